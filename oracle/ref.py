@@ -1,0 +1,206 @@
+"""ctypes front-end of the CPU oracle (``specroll_ref.c``).
+
+TEST INFRASTRUCTURE, NOT PRODUCT CODE: only the tests, the smoke check and the
+benchmark's CPU-baseline leg import this module.  It never touches the CUDA library.
+All arrays are host numpy arrays; bf16 tensors are uint16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "specroll_ref.c")
+_LIB = os.path.join(_HERE, "libspecroll_ref.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, OpenMP across independent rows only)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.specroll_ref_num_threads.restype = C.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().specroll_ref_num_threads())
+
+
+def _p(a: Optional[np.ndarray]):
+    if a is None:
+        return None
+    assert a.flags["C_CONTIGUOUS"], "oracle arrays must be contiguous"
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _chk(rc: int, what: str):
+    if rc != 0:
+        raise ValueError(f"oracle {what}: invalid arguments (code {rc})")
+
+
+def _as(a, dt):
+    return None if a is None else np.ascontiguousarray(a, dtype=dt)
+
+
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    x = _as(x, np.float64)
+    out = np.empty(x.shape, np.uint16)
+    lib().specroll_ref_round_bf16(C.c_int64(x.size), _p(x), _p(out))
+    return out
+
+
+def heads(h, A, bias, m=None, alpha=None, gamma=None, beta=None, ln_eps=1e-5, rms_eps=1e-6,
+          clip_c=0.0):
+    """Returns dict(xhat bf16, z fp64 (uncorrected), zc fp64 (corrected), zt bf16), all [B,K,d]."""
+    h, A, bias = _as(h, np.uint16), _as(A, np.uint16), _as(bias, np.uint16)
+    B, d = h.shape
+    K = A.shape[0]
+    assert A.shape == (K, d, d) and bias.shape == (K, d)
+    m, alpha = _as(m, np.float32), _as(alpha, np.float32)
+    gamma, beta = _as(gamma, np.uint16), _as(beta, np.uint16)
+    xhat = np.empty((B, K, d), np.uint16)
+    z = np.empty((B, K, d), np.float64)
+    zc = np.empty((B, K, d), np.float64)
+    zt = np.empty((B, K, d), np.uint16)
+    rc = lib().specroll_ref_heads(B, K, d, C.c_double(ln_eps), C.c_double(rms_eps),
+                                  C.c_double(clip_c), _p(h), _p(A), _p(bias), _p(gamma), _p(beta),
+                                  _p(m), _p(alpha), _p(xhat), _p(z), _p(zc), _p(zt))
+    _chk(rc, "heads")
+    return {"xhat": xhat, "z": z, "zc": zc, "zt": zt}
+
+
+def lm_logits(zt, W):
+    zt, W = _as(zt, np.uint16), _as(W, np.uint16)
+    zt2 = zt.reshape(-1, zt.shape[-1])
+    M, d = zt2.shape
+    V = W.shape[0]
+    out = np.empty((M, V), np.float64)
+    _chk(lib().specroll_ref_lm_logits(M, V, d, _p(zt2), _p(W), _p(out)), "lm_logits")
+    return out
+
+
+def topk(logits, k):
+    logits = _as(logits, np.float64)
+    M, V = logits.shape
+    cid = np.empty((M, k), np.int32)
+    cl = np.empty((M, k), np.float32)
+    _chk(lib().specroll_ref_topk(M, V, k, _p(logits), _p(cid), _p(cl)), "topk")
+    return cid, cl
+
+
+def lm_topk(zt, W, k):
+    zt, W = _as(zt, np.uint16), _as(W, np.uint16)
+    zt2 = zt.reshape(-1, zt.shape[-1])
+    M, d = zt2.shape
+    V = W.shape[0]
+    cid = np.empty((M, k), np.int32)
+    cl = np.empty((M, k), np.float32)
+    _chk(lib().specroll_ref_lm_topk(M, V, d, k, _p(zt2), _p(W), _p(cid), _p(cl)), "lm_topk")
+    return cid, cl
+
+
+def tree_draw(parent, anchor, cand_id, cand_logit, u_draw, temperature=1.0):
+    parent, anchor = _as(parent, np.int32), _as(anchor, np.int32)
+    cand_id, cand_logit = _as(cand_id, np.int32), _as(cand_logit, np.float32)
+    u_draw = _as(u_draw, np.float32)
+    B, K, k = cand_id.shape
+    N = parent.shape[0]
+    assert u_draw.shape == (B, N) and anchor.shape == (B,)
+    tok = np.empty((B, N), np.int32)
+    tc = np.empty((B, N), np.uint8)
+    sq = np.empty((B, N), np.float64)
+    rc = lib().specroll_ref_tree_draw(B, N, K, k, C.c_double(float(np.float32(temperature))), _p(parent), _p(anchor),
+                                      _p(cand_id), _p(cand_logit), _p(u_draw), _p(tok), _p(tc),
+                                      _p(sq))
+    _chk(rc, "tree_draw")
+    return {"tree_tok": tok, "tree_cand": tc, "slot_q": sq}
+
+
+def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0, ln_eps=1e-5,
+            rms_eps=1e-6, clip_c=0.0, gamma=None, beta=None):
+    h, A, bias, W = (_as(x, np.uint16) for x in (h, A, bias, W))
+    anchor, parent = _as(anchor, np.int32), _as(parent, np.int32)
+    m, alpha, u_draw = _as(m, np.float32), _as(alpha, np.float32), _as(u_draw, np.float32)
+    gamma, beta = _as(gamma, np.uint16), _as(beta, np.uint16)
+    B, d = h.shape
+    K, V, N = A.shape[0], W.shape[0], parent.shape[0]
+    cid = np.empty((B, K, k), np.int32)
+    cl = np.empty((B, K, k), np.float32)
+    tok = np.empty((B, N), np.int32)
+    tc = np.empty((B, N), np.uint8)
+    sq = np.empty((B, N), np.float64)
+    rc = lib().specroll_ref_propose(B, N, K, k, d, V, C.c_double(float(np.float32(temperature))), C.c_double(ln_eps),
+                                    C.c_double(rms_eps), C.c_double(clip_c), _p(h), _p(anchor),
+                                    _p(A), _p(bias), _p(gamma), _p(beta), _p(W), _p(m), _p(alpha),
+                                    _p(parent), _p(u_draw), _p(cid), _p(cl), _p(tok), _p(tc), _p(sq))
+    _chk(rc, "propose")
+    return {"cand_id": cid, "cand_logit": cl, "tree_tok": tok, "tree_cand": tc, "slot_q": sq}
+
+
+def tree_attn(Q, Kc, Vc, kv_indptr, Kt, Vt, parent, scale=None, want_lse=False):
+    Q, Kc, Vc, Kt, Vt = (_as(x, np.uint16) for x in (Q, Kc, Vc, Kt, Vt))
+    kv_indptr, parent = _as(kv_indptr, np.int32), _as(parent, np.int32)
+    B, N, Hq, D = Q.shape
+    Hkv = Kt.shape[2]
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    O64 = np.empty((B, N, Hq, D), np.float64)
+    Obf = np.empty((B, N, Hq, D), np.uint16)
+    lse = np.empty((B, N, Hq), np.float64) if want_lse else None
+    rc = lib().specroll_ref_tree_attn(B, N, Hq, Hkv, D, C.c_double(scale), _p(Q), _p(Kc), _p(Vc),
+                                      _p(kv_indptr), _p(Kt), _p(Vt), _p(parent), _p(O64), _p(Obf),
+                                      _p(lse))
+    _chk(rc, "tree_attn")
+    out = {"O64": O64, "Obf": Obf}
+    if want_lse:
+        out["lse"] = lse
+    return out
+
+
+def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin,
+           temperature=1.0):
+    logits = _as(logits, np.uint16)
+    parent, tree_tok = _as(parent, np.int32), _as(tree_tok, np.int32)
+    tree_cand, cand_id = _as(tree_cand, np.uint8), _as(cand_id, np.int32)
+    cand_logit, u_acc, u_fin = (_as(x, np.float32) for x in (cand_logit, u_acc, u_fin))
+    B, N, V = logits.shape
+    _, K, k = cand_id.shape
+    n_acc = np.empty(B, np.int32)
+    path = np.empty((B, K + 1), np.int32)
+    out_tok = np.empty((B, K + 1), np.int32)
+    term_node = np.empty(B, np.int32)
+    term_kind = np.empty(B, np.int32)
+    row_max = np.empty((B, N), np.float64)
+    row_sum = np.empty((B, N), np.float64)
+    mm = np.empty(B, np.float64)
+    fm = np.empty(B, np.float64)
+    rc = lib().specroll_ref_verify(B, N, K, k, V, C.c_double(float(np.float32(temperature))), _p(logits), _p(parent),
+                                   _p(tree_tok), _p(tree_cand), _p(cand_id), _p(cand_logit),
+                                   _p(u_acc), _p(u_fin), _p(n_acc), _p(path), _p(out_tok),
+                                   _p(term_node), _p(term_kind), _p(row_max), _p(row_sum), _p(mm),
+                                   _p(fm))
+    _chk(rc, "verify")
+    return {"n_acc": n_acc, "path_node": path, "out_tok": out_tok, "term_node": term_node,
+            "term_kind": term_kind, "row_max": row_max, "row_sum": row_sum, "min_margin": mm,
+            "fin_margin": fm}
+
+
+def node_budget(C_hw, B_active, N_min=1, N_max=10) -> int:
+    f = lib().specroll_ref_node_budget
+    f.restype = C.c_int32
+    return int(f(C.c_int32(C_hw), C.c_int32(B_active), C.c_int32(N_min), C.c_int32(N_max)))
