@@ -1,0 +1,174 @@
+/*
+ * specroll.h -- C ABI of the SpecRoll per-step speculative hot path for NVIDIA B200 (sm_100a).
+ *
+ * One speculative round of the rollout engine (Algorithm "One exact speculative round") is,
+ * per step: proposal -> packed target forward (tree attention in every layer) -> exact
+ * node-wise verification.  This library provides those three pieces as stateless calls.
+ *
+ * Conventions (all entry points):
+ *   - Pointers whose name ends in _host are HOST pointers, read during the call only.
+ *     Every other pointer is a DEVICE pointer owned by the caller; the library never
+ *     allocates, frees or retains memory and never synchronises the device.
+ *   - bf16 tensors are passed as `const void*` / `void*` to 2-byte bf16 elements.
+ *   - All tensors are dense, row-major, 16-byte aligned at their base.
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t; NULL = default stream).
+ *   - Scratch memory comes from `workspace` (device, 256-byte aligned), whose size is given
+ *     by the matching *_workspace_bytes query.  Calls that share a workspace must not
+ *     overlap on the device.
+ *   - Return value: SPECROLL_OK or an error code; on error nothing has been enqueued
+ *     (except SPECROLL_ECUDA, where earlier launches of the call may have been).
+ *   - Tree topology: parent_host[N] with parent[0] = -1 and 0 <= parent[n] < n; the tree is
+ *     shared by all B sequences of a call.  depth(n) <= K, every node has <= k children,
+ *     N <= 64.  The children of a node, in increasing node index, are its ordered slots.
+ *     Node 0 is the anchor (an exact target sample) and carries no proposal.
+ */
+#ifndef SPECROLL_H
+#define SPECROLL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPECROLL_OK 0
+#define SPECROLL_EINVAL 1     /* bad shape / limit / NULL pointer / malformed topology */
+#define SPECROLL_EALIGN 2     /* a base pointer is not 16-byte aligned */
+#define SPECROLL_EWORKSPACE 3 /* workspace too small or misaligned */
+#define SPECROLL_ECUDA 4      /* a CUDA runtime call or kernel launch failed */
+#define SPECROLL_ETIMEOUT 5   /* a bounded device-side wait ran out (read from a status word) */
+
+#define SPECROLL_MAX_NODES 64
+#define SPECROLL_MAX_HEADS 8
+#define SPECROLL_MAX_TOPK 64
+
+/* Library version (major * 10000 + minor * 100 + patch). */
+int specroll_version(void);
+
+/* Human-readable text for a return code; for SPECROLL_ECUDA includes the last CUDA error
+ * string seen by the calling thread.  The pointer stays valid until the thread's next call. */
+const char *specroll_strerror(int code);
+
+/* Concurrency-aware node budget, Eq. "verification-budget" (Sec. 3.2):
+ *   N_t = clip(floor(C_hw / B_active), N_min, N_max);  B_active < 1 gives N_max. */
+int32_t specroll_node_budget(int32_t C_hw, int32_t B_active, int32_t N_min, int32_t N_max);
+
+/* ------------------------------------------------------------------------------------------
+ * Proposal (Sec. 3.2 Eq. "heads"; App. C "Future-token proposer"; Sec. 3.4 Eq.
+ * "reflex-correction"; App. B.1 Eq. "slotq" / "childlist").
+ *
+ * For every sequence b and head h (predicting position t+h+1):
+ *   x^   = LN(h_b) * gamma_h + beta_h           (fp32 statistics, biased variance; bf16 out)
+ *   z    = h_b + SiLU(A_h x^ + bias_h)          (bf16 tensor-core product, fp32 accumulate)
+ *   z~   = z + alpha_{b,h} RMS(z) m_{b,h} / (RMS(m_{b,h}) + rms_eps), optionally rescaled so
+ *          that |z~ - z|_2 <= clip_c |z|_2; alpha = 0 (or m/alpha NULL) abstains; bf16 out
+ *   l_v  = W_v . z~  for all v (never written to memory); the k largest, ordered by
+ *          (logit descending, token id ascending), go to cand_logit / cand_id
+ * and the tree is drawn: node n >= 1 with parent u and depth dd takes a token from head dd's
+ * candidates not already used by an earlier child of u, with probability softmax(l / T)
+ * renormalised on that remaining set (inverse CDF in candidate order, uniform u_draw[b,n]).
+ *
+ * Shapes: h[B,d] bf16; anchor_tok[B] i32; A[K,d,d] bf16 (row = output unit); bias[K,d] bf16;
+ * ln_gamma/ln_beta[K,d] bf16 or NULL (1 / 0); W[V,d] bf16 (row = token); m[B,K,d] fp32 or NULL;
+ * alpha[B,K] fp32 or NULL; u_draw[B,N] fp32 in [0,1).
+ * Outputs: cand_id[B,K,k] i32; cand_logit[B,K,k] fp32; tree_tok[B,N] i32 (node 0 = anchor);
+ * tree_cand[B,N] u8 (slot of the node's token in its head's list; 255 for node 0);
+ * slot_q[B,N] fp32 (probability the node's token had when drawn; 1 for node 0).
+ * Limits: d % 64 == 0, V % 8 == 0, 1 <= k <= 64, K <= 8, N <= 64.
+ */
+typedef struct {
+    int32_t B, N, K, k, d, V;
+    float temperature; /* T > 0 */
+    float ln_eps;      /* LayerNorm epsilon (1e-5 if the caller has no other value) */
+    float rms_eps;     /* epsilon of the RMS normalisation of the memory */
+    float clip_c;      /* <= 0: no L2 clip */
+    int32_t flags;     /* reserved, must be 0 */
+} specroll_propose_desc;
+
+size_t specroll_propose_workspace_bytes(const specroll_propose_desc *desc);
+
+int specroll_propose(const specroll_propose_desc *desc, const void *h, const int32_t *anchor_tok,
+                     const void *A, const void *bias, const void *ln_gamma, const void *ln_beta,
+                     const void *W, const float *m, const float *alpha,
+                     const int32_t *parent_host, const float *u_draw, int32_t *cand_id,
+                     float *cand_logit, int32_t *tree_tok, uint8_t *tree_cand, float *slot_q,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* The last step of the proposal alone (App. B.1): draw the tree from given candidate lists.
+ * Same arguments and outputs as the corresponding ones of specroll_propose; needs no workspace. */
+int specroll_tree_draw(int32_t B, int32_t N, int32_t K, int32_t k, float temperature,
+                       const int32_t *parent_host, const int32_t *anchor_tok,
+                       const int32_t *cand_id, const float *cand_logit, const float *u_draw,
+                       int32_t *tree_tok, uint8_t *tree_cand, float *slot_q, void *cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Tree-verification attention of one layer (App. B.1 Eq. "nodep": the packed forward must
+ * equal an ordinary autoregressive forward at every node's own prefix).
+ *
+ * For sequence b, node n, query head hq (KV head hq / (Hq/Hkv)):
+ *   O = softmax(scale * q . [K_cache(b) ; K_tree(b, anc(n))]^T) [V_cache(b) ; V_tree(b, anc(n))]
+ * where anc(n) are the ancestors of n including n.
+ *
+ * Shapes: Q[B,N,Hq,D] bf16; Kc,Vc[T_kv,Hkv,D] bf16, sequence b owning rows
+ * kv_indptr[b] .. kv_indptr[b+1]-1; kv_indptr_dev/_host[B+1] i32 (same values; the host copy
+ * sizes the launch so no device read-back is needed); Kt,Vt[B,N,Hkv,D] bf16.
+ * Outputs: O[B,N,Hq,D] bf16; lse[B,N,Hq] fp32 or NULL (natural-log sum-exp of the scaled scores).
+ * Limits: D == 64 or 128, Hq % Hkv == 0, N <= 64.
+ */
+typedef struct {
+    int32_t B, N, Hq, Hkv, D;
+    float scale;   /* softmax scale; the method uses 1/sqrt(D) */
+    int32_t flags; /* reserved, must be 0 */
+} specroll_attn_desc;
+
+size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *desc,
+                                          const int32_t *kv_indptr_host);
+
+int specroll_tree_attn(const specroll_attn_desc *desc, const void *Q, const void *Kc,
+                       const void *Vc, const int32_t *kv_indptr_dev,
+                       const int32_t *kv_indptr_host, const void *Kt, const void *Vt,
+                       const int32_t *parent_host, void *O, float *lse, void *workspace,
+                       size_t workspace_bytes, void *cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Exact target verification (App. B.2 Eq. "nodeaccept" / "noderesidual", Algorithm "Exact
+ * node-wise tree verification").
+ *
+ * p_n = softmax(logits[b,n,:] / T) at every node.  Starting at the root u with residual
+ * r = p_u, the children of u are tested in slot order: child c with token y is accepted iff
+ * u_acc[b,c] < min(1, r(y) / q(y)), q being the slot's proposal (recomputed from
+ * cand_logit exactly as the proposal drew it); on rejection r <- [r - q]_+ / sum[r - q]_+.
+ * An accepted child becomes u.  The round ends with one more token drawn with u_fin[b] by
+ * inverse CDF in token-id order: from the final residual when every child of u was rejected
+ * (fallback), or from p_u when u was accepted and has no children (bonus).
+ *
+ * Shapes: logits[B,N,V] bf16; tree_tok[B,N] i32; tree_cand[B,N] u8; cand_id[B,K,k] i32;
+ * cand_logit[B,K,k] fp32; u_acc[B,N] fp32; u_fin[B] fp32 (uniforms in [0,1)).
+ * Outputs: n_acc[B] i32 (accepted proposals); path_node[B,K+1] i32 (node at each depth of the
+ * committed path, -1 after); out_tok[B,K+1] i32 (accepted tokens, then the terminal token, -1
+ * after); term_node[B]; term_kind[B] (0 fallback, 1 bonus); row_max,row_sum[B,N] fp32
+ * (max logit and sum exp((l - max)/T) of every node); min_margin[B] fp32 or NULL (smallest
+ * |u - ratio| over the tested slots; +inf if none).
+ * Limits: V % 8 == 0, k <= 64, K <= 8, N <= 64.
+ */
+typedef struct {
+    int32_t B, N, K, k, V;
+    float temperature;
+    int32_t flags; /* reserved, must be 0 */
+} specroll_verify_desc;
+
+size_t specroll_verify_workspace_bytes(const specroll_verify_desc *desc);
+
+int specroll_verify(const specroll_verify_desc *desc, const void *logits,
+                    const int32_t *parent_host, const int32_t *tree_tok,
+                    const uint8_t *tree_cand, const int32_t *cand_id, const float *cand_logit,
+                    const float *u_acc, const float *u_fin, int32_t *n_acc, int32_t *path_node,
+                    int32_t *out_tok, int32_t *term_node, int32_t *term_kind, float *row_max,
+                    float *row_sum, float *min_margin, void *workspace, size_t workspace_bytes,
+                    void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECROLL_H */

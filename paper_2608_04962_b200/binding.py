@@ -1,0 +1,275 @@
+"""Thin Python binding of the C-ABI library ``libspecroll.so``.
+
+Argument marshalling only: every function checks dtype / device / contiguity of torch
+tensors, allocates outputs and the workspace with torch, and passes raw pointers to the
+entry point of the same name.  No step of the method runs in Python.  The library is loaded
+on first use and loading fails loudly when it has not been built: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspecroll.so")
+_lib = None
+
+EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
+           "specroll_propose_workspace_bytes", "specroll_propose", "specroll_tree_draw",
+           "specroll_tree_attn_workspace_bytes", "specroll_tree_attn",
+           "specroll_verify_workspace_bytes", "specroll_verify")
+
+
+class SpecrollError(RuntimeError):
+    pass
+
+
+class ProposeDesc(C.Structure):
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("K", C.c_int32), ("k", C.c_int32),
+                ("d", C.c_int32), ("V", C.c_int32), ("temperature", C.c_float),
+                ("ln_eps", C.c_float), ("rms_eps", C.c_float), ("clip_c", C.c_float),
+                ("flags", C.c_int32)]
+
+
+class AttnDesc(C.Structure):
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
+                ("D", C.c_int32), ("scale", C.c_float), ("flags", C.c_int32)]
+
+
+class VerifyDesc(C.Structure):
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("K", C.c_int32), ("k", C.c_int32),
+                ("V", C.c_int32), ("temperature", C.c_float), ("flags", C.c_int32)]
+
+
+def lib():
+    """The loaded library.  Raises if it is missing: the CUDA path is the only path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise SpecrollError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2608_04962_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        l = C.CDLL(LIB_PATH)
+        l.specroll_version.restype = C.c_int
+        l.specroll_strerror.restype = C.c_char_p
+        l.specroll_strerror.argtypes = [C.c_int]
+        l.specroll_node_budget.restype = C.c_int32
+        l.specroll_node_budget.argtypes = [C.c_int32] * 4
+        for n in ("specroll_propose_workspace_bytes", "specroll_verify_workspace_bytes",
+                  "specroll_tree_attn_workspace_bytes"):
+            getattr(l, n).restype = C.c_size_t
+        for n in ("specroll_propose", "specroll_tree_draw", "specroll_tree_attn", "specroll_verify"):
+            getattr(l, n).restype = C.c_int
+        _lib = l
+    return _lib
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise SpecrollError(f"{what}: {lib().specroll_strerror(rc).decode()} (code {rc})")
+
+
+def _dev(t: Optional[torch.Tensor], dtype, name: str):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise SpecrollError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise SpecrollError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise SpecrollError(f"{name} must be contiguous")
+    return C.c_void_p(t.data_ptr())
+
+
+def _host_i32(a, name: str) -> np.ndarray:
+    a = np.ascontiguousarray(np.asarray(a), dtype=np.int32)
+    if a.ndim != 1:
+        raise SpecrollError(f"{name} must be one-dimensional")
+    return a
+
+
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def version() -> int:
+    return int(lib().specroll_version())
+
+
+def node_budget(C_hw: int, B_active: int, N_min: int = 1, N_max: int = 10) -> int:
+    return int(lib().specroll_node_budget(C_hw, B_active, N_min, N_max))
+
+
+# ----------------------------------------------------------------------------------- propose
+
+
+def propose_workspace_bytes(B, N, K, k, d, V, temperature=1.0, ln_eps=1e-5, rms_eps=1e-6,
+                            clip_c=0.0) -> int:
+    desc = ProposeDesc(B, N, K, k, d, V, temperature, ln_eps, rms_eps, clip_c, 0)
+    return int(lib().specroll_propose_workspace_bytes(C.byref(desc)))
+
+
+def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0, ln_eps=1e-5,
+            rms_eps=1e-6, clip_c=0.0, ln_gamma=None, ln_beta=None, workspace=None,
+            out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """specroll_propose.  Device tensors in, dict of device tensors out."""
+    parent = _host_i32(parent, "parent")
+    B, d = h.shape
+    K, V, N = A.shape[0], W.shape[0], parent.shape[0]
+    if tuple(A.shape) != (K, d, d) or tuple(bias.shape) != (K, d) or W.shape[1] != d:
+        raise SpecrollError("propose: inconsistent weight shapes")
+    if tuple(u_draw.shape) != (B, N) or tuple(anchor.shape) != (B,):
+        raise SpecrollError("propose: inconsistent u_draw / anchor shapes")
+    if m is not None and tuple(m.shape) != (B, K, d):
+        raise SpecrollError("propose: m must be [B,K,d]")
+    if alpha is not None and tuple(alpha.shape) != (B, K):
+        raise SpecrollError("propose: alpha must be [B,K]")
+    desc = ProposeDesc(B, N, K, k, d, V, temperature, ln_eps, rms_eps, clip_c, 0)
+    dev = h.device
+    if out is None:
+        out = {"cand_id": torch.empty((B, K, k), dtype=torch.int32, device=dev),
+               "cand_logit": torch.empty((B, K, k), dtype=torch.float32, device=dev),
+               "tree_tok": torch.empty((B, N), dtype=torch.int32, device=dev),
+               "tree_cand": torch.empty((B, N), dtype=torch.uint8, device=dev),
+               "slot_q": torch.empty((B, N), dtype=torch.float32, device=dev)}
+    if workspace is None:
+        workspace = _workspace(lib().specroll_propose_workspace_bytes(C.byref(desc)), dev)
+    bf = torch.bfloat16
+    rc = lib().specroll_propose(
+        C.byref(desc), _dev(h, bf, "h"), _dev(anchor, torch.int32, "anchor"), _dev(A, bf, "A"),
+        _dev(bias, bf, "bias"), _dev(ln_gamma, bf, "ln_gamma"), _dev(ln_beta, bf, "ln_beta"),
+        _dev(W, bf, "W"), _dev(m, torch.float32, "m"), _dev(alpha, torch.float32, "alpha"),
+        parent.ctypes.data_as(C.c_void_p), _dev(u_draw, torch.float32, "u_draw"),
+        _dev(out["cand_id"], torch.int32, "cand_id"), _dev(out["cand_logit"], torch.float32, "cand_logit"),
+        _dev(out["tree_tok"], torch.int32, "tree_tok"), _dev(out["tree_cand"], torch.uint8, "tree_cand"),
+        _dev(out["slot_q"], torch.float32, "slot_q"), C.c_void_p(workspace.data_ptr()),
+        C.c_size_t(workspace.numel()), _stream())
+    _check(rc, "specroll_propose")
+    return out
+
+
+def tree_draw(parent, anchor, cand_id, cand_logit, u_draw, temperature=1.0) -> Dict[str, torch.Tensor]:
+    """specroll_tree_draw."""
+    parent = _host_i32(parent, "parent")
+    B, K, k = cand_id.shape
+    N = parent.shape[0]
+    dev = cand_id.device
+    out = {"tree_tok": torch.empty((B, N), dtype=torch.int32, device=dev),
+           "tree_cand": torch.empty((B, N), dtype=torch.uint8, device=dev),
+           "slot_q": torch.empty((B, N), dtype=torch.float32, device=dev)}
+    rc = lib().specroll_tree_draw(
+        C.c_int32(B), C.c_int32(N), C.c_int32(K), C.c_int32(k), C.c_float(temperature),
+        parent.ctypes.data_as(C.c_void_p), _dev(anchor, torch.int32, "anchor"),
+        _dev(cand_id, torch.int32, "cand_id"), _dev(cand_logit, torch.float32, "cand_logit"),
+        _dev(u_draw, torch.float32, "u_draw"), _dev(out["tree_tok"], torch.int32, "tree_tok"),
+        _dev(out["tree_cand"], torch.uint8, "tree_cand"), _dev(out["slot_q"], torch.float32, "slot_q"),
+        _stream())
+    _check(rc, "specroll_tree_draw")
+    return out
+
+
+# ----------------------------------------------------------------------------------- attention
+
+
+def tree_attn_workspace_bytes(B, N, Hq, Hkv, D, kv_indptr_host, scale=None) -> int:
+    ip = _host_i32(kv_indptr_host, "kv_indptr_host")
+    desc = AttnDesc(B, N, Hq, Hkv, D, scale if scale is not None else 1.0 / float(np.sqrt(D)), 0)
+    return int(lib().specroll_tree_attn_workspace_bytes(C.byref(desc), ip.ctypes.data_as(C.c_void_p)))
+
+
+def tree_attn(Q, Kc, Vc, kv_indptr_dev, kv_indptr_host, Kt, Vt, parent, scale=None, want_lse=False,
+              workspace=None, out=None, lse=None):
+    """specroll_tree_attn.  Returns O (and lse when asked)."""
+    parent = _host_i32(parent, "parent")
+    ip = _host_i32(kv_indptr_host, "kv_indptr_host")
+    B, N, Hq, D = Q.shape
+    Hkv = Kt.shape[2]
+    if ip.shape[0] != B + 1 or tuple(Kt.shape) != (B, N, Hkv, D) or tuple(Vt.shape) != (B, N, Hkv, D):
+        raise SpecrollError("tree_attn: inconsistent shapes")
+    if Kc.shape[0] != int(ip[-1]) or tuple(Kc.shape[1:]) != (Hkv, D) or Vc.shape != Kc.shape:
+        raise SpecrollError("tree_attn: cache shape does not match kv_indptr")
+    if scale is None:
+        scale = 1.0 / float(np.sqrt(D))
+    desc = AttnDesc(B, N, Hq, Hkv, D, scale, 0)
+    dev = Q.device
+    if out is None:
+        out = torch.empty((B, N, Hq, D), dtype=torch.bfloat16, device=dev)
+    if want_lse and lse is None:
+        lse = torch.empty((B, N, Hq), dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = _workspace(lib().specroll_tree_attn_workspace_bytes(
+            C.byref(desc), ip.ctypes.data_as(C.c_void_p)), dev)
+    bf = torch.bfloat16
+    rc = lib().specroll_tree_attn(
+        C.byref(desc), _dev(Q, bf, "Q"), _dev(Kc, bf, "Kc"), _dev(Vc, bf, "Vc"),
+        _dev(kv_indptr_dev, torch.int32, "kv_indptr_dev"), ip.ctypes.data_as(C.c_void_p),
+        _dev(Kt, bf, "Kt"), _dev(Vt, bf, "Vt"), parent.ctypes.data_as(C.c_void_p),
+        _dev(out, bf, "O"), _dev(lse, torch.float32, "lse"), C.c_void_p(workspace.data_ptr()),
+        C.c_size_t(workspace.numel()), _stream())
+    _check(rc, "specroll_tree_attn")
+    return (out, lse) if want_lse else out
+
+
+# ----------------------------------------------------------------------------------- verify
+
+
+def verify_workspace_bytes(B, N, K, k, V, temperature=1.0) -> int:
+    desc = VerifyDesc(B, N, K, k, V, temperature, 0)
+    return int(lib().specroll_verify_workspace_bytes(C.byref(desc)))
+
+
+def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, temperature=1.0,
+           workspace=None, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """specroll_verify.  Device tensors in, dict of device tensors out."""
+    parent = _host_i32(parent, "parent")
+    B, N, V = logits.shape
+    _, K, k = cand_id.shape
+    if parent.shape[0] != N or tuple(tree_tok.shape) != (B, N) or tuple(u_acc.shape) != (B, N):
+        raise SpecrollError("verify: inconsistent shapes")
+    desc = VerifyDesc(B, N, K, k, V, temperature, 0)
+    dev = logits.device
+    i32, f32 = torch.int32, torch.float32
+    if out is None:
+        out = {"n_acc": torch.empty(B, dtype=i32, device=dev),
+               "path_node": torch.empty((B, K + 1), dtype=i32, device=dev),
+               "out_tok": torch.empty((B, K + 1), dtype=i32, device=dev),
+               "term_node": torch.empty(B, dtype=i32, device=dev),
+               "term_kind": torch.empty(B, dtype=i32, device=dev),
+               "row_max": torch.empty((B, N), dtype=f32, device=dev),
+               "row_sum": torch.empty((B, N), dtype=f32, device=dev),
+               "min_margin": torch.empty(B, dtype=f32, device=dev)}
+    if workspace is None:
+        workspace = _workspace(lib().specroll_verify_workspace_bytes(C.byref(desc)), dev)
+    rc = lib().specroll_verify(
+        C.byref(desc), _dev(logits, torch.bfloat16, "logits"), parent.ctypes.data_as(C.c_void_p),
+        _dev(tree_tok, i32, "tree_tok"), _dev(tree_cand, torch.uint8, "tree_cand"),
+        _dev(cand_id, i32, "cand_id"), _dev(cand_logit, f32, "cand_logit"), _dev(u_acc, f32, "u_acc"),
+        _dev(u_fin, f32, "u_fin"), _dev(out["n_acc"], i32, "n_acc"), _dev(out["path_node"], i32, "path_node"),
+        _dev(out["out_tok"], i32, "out_tok"), _dev(out["term_node"], i32, "term_node"),
+        _dev(out["term_kind"], i32, "term_kind"), _dev(out["row_max"], f32, "row_max"),
+        _dev(out["row_sum"], f32, "row_sum"), _dev(out.get("min_margin"), f32, "min_margin"),
+        C.c_void_p(workspace.data_ptr()), C.c_size_t(workspace.numel()), _stream())
+    _check(rc, "specroll_verify")
+    return out
+
+
+# ----------------------------------------------------------------------------------- helpers
+
+
+def bf16_tensor(bits: np.ndarray, device="cuda") -> torch.Tensor:
+    """uint16 bf16 bit patterns (host numpy) -> bf16 tensor on the device."""
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.view(torch.bfloat16).to(device)
+
+
+def bf16_bits(t: torch.Tensor) -> np.ndarray:
+    """bf16 tensor -> uint16 bit patterns on the host."""
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)

@@ -1,0 +1,68 @@
+// Entry points that need no kernel: version, error strings, node budget; plus the host-side
+// topology validation shared by the three steps.
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace specroll {
+
+static thread_local cudaError_t g_last_cuda = cudaSuccess;
+static thread_local char g_msg[256];
+
+int note_cuda_error(cudaError_t e) {
+    g_last_cuda = e;
+    return SPECROLL_ECUDA;
+}
+
+int build_topo(const int32_t *parent_host, int N, int K, int k, Topo *t, TopoMask *m) {
+    if (!parent_host || N < 1 || N > SPECROLL_MAX_NODES || parent_host[0] != -1) return SPECROLL_EINVAL;
+    memset(t, 0, sizeof(*t));
+    if (m) memset(m, 0, sizeof(*m));
+    t->N = N;
+    t->parent[0] = -1;
+    if (m) m->anc[0] = 1ull;
+    for (int n = 1; n < N; ++n) {
+        int p = parent_host[n];
+        if (p < 0 || p >= n) return SPECROLL_EINVAL;
+        t->parent[n] = (int8_t)p;
+        t->depth[n] = (int8_t)(t->depth[p] + 1);
+        t->n_child[p]++;
+        if (t->depth[n] > t->max_depth) t->max_depth = t->depth[n];
+        if (K >= 0 && t->depth[n] > K) return SPECROLL_EINVAL;
+        if (k >= 0 && t->n_child[p] > k) return SPECROLL_EINVAL;
+        if (m) m->anc[n] = m->anc[p] | (1ull << n);
+    }
+    return SPECROLL_OK;
+}
+
+}  // namespace specroll
+
+extern "C" {
+
+int specroll_version(void) { return 100; }
+
+const char *specroll_strerror(int code) {
+    using namespace specroll;
+    switch (code) {
+        case SPECROLL_OK: return "ok";
+        case SPECROLL_EINVAL: return "invalid argument (shape, limit, NULL pointer or malformed tree)";
+        case SPECROLL_EALIGN: return "a tensor base pointer is not 16-byte aligned";
+        case SPECROLL_EWORKSPACE: return "workspace too small or not 256-byte aligned";
+        case SPECROLL_ETIMEOUT: return "a bounded device-side wait ran out";
+        case SPECROLL_ECUDA:
+            snprintf(g_msg, sizeof(g_msg), "CUDA error: %s", cudaGetErrorString(g_last_cuda));
+            return g_msg;
+        default: return "unknown error code";
+    }
+}
+
+int32_t specroll_node_budget(int32_t C_hw, int32_t B_active, int32_t N_min, int32_t N_max) {
+    if (B_active < 1) return N_max;
+    int32_t n = C_hw / B_active;
+    if (n < N_min) n = N_min;
+    if (n > N_max) n = N_max;
+    return n;
+}
+
+}  // extern "C"

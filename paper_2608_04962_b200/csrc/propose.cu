@@ -1,0 +1,474 @@
+// Proposal step: LayerNorm -> K head MLPs -> bounded correction -> shared vocabulary projection
+// with a fused running top-k (logits never reach memory) -> top-k merge -> tree draw.
+#include <math.h>
+
+#include "common.cuh"
+#include "gemm_mma.cuh"
+
+namespace specroll {
+
+// ------------------------------------------------------------------------------ block reduce
+
+template <int THREADS>
+__device__ __forceinline__ float block_sum(float v, float *sh) {
+    v = warp_sum(v);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) sh[warp] = v;
+    __syncthreads();
+    float t = lane < THREADS / 32 ? sh[lane] : 0.f;
+    return warp_sum(t);
+}
+
+// ------------------------------------------------------------------------------ P1 LayerNorm
+
+constexpr int LN_THREADS = 256;
+
+// h[B,d] bf16 -> xhat[KX,B,d] bf16 with KX = K when an affine (gamma/beta) is given, else 1.
+__global__ void __launch_bounds__(LN_THREADS)
+layernorm_kernel(const __nv_bfloat16 *__restrict__ h, const __nv_bfloat16 *__restrict__ gamma,
+                 const __nv_bfloat16 *__restrict__ beta, __nv_bfloat16 *__restrict__ xhat, int B, int d,
+                 int KX, float eps) {
+    extern __shared__ float row[];  // d floats
+    __shared__ float red[LN_THREADS / 32];
+    const int b = blockIdx.x;
+    float s = 0.f;
+    for (int i = threadIdx.x; i < d; i += LN_THREADS) {
+        const float v = __bfloat162float(h[(size_t)b * d + i]);
+        row[i] = v;
+        s += v;
+    }
+    const float mu = block_sum<LN_THREADS>(s, red) / d;
+    float q = 0.f;
+    for (int i = threadIdx.x; i < d; i += LN_THREADS) {
+        const float t = row[i] - mu;
+        q += t * t;
+    }
+    const float var = block_sum<LN_THREADS>(q, red) / d;
+    const float rstd = 1.0f / sqrtf(var + eps);
+    for (int hd = 0; hd < KX; ++hd) {
+        for (int i = threadIdx.x; i < d; i += LN_THREADS) {
+            float x = (row[i] - mu) * rstd;
+            if (gamma) x *= __bfloat162float(gamma[(size_t)hd * d + i]);
+            if (beta) x += __bfloat162float(beta[(size_t)hd * d + i]);
+            xhat[((size_t)hd * B + b) * d + i] = __float2bfloat16_rn(x);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------ P2 head MLP
+
+using HeadTile = MmaTile<128, 64, 4, 2, 3>;  // 8 warps, warp tile 32 x 32
+
+// z[b,hd,o] = h[b,o] + SiLU(sum_i xhat[hd?,b,i] * A[hd,o,i] + bias[hd,o])      (fp32 out)
+__global__ void __launch_bounds__(HeadTile::THREADS)
+head_mlp_kernel(const __nv_bfloat16 *__restrict__ xhat, int KX, const __nv_bfloat16 *__restrict__ A,
+                const __nv_bfloat16 *__restrict__ bias, const __nv_bfloat16 *__restrict__ h,
+                float *__restrict__ z, int B, int K, int d) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    using T = HeadTile;
+    const int hd = blockIdx.z, m0 = blockIdx.y * T::BM, n0 = blockIdx.x * T::BN;
+    const __nv_bfloat16 *X = xhat + (KX > 1 ? (size_t)hd * B * d : 0);
+    const __nv_bfloat16 *Ah = A + (size_t)hd * d * d;
+    float acc[T::MT][T::NT][4];
+    T::run(smem, X, d, m0, B, Ah, d, n0, d, d, acc);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wm0 = (warp / T::WN) * T::WTM, wn0 = (warp % T::WN) * T::WTN;
+#pragma unroll
+    for (int i = 0; i < T::MT; ++i)
+#pragma unroll
+        for (int j = 0; j < T::NT; ++j)
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int row = m0 + wm0 + i * 16 + (lane >> 2) + (t >> 1) * 8;
+                const int col = n0 + wn0 + j * 8 + (lane & 3) * 2 + (t & 1);
+                if (row < B && col < d) {
+                    const float y = acc[i][j][t] + __bfloat162float(bias[(size_t)hd * d + col]);
+                    const float sl = y / (1.0f + __expf(-y));
+                    z[((size_t)row * K + hd) * d + col] = __bfloat162float(h[(size_t)row * d + col]) + sl;
+                }
+            }
+}
+
+// ------------------------------------------------------------------------------ P3 bounded correction
+
+constexpr int RX_THREADS = 256;
+
+// zt[r,:] = bf16(z[r,:] + coef * m[r,:]),  r = b*K + hd,
+// coef = alpha * RMS(z) / (RMS(m) + eps), shrunk so that |coef * m|_2 <= clip_c * |z|_2.
+__global__ void __launch_bounds__(RX_THREADS)
+reflex_kernel(const float *__restrict__ z, const float *__restrict__ m, const float *__restrict__ alpha,
+              __nv_bfloat16 *__restrict__ zt, int d, float rms_eps, float clip_c) {
+    __shared__ float red[RX_THREADS / 32];
+    const size_t r = blockIdx.x;
+    const float *zr = z + r * d;
+    const float a = (alpha && m) ? alpha[r] : 0.f;
+    float coef = 0.f;
+    if (a != 0.f) {  // uniform across the block
+        const float *mr = m + r * d;
+        float sz = 0.f, sm = 0.f;
+        for (int i = threadIdx.x; i < d; i += RX_THREADS) {
+            const float zv = zr[i], mv = mr[i];
+            sz += zv * zv;
+            sm += mv * mv;
+        }
+        sz = block_sum<RX_THREADS>(sz, red);
+        sm = block_sum<RX_THREADS>(sm, red);
+        const float rms_z = sqrtf(sz / d), rms_m = sqrtf(sm / d);
+        coef = a * rms_z / (rms_m + rms_eps);
+        const float nd = fabsf(coef) * sqrtf(sm), nz = sqrtf(sz);
+        if (clip_c > 0.f && nd > clip_c * nz) coef *= clip_c * nz / nd;
+        for (int i = threadIdx.x; i < d; i += RX_THREADS) zt[r * d + i] = __float2bfloat16_rn(zr[i] + coef * mr[i]);
+    } else {
+        for (int i = threadIdx.x; i < d; i += RX_THREADS) zt[r * d + i] = __float2bfloat16_rn(zr[i]);
+    }
+}
+
+// ------------------------------------------------------------------------------ P4 projection + top-k
+
+// Sorted (descending value; earlier insertion wins ties) list of the KMAX best seen so far.
+template <int KMAX>
+struct TopList {
+    float v[KMAX];
+    int32_t id[KMAX];
+    __device__ __forceinline__ void init() {
+#pragma unroll
+        for (int i = 0; i < KMAX; ++i) {
+            v[i] = -INFINITY;
+            id[i] = 0x7fffffff;
+        }
+    }
+    // candidates arrive in increasing id order, so "strictly greater" keeps the lowest id on ties
+    __device__ __forceinline__ void push(float x, int32_t t) {
+        if (!(x > v[KMAX - 1])) return;
+#pragma unroll
+        for (int i = KMAX - 1; i > 0; --i) {
+            if (x > v[i - 1]) {
+                v[i] = v[i - 1];
+                id[i] = id[i - 1];
+            } else if (x > v[i]) {  // v[i-1] >= x > v[i]
+                v[i] = x;
+                id[i] = t;
+            }
+        }
+        if (x > v[0]) {
+            v[0] = x;
+            id[0] = t;
+        }
+    }
+};
+
+using LmTile = MmaTile<128, 128, 2, 4, 3>;  // 8 warps, warp tile 64 x 32
+constexpr int LM_CSTRIDE = 129;            // fp32 staging tile row stride (conflict-free row scans)
+
+// Each CTA owns one block of 128 rows and a contiguous range of vocabulary tiles; thread r < 128
+// keeps the running top list of row r across those tiles.  Partial lists go to
+// pval/pid[M, n_groups, k]; a merge kernel finishes.
+template <int KMAX>
+__global__ void __launch_bounds__(LmTile::THREADS)
+lm_head_topk_kernel(const __nv_bfloat16 *__restrict__ Zt, const __nv_bfloat16 *__restrict__ W, int M,
+                    int V, int d, int k, int n_mblocks, int n_groups, int tiles_per_group,
+                    float *__restrict__ pval, int32_t *__restrict__ pid) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    using T = LmTile;
+    const int mb = blockIdx.x % n_mblocks, grp = blockIdx.x / n_mblocks;
+    const int m0 = mb * T::BM;
+    const int n_tiles = (V + T::BN - 1) / T::BN;
+    const int t_lo = grp * tiles_per_group, t_hi = min(n_tiles, t_lo + tiles_per_group);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wm0 = (warp / T::WN) * T::WTM, wn0 = (warp % T::WN) * T::WTN;
+    float *ctile = reinterpret_cast<float *>(smem);
+    TopList<KMAX> top;
+    top.init();
+    for (int tile = t_lo; tile < t_hi; ++tile) {
+        const int n0 = tile * T::BN;
+        float acc[T::MT][T::NT][4];
+        T::run(smem, Zt, d, m0, M, W, d, n0, V, d, acc);  // ends with a barrier: smem is free
+#pragma unroll
+        for (int i = 0; i < T::MT; ++i)
+#pragma unroll
+            for (int j = 0; j < T::NT; ++j)
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int row = wm0 + i * 16 + (lane >> 2) + (t >> 1) * 8;
+                    const int col = wn0 + j * 8 + (lane & 3) * 2 + (t & 1);
+                    ctile[row * LM_CSTRIDE + col] = acc[i][j][t];
+                }
+        __syncthreads();
+        if (threadIdx.x < T::BM) {
+            const float *rp = ctile + threadIdx.x * LM_CSTRIDE;
+            const int ncol = min(T::BN, V - n0);
+            for (int c = 0; c < ncol; ++c) top.push(rp[c], n0 + c);
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x < T::BM && m0 + threadIdx.x < M) {
+        const size_t o = ((size_t)(m0 + threadIdx.x) * n_groups + grp) * k;
+#pragma unroll
+        for (int i = 0; i < KMAX; ++i)
+            if (i < k) {
+                pval[o + i] = top.v[i];
+                pid[o + i] = top.id[i];
+            }
+    }
+}
+
+// One warp per row: k rounds of arg-best over the n_cand partial entries, order (value desc, id asc).
+__global__ void __launch_bounds__(128)
+topk_merge_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pid, int M, int n_cand, int k,
+                  int32_t *__restrict__ cand_id, float *__restrict__ cand_logit) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 4 + warp;
+    if (r >= M) return;
+    const float *v = pval + (size_t)r * n_cand;
+    const int32_t *id = pid + (size_t)r * n_cand;
+    float last_v = INFINITY;
+    int32_t last_id = -1;
+    for (int j = 0; j < k; ++j) {
+        float bv = -INFINITY;
+        int32_t bi = 0x7fffffff;
+        for (int c = lane; c < n_cand; c += 32) {
+            const float x = v[c];
+            const int32_t t = id[c];
+            // strictly after the previous pick in the (value desc, id asc) order
+            const bool after = (x < last_v) || (x == last_v && t > last_id);
+            if (after && (x > bv || (x == bv && t < bi))) {
+                bv = x;
+                bi = t;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) {
+                bv = ov;
+                bi = oi;
+            }
+        }
+        if (lane == 0) {
+            cand_id[(size_t)r * k + j] = bi;
+            cand_logit[(size_t)r * k + j] = bv;
+        }
+        last_v = bv;
+        last_id = bi;
+    }
+}
+
+// ------------------------------------------------------------------------------ P5 tree draw
+
+constexpr int DRAW_WARPS = 4;
+
+// One warp per sequence.  Lanes evaluate the exponentials; lane 0 does the short ordered sums so
+// that the arithmetic order is the plain sequential one.
+__global__ void __launch_bounds__(DRAW_WARPS * 32)
+tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__restrict__ anchor,
+                 const int32_t *__restrict__ cand_id, const float *__restrict__ cand_logit,
+                 const float *__restrict__ u_draw, int32_t *__restrict__ tree_tok,
+                 uint8_t *__restrict__ tree_cand, float *__restrict__ slot_q) {
+    __shared__ double sh_w[DRAW_WARPS][SPECROLL_MAX_TOPK];
+    __shared__ uint8_t sh_pick[DRAW_WARPS][SPECROLL_MAX_NODES];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * DRAW_WARPS + warp;
+    if (b >= B) return;
+    const int N = topo.N;
+    double *w = sh_w[warp];
+    uint8_t *pick = sh_pick[warp];
+    if (lane == 0) {
+        tree_tok[(size_t)b * N] = anchor[b];
+        tree_cand[(size_t)b * N] = 255;
+        slot_q[(size_t)b * N] = 1.0f;
+        pick[0] = 255;
+    }
+    __syncwarp();
+    for (int n = 1; n < N; ++n) {
+        const int u = topo.parent[n], hd = topo.depth[n] - 1;
+        const float *cl = cand_logit + ((size_t)b * K + hd) * k;
+        uint64_t taken = 0;
+        for (int e = 1; e < n; ++e)
+            if (topo.parent[e] == u) taken |= 1ull << pick[e];
+        // max over the remaining candidates
+        float mxf = -INFINITY;
+        for (int j = lane; j < k; j += 32)
+            if (!((taken >> j) & 1)) mxf = fmaxf(mxf, cl[j]);
+        mxf = warp_max(mxf);
+        for (int j = lane; j < k; j += 32)
+            w[j] = ((taken >> j) & 1) ? 0.0 : exp(((double)cl[j] - (double)mxf) / T);
+        __syncwarp();
+        if (lane == 0) {
+            double s = 0.0;
+            for (int j = 0; j < k; ++j) s += w[j];
+            const double uu = (double)u_draw[(size_t)b * N + n];
+            double cum = 0.0;
+            int sel = -1, last = -1;
+            for (int j = 0; j < k; ++j) {
+                if ((taken >> j) & 1) continue;
+                last = j;
+                cum += w[j] / s;
+                if (cum > uu) {
+                    sel = j;
+                    break;
+                }
+            }
+            if (sel < 0) sel = last;
+            pick[n] = (uint8_t)sel;
+            tree_tok[(size_t)b * N + n] = cand_id[((size_t)b * K + hd) * k + sel];
+            tree_cand[(size_t)b * N + n] = (uint8_t)sel;
+            slot_q[(size_t)b * N + n] = (float)(w[sel] / s);
+        }
+        __syncwarp();
+    }
+}
+
+// ------------------------------------------------------------------------------ host side
+
+struct ProposePlan {
+    int KX, M, n_mblocks, n_tiles, n_groups, tiles_per_group;
+    size_t off_xhat, off_z, off_zt, off_pval, off_pid, total;
+};
+
+static int make_plan(const specroll_propose_desc *d, bool affine, ProposePlan *p) {
+    if (!d || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->K < 1 || d->K > SPECROLL_MAX_HEADS ||
+        d->k < 1 || d->k > SPECROLL_MAX_TOPK || d->d < 64 || (d->d % 64) || d->V < 8 || (d->V % 8) ||
+        d->k > d->V || !(d->temperature > 0.f) || !(d->ln_eps >= 0.f) || !(d->rms_eps >= 0.f) ||
+        d->flags != 0)
+        return SPECROLL_EINVAL;
+    p->KX = affine ? d->K : 1;
+    p->M = d->B * d->K;
+    p->n_mblocks = (p->M + LmTile::BM - 1) / LmTile::BM;
+    p->n_tiles = (d->V + LmTile::BN - 1) / LmTile::BN;
+    int want = p->n_mblocks > 0 ? (2 * 148) / p->n_mblocks : 1;
+    if (want < 1) want = 1;
+    if (want > p->n_tiles) want = p->n_tiles;
+    p->tiles_per_group = (p->n_tiles + want - 1) / want;
+    p->n_groups = (p->n_tiles + p->tiles_per_group - 1) / p->tiles_per_group;
+    size_t o = 0;
+    const size_t B = d->B, K = d->K, dd = d->d, k = d->k;
+    p->off_xhat = o;
+    o += align_up((size_t)p->KX * B * dd * 2, 256);
+    p->off_z = o;
+    o += align_up(B * K * dd * 4, 256);
+    p->off_zt = o;
+    o += align_up(B * K * dd * 2, 256);
+    p->off_pval = o;
+    o += align_up((size_t)p->M * p->n_groups * k * 4, 256);
+    p->off_pid = o;
+    o += align_up((size_t)p->M * p->n_groups * k * 4, 256);
+    p->total = o + 256;
+    return SPECROLL_OK;
+}
+
+template <typename Kern>
+static int set_smem(Kern kern, int bytes) {
+    SR_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    return SPECROLL_OK;
+}
+
+static int launch_tree_draw(const Topo &topo, int B, int K, int k, float T, const int32_t *anchor,
+                            const int32_t *cand_id, const float *cand_logit, const float *u_draw,
+                            int32_t *tree_tok, uint8_t *tree_cand, float *slot_q, cudaStream_t st) {
+    if (B == 0) return SPECROLL_OK;
+    tree_draw_kernel<<<(B + DRAW_WARPS - 1) / DRAW_WARPS, DRAW_WARPS * 32, 0, st>>>(
+        topo, B, K, k, (double)T, anchor, cand_id, cand_logit, u_draw, tree_tok, tree_cand, slot_q);
+    SR_LAUNCH_CHECK();
+    return SPECROLL_OK;
+}
+
+}  // namespace specroll
+
+using namespace specroll;
+
+extern "C" size_t specroll_propose_workspace_bytes(const specroll_propose_desc *d) {
+    ProposePlan p;
+    if (make_plan(d, true, &p) != SPECROLL_OK) return 0;  // sized for the affine case (the larger one)
+    return p.total;
+}
+
+extern "C" int specroll_tree_draw(int32_t B, int32_t N, int32_t K, int32_t k, float temperature,
+                                  const int32_t *parent_host, const int32_t *anchor_tok,
+                                  const int32_t *cand_id, const float *cand_logit, const float *u_draw,
+                                  int32_t *tree_tok, uint8_t *tree_cand, float *slot_q, void *cuda_stream) {
+    if (B < 0 || K < 1 || K > SPECROLL_MAX_HEADS || k < 1 || k > SPECROLL_MAX_TOPK || !(temperature > 0.f))
+        return SPECROLL_EINVAL;
+    Topo topo;
+    if (build_topo(parent_host, N, K, k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (!anchor_tok || !cand_id || !cand_logit || !u_draw || !tree_tok || !tree_cand || !slot_q)
+        return SPECROLL_EINVAL;
+    return launch_tree_draw(topo, B, K, k, temperature, anchor_tok, cand_id, cand_logit, u_draw, tree_tok,
+                            tree_cand, slot_q, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, const int32_t *anchor_tok,
+                                const void *A, const void *bias, const void *ln_gamma, const void *ln_beta,
+                                const void *W, const float *m, const float *alpha,
+                                const int32_t *parent_host, const float *u_draw, int32_t *cand_id,
+                                float *cand_logit, int32_t *tree_tok, uint8_t *tree_cand, float *slot_q,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    ProposePlan p;
+    const bool affine = ln_gamma || ln_beta;
+    if (make_plan(d, affine, &p) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (!h || !anchor_tok || !A || !bias || !W || !u_draw || !cand_id || !cand_logit || !tree_tok ||
+        !tree_cand || !slot_q)
+        return SPECROLL_EINVAL;
+    Topo topo;
+    if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (!aligned16(h) || !aligned16(A) || !aligned16(bias) || !aligned16(W) || !aligned16(m) ||
+        !aligned16(ln_gamma) || !aligned16(ln_beta))
+        return SPECROLL_EALIGN;
+    if (d->B == 0) return SPECROLL_OK;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < p.total)
+        return SPECROLL_EWORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *ws = static_cast<char *>(workspace);
+    __nv_bfloat16 *xhat = reinterpret_cast<__nv_bfloat16 *>(ws + p.off_xhat);
+    float *z = reinterpret_cast<float *>(ws + p.off_z);
+    __nv_bfloat16 *zt = reinterpret_cast<__nv_bfloat16 *>(ws + p.off_zt);
+    float *pval = reinterpret_cast<float *>(ws + p.off_pval);
+    int32_t *pid = reinterpret_cast<int32_t *>(ws + p.off_pid);
+    const __nv_bfloat16 *hb = static_cast<const __nv_bfloat16 *>(h);
+    const int B = d->B, K = d->K, dd = d->d, k = d->k, V = d->V;
+
+    layernorm_kernel<<<B, LN_THREADS, dd * sizeof(float), st>>>(
+        hb, static_cast<const __nv_bfloat16 *>(ln_gamma), static_cast<const __nv_bfloat16 *>(ln_beta), xhat, B,
+        dd, p.KX, d->ln_eps);
+    SR_LAUNCH_CHECK();
+
+    {
+        int rc = set_smem(head_mlp_kernel, HeadTile::SMEM_BYTES);
+        if (rc) return rc;
+        dim3 grid((dd + HeadTile::BN - 1) / HeadTile::BN, (B + HeadTile::BM - 1) / HeadTile::BM, K);
+        head_mlp_kernel<<<grid, HeadTile::THREADS, HeadTile::SMEM_BYTES, st>>>(
+            xhat, p.KX, static_cast<const __nv_bfloat16 *>(A), static_cast<const __nv_bfloat16 *>(bias), hb, z,
+            B, K, dd);
+        SR_LAUNCH_CHECK();
+    }
+
+    reflex_kernel<<<B * K, RX_THREADS, 0, st>>>(z, m, alpha, zt, dd, d->rms_eps, d->clip_c);
+    SR_LAUNCH_CHECK();
+
+    {
+        const int grid = p.n_mblocks * p.n_groups;
+        const int smem = LmTile::SMEM_BYTES;  // >= 128 * 129 * 4 staging tile
+        static_assert(LmTile::SMEM_BYTES >= LmTile::BM * LM_CSTRIDE * 4, "staging tile must fit");
+        if (k <= 8) {
+            int rc = set_smem(lm_head_topk_kernel<8>, smem);
+            if (rc) return rc;
+            lm_head_topk_kernel<8><<<grid, LmTile::THREADS, smem, st>>>(
+                zt, static_cast<const __nv_bfloat16 *>(W), p.M, V, dd, k, p.n_mblocks, p.n_groups,
+                p.tiles_per_group, pval, pid);
+        } else {
+            int rc = set_smem(lm_head_topk_kernel<SPECROLL_MAX_TOPK>, smem);
+            if (rc) return rc;
+            lm_head_topk_kernel<SPECROLL_MAX_TOPK><<<grid, LmTile::THREADS, smem, st>>>(
+                zt, static_cast<const __nv_bfloat16 *>(W), p.M, V, dd, k, p.n_mblocks, p.n_groups,
+                p.tiles_per_group, pval, pid);
+        }
+        SR_LAUNCH_CHECK();
+    }
+
+    topk_merge_kernel<<<(p.M + 3) / 4, 128, 0, st>>>(pval, pid, p.M, p.n_groups * k, k, cand_id, cand_logit);
+    SR_LAUNCH_CHECK();
+
+    return launch_tree_draw(topo, B, K, k, d->temperature, anchor_tok, cand_id, cand_logit, u_draw, tree_tok,
+                            tree_cand, slot_q, st);
+}

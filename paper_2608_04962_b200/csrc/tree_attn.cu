@@ -1,0 +1,462 @@
+// Tree-verification attention, one layer: every tree node of every sequence attends to the
+// sequence's KV cache plus its own ancestors' tree rows.
+//
+// Work decomposition.  For one (sequence, KV head) all N*G query rows (G = Hq/Hkv query heads per
+// KV head) share the same keys and values, so they form the M dimension of one skinny GEMM pair:
+// each cached K/V element is read once for all of them.  A CTA owns a block of <= 128 of those
+// rows (one warp per 16 rows) and a contiguous chunk of the cache ("split-KV"); chunks are
+// sized on the host from the KV lengths so that long sequences are spread over many CTAs.
+// The tree's own K/V rows form one extra 64-token tile masked by the per-node ancestor bitmask;
+// it is processed by the CTA that owns the last chunk.  A sequence that needs a single chunk
+// writes its output directly; otherwise fp32 partials (O, running max, running sum) go to the
+// workspace and a second kernel combines them.
+//
+// Legacy tensor-core path: mma.sync m16n8k16 bf16 with fp32 accumulation, cp.async staging,
+// warp-shuffle online softmax in the log2 domain.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace specroll {
+
+constexpr int AT_BN = 64;       // KV tokens per tile
+constexpr int AT_STAGES = 3;
+constexpr int AT_MAX_WARPS = 8; // 128 query rows per CTA
+constexpr float LOG2E = 1.4426950408889634f;
+
+struct AttnArgs {
+    const __nv_bfloat16 *Q, *Kc, *Vc, *Kt, *Vt;
+    const int32_t *kv_indptr;
+    const int32_t *item_start;  // [B+1] exclusive prefix of the per-sequence chunk counts
+    __nv_bfloat16 *O;
+    float *lse;
+    float *part_o;   // [items, Hkv, rows_pad, D]
+    float *part_ml;  // [items, Hkv, rows_pad, 2]  (max in log2 units, sum)
+    int32_t B, N, Hq, Hkv, G, rows, rows_pad, n_rb, rows_per_block, chunk_tiles;
+    float scale_log2;  // scale * log2(e)
+};
+
+// item_start[b] = sum_{b' < b} max(1, ceil(tiles(b') / chunk_tiles))
+__global__ void attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles,
+                                 int32_t *__restrict__ item_start) {
+    // single thread: B is at most a few thousand and this runs concurrently with nothing
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        int acc = 0;
+        for (int b = 0; b < B; ++b) {
+            item_start[b] = acc;
+            const int L = kv_indptr[b + 1] - kv_indptr[b];
+            const int tiles = (L + AT_BN - 1) / AT_BN;
+            int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
+            acc += ns < 1 ? 1 : ns;
+        }
+        item_start[B] = acc;
+    }
+}
+
+template <int D>
+struct AttnSmem {
+    static constexpr int ROW_BYTES = D * 2;
+    static constexpr int CHUNKS = D / 8;  // 16-byte chunks per row
+    static constexpr int Q_BYTES = AT_MAX_WARPS * 16 * ROW_BYTES;
+    static constexpr int KV_BYTES = AT_BN * ROW_BYTES;
+    static constexpr int STAGE_BYTES = 2 * KV_BYTES;
+    static constexpr int TOTAL = Q_BYTES + AT_STAGES * STAGE_BYTES;
+    static __device__ __forceinline__ uint32_t off(int row, int chunk) {
+        return row * ROW_BYTES + ((chunk ^ (row & 7)) << 4);
+    }
+};
+
+template <int D>
+__global__ void __launch_bounds__(AT_MAX_WARPS * 32, 1)
+tree_attn_kernel(AttnArgs a, TopoMask mask) {
+    using S = AttnSmem<D>;
+    extern __shared__ __align__(128) unsigned char smem[];
+    const uint32_t sq = smem_u32(smem), skv = sq + S::Q_BYTES;
+    const int nthreads = blockDim.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- which work item
+    int bid = blockIdx.x;
+    const int rb = bid % a.n_rb;
+    bid /= a.n_rb;
+    const int hkv = bid % a.Hkv;
+    const int item = bid / a.Hkv;
+    int lo = 0, hi = a.B;  // largest b with item_start[b] <= item
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (a.item_start[mid] <= item) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int split = item - a.item_start[b];
+    const int n_splits = a.item_start[b + 1] - a.item_start[b];
+    const int kv0 = a.kv_indptr[b];
+    const int L = a.kv_indptr[b + 1] - kv0;
+    const int tiles_b = (L + AT_BN - 1) / AT_BN;
+    const int tps = (tiles_b + n_splits - 1) / n_splits;
+    const int t_lo = min(tiles_b, split * tps), t_hi = min(tiles_b, t_lo + tps);
+    const bool has_tree = (split == n_splits - 1);
+    const int n_it = (t_hi - t_lo) + (has_tree ? 1 : 0);
+
+    const int row0 = rb * a.rows_per_block;  // first query row (n*G+g) of this CTA
+    const int N = a.N, G = a.G;
+
+    // ---- Q tile -> smem (zero rows beyond `rows`)
+    {
+        const int nrow = a.rows_per_block;
+        for (int c = threadIdx.x; c < nrow * S::CHUNKS; c += nthreads) {
+            const int r = c / S::CHUNKS, ch = c % S::CHUNKS;
+            const int gr = row0 + r;
+            const bool ok = gr < a.rows;
+            const int n = ok ? gr / G : 0, g = ok ? gr % G : 0;
+            const __nv_bfloat16 *src = a.Q + (((size_t)b * N + n) * a.Hq + hkv * G + g) * D + ch * 8;
+            cp_async16(sq + S::off(r, ch), src, ok);
+        }
+        cp_async_commit();
+    }
+
+    auto load_tile = [&](int it, int stage) {
+        const uint32_t sk = skv + stage * S::STAGE_BYTES, sv = sk + S::KV_BYTES;
+        const bool tree = has_tree && (it == n_it - 1);
+        for (int c = threadIdx.x; c < AT_BN * S::CHUNKS; c += nthreads) {
+            const int r = c / S::CHUNKS, ch = c % S::CHUNKS;
+            const __nv_bfloat16 *ksrc, *vsrc;
+            bool ok;
+            if (!tree) {
+                const int tok = (t_lo + it) * AT_BN + r;
+                ok = tok < L;
+                const size_t o = ((size_t)(kv0 + (ok ? tok : 0)) * a.Hkv + hkv) * D + ch * 8;
+                ksrc = a.Kc + o;
+                vsrc = a.Vc + o;
+            } else {
+                ok = r < N;
+                const size_t o = (((size_t)b * N + (ok ? r : 0)) * a.Hkv + hkv) * D + ch * 8;
+                ksrc = a.Kt + o;
+                vsrc = a.Vt + o;
+            }
+            cp_async16(sk + S::off(r, ch), ksrc, ok);
+            cp_async16(sv + S::off(r, ch), vsrc, ok);
+        }
+    };
+
+#pragma unroll
+    for (int s = 0; s < AT_STAGES - 1; ++s) {
+        if (s < n_it) load_tile(s, s);
+        cp_async_commit();
+    }
+
+    // ---- per-thread state: rows g0 = lane/4 and g0+8 of this warp's 16-row slab
+    const int wrow = warp * 16;
+    const int r_lo = row0 + wrow + (lane >> 2), r_hi = r_lo + 8;
+    uint64_t anc_lo = 0, anc_hi = 0;
+    if (r_lo < a.rows) anc_lo = mask.anc[r_lo / G];
+    if (r_hi < a.rows) anc_hi = mask.anc[r_hi / G];
+
+    uint32_t qf[D / 16][4];
+    float oacc[D / 8][4];
+#pragma unroll
+    for (int j = 0; j < D / 8; ++j)
+#pragma unroll
+        for (int t = 0; t < 4; ++t) oacc[j][t] = 0.f;
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+
+    for (int it = 0; it < n_it; ++it) {
+        cp_async_wait<AT_STAGES - 2>();
+        __syncthreads();
+        if (it == 0) {
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk)
+                ldmatrix_x4(qf[kk], sq + S::off(wrow + (lane & 15), kk * 2 + (lane >> 4)));
+        }
+        {
+            const int nx = it + AT_STAGES - 1;
+            if (nx < n_it) load_tile(nx, nx % AT_STAGES);
+            cp_async_commit();
+        }
+        const uint32_t sk = skv + (it % AT_STAGES) * S::STAGE_BYTES, sv = sk + S::KV_BYTES;
+        const bool tree = has_tree && (it == n_it - 1);
+
+        // ---- S = Q K^T   (16 x 64 per warp)
+        float sacc[AT_BN / 8][4];
+#pragma unroll
+        for (int j = 0; j < AT_BN / 8; ++j)
+#pragma unroll
+            for (int t = 0; t < 4; ++t) sacc[j][t] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+#pragma unroll
+            for (int jp = 0; jp < AT_BN / 16; ++jp) {
+                uint32_t r[4];
+                const int row = jp * 16 + (lane & 7) + ((lane >> 4) << 3), ch = kk * 2 + ((lane >> 3) & 1);
+                ldmatrix_x4(r, sk + S::off(row, ch));
+                mma_bf16_16816(sacc[2 * jp], qf[kk], r[0], r[1]);
+                mma_bf16_16816(sacc[2 * jp + 1], qf[kk], r[2], r[3]);
+            }
+        }
+
+        // ---- scale, mask, online softmax (log2 domain)
+        const int tok0 = (t_lo + it) * AT_BN;
+        float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < AT_BN / 8; ++j) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int col = j * 8 + (lane & 3) * 2 + e;
+                bool ok_lo, ok_hi;
+                if (tree) {
+                    ok_lo = (anc_lo >> col) & 1;
+                    ok_hi = (anc_hi >> col) & 1;
+                } else {
+                    ok_lo = ok_hi = (tok0 + col) < L;
+                }
+                const float v_lo = ok_lo ? sacc[j][e] * a.scale_log2 : -INFINITY;
+                const float v_hi = ok_hi ? sacc[j][2 + e] * a.scale_log2 : -INFINITY;
+                sacc[j][e] = v_lo;
+                sacc[j][2 + e] = v_hi;
+                mx_lo = fmaxf(mx_lo, v_lo);
+                mx_hi = fmaxf(mx_hi, v_hi);
+            }
+        }
+        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+        const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+        const float ms_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, ms_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
+        const float al_lo = ex2_approx(m_lo - ms_lo), al_hi = ex2_approx(m_hi - ms_hi);
+        m_lo = mn_lo;
+        m_hi = mn_hi;
+        float ps_lo = 0.f, ps_hi = 0.f;
+        uint32_t pf[AT_BN / 16][4];
+#pragma unroll
+        for (int j = 0; j < AT_BN / 8; ++j) {
+            const float p0 = ex2_approx(sacc[j][0] - ms_lo), p1 = ex2_approx(sacc[j][1] - ms_lo);
+            const float p2 = ex2_approx(sacc[j][2] - ms_hi), p3 = ex2_approx(sacc[j][3] - ms_hi);
+            ps_lo += p0 + p1;
+            ps_hi += p2 + p3;
+            pf[j >> 1][(j & 1) * 2] = pack_bf16x2(p0, p1);
+            pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16x2(p2, p3);
+        }
+        l_lo = l_lo * al_lo + ps_lo;
+        l_hi = l_hi * al_hi + ps_hi;
+#pragma unroll
+        for (int j = 0; j < D / 8; ++j) {
+            oacc[j][0] *= al_lo;
+            oacc[j][1] *= al_lo;
+            oacc[j][2] *= al_hi;
+            oacc[j][3] *= al_hi;
+        }
+
+        // ---- O += P V
+#pragma unroll
+        for (int kk = 0; kk < AT_BN / 16; ++kk) {
+#pragma unroll
+            for (int dp = 0; dp < D / 16; ++dp) {
+                uint32_t r[4];
+                const int row = kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), ch = dp * 2 + (lane >> 4);
+                ldmatrix_x4_trans(r, sv + S::off(row, ch));
+                mma_bf16_16816(oacc[2 * dp], pf[kk], r[0], r[1]);
+                mma_bf16_16816(oacc[2 * dp + 1], pf[kk], r[2], r[3]);
+            }
+        }
+    }
+    cp_async_wait<0>();
+
+    // ---- finish
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        const int gr = half ? r_hi : r_lo;
+        if (gr >= a.rows) continue;
+        const float mrow = half ? m_hi : m_lo, lrow = half ? l_hi : l_lo;
+        const int n = gr / G, g = gr % G;
+        if (n_splits == 1) {
+            const float inv = lrow > 0.f ? 1.0f / lrow : 0.f;
+            __nv_bfloat16 *dst = a.O + (((size_t)b * N + n) * a.Hq + hkv * G + g) * D;
+#pragma unroll
+            for (int j = 0; j < D / 8; ++j) {
+                const uint32_t v = pack_bf16x2(oacc[j][half * 2] * inv, oacc[j][half * 2 + 1] * inv);
+                *reinterpret_cast<uint32_t *>(dst + j * 8 + (lane & 3) * 2) = v;
+            }
+            if (a.lse && (lane & 3) == 0)
+                a.lse[((size_t)b * N + n) * a.Hq + hkv * G + g] = (mrow + log2f(lrow)) * 0.6931471805599453f;
+        } else {
+            const size_t prow = ((size_t)item * a.Hkv + hkv) * a.rows_pad + gr;
+            float *dst = a.part_o + prow * D;
+#pragma unroll
+            for (int j = 0; j < D / 8; ++j)
+                *reinterpret_cast<float2 *>(dst + j * 8 + (lane & 3) * 2) =
+                    make_float2(oacc[j][half * 2], oacc[j][half * 2 + 1]);
+            if ((lane & 3) == 0) {
+                a.part_ml[prow * 2] = mrow;
+                a.part_ml[prow * 2 + 1] = lrow;
+            }
+        }
+    }
+}
+
+// One warp per (b, n, hq): merges the chunks of sequences that were split.
+template <int D>
+__global__ void __launch_bounds__(128) attn_combine_kernel(AttnArgs a) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t idx = (size_t)blockIdx.x * 4 + warp;
+    const size_t total = (size_t)a.B * a.N * a.Hq;
+    if (idx >= total) return;
+    const int hq = idx % a.Hq;
+    const int n = (idx / a.Hq) % a.N;
+    const int b = idx / ((size_t)a.Hq * a.N);
+    const int it0 = a.item_start[b], ns = a.item_start[b + 1] - it0;
+    if (ns == 1) return;
+    const int hkv = hq / a.G, gr = n * a.G + hq % a.G;
+    float M = -INFINITY;
+    for (int s = 0; s < ns; ++s) {
+        const size_t prow = ((size_t)(it0 + s) * a.Hkv + hkv) * a.rows_pad + gr;
+        M = fmaxf(M, a.part_ml[prow * 2]);
+    }
+    constexpr int PER = D / 32;
+    float acc[PER];
+#pragma unroll
+    for (int t = 0; t < PER; ++t) acc[t] = 0.f;
+    float lsum = 0.f;
+    for (int s = 0; s < ns; ++s) {
+        const size_t prow = ((size_t)(it0 + s) * a.Hkv + hkv) * a.rows_pad + gr;
+        const float ms = a.part_ml[prow * 2];
+        const float w = (ms == -INFINITY) ? 0.f : ex2_approx(ms - M);
+        lsum += w * a.part_ml[prow * 2 + 1];
+        const float *src = a.part_o + prow * D + lane * PER;
+#pragma unroll
+        for (int t = 0; t < PER; ++t) acc[t] += w * src[t];
+    }
+    const float inv = lsum > 0.f ? 1.0f / lsum : 0.f;
+    __nv_bfloat16 *dst = a.O + idx * D + lane * PER;
+#pragma unroll
+    for (int t = 0; t < PER; ++t) dst[t] = __float2bfloat16_rn(acc[t] * inv);
+    if (a.lse && lane == 0) a.lse[idx] = (M + log2f(lsum)) * 0.6931471805599453f;
+}
+
+// ------------------------------------------------------------------------------ host side
+
+struct AttnPlan {
+    int rows, n_rb, rows_per_block, rows_pad, chunk_tiles, items;
+    size_t off_items, off_po, off_pml, total;
+};
+
+static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
+    if (!d || !indptr_host || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->Hq < 1 || d->Hkv < 1 ||
+        (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || d->flags != 0)
+        return SPECROLL_EINVAL;
+    const int G = d->Hq / d->Hkv;
+    p->rows = d->N * G;
+    p->n_rb = (p->rows + AT_MAX_WARPS * 16 - 1) / (AT_MAX_WARPS * 16);
+    p->rows_per_block = ((p->rows + p->n_rb - 1) / p->n_rb + 15) / 16 * 16;
+    p->rows_pad = p->rows_per_block * p->n_rb;
+    long long tiles_total = 0;
+    int max_tiles = 0;
+    for (int b = 0; b < d->B; ++b) {
+        const int L = indptr_host[b + 1] - indptr_host[b];
+        if (L < 0) return SPECROLL_EINVAL;
+        const int t = (L + AT_BN - 1) / AT_BN;
+        tiles_total += t;
+        if (t > max_tiles) max_tiles = t;
+    }
+    // chunk length: about four CTAs' worth of work per SM over the whole launch, at least 8 tiles
+    // (512 tokens) so that the fp32 partials stay a small fraction of the KV bytes
+    long long ctas_per_tile = (long long)d->Hkv * p->n_rb;
+    long long ct = (tiles_total * ctas_per_tile + 148 * 4 - 1) / (148 * 4);
+    if (ct < 8) ct = 8;
+    if (ct > max_tiles) ct = max_tiles > 0 ? max_tiles : 1;
+    p->chunk_tiles = (int)ct;
+    int items = 0;
+    for (int b = 0; b < d->B; ++b) {
+        const int L = indptr_host[b + 1] - indptr_host[b];
+        const int t = (L + AT_BN - 1) / AT_BN;
+        const int ns = (t + p->chunk_tiles - 1) / p->chunk_tiles;
+        items += ns < 1 ? 1 : ns;
+    }
+    p->items = items;
+    size_t o = 0;
+    p->off_items = o;
+    o += align_up((size_t)(d->B + 1) * 4, 256);
+    p->off_po = o;
+    o += align_up((size_t)items * d->Hkv * p->rows_pad * d->D * 4, 256);
+    p->off_pml = o;
+    o += align_up((size_t)items * d->Hkv * p->rows_pad * 2 * 4, 256);
+    p->total = o + 256;
+    return SPECROLL_OK;
+}
+
+template <int D>
+static int launch_attn(const AttnArgs &a, const TopoMask &mask, const AttnPlan &p, int Hkv, size_t n_out,
+                       cudaStream_t st) {
+    using S = AttnSmem<D>;
+    SR_CUDA_TRY(cudaFuncSetAttribute(tree_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
+    const int threads = (p.rows_per_block / 16) * 32;
+    const unsigned grid = (unsigned)p.items * Hkv * p.n_rb;
+    tree_attn_kernel<D><<<grid, threads, S::TOTAL, st>>>(a, mask);
+    SR_LAUNCH_CHECK();
+    attn_combine_kernel<D><<<(unsigned)((n_out + 3) / 4), 128, 0, st>>>(a);
+    SR_LAUNCH_CHECK();
+    return SPECROLL_OK;
+}
+
+}  // namespace specroll
+
+using namespace specroll;
+
+extern "C" size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *d,
+                                                     const int32_t *kv_indptr_host) {
+    AttnPlan p;
+    if (make_attn_plan(d, kv_indptr_host, &p) != SPECROLL_OK) return 0;
+    return p.total;
+}
+
+extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, const void *Kc, const void *Vc,
+                                  const int32_t *kv_indptr_dev, const int32_t *kv_indptr_host, const void *Kt,
+                                  const void *Vt, const int32_t *parent_host, void *O, float *lse,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    AttnPlan p;
+    if (make_attn_plan(d, kv_indptr_host, &p) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (!Q || !kv_indptr_dev || !Kt || !Vt || !O) return SPECROLL_EINVAL;
+    const long long T_kv = kv_indptr_host[d->B] - kv_indptr_host[0];
+    if (T_kv > 0 && (!Kc || !Vc)) return SPECROLL_EINVAL;
+    Topo topo;
+    TopoMask mask;
+    if (build_topo(parent_host, d->N, -1, -1, &topo, &mask) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (!aligned16(Q) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(Kt) || !aligned16(Vt) || !aligned16(O))
+        return SPECROLL_EALIGN;
+    if (d->B == 0) return SPECROLL_OK;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < p.total)
+        return SPECROLL_EWORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *ws = static_cast<char *>(workspace);
+    AttnArgs a;
+    a.Q = static_cast<const __nv_bfloat16 *>(Q);
+    a.Kc = static_cast<const __nv_bfloat16 *>(Kc);
+    a.Vc = static_cast<const __nv_bfloat16 *>(Vc);
+    a.Kt = static_cast<const __nv_bfloat16 *>(Kt);
+    a.Vt = static_cast<const __nv_bfloat16 *>(Vt);
+    a.kv_indptr = kv_indptr_dev;
+    a.item_start = reinterpret_cast<int32_t *>(ws + p.off_items);
+    a.O = static_cast<__nv_bfloat16 *>(O);
+    a.lse = lse;
+    a.part_o = reinterpret_cast<float *>(ws + p.off_po);
+    a.part_ml = reinterpret_cast<float *>(ws + p.off_pml);
+    a.B = d->B;
+    a.N = d->N;
+    a.Hq = d->Hq;
+    a.Hkv = d->Hkv;
+    a.G = d->Hq / d->Hkv;
+    a.rows = p.rows;
+    a.rows_pad = p.rows_pad;
+    a.n_rb = p.n_rb;
+    a.rows_per_block = p.rows_per_block;
+    a.chunk_tiles = p.chunk_tiles;
+    a.scale_log2 = d->scale * LOG2E;
+    attn_prep_kernel<<<1, 32, 0, st>>>(kv_indptr_dev, d->B, p.chunk_tiles, reinterpret_cast<int32_t *>(ws + p.off_items));
+    SR_LAUNCH_CHECK();
+    const size_t n_out = (size_t)d->B * d->N * d->Hq;
+    if (d->D == 128) return launch_attn<128>(a, mask, p, d->Hkv, n_out, st);
+    return launch_attn<64>(a, mask, p, d->Hkv, n_out, st);
+}

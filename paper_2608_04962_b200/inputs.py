@@ -282,3 +282,15 @@ def verify_uniforms(w: Workload) -> Tuple[np.ndarray, np.ndarray]:
     u_acc = g.random(size=(w.B, w.N), dtype=np.float32)
     u_fin = g.random(size=(w.B,), dtype=np.float32)
     return u_acc, u_fin
+
+
+def synthetic_candidates(w: Workload) -> Tuple[np.ndarray, np.ndarray]:
+    """Stand-in candidate lists for verification-only runs: per (sequence, head) k distinct
+    token ids with logits sorted in descending order (gaps of a peaked head distribution)."""
+    g = rng(1000 * w.cfg_id + S_ACT + 700)
+    ids = np.empty((w.B, w.K, w.k), dtype=np.int32)
+    for b in range(w.B):
+        for hd in range(w.K):
+            ids[b, hd] = g.choice(w.V, size=w.k, replace=False)
+    lg = -np.sort(-(g.standard_normal(size=(w.B, w.K, w.k), dtype=np.float32) * np.float32(1.5)), axis=-1)
+    return ids, np.ascontiguousarray(lg, dtype=np.float32)

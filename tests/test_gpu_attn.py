@@ -1,0 +1,86 @@
+"""GPU parity: specroll_tree_attn against the CPU oracle on identical seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2608_04962_b200 import binding as S
+from paper_2608_04962_b200 import inputs as I
+from tests.util import dev, dev_bf16, host
+
+pytestmark = pytest.mark.gpu
+
+O_ATOL = 1e-2          # max abs error of the attention output (bf16 inputs, fp32 accumulate)
+
+
+def run_both(w, x, lengths=None):
+    if lengths is not None:
+        lengths = np.asarray(lengths, np.int32)
+        ip = np.zeros(w.B + 1, np.int32)
+        np.cumsum(lengths, out=ip[1:])
+        g = I.rng(4242)
+        x = dict(x)
+        x["kv_indptr"] = ip
+        x["Kc"] = I.f32_to_bf16_bits(g.standard_normal((int(ip[-1]), w.Hkv, w.D), dtype=np.float32))
+        x["Vc"] = I.f32_to_bf16_bits(g.standard_normal((int(ip[-1]), w.Hkv, w.D), dtype=np.float32))
+    o = ref.tree_attn(x["Q"], x["Kc"], x["Vc"], x["kv_indptr"], x["Kt"], x["Vt"], x["parent"], want_lse=True)
+    O, lse = S.tree_attn(dev_bf16(x["Q"]), dev_bf16(x["Kc"]), dev_bf16(x["Vc"]), dev(x["kv_indptr"]),
+                         x["kv_indptr"], dev_bf16(x["Kt"]), dev_bf16(x["Vt"]), x["parent"], want_lse=True)
+    torch.cuda.synchronize()
+    return o, host(O.float()).astype(np.float64), host(lse).astype(np.float64)
+
+
+def check(o, O, lse):
+    err = np.abs(O - o["O64"]).max()
+    assert err <= O_ATOL, err
+    np.testing.assert_allclose(lse, o["lse"], atol=2e-3, rtol=0)
+    return err
+
+
+def test_tiny_config():
+    w = I.WORKLOADS["tiny"]
+    o, O, lse = run_both(w, I.attn_inputs(w))
+    check(o, O, lse)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,N", [(12, 2, 128, 16), (28, 4, 128, 32), (40, 8, 128, 48), (10, 2, 64, 13),
+                                        (28, 4, 128, 64), (4, 4, 128, 1), (14, 2, 64, 37)])
+def test_group_sizes_head_dims_and_tree_sizes(Hq, Hkv, D, N):
+    # G = 6, 7, 5, 5, 7, 1, 7; rows = 96, 224, 240, 65, 448, 1, 259 (one to four row blocks)
+    K = 5
+    w = I.scaled(I.WORKLOADS["qwen7b"], B=5, N=N, K=K, Hq=Hq, Hkv=Hkv, D=D, kv_a=300, kv_b=900)
+    x = I.attn_inputs(w)
+    o, O, lse = run_both(w, x, lengths=[700, 64, 1, 333, 129])
+    check(o, O, lse)
+
+
+def test_ragged_lengths_empty_cache_and_split_kv():
+    # one long sequence forces several chunks per sequence; zero-length and sub-tile caches ride along
+    w = I.scaled(I.WORKLOADS["qwen1.5b"], B=7, N=16)
+    x = I.attn_inputs(w)
+    o, O, lse = run_both(w, x, lengths=[0, 5000, 63, 64, 65, 2049, 777])
+    check(o, O, lse)
+    # the same data with everything short: single-chunk direct-write path
+    o2, O2, lse2 = run_both(w, x, lengths=[0, 17, 63, 64, 65, 100, 1])
+    check(o2, O2, lse2)
+
+
+def test_reduced_batches_of_the_large_configs():
+    for name, B in (("qwen1.5b", 12), ("qwen7b", 4), ("qwen14b", 2)):
+        w = I.scaled(I.WORKLOADS[name], B=B)
+        o, O, lse = run_both(w, I.attn_inputs(w))
+        check(o, O, lse)
+
+
+def test_scale_argument_and_topology_errors():
+    w = I.scaled(I.WORKLOADS["tiny"], B=2)
+    x = I.attn_inputs(w)
+    args = (dev_bf16(x["Q"]), dev_bf16(x["Kc"]), dev_bf16(x["Vc"]), dev(x["kv_indptr"]), x["kv_indptr"],
+            dev_bf16(x["Kt"]), dev_bf16(x["Vt"]))
+    O = S.tree_attn(*args, x["parent"], scale=0.05)
+    want = ref.tree_attn(x["Q"], x["Kc"], x["Vc"], x["kv_indptr"], x["Kt"], x["Vt"], x["parent"], scale=0.05)
+    assert np.abs(host(O.float()) - want["O64"]).max() <= O_ATOL
+    bad = x["parent"].copy()
+    bad[2] = 2
+    with pytest.raises(S.SpecrollError):
+        S.tree_attn(*args, bad)

@@ -1,0 +1,129 @@
+"""GPU parity: specroll_propose / specroll_tree_draw against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2608_04962_b200 import binding as S
+from paper_2608_04962_b200 import inputs as I
+from tests.util import dev, dev_bf16, host
+
+pytestmark = pytest.mark.gpu
+
+TIE = 1e-3             # top-k sets may differ only among logits within this distance of the k-th
+
+
+def gpu_propose(w, x, **kw):
+    g = S.propose(dev_bf16(x["h"]), dev(x["anchor"]), dev_bf16(x["A"]), dev_bf16(x["bias"]), dev_bf16(x["W"]),
+                  dev(x["m"]) if x.get("m") is not None else None,
+                  dev(x["alpha"]) if x.get("alpha") is not None else None,
+                  x["parent"], dev(x["u_draw"]), k=w.k, temperature=w.temperature, clip_c=w.clip_c, **kw)
+    torch.cuda.synchronize()
+    return {k: host(v) for k, v in g.items()}
+
+
+def check_candidates(w, x, g, logit_atol, **okw):
+    """Top-k sets against the oracle's full logits, tie-aware; returns rows whose lists are identical."""
+    hd = ref.heads(x["h"], x["A"], x["bias"], m=x.get("m"), alpha=x.get("alpha"), clip_c=w.clip_c, **okw)
+    full = ref.lm_logits(hd["zt"], x["W"])                      # [B*K, V] fp64
+    oid, ol = ref.topk(full, w.k)
+    gid = g["cand_id"].reshape(-1, w.k)
+    gl = g["cand_logit"].reshape(-1, w.k).astype(np.float64)
+    kth = ol[:, -1].astype(np.float64)
+    rows = np.arange(full.shape[0])[:, None]
+    assert (gid >= 0).all() and (gid < w.V).all()
+    assert (np.sort(gid, 1)[:, 1:] != np.sort(gid, 1)[:, :-1]).all()          # distinct
+    picked = full[rows, gid]
+    assert (picked >= kth[:, None] - TIE).all()                               # nothing clearly outside
+    must = full > (kth[:, None] + TIE)                                        # clearly inside
+    got = np.zeros_like(must)
+    got[rows, gid] = True
+    assert (got | ~must).all()
+    np.testing.assert_allclose(gl, picked, atol=logit_atol, rtol=0)           # reported logits
+    assert (np.diff(gl, axis=1) <= 0).all()                                   # sorted descending
+    same = (gid == oid).all(1)
+    return same.reshape(w.B, w.K), oid.reshape(w.B, w.K, w.k), ol.reshape(w.B, w.K, w.k)
+
+
+def check_tree(w, x, g, same, T=1.0):
+    """Where a sequence's candidate lists equal the oracle's, the drawn tree must too."""
+    d = ref.tree_draw(x["parent"], x["anchor"], g["cand_id"], g["cand_logit"], x["u_draw"], temperature=T)
+    # the oracle draw from the GPU's own lists isolates the draw step: exact tokens expected
+    assert np.array_equal(g["tree_tok"], d["tree_tok"])
+    assert np.array_equal(g["tree_cand"], d["tree_cand"])
+    np.testing.assert_allclose(g["slot_q"], d["slot_q"], rtol=1e-5)
+    assert (g["tree_tok"][:, 0] == x["anchor"]).all()
+
+
+@pytest.mark.parametrize("peaked", [False, True])
+def test_tiny_config(peaked):
+    w = I.WORKLOADS["tiny"]
+    x = I.propose_inputs(w, peaked=peaked)
+    g = gpu_propose(w, x)
+    same, _, _ = check_candidates(w, x, g, logit_atol=2e-2 if peaked else 2e-5)
+    check_tree(w, x, g, same)
+    if peaked:
+        assert same.mean() > 0.9
+
+
+@pytest.mark.parametrize("B,K,k,d,V,N", [(37, 4, 8, 512, 3000, 16), (130, 2, 8, 256, 1288, 9),
+                                         (9, 5, 16, 320, 2056, 24), (64, 4, 8, 1536, 8192, 16)])
+def test_ragged_shapes(B, K, k, d, V, N):
+    # rows and vocabulary not multiples of the 128-wide tiles; k above the fast-path size
+    w = I.scaled(I.WORKLOADS["qwen1.5b"], B=B, K=K, k=k, d=d, V=V, N=N, alpha_heads=(0.025, 0.01, 0.006, 0.004, 0.003)[:K])
+    x = I.propose_inputs(w, peaked=True)
+    g = gpu_propose(w, x)
+    same, _, _ = check_candidates(w, x, g, logit_atol=5e-2)
+    check_tree(w, x, g, same)
+    assert same.mean() > 0.9
+
+
+def test_reflex_abstain_clip_and_affine_layernorm():
+    w = I.scaled(I.WORKLOADS["tiny"], B=16, V=2048)
+    x = I.propose_inputs(w, peaked=True)
+    # (a) no memory at all
+    x0 = dict(x, m=None, alpha=None)
+    g0 = gpu_propose(w, x0)
+    check_candidates(w, x0, g0, logit_atol=2e-2)
+    # (b) strong correction so that the clip binds everywhere and changes the candidates
+    x1 = dict(x, alpha=np.full((w.B, w.K), 0.5, np.float32))
+    g1 = gpu_propose(w, x1)
+    check_candidates(w, x1, g1, logit_atol=2e-2)
+    assert (g1["cand_id"] != g0["cand_id"]).any()
+    # (c) per-head LayerNorm affine
+    gg = I.rng(31)
+    gam = I.f32_to_bf16_bits(gg.uniform(0.5, 1.5, (w.K, w.d)).astype(np.float32))
+    bet = I.f32_to_bf16_bits((0.1 * gg.standard_normal((w.K, w.d))).astype(np.float32))
+    g2 = gpu_propose(w, x, ln_gamma=dev_bf16(gam), ln_beta=dev_bf16(bet))
+    check_candidates(w, x, g2, logit_atol=2e-2, gamma=gam, beta=bet)
+
+
+def test_tree_draw_alone_matches_exactly():
+    for name in ("qwen1.5b", "qwen7b", "qwen14b"):
+        w = I.scaled(I.WORKLOADS[name], B=200)
+        parent = I.topology(w)
+        cid, cl = I.synthetic_candidates(w)
+        u = I.uniforms24(3, (w.B, w.N))
+        anchor = np.arange(w.B, dtype=np.int32)
+        for T in (1.0, 0.6):
+            o = ref.tree_draw(parent, anchor, cid, cl, u, temperature=T)
+            g = S.tree_draw(parent, dev(anchor), dev(cid), dev(cl), dev(u), temperature=T)
+            assert np.array_equal(host(g["tree_tok"]), o["tree_tok"])
+            assert np.array_equal(host(g["tree_cand"]), o["tree_cand"])
+            np.testing.assert_allclose(host(g["slot_q"]), o["slot_q"], rtol=1e-6)
+    # the paper's nominal (5,4,0) allocation
+    parent = I.paper_540_topology()
+    w = I.scaled(I.WORKLOADS["tiny"], B=50, N=10, K=3, k=8, V=4096)
+    cid, cl = I.synthetic_candidates(w)
+    u = I.uniforms24(4, (w.B, 10))
+    o = ref.tree_draw(parent, np.zeros(w.B, np.int32), cid, cl, u)
+    g = S.tree_draw(parent, dev(np.zeros(w.B, np.int32)), dev(cid), dev(cl), dev(u))
+    assert np.array_equal(host(g["tree_tok"]), o["tree_tok"])
+
+
+def test_bad_arguments():
+    w = I.scaled(I.WORKLOADS["tiny"], B=2)
+    x = I.propose_inputs(w)
+    bad = dict(x, parent=np.array([-1, 0, 0, 0, 1, 2, 3, 3], np.int32))   # three children > k = 2
+    with pytest.raises(S.SpecrollError):
+        gpu_propose(w, bad)

@@ -1,0 +1,126 @@
+"""GPU parity: specroll_verify against the CPU oracle on identical seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2608_04962_b200 import binding as S
+from paper_2608_04962_b200 import inputs as I
+from tests.util import dev, dev_bf16, host
+
+pytestmark = pytest.mark.gpu
+
+NEAR_TIE = 1e-4        # |u - ratio| below this may flip the decision (counted)
+P_RTOL = 1e-3          # relative tolerance on normalised probabilities
+
+
+def run_both(w, parent, logits, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin):
+    o = ref.verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin,
+                   temperature=w.temperature)
+    g = S.verify(dev_bf16(logits), parent, dev(tree_tok), dev(tree_cand), dev(cand_id), dev(cand_logit),
+                 dev(u_acc), dev(u_fin), temperature=w.temperature)
+    torch.cuda.synchronize()
+    return o, {k: host(v) for k, v in g.items()}
+
+
+def check(w, o, g, logits):
+    B = w.B
+    # softmax statistics: max is exact (a bf16 value), the normaliser to 1e-3 relative
+    assert np.array_equal(g["row_max"].astype(np.float64), o["row_max"])
+    np.testing.assert_allclose(g["row_sum"], o["row_sum"], rtol=P_RTOL)
+    assert np.abs(g["row_sum"] / o["row_sum"] - 1).max() < 2e-5   # what bit-exact acceptance needs
+    same = (g["n_acc"] == o["n_acc"]) & (g["path_node"] == o["path_node"]).all(1) & \
+           (g["out_tok"] == o["out_tok"]).all(1) & (g["term_node"] == o["term_node"]) & \
+           (g["term_kind"] == o["term_kind"])
+    bad = np.flatnonzero(~same)
+    near = 0
+    for b in bad:
+        walk_same = g["n_acc"][b] == o["n_acc"][b] and (g["path_node"][b] == o["path_node"][b]).all()
+        if not walk_same:
+            assert o["min_margin"][b] < NEAR_TIE, (b, o["min_margin"][b], g["n_acc"][b], o["n_acc"][b])
+        else:
+            # only the terminal inverse-CDF draw differs: neighbouring token at a bracket edge
+            n = o["n_acc"][b]
+            assert (g["out_tok"][b, :n] == o["out_tok"][b, :n]).all()
+            assert o["fin_margin"][b] < 1e-6, (b, o["fin_margin"][b])
+        near += 1
+    assert near <= max(1, int(1e-3 * B)) and near / max(B, 1) < (1e-3 if B >= 1000 else 1.0), (near, B)
+    ok = np.isfinite(o["min_margin"])
+    mm_ok = np.abs(g["min_margin"][ok] - o["min_margin"][ok]) <= 1e-3 * np.maximum(1.0, o["min_margin"][ok])
+    assert mm_ok[same[ok]].all()
+    return len(bad)
+
+
+def test_tiny_config_with_oracle_proposals():
+    w = I.WORKLOADS["tiny"]
+    x = I.propose_inputs(w, peaked=True)
+    pr = ref.propose(x["h"], x["anchor"], x["A"], x["bias"], x["W"], x["m"], x["alpha"], x["parent"],
+                     x["u_draw"], k=w.k, clip_c=w.clip_c)
+    u_acc, u_fin = I.verify_uniforms(w)
+    for flat in (False, True):
+        lg = I.target_logits(w, x["parent"], pr["tree_tok"], flat=flat)
+        o, g = run_both(w, x["parent"], lg, pr["tree_tok"], pr["tree_cand"], pr["cand_id"], pr["cand_logit"],
+                        u_acc, u_fin)
+        check(w, o, g, lg)
+
+
+@pytest.mark.parametrize("name,B,V,T", [("qwen1.5b", 48, 151936, 1.0), ("qwen7b", 24, 152064, 0.7),
+                                        ("qwen14b", 12, 152064, 1.0), ("qwen1.5b", 300, 4104, 1.3)])
+def test_reduced_batches_of_the_large_configs(name, B, V, T):
+    w = I.scaled(I.WORKLOADS[name], B=B, V=V, temperature=T)
+    parent = I.topology(w)
+    cid, cl = I.synthetic_candidates(w)
+    u_draw = I.uniforms24(77, (w.B, w.N))
+    d = ref.tree_draw(parent, np.zeros(w.B, np.int32), cid, cl, u_draw, temperature=T)
+    lg = I.target_logits(w, parent, d["tree_tok"])
+    u_acc, u_fin = I.verify_uniforms(w)
+    o, g = run_both(w, parent, lg, d["tree_tok"], d["tree_cand"], cid, cl, u_acc, u_fin)
+    check(w, o, g, lg)
+    assert o["n_acc"].max() >= 1          # the workload does accept something
+    # accepted-length statistics of the two sides agree
+    assert abs(g["n_acc"].mean() - o["n_acc"].mean()) < 0.05
+
+
+def test_many_sequences_small_vocab_mismatch_budget():
+    # 20000 sequences: the 0.1 % budget on near-tie decisions is measurable here
+    w = I.scaled(I.WORKLOADS["tiny"], B=20000, V=64, K=3, k=4, N=8)
+    parent = I.topology(w)
+    cid, cl = I.synthetic_candidates(w)
+    d = ref.tree_draw(parent, np.zeros(w.B, np.int32), cid, cl, I.uniforms24(5, (w.B, w.N)))
+    lg = I.target_logits(w, parent, d["tree_tok"], boost=3.0)
+    u_acc, u_fin = I.verify_uniforms(w)
+    o, g = run_both(w, parent, lg, d["tree_tok"], d["tree_cand"], cid, cl, u_acc, u_fin)
+    n_bad = check(w, o, g, lg)
+    assert n_bad / w.B < 1e-3
+    near = np.mean(o["min_margin"] < NEAR_TIE)
+    assert near < 1e-3 * 8                 # near ties are rare in the workload itself
+
+
+def test_lone_root_and_chain_and_star_topologies():
+    for parent in ([-1], [-1, 0, 1, 2], [-1, 0, 0, 0, 0]):
+        N = len(parent)
+        w = I.scaled(I.WORKLOADS["tiny"], B=16, N=N, V=512, K=3, k=4, fixed_parent=tuple(parent))
+        parent = np.array(parent, np.int32)
+        cid, cl = I.synthetic_candidates(w)
+        d = ref.tree_draw(parent, np.zeros(w.B, np.int32), cid, cl, I.uniforms24(9, (w.B, N)))
+        lg = I.target_logits(w, parent, d["tree_tok"], boost=6.0)
+        u_acc, u_fin = I.verify_uniforms(w)
+        o, g = run_both(w, parent, lg, d["tree_tok"], d["tree_cand"], cid, cl, u_acc, u_fin)
+        check(w, o, g, lg)
+
+
+def test_bad_arguments_are_refused_without_touching_the_device():
+    w = I.scaled(I.WORKLOADS["tiny"], B=2)
+    parent = I.topology(w)
+    cid, cl = I.synthetic_candidates(w)
+    lg = dev_bf16(np.zeros((w.B, w.N, w.V), np.uint16))
+    args = (dev(np.zeros((w.B, w.N), np.int32)), dev(np.zeros((w.B, w.N), np.uint8)), dev(cid), dev(cl),
+            dev(np.zeros((w.B, w.N), np.float32)), dev(np.zeros(w.B, np.float32)))
+    bad_parent = parent.copy()
+    bad_parent[3] = 5                      # not topological
+    with pytest.raises(S.SpecrollError):
+        S.verify(lg, bad_parent, *args)
+    with pytest.raises(S.SpecrollError):
+        S.verify(lg, parent, *args, temperature=0.0)
+    with pytest.raises(S.SpecrollError):
+        S.verify(lg, parent, *args, workspace=torch.empty(256, dtype=torch.uint8, device="cuda")[:16])
