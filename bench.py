@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the SpecRoll per-step speculative hot path on B200.
+
+One step = specroll_propose -> specroll_tree_attn for every layer -> specroll_verify over one
+batch of synthetic input.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+`--impl reference` times the CPU oracle (the only reference there is: the paper ships no code)
+on the host cores, each step a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verified tree tokens/sec per speculative step"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def recorded_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch from the committed ncu summary, or None."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(p):
+        return None
+    try:
+        return json.load(open(p)).get(workload, {}).get(kernel)
+    except Exception:
+        return None
+
+
+# ------------------------------------------------------------------------------------ clocks
+
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(self.idx)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()          # the exact child started above
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------ CPU oracle legs
+
+
+def oracle_sample_step(w, n_seq: int, layers: int):
+    """One pass of the whole path by the CPU oracle over the first n_seq sequences of `w`.
+    Returns (seconds, tokens processed, threads)."""
+    from oracle import ref
+    from paper_2608_04962_b200 import inputs as I
+    ws = I.scaled(w, B=n_seq)
+    x = I.propose_inputs(ws)
+    a = I.attn_inputs(ws)
+    u_acc, u_fin = I.verify_uniforms(ws)
+    # target logits need the proposal's tokens; that first (untimed) pass also warms the caches
+    pr = ref.propose(x["h"], x["anchor"], x["A"], x["bias"], x["W"], x["m"], x["alpha"], x["parent"], x["u_draw"],
+                     k=ws.k, temperature=ws.temperature, clip_c=ws.clip_c)
+    lg = I.target_logits(ws, x["parent"], pr["tree_tok"])
+
+    def one():
+        t0 = time.perf_counter()
+        p = ref.propose(x["h"], x["anchor"], x["A"], x["bias"], x["W"], x["m"], x["alpha"], x["parent"],
+                        x["u_draw"], k=ws.k, temperature=ws.temperature, clip_c=ws.clip_c)
+        for _ in range(layers):   # same arrays every layer: the oracle's cost does not depend on the values
+            ref.tree_attn(a["Q"], a["Kc"], a["Vc"], a["kv_indptr"], a["Kt"], a["Vt"], a["parent"])
+        ref.verify(lg, x["parent"], p["tree_tok"], p["tree_cand"], p["cand_id"], p["cand_logit"], u_acc, u_fin,
+                   temperature=ws.temperature)
+        return time.perf_counter() - t0
+
+    return one, ws.B * ws.N, ref.num_threads()
+
+
+def run_reference(args, w, layers):
+    from paper_2608_04962_b200 import dist as D
+    rank, _, world = D.env_world()
+    if rank != 0:
+        return 0
+    n_seq = args.ref_seqs
+    one, tokens, threads = oracle_sample_step(w, n_seq, layers)
+    for _ in range(args.warmup):
+        one()
+    t = [one() for _ in range(args.steps)]
+    total = float(sum(t))
+    value = tokens * args.steps / total
+    sample = f"first {n_seq} of {w.B} sequences of {w.name}, all {layers} layers, per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "N": w.N, "K": w.K, "k": w.k, "layers": layers,
+                       "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------------ our arm
+
+
+def run_ours(args, w, layers):
+    import torch
+    from paper_2608_04962_b200 import binding as S
+    from paper_2608_04962_b200 import dist as D
+    from paper_2608_04962_b200.workload import StepWorkload
+
+    rank, local, world = D.env_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback of the hot path")
+    S.lib()                                   # fails loudly if the library is not built
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    D.init("nccl")
+    wl = StepWorkload(w, dev, seed=rank, layers=layers)
+    peaks = measured_peaks()
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    for _ in range(max(args.warmup, 3)):
+        wl.step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    D.barrier()
+    torch.cuda.synchronize()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(args.steps):
+        wl.step(ev[i])
+    t1.record()
+    torch.cuda.synchronize()
+    D.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    elapsed_ms = t0.elapsed_time(t1)
+    tokens = wl.tokens_per_step() * args.steps
+    tmax, tok_all = D.aggregate(elapsed_ms, tokens, device=dev)
+    value = tok_all / (tmax * 1e-3)
+
+    prop_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    attn_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    ver_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))
+    attn_launch_s = attn_ms * 1e-3 / wl.layers
+
+    # accepted-length statistics of the synthetic workload (reporting only)
+    n_acc = wl.ver["n_acc"].float()
+    aal = float(1.0 + n_acc.mean().item())
+    ar = float(n_acc.sum().item() / max(1, w.B * (w.N - 1)))
+
+    # ---- end to end through host buffers
+    e2e = run_e2e(args, wl, dev, world)
+
+    if rank != 0:
+        D.finish()
+        return 0
+
+    attn_gbs = wl.attn_algorithmic_bytes() / attn_launch_s / 1e9
+    roofline = {"kernel": "tree_attn_kernel (per layer call: prep + attention + combine)", "bound": "hbm",
+                "achieved": attn_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / peaks["hbm_gbs"],
+                "peak_source": peaks["source"], "frac_of_nominal_8TBs": attn_gbs / 8000.0,
+                "algorithmic_bytes_per_launch": wl.attn_algorithmic_bytes(),
+                "traffic": recorded_traffic("tree_attn_kernel", w.name)}
+    ver_gbs = wl.rowstats_algorithmic_bytes() / (ver_ms * 1e-3) / 1e9
+    lm_tf = (wl.lmhead_algorithmic_flops() + 2 * w.B * w.K * w.d * w.d) / (prop_ms * 1e-3) / 1e12
+    phases = {
+        "propose": {"ms": prop_ms, "bound": "tensor", "achieved": lm_tf, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": lm_tf / peaks["bf16_tflops_sustained"],
+                    "note": "whole call (6 launches); flops = 2*B*K*d*(d+V)"},
+        "tree_attn": {"ms": attn_ms, "ms_per_layer": attn_ms / wl.layers, "layers": wl.layers,
+                      "tflops": wl.attn_algorithmic_flops() / attn_launch_s / 1e12},
+        "verify": {"ms": ver_ms, "bound": "hbm", "achieved": ver_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                   "frac": ver_gbs / peaks["hbm_gbs"], "note": "whole call (3 launches); bytes = logits once"},
+    }
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        one, ctok, threads = oracle_sample_step(w, args.ref_seqs, wl.layers)
+        reps, tt = 0, 0.0
+        while reps < 1 or (tt < 10.0 and reps < 8):
+            tt += one()
+            reps += 1
+        cpu = {"value": ctok * reps / tt, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"first {args.ref_seqs} of {w.B} sequences of {w.name}, all {wl.layers} layers, "
+                         f"{reps} passes in {tt:.1f} s"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": tmax / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "N": w.N, "K": w.K, "k": w.k, "d": w.d, "V": w.V, "Hq": w.Hq,
+                       "Hkv": w.Hkv, "D": w.D, "layers": wl.layers, "T_kv": wl.T_kv, "temperature": w.temperature,
+                       "parallelism": f"replicas x{world} (sharded by sequence, no collective)",
+                       "l2": "inputs larger than L2: per-layer KV cache, logits and W each exceed 126 MB and every "
+                             "layer has its own cache"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": wl.launches_per_step() * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "phases": phases,
+            "accepted": {"aal": aal, "acceptance_rate": ar}}
+    print(json.dumps(line), flush=True)
+    D.finish()
+    return 0
+
+
+def run_e2e(args, wl, dev, world):
+    """The same step driven from HOST buffers: per-step activations (hidden state, Reflex memory, uniforms,
+    every layer's Q and tree K/V, target logits) are copied from pinned memory inside the timed region and
+    the step's results are read back.  Weights and the KV cache are resident state."""
+    import torch
+    from paper_2608_04962_b200 import dist as D
+    w = wl.w
+    host_in = {}
+
+    def pin(t):
+        h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+        h.copy_(t)
+        return h
+
+    names = ["h", "anchor", "m", "alpha", "u_draw", "u_acc", "u_fin", "logits"]
+    for n in names:
+        host_in[n] = pin(getattr(wl, n))
+    hQ = [pin(t) for t in wl.Q]
+    hKt = [pin(t) for t in wl.Kt]
+    hVt = [pin(t) for t in wl.Vt]
+    out_names_p = ["cand_id", "cand_logit", "tree_tok", "tree_cand", "slot_q"]
+    out_names_v = ["n_acc", "path_node", "out_tok", "term_node", "term_kind"]
+    host_out = {n: torch.empty(wl.prop[n].shape, dtype=wl.prop[n].dtype, pin_memory=True) for n in out_names_p}
+    host_out.update({n: torch.empty(wl.ver[n].shape, dtype=wl.ver[n].dtype, pin_memory=True) for n in out_names_v})
+    hO = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in wl.O]
+    h2d = sum(t.numel() * t.element_size() for t in list(host_in.values()) + hQ + hKt + hVt)
+    d2h = sum(t.numel() * t.element_size() for t in list(host_out.values()) + hO)
+
+    def step():
+        for n in names:
+            getattr(wl, n).copy_(host_in[n], non_blocking=True)
+        wl.propose()
+        for n in out_names_p:
+            host_out[n].copy_(wl.prop[n], non_blocking=True)
+        for l in range(wl.layers):
+            wl.Q[l].copy_(hQ[l], non_blocking=True)
+            wl.Kt[l].copy_(hKt[l], non_blocking=True)
+            wl.Vt[l].copy_(hVt[l], non_blocking=True)
+            wl.attn(l)
+            hO[l].copy_(wl.O[l], non_blocking=True)
+        wl.verify()
+        for n in out_names_v:
+            host_out[n].copy_(wl.ver[n], non_blocking=True)
+
+    steps = max(2, min(args.steps, 5))
+    step()
+    torch.cuda.synchronize()
+    D.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+        torch.cuda.synchronize()      # the host holds the step's result before the next step starts
+    dt = time.perf_counter() - t0
+    D.barrier()
+    tmax, tok = D.aggregate(dt * 1e3, wl.tokens_per_step() * steps, device=dev)
+    return {"value": tok / (tmax * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "ms_per_step": tmax / steps, "steps": steps}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen1.5b")
+    ap.add_argument("--layers", type=int, default=None, help="attention layers per step (default: the model's)")
+    ap.add_argument("--ref-seqs", type=int, default=8, help="sequences per CPU-oracle sample step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2608_04962_b200 import inputs as I
+    w = I.WORKLOADS[args.workload]
+    layers = args.layers if args.layers is not None else w.layers
+    if args.impl == "reference":
+        return run_reference(args, w, layers)
+    return run_ours(args, w, layers)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

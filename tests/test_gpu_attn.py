@@ -30,9 +30,16 @@ def run_both(w, x, lengths=None):
     return o, host(O.float()).astype(np.float64), host(lse).astype(np.float64)
 
 
-def check(o, O, lse):
-    err = np.abs(O - o["O64"]).max()
-    assert err <= O_ATOL, err
+def check(o, O, lse, edge=False):
+    """edge=False: the bar of the workloads (cache length >= 64, so |O| < 1): max abs <= 1e-2.
+    edge=True: degenerate caches (0 or 1 cached tokens) give |O| of several units, where the bf16
+    output spacing alone (2^-8 |O|) exceeds 1e-2; there the bound scales with max(1, |O|)."""
+    diff = np.abs(O - o["O64"])
+    if edge:
+        assert (diff <= O_ATOL * np.maximum(1.0, np.abs(o["O64"]))).all(), diff.max()
+    else:
+        assert diff.max() <= O_ATOL, diff.max()
+    err = diff.max()
     np.testing.assert_allclose(lse, o["lse"], atol=2e-3, rtol=0)
     return err
 
@@ -51,6 +58,8 @@ def test_group_sizes_head_dims_and_tree_sizes(Hq, Hkv, D, N):
     w = I.scaled(I.WORKLOADS["qwen7b"], B=5, N=N, K=K, Hq=Hq, Hkv=Hkv, D=D, kv_a=300, kv_b=900)
     x = I.attn_inputs(w)
     o, O, lse = run_both(w, x, lengths=[700, 64, 1, 333, 129])
+    check(o, O, lse, edge=True)
+    o, O, lse = run_both(w, x, lengths=[700, 64, 70, 333, 129])
     check(o, O, lse)
 
 
@@ -59,10 +68,12 @@ def test_ragged_lengths_empty_cache_and_split_kv():
     w = I.scaled(I.WORKLOADS["qwen1.5b"], B=7, N=16)
     x = I.attn_inputs(w)
     o, O, lse = run_both(w, x, lengths=[0, 5000, 63, 64, 65, 2049, 777])
-    check(o, O, lse)
+    check(o, O, lse, edge=True)
     # the same data with everything short: single-chunk direct-write path
     o2, O2, lse2 = run_both(w, x, lengths=[0, 17, 63, 64, 65, 100, 1])
-    check(o2, O2, lse2)
+    check(o2, O2, lse2, edge=True)
+    o3, O3, lse3 = run_both(w, x, lengths=[64, 5000, 80, 64, 65, 2049, 777])
+    check(o3, O3, lse3)
 
 
 def test_reduced_batches_of_the_large_configs():
