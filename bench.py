@@ -211,7 +211,7 @@ def run_ours(args, w, layers):
     ar = float(n_acc.sum().item() / max(1, w.B * (w.N - 1)))
 
     # ---- end to end through host buffers
-    e2e = run_e2e(args, wl, dev, world)
+    e2e = None if args.no_e2e else run_e2e(args, wl, dev, world)
 
     if rank != 0:
         D.finish()
@@ -331,6 +331,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="attention layers per step (default: the model's)")
     ap.add_argument("--ref-seqs", type=int, default=8, help="sequences per CPU-oracle sample step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     from paper_2608_04962_b200 import inputs as I
     w = I.WORKLOADS[args.workload]
