@@ -38,6 +38,7 @@ extern "C" {
 #define SPECROLL_EWORKSPACE 3 /* workspace too small or misaligned */
 #define SPECROLL_ECUDA 4      /* a CUDA runtime call or kernel launch failed */
 #define SPECROLL_ETIMEOUT 5   /* a bounded device-side wait ran out (read from a status word) */
+#define SPECROLL_ELIMIT 6     /* problem larger than the fixed limit of an allocation-free entry point */
 
 #define SPECROLL_MAX_NODES 64
 #define SPECROLL_MAX_HEADS 8
@@ -167,6 +168,44 @@ int specroll_verify(const specroll_verify_desc *desc, const void *logits,
                     int32_t *out_tok, int32_t *term_node, int32_t *term_kind, float *row_max,
                     float *row_sum, float *min_margin, void *workspace, size_t workspace_bytes,
                     void *cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Allocation-free variant of specroll_verify.  (The paper has no counterpart: this is a
+ * deployment convenience of this library, not a step of the method.)
+ *
+ * Who needs it: hosts that cannot supply a workspace because they cannot allocate device memory
+ * at the point of the call.  Examples are a rollout server that hands the whole device to its
+ * KV-cache pool at start-up and then runs with allocation switched off (a cudaMalloc there either
+ * fails for lack of memory or stalls every stream while the driver serialises the device), and a
+ * plain-C client that only receives device pointers from another component and owns no allocator.
+ *
+ * Same arguments, outputs and results as specroll_verify, minus `workspace`: the scratch is a
+ * fixed array inside the library image (about 0.2 MB, present once on every GPU that loads the
+ * library, until the process exits).  The call performs no cudaMalloc/cudaFree and calls no
+ * allocating routine.
+ *
+ * Limits: B <= SPECROLL_STATIC_MAX_B and B * k <= SPECROLL_STATIC_MAX_BK; anything larger returns
+ * SPECROLL_ELIMIT and enqueues nothing (use specroll_verify with a caller workspace instead).
+ *
+ * First use on a device: the first call made with a given device current looks up the scratch
+ * array's device address (cudaGetSymbolAddress) and remembers it.  Make that first call outside
+ * any stream capture.  Later calls on that device do no set-up.
+ *
+ * Sharing: every call on a device uses the same array and finds the previous call's contents in
+ * it.  Nothing in it needs to start at zero (each call overwrites every entry it later reads), but
+ * two calls that overlap on the GPU (different streams, or different host threads without ordering)
+ * race on it.  Serialise them, or use specroll_verify with separate workspaces.
+ */
+#define SPECROLL_STATIC_MAX_B 4096
+#define SPECROLL_STATIC_MAX_BK 16384
+
+int specroll_verify_static(const specroll_verify_desc *desc, const void *logits,
+                           const int32_t *parent_host, const int32_t *tree_tok,
+                           const uint8_t *tree_cand, const int32_t *cand_id, const float *cand_logit,
+                           const float *u_acc, const float *u_fin, int32_t *n_acc,
+                           int32_t *path_node, int32_t *out_tok, int32_t *term_node,
+                           int32_t *term_kind, float *row_max, float *row_sum, float *min_margin,
+                           void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -50,6 +50,9 @@ const char *specroll_strerror(int code) {
         case SPECROLL_EALIGN: return "a tensor base pointer is not 16-byte aligned";
         case SPECROLL_EWORKSPACE: return "workspace too small or not 256-byte aligned";
         case SPECROLL_ETIMEOUT: return "a bounded device-side wait ran out";
+        case SPECROLL_ELIMIT:
+            return "problem exceeds the fixed size limit of this allocation-free entry point (use the "
+                   "variant that takes a caller workspace)";
         case SPECROLL_ECUDA:
             snprintf(g_msg, sizeof(g_msg), "CUDA error: %s", cudaGetErrorString(g_last_cuda));
             return g_msg;

@@ -13,6 +13,8 @@
 //                       the plain softmax mass.
 #include <math.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace specroll {
@@ -508,4 +510,51 @@ extern "C" int specroll_verify(const specroll_verify_desc *d, const void *logits
     terminal_kernel<<<d->B, TERM_THREADS, 0, st>>>(ta);
     SR_LAUNCH_CHECK();
     return SPECROLL_OK;
+}
+
+// ------------------------------------------------------------------------------ allocation-free variant
+//
+// Scratch of specroll_verify_static: lives in the library image, one copy per GPU that loads the
+// library, held until the process exits.  Layout = the workspace layout of specroll_verify for the
+// largest admitted problem (SPECROLL_STATIC_MAX_B sequences, SPECROLL_STATIC_MAX_BK residual entries).
+namespace specroll {
+constexpr size_t STATIC_SCRATCH_BYTES =
+    (SPECROLL_STATIC_MAX_BK * sizeof(double) + 255) / 256 * 256 +
+    (SPECROLL_STATIC_MAX_BK * sizeof(int32_t) + 255) / 256 * 256 +
+    (SPECROLL_STATIC_MAX_B * sizeof(int32_t) + 255) / 256 * 256 + 256;
+static __device__ __align__(256) unsigned char g_verify_scratch[STATIC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+static void *g_scratch_addr[MAX_DEVICES];  // device address of g_verify_scratch, per device ordinal
+static std::mutex g_scratch_mutex;
+}  // namespace specroll
+
+extern "C" int specroll_verify_static(const specroll_verify_desc *d, const void *logits,
+                                      const int32_t *parent_host, const int32_t *tree_tok,
+                                      const uint8_t *tree_cand, const int32_t *cand_id,
+                                      const float *cand_logit, const float *u_acc, const float *u_fin,
+                                      int32_t *n_acc, int32_t *path_node, int32_t *out_tok,
+                                      int32_t *term_node, int32_t *term_kind, float *row_max,
+                                      float *row_sum, float *min_margin, void *cuda_stream) {
+    if (check_verify_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (d->B > SPECROLL_STATIC_MAX_B || (long long)d->B * d->k > SPECROLL_STATIC_MAX_BK) return SPECROLL_ELIMIT;
+    if (specroll_verify_workspace_bytes(d) > STATIC_SCRATCH_BYTES) return SPECROLL_ELIMIT;
+    int dev = -1;
+    SR_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return SPECROLL_ELIMIT;
+    void *scratch = nullptr;
+    {
+        // In host code the array's name is only a handle; the kernels need its device address,
+        // which differs per GPU.  Looked up once per device, with that device current.
+        std::lock_guard<std::mutex> lock(g_scratch_mutex);
+        if (!g_scratch_addr[dev]) {
+            void *p = nullptr;
+            SR_CUDA_TRY(cudaGetSymbolAddress(&p, g_verify_scratch));
+            g_scratch_addr[dev] = p;
+        }
+        scratch = g_scratch_addr[dev];
+    }
+    return specroll_verify(d, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
+                           path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, scratch,
+                           STATIC_SCRATCH_BYTES, cuda_stream);
 }
