@@ -84,8 +84,12 @@ typedef struct {
     float ln_eps;      /* LayerNorm epsilon (1e-5 if the caller has no other value) */
     float rms_eps;     /* epsilon of the RMS normalisation of the memory */
     float clip_c;      /* <= 0: no L2 clip */
-    int32_t flags;     /* reserved, must be 0 */
+    int32_t flags;     /* 0, or SPECROLL_PROPOSE_LEGACY_MMA */
 } specroll_propose_desc;
+
+/* Run the vocabulary projection on the mma.sync kernel instead of the tcgen05 one (kept for
+ * comparison and for k > 8, where it is used anyway). */
+#define SPECROLL_PROPOSE_LEGACY_MMA 1
 
 size_t specroll_propose_workspace_bytes(const specroll_propose_desc *desc);
 
@@ -95,6 +99,12 @@ int specroll_propose(const specroll_propose_desc *desc, const void *h, const int
                      const int32_t *parent_host, const float *u_draw, int32_t *cand_id,
                      float *cand_logit, int32_t *tree_tok, uint8_t *tree_cand, float *slot_q,
                      void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Reads back the status word the last specroll_propose on this workspace left behind: SPECROLL_OK,
+ * or SPECROLL_ETIMEOUT if a bounded wait inside a kernel ran out (results are then invalid).
+ * Unlike the other calls this one synchronises `cuda_stream`.  (Housekeeping; the paper has no
+ * counterpart.) */
+int specroll_propose_status(const void *workspace, void *cuda_stream);
 
 /* The last step of the proposal alone (App. B.1): draw the tree from given candidate lists.
  * Same arguments and outputs as the corresponding ones of specroll_propose; needs no workspace. */

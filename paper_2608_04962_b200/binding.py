@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libspecroll.so")
 _lib = None
 
 EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
-           "specroll_propose_workspace_bytes", "specroll_propose", "specroll_tree_draw",
+           "specroll_propose_workspace_bytes", "specroll_propose", "specroll_propose_status",
+           "specroll_tree_draw",
            "specroll_tree_attn_workspace_bytes", "specroll_tree_attn",
            "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static")
 
@@ -62,7 +63,8 @@ def lib():
         for n in ("specroll_propose_workspace_bytes", "specroll_verify_workspace_bytes",
                   "specroll_tree_attn_workspace_bytes"):
             getattr(l, n).restype = C.c_size_t
-        for n in ("specroll_propose", "specroll_tree_draw", "specroll_tree_attn", "specroll_verify",
+        for n in ("specroll_propose", "specroll_propose_status", "specroll_tree_draw", "specroll_tree_attn",
+                  "specroll_verify",
                   "specroll_verify_static"):
             getattr(l, n).restype = C.c_int
         _lib = l
@@ -120,8 +122,10 @@ def propose_workspace_bytes(B, N, K, k, d, V, temperature=1.0, ln_eps=1e-5, rms_
 
 def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0, ln_eps=1e-5,
             rms_eps=1e-6, clip_c=0.0, ln_gamma=None, ln_beta=None, workspace=None,
-            out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
-    """specroll_propose.  Device tensors in, dict of device tensors out."""
+            out: Optional[Dict[str, torch.Tensor]] = None, flags: int = 0,
+            check_status: bool = False) -> Dict[str, torch.Tensor]:
+    """specroll_propose.  Device tensors in, dict of device tensors out.
+    ``check_status`` also calls specroll_propose_status (synchronises the stream)."""
     parent = _host_i32(parent, "parent")
     B, d = h.shape
     K, V, N = A.shape[0], W.shape[0], parent.shape[0]
@@ -133,7 +137,7 @@ def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0,
         raise SpecrollError("propose: m must be [B,K,d]")
     if alpha is not None and tuple(alpha.shape) != (B, K):
         raise SpecrollError("propose: alpha must be [B,K]")
-    desc = ProposeDesc(B, N, K, k, d, V, temperature, ln_eps, rms_eps, clip_c, 0)
+    desc = ProposeDesc(B, N, K, k, d, V, temperature, ln_eps, rms_eps, clip_c, flags)
     dev = h.device
     if out is None:
         out = {"cand_id": torch.empty((B, K, k), dtype=torch.int32, device=dev),
@@ -154,6 +158,8 @@ def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0,
         _dev(out["slot_q"], torch.float32, "slot_q"), C.c_void_p(workspace.data_ptr()),
         C.c_size_t(workspace.numel()), _stream())
     _check(rc, "specroll_propose")
+    if check_status:
+        _check(lib().specroll_propose_status(C.c_void_p(workspace.data_ptr()), _stream()), "specroll_propose_status")
     return out
 
 

@@ -324,26 +324,35 @@ tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__rest
 
 struct ProposePlan {
     int KX, M, n_mblocks, n_tiles, n_groups, tiles_per_group;
-    size_t off_xhat, off_z, off_zt, off_pval, off_pid, total;
+    bool use_tc;  // tcgen05 projection kernel (k <= 8); otherwise the mma.sync one
+    size_t off_status, off_xhat, off_z, off_zt, off_pval, off_pid, total;
 };
+
+// lm_head_tc.cu
+int launch_lm_head_tc(const void *Zt, const void *W, int M, int V, int d, int k, int n_mblocks, int n_groups,
+                      int tiles_per_group, float *pval, int32_t *pid, int32_t *status, cudaStream_t st);
 
 static int make_plan(const specroll_propose_desc *d, bool affine, ProposePlan *p) {
     if (!d || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->K < 1 || d->K > SPECROLL_MAX_HEADS ||
         d->k < 1 || d->k > SPECROLL_MAX_TOPK || d->d < 64 || (d->d % 64) || d->V < 8 || (d->V % 8) ||
         d->k > d->V || !(d->temperature > 0.f) || !(d->ln_eps >= 0.f) || !(d->rms_eps >= 0.f) ||
-        d->flags != 0)
+        (d->flags & ~SPECROLL_PROPOSE_LEGACY_MMA) != 0 || d->d > 12288)
         return SPECROLL_EINVAL;
     p->KX = affine ? d->K : 1;
     p->M = d->B * d->K;
-    p->n_mblocks = (p->M + LmTile::BM - 1) / LmTile::BM;
-    p->n_tiles = (d->V + LmTile::BN - 1) / LmTile::BN;
-    int want = p->n_mblocks > 0 ? (2 * 148) / p->n_mblocks : 1;
+    p->use_tc = d->k <= 8 && !(d->flags & SPECROLL_PROPOSE_LEGACY_MMA);
+    const int bn = p->use_tc ? 256 : LmTile::BN;
+    p->n_mblocks = (p->M + LmTile::BM - 1) / LmTile::BM;  // both kernels use 128-row blocks
+    p->n_tiles = (d->V + bn - 1) / bn;
+    int want = p->n_mblocks > 0 ? ((p->use_tc ? 1 : 2) * 148) / p->n_mblocks : 1;
     if (want < 1) want = 1;
     if (want > p->n_tiles) want = p->n_tiles;
     p->tiles_per_group = (p->n_tiles + want - 1) / want;
     p->n_groups = (p->n_tiles + p->tiles_per_group - 1) / p->tiles_per_group;
     size_t o = 0;
     const size_t B = d->B, K = d->K, dd = d->d, k = d->k;
+    p->off_status = o;
+    o += 256;
     p->off_xhat = o;
     o += align_up((size_t)p->KX * B * dd * 2, 256);
     p->off_z = o;
@@ -382,6 +391,15 @@ extern "C" size_t specroll_propose_workspace_bytes(const specroll_propose_desc *
     ProposePlan p;
     if (make_plan(d, true, &p) != SPECROLL_OK) return 0;  // sized for the affine case (the larger one)
     return p.total;
+}
+
+extern "C" int specroll_propose_status(const void *workspace, void *cuda_stream) {
+    if (!workspace) return SPECROLL_EINVAL;
+    int32_t word = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    SR_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st));
+    SR_CUDA_TRY(cudaStreamSynchronize(st));
+    return word == 0 ? SPECROLL_OK : (int)word;
 }
 
 extern "C" int specroll_tree_draw(int32_t B, int32_t N, int32_t K, int32_t k, float temperature,
@@ -427,6 +445,8 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
     int32_t *pid = reinterpret_cast<int32_t *>(ws + p.off_pid);
     const __nv_bfloat16 *hb = static_cast<const __nv_bfloat16 *>(h);
     const int B = d->B, K = d->K, dd = d->d, k = d->k, V = d->V;
+    int32_t *status = reinterpret_cast<int32_t *>(ws + p.off_status);
+    SR_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
 
     layernorm_kernel<<<B, LN_THREADS, dd * sizeof(float), st>>>(
         hb, static_cast<const __nv_bfloat16 *>(ln_gamma), static_cast<const __nv_bfloat16 *>(ln_beta), xhat, B,
@@ -450,7 +470,11 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
         const int grid = p.n_mblocks * p.n_groups;
         const int smem = LmTile::SMEM_BYTES;  // >= 128 * 129 * 4 staging tile
         static_assert(LmTile::SMEM_BYTES >= LmTile::BM * LM_CSTRIDE * 4, "staging tile must fit");
-        if (k <= 8) {
+        if (p.use_tc) {
+            int rc = launch_lm_head_tc(zt, W, p.M, V, dd, k, p.n_mblocks, p.n_groups, p.tiles_per_group, pval, pid,
+                                       status, st);
+            if (rc) return rc;
+        } else if (k <= 8) {
             int rc = set_smem(lm_head_topk_kernel<8>, smem);
             if (rc) return rc;
             lm_head_topk_kernel<8><<<grid, LmTile::THREADS, smem, st>>>(

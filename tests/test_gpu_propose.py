@@ -22,7 +22,8 @@ def gpu_propose(w, x, **kw):
     g = S.propose(dev_bf16(x["h"]), dev(x["anchor"]), dev_bf16(x["A"]), dev_bf16(x["bias"]), dev_bf16(x["W"]),
                   dev(x["m"]) if x.get("m") is not None else None,
                   dev(x["alpha"]) if x.get("alpha") is not None else None,
-                  x["parent"], dev(x["u_draw"]), k=w.k, temperature=w.temperature, clip_c=w.clip_c, **kw)
+                  x["parent"], dev(x["u_draw"]), k=w.k, temperature=w.temperature, clip_c=w.clip_c,
+                  check_status=True, **kw)
     torch.cuda.synchronize()
     return {k: host(v) for k, v in g.items()}
 
@@ -81,6 +82,16 @@ def test_ragged_shapes(B, K, k, d, V, N):
     same, _, _ = check_candidates(w, x, g, logit_atol=LOGIT_ATOL)
     check_tree(w, x, g, same)
     assert same.mean() > 0.9
+
+
+def test_legacy_projection_kernel_agrees():
+    # the mma.sync projection (flag) and the tcgen05 one must both match the oracle
+    w = I.scaled(I.WORKLOADS["qwen1.5b"], B=40, K=4, k=8, d=512, V=5000, N=16)
+    x = I.propose_inputs(w, peaked=True)
+    for flags in (0, 1):
+        g = gpu_propose(w, x, flags=flags)
+        same, _, _ = check_candidates(w, x, g, logit_atol=LOGIT_ATOL)
+        assert same.mean() > 0.9
 
 
 def test_reflex_abstain_clip_and_affine_layernorm():
