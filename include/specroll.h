@@ -100,11 +100,11 @@ int specroll_propose(const specroll_propose_desc *desc, const void *h, const int
                      float *cand_logit, int32_t *tree_tok, uint8_t *tree_cand, float *slot_q,
                      void *workspace, size_t workspace_bytes, void *cuda_stream);
 
-/* Reads back the status word the last specroll_propose on this workspace left behind: SPECROLL_OK,
- * or SPECROLL_ETIMEOUT if a bounded wait inside a kernel ran out (results are then invalid).
- * Unlike the other calls this one synchronises `cuda_stream`.  (Housekeeping; the paper has no
- * counterpart.) */
-int specroll_propose_status(const void *workspace, void *cuda_stream);
+/* Reads back the status word that the last specroll_propose or specroll_tree_attn using this
+ * workspace left behind: SPECROLL_OK, or SPECROLL_ETIMEOUT if a bounded wait inside a kernel ran
+ * out (the call's results are then invalid).  Unlike the other calls this one synchronises
+ * `cuda_stream`.  (Housekeeping; the paper has no counterpart.) */
+int specroll_workspace_status(const void *workspace, void *cuda_stream);
 
 /* The last step of the proposal alone (App. B.1): draw the tree from given candidate lists.
  * Same arguments and outputs as the corresponding ones of specroll_propose; needs no workspace. */
@@ -129,9 +129,12 @@ int specroll_tree_draw(int32_t B, int32_t N, int32_t K, int32_t k, float tempera
  */
 typedef struct {
     int32_t B, N, Hq, Hkv, D;
-    float scale;   /* softmax scale; the method uses 1/sqrt(D) */
-    int32_t flags; /* reserved, must be 0 */
+    float scale;   /* softmax scale (> 0); the method uses 1/sqrt(D) */
+    int32_t flags; /* 0, or SPECROLL_ATTN_LEGACY_MMA */
 } specroll_attn_desc;
+
+/* Run the attention on the mma.sync kernel instead of the tcgen05 one (kept for comparison). */
+#define SPECROLL_ATTN_LEGACY_MMA 1
 
 size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *desc,
                                           const int32_t *kv_indptr_host);

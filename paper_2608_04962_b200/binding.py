@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libspecroll.so")
 _lib = None
 
 EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
-           "specroll_propose_workspace_bytes", "specroll_propose", "specroll_propose_status",
+           "specroll_propose_workspace_bytes", "specroll_propose", "specroll_workspace_status",
            "specroll_tree_draw",
            "specroll_tree_attn_workspace_bytes", "specroll_tree_attn",
            "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static")
@@ -63,7 +63,7 @@ def lib():
         for n in ("specroll_propose_workspace_bytes", "specroll_verify_workspace_bytes",
                   "specroll_tree_attn_workspace_bytes"):
             getattr(l, n).restype = C.c_size_t
-        for n in ("specroll_propose", "specroll_propose_status", "specroll_tree_draw", "specroll_tree_attn",
+        for n in ("specroll_propose", "specroll_workspace_status", "specroll_tree_draw", "specroll_tree_attn",
                   "specroll_verify",
                   "specroll_verify_static"):
             getattr(l, n).restype = C.c_int
@@ -125,7 +125,7 @@ def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0,
             out: Optional[Dict[str, torch.Tensor]] = None, flags: int = 0,
             check_status: bool = False) -> Dict[str, torch.Tensor]:
     """specroll_propose.  Device tensors in, dict of device tensors out.
-    ``check_status`` also calls specroll_propose_status (synchronises the stream)."""
+    ``check_status`` also calls specroll_workspace_status (synchronises the stream)."""
     parent = _host_i32(parent, "parent")
     B, d = h.shape
     K, V, N = A.shape[0], W.shape[0], parent.shape[0]
@@ -159,7 +159,7 @@ def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0,
         C.c_size_t(workspace.numel()), _stream())
     _check(rc, "specroll_propose")
     if check_status:
-        _check(lib().specroll_propose_status(C.c_void_p(workspace.data_ptr()), _stream()), "specroll_propose_status")
+        _check(lib().specroll_workspace_status(C.c_void_p(workspace.data_ptr()), _stream()), "specroll_workspace_status")
     return out
 
 
@@ -193,8 +193,9 @@ def tree_attn_workspace_bytes(B, N, Hq, Hkv, D, kv_indptr_host, scale=None) -> i
 
 
 def tree_attn(Q, Kc, Vc, kv_indptr_dev, kv_indptr_host, Kt, Vt, parent, scale=None, want_lse=False,
-              workspace=None, out=None, lse=None):
-    """specroll_tree_attn.  Returns O (and lse when asked)."""
+              workspace=None, out=None, lse=None, flags: int = 0, check_status: bool = False):
+    """specroll_tree_attn.  Returns O (and lse when asked).
+    ``check_status`` also calls specroll_workspace_status (synchronises the stream)."""
     parent = _host_i32(parent, "parent")
     ip = _host_i32(kv_indptr_host, "kv_indptr_host")
     B, N, Hq, D = Q.shape
@@ -205,7 +206,7 @@ def tree_attn(Q, Kc, Vc, kv_indptr_dev, kv_indptr_host, Kt, Vt, parent, scale=No
         raise SpecrollError("tree_attn: cache shape does not match kv_indptr")
     if scale is None:
         scale = 1.0 / float(np.sqrt(D))
-    desc = AttnDesc(B, N, Hq, Hkv, D, scale, 0)
+    desc = AttnDesc(B, N, Hq, Hkv, D, scale, flags)
     dev = Q.device
     if out is None:
         out = torch.empty((B, N, Hq, D), dtype=torch.bfloat16, device=dev)
@@ -222,6 +223,9 @@ def tree_attn(Q, Kc, Vc, kv_indptr_dev, kv_indptr_host, Kt, Vt, parent, scale=No
         _dev(out, bf, "O"), _dev(lse, torch.float32, "lse"), C.c_void_p(workspace.data_ptr()),
         C.c_size_t(workspace.numel()), _stream())
     _check(rc, "specroll_tree_attn")
+    if check_status:
+        _check(lib().specroll_workspace_status(C.c_void_p(workspace.data_ptr()), _stream()),
+               "specroll_workspace_status")
     return (out, lse) if want_lse else out
 
 

@@ -393,7 +393,7 @@ extern "C" size_t specroll_propose_workspace_bytes(const specroll_propose_desc *
     return p.total;
 }
 
-extern "C" int specroll_propose_status(const void *workspace, void *cuda_stream) {
+extern "C" int specroll_workspace_status(const void *workspace, void *cuda_stream) {
     if (!workspace) return SPECROLL_EINVAL;
     int32_t word = 0;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

@@ -16,6 +16,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "tree_attn.cuh"
 
 namespace specroll {
 
@@ -24,20 +25,8 @@ constexpr int AT_STAGES = 3;
 constexpr int AT_MAX_WARPS = 8; // 128 query rows per CTA
 constexpr float LOG2E = 1.4426950408889634f;
 
-struct AttnArgs {
-    const __nv_bfloat16 *Q, *Kc, *Vc, *Kt, *Vt;
-    const int32_t *kv_indptr;
-    const int32_t *item_start;  // [B+1] exclusive prefix of the per-sequence chunk counts
-    __nv_bfloat16 *O;
-    float *lse;
-    float *part_o;   // [items, Hkv, rows_pad, D]
-    float *part_ml;  // [items, Hkv, rows_pad, 2]  (max in log2 units, sum)
-    int32_t B, N, Hq, Hkv, G, rows, rows_pad, n_rb, rows_per_block, chunk_tiles;
-    float scale_log2;  // scale * log2(e)
-};
-
 // item_start[b] = sum_{b' < b} max(1, ceil(tiles(b') / chunk_tiles))
-__global__ void attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles,
+__global__ void attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles, int tile_tokens,
                                  int32_t *__restrict__ item_start) {
     // single thread: B is at most a few thousand and this runs concurrently with nothing
     if (threadIdx.x == 0 && blockIdx.x == 0) {
@@ -45,7 +34,7 @@ __global__ void attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, i
         for (int b = 0; b < B; ++b) {
             item_start[b] = acc;
             const int L = kv_indptr[b + 1] - kv_indptr[b];
-            const int tiles = (L + AT_BN - 1) / AT_BN;
+            const int tiles = (L + tile_tokens - 1) / tile_tokens;
             int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
             acc += ns < 1 ? 1 : ns;
         }
@@ -339,15 +328,20 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(AttnArgs a) {
 // ------------------------------------------------------------------------------ host side
 
 struct AttnPlan {
-    int rows, n_rb, rows_per_block, rows_pad, chunk_tiles, items;
-    size_t off_items, off_po, off_pml, total;
+    int rows, n_rb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens;
+    bool use_tc;
+    size_t off_status, off_items, off_po, off_pml, total;
 };
 
 static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
     if (!d || !indptr_host || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->Hq < 1 || d->Hkv < 1 ||
-        (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || d->flags != 0)
+        (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || (d->flags & ~SPECROLL_ATTN_LEGACY_MMA) != 0 ||
+        !(d->scale > 0.f))
         return SPECROLL_EINVAL;
     const int G = d->Hq / d->Hkv;
+    p->use_tc = !(d->flags & SPECROLL_ATTN_LEGACY_MMA);
+    p->tile_tokens = p->use_tc ? 128 : AT_BN;
+    const int TT = p->tile_tokens;
     p->rows = d->N * G;
     p->n_rb = (p->rows + AT_MAX_WARPS * 16 - 1) / (AT_MAX_WARPS * 16);
     p->rows_per_block = ((p->rows + p->n_rb - 1) / p->n_rb + 15) / 16 * 16;
@@ -357,26 +351,28 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     for (int b = 0; b < d->B; ++b) {
         const int L = indptr_host[b + 1] - indptr_host[b];
         if (L < 0) return SPECROLL_EINVAL;
-        const int t = (L + AT_BN - 1) / AT_BN;
+        const int t = (L + TT - 1) / TT;
         tiles_total += t;
         if (t > max_tiles) max_tiles = t;
     }
-    // chunk length: about four CTAs' worth of work per SM over the whole launch, at least 8 tiles
-    // (512 tokens) so that the fp32 partials stay a small fraction of the KV bytes
+    // chunk length: about four CTAs' worth of work per SM over the whole launch, at least 512
+    // tokens so that the fp32 partials stay a small fraction of the KV bytes
     long long ctas_per_tile = (long long)d->Hkv * p->n_rb;
     long long ct = (tiles_total * ctas_per_tile + 148 * 4 - 1) / (148 * 4);
-    if (ct < 8) ct = 8;
+    if (ct < 512 / TT) ct = 512 / TT;
     if (ct > max_tiles) ct = max_tiles > 0 ? max_tiles : 1;
     p->chunk_tiles = (int)ct;
     int items = 0;
     for (int b = 0; b < d->B; ++b) {
         const int L = indptr_host[b + 1] - indptr_host[b];
-        const int t = (L + AT_BN - 1) / AT_BN;
+        const int t = (L + TT - 1) / TT;
         const int ns = (t + p->chunk_tiles - 1) / p->chunk_tiles;
         items += ns < 1 ? 1 : ns;
     }
     p->items = items;
     size_t o = 0;
+    p->off_status = o;
+    o += 256;
     p->off_items = o;
     o += align_up((size_t)(d->B + 1) * 4, 256);
     p->off_po = o;
@@ -453,10 +449,22 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
     a.n_rb = p.n_rb;
     a.rows_per_block = p.rows_per_block;
     a.chunk_tiles = p.chunk_tiles;
+    a.tile_tokens = p.tile_tokens;
     a.scale_log2 = d->scale * LOG2E;
-    attn_prep_kernel<<<1, 32, 0, st>>>(kv_indptr_dev, d->B, p.chunk_tiles, reinterpret_cast<int32_t *>(ws + p.off_items));
+    int32_t *status = reinterpret_cast<int32_t *>(ws + p.off_status);
+    SR_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    attn_prep_kernel<<<1, 32, 0, st>>>(kv_indptr_dev, d->B, p.chunk_tiles, p.tile_tokens,
+                                       reinterpret_cast<int32_t *>(ws + p.off_items));
     SR_LAUNCH_CHECK();
     const size_t n_out = (size_t)d->B * d->N * d->Hq;
+    if (p.use_tc) {
+        int rc = launch_attn_tc(a, mask, d->D, p.items, T_kv, status, st);
+        if (rc != SPECROLL_OK) return rc;
+        if (d->D == 128) attn_combine_kernel<128><<<(unsigned)((n_out + 3) / 4), 128, 0, st>>>(a);
+        else attn_combine_kernel<64><<<(unsigned)((n_out + 3) / 4), 128, 0, st>>>(a);
+        SR_LAUNCH_CHECK();
+        return SPECROLL_OK;
+    }
     if (d->D == 128) return launch_attn<128>(a, mask, p, d->Hkv, n_out, st);
     return launch_attn<64>(a, mask, p, d->Hkv, n_out, st);
 }

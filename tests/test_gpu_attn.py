@@ -11,6 +11,14 @@ from tests.util import dev, dev_bf16, host
 pytestmark = pytest.mark.gpu
 
 O_ATOL = 1e-2          # max abs error of the attention output (bf16 inputs, fp32 accumulate)
+FLAGS = {"v": 0}       # 0: tcgen05 kernel, 1: legacy mma.sync kernel
+
+
+@pytest.fixture(params=[0, 1], ids=["tcgen05", "mma"], autouse=True)
+def _both_kernels(request):
+    FLAGS["v"] = request.param
+    yield
+    FLAGS["v"] = 0
 
 
 def run_both(w, x, lengths=None):
@@ -25,7 +33,8 @@ def run_both(w, x, lengths=None):
         x["Vc"] = I.f32_to_bf16_bits(g.standard_normal((int(ip[-1]), w.Hkv, w.D), dtype=np.float32))
     o = ref.tree_attn(x["Q"], x["Kc"], x["Vc"], x["kv_indptr"], x["Kt"], x["Vt"], x["parent"], want_lse=True)
     O, lse = S.tree_attn(dev_bf16(x["Q"]), dev_bf16(x["Kc"]), dev_bf16(x["Vc"]), dev(x["kv_indptr"]),
-                         x["kv_indptr"], dev_bf16(x["Kt"]), dev_bf16(x["Vt"]), x["parent"], want_lse=True)
+                         x["kv_indptr"], dev_bf16(x["Kt"]), dev_bf16(x["Vt"]), x["parent"], want_lse=True,
+                         flags=FLAGS["v"], check_status=True)
     torch.cuda.synchronize()
     return o, host(O.float()).astype(np.float64), host(lse).astype(np.float64)
 
