@@ -2,16 +2,19 @@
 //
 // Same decomposition as the legacy kernel: for one (sequence, KV head) the N*G query rows form the
 // M dimension; a CTA owns up to 128 of them and one chunk of the cache (split-KV), and streams
-// 128-token K/V tiles.  Warp roles (192 threads, one CTA per SM):
-//   warp 0    TMA producer: K and V tiles (3-D tensor maps over [token, kv head, D], 128-byte
-//             swizzle), three stages, separate barriers for K and V
-//   warp 1    allocates TMEM, issues  S = Q K^T  (M=128, N=128, A and B from shared memory) and
-//             O += P V  (M=128, N=D, A = P from TMEM, B = V tile read MN-major from shared memory)
-//   warps 2-5 softmax: thread = query row = TMEM lane, so row max / row sum need no shuffles;
-//             P goes back to TMEM as packed bf16; the running output stays in TMEM and is rescaled
-//             only when a row's maximum grows by more than 2^8 (rare), by the thread that owns the row
-// S is double-buffered so the next tile's Q K^T overlaps this tile's softmax.
-// TMEM columns: O [0,128)  S0 [128,256)  S1 [256,384)  P0 [384,448)  P1 [448,512).
+// 128-token K/V tiles.  Warp roles (320 threads, one CTA per SM):
+//   warp 0     TMA producer: K and V tiles (3-D tensor maps over [token, kv head, D], 128-byte
+//              swizzle), three stages, separate barriers for K and V
+//   warp 1     allocates TMEM, issues  S = Q K^T  (M=128, N=128, A and B from shared memory) and
+//              O += P V  (M=128, N=D, A = P from TMEM, B = V tile read MN-major from shared memory)
+//   warps 2-5  softmax group 0: even tiles      } thread = query row = TMEM lane, so row max and
+//   warps 6-9  softmax group 1: odd tiles       } row sum need no shuffles
+// The two softmax groups are independent: each keeps its own running (reference max, sum) per row
+// and its own output accumulator in TMEM, exactly like two KV splits, and they are merged at the
+// end of the CTA.  P overwrites the first half of its S buffer in place (packed bf16).  An output
+// accumulator is rescaled only when a row's maximum grows by more than 2^8 (rare), by the thread
+// that owns the row.
+// TMEM columns: O0 [0,128)  O1 [128,256)  S0/P0 [256,384)  S1/P1 [384,512).
 #include <math.h>
 
 #include "tc05.cuh"
@@ -21,10 +24,10 @@ namespace specroll {
 
 namespace attc {
 constexpr int BN = 128;
-constexpr int THREADS = 192;
+constexpr int THREADS = 320;
 constexpr int STAGES = 3;
 constexpr int TMEM_COLS = 512;
-constexpr uint32_t O_COL = 0, S_COL = 128, P_COL = 384;  // S_COL + 128*buf, P_COL + 64*buf
+constexpr uint32_t O_COL = 0, S_COL = 256;  // O_COL + 128*group, S_COL + 128*group
 constexpr float RESCALE_LOG2 = 8.0f;
 constexpr int BOX_BYTES = BN * 128;  // 128 rows x 128 bytes (64 bf16) = one TMA box
 
@@ -34,10 +37,16 @@ struct Cfg {
     static constexpr int Q_BYTES = NBOX * BOX_BYTES;
     static constexpr int KV_BYTES = NBOX * BOX_BYTES;  // one K tile or one V tile
     static constexpr int STAGE_BYTES = 2 * KV_BYTES;
-    static constexpr int USED = Q_BYTES + STAGES * STAGE_BYTES + 1024 + 256;
+    static constexpr int N_BARS = 3 * STAGES + 6;
+    static constexpr int EXTRA = 8 * N_BARS + 16 + 128 * 8;  // barriers, TMEM slot + abort flag, merge scratch
+    static constexpr int USED = Q_BYTES + STAGES * STAGE_BYTES + 1024 + EXTRA;
     // at least ~118 KB so that two CTAs can never share an SM (each allocates all of TMEM)
     static constexpr int SMEM = USED > 120832 ? USED : 120832;
 };
+
+__device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 }  // namespace attc
 
 template <int D>
@@ -57,12 +66,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     auto k_full = [&](int s) { return bar0 + 8u * s; };
     auto v_full = [&](int s) { return bar0 + 8u * (STAGES + s); };
     auto kv_empty = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };
-    auto s_full = [&](int b) { return bar0 + 8u * (3 * STAGES + b); };
-    auto p_ready = [&](int b) { return bar0 + 8u * (3 * STAGES + 2 + b); };
-    const uint32_t pv_done = bar0 + 8u * (3 * STAGES + 4);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(aligned + C::Q_BYTES + STAGES * C::STAGE_BYTES +
-                                                       8 * (3 * STAGES + 5));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    auto s_full = [&](int g) { return bar0 + 8u * (3 * STAGES + g); };
+    auto p_ready = [&](int g) { return bar0 + 8u * (3 * STAGES + 2 + g); };
+    auto pv_done = [&](int g) { return bar0 + 8u * (3 * STAGES + 4 + g); };
+    unsigned char *extra = aligned + C::Q_BYTES + STAGES * C::STAGE_BYTES + 8 * C::N_BARS;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(extra);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(extra + 4);
+    float2 *merge_ml = reinterpret_cast<float2 *>(extra + 16);  // group 1's (max, sum) per row
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -99,8 +109,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         for (int i = 0; i < 2; ++i) {
             mbar_init(s_full(i), 1);
             mbar_init(p_ready(i), 128);
+            mbar_init(pv_done(i), 1);
         }
-        mbar_init(pv_done, 1);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tmK);
@@ -175,6 +185,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
+        // tcgen05.mma operations of one thread execute in issue order, which is what lets S of
+        // tile j+2 overwrite the buffer whose P (tile j) the previous P V has read.
         if (lane == 0 && n_it > 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, BN, false, false);
             constexpr uint32_t idesc_pv = idesc_bf16(128, D, false, true);  // V is read MN-major
@@ -200,64 +212,79 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     tc_fence_after();
                     issue_s(j + 1);
                 }
-                if (!mbar_wait(p_ready(j & 1), (uint32_t)(j >> 1) & 1u, abort_flag)) break;
+                const int g = j & 1;
+                if (!mbar_wait(p_ready(g), (uint32_t)(j >> 1) & 1u, abort_flag)) break;
                 const int s = j % STAGES;
                 if (!mbar_wait(v_full(s), (uint32_t)(j / STAGES) & 1u, abort_flag)) break;
                 tc_fence_after();
                 const uint32_t vs = kv_s + s * C::STAGE_BYTES + C::KV_BYTES;
-                const uint32_t p_t = tmem_base + P_COL + 64u * (uint32_t)(j & 1);
+                const uint32_t p_t = tmem_base + S_COL + 128u * (uint32_t)g;
+                const uint32_t o_t = tmem_base + O_COL + 128u * (uint32_t)g;
 #pragma unroll
                 for (int kk = 0; kk < BN / 16; ++kk) {
                     // 16 tokens per step: 2048 bytes down the V tile, 8 packed columns along P
-                    umma_ts(tmem_base + O_COL, p_t + 8u * kk, smem_desc_sw128(vs + kk * 2048, 1024, BOX_BYTES), idesc_pv,
-                            (j > 0 || kk > 0) ? 1u : 0u);
+                    umma_ts(o_t, p_t + 8u * kk, smem_desc_sw128(vs + kk * 2048, 1024, BOX_BYTES), idesc_pv,
+                            (j > 1 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(kv_empty(s));
-                umma_commit(pv_done);
+                umma_commit(pv_done(g));
             }
         }
     } else {
-        // ------------------------------------------------------------------ softmax / output (warps 2..5)
-        const int lg = warp & 3;
+        // ------------------------------------------------------------------ softmax groups (warps 2..9)
+        const int grp = (warp - 2) >> 2;  // 0: even tiles, 1: odd tiles
+        const int lg = warp & 3;          // TMEM lane group of this warp
         const int row = lg * 32 + lane;
         const int gr = row0 + row;
         const bool row_ok = row < a.rows_per_block && gr < a.rows;
         const uint64_t anc = row_ok ? mask.anc[gr / G] : 0ull;
         const uint32_t t_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
+        const uint32_t s_t = t_lane + S_COL + 128u * (uint32_t)grp;
+        const uint32_t o_t = t_lane + O_COL + 128u * (uint32_t)grp;
         const float sc = a.scale_log2;
         float m_used = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int j = 0; j < n_it; ++j) {
-            const int buf = j & 1;
-            ok = mbar_wait(s_full(buf), (uint32_t)(j >> 1) & 1u, abort_flag);
+        int n_mine = 0;
+        for (int j = grp; j < n_it; j += 2, ++n_mine) {
+            const int i = j >> 1;  // this group's i-th tile
+            ok = mbar_wait(s_full(grp), (uint32_t)i & 1u, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             const bool tree = has_tree && (j == n_it - 1);
-            const int limit = tree ? 64 : (L - (t_lo + j) * BN);  // columns >= limit are not in this sequence
-            const uint32_t s_t = t_lane + S_COL + 128u * (uint32_t)buf;
-            // pass 1: row maximum over the admissible columns
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t r[32];
-                tmem_ld32(s_t + (uint32_t)c, r);
-                tmem_ld_wait();
-                if (tree) {
-                    const uint32_t bits = (c < 64) ? (uint32_t)(anc >> c) : 0u;
+            const int limit = tree ? 64 : (L - (t_lo + j) * BN);  // columns >= limit are outside the sequence
+            const bool full = !tree && limit >= BN;
+            uint32_t r[4][32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if ((bits >> i) & 1u) mx = fmaxf(mx, __uint_as_float(r[i]));
-                } else if (c + 32 <= limit) {
+            for (int c = 0; c < 4; ++c) tmem_ld32(s_t + 32u * c, r[c]);
+            tmem_ld_wait();
+            // admissible-column masks of the four 32-column groups
+            uint32_t bits[4];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
-                } else {
+            for (int c = 0; c < 4; ++c) {
+                if (full) bits[c] = 0xffffffffu;
+                else if (tree) bits[c] = (c < 2) ? (uint32_t)(anc >> (32 * c)) : 0u;
+                else bits[c] = (32 * c + 32 <= limit) ? 0xffffffffu : ((32 * c >= limit) ? 0u : ((1u << (limit - 32 * c)) - 1u));
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+            if (full) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (c + i < limit) mx = fmaxf(mx, __uint_as_float(r[i]));
+                for (int i2 = 0; i2 < 32; ++i2) {
+                    mx0 = fmaxf(mx0, __uint_as_float(r[0][i2]));
+                    mx1 = fmaxf(mx1, __uint_as_float(r[1][i2]));
+                    mx2 = fmaxf(mx2, __uint_as_float(r[2][i2]));
+                    mx3 = fmaxf(mx3, __uint_as_float(r[3][i2]));
+                }
+            } else {
+#pragma unroll
+                for (int i2 = 0; i2 < 32; ++i2) {
+                    if ((bits[0] >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(r[0][i2]));
+                    if ((bits[1] >> i2) & 1u) mx1 = fmaxf(mx1, __uint_as_float(r[1][i2]));
+                    if ((bits[2] >> i2) & 1u) mx2 = fmaxf(mx2, __uint_as_float(r[2][i2]));
+                    if ((bits[3] >> i2) & 1u) mx3 = fmaxf(mx3, __uint_as_float(r[3][i2]));
                 }
             }
-            const float mt = mx * sc;  // scale > 0; -inf stays -inf
+            const float mt = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc;  // scale > 0; -inf stays -inf
             float alpha = 1.f;
             const bool need = mt > m_used + RESCALE_LOG2;  // also true on the first admissible tile
             if (need) {
@@ -265,99 +292,107 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 m_used = mt;
                 l *= alpha;
             }
-            if (__any_sync(0xffffffffu, need) && j > 0) {
-                // rows of this warp change their reference maximum: rescale their running outputs in TMEM.
-                // The previous tile's P V must have landed first.
-                ok = mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, abort_flag);
+            if (__any_sync(0xffffffffu, need) && i > 0) {
+                // rows of this warp change their reference maximum: rescale their running outputs in
+                // TMEM.  This group's previous P V must have landed first.
+                ok = mbar_wait(pv_done(grp), (uint32_t)(i - 1) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll 1
                 for (int c = 0; c < D; c += 32) {
-                    uint32_t r[32];
-                    tmem_ld32(t_lane + O_COL + (uint32_t)c, r);
+                    uint32_t o[32];
+                    tmem_ld32(o_t + (uint32_t)c, o);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                    tmem_st32(t_lane + O_COL + (uint32_t)c, r);
+                    for (int i2 = 0; i2 < 32; ++i2) o[i2] = __float_as_uint(__uint_as_float(o[i2]) * alpha);
+                    tmem_st32(o_t + (uint32_t)c, o);
                 }
                 tmem_st_wait();
             }
             const float mref = (m_used == -INFINITY) ? 0.f : m_used;
-            // pass 2: p = 2^(s*scale - m), packed bf16 pairs into the P buffer
-            float lsum = 0.f;
-            const uint32_t p_t = t_lane + P_COL + 64u * (uint32_t)buf;
-#pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t r[32];
-                tmem_ld32(s_t + (uint32_t)c, r);
-                tmem_ld_wait();
-                uint32_t bits;
-                if (tree) bits = (c < 64) ? (uint32_t)(anc >> c) : 0u;
-                else bits = (c + 32 <= limit) ? 0xffffffffu : ((c >= limit) ? 0u : ((1u << (limit - c)) - 1u));
+            // p = 2^(s*scale - m), packed bf16 pairs written over the first 64 columns of the S buffer
+            float ls0 = 0.f, ls1 = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float p0 = ex2_approx(fmaf(__uint_as_float(r[i]), sc, -mref));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(r[i + 1]), sc, -mref));
-                    p0 = ((bits >> i) & 1u) ? p0 : 0.f;
-                    p1 = ((bits >> (i + 1)) & 1u) ? p1 : 0.f;
-                    lsum += p0 + p1;
-                    pk[i >> 1] = pack_bf16x2(p0, p1);
+                for (int i2 = 0; i2 < 32; i2 += 2) {
+                    float p0 = ex2_approx(fmaf(__uint_as_float(r[c][i2]), sc, -mref));
+                    float p1 = ex2_approx(fmaf(__uint_as_float(r[c][i2 + 1]), sc, -mref));
+                    if (!full) {
+                        p0 = ((bits[c] >> i2) & 1u) ? p0 : 0.f;
+                        p1 = ((bits[c] >> (i2 + 1)) & 1u) ? p1 : 0.f;
+                    }
+                    ls0 += p0;
+                    ls1 += p1;
+                    pk[i2 >> 1] = pack_bf16x2(p0, p1);
                 }
-                tmem_st16(p_t + (uint32_t)(c >> 1), pk);
+                tmem_st16(s_t + 16u * c, pk);
             }
             tmem_st_wait();
-            l += lsum;
+            l += ls0 + ls1;
             tc_fence_before();
-            mbar_arrive(p_ready(buf));
+            mbar_arrive(p_ready(grp));
         }
-        // ---- output
-        if (ok && n_it > 0) {
-            ok = mbar_wait(pv_done, (uint32_t)(n_it - 1) & 1u, abort_flag);
+        // ---- wait for this group's last P V, then merge the two groups and write the output
+        if (ok && n_mine > 0) {
+            ok = mbar_wait(pv_done(grp), (uint32_t)(n_mine - 1) & 1u, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if (ok) {
-            tc_fence_after();
+        if (grp == 1) merge_ml[row] = make_float2(m_used, (ok && n_mine > 0) ? l : 0.f);
+        tc_fence_before();
+        named_barrier_sync(1, 256);
+        tc_fence_after();
+        const bool all_ok = !*abort_flag;
+        if (grp == 0 && all_ok) {
+            const float2 other = merge_ml[row];
+            const float m1 = other.x, l1 = other.y;
+            const bool have0 = n_mine > 0 && l > 0.f, have1 = l1 > 0.f;
+            const float M = fmaxf(have0 ? m_used : -INFINITY, have1 ? m1 : -INFINITY);
+            const float w0 = have0 ? ex2_approx(m_used - M) : 0.f, w1 = have1 ? ex2_approx(m1 - M) : 0.f;
+            const float lt = w0 * l + w1 * l1;
             const int n = row_ok ? gr / G : 0, g = row_ok ? gr % G : 0;
             const bool direct = (n_splits == 1);
-            const float inv = (direct && l > 0.f) ? 1.0f / l : (direct ? 0.f : 1.0f);
+            const float inv = direct ? (lt > 0.f ? 1.0f / lt : 0.f) : 1.0f;
+            const float f0 = w0 * inv, f1 = w1 * inv;
             __nv_bfloat16 *dst_o = a.O + (((size_t)b * N + n) * a.Hq + hkv * G + g) * D;
             const size_t prow = ((size_t)item * a.Hkv + hkv) * a.rows_pad + (row_ok ? gr : 0);
             float *dst_p = a.part_o + prow * D;
+            const bool any0 = __any_sync(0xffffffffu, have0), any1 = __any_sync(0xffffffffu, have1);
 #pragma unroll 1
             for (int c = 0; c < D; c += 32) {
-                uint32_t r[32];
-                if (n_it > 0) {
-                    tmem_ld32(t_lane + O_COL + (uint32_t)c, r);
-                    tmem_ld_wait();
-                } else {
+                uint32_t o0[32], o1[32];
+                if (any0) tmem_ld32(t_lane + O_COL + (uint32_t)c, o0);
+                if (any1) tmem_ld32(t_lane + O_COL + 128u + (uint32_t)c, o1);
+                tmem_ld_wait();
+                float v[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = 0u;
-                }
+                for (int i2 = 0; i2 < 32; ++i2)
+                    v[i2] = (have0 ? __uint_as_float(o0[i2]) * f0 : 0.f) + (have1 ? __uint_as_float(o1[i2]) * f1 : 0.f);
                 if (!row_ok) continue;
                 if (direct) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 v;
-                        v.x = pack_bf16x2(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
-                        v.y = pack_bf16x2(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-                        v.z = pack_bf16x2(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
-                        v.w = pack_bf16x2(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(dst_o + c + i) = v;
+                    for (int i2 = 0; i2 < 32; i2 += 8) {
+                        uint4 u;
+                        u.x = pack_bf16x2(v[i2], v[i2 + 1]);
+                        u.y = pack_bf16x2(v[i2 + 2], v[i2 + 3]);
+                        u.z = pack_bf16x2(v[i2 + 4], v[i2 + 5]);
+                        u.w = pack_bf16x2(v[i2 + 6], v[i2 + 7]);
+                        *reinterpret_cast<uint4 *>(dst_o + c + i2) = u;
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        *reinterpret_cast<uint4 *>(dst_p + c + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+                    for (int i2 = 0; i2 < 32; i2 += 4)
+                        *reinterpret_cast<float4 *>(dst_p + c + i2) = make_float4(v[i2], v[i2 + 1], v[i2 + 2], v[i2 + 3]);
                 }
             }
             if (row_ok) {
                 if (direct) {
-                    if (a.lse) a.lse[((size_t)b * N + n) * a.Hq + hkv * G + g] = (m_used + log2f(l)) * 0.6931471805599453f;
+                    if (a.lse) a.lse[((size_t)b * N + n) * a.Hq + hkv * G + g] = (M + log2f(lt)) * 0.6931471805599453f;
                 } else {
-                    a.part_ml[prow * 2] = m_used;
-                    a.part_ml[prow * 2 + 1] = l;
+                    a.part_ml[prow * 2] = M;
+                    a.part_ml[prow * 2 + 1] = lt;
                 }
             }
         }
