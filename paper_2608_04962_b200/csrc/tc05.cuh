@@ -16,8 +16,9 @@ namespace specroll {
 int make_tmap_2d_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint64_t ld_elems,
                       uint32_t box_rows);
 
-// Host: 3-D bf16 tensor [n2, n1, n0] (n0 innermost and contiguous), box [box2, 1, 64], 128-byte swizzle.
-int make_tmap_3d_bf16(CUtensorMap *map, const void *base, uint64_t n0, uint64_t n1, uint64_t n2, uint32_t box2);
+// Host: 3-D bf16 tensor [n2, n1, n0] (n0 innermost and contiguous), box [box2, box1, 64], 128-byte swizzle.
+int make_tmap_3d_bf16(CUtensorMap *map, const void *base, uint64_t n0, uint64_t n1, uint64_t n2, uint32_t box1,
+                      uint32_t box2);
 
 #ifdef __CUDACC__
 

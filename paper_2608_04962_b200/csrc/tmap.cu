@@ -22,13 +22,14 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// 3-D bf16 tensor [n2, n1, n0] (n0 innermost, contiguous), box [box2, 1, 64], 128-byte swizzle.
-int make_tmap_3d_bf16(CUtensorMap *map, const void *base, uint64_t n0, uint64_t n1, uint64_t n2, uint32_t box2) {
+// 3-D bf16 tensor [n2, n1, n0] (n0 innermost, contiguous), box [box2, box1, 64], 128-byte swizzle.
+int make_tmap_3d_bf16(CUtensorMap *map, const void *base, uint64_t n0, uint64_t n1, uint64_t n2, uint32_t box1,
+                      uint32_t box2) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return note_cuda_error(cudaErrorNotSupported);
     cuuint64_t dims[3] = {n0, n1, n2};
     cuuint64_t strides[2] = {n0 * 2, n0 * n1 * 2};
-    cuuint32_t box[3] = {64, 1, box2};
+    cuuint32_t box[3] = {64, box1, box2};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

@@ -25,21 +25,113 @@ constexpr int AT_STAGES = 3;
 constexpr int AT_MAX_WARPS = 8; // 128 query rows per CTA
 constexpr float LOG2E = 1.4426950408889634f;
 
-// item_start[b] = sum_{b' < b} max(1, ceil(tiles(b') / chunk_tiles))
-__global__ void attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles, int tile_tokens,
-                                 int32_t *__restrict__ item_start) {
-    // single thread: B is at most a few thousand and this runs concurrently with nothing
-    if (threadIdx.x == 0 && blockIdx.x == 0) {
-        int acc = 0;
-        for (int b = 0; b < B; ++b) {
-            item_start[b] = acc;
-            const int L = kv_indptr[b + 1] - kv_indptr[b];
-            const int tiles = (L + tile_tokens - 1) / tile_tokens;
-            int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
-            acc += ns < 1 ? 1 : ns;
-        }
-        item_start[B] = acc;
+constexpr int PREP_THREADS = 1024;
+constexpr int PREP_MAX_B = 4096;  // sequences the prep kernel can order (4 per thread)
+
+// Exclusive scan of n <= 4 * PREP_THREADS ints held in shared memory, in place; returns the total.
+__device__ int block_exclusive_scan(int *data, int n, int *warp_tot) {
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    int v[4], s = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int idx = 4 * t + i;
+        v[i] = idx < n ? data[idx] : 0;
+        s += v[i];
     }
+    int incl = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += x;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = warp_tot[lane];
+        int wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int x = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += x;
+        }
+        warp_tot[lane] = wi - w;  // exclusive prefix of the warp totals
+        if (lane == 31) warp_tot[32] = wi;
+    }
+    __syncthreads();
+    int run = warp_tot[warp] + incl - s;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int idx = 4 * t + i;
+        if (idx < n) data[idx] = run;
+        run += v[i];
+    }
+    const int total = warp_tot[32];
+    __syncthreads();
+    return total;
+}
+
+// One block.  Per sequence: number of chunks ns = max(1, ceil(tiles / chunk_tiles)).
+//   item_start[b]   exclusive prefix of ns in sequence order            (both kernels)
+//   seq_at_rank[r], sorted_start[r]   work order: sequences by decreasing tiles-per-chunk, and the
+//                   exclusive prefix of ns in that order                  (tcgen05 kernel, B <= PREP_MAX_B)
+// Also clears the status word and the scheduling counters.
+__global__ void __launch_bounds__(PREP_THREADS)
+attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles, int tile_tokens,
+                 int32_t *__restrict__ item_start, int32_t *__restrict__ sorted_start,
+                 int32_t *__restrict__ seq_at_rank, int32_t *__restrict__ status, int32_t *__restrict__ counters,
+                 int n_counters) {
+    __shared__ unsigned short sh_ns[PREP_MAX_B];  // chunk counts fit 16 bits (checked on the host)
+    __shared__ int sh_cost[PREP_MAX_B];
+    __shared__ int sh_tmp[PREP_MAX_B];
+    __shared__ int warp_tot[33];
+    const int t = threadIdx.x;
+    if (t == 0) *status = 0;
+    for (int i = t; i < n_counters; i += PREP_THREADS) counters[i] = 0;
+    if (B > PREP_MAX_B) {
+        // too many sequences to order here: sequence-order prefix only (legacy kernel)
+        if (t == 0) {
+            int acc = 0;
+            for (int b = 0; b < B; ++b) {
+                item_start[b] = acc;
+                const int L = kv_indptr[b + 1] - kv_indptr[b];
+                const int tiles = (L + tile_tokens - 1) / tile_tokens;
+                const int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
+                acc += ns < 1 ? 1 : ns;
+            }
+            item_start[B] = acc;
+        }
+        return;
+    }
+    for (int b = t; b < B; b += PREP_THREADS) {
+        const int L = kv_indptr[b + 1] - kv_indptr[b];
+        const int tiles = (L + tile_tokens - 1) / tile_tokens;
+        int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
+        if (ns < 1) ns = 1;
+        sh_ns[b] = (unsigned short)ns;
+        sh_cost[b] = (tiles + ns - 1) / ns;  // tiles per chunk
+        sh_tmp[b] = ns;
+    }
+    __syncthreads();
+    const int total = block_exclusive_scan(sh_tmp, B, warp_tot);
+    for (int b = t; b < B; b += PREP_THREADS) item_start[b] = sh_tmp[b];
+    if (t == 0) item_start[B] = total;
+    if (!sorted_start) return;
+    __syncthreads();
+    // rank by counting: position of b in the order (cost descending, index ascending)
+    for (int b = t; b < B; b += PREP_THREADS) {
+        const int c = sh_cost[b];
+        int r = 0;
+        for (int o = 0; o < B; ++o) {
+            const int co = sh_cost[o];
+            r += (co > c) || (co == c && o < b);
+        }
+        seq_at_rank[r] = b;
+        sh_tmp[r] = (int)sh_ns[b];
+    }
+    __syncthreads();
+    const int total2 = block_exclusive_scan(sh_tmp, B, warp_tot);
+    for (int r = t; r < B; r += PREP_THREADS) sorted_start[r] = sh_tmp[r];
+    if (t == 0) sorted_start[B] = total2;
 }
 
 template <int D>
@@ -328,9 +420,9 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(AttnArgs a) {
 // ------------------------------------------------------------------------------ host side
 
 struct AttnPlan {
-    int rows, n_rb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens;
+    int rows, n_rb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens, nodes_per_block, n_counters;
     bool use_tc;
-    size_t off_status, off_items, off_po, off_pml, total;
+    size_t off_status, off_items, off_sorted, off_rank, off_counters, off_po, off_pml, total;
 };
 
 static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
@@ -339,12 +431,24 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
         !(d->scale > 0.f))
         return SPECROLL_EINVAL;
     const int G = d->Hq / d->Hkv;
-    p->use_tc = !(d->flags & SPECROLL_ATTN_LEGACY_MMA);
+    // the tcgen05 kernel needs whole nodes per 128-row block and at most PREP_MAX_B sequences
+    p->use_tc = !(d->flags & SPECROLL_ATTN_LEGACY_MMA) && G <= 128 && d->B <= PREP_MAX_B;
     p->tile_tokens = p->use_tc ? 128 : AT_BN;
     const int TT = p->tile_tokens;
     p->rows = d->N * G;
-    p->n_rb = (p->rows + AT_MAX_WARPS * 16 - 1) / (AT_MAX_WARPS * 16);
-    p->rows_per_block = ((p->rows + p->n_rb - 1) / p->n_rb + 15) / 16 * 16;
+    if (p->use_tc) {
+        // row blocks are whole nodes: (node, head-in-group) rows of a block are one TMA box
+        int npb = 128 / G;
+        const int nb = (d->N + npb - 1) / npb;
+        npb = (d->N + nb - 1) / nb;  // even out the blocks
+        p->nodes_per_block = npb;
+        p->n_rb = nb;
+        p->rows_per_block = npb * G;
+    } else {
+        p->nodes_per_block = 0;
+        p->n_rb = (p->rows + AT_MAX_WARPS * 16 - 1) / (AT_MAX_WARPS * 16);
+        p->rows_per_block = ((p->rows + p->n_rb - 1) / p->n_rb + 15) / 16 * 16;
+    }
     p->rows_pad = p->rows_per_block * p->n_rb;
     long long tiles_total = 0;
     int max_tiles = 0;
@@ -370,11 +474,19 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
         items += ns < 1 ? 1 : ns;
     }
     p->items = items;
+    if (max_tiles / p->chunk_tiles + 1 > 65535) return SPECROLL_EINVAL;
+    p->n_counters = 64 + d->B * d->Hkv * p->n_rb;  // [0]: work counter; [64 ...]: per (b, hkv, rb) arrivals
     size_t o = 0;
     p->off_status = o;
     o += 256;
     p->off_items = o;
     o += align_up((size_t)(d->B + 1) * 4, 256);
+    p->off_sorted = o;
+    o += align_up((size_t)(d->B + 1) * 4, 256);
+    p->off_rank = o;
+    o += align_up((size_t)(d->B + 1) * 4, 256);
+    p->off_counters = o;
+    o += align_up((size_t)p->n_counters * 4, 256);
     p->off_po = o;
     o += align_up((size_t)items * d->Hkv * p->rows_pad * d->D * 4, 256);
     p->off_pml = o;
@@ -452,19 +564,22 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
     a.tile_tokens = p.tile_tokens;
     a.scale_log2 = d->scale * LOG2E;
     int32_t *status = reinterpret_cast<int32_t *>(ws + p.off_status);
-    SR_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
-    attn_prep_kernel<<<1, 32, 0, st>>>(kv_indptr_dev, d->B, p.chunk_tiles, p.tile_tokens,
-                                       reinterpret_cast<int32_t *>(ws + p.off_items));
+    int32_t *counters = reinterpret_cast<int32_t *>(ws + p.off_counters);
+    int32_t *sorted_start = reinterpret_cast<int32_t *>(ws + p.off_sorted);
+    int32_t *seq_at_rank = reinterpret_cast<int32_t *>(ws + p.off_rank);
+    a.sorted_start = sorted_start;
+    a.seq_at_rank = seq_at_rank;
+    a.work_counter = counters;
+    a.split_counters = counters + 64;
+    a.total_work = p.items * d->Hkv * p.n_rb;
+    a.nodes_per_block = p.nodes_per_block;
+    attn_prep_kernel<<<1, PREP_THREADS, 0, st>>>(kv_indptr_dev, d->B, p.chunk_tiles, p.tile_tokens,
+                                                 reinterpret_cast<int32_t *>(ws + p.off_items),
+                                                 p.use_tc ? sorted_start : nullptr, seq_at_rank, status, counters,
+                                                 p.n_counters);
     SR_LAUNCH_CHECK();
     const size_t n_out = (size_t)d->B * d->N * d->Hq;
-    if (p.use_tc) {
-        int rc = launch_attn_tc(a, mask, d->D, p.items, T_kv, status, st);
-        if (rc != SPECROLL_OK) return rc;
-        if (d->D == 128) attn_combine_kernel<128><<<(unsigned)((n_out + 3) / 4), 128, 0, st>>>(a);
-        else attn_combine_kernel<64><<<(unsigned)((n_out + 3) / 4), 128, 0, st>>>(a);
-        SR_LAUNCH_CHECK();
-        return SPECROLL_OK;
-    }
+    if (p.use_tc) return launch_attn_tc(a, mask, d->D, T_kv, status, st);  // merges split sequences itself
     if (d->D == 128) return launch_attn<128>(a, mask, p, d->Hkv, n_out, st);
     return launch_attn<64>(a, mask, p, d->Hkv, n_out, st);
 }

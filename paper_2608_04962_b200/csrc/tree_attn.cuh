@@ -8,7 +8,7 @@ namespace specroll {
 struct AttnArgs {
     const __nv_bfloat16 *Q, *Kc, *Vc, *Kt, *Vt;
     const int32_t *kv_indptr;
-    const int32_t *item_start;  // [B+1] exclusive prefix of the per-sequence chunk counts
+    const int32_t *item_start;  // [B+1] exclusive prefix of the per-sequence chunk counts (sequence order)
     __nv_bfloat16 *O;
     float *lse;
     float *part_o;   // [items, Hkv, rows_pad, D]   un-normalised partial outputs of split sequences
@@ -16,10 +16,16 @@ struct AttnArgs {
     int32_t B, N, Hq, Hkv, G, rows, rows_pad, n_rb, rows_per_block, chunk_tiles;
     int32_t tile_tokens;  // KV tokens per tile: 64 (mma.sync kernel) or 128 (tcgen05 kernel)
     float scale_log2;     // scale * log2(e)
+    // ---- tcgen05 kernel only: work order and counters written by the prep kernel
+    const int32_t *sorted_start;  // [B+1] exclusive prefix of the chunk counts in work order
+    const int32_t *seq_at_rank;   // [B]   sequence at each position of the work order (longest chunks first)
+    int32_t *work_counter;        // next work unit to hand out
+    int32_t *split_counters;      // [B, Hkv, n_rb] chunks of a (sequence, kv head, row block) that have finished
+    int32_t total_work;           // items * Hkv * n_rb
+    int32_t nodes_per_block;      // rows_per_block = nodes_per_block * G
 };
 
 // tcgen05 kernel (tree_attn_tc.cu).  T_kv = total cached tokens.  Launches the main kernel only.
-int launch_attn_tc(const AttnArgs &a, const TopoMask &mask, int D, int items, long long T_kv, int32_t *status,
-                   cudaStream_t st);
+int launch_attn_tc(const AttnArgs &a, const TopoMask &mask, int D, long long T_kv, int32_t *status, cudaStream_t st);
 
 }  // namespace specroll
