@@ -433,7 +433,7 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     const int G = d->Hq / d->Hkv;
     // the tcgen05 kernel needs whole nodes per 128-row block and at most PREP_MAX_B sequences
     p->use_tc = !(d->flags & SPECROLL_ATTN_LEGACY_MMA) && G <= 128 && d->B <= PREP_MAX_B;
-    p->tile_tokens = p->use_tc ? 128 : AT_BN;
+    p->tile_tokens = AT_BN;  // both kernels stream 64-token tiles
     const int TT = p->tile_tokens;
     p->rows = d->N * G;
     if (p->use_tc) {

@@ -1,24 +1,26 @@
 // Tree-verification attention on the 5th-generation tensor cores (tcgen05 + TMEM), one layer.
 //
 // Decomposition: for one (sequence, KV head) the N*G query rows form the M dimension; a work unit
-// is up to 128 of them (whole nodes) times one chunk of the cache (split-KV), streamed as 128-token
+// is up to 128 of them (whole nodes) times one chunk of the cache (split-KV), streamed as 64-token
 // K/V tiles.  The kernel is persistent: one CTA per SM takes work units from a global counter, in an
 // order prepared on the device (longest chunks first), and its pipeline runs across unit boundaries.
 // Warp roles (320 threads):
 //   warp 0     scheduler + TMA producer: fetches the next unit, publishes its descriptor in a
 //              two-slot ring, loads the Q block (3-D box over [node, head, D]) and the K and V tiles
-//              (3-D boxes over [token, kv head, D], 128-byte swizzle, three stages)
-//   warp 1     allocates TMEM, issues  S = Q K^T  (M=128, N=128, operands from shared memory) and
-//              O += P V  (M=128, N=D, A = P from TMEM, B = V tile read MN-major from shared memory)
+//              (3-D boxes over [token, kv head, D], 128-byte swizzle, six stages)
+//   warp 1     allocates TMEM, issues  S = Q K^T  (M=128, N=64, operands from shared memory) and
+//              O += P V  (M=128, N=D, A = P from TMEM, B = V tile read MN-major from shared memory);
+//              S runs four tiles ahead of P V
 //   warps 2-5  softmax group 0: even tiles      } thread = query row = TMEM lane, so row max and
 //   warps 6-9  softmax group 1: odd tiles       } row sum need no shuffles
 // The two softmax groups are independent: each keeps its own running (reference max, sum) per row
 // and its own output accumulator in TMEM, exactly like two KV splits, and they are merged at the
-// end of the unit.  P overwrites the first half of its S buffer in place (packed bf16).  An output
+// end of the unit.  Each group has two S buffers, so its next S tile is ready when it finishes
+// the current one.  P overwrites the first half of its S buffer in place (packed bf16).  An output
 // accumulator is rescaled only when a row's maximum grows by more than 2^8 (rare), by the thread
 // that owns the row.  Chunks of a split sequence leave fp32 partials in the workspace; the CTA that
 // finishes a sequence's last chunk (atomic ticket, nobody waits) merges them.
-// TMEM columns: O0 [0,128)  O1 [128,256)  S0/P0 [256,384)  S1/P1 [384,512).
+// TMEM columns: O0 [0,128)  O1 [128,256)  S/P of group g, buffer h: [256 + 128 g + 64 h, +64).
 #include <math.h>
 
 #include "tc05.cuh"
@@ -27,14 +29,16 @@
 namespace specroll {
 
 namespace attc {
-constexpr int BN = 128;
+constexpr int BN = 64;        // KV tokens per tile
+constexpr int AHEAD = 4;      // S tiles in flight ahead of P V (two per softmax group)
 constexpr int THREADS = 320;
-constexpr int STAGES = 3;
+constexpr int STAGES = 6;
 constexpr int TMEM_COLS = 512;
-constexpr uint32_t O_COL = 0, S_COL = 256;  // O_COL + 128*group, S_COL + 128*group
+constexpr uint32_t O_COL = 0, S_COL = 256;  // O_COL + 128*group ; S_COL + 128*group + 64*buffer
 constexpr float RESCALE_LOG2 = 8.0f;
-constexpr int BOX_BYTES = BN * 128;  // 128 rows x 128 bytes (64 bf16)
-constexpr int N_BARS = 3 * STAGES + 6 + 2 + 4 + 3;
+constexpr int Q_BOX_BYTES = 128 * 128;  // 128 query rows x 128 bytes (64 bf16)
+constexpr int KV_BOX_BYTES = BN * 128;  // 64 tokens x 128 bytes
+constexpr int N_BARS = 3 * STAGES + 21;
 
 struct UnitDesc {
     int32_t valid, b, hkv, rb, n_splits, kv0, L, t_lo, n_it, has_tree, item, item0;
@@ -43,8 +47,8 @@ struct UnitDesc {
 template <int D>
 struct Cfg {
     static constexpr int NBOX = D / 64;
-    static constexpr int Q_BYTES = NBOX * BOX_BYTES;
-    static constexpr int KV_BYTES = NBOX * BOX_BYTES;  // one K tile or one V tile
+    static constexpr int Q_BYTES = NBOX * Q_BOX_BYTES;
+    static constexpr int KV_BYTES = NBOX * KV_BOX_BYTES;  // one K tile or one V tile
     static constexpr int STAGE_BYTES = 2 * KV_BYTES;
     static constexpr int BAR_BYTES = (8 * N_BARS + 15) / 16 * 16;
     static constexpr int EXTRA = BAR_BYTES + 16 + 128 * 8 + 2 * 64;  // barriers, slot/abort/ticket, merge, ring
@@ -83,14 +87,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     auto k_full = [&](int s) { return bar0 + 8u * s; };
     auto v_full = [&](int s) { return bar0 + 8u * (STAGES + s); };
     auto kv_empty = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };
-    auto s_full = [&](int g) { return bar0 + 8u * (3 * STAGES + g); };
-    auto p_ready = [&](int g) { return bar0 + 8u * (3 * STAGES + 2 + g); };
-    auto pv_done = [&](int g) { return bar0 + 8u * (3 * STAGES + 4 + g); };
-    const uint32_t q_full = bar0 + 8u * (3 * STAGES + 6), q_free = bar0 + 8u * (3 * STAGES + 7);
-    auto unit_full = [&](int s) { return bar0 + 8u * (3 * STAGES + 8 + s); };
-    auto unit_empty = [&](int s) { return bar0 + 8u * (3 * STAGES + 10 + s); };
-    const uint32_t sync_a = bar0 + 8u * (3 * STAGES + 12), sync_b = bar0 + 8u * (3 * STAGES + 13);
-    const uint32_t sync_g0 = bar0 + 8u * (3 * STAGES + 14);
+    constexpr int B1 = 3 * STAGES;
+    auto s_full = [&](int g, int h) { return bar0 + 8u * (B1 + 2 * g + h); };
+    // one P barrier per S buffer: a group may finish two tiles before the MMA thread looks, and a
+    // single barrier would then have flipped twice and hide the first completion
+    auto p_ready = [&](int g, int h) { return bar0 + 8u * (B1 + 4 + 2 * g + h); };
+    // likewise one "P V done" barrier per S buffer: two P V of a group can be pending at once, and on a
+    // single barrier the completion of the older one would pass for the completion of the newer one
+    auto pv_done = [&](int g, int h) { return bar0 + 8u * (B1 + 8 + 2 * g + h); };
+    const uint32_t q_full = bar0 + 8u * (B1 + 12), q_free = bar0 + 8u * (B1 + 13);
+    auto unit_full = [&](int s) { return bar0 + 8u * (B1 + 14 + s); };
+    auto unit_empty = [&](int s) { return bar0 + 8u * (B1 + 16 + s); };
+    const uint32_t sync_a = bar0 + 8u * (B1 + 18), sync_b = bar0 + 8u * (B1 + 19), sync_g0 = bar0 + 8u * (B1 + 20);
     unsigned char *extra = aligned + C::Q_BYTES + STAGES * C::STAGE_BYTES + C::BAR_BYTES;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(extra);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(extra + 4);
@@ -108,9 +116,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             mbar_init(kv_empty(s), 1);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(s_full(i), 1);
-            mbar_init(p_ready(i), 128);
-            mbar_init(pv_done(i), 1);
+            mbar_init(s_full(i, 0), 1);
+            mbar_init(s_full(i, 1), 1);
+            mbar_init(p_ready(i, 0), 128);
+            mbar_init(p_ready(i, 1), 128);
+            mbar_init(pv_done(i, 0), 1);
+            mbar_init(pv_done(i, 1), 1);
             mbar_init(unit_full(i), 1);
             mbar_init(unit_empty(i), 257);  // the MMA thread and the 256 softmax threads
         }
@@ -204,7 +215,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 mbar_arrive_expect_tx(q_full, (uint32_t)(C::NBOX * 128 * a.rows_per_block));
 #pragma unroll
                 for (int bx = 0; bx < C::NBOX; ++bx)
-                    tma_load_3d(q_s + bx * BOX_BYTES, &tmQ, bx * 64, hkv * G, b * N + rb * a.nodes_per_block, q_full);
+                    tma_load_3d(q_s + bx * Q_BOX_BYTES, &tmQ, bx * 64, hkv * G, b * N + rb * a.nodes_per_block, q_full);
                 q_inflight = true;
                 // ---- K/V tiles
                 for (int it = 0; it < n_it; ++it, ++gt) {
@@ -222,11 +233,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     mbar_arrive_expect_tx(k_full(s), C::KV_BYTES);
 #pragma unroll
                     for (int bx = 0; bx < C::NBOX; ++bx)
-                        tma_load_3d(ks + bx * BOX_BYTES, mk, bx * 64, hkv, tok, k_full(s));
+                        tma_load_3d(ks + bx * KV_BOX_BYTES, mk, bx * 64, hkv, tok, k_full(s));
                     mbar_arrive_expect_tx(v_full(s), C::KV_BYTES);
 #pragma unroll
                     for (int bx = 0; bx < C::NBOX; ++bx)
-                        tma_load_3d(vs + bx * BOX_BYTES, mv, bx * 64, hkv, tok, v_full(s));
+                        tma_load_3d(vs + bx * KV_BOX_BYTES, mv, bx * 64, hkv, tok, v_full(s));
                     issued[s] = (int)ph;
                 }
                 if (ok) q_inflight = false;  // the MMA thread has consumed q_full before its first S
@@ -252,8 +263,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        // tcgen05.mma operations of one thread execute in issue order, which is what lets S of
-        // tile j+2 overwrite the buffer whose P (tile j) the previous P V has read.
+        // tcgen05.mma operations of one thread execute in issue order, which is what lets an S tile
+        // overwrite the buffer whose P the previously issued P V has read.
         if (lane == 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, BN, false, false);
             constexpr uint32_t idesc_pv = idesc_bf16(128, D, false, true);  // V is read MN-major
@@ -268,38 +279,37 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (!valid) break;
                 if (!mbar_wait(q_full, u & 1u, abort_flag)) break;
                 tc_fence_after();
-                auto issue_s = [&](int j) {
-                    const uint32_t ks = kv_s + ((gt + (uint32_t)j) % STAGES) * C::STAGE_BYTES;
-                    const uint32_t d_t = tmem_base + S_COL + 128u * (uint32_t)(j & 1);
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = (uint32_t)(kk >> 2) * BOX_BYTES + (uint32_t)(kk & 3) * 32u;
-                        umma_ss(d_t, smem_desc_sw128(q_s + off, 1024, 0), smem_desc_sw128(ks + off, 1024, 0), idesc_s,
-                                kk > 0 ? 1u : 0u);
-                    }
-                    umma_commit(s_full(j & 1));
-                    if (j == n_it - 1) umma_commit(q_free);  // last S of the unit: Q may be replaced after it
-                };
                 if (n_it == 0) {
                     umma_commit(q_free);
                     continue;
                 }
-                ok = mbar_wait(k_full((int)(gt % STAGES)), (gt / STAGES) & 1u, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                issue_s(0);
-                for (int j = 0; j < n_it; ++j) {
-                    if (j + 1 < n_it) {
-                        const uint32_t g1 = gt + (uint32_t)j + 1u;
-                        if (!mbar_wait(k_full((int)(g1 % STAGES)), (g1 / STAGES) & 1u, abort_flag)) {
-                            ok = false;
-                            break;
-                        }
-                        tc_fence_after();
-                        issue_s(j + 1);
-                    }
+                // S of tile j -> buffer (group j&1, parity of that group's tile count); waits for the K tile
+                auto issue_s = [&](int j) -> bool {
+                    const uint32_t gj = gt + (uint32_t)j;
+                    const int s = (int)(gj % STAGES);
+                    if (!mbar_wait(k_full(s), (gj / STAGES) & 1u, abort_flag)) return false;
+                    tc_fence_after();
                     const int g = j & 1;
-                    if (!mbar_wait(p_ready(g), (cnt[g] + (uint32_t)(j >> 1)) & 1u, abort_flag)) {
+                    const uint32_t c = cnt[g] + (uint32_t)(j >> 1);
+                    const int h = (int)(c & 1u);
+                    const uint32_t ks = kv_s + s * C::STAGE_BYTES;
+                    const uint32_t d_t = tmem_base + S_COL + 128u * (uint32_t)g + 64u * (uint32_t)h;
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t qoff = (uint32_t)(kk >> 2) * Q_BOX_BYTES + (uint32_t)(kk & 3) * 32u;
+                        const uint32_t koff = (uint32_t)(kk >> 2) * KV_BOX_BYTES + (uint32_t)(kk & 3) * 32u;
+                        umma_ss(d_t, smem_desc_sw128(q_s + qoff, 1024, 0), smem_desc_sw128(ks + koff, 1024, 0), idesc_s,
+                                kk > 0 ? 1u : 0u);
+                    }
+                    umma_commit(s_full(g, h));
+                    if (j == n_it - 1) umma_commit(q_free);  // last S of the unit: Q may be replaced after it
+                    return true;
+                };
+                for (int j = 0; j < AHEAD && j < n_it && ok; ++j) ok = issue_s(j);
+                for (int j = 0; j < n_it && ok; ++j) {
+                    const int g = j & 1;
+                    const uint32_t c = cnt[g] + (uint32_t)(j >> 1);
+                    if (!mbar_wait(p_ready(g, (int)(c & 1u)), (c >> 1) & 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
@@ -311,16 +321,17 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                     tc_fence_after();
                     const uint32_t vs = kv_s + s * C::STAGE_BYTES + C::KV_BYTES;
-                    const uint32_t p_t = tmem_base + S_COL + 128u * (uint32_t)g;
+                    const uint32_t p_t = tmem_base + S_COL + 128u * (uint32_t)g + 64u * (c & 1u);
                     const uint32_t o_t = tmem_base + O_COL + 128u * (uint32_t)g;
 #pragma unroll
                     for (int kk = 0; kk < BN / 16; ++kk) {
                         // 16 tokens per step: 2048 bytes down the V tile, 8 packed columns along P
-                        umma_ts(o_t, p_t + 8u * kk, smem_desc_sw128(vs + kk * 2048, 1024, BOX_BYTES), idesc_pv,
+                        umma_ts(o_t, p_t + 8u * kk, smem_desc_sw128(vs + kk * 2048, 1024, KV_BOX_BYTES), idesc_pv,
                                 (j > 1 || kk > 0) ? 1u : 0u);
                     }
                     umma_commit(kv_empty(s));
-                    umma_commit(pv_done(g));
+                    umma_commit(pv_done(g, (int)(c & 1u)));
+                    if (j + AHEAD < n_it) ok = issue_s(j + AHEAD);  // reuses the buffer this P V has just read
                 }
                 gt += (uint32_t)n_it;
                 cnt[0] += (uint32_t)((n_it + 1) >> 1);
@@ -333,7 +344,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const int lg = warp & 3;          // TMEM lane group of this warp
         const int row = lg * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
-        const uint32_t s_t = t_lane + S_COL + 128u * (uint32_t)grp;
         const uint32_t o_t = t_lane + O_COL + 128u * (uint32_t)grp;
         const float sc = a.scale_log2;
         uint32_t cnt = 0;  // tiles this group has processed so far (all units)
@@ -357,40 +367,41 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             int n_mine = 0;
             for (int j = grp; j < n_it; j += 2, ++n_mine) {
                 const uint32_t c_idx = cnt + (uint32_t)n_mine;
-                ok = mbar_wait(s_full(grp), c_idx & 1u, abort_flag);
+                const int h = (int)(c_idx & 1u);
+                ok = mbar_wait(s_full(grp, h), (c_idx >> 1) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
+                const uint32_t s_t = t_lane + S_COL + 128u * (uint32_t)grp + 64u * (uint32_t)h;
                 const bool tree = has_tree && (j == n_it - 1);
-                const int limit = tree ? 64 : (L - (t_lo + j) * BN);  // columns >= limit are outside the sequence
+                const int limit = tree ? BN : (L - (t_lo + j) * BN);  // columns >= limit are outside the sequence
                 const bool full = !tree && limit >= BN;
-                uint32_t bits[4];  // admissible columns of the four 32-column groups
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (full) bits[c] = 0xffffffffu;
-                    else if (tree) bits[c] = (c < 2) ? (uint32_t)(anc >> (32 * c)) : 0u;
-                    else bits[c] = (32 * c + 32 <= limit) ? 0xffffffffu : ((32 * c >= limit) ? 0u : ((1u << (limit - 32 * c)) - 1u));
+                uint32_t r0[32], r1[32];
+                tmem_ld32(s_t, r0);
+                tmem_ld32(s_t + 32u, r1);
+                tmem_ld_wait();
+                uint32_t bits0, bits1;  // admissible columns 0..31 and 32..63
+                if (full) {
+                    bits0 = bits1 = 0xffffffffu;
+                } else if (tree) {
+                    bits0 = (uint32_t)anc;
+                    bits1 = (uint32_t)(anc >> 32);
+                } else {
+                    bits0 = limit >= 32 ? 0xffffffffu : ((1u << limit) - 1u);
+                    bits1 = limit >= 64 ? 0xffffffffu : (limit <= 32 ? 0u : ((1u << (limit - 32)) - 1u));
                 }
-                // pass 1: row maximum, 64 columns at a time (keeps the live registers well under the limit)
                 float mx0 = -INFINITY, mx1 = -INFINITY;
+                if (full) {
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t r0[32], r1[32];
-                    tmem_ld32(s_t + 64u * h, r0);
-                    tmem_ld32(s_t + 64u * h + 32u, r1);
-                    tmem_ld_wait();
-                    if (full) {
+                    for (int i2 = 0; i2 < 32; ++i2) {
+                        mx0 = fmaxf(mx0, __uint_as_float(r0[i2]));
+                        mx1 = fmaxf(mx1, __uint_as_float(r1[i2]));
+                    }
+                } else {
 #pragma unroll
-                        for (int i2 = 0; i2 < 32; ++i2) {
-                            mx0 = fmaxf(mx0, __uint_as_float(r0[i2]));
-                            mx1 = fmaxf(mx1, __uint_as_float(r1[i2]));
-                        }
-                    } else {
-#pragma unroll
-                        for (int i2 = 0; i2 < 32; ++i2) {
-                            if ((bits[2 * h] >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(r0[i2]));
-                            if ((bits[2 * h + 1] >> i2) & 1u) mx1 = fmaxf(mx1, __uint_as_float(r1[i2]));
-                        }
+                    for (int i2 = 0; i2 < 32; ++i2) {
+                        if ((bits0 >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(r0[i2]));
+                        if ((bits1 >> i2) & 1u) mx1 = fmaxf(mx1, __uint_as_float(r1[i2]));
                     }
                 }
                 const float mt = fmaxf(mx0, mx1) * sc;  // scale > 0; -inf stays -inf
@@ -404,7 +415,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (__any_sync(0xffffffffu, need) && n_mine > 0) {
                     // rows of this warp change their reference maximum: rescale their running outputs
                     // in TMEM.  This group's previous P V must have landed first.
-                    ok = mbar_wait(pv_done(grp), (c_idx - 1u) & 1u, abort_flag);
+                    ok = mbar_wait(pv_done(grp, (int)((c_idx - 1u) & 1u)), ((c_idx - 1u) >> 1) & 1u, abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
@@ -420,36 +431,38 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     tmem_st_wait();
                 }
                 const float mref = (m_used == -INFINITY) ? 0.f : m_used;
-                // p = 2^(s*scale - m), packed bf16 pairs written over the first 64 columns of the S buffer
-                // (second read of S, 32 columns at a time; P chunk c lands on columns the reads have passed)
+                // p = 2^(s*scale - m), packed bf16 pairs written over the first 32 columns of the S buffer
                 float ls0 = 0.f, ls1 = 0.f;
+                uint32_t pk0[16], pk1[16];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32], pk[16];
-                    tmem_ld32(s_t + 32u * c, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i2 = 0; i2 < 32; i2 += 2) {
-                        float p0 = ex2_approx(fmaf(__uint_as_float(r[i2]), sc, -mref));
-                        float p1 = ex2_approx(fmaf(__uint_as_float(r[i2 + 1]), sc, -mref));
-                        if (!full) {
-                            p0 = ((bits[c] >> i2) & 1u) ? p0 : 0.f;
-                            p1 = ((bits[c] >> (i2 + 1)) & 1u) ? p1 : 0.f;
-                        }
-                        ls0 += p0;
-                        ls1 += p1;
-                        pk[i2 >> 1] = pack_bf16x2(p0, p1);
+                for (int i2 = 0; i2 < 32; i2 += 2) {
+                    float p0 = ex2_approx(fmaf(__uint_as_float(r0[i2]), sc, -mref));
+                    float p1 = ex2_approx(fmaf(__uint_as_float(r0[i2 + 1]), sc, -mref));
+                    float p2 = ex2_approx(fmaf(__uint_as_float(r1[i2]), sc, -mref));
+                    float p3 = ex2_approx(fmaf(__uint_as_float(r1[i2 + 1]), sc, -mref));
+                    if (!full) {
+                        p0 = ((bits0 >> i2) & 1u) ? p0 : 0.f;
+                        p1 = ((bits0 >> (i2 + 1)) & 1u) ? p1 : 0.f;
+                        p2 = ((bits1 >> i2) & 1u) ? p2 : 0.f;
+                        p3 = ((bits1 >> (i2 + 1)) & 1u) ? p3 : 0.f;
                     }
-                    tmem_st16(s_t + 16u * c, pk);
+                    ls0 += p0 + p1;
+                    ls1 += p2 + p3;
+                    pk0[i2 >> 1] = pack_bf16x2(p0, p1);
+                    pk1[i2 >> 1] = pack_bf16x2(p2, p3);
                 }
+                tmem_st16(s_t, pk0);
+                tmem_st16(s_t + 16u, pk1);
                 tmem_st_wait();
                 l += ls0 + ls1;
                 tc_fence_before();
-                mbar_arrive(p_ready(grp));
+                mbar_arrive(p_ready(grp, h));
             }
             // ---- wait for this group's last P V of the unit
             if (ok && n_mine > 0) {
-                ok = mbar_wait(pv_done(grp), (cnt + (uint32_t)n_mine - 1u) & 1u, abort_flag);
+                // (operations complete in issue order, so the last P V covers the one before it)
+                const uint32_t c_last = cnt + (uint32_t)n_mine - 1u;
+                ok = mbar_wait(pv_done(grp, (int)(c_last & 1u)), (c_last >> 1) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
             }
             cnt += (uint32_t)n_mine;
