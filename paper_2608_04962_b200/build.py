@@ -34,7 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     objs = []
     procs = []
     os.makedirs(os.path.join(HERE, "build"), exist_ok=True)
-    flags = list(FLAGS)
+    flags = list(FLAGS) + os.environ.get("SPECROLL_NVCC_FLAGS", "").split()
     if verbose:
         flags = flags + ["-Xptxas", "-v"]
     for src in sources():

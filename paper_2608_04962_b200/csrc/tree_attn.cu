@@ -78,8 +78,8 @@ __device__ int block_exclusive_scan(int *data, int n, int *warp_tot) {
 __global__ void __launch_bounds__(PREP_THREADS)
 attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles, int tile_tokens,
                  int32_t *__restrict__ item_start, int32_t *__restrict__ sorted_start,
-                 int32_t *__restrict__ seq_at_rank, int32_t *__restrict__ status, int32_t *__restrict__ counters,
-                 int n_counters) {
+                 int32_t *__restrict__ seq_at_rank, int32_t *__restrict__ unit_tab, int32_t *__restrict__ status,
+                 int32_t *__restrict__ counters, int n_counters) {
     __shared__ unsigned short sh_ns[PREP_MAX_B];  // chunk counts fit 16 bits (checked on the host)
     __shared__ int sh_cost[PREP_MAX_B];
     __shared__ int sh_tmp[PREP_MAX_B];
@@ -132,6 +132,27 @@ attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles, 
     const int total2 = block_exclusive_scan(sh_tmp, B, warp_tot);
     for (int r = t; r < B; r += PREP_THREADS) sorted_start[r] = sh_tmp[r];
     if (t == 0) sorted_start[B] = total2;
+    // per-chunk table in work order, so that the scheduler decodes a work unit with one 32-byte load
+    if (unit_tab) {
+        __syncthreads();
+        for (int b = t; b < B; b += PREP_THREADS) {
+            // recompute this sequence's rank (same rule as above) to find where its chunks go
+            const int c = sh_cost[b];
+            int r = 0;
+            for (int o = 0; o < B; ++o) {
+                const int co = sh_cost[o];
+                r += (co > c) || (co == c && o < b);
+            }
+            const int ns = (int)sh_ns[b];
+            const int kv0 = kv_indptr[b], L = kv_indptr[b + 1] - kv0;
+            const int first = item_start[b];  // written by this block; visible after the barriers above
+            int4 *dst = reinterpret_cast<int4 *>(unit_tab) + 2 * (size_t)sh_tmp[r];
+            for (int s = 0; s < ns; ++s) {
+                dst[2 * s] = make_int4(b, s, ns, first);
+                dst[2 * s + 1] = make_int4(kv0, L, 0, 0);
+            }
+        }
+    }
 }
 
 template <int D>
@@ -422,7 +443,7 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(AttnArgs a) {
 struct AttnPlan {
     int rows, n_rb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens, nodes_per_block, n_counters;
     bool use_tc;
-    size_t off_status, off_items, off_sorted, off_rank, off_counters, off_po, off_pml, total;
+    size_t off_status, off_items, off_sorted, off_rank, off_tab, off_counters, off_po, off_pml, total;
 };
 
 static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
@@ -433,7 +454,7 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     const int G = d->Hq / d->Hkv;
     // the tcgen05 kernel needs whole nodes per 128-row block and at most PREP_MAX_B sequences
     p->use_tc = !(d->flags & SPECROLL_ATTN_LEGACY_MMA) && G <= 128 && d->B <= PREP_MAX_B;
-    p->tile_tokens = AT_BN;  // both kernels stream 64-token tiles
+    p->tile_tokens = p->use_tc ? 128 : AT_BN;  // KV tokens per tile of the chosen kernel
     const int TT = p->tile_tokens;
     p->rows = d->N * G;
     if (p->use_tc) {
@@ -462,7 +483,8 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     // chunk length: about four CTAs' worth of work per SM over the whole launch, at least 512
     // tokens so that the fp32 partials stay a small fraction of the KV bytes
     long long ctas_per_tile = (long long)d->Hkv * p->n_rb;
-    long long ct = (tiles_total * ctas_per_tile + 148 * 4 - 1) / (148 * 4);
+    const int per_sm_div = p->use_tc ? 2 : 4;  // the persistent kernel balances dynamically: fewer, larger chunks
+    long long ct = (tiles_total * ctas_per_tile + 148 * per_sm_div - 1) / (148 * per_sm_div);
     if (ct < 512 / TT) ct = 512 / TT;
     if (ct > max_tiles) ct = max_tiles > 0 ? max_tiles : 1;
     p->chunk_tiles = (int)ct;
@@ -485,6 +507,8 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     o += align_up((size_t)(d->B + 1) * 4, 256);
     p->off_rank = o;
     o += align_up((size_t)(d->B + 1) * 4, 256);
+    p->off_tab = o;
+    o += align_up((size_t)items * 32, 256);
     p->off_counters = o;
     o += align_up((size_t)p->n_counters * 4, 256);
     p->off_po = o;
@@ -567,16 +591,18 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
     int32_t *counters = reinterpret_cast<int32_t *>(ws + p.off_counters);
     int32_t *sorted_start = reinterpret_cast<int32_t *>(ws + p.off_sorted);
     int32_t *seq_at_rank = reinterpret_cast<int32_t *>(ws + p.off_rank);
+    int32_t *unit_tab = reinterpret_cast<int32_t *>(ws + p.off_tab);
     a.sorted_start = sorted_start;
     a.seq_at_rank = seq_at_rank;
+    a.unit_tab = unit_tab;
     a.work_counter = counters;
     a.split_counters = counters + 64;
     a.total_work = p.items * d->Hkv * p.n_rb;
     a.nodes_per_block = p.nodes_per_block;
     attn_prep_kernel<<<1, PREP_THREADS, 0, st>>>(kv_indptr_dev, d->B, p.chunk_tiles, p.tile_tokens,
                                                  reinterpret_cast<int32_t *>(ws + p.off_items),
-                                                 p.use_tc ? sorted_start : nullptr, seq_at_rank, status, counters,
-                                                 p.n_counters);
+                                                 p.use_tc ? sorted_start : nullptr, seq_at_rank,
+                                                 p.use_tc ? unit_tab : nullptr, status, counters, p.n_counters);
     SR_LAUNCH_CHECK();
     const size_t n_out = (size_t)d->B * d->N * d->Hq;
     if (p.use_tc) return launch_attn_tc(a, mask, d->D, T_kv, status, st);  // merges split sequences itself

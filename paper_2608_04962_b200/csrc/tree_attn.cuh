@@ -19,6 +19,7 @@ struct AttnArgs {
     // ---- tcgen05 kernel only: work order and counters written by the prep kernel
     const int32_t *sorted_start;  // [B+1] exclusive prefix of the chunk counts in work order
     const int32_t *seq_at_rank;   // [B]   sequence at each position of the work order (longest chunks first)
+    const int32_t *unit_tab;      // [items][8] per chunk in work order: b, chunk, n_chunks, first item, kv0, L, 0, 0
     int32_t *work_counter;        // next work unit to hand out
     int32_t *split_counters;      // [B, Hkv, n_rb] chunks of a (sequence, kv head, row block) that have finished
     int32_t total_work;           // items * Hkv * n_rb

@@ -1,26 +1,27 @@
 // Tree-verification attention on the 5th-generation tensor cores (tcgen05 + TMEM), one layer.
 //
 // Decomposition: for one (sequence, KV head) the N*G query rows form the M dimension; a work unit
-// is up to 128 of them (whole nodes) times one chunk of the cache (split-KV), streamed as 64-token
+// is up to 128 of them (whole nodes) times one chunk of the cache (split-KV), streamed as 128-token
 // K/V tiles.  The kernel is persistent: one CTA per SM takes work units from a global counter, in an
 // order prepared on the device (longest chunks first), and its pipeline runs across unit boundaries.
 // Warp roles (320 threads):
 //   warp 0     scheduler + TMA producer: fetches the next unit, publishes its descriptor in a
 //              two-slot ring, loads the Q block (3-D box over [node, head, D]) and the K and V tiles
-//              (3-D boxes over [token, kv head, D], 128-byte swizzle, six stages)
-//   warp 1     allocates TMEM, issues  S = Q K^T  (M=128, N=64, operands from shared memory) and
-//              O += P V  (M=128, N=D, A = P from TMEM, B = V tile read MN-major from shared memory);
-//              S runs four tiles ahead of P V
-//   warps 2-5  softmax group 0: even tiles      } thread = query row = TMEM lane, so row max and
-//   warps 6-9  softmax group 1: odd tiles       } row sum need no shuffles
-// The two softmax groups are independent: each keeps its own running (reference max, sum) per row
-// and its own output accumulator in TMEM, exactly like two KV splits, and they are merged at the
-// end of the unit.  Each group has two S buffers, so its next S tile is ready when it finishes
-// the current one.  P overwrites the first half of its S buffer in place (packed bf16).  An output
-// accumulator is rescaled only when a row's maximum grows by more than 2^8 (rare), by the thread
-// that owns the row.  Chunks of a split sequence leave fp32 partials in the workspace; the CTA that
-// finishes a sequence's last chunk (atomic ticket, nobody waits) merges them.
-// TMEM columns: O0 [0,128)  O1 [128,256)  S/P of group g, buffer h: [256 + 128 g + 64 h, +64).
+//              (3-D boxes over [token, kv head, D], 128-byte swizzle).  K and V have separate rings
+//              (4 and 2 stages): K is needed early, because S runs ahead, and is released as soon as
+//              its S is computed; V is needed late and released after P V.
+//   warp 1     allocates TMEM, issues  S = Q K^T  (M=128, N=128, operands from shared memory), up to
+//              three tiles ahead, and  O += P V  (M=128, N=D, A = P from TMEM, B = V tile read
+//              MN-major from shared memory)
+//   warps 2-9  softmax: TWO threads per query row (warps w and w+4 own the same 32 TMEM lanes and
+//              take columns 0-63 / 64-127 of each S tile), so the per-tile latency between "S ready"
+//              and "P ready" is half of the one-thread-per-row form.  The pair exchanges its two
+//              partial row maxima through shared memory once per tile.
+// P overwrites the first half of its S buffer in place (packed bf16).  The output accumulator is
+// rescaled only when a row's maximum grows by more than 2^8 (rare).  Chunks of a split sequence
+// leave fp32 partials in the workspace; the CTA that finishes a sequence's last chunk (atomic
+// ticket, nobody waits) merges them.
+// TMEM columns: O [0,128)   S/P buffer i: [128 + 128 i, +128), i = tile mod 3.
 #include <math.h>
 
 #include "tc05.cuh"
@@ -28,17 +29,37 @@
 
 namespace specroll {
 
+// Optional pipeline trace (build with -DSPECROLL_TRACE): CTA 0 records (event, index, SM clock) per role.
+#ifdef SPECROLL_TRACE
+__device__ unsigned long long g_trace[4][8192];
+__device__ unsigned int g_trace_n[4];
+#define SR_TRACE(role, ev, idx)                                                                       \
+    do {                                                                                              \
+        if (blockIdx.x == 0) {                                                                        \
+            const unsigned n_ = g_trace_n[role]++;                                                    \
+            if (n_ < 4096) {                                                                          \
+                g_trace[role][2 * n_] = ((unsigned long long)(ev) << 32) | (unsigned)(idx);           \
+                g_trace[role][2 * n_ + 1] = (unsigned long long)clock64();                            \
+            }                                                                                         \
+        }                                                                                             \
+    } while (0)
+#else
+#define SR_TRACE(role, ev, idx)
+#endif
+
 namespace attc {
-constexpr int BN = 64;        // KV tokens per tile
-constexpr int AHEAD = 4;      // S tiles in flight ahead of P V (two per softmax group)
+constexpr int BN = 128;       // KV tokens per tile
 constexpr int THREADS = 320;
-constexpr int STAGES = 6;
+constexpr int KS = 4, VS = 2, SB = 3;  // K stages, V stages, S buffers
 constexpr int TMEM_COLS = 512;
-constexpr uint32_t O_COL = 0, S_COL = 256;  // O_COL + 128*group ; S_COL + 128*group + 64*buffer
+constexpr uint32_t O_COL = 0, S_COL = 128;
 constexpr float RESCALE_LOG2 = 8.0f;
-constexpr int Q_BOX_BYTES = 128 * 128;  // 128 query rows x 128 bytes (64 bf16)
-constexpr int KV_BOX_BYTES = BN * 128;  // 64 tokens x 128 bytes
-constexpr int N_BARS = 3 * STAGES + 21;
+constexpr int BOX_BYTES = BN * 128;  // 128 rows x 128 bytes (64 bf16)
+// barrier slots
+constexpr int B_KFULL = 0, B_KEMPTY = B_KFULL + KS, B_VFULL = B_KEMPTY + KS, B_VEMPTY = B_VFULL + VS,
+              B_SFULL = B_VEMPTY + VS, B_PREADY = B_SFULL + SB, B_PVDONE = B_PREADY + SB, B_QFULL = B_PVDONE + SB,
+              B_QFREE = B_QFULL + 1, B_UFULL = B_QFREE + 1, B_UEMPTY = B_UFULL + 2, B_PAIR = B_UEMPTY + 2,
+              B_ALL = B_PAIR + 4, N_BARS = B_ALL + 1;
 
 struct UnitDesc {
     int32_t valid, b, hkv, rb, n_splits, kv0, L, t_lo, n_it, has_tree, item, item0;
@@ -47,20 +68,22 @@ struct UnitDesc {
 template <int D>
 struct Cfg {
     static constexpr int NBOX = D / 64;
-    static constexpr int Q_BYTES = NBOX * Q_BOX_BYTES;
-    static constexpr int KV_BYTES = NBOX * KV_BOX_BYTES;  // one K tile or one V tile
-    static constexpr int STAGE_BYTES = 2 * KV_BYTES;
+    static constexpr int Q_BYTES = NBOX * BOX_BYTES;
+    static constexpr int KV_BYTES = NBOX * BOX_BYTES;  // one K tile or one V tile
     static constexpr int BAR_BYTES = (8 * N_BARS + 15) / 16 * 16;
-    static constexpr int EXTRA = BAR_BYTES + 16 + 128 * 8 + 2 * 64;  // barriers, slot/abort/ticket, merge, ring
-    static constexpr int USED = Q_BYTES + STAGES * STAGE_BYTES + 1024 + EXTRA;
+    static constexpr int EXTRA = BAR_BYTES + 16 + 4 * 128 * 4 + 2 * 64;  // barriers, slot/abort/ticket, pair exchange, ring
+    // The operand tiles need 1024-byte alignment.  The dynamic shared window starts 1024-aligned on this
+    // architecture (checked at run time), so only a small slack is budgeted.
+    static constexpr int SLACK = 256;
+    static constexpr int USED = Q_BYTES + (KS + VS) * KV_BYTES + SLACK + EXTRA;
     // at least ~118 KB so that two CTAs can never share an SM (each allocates all of TMEM)
     static constexpr int SMEM = USED > 120832 ? USED : 120832;
     static_assert(sizeof(UnitDesc) <= 64, "ring slot");
     static_assert(USED <= 232448, "shared memory budget");
 };
 
-// Group rendezvous on an mbarrier (count = number of participants) with the same bounded wait as every
-// other wait here: a hardware named barrier would hang if a participant had left through the abort path.
+// Rendezvous on an mbarrier (count = number of participants) with the same bounded wait as every other
+// wait here: a hardware named barrier would hang if a participant had left through the abort path.
 __device__ __forceinline__ bool group_sync(uint32_t bar, uint32_t &uses, volatile int *abort_flag) {
     mbar_arrive(bar);
     const bool ok = mbar_wait(bar, uses & 1u, abort_flag);
@@ -77,59 +100,39 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     int32_t *__restrict__ status) {
     using namespace attc;
     using C = Cfg<D>;
+    constexpr int DH = D / 2;  // output columns per thread of a pair
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char *aligned = smem_raw + (base - raw);
     const uint32_t q_s = base;
-    const uint32_t kv_s = base + C::Q_BYTES;
-    const uint32_t bar0 = kv_s + STAGES * C::STAGE_BYTES;
-    auto k_full = [&](int s) { return bar0 + 8u * s; };
-    auto v_full = [&](int s) { return bar0 + 8u * (STAGES + s); };
-    auto kv_empty = [&](int s) { return bar0 + 8u * (2 * STAGES + s); };
-    constexpr int B1 = 3 * STAGES;
-    auto s_full = [&](int g, int h) { return bar0 + 8u * (B1 + 2 * g + h); };
-    // one P barrier per S buffer: a group may finish two tiles before the MMA thread looks, and a
-    // single barrier would then have flipped twice and hide the first completion
-    auto p_ready = [&](int g, int h) { return bar0 + 8u * (B1 + 4 + 2 * g + h); };
-    // likewise one "P V done" barrier per S buffer: two P V of a group can be pending at once, and on a
-    // single barrier the completion of the older one would pass for the completion of the newer one
-    auto pv_done = [&](int g, int h) { return bar0 + 8u * (B1 + 8 + 2 * g + h); };
-    const uint32_t q_full = bar0 + 8u * (B1 + 12), q_free = bar0 + 8u * (B1 + 13);
-    auto unit_full = [&](int s) { return bar0 + 8u * (B1 + 14 + s); };
-    auto unit_empty = [&](int s) { return bar0 + 8u * (B1 + 16 + s); };
-    const uint32_t sync_a = bar0 + 8u * (B1 + 18), sync_b = bar0 + 8u * (B1 + 19), sync_g0 = bar0 + 8u * (B1 + 20);
-    unsigned char *extra = aligned + C::Q_BYTES + STAGES * C::STAGE_BYTES + C::BAR_BYTES;
+    const uint32_t k_s = base + C::Q_BYTES;
+    const uint32_t v_s = k_s + KS * C::KV_BYTES;
+    const uint32_t bar0 = v_s + VS * C::KV_BYTES;
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    unsigned char *extra = aligned + C::Q_BYTES + (KS + VS) * C::KV_BYTES + C::BAR_BYTES;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(extra);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(extra + 4);
     volatile int *ticket = reinterpret_cast<volatile int *>(extra + 8);
-    float2 *merge_ml = reinterpret_cast<float2 *>(extra + 16);  // group 1's (max, sum) per row
-    volatile UnitDesc *ring = reinterpret_cast<volatile UnitDesc *>(extra + 16 + 128 * 8);  // 2 slots of 64 bytes
+    volatile float *xch = reinterpret_cast<volatile float *>(extra + 16);  // [2 parities][2 halves][128 rows]
+    volatile UnitDesc *ring = reinterpret_cast<volatile UnitDesc *>(extra + 16 + 4 * 128 * 4);  // 2 slots of 64 bytes
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int N = a.N, G = a.G;
+    if (base - raw > (uint32_t)C::SLACK) {  // uniform: the whole CTA leaves before touching anything
+        if (threadIdx.x == 0) atomicExch(status, SPECROLL_ECUDA);
+        return;
+    }
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(k_full(s), 1);
-            mbar_init(v_full(s), 1);
-            mbar_init(kv_empty(s), 1);
+        for (int i = 0; i < N_BARS; ++i) {
+            uint32_t count = 1;
+            if (i >= B_PREADY && i < B_PREADY + SB) count = 256;
+            if (i >= B_UEMPTY && i < B_UEMPTY + 2) count = 257;  // the MMA thread and the 256 softmax threads
+            if (i >= B_PAIR && i < B_PAIR + 4) count = 64;
+            if (i == B_ALL) count = 256;
+            mbar_init(bar(i), count);
         }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(s_full(i, 0), 1);
-            mbar_init(s_full(i, 1), 1);
-            mbar_init(p_ready(i, 0), 128);
-            mbar_init(p_ready(i, 1), 128);
-            mbar_init(pv_done(i, 0), 1);
-            mbar_init(pv_done(i, 1), 1);
-            mbar_init(unit_full(i), 1);
-            mbar_init(unit_empty(i), 257);  // the MMA thread and the 256 softmax threads
-        }
-        mbar_init(q_full, 1);
-        mbar_init(q_free, 1);
-        mbar_init(sync_a, 256);
-        mbar_init(sync_b, 256);
-        mbar_init(sync_g0, 128);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tmQ);
@@ -154,14 +157,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------------ scheduler + TMA producer
         if (lane == 0) {
-            int issued[STAGES];
+            bool ok = true;
+            uint32_t kt = 0, vt = 0;   // K and V tiles loaded so far (all units)
+            // V loads trail K loads by two tiles, carried over unit boundaries: (map, kv head, token) of pending V tiles
+            const CUtensorMap *pv_map[2];
+            int pv_h[2], pv_tok[2];
+            int n_pend = 0;
+            auto load_v = [&](const CUtensorMap *mv, int hkv, int tok) -> bool {
+                const int s = (int)(vt % VS);
+                if (!mbar_wait(bar(B_VEMPTY + s), ((vt / VS) & 1u) ^ 1u, abort_flag)) return false;
+                const uint32_t dst = v_s + s * C::KV_BYTES;
+                mbar_arrive_expect_tx(bar(B_VFULL + s), C::KV_BYTES);
 #pragma unroll
-            for (int s = 0; s < STAGES; ++s) issued[s] = -1;
-            bool ok = true, q_inflight = false;
-            uint32_t gt = 0;  // K/V tiles loaded so far (all units)
+                for (int bx = 0; bx < C::NBOX; ++bx) tma_load_3d(dst + bx * BOX_BYTES, mv, bx * 64, hkv, tok, bar(B_VFULL + s));
+                ++vt;
+                return true;
+            };
             for (uint32_t u = 0; ok; ++u) {
                 const int slot = (int)(u & 1u);
-                if (!mbar_wait(unit_empty(slot), ((u >> 1) & 1u) ^ 1u, abort_flag)) {
+                if (!mbar_wait(bar(B_UEMPTY + slot), ((u >> 1) & 1u) ^ 1u, abort_flag)) {
                     ok = false;
                     break;
                 }
@@ -169,31 +183,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 volatile UnitDesc *d = ring + slot;
                 if (w >= a.total_work) {
                     d->valid = 0;
-                    mbar_arrive(unit_full(slot));
+                    mbar_arrive(bar(B_UFULL + slot));
                     break;
                 }
-                // ---- decode: w = (position in work order * Hkv + hkv) * n_rb + rb
+                // ---- decode: w = (chunk position in work order * Hkv + hkv) * n_rb + rb; one table row per chunk
                 int t = w;
                 const int rb = t % a.n_rb;
                 t /= a.n_rb;
                 const int hkv = t % a.Hkv;
                 const int si = t / a.Hkv;
-                int lo = 0, hi = a.B;  // largest rank r with sorted_start[r] <= si
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (a.sorted_start[mid] <= si) lo = mid; else hi = mid;
-                }
-                const int b = a.seq_at_rank[lo];
-                const int split = si - a.sorted_start[lo];
-                const int n_splits = a.sorted_start[lo + 1] - a.sorted_start[lo];
-                const int kv0 = a.kv_indptr[b];
-                const int L = a.kv_indptr[b + 1] - kv0;
+                const int4 e0 = __ldg(reinterpret_cast<const int4 *>(a.unit_tab) + 2 * (size_t)si);
+                const int4 e1 = __ldg(reinterpret_cast<const int4 *>(a.unit_tab) + 2 * (size_t)si + 1);
+                const int b = e0.x, split = e0.y, n_splits = e0.z, item0 = e0.w, kv0 = e1.x, L = e1.y;
                 const int tiles_b = (L + BN - 1) / BN;
                 const int tps = (tiles_b + n_splits - 1) / n_splits;
                 const int t_lo = min(tiles_b, split * tps), t_hi = min(tiles_b, t_lo + tps);
                 const int has_tree = (split == n_splits - 1) ? 1 : 0;
                 const int n_it = (t_hi - t_lo) + has_tree;
-                const int item0 = a.item_start[b];
                 d->valid = 1;
                 d->b = b;
                 d->hkv = hkv;
@@ -206,188 +212,193 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 d->has_tree = has_tree;
                 d->item = item0 + split;
                 d->item0 = item0;
-                mbar_arrive(unit_full(slot));  // release: the descriptor is visible to whoever acquires
+                mbar_arrive(bar(B_UFULL + slot));  // release: the descriptor is visible to whoever acquires
+                SR_TRACE(0, 0, u);
                 // ---- Q block of this unit, once every S of the previous unit has been computed
-                if (u > 0 && !mbar_wait(q_free, (u - 1u) & 1u, abort_flag)) {
+                if (u > 0 && !mbar_wait(bar(B_QFREE), (u - 1u) & 1u, abort_flag)) {
                     ok = false;
                     break;
                 }
-                mbar_arrive_expect_tx(q_full, (uint32_t)(C::NBOX * 128 * a.rows_per_block));
+                mbar_arrive_expect_tx(bar(B_QFULL), (uint32_t)(C::NBOX * 128 * a.rows_per_block));
 #pragma unroll
                 for (int bx = 0; bx < C::NBOX; ++bx)
-                    tma_load_3d(q_s + bx * Q_BOX_BYTES, &tmQ, bx * 64, hkv * G, b * N + rb * a.nodes_per_block, q_full);
-                q_inflight = true;
-                // ---- K/V tiles
-                for (int it = 0; it < n_it; ++it, ++gt) {
-                    const int s = (int)(gt % STAGES);
-                    const uint32_t ph = (gt / STAGES) & 1u;
-                    if (!mbar_wait(kv_empty(s), ph ^ 1u, abort_flag)) {
+                    tma_load_3d(q_s + bx * BOX_BYTES, &tmQ, bx * 64, hkv * G, b * N + rb * a.nodes_per_block, bar(B_QFULL));
+                // ---- K tiles, each followed by the V tile from two tiles back
+                for (int it = 0; it < n_it && ok; ++it) {
+                    const int s = (int)(kt % KS);
+                    if (!mbar_wait(bar(B_KEMPTY + s), ((kt / KS) & 1u) ^ 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
                     const bool tree = has_tree && (it == n_it - 1);
                     const int tok = tree ? b * N : kv0 + (t_lo + it) * BN;
                     const CUtensorMap *mk = tree ? &tmKt : &tmK;
-                    const CUtensorMap *mv = tree ? &tmVt : &tmV;
-                    const uint32_t ks = kv_s + s * C::STAGE_BYTES, vs = ks + C::KV_BYTES;
-                    mbar_arrive_expect_tx(k_full(s), C::KV_BYTES);
+                    const uint32_t dst = k_s + s * C::KV_BYTES;
+                    mbar_arrive_expect_tx(bar(B_KFULL + s), C::KV_BYTES);
 #pragma unroll
-                    for (int bx = 0; bx < C::NBOX; ++bx)
-                        tma_load_3d(ks + bx * KV_BOX_BYTES, mk, bx * 64, hkv, tok, k_full(s));
-                    mbar_arrive_expect_tx(v_full(s), C::KV_BYTES);
-#pragma unroll
-                    for (int bx = 0; bx < C::NBOX; ++bx)
-                        tma_load_3d(vs + bx * KV_BOX_BYTES, mv, bx * 64, hkv, tok, v_full(s));
-                    issued[s] = (int)ph;
-                }
-                if (ok) q_inflight = false;  // the MMA thread has consumed q_full before its first S
-            }
-            if (!ok) {
-                // aborting: give the copies already in flight time to land before the CTA goes away
-                const unsigned long long t0 = globaltimer_ns();
-                bool pending = true;
-                while (pending && globaltimer_ns() - t0 < 100000000ull) {
-                    pending = false;
-#pragma unroll
-                    for (int s = 0; s < STAGES; ++s)
-                        if (issued[s] >= 0 && !(mbar_try_wait(k_full(s), (uint32_t)issued[s]) &&
-                                                mbar_try_wait(v_full(s), (uint32_t)issued[s])))
-                            pending = true;
-                }
-                if (q_inflight) {
-                    const unsigned long long t1 = globaltimer_ns();
-                    while (!mbar_try_wait(q_full, 0u) && !mbar_try_wait(q_full, 1u) && globaltimer_ns() - t1 < 100000000ull) {
+                    for (int bx = 0; bx < C::NBOX; ++bx) tma_load_3d(dst + bx * BOX_BYTES, mk, bx * 64, hkv, tok, bar(B_KFULL + s));
+                    ++kt;
+                    SR_TRACE(0, 1, kt);
+                    if (n_pend == 2) {
+                        ok = load_v(pv_map[0], pv_h[0], pv_tok[0]);
+                        pv_map[0] = pv_map[1];
+                        pv_h[0] = pv_h[1];
+                        pv_tok[0] = pv_tok[1];
+                        n_pend = 1;
                     }
+                    pv_map[n_pend] = tree ? &tmVt : &tmV;
+                    pv_h[n_pend] = hkv;
+                    pv_tok[n_pend] = tok;
+                    ++n_pend;
+                }
+                // the unit's last V tiles go out now if their stages are already free; otherwise they wait
+                // behind the next unit's Q and first K tiles (never block here)
+                while (ok && n_pend > 0 && mbar_try_wait(bar(B_VEMPTY + (int)(vt % VS)), ((vt / VS) & 1u) ^ 1u)) {
+                    ok = load_v(pv_map[0], pv_h[0], pv_tok[0]);
+                    pv_map[0] = pv_map[1];
+                    pv_h[0] = pv_h[1];
+                    pv_tok[0] = pv_tok[1];
+                    --n_pend;
+                }
+            }
+            // flush the V tiles still pending (the last two tiles of the last unit)
+            for (int i = 0; i < n_pend && ok; ++i) ok = load_v(pv_map[i], pv_h[i], pv_tok[i]);
+            if (!ok) {
+                // aborting: give copies in flight time to land before the CTA goes away
+                const unsigned long long t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 20000000ull) {
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        // tcgen05.mma operations of one thread execute in issue order, which is what lets an S tile
-        // overwrite the buffer whose P the previously issued P V has read.
+        // tcgen05.mma operations of one thread execute in issue order, which is what lets S of tile t+3
+        // overwrite the buffer whose P (tile t) the previously issued P V has read.
         if (lane == 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, BN, false, false);
             constexpr uint32_t idesc_pv = idesc_bf16(128, D, false, true);  // V is read MN-major
-            uint32_t gt = 0;            // K/V tiles consumed so far (all units)
-            uint32_t cnt[2] = {0u, 0u};  // tiles handed to each softmax group so far
+            // Descriptors are assembled from precomputed halves: the high word is constant, the low word is
+            // the operand's shared-memory address / 16 (14 bits) plus, for V, LBO / 16 << 16.
+            constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO 1024, version, 128B swizzle
+            constexpr uint32_t V_LBO = ((uint32_t)BOX_BYTES >> 4) << 16;
+            constexpr uint32_t BOXU = (uint32_t)BOX_BYTES >> 4;
+            uint32_t q_lo[D / 16];
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) q_lo[kk] = (q_s >> 4) + (uint32_t)(kk >> 2) * BOXU + (uint32_t)(kk & 3) * 2u;
+            auto desc = [](uint32_t lo) -> uint64_t { return ((uint64_t)DESC_HI << 32) | (uint64_t)lo; };
+            uint32_t gt = 0;  // tiles issued so far (all units)
             bool ok = true;
             for (uint32_t u = 0; ok; ++u) {
                 const int slot = (int)(u & 1u);
-                if (!mbar_wait(unit_full(slot), (u >> 1) & 1u, abort_flag)) break;
+                if (!mbar_wait(bar(B_UFULL + slot), (u >> 1) & 1u, abort_flag)) break;
                 const int valid = ring[slot].valid, n_it = ring[slot].n_it;
-                mbar_arrive(unit_empty(slot));
+                mbar_arrive(bar(B_UEMPTY + slot));
                 if (!valid) break;
-                if (!mbar_wait(q_full, u & 1u, abort_flag)) break;
+                if (!mbar_wait(bar(B_QFULL), u & 1u, abort_flag)) break;
                 tc_fence_after();
                 if (n_it == 0) {
-                    umma_commit(q_free);
+                    umma_commit(bar(B_QFREE));
                     continue;
                 }
-                // S of tile j -> buffer (group j&1, parity of that group's tile count); waits for the K tile
                 auto issue_s = [&](int j) -> bool {
-                    const uint32_t gj = gt + (uint32_t)j;
-                    const int s = (int)(gj % STAGES);
-                    if (!mbar_wait(k_full(s), (gj / STAGES) & 1u, abort_flag)) return false;
+                    const uint32_t t = gt + (uint32_t)j;
+                    const int ks = (int)(t % KS);
+                    if (!mbar_wait(bar(B_KFULL + ks), (t / KS) & 1u, abort_flag)) return false;
                     tc_fence_after();
-                    const int g = j & 1;
-                    const uint32_t c = cnt[g] + (uint32_t)(j >> 1);
-                    const int h = (int)(c & 1u);
-                    const uint32_t ks = kv_s + s * C::STAGE_BYTES;
-                    const uint32_t d_t = tmem_base + S_COL + 128u * (uint32_t)g + 64u * (uint32_t)h;
+                    const uint32_t k_lo = (k_s + ks * C::KV_BYTES) >> 4;
+                    const uint32_t d_t = tmem_base + S_COL + 128u * (t % SB);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t qoff = (uint32_t)(kk >> 2) * Q_BOX_BYTES + (uint32_t)(kk & 3) * 32u;
-                        const uint32_t koff = (uint32_t)(kk >> 2) * KV_BOX_BYTES + (uint32_t)(kk & 3) * 32u;
-                        umma_ss(d_t, smem_desc_sw128(q_s + qoff, 1024, 0), smem_desc_sw128(ks + koff, 1024, 0), idesc_s,
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        umma_ss(d_t, desc(q_lo[kk]), desc(k_lo + (uint32_t)(kk >> 2) * BOXU + (uint32_t)(kk & 3) * 2u), idesc_s,
                                 kk > 0 ? 1u : 0u);
-                    }
-                    umma_commit(s_full(g, h));
-                    if (j == n_it - 1) umma_commit(q_free);  // last S of the unit: Q may be replaced after it
+                    umma_commit(bar(B_SFULL + (int)(t % SB)));
+                    umma_commit(bar(B_KEMPTY + ks));  // the K tile is free once this S has been computed
+                    SR_TRACE(1, 1, t);
+                    if (j == n_it - 1) umma_commit(bar(B_QFREE));  // last S of the unit: Q may be replaced after it
                     return true;
                 };
-                for (int j = 0; j < AHEAD && j < n_it && ok; ++j) ok = issue_s(j);
+                for (int j = 0; j < SB && j < n_it && ok; ++j) ok = issue_s(j);
                 for (int j = 0; j < n_it && ok; ++j) {
-                    const int g = j & 1;
-                    const uint32_t c = cnt[g] + (uint32_t)(j >> 1);
-                    if (!mbar_wait(p_ready(g, (int)(c & 1u)), (c >> 1) & 1u, abort_flag)) {
+                    const uint32_t t = gt + (uint32_t)j;
+                    const int sb = (int)(t % SB), vs = (int)(t % VS);
+                    if (!mbar_wait(bar(B_PREADY + sb), (t / SB) & 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
-                    const uint32_t gj = gt + (uint32_t)j;
-                    const int s = (int)(gj % STAGES);
-                    if (!mbar_wait(v_full(s), (gj / STAGES) & 1u, abort_flag)) {
+                    SR_TRACE(1, 2, t);
+                    if (!mbar_wait(bar(B_VFULL + vs), (t / VS) & 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t vs = kv_s + s * C::STAGE_BYTES + C::KV_BYTES;
-                    const uint32_t p_t = tmem_base + S_COL + 128u * (uint32_t)g + 64u * (c & 1u);
-                    const uint32_t o_t = tmem_base + O_COL + 128u * (uint32_t)g;
+                    const uint32_t v_lo = ((v_s + vs * C::KV_BYTES) >> 4) | V_LBO;
+                    const uint32_t p_t = tmem_base + S_COL + 128u * (uint32_t)sb;
+                    const uint32_t acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
                     for (int kk = 0; kk < BN / 16; ++kk) {
-                        // 16 tokens per step: 2048 bytes down the V tile, 8 packed columns along P
-                        umma_ts(o_t, p_t + 8u * kk, smem_desc_sw128(vs + kk * 2048, 1024, KV_BOX_BYTES), idesc_pv,
-                                (j > 1 || kk > 0) ? 1u : 0u);
+                        // 16 tokens per step: 2048 bytes (128 address units) down the V tile, 8 packed columns along P
+                        umma_ts(tmem_base + O_COL, p_t + 8u * kk, desc(v_lo + 128u * kk), idesc_pv, kk > 0 ? 1u : acc0);
                     }
-                    umma_commit(kv_empty(s));
-                    umma_commit(pv_done(g, (int)(c & 1u)));
-                    if (j + AHEAD < n_it) ok = issue_s(j + AHEAD);  // reuses the buffer this P V has just read
+                    umma_commit(bar(B_VEMPTY + vs));
+                    umma_commit(bar(B_PVDONE + sb));
+                    SR_TRACE(1, 3, t);
+                    if (j + SB < n_it) ok = issue_s(j + SB);  // reuses the buffer this P V has just read
                 }
                 gt += (uint32_t)n_it;
-                cnt[0] += (uint32_t)((n_it + 1) >> 1);
-                cnt[1] += (uint32_t)(n_it >> 1);
             }
         }
     } else {
-        // ------------------------------------------------------------------ softmax groups (warps 2..9)
-        const int grp = (warp - 2) >> 2;  // 0: even tiles, 1: odd tiles
-        const int lg = warp & 3;          // TMEM lane group of this warp
+        // ------------------------------------------------------------------ softmax (warps 2..9)
+        const int half = (warp - 2) >> 2;  // which 64 of a tile's 128 columns, and which D/2 of the output columns
+        const int lg = warp & 3;           // TMEM lane group of this warp
         const int row = lg * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
-        const uint32_t o_t = t_lane + O_COL + 128u * (uint32_t)grp;
+        const uint32_t o_t = t_lane + O_COL + (uint32_t)(half * DH);
         const float sc = a.scale_log2;
-        uint32_t cnt = 0;  // tiles this group has processed so far (all units)
-        uint32_t use_a = 0, use_b = 0, use_g0 = 0;
+        uint32_t gt = 0;  // tiles processed so far (all units)
+        uint32_t use_pair = 0, use_all = 0;
+        const uint32_t pair_bar = bar(B_PAIR + lg);
         bool ok = true;
         for (uint32_t u = 0; ok; ++u) {
             const int slot = (int)(u & 1u);
-            ok = mbar_wait(unit_full(slot), (u >> 1) & 1u, abort_flag);
+            ok = mbar_wait(bar(B_UFULL + slot), (u >> 1) & 1u, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const int valid = ring[slot].valid, b = ring[slot].b, hkv = ring[slot].hkv, rb = ring[slot].rb;
             const int n_splits = ring[slot].n_splits, L = ring[slot].L, t_lo = ring[slot].t_lo;
             const int n_it = ring[slot].n_it, has_tree = ring[slot].has_tree, item = ring[slot].item;
             const int item0 = ring[slot].item0;
-            mbar_arrive(unit_empty(slot));
+            mbar_arrive(bar(B_UEMPTY + slot));
             if (!valid) break;
             const int gr = rb * a.rows_per_block + row;
             const bool row_ok = row < a.rows_per_block && gr < a.rows;
             const uint64_t anc = row_ok ? mask.anc[gr / G] : 0ull;
-            float m_used = -INFINITY, l = 0.f;
-            int n_mine = 0;
-            for (int j = grp; j < n_it; j += 2, ++n_mine) {
-                const uint32_t c_idx = cnt + (uint32_t)n_mine;
-                const int h = (int)(c_idx & 1u);
-                ok = mbar_wait(s_full(grp, h), (c_idx >> 1) & 1u, abort_flag);
+            float m_used = -INFINITY, l = 0.f;  // l: this thread's share (its 64 columns of every tile)
+            for (int j = 0; j < n_it; ++j) {
+                const uint32_t t = gt + (uint32_t)j;
+                const int sb = (int)(t % SB);
+                ok = mbar_wait(bar(B_SFULL + sb), (t / SB) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t s_t = t_lane + S_COL + 128u * (uint32_t)grp + 64u * (uint32_t)h;
+                if (lg == 0 && lane == 0) SR_TRACE(2 + half, 1, t);
+                const uint32_t s_t = t_lane + S_COL + 128u * (uint32_t)sb;
                 const bool tree = has_tree && (j == n_it - 1);
-                const int limit = tree ? BN : (L - (t_lo + j) * BN);  // columns >= limit are outside the sequence
-                const bool full = !tree && limit >= BN;
+                // columns >= limit are outside the sequence; this thread's columns start at 64 * half
+                const int limit = (tree ? 64 : (L - (t_lo + j) * BN)) - 64 * half;
+                const bool full = !tree && limit >= 64;
                 uint32_t r0[32], r1[32];
-                tmem_ld32(s_t, r0);
-                tmem_ld32(s_t + 32u, r1);
+                tmem_ld32(s_t + 64u * half, r0);
+                tmem_ld32(s_t + 64u * half + 32u, r1);
                 tmem_ld_wait();
-                uint32_t bits0, bits1;  // admissible columns 0..31 and 32..63
+                uint32_t bits0, bits1;  // admissible columns among this thread's 64
                 if (full) {
                     bits0 = bits1 = 0xffffffffu;
                 } else if (tree) {
-                    bits0 = (uint32_t)anc;
-                    bits1 = (uint32_t)(anc >> 32);
+                    bits0 = half == 0 ? (uint32_t)anc : 0u;
+                    bits1 = half == 0 ? (uint32_t)(anc >> 32) : 0u;
                 } else {
-                    bits0 = limit >= 32 ? 0xffffffffu : ((1u << limit) - 1u);
+                    bits0 = limit >= 32 ? 0xffffffffu : (limit <= 0 ? 0u : ((1u << limit) - 1u));
                     bits1 = limit >= 64 ? 0xffffffffu : (limit <= 32 ? 0u : ((1u << (limit - 32)) - 1u));
                 }
                 float mx0 = -INFINITY, mx1 = -INFINITY;
@@ -404,7 +415,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         if ((bits1 >> i2) & 1u) mx1 = fmaxf(mx1, __uint_as_float(r1[i2]));
                     }
                 }
-                const float mt = fmaxf(mx0, mx1) * sc;  // scale > 0; -inf stays -inf
+                // exchange the partial maximum with the thread that has the row's other 64 columns.  After
+                // this rendezvous both threads have also finished reading S, so P may overwrite it.
+                // (two exchange slots, alternating, so that a fast thread's next write cannot overtake a slow read)
+                const float mine = fmaxf(mx0, mx1);
+                const int px = (int)(use_pair & 1u) * 256;
+                xch[px + half * 128 + row] = mine;
+                tc_fence_before();
+                ok = group_sync(pair_bar, use_pair, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const float mt = fmaxf(mine, xch[px + (half ^ 1) * 128 + row]) * sc;  // scale > 0; -inf stays -inf
                 float alpha = 1.f;
                 const bool need = mt > m_used + RESCALE_LOG2;  // also true on the first admissible tile
                 if (need) {
@@ -412,15 +434,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     m_used = mt;
                     l *= alpha;
                 }
-                if (__any_sync(0xffffffffu, need) && n_mine > 0) {
-                    // rows of this warp change their reference maximum: rescale their running outputs
-                    // in TMEM.  This group's previous P V must have landed first.
-                    ok = mbar_wait(pv_done(grp, (int)((c_idx - 1u) & 1u)), ((c_idx - 1u) >> 1) & 1u, abort_flag);
+                if (__any_sync(0xffffffffu, need) && j > 0) {
+                    // rows of this warp change their reference maximum: rescale this thread's half of their
+                    // running outputs in TMEM.  The previous tile's P V must have landed first.
+                    ok = mbar_wait(bar(B_PVDONE + (int)((t - 1u) % SB)), ((t - 1u) / SB) & 1u, abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll 1
-                    for (int c = 0; c < D; c += 32) {
+                    for (int c = 0; c < DH; c += 32) {
                         uint32_t o[32];
                         tmem_ld32(o_t + (uint32_t)c, o);
                         tmem_ld_wait();
@@ -431,7 +453,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     tmem_st_wait();
                 }
                 const float mref = (m_used == -INFINITY) ? 0.f : m_used;
-                // p = 2^(s*scale - m), packed bf16 pairs written over the first 32 columns of the S buffer
+                // p = 2^(s*scale - m), packed bf16 pairs: this thread's 64 columns become 32 packed columns
                 float ls0 = 0.f, ls1 = 0.f;
                 uint32_t pk0[16], pk1[16];
 #pragma unroll
@@ -451,83 +473,83 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     pk0[i2 >> 1] = pack_bf16x2(p0, p1);
                     pk1[i2 >> 1] = pack_bf16x2(p2, p3);
                 }
-                tmem_st16(s_t, pk0);
-                tmem_st16(s_t + 16u, pk1);
+                tmem_st16(s_t + 32u * half, pk0);
+                tmem_st16(s_t + 32u * half + 16u, pk1);
                 tmem_st_wait();
                 l += ls0 + ls1;
                 tc_fence_before();
-                mbar_arrive(p_ready(grp, h));
+                mbar_arrive(bar(B_PREADY + sb));
+                if (lg == 0 && lane == 0) SR_TRACE(2 + half, 2, t);
             }
-            // ---- wait for this group's last P V of the unit
-            if (ok && n_mine > 0) {
-                // (operations complete in issue order, so the last P V covers the one before it)
-                const uint32_t c_last = cnt + (uint32_t)n_mine - 1u;
-                ok = mbar_wait(pv_done(grp, (int)(c_last & 1u)), (c_last >> 1) & 1u, abort_flag);
+            // ---- wait for the unit's last P V (operations complete in issue order, so it covers all of them)
+            if (ok && n_it > 0) {
+                const uint32_t tl = gt + (uint32_t)n_it - 1u;
+                ok = mbar_wait(bar(B_PVDONE + (int)(tl % SB)), (tl / SB) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
             }
-            cnt += (uint32_t)n_mine;
-            if (grp == 1) merge_ml[row] = make_float2(m_used, (ok && n_mine > 0) ? l : 0.f);
-            tc_fence_before();
-            if (!group_sync(sync_a, use_a, abort_flag)) ok = false;
+            gt += (uint32_t)n_it;
+            if (lg == 0 && lane == 0) SR_TRACE(2 + half, 3, u);
+            // ---- row sum = the pair's two shares
+            const int pxl = (int)(use_pair & 1u) * 256;
+            xch[pxl + half * 128 + row] = l;
+            if (ok) ok = group_sync(pair_bar, use_pair, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
             tc_fence_after();
-            if (grp == 0 && ok) {
-                // ---- merge the two groups; write the output, or this chunk's partial
-                const float2 other = merge_ml[row];
-                const float m1 = other.x, l1 = other.y;
-                const bool have0 = n_mine > 0 && l > 0.f, have1 = l1 > 0.f;
-                const float M = fmaxf(have0 ? m_used : -INFINITY, have1 ? m1 : -INFINITY);
-                const float w0 = have0 ? ex2_approx(m_used - M) : 0.f, w1 = have1 ? ex2_approx(m1 - M) : 0.f;
-                const float lt = w0 * l + w1 * l1;
+            const float lt = l + xch[pxl + (half ^ 1) * 128 + row];
+            {
+                // ---- output (or this chunk's partial): this thread's D/2 columns of its row
                 const int n = row_ok ? gr / G : 0, g = row_ok ? gr % G : 0;
                 const bool direct = (n_splits == 1);
                 const float inv = direct ? (lt > 0.f ? 1.0f / lt : 0.f) : 1.0f;
-                const float f0 = w0 * inv, f1 = w1 * inv;
-                __nv_bfloat16 *dst_o = a.O + (((size_t)b * N + n) * a.Hq + hkv * G + g) * D;
-                const size_t prow = ((size_t)item * a.Hkv + hkv) * a.rows_pad + (row_ok ? gr : 0);
-                float *dst_p = a.part_o + prow * D;
-                const bool any0 = __any_sync(0xffffffffu, have0), any1 = __any_sync(0xffffffffu, have1);
+                __nv_bfloat16 *dst_o = a.O + (((size_t)b * N + n) * a.Hq + hkv * G + g) * D + half * DH;
+                // partials are stored [unit][float4 column][row] so that a warp's stores are contiguous
+                const size_t pbase = ((size_t)item * a.Hkv + hkv) * (size_t)(D / 4) * a.rows_pad;
+                float4 *dst_p = reinterpret_cast<float4 *>(a.part_o) + pbase + (size_t)(half * (DH / 4)) * a.rows_pad + gr;
 #pragma unroll 1
-                for (int c = 0; c < D; c += 32) {
-                    uint32_t o0[32], o1[32];
-                    if (any0) tmem_ld32(t_lane + O_COL + (uint32_t)c, o0);
-                    if (any1) tmem_ld32(t_lane + O_COL + 128u + (uint32_t)c, o1);
-                    tmem_ld_wait();
-                    float v[32];
+                for (int c = 0; c < DH; c += 32) {
+                    uint32_t o[32];
+                    if (n_it > 0) {
+                        tmem_ld32(o_t + (uint32_t)c, o);
+                        tmem_ld_wait();
+                    } else {
 #pragma unroll
-                    for (int i2 = 0; i2 < 32; ++i2)
-                        v[i2] = (have0 ? __uint_as_float(o0[i2]) * f0 : 0.f) + (have1 ? __uint_as_float(o1[i2]) * f1 : 0.f);
+                        for (int i2 = 0; i2 < 32; ++i2) o[i2] = 0u;
+                    }
                     if (!row_ok) continue;
                     if (direct) {
 #pragma unroll
                         for (int i2 = 0; i2 < 32; i2 += 8) {
                             uint4 q4;
-                            q4.x = pack_bf16x2(v[i2], v[i2 + 1]);
-                            q4.y = pack_bf16x2(v[i2 + 2], v[i2 + 3]);
-                            q4.z = pack_bf16x2(v[i2 + 4], v[i2 + 5]);
-                            q4.w = pack_bf16x2(v[i2 + 6], v[i2 + 7]);
+                            q4.x = pack_bf16x2(__uint_as_float(o[i2]) * inv, __uint_as_float(o[i2 + 1]) * inv);
+                            q4.y = pack_bf16x2(__uint_as_float(o[i2 + 2]) * inv, __uint_as_float(o[i2 + 3]) * inv);
+                            q4.z = pack_bf16x2(__uint_as_float(o[i2 + 4]) * inv, __uint_as_float(o[i2 + 5]) * inv);
+                            q4.w = pack_bf16x2(__uint_as_float(o[i2 + 6]) * inv, __uint_as_float(o[i2 + 7]) * inv);
                             *reinterpret_cast<uint4 *>(dst_o + c + i2) = q4;
                         }
                     } else {
 #pragma unroll
                         for (int i2 = 0; i2 < 32; i2 += 4)
-                            *reinterpret_cast<float4 *>(dst_p + c + i2) = make_float4(v[i2], v[i2 + 1], v[i2 + 2], v[i2 + 3]);
+                            dst_p[(size_t)((c + i2) / 4) * a.rows_pad] =
+                                make_float4(__uint_as_float(o[i2]), __uint_as_float(o[i2 + 1]), __uint_as_float(o[i2 + 2]),
+                                            __uint_as_float(o[i2 + 3]));
                     }
                 }
-                if (row_ok) {
+                const size_t prow = ((size_t)item * a.Hkv + hkv) * a.rows_pad + (row_ok ? gr : 0);
+                if (row_ok && half == 0) {
                     if (direct) {
-                        if (a.lse) a.lse[((size_t)b * N + n) * a.Hq + hkv * G + g] = (M + log2f(lt)) * 0.6931471805599453f;
+                        if (a.lse) a.lse[((size_t)b * N + n) * a.Hq + hkv * G + g] = (m_used + log2f(lt)) * 0.6931471805599453f;
                     } else {
-                        a.part_ml[prow * 2] = M;
+                        a.part_ml[prow * 2] = m_used;
                         a.part_ml[prow * 2 + 1] = lt;
                     }
                 }
                 if (!direct) {
                     // ---- the chunk that arrives last merges all chunks of this (sequence, kv head, row block)
                     __threadfence();
-                    bool ok3 = group_sync(sync_g0, use_g0, abort_flag);
-                    if (row == 0) *ticket = atomicAdd(a.split_counters + ((size_t)b * a.Hkv + hkv) * a.n_rb + rb, 1);
-                    ok3 = group_sync(sync_g0, use_g0, abort_flag) && ok3;
+                    bool ok3 = group_sync(bar(B_ALL), use_all, abort_flag);
+                    if (half == 0 && row == 0) *ticket = atomicAdd(a.split_counters + ((size_t)b * a.Hkv + hkv) * a.n_rb + rb, 1);
+                    ok3 = group_sync(bar(B_ALL), use_all, abort_flag) && ok3;
                     if (ok3 && *ticket == n_splits - 1 && row_ok) {
                         __threadfence();
                         float Mx = -INFINITY;
@@ -543,7 +565,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         }
                         const float invl = lsum > 0.f ? 1.0f / lsum : 0.f;
 #pragma unroll 1
-                        for (int c = 0; c < D; c += 32) {
+                        for (int c = 0; c < DH; c += 32) {
                             float acc[32];
 #pragma unroll
                             for (int i2 = 0; i2 < 32; ++i2) acc[i2] = 0.f;
@@ -551,10 +573,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                                 const size_t pr = ((size_t)(item0 + s) * a.Hkv + hkv) * a.rows_pad + gr;
                                 const float ms = __ldcg(a.part_ml + pr * 2);
                                 const float ws = (ms == -INFINITY) ? 0.f : ex2_approx(ms - Mx) * invl;
-                                const float4 *src = reinterpret_cast<const float4 *>(a.part_o + pr * D + c);
+                                const float4 *src = reinterpret_cast<const float4 *>(a.part_o) +
+                                                    ((size_t)(item0 + s) * a.Hkv + hkv) * (size_t)(D / 4) * a.rows_pad +
+                                                    (size_t)((half * DH + c) / 4) * a.rows_pad + gr;
 #pragma unroll
                                 for (int i2 = 0; i2 < 8; ++i2) {
-                                    const float4 x = __ldcg(src + i2);
+                                    const float4 x = __ldcg(src + (size_t)i2 * a.rows_pad);
                                     acc[4 * i2] += ws * x.x;
                                     acc[4 * i2 + 1] += ws * x.y;
                                     acc[4 * i2 + 2] += ws * x.z;
@@ -571,15 +595,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                                 *reinterpret_cast<uint4 *>(dst_o + c + i2) = q4;
                             }
                         }
-                        if (a.lse) a.lse[((size_t)b * N + n) * a.Hq + hkv * G + g] = (Mx + log2f(lsum)) * 0.6931471805599453f;
+                        if (a.lse && half == 0)
+                            a.lse[((size_t)b * N + n) * a.Hq + hkv * G + g] = (Mx + log2f(lsum)) * 0.6931471805599453f;
                     }
                 }
             }
-            // group 1 must not start the next unit's tiles (its P V overwrites O1) before group 0 has read O1
+            if (lg == 0 && lane == 0) SR_TRACE(2 + half, 4, u);
+            // No rendezvous is needed before the next unit: its first P V (which overwrites O) waits for the
+            // P of all 256 threads, and each of them arrives there only after it has finished reading O here.
             tc_fence_before();
-            if (!group_sync(sync_b, use_b, abort_flag)) ok = false;
-            ok = __all_sync(0xffffffffu, ok);
-            tc_fence_after();
         }
     }
 
@@ -621,6 +645,17 @@ static int launch_tc(const AttnArgs &a, const TopoMask &mask, long long T_kv, in
     SR_LAUNCH_CHECK();
     return SPECROLL_OK;
 }
+
+#ifdef SPECROLL_TRACE
+extern "C" int specroll_debug_trace_reset(void) {
+    unsigned int z[4] = {0, 0, 0, 0};
+    return cudaMemcpyToSymbol(g_trace_n, z, sizeof(z)) == cudaSuccess ? 0 : 4;
+}
+extern "C" int specroll_debug_trace_read(unsigned long long *dst, unsigned int *counts) {
+    if (cudaMemcpyFromSymbol(counts, g_trace_n, 16) != cudaSuccess) return 4;
+    return cudaMemcpyFromSymbol(dst, g_trace, sizeof(unsigned long long) * 4 * 8192) == cudaSuccess ? 0 : 4;
+}
+#endif
 
 int launch_attn_tc(const AttnArgs &a, const TopoMask &mask, int D, long long T_kv, int32_t *status, cudaStream_t st) {
     if (D == 128) return launch_tc<128>(a, mask, T_kv, status, st);
