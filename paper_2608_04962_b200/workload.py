@@ -140,7 +140,7 @@ class StepWorkload:
             events[3].record()
 
     # ---- bookkeeping for the report
-    LAUNCHES_PROPOSE, LAUNCHES_ATTN, LAUNCHES_VERIFY = 6, 3, 3
+    LAUNCHES_PROPOSE, LAUNCHES_ATTN, LAUNCHES_VERIFY = 6, 2, 3   # kernels per call
 
     def launches_per_step(self) -> int:
         return self.LAUNCHES_PROPOSE + self.layers * self.LAUNCHES_ATTN + self.LAUNCHES_VERIFY
