@@ -237,7 +237,7 @@ def run_ours(args, w, layers):
                 "achieved": attn_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / peaks["hbm_gbs"],
                 "peak_source": peaks["source"], "frac_of_nominal_8TBs": attn_gbs / 8000.0,
                 "algorithmic_bytes_per_launch": wl.attn_algorithmic_bytes(),
-                "traffic": recorded_traffic("tree_attn_kernel", w.name)}
+                "traffic": recorded_traffic("tree_attn_tc_kernel", w.name)}
     ver_gbs = wl.rowstats_algorithmic_bytes() / (ver_ms * 1e-3) / 1e9
     lm_tf = (wl.lmhead_algorithmic_flops() + 2 * w.B * w.K * w.d * w.d) / (prop_ms * 1e-3) / 1e12
     phases = {
