@@ -107,6 +107,11 @@ def version() -> int:
     return int(lib().specroll_version())
 
 
+def workspace_status(workspace: torch.Tensor) -> int:
+    """specroll_workspace_status: 0, or the error code a kernel left in this workspace (synchronises)."""
+    return int(lib().specroll_workspace_status(C.c_void_p(workspace.data_ptr()), _stream()))
+
+
 def node_budget(C_hw: int, B_active: int, N_min: int = 1, N_max: int = 10) -> int:
     return int(lib().specroll_node_budget(C_hw, B_active, N_min, N_max))
 
