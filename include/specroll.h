@@ -130,11 +130,15 @@ int specroll_tree_draw(int32_t B, int32_t N, int32_t K, int32_t k, float tempera
 typedef struct {
     int32_t B, N, Hq, Hkv, D;
     float scale;   /* softmax scale (> 0); the method uses 1/sqrt(D) */
-    int32_t flags; /* 0, or SPECROLL_ATTN_LEGACY_MMA */
+    int32_t flags; /* 0, or an OR of the SPECROLL_ATTN_* flags below */
 } specroll_attn_desc;
 
 /* Run the attention on the mma.sync kernel instead of the tcgen05 one (kept for comparison). */
 #define SPECROLL_ATTN_LEGACY_MMA 1
+/* The workspace still holds the work plan of an earlier specroll_tree_attn call with the same
+ * descriptor and the same kv_indptr values (typically the previous layer of the same step): do not
+ * rebuild it.  Tensors (Q, K, V, O) may differ.  Ignored by the mma.sync kernel. */
+#define SPECROLL_ATTN_REUSE_PLAN 2
 
 size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *desc,
                                           const int32_t *kv_indptr_host);

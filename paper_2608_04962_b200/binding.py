@@ -25,6 +25,11 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
            "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static")
 
 
+PROPOSE_LEGACY_MMA = 1
+ATTN_LEGACY_MMA = 1
+ATTN_REUSE_PLAN = 2
+
+
 class SpecrollError(RuntimeError):
     pass
 

@@ -448,7 +448,7 @@ struct AttnPlan {
 
 static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
     if (!d || !indptr_host || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->Hq < 1 || d->Hkv < 1 ||
-        (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || (d->flags & ~SPECROLL_ATTN_LEGACY_MMA) != 0 ||
+        (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || (d->flags & ~(SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN)) != 0 ||
         !(d->scale > 0.f))
         return SPECROLL_EINVAL;
     const int G = d->Hq / d->Hkv;
@@ -599,11 +599,14 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
     a.split_counters = counters + 64;
     a.total_work = p.items * d->Hkv * p.n_rb;
     a.nodes_per_block = p.nodes_per_block;
-    attn_prep_kernel<<<1, PREP_THREADS, 0, st>>>(kv_indptr_dev, d->B, p.chunk_tiles, p.tile_tokens,
-                                                 reinterpret_cast<int32_t *>(ws + p.off_items),
-                                                 p.use_tc ? sorted_start : nullptr, seq_at_rank,
-                                                 p.use_tc ? unit_tab : nullptr, status, counters, p.n_counters);
-    SR_LAUNCH_CHECK();
+    if (!(p.use_tc && (d->flags & SPECROLL_ATTN_REUSE_PLAN))) {
+        // (the tcgen05 kernel leaves its scheduling counters cleared, so a kept plan can be run again as is)
+        attn_prep_kernel<<<1, PREP_THREADS, 0, st>>>(kv_indptr_dev, d->B, p.chunk_tiles, p.tile_tokens,
+                                                     reinterpret_cast<int32_t *>(ws + p.off_items),
+                                                     p.use_tc ? sorted_start : nullptr, seq_at_rank,
+                                                     p.use_tc ? unit_tab : nullptr, status, counters, p.n_counters);
+        SR_LAUNCH_CHECK();
+    }
     const size_t n_out = (size_t)d->B * d->N * d->Hq;
     if (p.use_tc) return launch_attn_tc(a, mask, d->D, T_kv, status, st);  // merges split sequences itself
     if (d->D == 128) return launch_attn<128>(a, mask, p, d->Hkv, n_out, st);

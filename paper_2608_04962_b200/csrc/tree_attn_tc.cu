@@ -610,10 +610,24 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // ------------------------------------------------------------------ teardown
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0 && *abort_flag) atomicExch(status, SPECROLL_ETIMEOUT);
+    if (threadIdx.x == 0) {
+        if (*abort_flag) atomicExch(status, SPECROLL_ETIMEOUT);
+        // the CTA that leaves last clears the scheduling counters, so the same plan can be launched again
+        __threadfence();
+        *ticket = (atomicAdd(a.work_counter + 1, 1) == (int)gridDim.x - 1) ? 1 : 0;
+    }
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+    __syncthreads();
+    if (*ticket) {
+        const int n_split = a.B * a.Hkv * a.n_rb;
+        for (int i = threadIdx.x; i < n_split; i += THREADS) a.split_counters[i] = 0;
+        if (threadIdx.x == 0) {
+            a.work_counter[0] = 0;
+            a.work_counter[1] = 0;
+        }
     }
 }
 

@@ -113,9 +113,10 @@ class StepWorkload:
         return self.prop
 
     def attn(self, layer: int):
+        # every layer of a step sees the same KV lengths: layers after the first reuse the work plan
         return S.tree_attn(self.Q[layer], self.Kc[layer], self.Vc[layer], self.kv_indptr, self.kv_indptr_host,
                            self.Kt[layer], self.Vt[layer], self.parent, workspace=self.ws_attn,
-                           out=self.O[layer])
+                           out=self.O[layer], flags=S.ATTN_REUSE_PLAN if layer > 0 else 0)
 
     def verify(self):
         p = self.prop
@@ -143,7 +144,8 @@ class StepWorkload:
     LAUNCHES_PROPOSE, LAUNCHES_ATTN, LAUNCHES_VERIFY = 6, 2, 3   # kernels per call
 
     def launches_per_step(self) -> int:
-        return self.LAUNCHES_PROPOSE + self.layers * self.LAUNCHES_ATTN + self.LAUNCHES_VERIFY
+        # the attention prep kernel runs for the first layer only (the plan is reused afterwards)
+        return self.LAUNCHES_PROPOSE + 1 + self.layers * (self.LAUNCHES_ATTN - 1) + self.LAUNCHES_VERIFY
 
     def tokens_per_step(self) -> int:
         return self.w.B * self.w.N

@@ -104,3 +104,27 @@ def test_scale_argument_and_topology_errors():
     bad[2] = 2
     with pytest.raises(S.SpecrollError):
         S.tree_attn(*args, bad)
+
+
+def test_plan_reuse_across_layers():
+    # second call keeps the first call's work plan (same KV lengths, different tensors), as the layers of a
+    # step do; results must still match the oracle, also for a third call
+    if FLAGS["v"] != 0:
+        pytest.skip("plan reuse is a feature of the tcgen05 kernel")
+    w = I.scaled(I.WORKLOADS["qwen7b"], B=6, N=32)
+    lengths = np.array([3000, 64, 700, 129, 5000, 1], np.int32)
+    ip = np.zeros(w.B + 1, np.int32)
+    np.cumsum(lengths, out=ip[1:])
+    ws = None
+    for layer in range(3):
+        x = I.attn_inputs(w, layer=layer)
+        g = I.rng(900 + layer)
+        Kc = I.f32_to_bf16_bits(g.standard_normal((int(ip[-1]), w.Hkv, w.D), dtype=np.float32))
+        Vc = I.f32_to_bf16_bits(g.standard_normal((int(ip[-1]), w.Hkv, w.D), dtype=np.float32))
+        o = ref.tree_attn(x["Q"], Kc, Vc, ip, x["Kt"], x["Vt"], x["parent"])
+        if ws is None:
+            ws = torch.empty(S.tree_attn_workspace_bytes(w.B, w.N, w.Hq, w.Hkv, w.D, ip), dtype=torch.uint8, device="cuda")
+        O = S.tree_attn(dev_bf16(x["Q"]), dev_bf16(Kc), dev_bf16(Vc), dev(ip), ip, dev_bf16(x["Kt"]), dev_bf16(x["Vt"]),
+                        x["parent"], workspace=ws, flags=S.ATTN_REUSE_PLAN if layer > 0 else 0, check_status=True)
+        diff = np.abs(host(O.float()) - o["O64"])
+        assert (diff <= O_ATOL * np.maximum(1.0, np.abs(o["O64"]))).all(), (layer, diff.max())
