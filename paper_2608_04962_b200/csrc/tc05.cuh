@@ -65,7 +65,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (((++spins) & 127u) == 0u) {
             if (*abort_flag) return false;
             if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
-                *abort_flag = 1;
+                // records which wait gave up: barrier address (shared window) and the parity waited for
+                *abort_flag = (int)(0x40000000u | (parity << 24) | (bar & 0xffffffu));
                 return false;
             }
         }

@@ -441,7 +441,8 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(AttnArgs a) {
 // ------------------------------------------------------------------------------ host side
 
 struct AttnPlan {
-    int rows, n_rb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens, nodes_per_block, n_counters;
+    int rows, n_rb, nrb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens, nodes_per_block, n_counters;
+    int merge_mode;  // tcgen05 path: 0 = split sequences are merged inside the attention kernel, 2 = by a kernel after it
     bool use_tc;
     size_t off_status, off_items, off_sorted, off_rank, off_tab, off_counters, off_po, off_pml, total;
 };
@@ -459,13 +460,26 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     p->rows = d->N * G;
     if (p->use_tc) {
         // row blocks are whole nodes: (node, head-in-group) rows of a block are one TMA box
+        // and, when one block does not hold all rows, a work unit carries two blocks that share each K/V tile
         int npb = 128 / G;
-        const int nb = (d->N + npb - 1) / npb;
+        int nb = (d->N + npb - 1) / npb;
+        p->nrb = nb > 1 ? 2 : 1;
+        if (nb > 1 && (nb & 1)) {
+            ++nb;
+            if (nb > d->N) return SPECROLL_EINVAL;  // cannot happen for N >= 2 (nb is at most N)
+        }
         npb = (d->N + nb - 1) / nb;  // even out the blocks
+        if ((nb - 1) * npb >= d->N) {  // evening out left the last block empty: fall back to one block per unit
+            npb = 128 / G;
+            nb = (d->N + npb - 1) / npb;
+            npb = (d->N + nb - 1) / nb;
+            p->nrb = 1;
+        }
         p->nodes_per_block = npb;
         p->n_rb = nb;
         p->rows_per_block = npb * G;
     } else {
+        p->nrb = 1;
         p->nodes_per_block = 0;
         p->n_rb = (p->rows + AT_MAX_WARPS * 16 - 1) / (AT_MAX_WARPS * 16);
         p->rows_per_block = ((p->rows + p->n_rb - 1) / p->n_rb + 15) / 16 * 16;
@@ -482,7 +496,7 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     }
     // chunk length: about four CTAs' worth of work per SM over the whole launch, at least 512
     // tokens so that the fp32 partials stay a small fraction of the KV bytes
-    long long ctas_per_tile = (long long)d->Hkv * p->n_rb;
+    long long ctas_per_tile = (long long)d->Hkv * p->n_rb / p->nrb;
     const int per_sm_div = p->use_tc ? 2 : 4;  // the persistent kernel balances dynamically: fewer, larger chunks
     long long ct = (tiles_total * ctas_per_tile + 148 * per_sm_div - 1) / (148 * per_sm_div);
     if (ct < 512 / TT) ct = 512 / TT;
@@ -497,6 +511,9 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     }
     p->items = items;
     if (max_tiles / p->chunk_tiles + 1 > 65535) return SPECROLL_EINVAL;
+    // A sequence cut into many chunks is merged by a kernel of its own, over the whole GPU; with few chunks the
+    // CTA that finishes a sequence's last chunk merges them while the others keep streaming.
+    p->merge_mode = (p->use_tc && (max_tiles + p->chunk_tiles - 1) / p->chunk_tiles >= 5) ? 2 : 0;
     p->n_counters = 64 + d->B * d->Hkv * p->n_rb;  // [0]: work counter; [64 ...]: per (b, hkv, rb) arrivals
     size_t o = 0;
     p->off_status = o;
@@ -597,7 +614,9 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
     a.unit_tab = unit_tab;
     a.work_counter = counters;
     a.split_counters = counters + 64;
-    a.total_work = p.items * d->Hkv * p.n_rb;
+    a.total_work = p.items * d->Hkv * (p.n_rb / p.nrb);
+    a.nrb = p.nrb;
+    a.merge_mode = p.merge_mode;
     a.nodes_per_block = p.nodes_per_block;
     if (!(p.use_tc && (d->flags & SPECROLL_ATTN_REUSE_PLAN))) {
         // (the tcgen05 kernel leaves its scheduling counters cleared, so a kept plan can be run again as is)
@@ -608,7 +627,11 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
         SR_LAUNCH_CHECK();
     }
     const size_t n_out = (size_t)d->B * d->N * d->Hq;
-    if (p.use_tc) return launch_attn_tc(a, mask, d->D, T_kv, status, st);  // merges split sequences itself
+    if (p.use_tc) {
+        const int rc = launch_attn_tc(a, mask, d->D, T_kv, status, st);
+        if (rc != SPECROLL_OK || p.merge_mode != 2 || p.items <= d->B) return rc;
+        return launch_attn_merge_tc(a, d->D, p.items, st);
+    }
     if (d->D == 128) return launch_attn<128>(a, mask, p, d->Hkv, n_out, st);
     return launch_attn<64>(a, mask, p, d->Hkv, n_out, st);
 }

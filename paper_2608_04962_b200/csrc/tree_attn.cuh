@@ -22,11 +22,15 @@ struct AttnArgs {
     const int32_t *unit_tab;      // [items][8] per chunk in work order: b, chunk, n_chunks, first item, kv0, L, 0, 0
     int32_t *work_counter;        // next work unit to hand out
     int32_t *split_counters;      // [B, Hkv, n_rb] chunks of a (sequence, kv head, row block) that have finished
-    int32_t total_work;           // items * Hkv * n_rb
+    int32_t total_work;           // items * Hkv * n_rb / nrb
     int32_t nodes_per_block;      // rows_per_block = nodes_per_block * G
+    int32_t nrb;                  // row blocks per work unit: 1, or 2 (then n_rb is even)
+    int32_t merge_mode;           // chunks of a split sequence are merged 0: by the CTA that finishes last; 2: by a later kernel
 };
 
 // tcgen05 kernel (tree_attn_tc.cu).  T_kv = total cached tokens.  Launches the main kernel only.
 int launch_attn_tc(const AttnArgs &a, const TopoMask &mask, int D, long long T_kv, int32_t *status, cudaStream_t st);
+// Merges the chunks of split sequences after launch_attn_tc when a.merge_mode == 2.  items = chunks in the plan.
+int launch_attn_merge_tc(const AttnArgs &a, int D, int items, cudaStream_t st);
 
 }  // namespace specroll

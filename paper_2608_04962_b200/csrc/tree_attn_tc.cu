@@ -1,27 +1,29 @@
 // Tree-verification attention on the 5th-generation tensor cores (tcgen05 + TMEM), one layer.
 //
-// Decomposition: for one (sequence, KV head) the N*G query rows form the M dimension; a work unit
-// is up to 128 of them (whole nodes) times one chunk of the cache (split-KV), streamed as 128-token
-// K/V tiles.  The kernel is persistent: one CTA per SM takes work units from a global counter, in an
-// order prepared on the device (longest chunks first), and its pipeline runs across unit boundaries.
-// Warp roles (320 threads):
+// Decomposition: for one (sequence, KV head) the N*G query rows form the M dimension, cut into row
+// blocks of up to 128 rows (whole nodes).  A work unit is NRB row blocks (1 when all rows fit one
+// block, else 2) times one chunk of the cache (split-KV), streamed as 128-token K/V tiles that all
+// row blocks of the unit share.  The kernel is persistent: one CTA per SM takes work units from a
+// global counter, in an order prepared on the device (longest chunks first), and its pipeline runs
+// across unit boundaries.  Warp roles (64 + 256*NRB threads):
 //   warp 0     scheduler + TMA producer: fetches the next unit, publishes its descriptor in a
-//              two-slot ring, loads the Q block (3-D box over [node, head, D]) and the K and V tiles
-//              (3-D boxes over [token, kv head, D], 128-byte swizzle).  K and V have separate rings
-//              (4 and 2 stages): K is needed early, because S runs ahead, and is released as soon as
-//              its S is computed; V is needed late and released after P V.
-//   warp 1     allocates TMEM, issues  S = Q K^T  (M=128, N=128, operands from shared memory), up to
-//              three tiles ahead, and  O += P V  (M=128, N=D, A = P from TMEM, B = V tile read
-//              MN-major from shared memory)
-//   warps 2-9  softmax: TWO threads per query row (warps w and w+4 own the same 32 TMEM lanes and
-//              take columns 0-63 / 64-127 of each S tile), so the per-tile latency between "S ready"
-//              and "P ready" is half of the one-thread-per-row form.  The pair exchanges its two
-//              partial row maxima through shared memory once per tile.
-// P overwrites the first half of its S buffer in place (packed bf16).  The output accumulator is
-// rescaled only when a row's maximum grows by more than 2^8 (rare).  Chunks of a split sequence
-// leave fp32 partials in the workspace; the CTA that finishes a sequence's last chunk (atomic
-// ticket, nobody waits) merges them.
-// TMEM columns: O [0,128)   S/P buffer i: [128 + 128 i, +128), i = tile mod 3.
+//              two-slot ring, loads the Q blocks (3-D box over [node, head, D]) and the K and V tiles
+//              (3-D boxes over [token, kv head, D], 128-byte swizzle).  K and V have separate rings:
+//              K is needed early and is released as soon as its S is computed; V is needed late.
+//   warp 1     allocates TMEM, issues  S = Q K^T  (M=128, N=128, operands from shared memory) and
+//              O += P V  (M=128, N=D, A = P from TMEM, B = V tile read MN-major from shared memory).
+//              NRB=1: three S buffers, S runs three tiles ahead.  NRB=2: one S buffer per row block;
+//              the two blocks alternate on the tensor pipe, each one's softmax hiding under the
+//              other's MMAs.
+//   8 warps per row block: softmax with TWO threads per query row (warps w and w+4 own the same 32
+//              TMEM lanes and take columns 0-63 / 64-127 of each S tile).  The pair exchanges its
+//              two partial row maxima through shared memory once per tile.
+// P is written back to TMEM over parts of S that its writer has already read (columns [0,32) by
+// the first thread of a pair, [96,128) by the second), as packed bf16.  An output accumulator is
+// rescaled only when a row's reference maximum grows by more than 2^8 (rare).  Chunks of a split
+// sequence leave fp32 partials in the workspace; the CTA that finishes a sequence's last chunk
+// (atomic ticket, nobody waits) merges them.
+// TMEM columns: O of block b: [128 b, +128);  S/P buffer i of block b: [128 NRB + 128 (b SB + i), +128).
 #include <math.h>
 
 #include "tc05.cuh"
@@ -48,36 +50,40 @@ __device__ unsigned int g_trace_n[4];
 #endif
 
 namespace attc {
-constexpr int BN = 128;       // KV tokens per tile
-constexpr int THREADS = 320;
-constexpr int KS = 4, VS = 2, SB = 3;  // K stages, V stages, S buffers
+constexpr int BN = 128;  // KV tokens per tile
+constexpr int VS = 2;    // V stages
 constexpr int TMEM_COLS = 512;
-constexpr uint32_t O_COL = 0, S_COL = 128;
 constexpr float RESCALE_LOG2 = 8.0f;
 constexpr int BOX_BYTES = BN * 128;  // 128 rows x 128 bytes (64 bf16)
-// barrier slots
-constexpr int B_KFULL = 0, B_KEMPTY = B_KFULL + KS, B_VFULL = B_KEMPTY + KS, B_VEMPTY = B_VFULL + VS,
-              B_SFULL = B_VEMPTY + VS, B_PREADY = B_SFULL + SB, B_PVDONE = B_PREADY + SB, B_QFULL = B_PVDONE + SB,
-              B_QFREE = B_QFULL + 1, B_UFULL = B_QFREE + 1, B_UEMPTY = B_UFULL + 2, B_PAIR = B_UEMPTY + 2,
-              B_ALL = B_PAIR + 4, N_BARS = B_ALL + 1;
 
 struct UnitDesc {
     int32_t valid, b, hkv, rb, n_splits, kv0, L, t_lo, n_it, has_tree, item, item0;
 };
 
-template <int D>
+template <int D, int NRB>
 struct Cfg {
     static constexpr int NBOX = D / 64;
-    static constexpr int Q_BYTES = NBOX * BOX_BYTES;
+    static constexpr int SB = NRB == 1 ? 3 : 1;  // S buffers per row block
+    static constexpr int KS = NRB == 1 ? 4 : 3;  // K stages
+    static constexpr int THREADS = 64 + 256 * NRB;
+    static constexpr int QB_BYTES = NBOX * BOX_BYTES;  // one Q block
+    static constexpr int Q_BYTES = NRB * QB_BYTES;
     static constexpr int KV_BYTES = NBOX * BOX_BYTES;  // one K tile or one V tile
+    // barrier slots
+    static constexpr int B_KFULL = 0, B_KEMPTY = B_KFULL + KS, B_VFULL = B_KEMPTY + KS, B_VEMPTY = B_VFULL + VS,
+                         B_SFULL = B_VEMPTY + VS, B_PREADY = B_SFULL + NRB * SB, B_PVDONE = B_PREADY + NRB * SB,
+                         B_QFULL = B_PVDONE + NRB * SB, B_QFREE = B_QFULL + 1, B_UFULL = B_QFREE + 1,
+                         B_UEMPTY = B_UFULL + 2, B_PAIR = B_UEMPTY + 2, B_ALL = B_PAIR + 4 * NRB, N_BARS = B_ALL + NRB;
     static constexpr int BAR_BYTES = (8 * N_BARS + 15) / 16 * 16;
-    static constexpr int EXTRA = BAR_BYTES + 16 + 4 * 128 * 4 + 2 * 64;  // barriers, slot/abort/ticket, pair exchange, ring
+    static constexpr int XCH_BYTES = NRB * 1024;  // per (block, lane group) 256 bytes: maxima as bf16 or row sums as fp32
+    static constexpr int EXTRA = BAR_BYTES + 16 + XCH_BYTES + 2 * 64;  // barriers, slot/abort/tickets, exchange, ring
     // The operand tiles need 1024-byte alignment.  The dynamic shared window starts 1024-aligned on this
     // architecture (checked at run time), so only a small slack is budgeted.
     static constexpr int SLACK = 256;
     static constexpr int USED = Q_BYTES + (KS + VS) * KV_BYTES + SLACK + EXTRA;
     // at least ~118 KB so that two CTAs can never share an SM (each allocates all of TMEM)
     static constexpr int SMEM = USED > 120832 ? USED : 120832;
+    static constexpr uint32_t O_COL = 0, S_COL = 128 * NRB;
     static_assert(sizeof(UnitDesc) <= 64, "ring slot");
     static_assert(USED <= 232448, "shared memory budget");
 };
@@ -90,17 +96,23 @@ __device__ __forceinline__ bool group_sync(uint32_t bar, uint32_t &uses, volatil
     ++uses;
     return ok;
 }
+
+__device__ __forceinline__ unsigned short bf16_bits_rn(float x) {
+    return __bfloat16_as_ushort(__float2bfloat16_rn(x));
+}
+__device__ __forceinline__ float bf16_bits_to_float(unsigned short b) { return __uint_as_float((uint32_t)b << 16); }
 }  // namespace attc
 
-template <int D>
-__global__ void __launch_bounds__(attc::THREADS, 1)
+template <int D, int NRB>
+__global__ void __launch_bounds__(attc::Cfg<D, NRB>::THREADS, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKt,
                     const __grid_constant__ CUtensorMap tmVt, AttnArgs a, TopoMask mask,
                     int32_t *__restrict__ status) {
     using namespace attc;
-    using C = Cfg<D>;
+    using C = Cfg<D, NRB>;
     constexpr int DH = D / 2;  // output columns per thread of a pair
+    constexpr int SB = C::SB, KS = C::KS, THREADS = C::THREADS;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -113,9 +125,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     unsigned char *extra = aligned + C::Q_BYTES + (KS + VS) * C::KV_BYTES + C::BAR_BYTES;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(extra);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(extra + 4);
-    volatile int *ticket = reinterpret_cast<volatile int *>(extra + 8);
-    volatile float *xch = reinterpret_cast<volatile float *>(extra + 16);  // [2 parities][2 halves][128 rows]
-    volatile UnitDesc *ring = reinterpret_cast<volatile UnitDesc *>(extra + 16 + 4 * 128 * 4);  // 2 slots of 64 bytes
+    volatile int *tickets = reinterpret_cast<volatile int *>(extra + 8);  // one per row block
+    unsigned char *xch_base = extra + 16;
+    volatile UnitDesc *ring = reinterpret_cast<volatile UnitDesc *>(extra + 16 + C::XCH_BYTES);  // 2 slots of 64 bytes
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int N = a.N, G = a.G;
@@ -125,12 +137,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < N_BARS; ++i) {
+        for (int i = 0; i < C::N_BARS; ++i) {
             uint32_t count = 1;
-            if (i >= B_PREADY && i < B_PREADY + SB) count = 256;
-            if (i >= B_UEMPTY && i < B_UEMPTY + 2) count = 257;  // the MMA thread and the 256 softmax threads
-            if (i >= B_PAIR && i < B_PAIR + 4) count = 64;
-            if (i == B_ALL) count = 256;
+            if (i >= C::B_PREADY && i < C::B_PREADY + NRB * SB) count = 256;
+            if (i >= C::B_UEMPTY && i < C::B_UEMPTY + 2) count = 1 + 256 * NRB;  // MMA thread + softmax threads
+            if (i >= C::B_PAIR && i < C::B_PAIR + 4 * NRB) count = 64;
+            if (i >= C::B_ALL && i < C::B_ALL + NRB) count = 256;
             mbar_init(bar(i), count);
         }
         *abort_flag = 0;
@@ -145,7 +157,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
-    // The Q block's TMA box covers rows_per_block rows; the rest of the 128-row operand stays zero.
+    // A Q block's TMA box covers rows_per_block rows; the rest of each 128-row operand stays zero.
     for (int c = threadIdx.x; c < C::Q_BYTES / 16; c += THREADS)
         reinterpret_cast<uint4 *>(aligned)[c] = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async();
@@ -153,29 +165,31 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    const int units_per_chunk = a.n_rb / NRB;  // row-block groups per (chunk, kv head)
 
     if (warp == 0) {
         // ------------------------------------------------------------------ scheduler + TMA producer
         if (lane == 0) {
             bool ok = true;
-            uint32_t kt = 0, vt = 0;   // K and V tiles loaded so far (all units)
+            uint32_t kt = 0, vt = 0;  // K and V tiles loaded so far (all units)
             // V loads trail K loads by two tiles, carried over unit boundaries: (map, kv head, token) of pending V tiles
             const CUtensorMap *pv_map[2];
             int pv_h[2], pv_tok[2];
             int n_pend = 0;
             auto load_v = [&](const CUtensorMap *mv, int hkv, int tok) -> bool {
                 const int s = (int)(vt % VS);
-                if (!mbar_wait(bar(B_VEMPTY + s), ((vt / VS) & 1u) ^ 1u, abort_flag)) return false;
+                if (!mbar_wait(bar(C::B_VEMPTY + s), ((vt / VS) & 1u) ^ 1u, abort_flag)) return false;
                 const uint32_t dst = v_s + s * C::KV_BYTES;
-                mbar_arrive_expect_tx(bar(B_VFULL + s), C::KV_BYTES);
+                mbar_arrive_expect_tx(bar(C::B_VFULL + s), C::KV_BYTES);
 #pragma unroll
-                for (int bx = 0; bx < C::NBOX; ++bx) tma_load_3d(dst + bx * BOX_BYTES, mv, bx * 64, hkv, tok, bar(B_VFULL + s));
+                for (int bx = 0; bx < C::NBOX; ++bx)
+                    tma_load_3d(dst + bx * BOX_BYTES, mv, bx * 64, hkv, tok, bar(C::B_VFULL + s));
                 ++vt;
                 return true;
             };
             for (uint32_t u = 0; ok; ++u) {
                 const int slot = (int)(u & 1u);
-                if (!mbar_wait(bar(B_UEMPTY + slot), ((u >> 1) & 1u) ^ 1u, abort_flag)) {
+                if (!mbar_wait(bar(C::B_UEMPTY + slot), ((u >> 1) & 1u) ^ 1u, abort_flag)) {
                     ok = false;
                     break;
                 }
@@ -183,13 +197,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 volatile UnitDesc *d = ring + slot;
                 if (w >= a.total_work) {
                     d->valid = 0;
-                    mbar_arrive(bar(B_UFULL + slot));
+                    mbar_arrive(bar(C::B_UFULL + slot));
                     break;
                 }
-                // ---- decode: w = (chunk position in work order * Hkv + hkv) * n_rb + rb; one table row per chunk
+                // ---- decode: w = (chunk position in work order * Hkv + hkv) * units_per_chunk + row-block group
                 int t = w;
-                const int rb = t % a.n_rb;
-                t /= a.n_rb;
+                const int rb = (t % units_per_chunk) * NRB;
+                t /= units_per_chunk;
                 const int hkv = t % a.Hkv;
                 const int si = t / a.Hkv;
                 const int4 e0 = __ldg(reinterpret_cast<const int4 *>(a.unit_tab) + 2 * (size_t)si);
@@ -212,21 +226,24 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 d->has_tree = has_tree;
                 d->item = item0 + split;
                 d->item0 = item0;
-                mbar_arrive(bar(B_UFULL + slot));  // release: the descriptor is visible to whoever acquires
+                mbar_arrive(bar(C::B_UFULL + slot));  // release: the descriptor is visible to whoever acquires
                 SR_TRACE(0, 0, u);
-                // ---- Q block of this unit, once every S of the previous unit has been computed
-                if (u > 0 && !mbar_wait(bar(B_QFREE), (u - 1u) & 1u, abort_flag)) {
+                // ---- Q blocks of this unit, once every S of the previous unit has been computed
+                if (u > 0 && !mbar_wait(bar(C::B_QFREE), (u - 1u) & 1u, abort_flag)) {
                     ok = false;
                     break;
                 }
-                mbar_arrive_expect_tx(bar(B_QFULL), (uint32_t)(C::NBOX * 128 * a.rows_per_block));
+                mbar_arrive_expect_tx(bar(C::B_QFULL), (uint32_t)(NRB * C::NBOX * 128 * a.rows_per_block));
 #pragma unroll
-                for (int bx = 0; bx < C::NBOX; ++bx)
-                    tma_load_3d(q_s + bx * BOX_BYTES, &tmQ, bx * 64, hkv * G, b * N + rb * a.nodes_per_block, bar(B_QFULL));
+                for (int blk = 0; blk < NRB; ++blk)
+#pragma unroll
+                    for (int bx = 0; bx < C::NBOX; ++bx)
+                        tma_load_3d(q_s + blk * C::QB_BYTES + bx * BOX_BYTES, &tmQ, bx * 64, hkv * G,
+                                    b * N + (rb + blk) * a.nodes_per_block, bar(C::B_QFULL));
                 // ---- K tiles, each followed by the V tile from two tiles back
                 for (int it = 0; it < n_it && ok; ++it) {
                     const int s = (int)(kt % KS);
-                    if (!mbar_wait(bar(B_KEMPTY + s), ((kt / KS) & 1u) ^ 1u, abort_flag)) {
+                    if (!mbar_wait(bar(C::B_KEMPTY + s), ((kt / KS) & 1u) ^ 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
@@ -234,9 +251,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     const int tok = tree ? b * N : kv0 + (t_lo + it) * BN;
                     const CUtensorMap *mk = tree ? &tmKt : &tmK;
                     const uint32_t dst = k_s + s * C::KV_BYTES;
-                    mbar_arrive_expect_tx(bar(B_KFULL + s), C::KV_BYTES);
+                    mbar_arrive_expect_tx(bar(C::B_KFULL + s), C::KV_BYTES);
 #pragma unroll
-                    for (int bx = 0; bx < C::NBOX; ++bx) tma_load_3d(dst + bx * BOX_BYTES, mk, bx * 64, hkv, tok, bar(B_KFULL + s));
+                    for (int bx = 0; bx < C::NBOX; ++bx)
+                        tma_load_3d(dst + bx * BOX_BYTES, mk, bx * 64, hkv, tok, bar(C::B_KFULL + s));
                     ++kt;
                     SR_TRACE(0, 1, kt);
                     if (n_pend == 2) {
@@ -251,9 +269,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     pv_tok[n_pend] = tok;
                     ++n_pend;
                 }
+                // The next unit's Q waits for this unit's last S, which is issued after the P V of the tile SB
+                // before it: with a single S buffer that P V needs the second-to-last V tile, so it must go
+                // out now (its stage depends on earlier tiles only).
+                if (SB == 1 && ok && n_pend == 2) {
+                    ok = load_v(pv_map[0], pv_h[0], pv_tok[0]);
+                    pv_map[0] = pv_map[1];
+                    pv_h[0] = pv_h[1];
+                    pv_tok[0] = pv_tok[1];
+                    n_pend = 1;
+                }
                 // the unit's last V tiles go out now if their stages are already free; otherwise they wait
                 // behind the next unit's Q and first K tiles (never block here)
-                while (ok && n_pend > 0 && mbar_try_wait(bar(B_VEMPTY + (int)(vt % VS)), ((vt / VS) & 1u) ^ 1u)) {
+                while (ok && n_pend > 0 && mbar_try_wait(bar(C::B_VEMPTY + (int)(vt % VS)), ((vt / VS) & 1u) ^ 1u)) {
                     ok = load_v(pv_map[0], pv_h[0], pv_tok[0]);
                     pv_map[0] = pv_map[1];
                     pv_h[0] = pv_h[1];
@@ -272,8 +300,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        // tcgen05.mma operations of one thread execute in issue order, which is what lets S of tile t+3
-        // overwrite the buffer whose P (tile t) the previously issued P V has read.
+        // tcgen05.mma operations of one thread execute in issue order, which is what lets an S tile
+        // overwrite the buffer whose P the previously issued P V has read.
         if (lane == 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, BN, false, false);
             constexpr uint32_t idesc_pv = idesc_bf16(128, D, false, true);  // V is read MN-major
@@ -282,93 +310,166 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO 1024, version, 128B swizzle
             constexpr uint32_t V_LBO = ((uint32_t)BOX_BYTES >> 4) << 16;
             constexpr uint32_t BOXU = (uint32_t)BOX_BYTES >> 4;
-            uint32_t q_lo[D / 16];
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) q_lo[kk] = (q_s >> 4) + (uint32_t)(kk >> 2) * BOXU + (uint32_t)(kk & 3) * 2u;
             auto desc = [](uint32_t lo) -> uint64_t { return ((uint64_t)DESC_HI << 32) | (uint64_t)lo; };
             uint32_t gt = 0;  // tiles issued so far (all units)
             bool ok = true;
             for (uint32_t u = 0; ok; ++u) {
                 const int slot = (int)(u & 1u);
-                if (!mbar_wait(bar(B_UFULL + slot), (u >> 1) & 1u, abort_flag)) break;
+                if (!mbar_wait(bar(C::B_UFULL + slot), (u >> 1) & 1u, abort_flag)) break;
                 const int valid = ring[slot].valid, n_it = ring[slot].n_it;
-                mbar_arrive(bar(B_UEMPTY + slot));
+                mbar_arrive(bar(C::B_UEMPTY + slot));
                 if (!valid) break;
-                if (!mbar_wait(bar(B_QFULL), u & 1u, abort_flag)) break;
+                if (!mbar_wait(bar(C::B_QFULL), u & 1u, abort_flag)) break;
                 tc_fence_after();
                 if (n_it == 0) {
-                    umma_commit(bar(B_QFREE));
+                    umma_commit(bar(C::B_QFREE));
                     continue;
                 }
-                auto issue_s = [&](int j) -> bool {
+                // S of tile j for row block blk; the first block to need a K tile waits for it, the last releases it
+                auto issue_s = [&](int j, int blk) -> bool {
                     const uint32_t t = gt + (uint32_t)j;
                     const int ks = (int)(t % KS);
-                    if (!mbar_wait(bar(B_KFULL + ks), (t / KS) & 1u, abort_flag)) return false;
-                    tc_fence_after();
+                    if (blk == 0) {
+                        if (!mbar_wait(bar(C::B_KFULL + ks), (t / KS) & 1u, abort_flag)) return false;
+                        tc_fence_after();
+                    }
                     const uint32_t k_lo = (k_s + ks * C::KV_BYTES) >> 4;
-                    const uint32_t d_t = tmem_base + S_COL + 128u * (t % SB);
+                    const uint32_t q_lo = (q_s + blk * C::QB_BYTES) >> 4;
+                    const int sb = blk * SB + (int)(t % SB);
+                    const uint32_t d_t = tmem_base + C::S_COL + 128u * (uint32_t)sb;
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        umma_ss(d_t, desc(q_lo[kk]), desc(k_lo + (uint32_t)(kk >> 2) * BOXU + (uint32_t)(kk & 3) * 2u), idesc_s,
-                                kk > 0 ? 1u : 0u);
-                    umma_commit(bar(B_SFULL + (int)(t % SB)));
-                    umma_commit(bar(B_KEMPTY + ks));  // the K tile is free once this S has been computed
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = (uint32_t)(kk >> 2) * BOXU + (uint32_t)(kk & 3) * 2u;
+                        umma_ss(d_t, desc(q_lo + off), desc(k_lo + off), idesc_s, kk > 0 ? 1u : 0u);
+                    }
+                    umma_commit(bar(C::B_SFULL + sb));
                     SR_TRACE(1, 1, t);
-                    if (j == n_it - 1) umma_commit(bar(B_QFREE));  // last S of the unit: Q may be replaced after it
+                    if (blk == NRB - 1) {
+                        umma_commit(bar(C::B_KEMPTY + ks));  // the K tile is free once its last S has been computed
+                        if (j == n_it - 1) umma_commit(bar(C::B_QFREE));  // last S of the unit: Q may be replaced
+                    }
                     return true;
                 };
-                for (int j = 0; j < SB && j < n_it && ok; ++j) ok = issue_s(j);
+                for (int j = 0; j < SB && j < n_it && ok; ++j)
+                    for (int blk = 0; blk < NRB && ok; ++blk) ok = issue_s(j, blk);
                 for (int j = 0; j < n_it && ok; ++j) {
                     const uint32_t t = gt + (uint32_t)j;
-                    const int sb = (int)(t % SB), vs = (int)(t % VS);
-                    if (!mbar_wait(bar(B_PREADY + sb), (t / SB) & 1u, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
-                    SR_TRACE(1, 2, t);
-                    if (!mbar_wait(bar(B_VFULL + vs), (t / VS) & 1u, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after();
-                    const uint32_t v_lo = ((v_s + vs * C::KV_BYTES) >> 4) | V_LBO;
-                    const uint32_t p_t = tmem_base + S_COL + 128u * (uint32_t)sb;
-                    const uint32_t acc0 = j > 0 ? 1u : 0u;
+                    const int vs = (int)(t % VS);
+                    for (int blk = 0; blk < NRB && ok; ++blk) {
+                        const int sb = blk * SB + (int)(t % SB);
+                        if (!mbar_wait(bar(C::B_PREADY + sb), (t / SB) & 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        SR_TRACE(1, 2, t);
+                        if (blk == 0 && !mbar_wait(bar(C::B_VFULL + vs), (t / VS) & 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t v_lo = ((v_s + vs * C::KV_BYTES) >> 4) | V_LBO;
+                        const uint32_t p_t = tmem_base + C::S_COL + 128u * (uint32_t)sb;
+                        const uint32_t o_t = tmem_base + C::O_COL + 128u * (uint32_t)blk;
+                        const uint32_t acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
-                    for (int kk = 0; kk < BN / 16; ++kk) {
-                        // 16 tokens per step: 2048 bytes (128 address units) down the V tile, 8 packed columns along P
-                        umma_ts(tmem_base + O_COL, p_t + 8u * kk, desc(v_lo + 128u * kk), idesc_pv, kk > 0 ? 1u : acc0);
+                        for (int kk = 0; kk < BN / 16; ++kk) {
+                            // 16 tokens per step: 2048 bytes (128 address units) down the V tile; P of tokens 0-63
+                            // sits in columns [0,32), of tokens 64-127 in columns [96,128), 8 packed columns per step
+                            const uint32_t pcol = kk < 4 ? 8u * kk : 64u + 8u * kk;
+                            umma_ts(o_t, p_t + pcol, desc(v_lo + 128u * kk), idesc_pv, kk > 0 ? 1u : acc0);
+                        }
+                        if (blk == NRB - 1) umma_commit(bar(C::B_VEMPTY + vs));
+                        umma_commit(bar(C::B_PVDONE + sb));
+                        SR_TRACE(1, 3, t);
+                        if (j + SB < n_it) ok = issue_s(j + SB, blk);  // reuses the buffer this P V has just read
                     }
-                    umma_commit(bar(B_VEMPTY + vs));
-                    umma_commit(bar(B_PVDONE + sb));
-                    SR_TRACE(1, 3, t);
-                    if (j + SB < n_it) ok = issue_s(j + SB);  // reuses the buffer this P V has just read
                 }
                 gt += (uint32_t)n_it;
             }
         }
     } else {
-        // ------------------------------------------------------------------ softmax (warps 2..9)
-        const int half = (warp - 2) >> 2;  // which 64 of a tile's 128 columns, and which D/2 of the output columns
-        const int lg = warp & 3;           // TMEM lane group of this warp
+        // ------------------------------------------------------------------ softmax (8 warps per row block)
+        const int ws = warp - 2;
+        const int blk = ws >> 3;            // row block of the unit
+        const int half = (ws & 7) >> 2;     // which 64 of a tile's 128 columns, and which D/2 output columns
+        const int lg = warp & 3;            // TMEM lane group of this warp
         const int row = lg * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
-        const uint32_t o_t = t_lane + O_COL + (uint32_t)(half * DH);
+        const uint32_t o_t = t_lane + C::O_COL + 128u * (uint32_t)blk + (uint32_t)(half * DH);
         const float sc = a.scale_log2;
+        // exchange area of this (row block, lane group), 256 bytes, touched by the group's two warps only:
+        // maxima as bf16 [2 slots][2 halves][32 lanes]; row sums as fp32 [2 halves][32 lanes]
+        volatile unsigned short *xm = reinterpret_cast<volatile unsigned short *>(xch_base + blk * 1024 + lg * 256);
+        volatile float *xl = reinterpret_cast<volatile float *>(xch_base + blk * 1024 + lg * 256);
+        volatile int *ticket = tickets + blk;
+        const int tix = (ws & 7) * 32 + lane;  // thread index within the row block
+        // Sums the partials of all chunks of one (sequence, kv head, row block); run by the 256 threads of a row
+        // block, each for its D/2 columns of its row, after the tickets showed that every chunk has been written.
+        auto merge_group = [&](int b, int hkv, int rb, int n_splits, int item0) {
+            const int gr = rb * a.rows_per_block + row;
+            if (!(row < a.rows_per_block && gr < a.rows)) return;
+            const int n = gr / G, g = gr % G;
+            __nv_bfloat16 *dst_o = a.O + (((size_t)b * N + n) * a.Hq + hkv * G + g) * D + half * DH;
+            float Mx = -INFINITY;
+            for (int s = 0; s < n_splits; ++s) {
+                const size_t pr = ((size_t)(item0 + s) * a.Hkv + hkv) * a.rows_pad + gr;
+                Mx = fmaxf(Mx, __ldcg(a.part_ml + pr * 2));
+            }
+            float lsum = 0.f;
+            for (int s = 0; s < n_splits; ++s) {
+                const size_t pr = ((size_t)(item0 + s) * a.Hkv + hkv) * a.rows_pad + gr;
+                const float ms = __ldcg(a.part_ml + pr * 2);
+                lsum += ((ms == -INFINITY) ? 0.f : ex2_approx(ms - Mx)) * __ldcg(a.part_ml + pr * 2 + 1);
+            }
+            const float invl = lsum > 0.f ? 1.0f / lsum : 0.f;
+#pragma unroll 1
+            for (int c = 0; c < DH; c += 32) {
+                float acc[32];
+#pragma unroll
+                for (int i2 = 0; i2 < 32; ++i2) acc[i2] = 0.f;
+                for (int s = 0; s < n_splits; ++s) {
+                    const size_t pr = ((size_t)(item0 + s) * a.Hkv + hkv) * a.rows_pad + gr;
+                    const float ms = __ldcg(a.part_ml + pr * 2);
+                    const float wgt = (ms == -INFINITY) ? 0.f : ex2_approx(ms - Mx) * invl;
+                    const float4 *src = reinterpret_cast<const float4 *>(a.part_o) +
+                                        ((size_t)(item0 + s) * a.Hkv + hkv) * (size_t)(D / 4) * a.rows_pad +
+                                        (size_t)((half * DH + c) / 4) * a.rows_pad + gr;
+#pragma unroll
+                    for (int i2 = 0; i2 < 8; ++i2) {
+                        const float4 x = __ldcg(src + (size_t)i2 * a.rows_pad);
+                        acc[4 * i2] += wgt * x.x;
+                        acc[4 * i2 + 1] += wgt * x.y;
+                        acc[4 * i2 + 2] += wgt * x.z;
+                        acc[4 * i2 + 3] += wgt * x.w;
+                    }
+                }
+#pragma unroll
+                for (int i2 = 0; i2 < 32; i2 += 8) {
+                    uint4 q4;
+                    q4.x = pack_bf16x2(acc[i2], acc[i2 + 1]);
+                    q4.y = pack_bf16x2(acc[i2 + 2], acc[i2 + 3]);
+                    q4.z = pack_bf16x2(acc[i2 + 4], acc[i2 + 5]);
+                    q4.w = pack_bf16x2(acc[i2 + 6], acc[i2 + 7]);
+                    *reinterpret_cast<uint4 *>(dst_o + c + i2) = q4;
+                }
+            }
+            if (a.lse && half == 0)
+                a.lse[((size_t)b * N + n) * a.Hq + hkv * G + g] = (Mx + log2f(lsum)) * 0.6931471805599453f;
+        };
         uint32_t gt = 0;  // tiles processed so far (all units)
         uint32_t use_pair = 0, use_all = 0;
-        const uint32_t pair_bar = bar(B_PAIR + lg);
+        const uint32_t pair_bar = bar(C::B_PAIR + blk * 4 + lg), all_bar = bar(C::B_ALL + blk);
         bool ok = true;
         for (uint32_t u = 0; ok; ++u) {
             const int slot = (int)(u & 1u);
-            ok = mbar_wait(bar(B_UFULL + slot), (u >> 1) & 1u, abort_flag);
+            ok = mbar_wait(bar(C::B_UFULL + slot), (u >> 1) & 1u, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const int valid = ring[slot].valid, b = ring[slot].b, hkv = ring[slot].hkv, rb = ring[slot].rb;
+            const int valid = ring[slot].valid, b = ring[slot].b, hkv = ring[slot].hkv, rb = ring[slot].rb + blk;
             const int n_splits = ring[slot].n_splits, L = ring[slot].L, t_lo = ring[slot].t_lo;
             const int n_it = ring[slot].n_it, has_tree = ring[slot].has_tree, item = ring[slot].item;
             const int item0 = ring[slot].item0;
-            mbar_arrive(bar(B_UEMPTY + slot));
+            mbar_arrive(bar(C::B_UEMPTY + slot));
             if (!valid) break;
             const int gr = rb * a.rows_per_block + row;
             const bool row_ok = row < a.rows_per_block && gr < a.rows;
@@ -376,22 +477,18 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             float m_used = -INFINITY, l = 0.f;  // l: this thread's share (its 64 columns of every tile)
             for (int j = 0; j < n_it; ++j) {
                 const uint32_t t = gt + (uint32_t)j;
-                const int sb = (int)(t % SB);
-                ok = mbar_wait(bar(B_SFULL + sb), (t / SB) & 1u, abort_flag);
+                const int sb = blk * SB + (int)(t % SB);
+                ok = mbar_wait(bar(C::B_SFULL + sb), (t / SB) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                if (lg == 0 && lane == 0) SR_TRACE(2 + half, 1, t);
-                const uint32_t s_t = t_lane + S_COL + 128u * (uint32_t)sb;
+                if ((ws & 7) == 0 && lane == 0) SR_TRACE(2 + blk, 1, t);
+                const uint32_t s_t = t_lane + C::S_COL + 128u * (uint32_t)sb;
                 const bool tree = has_tree && (j == n_it - 1);
                 // columns >= limit are outside the sequence; this thread's columns start at 64 * half
                 const int limit = (tree ? 64 : (L - (t_lo + j) * BN)) - 64 * half;
                 const bool full = !tree && limit >= 64;
-                uint32_t r0[32], r1[32];
-                tmem_ld32(s_t + 64u * half, r0);
-                tmem_ld32(s_t + 64u * half + 32u, r1);
-                tmem_ld_wait();
-                uint32_t bits0, bits1;  // admissible columns among this thread's 64
+                uint32_t bits0, bits1;  // admissible columns among this thread's 64, in two groups of 32
                 if (full) {
                     bits0 = bits1 = 0xffffffffu;
                 } else if (tree) {
@@ -401,32 +498,46 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     bits0 = limit >= 32 ? 0xffffffffu : (limit <= 0 ? 0u : ((1u << limit) - 1u));
                     bits1 = limit >= 64 ? 0xffffffffu : (limit <= 32 ? 0u : ((1u << (limit - 32)) - 1u));
                 }
+                // ---- pass 1: maximum of this thread's 64 columns
+                uint32_t r0[32], r1[32];
                 float mx0 = -INFINITY, mx1 = -INFINITY;
-                if (full) {
+                auto max_group = [&](const uint32_t(&src)[32], uint32_t bc) {
+                    if (full) {
 #pragma unroll
-                    for (int i2 = 0; i2 < 32; ++i2) {
-                        mx0 = fmaxf(mx0, __uint_as_float(r0[i2]));
-                        mx1 = fmaxf(mx1, __uint_as_float(r1[i2]));
-                    }
-                } else {
+                        for (int i2 = 0; i2 < 32; i2 += 2) {
+                            mx0 = fmaxf(mx0, __uint_as_float(src[i2]));
+                            mx1 = fmaxf(mx1, __uint_as_float(src[i2 + 1]));
+                        }
+                    } else {
 #pragma unroll
-                    for (int i2 = 0; i2 < 32; ++i2) {
-                        if ((bits0 >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(r0[i2]));
-                        if ((bits1 >> i2) & 1u) mx1 = fmaxf(mx1, __uint_as_float(r1[i2]));
+                        for (int i2 = 0; i2 < 32; ++i2)
+                            if ((bc >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(src[i2]));
                     }
+                };
+                if constexpr (NRB == 1) {
+                    tmem_ld32(s_t + 64u * half, r0);
+                    tmem_ld32(s_t + 64u * half + 32u, r1);
+                    tmem_ld_wait();
+                    max_group(r0, bits0);
+                    max_group(r1, bits1);
+                } else {  // fewer registers: one group at a time, and both are read again in pass 2
+                    tmem_ld32(s_t + 64u * half, r0);
+                    tmem_ld_wait();
+                    max_group(r0, bits0);
+                    tmem_ld32(s_t + 64u * half + 32u, r0);
+                    tmem_ld_wait();
+                    max_group(r0, bits1);
                 }
-                // exchange the partial maximum with the thread that has the row's other 64 columns.  After
-                // this rendezvous both threads have also finished reading S, so P may overwrite it.
-                // (two exchange slots, alternating, so that a fast thread's next write cannot overtake a slow read)
-                const float mine = fmaxf(mx0, mx1);
-                const int px = (int)(use_pair & 1u) * 256;
-                xch[px + half * 128 + row] = mine;
-                tc_fence_before();
+                // ---- exchange the partial maximum with the thread that has the row's other 64 columns.  It
+                //      travels as bf16: any common reference close to the true maximum will do.  Two slots,
+                //      alternating, so that a fast thread's next write cannot overtake a slow read.
+                const unsigned short mine = bf16_bits_rn(fmaxf(mx0, mx1));
+                const int px = (int)(use_pair & 1u) * 64;
+                xm[px + half * 32 + lane] = mine;
                 ok = group_sync(pair_bar, use_pair, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                tc_fence_after();
-                const float mt = fmaxf(mine, xch[px + (half ^ 1) * 128 + row]) * sc;  // scale > 0; -inf stays -inf
+                const float mt = fmaxf(bf16_bits_to_float(mine), bf16_bits_to_float(xm[px + (half ^ 1) * 32 + lane])) * sc;
                 float alpha = 1.f;
                 const bool need = mt > m_used + RESCALE_LOG2;  // also true on the first admissible tile
                 if (need) {
@@ -437,7 +548,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (__any_sync(0xffffffffu, need) && j > 0) {
                     // rows of this warp change their reference maximum: rescale this thread's half of their
                     // running outputs in TMEM.  The previous tile's P V must have landed first.
-                    ok = mbar_wait(bar(B_PVDONE + (int)((t - 1u) % SB)), ((t - 1u) / SB) & 1u, abort_flag);
+                    const int sbp = blk * SB + (int)((t - 1u) % SB);
+                    ok = mbar_wait(bar(C::B_PVDONE + sbp), ((t - 1u) / SB) & 1u, abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
@@ -453,50 +565,71 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     tmem_st_wait();
                 }
                 const float mref = (m_used == -INFINITY) ? 0.f : m_used;
-                // p = 2^(s*scale - m), packed bf16 pairs: this thread's 64 columns become 32 packed columns
+                // ---- pass 2: p = 2^(s*scale - m) as packed bf16 pairs.  Each 32-column group becomes 16 packed
+                //      columns, stored over S columns this thread has already read: [0,32) for the first thread
+                //      of the pair, [96,128) for the second.
                 float ls0 = 0.f, ls1 = 0.f;
-                uint32_t pk0[16], pk1[16];
+                auto exp_group = [&](const uint32_t(&src)[32], uint32_t bc, uint32_t dst_col) {
+                    uint32_t pk[16];
 #pragma unroll
-                for (int i2 = 0; i2 < 32; i2 += 2) {
-                    float p0 = ex2_approx(fmaf(__uint_as_float(r0[i2]), sc, -mref));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(r0[i2 + 1]), sc, -mref));
-                    float p2 = ex2_approx(fmaf(__uint_as_float(r1[i2]), sc, -mref));
-                    float p3 = ex2_approx(fmaf(__uint_as_float(r1[i2 + 1]), sc, -mref));
-                    if (!full) {
-                        p0 = ((bits0 >> i2) & 1u) ? p0 : 0.f;
-                        p1 = ((bits0 >> (i2 + 1)) & 1u) ? p1 : 0.f;
-                        p2 = ((bits1 >> i2) & 1u) ? p2 : 0.f;
-                        p3 = ((bits1 >> (i2 + 1)) & 1u) ? p3 : 0.f;
+                    for (int i2 = 0; i2 < 32; i2 += 2) {
+                        float p0 = ex2_approx(fmaf(__uint_as_float(src[i2]), sc, -mref));
+                        float p1 = ex2_approx(fmaf(__uint_as_float(src[i2 + 1]), sc, -mref));
+                        if (!full) {
+                            p0 = ((bc >> i2) & 1u) ? p0 : 0.f;
+                            p1 = ((bc >> (i2 + 1)) & 1u) ? p1 : 0.f;
+                        }
+                        ls0 += p0;
+                        ls1 += p1;
+                        pk[i2 >> 1] = pack_bf16x2(p0, p1);
                     }
-                    ls0 += p0 + p1;
-                    ls1 += p2 + p3;
-                    pk0[i2 >> 1] = pack_bf16x2(p0, p1);
-                    pk1[i2 >> 1] = pack_bf16x2(p2, p3);
+                    tmem_st16(dst_col, pk);
+                };
+                if constexpr (NRB == 1) {
+                    exp_group(r0, bits0, s_t + 96u * half);
+                    exp_group(r1, bits1, s_t + 96u * half + 16u);
+                } else {
+                    // second read of S; the second thread of a pair takes its upper group first, so that P
+                    // never lands on columns it has yet to read
+                    if (half == 0) {
+                        tmem_ld32(s_t, r0);
+                        tmem_ld_wait();
+                        exp_group(r0, bits0, s_t);
+                        tmem_ld32(s_t + 32u, r0);
+                        tmem_ld_wait();
+                        exp_group(r0, bits1, s_t + 16u);
+                    } else {
+                        tmem_ld32(s_t + 96u, r0);
+                        tmem_ld_wait();
+                        exp_group(r0, bits1, s_t + 112u);
+                        tmem_ld32(s_t + 64u, r0);
+                        tmem_ld_wait();
+                        exp_group(r0, bits0, s_t + 96u);
+                    }
                 }
-                tmem_st16(s_t + 32u * half, pk0);
-                tmem_st16(s_t + 32u * half + 16u, pk1);
                 tmem_st_wait();
                 l += ls0 + ls1;
                 tc_fence_before();
-                mbar_arrive(bar(B_PREADY + sb));
-                if (lg == 0 && lane == 0) SR_TRACE(2 + half, 2, t);
+                mbar_arrive(bar(C::B_PREADY + sb));
+                if ((ws & 7) == 0 && lane == 0) SR_TRACE(2 + blk, 2, t);
             }
-            // ---- wait for the unit's last P V (operations complete in issue order, so it covers all of them)
+            // ---- wait for the unit's last P V of this block (operations complete in issue order, so it covers all)
             if (ok && n_it > 0) {
                 const uint32_t tl = gt + (uint32_t)n_it - 1u;
-                ok = mbar_wait(bar(B_PVDONE + (int)(tl % SB)), (tl / SB) & 1u, abort_flag);
+                ok = mbar_wait(bar(C::B_PVDONE + blk * SB + (int)(tl % SB)), (tl / SB) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
             }
             gt += (uint32_t)n_it;
-            if (lg == 0 && lane == 0) SR_TRACE(2 + half, 3, u);
-            // ---- row sum = the pair's two shares
-            const int pxl = (int)(use_pair & 1u) * 256;
-            xch[pxl + half * 128 + row] = l;
+            if ((ws & 7) == 0 && lane == 0) SR_TRACE(2 + blk, 3, u);
+            // ---- row sum = the pair's two shares (fp32 through the same area: rendezvous before reusing it)
+            if (ok) ok = group_sync(pair_bar, use_pair, abort_flag);
+            xl[half * 32 + lane] = l;
             if (ok) ok = group_sync(pair_bar, use_pair, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const float lt = l + xch[pxl + (half ^ 1) * 128 + row];
+            const float lt = l + xl[(half ^ 1) * 32 + lane];
+            if (ok) ok = group_sync(pair_bar, use_pair, abort_flag);  // both have read before the area is reused
             {
                 // ---- output (or this chunk's partial): this thread's D/2 columns of its row
                 const int n = row_ok ? gr / G : 0, g = row_ok ? gr % G : 0;
@@ -505,7 +638,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 __nv_bfloat16 *dst_o = a.O + (((size_t)b * N + n) * a.Hq + hkv * G + g) * D + half * DH;
                 // partials are stored [unit][float4 column][row] so that a warp's stores are contiguous
                 const size_t pbase = ((size_t)item * a.Hkv + hkv) * (size_t)(D / 4) * a.rows_pad;
-                float4 *dst_p = reinterpret_cast<float4 *>(a.part_o) + pbase + (size_t)(half * (DH / 4)) * a.rows_pad + gr;
+                float4 *dst_p = reinterpret_cast<float4 *>(a.part_o) + pbase + (size_t)(half * (DH / 4)) * a.rows_pad +
+                                (row_ok ? gr : 0);
 #pragma unroll 1
                 for (int c = 0; c < DH; c += 32) {
                     uint32_t o[32];
@@ -545,64 +679,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                 }
                 if (!direct) {
-                    // ---- the chunk that arrives last merges all chunks of this (sequence, kv head, row block)
-                    __threadfence();
-                    bool ok3 = group_sync(bar(B_ALL), use_all, abort_flag);
-                    if (half == 0 && row == 0) *ticket = atomicAdd(a.split_counters + ((size_t)b * a.Hkv + hkv) * a.n_rb + rb, 1);
-                    ok3 = group_sync(bar(B_ALL), use_all, abort_flag) && ok3;
-                    if (ok3 && *ticket == n_splits - 1 && row_ok) {
+                    // Unless a later kernel does the merging: the chunk whose ticket comes last merges all chunks
+                    // of this (sequence, kv head, row block).  Nobody waits for anybody.
+                    if (a.merge_mode == 0) {
                         __threadfence();
-                        float Mx = -INFINITY;
-                        for (int s = 0; s < n_splits; ++s) {
-                            const size_t pr = ((size_t)(item0 + s) * a.Hkv + hkv) * a.rows_pad + gr;
-                            Mx = fmaxf(Mx, __ldcg(a.part_ml + pr * 2));
+                        bool ok3 = group_sync(all_bar, use_all, abort_flag);
+                        if (tix == 0) *ticket = atomicAdd(a.split_counters + (b * a.Hkv + hkv) * a.n_rb + rb, 1);
+                        ok3 = group_sync(all_bar, use_all, abort_flag) && ok3;
+                        if (ok3 && *ticket == n_splits - 1) {
+                            __threadfence();
+                            merge_group(b, hkv, rb, n_splits, item0);
                         }
-                        float lsum = 0.f;
-                        for (int s = 0; s < n_splits; ++s) {
-                            const size_t pr = ((size_t)(item0 + s) * a.Hkv + hkv) * a.rows_pad + gr;
-                            const float ms = __ldcg(a.part_ml + pr * 2);
-                            lsum += ((ms == -INFINITY) ? 0.f : ex2_approx(ms - Mx)) * __ldcg(a.part_ml + pr * 2 + 1);
-                        }
-                        const float invl = lsum > 0.f ? 1.0f / lsum : 0.f;
-#pragma unroll 1
-                        for (int c = 0; c < DH; c += 32) {
-                            float acc[32];
-#pragma unroll
-                            for (int i2 = 0; i2 < 32; ++i2) acc[i2] = 0.f;
-                            for (int s = 0; s < n_splits; ++s) {
-                                const size_t pr = ((size_t)(item0 + s) * a.Hkv + hkv) * a.rows_pad + gr;
-                                const float ms = __ldcg(a.part_ml + pr * 2);
-                                const float ws = (ms == -INFINITY) ? 0.f : ex2_approx(ms - Mx) * invl;
-                                const float4 *src = reinterpret_cast<const float4 *>(a.part_o) +
-                                                    ((size_t)(item0 + s) * a.Hkv + hkv) * (size_t)(D / 4) * a.rows_pad +
-                                                    (size_t)((half * DH + c) / 4) * a.rows_pad + gr;
-#pragma unroll
-                                for (int i2 = 0; i2 < 8; ++i2) {
-                                    const float4 x = __ldcg(src + (size_t)i2 * a.rows_pad);
-                                    acc[4 * i2] += ws * x.x;
-                                    acc[4 * i2 + 1] += ws * x.y;
-                                    acc[4 * i2 + 2] += ws * x.z;
-                                    acc[4 * i2 + 3] += ws * x.w;
-                                }
-                            }
-#pragma unroll
-                            for (int i2 = 0; i2 < 32; i2 += 8) {
-                                uint4 q4;
-                                q4.x = pack_bf16x2(acc[i2], acc[i2 + 1]);
-                                q4.y = pack_bf16x2(acc[i2 + 2], acc[i2 + 3]);
-                                q4.z = pack_bf16x2(acc[i2 + 4], acc[i2 + 5]);
-                                q4.w = pack_bf16x2(acc[i2 + 6], acc[i2 + 7]);
-                                *reinterpret_cast<uint4 *>(dst_o + c + i2) = q4;
-                            }
-                        }
-                        if (a.lse && half == 0)
-                            a.lse[((size_t)b * N + n) * a.Hq + hkv * G + g] = (Mx + log2f(lsum)) * 0.6931471805599453f;
                     }
                 }
             }
-            if (lg == 0 && lane == 0) SR_TRACE(2 + half, 4, u);
-            // No rendezvous is needed before the next unit: its first P V (which overwrites O) waits for the
-            // P of all 256 threads, and each of them arrives there only after it has finished reading O here.
+            if ((ws & 7) == 0 && lane == 0) SR_TRACE(2 + blk, 4, u);
+            // No rendezvous is needed before the next unit: its first P V of this block (which overwrites O)
+            // waits for the P of all 256 threads of the block, and each arrives only after reading O here.
             tc_fence_before();
         }
     }
@@ -611,17 +704,22 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0) {
-        if (*abort_flag) atomicExch(status, SPECROLL_ETIMEOUT);
+        if (*abort_flag) {
+            // status word 1: index of the barrier whose wait ran out, parity in bit 8 (diagnostic only)
+            if (atomicExch(status, SPECROLL_ETIMEOUT) == 0)
+                status[1] = (int)((((uint32_t)*abort_flag & 0xffffffu) - bar0) / 8u) | (((*abort_flag >> 24) & 1) << 8) |
+                            (int)(blockIdx.x << 16);
+        }
         // the CTA that leaves last clears the scheduling counters, so the same plan can be launched again
         __threadfence();
-        *ticket = (atomicAdd(a.work_counter + 1, 1) == (int)gridDim.x - 1) ? 1 : 0;
+        tickets[0] = (atomicAdd(a.work_counter + 1, 1) == (int)gridDim.x - 1) ? 1 : 0;
     }
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
     __syncthreads();
-    if (*ticket) {
+    if (tickets[0]) {
         const int n_split = a.B * a.Hkv * a.n_rb;
         for (int i = threadIdx.x; i < n_split; i += THREADS) a.split_counters[i] = 0;
         if (threadIdx.x == 0) {
@@ -631,9 +729,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
 }
 
-template <int D>
+template <int D, int NRB>
 static int launch_tc(const AttnArgs &a, const TopoMask &mask, long long T_kv, int32_t *status, cudaStream_t st) {
-    using C = attc::Cfg<D>;
+    using C = attc::Cfg<D, NRB>;
     CUtensorMap tmQ, tmK, tmV, tmKt, tmVt;
     int rc;
     const uint64_t tree_rows = (uint64_t)a.B * a.N;
@@ -652,10 +750,75 @@ static int launch_tc(const AttnArgs &a, const TopoMask &mask, long long T_kv, in
         int dev = 0;
         SR_CUDA_TRY(cudaGetDevice(&dev));
         SR_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-        SR_CUDA_TRY(cudaFuncSetAttribute(tree_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+        SR_CUDA_TRY(cudaFuncSetAttribute(tree_attn_tc_kernel<D, NRB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
     }
     const unsigned grid = (unsigned)(a.total_work < n_sm ? a.total_work : n_sm);
-    tree_attn_tc_kernel<D><<<grid, attc::THREADS, C::SMEM, st>>>(tmQ, tmK, tmV, tmKt, tmVt, a, mask, status);
+    tree_attn_tc_kernel<D, NRB><<<grid, C::THREADS, C::SMEM, st>>>(tmQ, tmK, tmV, tmKt, tmVt, a, mask, status);
+    SR_LAUNCH_CHECK();
+    return SPECROLL_OK;
+}
+
+// Sums the chunks of every split sequence (the plan uses this instead of merging inside the attention kernel
+// when some sequence has many chunks: there the last chunk's CTA would sit on a long chain of dependent loads).
+// grid = (chunks in work order, Hkv * n_rb, D / 32); only the block of a split sequence's first chunk works.
+// 256 threads: 128 rows x 2 groups of 4 float4 columns.
+template <int D>
+__global__ void __launch_bounds__(256) attn_merge_tc_kernel(AttnArgs a) {
+    const int4 e0 = __ldg(reinterpret_cast<const int4 *>(a.unit_tab) + 2 * (size_t)blockIdx.x);
+    const int b = e0.x, n_splits = e0.z, item0 = e0.w;
+    if (e0.y != 0 || n_splits < 2) return;
+    const int hkv = blockIdx.y / a.n_rb, rb = blockIdx.y % a.n_rb;
+    const int row = threadIdx.x & 127, cg = threadIdx.x >> 7;
+    const int gr = rb * a.rows_per_block + row;
+    if (row >= a.rows_per_block || gr >= a.rows) return;
+    const int c4 = blockIdx.z * 8 + cg * 4;  // first of this thread's 4 float4 columns
+    const size_t unit_ml = (size_t)a.Hkv * a.rows_pad, unit_o = (size_t)a.Hkv * (D / 4) * a.rows_pad;
+    const float *ml = a.part_ml + 2 * (((size_t)item0 * a.Hkv + hkv) * a.rows_pad + gr);
+    const float4 *po = reinterpret_cast<const float4 *>(a.part_o) + ((size_t)item0 * a.Hkv + hkv) * (size_t)(D / 4) * a.rows_pad +
+                       (size_t)c4 * a.rows_pad + gr;
+    float Mx = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) Mx = fmaxf(Mx, __ldcg(ml + 2 * s * unit_ml));
+    float lsum = 0.f;
+    float4 acc[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int s = 0; s < n_splits; ++s) {
+        const float ms = __ldcg(ml + 2 * s * unit_ml), ls = __ldcg(ml + 2 * s * unit_ml + 1);
+        const float wgt = (ms == -INFINITY) ? 0.f : ex2_approx(ms - Mx);
+        lsum += wgt * ls;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 x = __ldcg(po + s * unit_o + (size_t)i * a.rows_pad);
+            acc[i].x += wgt * x.x;
+            acc[i].y += wgt * x.y;
+            acc[i].z += wgt * x.z;
+            acc[i].w += wgt * x.w;
+        }
+    }
+    const float inv = lsum > 0.f ? 1.0f / lsum : 0.f;
+    const int n = gr / a.G, g = gr % a.G;
+    __nv_bfloat16 *dst = a.O + (((size_t)b * a.N + n) * a.Hq + hkv * a.G + g) * D + c4 * 4;
+    uint4 q0, q1;
+    q0.x = pack_bf16x2(acc[0].x * inv, acc[0].y * inv);
+    q0.y = pack_bf16x2(acc[0].z * inv, acc[0].w * inv);
+    q0.z = pack_bf16x2(acc[1].x * inv, acc[1].y * inv);
+    q0.w = pack_bf16x2(acc[1].z * inv, acc[1].w * inv);
+    q1.x = pack_bf16x2(acc[2].x * inv, acc[2].y * inv);
+    q1.y = pack_bf16x2(acc[2].z * inv, acc[2].w * inv);
+    q1.z = pack_bf16x2(acc[3].x * inv, acc[3].y * inv);
+    q1.w = pack_bf16x2(acc[3].z * inv, acc[3].w * inv);
+    reinterpret_cast<uint4 *>(dst)[0] = q0;
+    reinterpret_cast<uint4 *>(dst)[1] = q1;
+    if (a.lse && c4 == 0) a.lse[((size_t)b * a.N + n) * a.Hq + hkv * a.G + g] = (Mx + log2f(lsum)) * 0.6931471805599453f;
+}
+
+int launch_attn_merge_tc(const AttnArgs &a, int D, int items, cudaStream_t st) {
+    const dim3 grid((unsigned)items, (unsigned)(a.Hkv * a.n_rb), (unsigned)(D / 32));
+    if (D == 128)
+        attn_merge_tc_kernel<128><<<grid, 256, 0, st>>>(a);
+    else
+        attn_merge_tc_kernel<64><<<grid, 256, 0, st>>>(a);
     SR_LAUNCH_CHECK();
     return SPECROLL_OK;
 }
@@ -672,8 +835,12 @@ extern "C" int specroll_debug_trace_read(unsigned long long *dst, unsigned int *
 #endif
 
 int launch_attn_tc(const AttnArgs &a, const TopoMask &mask, int D, long long T_kv, int32_t *status, cudaStream_t st) {
-    if (D == 128) return launch_tc<128>(a, mask, T_kv, status, st);
-    return launch_tc<64>(a, mask, T_kv, status, st);
+    if (a.nrb == 2) {
+        if (D == 128) return launch_tc<128, 2>(a, mask, T_kv, status, st);
+        return launch_tc<64, 2>(a, mask, T_kv, status, st);
+    }
+    if (D == 128) return launch_tc<128, 1>(a, mask, T_kv, status, st);
+    return launch_tc<64, 1>(a, mask, T_kv, status, st);
 }
 
 }  // namespace specroll
