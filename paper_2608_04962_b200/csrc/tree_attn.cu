@@ -460,21 +460,14 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     p->rows = d->N * G;
     if (p->use_tc) {
         // row blocks are whole nodes: (node, head-in-group) rows of a block are one TMA box
-        // and, when one block does not hold all rows, a work unit carries two blocks that share each K/V tile
+        // The softmax of a row block costs the same whether the block is full or not, so the rows go into as
+        // few blocks as possible.  An even number of blocks is processed two per work unit (they share every
+        // K/V tile in shared memory); an odd number one per unit (the blocks' units run side by side on
+        // different SMs and the tile comes from L2 after the first read).
         int npb = 128 / G;
-        int nb = (d->N + npb - 1) / npb;
-        p->nrb = nb > 1 ? 2 : 1;
-        if (nb > 1 && (nb & 1)) {
-            ++nb;
-            if (nb > d->N) return SPECROLL_EINVAL;  // cannot happen for N >= 2 (nb is at most N)
-        }
+        const int nb = (d->N + npb - 1) / npb;
         npb = (d->N + nb - 1) / nb;  // even out the blocks
-        if ((nb - 1) * npb >= d->N) {  // evening out left the last block empty: fall back to one block per unit
-            npb = 128 / G;
-            nb = (d->N + npb - 1) / npb;
-            npb = (d->N + nb - 1) / nb;
-            p->nrb = 1;
-        }
+        p->nrb = (nb % 2 == 0) ? 2 : 1;
         p->nodes_per_block = npb;
         p->n_rb = nb;
         p->rows_per_block = npb * G;
