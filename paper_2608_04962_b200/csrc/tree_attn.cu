@@ -16,6 +16,14 @@
 #include <math.h>
 
 #include "common.cuh"
+#include <string.h>
+
+#include <algorithm>
+#include <functional>
+#include <mutex>
+#include <queue>
+#include <vector>
+
 #include "tree_attn.cuh"
 
 namespace specroll {
@@ -440,6 +448,43 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(AttnArgs a) {
 
 // ------------------------------------------------------------------------------ host side
 
+constexpr int PLAN_SMS = 148;  // SMs the chunking is planned for
+
+// Estimated finishing time, in quarter tiles, of the persistent tcgen05 kernel when sequences of the given tile
+// counts (sorted, longest first) are cut into chunks of at most ct tiles: work units go, in the order the device
+// uses, to whichever of PLAN_SMS CTAs is free first.  A unit costs its K/V tiles, one more for the tree tile of a
+// sequence's last chunk, one for the hand-over between units; a chunk of a split sequence adds one for its
+// partial, and the last one the merge when the attention kernel does it (fewer than 5 chunks per sequence).
+static long long estimate_makespan(const std::vector<int> &tiles, int ct, int copies) {
+    struct Chunk { int tps, cost; };
+    std::vector<Chunk> chunks;
+    int max_ns = 1;
+    for (int t : tiles) max_ns = std::max(max_ns, (t + ct - 1) / ct);
+    const bool merge_inline = max_ns < 5;
+    for (int t : tiles) {
+        const int ns = std::max(1, (t + ct - 1) / ct), tps = (t + ns - 1) / ns;
+        for (int s = 0; s < ns; ++s) {
+            const int lo = std::min(t, s * tps), hi = std::min(t, lo + tps);
+            int cost = 4 * (hi - lo) + 4;
+            if (s == ns - 1) cost += 4;
+            if (ns > 1) cost += 4 + ((merge_inline && s == ns - 1) ? 6 * ns : 0);
+            chunks.push_back({tps, cost});
+        }
+    }
+    std::stable_sort(chunks.begin(), chunks.end(), [](const Chunk &x, const Chunk &y) { return x.tps > y.tps; });
+    std::priority_queue<long long, std::vector<long long>, std::greater<long long>> sms;
+    for (int i = 0; i < PLAN_SMS; ++i) sms.push(0);
+    long long end = 0;
+    for (const Chunk &c : chunks)
+        for (int k = 0; k < copies; ++k) {
+            const long long t = sms.top() + c.cost;
+            sms.pop();
+            sms.push(t);
+            end = std::max(end, t);
+        }
+    return end;
+}
+
 struct AttnPlan {
     int rows, n_rb, nrb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens, nodes_per_block, n_counters;
     int merge_mode;  // tcgen05 path: 0 = split sequences are merged inside the attention kernel, 2 = by a kernel after it
@@ -447,7 +492,7 @@ struct AttnPlan {
     size_t off_status, off_items, off_sorted, off_rank, off_tab, off_counters, off_po, off_pml, total;
 };
 
-static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
+static int compute_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
     if (!d || !indptr_host || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->Hq < 1 || d->Hkv < 1 ||
         (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || (d->flags & ~(SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN)) != 0 ||
         !(d->scale > 0.f))
@@ -487,13 +532,38 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
         tiles_total += t;
         if (t > max_tiles) max_tiles = t;
     }
-    // chunk length: about four CTAs' worth of work per SM over the whole launch, at least 512
-    // tokens so that the fp32 partials stay a small fraction of the KV bytes
-    long long ctas_per_tile = (long long)d->Hkv * p->n_rb / p->nrb;
-    const int per_sm_div = p->use_tc ? 2 : 4;  // the persistent kernel balances dynamically: fewer, larger chunks
-    long long ct = (tiles_total * ctas_per_tile + 148 * per_sm_div - 1) / (148 * per_sm_div);
-    if (ct < 512 / TT) ct = 512 / TT;
-    if (ct > max_tiles) ct = max_tiles > 0 ? max_tiles : 1;
+    // chunk length.  Legacy kernel: about four CTAs' worth of work per SM over the whole launch.  tcgen05 kernel:
+    // the candidate whose estimated finishing time is lowest (the kernel hands the units, longest first, to
+    // whichever CTA is free, which a few microseconds of host time can play through).  At least 512 tokens,
+    // so that the fp32 partials stay a small fraction of the KV bytes.
+    const long long ctas_per_tile = (long long)d->Hkv * p->n_rb / p->nrb;
+    auto chunk_for = [&](int per_sm_pct) -> int {
+        long long c = (tiles_total * ctas_per_tile * 100 + (long long)PLAN_SMS * per_sm_pct - 1) / ((long long)PLAN_SMS * per_sm_pct);
+        if (c < 512 / TT) c = 512 / TT;
+        if (c > max_tiles) c = max_tiles > 0 ? max_tiles : 1;
+        return (int)c;
+    };
+    long long ct = chunk_for(p->use_tc ? 100 : 400);
+    if (p->use_tc && d->B > 0 && tiles_total * ctas_per_tile <= (1LL << 22)) {
+        std::vector<int> tiles((size_t)d->B);
+        for (int b = 0; b < d->B; ++b) tiles[(size_t)b] = (indptr_host[b + 1] - indptr_host[b] + TT - 1) / TT;
+        std::sort(tiles.begin(), tiles.end(), std::greater<int>());
+        static const int pcts[] = {75, 100, 125, 150, 200, 300};
+        long long best = -1;
+        int seen[6], n_seen = 0;
+        for (int pct : pcts) {
+            const int c = chunk_for(pct);
+            bool dup = false;
+            for (int i = 0; i < n_seen; ++i) dup |= (seen[i] == c);
+            if (dup) continue;
+            seen[n_seen++] = c;
+            const long long m = estimate_makespan(tiles, c, (int)ctas_per_tile);
+            if (best < 0 || m < best) {
+                best = m;
+                ct = c;
+            }
+        }
+    }
     p->chunk_tiles = (int)ct;
     int items = 0;
     for (int b = 0; b < d->B; ++b) {
@@ -546,6 +616,37 @@ static int launch_attn(const AttnArgs &a, const TopoMask &mask, const AttnPlan &
 }  // namespace specroll
 
 using namespace specroll;
+
+// Plans are remembered for the last few (shape, lengths) seen: every layer of a step asks for the same one.
+static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
+    struct Entry {
+        int key[7];
+        std::vector<int32_t> indptr;
+        AttnPlan plan;
+    };
+    static std::mutex mu;
+    static Entry cache[4];
+    static unsigned next = 0;
+    if (!d || !indptr_host || d->B < 0 || d->B > (1 << 24)) return compute_attn_plan(d, indptr_host, p);
+    // what the key leaves out is checked here, so that a remembered plan never answers for an invalid call
+    if ((d->flags & ~(SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN)) != 0 || !(d->scale > 0.f)) return SPECROLL_EINVAL;
+    const int key[7] = {d->B, d->N, d->Hq, d->Hkv, d->D, (int)(d->flags & SPECROLL_ATTN_LEGACY_MMA), 1};
+    const size_t n = (size_t)d->B + 1;
+    std::lock_guard<std::mutex> lock(mu);
+    for (Entry &e : cache)
+        if (memcmp(e.key, key, sizeof(key)) == 0 && e.indptr.size() == n &&
+            memcmp(e.indptr.data(), indptr_host, n * sizeof(int32_t)) == 0) {
+            *p = e.plan;
+            return SPECROLL_OK;
+        }
+    const int rc = compute_attn_plan(d, indptr_host, p);
+    if (rc != SPECROLL_OK) return rc;
+    Entry &e = cache[next++ % 4];
+    memcpy(e.key, key, sizeof(key));
+    e.indptr.assign(indptr_host, indptr_host + n);
+    e.plan = *p;
+    return SPECROLL_OK;
+}
 
 extern "C" size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *d,
                                                      const int32_t *kv_indptr_host) {
