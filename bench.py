@@ -305,21 +305,57 @@ def run_e2e(args, wl, dev, world):
     h2d = sum(t.numel() * t.element_size() for t in list(host_in.values()) + hQ + hKt + hVt)
     d2h = sum(t.numel() * t.element_size() for t in list(host_out.values()) + hO)
 
+    # Three streams: uploads, the kernels, downloads.  A kernel waits only for the upload of its own inputs, so
+    # the bulk of the bytes (target logits, needed last) crosses PCIe while the proposal and the attention layers
+    # run, and results go back while later layers compute (the link is full duplex).
+    s_cmp = torch.cuda.current_stream(dev)
+    s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    n_ev = 2 * wl.layers + 4
+    evs = [torch.cuda.Event() for _ in range(n_ev)]
+
     def step():
-        for n in names:
-            getattr(wl, n).copy_(host_in[n], non_blocking=True)
+        ev = iter(evs)
+        small = [n for n in names if n != "logits"]
+        with torch.cuda.stream(s_in):
+            for n in small:
+                getattr(wl, n).copy_(host_in[n], non_blocking=True)
+            e_small = next(ev)
+            e_small.record(s_in)
+            e_layer = []
+            for l in range(wl.layers):
+                wl.Q[l].copy_(hQ[l], non_blocking=True)
+                wl.Kt[l].copy_(hKt[l], non_blocking=True)
+                wl.Vt[l].copy_(hVt[l], non_blocking=True)
+                e = next(ev)
+                e.record(s_in)
+                e_layer.append(e)
+            wl.logits.copy_(host_in["logits"], non_blocking=True)
+            e_logits = next(ev)
+            e_logits.record(s_in)
+        s_cmp.wait_event(e_small)
         wl.propose()
-        for n in out_names_p:
-            host_out[n].copy_(wl.prop[n], non_blocking=True)
+        e = next(ev)
+        e.record(s_cmp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(e)
+            for n in out_names_p:
+                host_out[n].copy_(wl.prop[n], non_blocking=True)
         for l in range(wl.layers):
-            wl.Q[l].copy_(hQ[l], non_blocking=True)
-            wl.Kt[l].copy_(hKt[l], non_blocking=True)
-            wl.Vt[l].copy_(hVt[l], non_blocking=True)
+            s_cmp.wait_event(e_layer[l])
             wl.attn(l)
-            hO[l].copy_(wl.O[l], non_blocking=True)
+            e = next(ev)
+            e.record(s_cmp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(e)
+                hO[l].copy_(wl.O[l], non_blocking=True)
+        s_cmp.wait_event(e_logits)
         wl.verify()
-        for n in out_names_v:
-            host_out[n].copy_(wl.ver[n], non_blocking=True)
+        e = next(ev)
+        e.record(s_cmp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(e)
+            for n in out_names_v:
+                host_out[n].copy_(wl.ver[n], non_blocking=True)
 
     steps = max(2, min(args.steps, 5))
     step()
