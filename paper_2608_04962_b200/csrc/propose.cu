@@ -266,57 +266,65 @@ tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__rest
                  const int32_t *__restrict__ cand_id, const float *__restrict__ cand_logit,
                  const float *__restrict__ u_draw, int32_t *__restrict__ tree_tok,
                  uint8_t *__restrict__ tree_cand, float *__restrict__ slot_q) {
-    __shared__ double sh_w[DRAW_WARPS][SPECROLL_MAX_TOPK];
-    __shared__ uint8_t sh_pick[DRAW_WARPS][SPECROLL_MAX_NODES];
+    // Softmax weights of every head's candidates, relative to the head's largest logit, once per sequence: a
+    // child's distribution is these weights renormalised over the candidates its earlier siblings left.
+    __shared__ double sh_w[DRAW_WARPS][SPECROLL_MAX_HEADS][SPECROLL_MAX_TOPK];
+    __shared__ unsigned long long sh_taken[DRAW_WARPS][SPECROLL_MAX_NODES];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x * DRAW_WARPS + warp;
     if (b >= B) return;
     const int N = topo.N;
-    double *w = sh_w[warp];
-    uint8_t *pick = sh_pick[warp];
-    if (lane == 0) {
-        tree_tok[(size_t)b * N] = anchor[b];
-        tree_cand[(size_t)b * N] = 255;
-        slot_q[(size_t)b * N] = 1.0f;
-        pick[0] = 255;
+    for (int hd = 0; hd < K; ++hd) {
+        const float *cl = cand_logit + ((size_t)b * K + hd) * k;
+        float mxf = -INFINITY;
+        for (int j = lane; j < k; j += 32) mxf = fmaxf(mxf, cl[j]);
+        mxf = warp_max(mxf);
+        for (int j = lane; j < k; j += 32) sh_w[warp][hd][j] = exp(((double)cl[j] - (double)mxf) / T);
     }
+    for (int n = lane; n < N; n += 32) sh_taken[warp][n] = 0ull;
     __syncwarp();
+    if (lane != 0) return;
+    tree_tok[(size_t)b * N] = anchor[b];
+    tree_cand[(size_t)b * N] = 255;
+    slot_q[(size_t)b * N] = 1.0f;
     for (int n = 1; n < N; ++n) {
         const int u = topo.parent[n], hd = topo.depth[n] - 1;
-        const float *cl = cand_logit + ((size_t)b * K + hd) * k;
-        uint64_t taken = 0;
-        for (int e = 1; e < n; ++e)
-            if (topo.parent[e] == u) taken |= 1ull << pick[e];
-        // max over the remaining candidates
-        float mxf = -INFINITY;
-        for (int j = lane; j < k; j += 32)
-            if (!((taken >> j) & 1)) mxf = fmaxf(mxf, cl[j]);
-        mxf = warp_max(mxf);
-        for (int j = lane; j < k; j += 32)
-            w[j] = ((taken >> j) & 1) ? 0.0 : exp(((double)cl[j] - (double)mxf) / T);
-        __syncwarp();
-        if (lane == 0) {
-            double s = 0.0;
-            for (int j = 0; j < k; ++j) s += w[j];
-            const double uu = (double)u_draw[(size_t)b * N + n];
-            double cum = 0.0;
-            int sel = -1, last = -1;
+        double *w = sh_w[warp][hd];
+        const unsigned long long taken = sh_taken[warp][u];
+        double s = 0.0;
+        for (int j = 0; j < k; ++j)
+            if (!((taken >> j) & 1ull)) s += w[j];
+        if (!(s > 0.0)) {
+            // every remaining weight underflowed against a taken candidate's logit: take the reference among
+            // the remaining ones instead (from here on this head's weights are relative to it)
+            const float *cl = cand_logit + ((size_t)b * K + hd) * k;
+            float mxf = -INFINITY;
+            for (int j = 0; j < k; ++j)
+                if (!((taken >> j) & 1ull)) mxf = fmaxf(mxf, cl[j]);
+            s = 0.0;
             for (int j = 0; j < k; ++j) {
-                if ((taken >> j) & 1) continue;
-                last = j;
-                cum += w[j] / s;
-                if (cum > uu) {
-                    sel = j;
-                    break;
-                }
+                w[j] = ((taken >> j) & 1ull) ? 0.0 : exp(((double)cl[j] - (double)mxf) / T);
+                s += w[j];
             }
-            if (sel < 0) sel = last;
-            pick[n] = (uint8_t)sel;
-            tree_tok[(size_t)b * N + n] = cand_id[((size_t)b * K + hd) * k + sel];
-            tree_cand[(size_t)b * N + n] = (uint8_t)sel;
-            slot_q[(size_t)b * N + n] = (float)(w[sel] / s);
         }
-        __syncwarp();
+        // first remaining candidate whose cumulative probability exceeds the uniform (compared as masses)
+        const double thr = (double)u_draw[(size_t)b * N + n] * s;
+        double cum = 0.0;
+        int sel = -1, last = -1;
+        for (int j = 0; j < k; ++j) {
+            if ((taken >> j) & 1ull) continue;
+            last = j;
+            cum += w[j];
+            if (cum > thr) {
+                sel = j;
+                break;
+            }
+        }
+        if (sel < 0) sel = last;
+        sh_taken[warp][u] = taken | (1ull << sel);
+        tree_tok[(size_t)b * N + n] = cand_id[((size_t)b * K + hd) * k + sel];
+        tree_cand[(size_t)b * N + n] = (uint8_t)sel;
+        slot_q[(size_t)b * N + n] = (float)(w[sel] / s);
     }
 }
 

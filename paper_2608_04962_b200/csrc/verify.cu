@@ -22,7 +22,8 @@ namespace specroll {
 constexpr int RS_THREADS = 256;
 constexpr int RS_UNROLL = 4;
 constexpr int WALK_WARPS = 4;
-constexpr int TERM_THREADS = 1024;
+constexpr int TERM_THREADS = 512;  // two CTAs per SM
+constexpr int TERM_WARPS = TERM_THREADS / 32;
 constexpr float NEG_INF = -INFINITY;
 
 // ------------------------------------------------------------------------------ row statistics
@@ -273,11 +274,21 @@ __device__ __forceinline__ double warp_incl_scan(double v, int lane) {
     return v;
 }
 
+// The vocabulary is cut into TERM_WARPS warp segments of vpw 8-token vectors, each walked in slices of 32 vectors (one per
+// lane).  Pass 1 (all warps, independent loads) leaves the fp64 mass of every slice in shared memory; the walk's
+// residual entries then replace the plain mass of their tokens; two scans pick the segment and the slice that
+// hold u * total, and only that slice is read again to find the token.
+__host__ __device__ inline int term_slices(int V) {
+    const int nvec = V >> 3, vpw = (nvec + TERM_WARPS - 1) / TERM_WARPS;
+    return (vpw + 31) / 32;
+}
+
 __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
+    extern __shared__ double sh_slice[];  // [TERM_WARPS][n_sl]
     __shared__ double sh_seg[32];
     __shared__ double sh_ovm[SPECROLL_MAX_TOPK];
     __shared__ int32_t sh_ovid[SPECROLL_MAX_TOPK];
-    __shared__ int sh_pick[2];  // target warp, -1 if none
+    __shared__ int sh_pick[2];     // target warp, -1 if none
     __shared__ double sh_base[2];  // mass before the target warp's segment; target
 
     const int b = blockIdx.x;
@@ -288,38 +299,60 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
     const uint16_t *lg = a.logits + ((size_t)b * a.N + node) * a.V;
     const uint4 *p = reinterpret_cast<const uint4 *>(lg);
     const int nvec = a.V >> 3;
-    const int vpw = (nvec + 31) / 32;  // vectors per warp segment
-    const int v_lo = warp * vpw, v_hi = min(nvec, v_lo + vpw);
+    const int vpw = (nvec + TERM_WARPS - 1) / TERM_WARPS;  // vectors per warp segment
+    const int n_sl = (vpw + 31) / 32;                      // slices per segment
+    const int v_lo = min(nvec, warp * vpw), v_hi = min(nvec, v_lo + vpw);
 
     if (threadIdx.x < nov) {
         sh_ovm[threadIdx.x] = a.ws_ovm[(size_t)b * a.k + threadIdx.x];
         sh_ovid[threadIdx.x] = a.ws_ovid[(size_t)b * a.k + threadIdx.x];
     }
-    __syncthreads();
 
-    // level A: mass of every warp segment (plain softmax mass, then the overrides' corrections)
-    double acc = 0.0;
-    for (int i = v_lo + lane; i < v_hi; i += 32) {
-        float e[8];
-        masses8(ld_nc_v4(p + i), M, a.c, e);
+    // pass 1: plain softmax mass of every slice, eight slices' loads in flight
+    for (int s0 = 0; s0 < n_sl; s0 += 8) {
+        uint4 v[8];
 #pragma unroll
-        for (int t = 0; t < 8; ++t) acc += (double)e[t];
+        for (int q = 0; q < 8; ++q) {
+            const int i = v_lo + (s0 + q) * 32 + lane;
+            v[q] = (s0 + q < n_sl && i < v_hi) ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);  // -inf: no mass
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            float e[8];
+            masses8(v[q], M, a.c, e);
+            double acc = 0.0;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) acc += (double)e[t];
+            acc = warp_sum(acc);
+            if (lane == 0 && s0 + q < n_sl) sh_slice[warp * n_sl + s0 + q] = acc;
+        }
     }
-    for (int j = lane; j < nov; j += 32) {
-        const int t = sh_ovid[j];
-        if (t >= v_lo * 8 && t < v_hi * 8)
-            acc += sh_ovm[j] - (double)ex2_approx((bf16_bits_to_float(lg[t]) - M) * a.c);
+    __syncthreads();
+    // the walk's residual entries replace the plain mass of their tokens (at most k of them: one thread)
+    if (threadIdx.x == 0) {
+        for (int j = 0; j < nov; ++j) {
+            const int t = sh_ovid[j], vi = t >> 3;
+            const int w = min(TERM_WARPS - 1, vi / vpw), sl = (vi - w * vpw) >> 5;
+            sh_slice[w * n_sl + sl] += sh_ovm[j] - (double)ex2_approx((bf16_bits_to_float(lg[t]) - M) * a.c);
+        }
     }
-    acc = warp_sum(acc);
-    if (lane == 0) sh_seg[warp] = acc;
+    __syncthreads();
+    // segment masses
+    {
+        double acc = 0.0;
+        for (int sl = lane; sl < n_sl; sl += 32) acc += sh_slice[warp * n_sl + sl];
+        acc = warp_sum(acc);
+        if (lane == 0) sh_seg[warp] = acc;
+    }
     __syncthreads();
     if (warp == 0) {
-        const double incl = warp_incl_scan(sh_seg[lane], lane);
+        const double seg = lane < TERM_WARPS ? sh_seg[lane] : 0.0;
+        const double incl = warp_incl_scan(seg, lane);
         const double total = __shfl_sync(0xffffffffu, incl, 31);
         const double target = (double)a.u_fin[b] * total;
-        const unsigned hit = __ballot_sync(0xffffffffu, incl > target);
+        const unsigned hit = __ballot_sync(0xffffffffu, lane < TERM_WARPS && incl > target);
         const int wsel = hit ? (__ffs(hit) - 1) : -1;
-        const double base = __shfl_sync(0xffffffffu, incl - sh_seg[lane], wsel < 0 ? 0 : wsel);
+        const double base = __shfl_sync(0xffffffffu, incl - seg, wsel < 0 ? 0 : wsel);
         if (lane == 0) {
             sh_pick[0] = wsel;
             sh_base[0] = base;
@@ -346,67 +379,102 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
     }
     if (warp != wsel) return;
 
-    // levels B and C: inside the selected segment, 32 vectors at a time
+    // the slice inside the selected segment: first one whose running mass exceeds the target; if rounding made
+    // the slices fall short of the segment's own sum, the last slice with positive mass
     const double target = sh_base[1];
     double base = sh_base[0];
-    int found = -1;
-    int last_pos = -1;  // last token with positive mass seen so far in this segment (lane-local)
-    for (int i0 = v_lo; i0 < v_hi && found < 0; i0 += 32) {
-        const int i = i0 + lane;
-        double ms[8];
-        double lsum = 0.0;
-        if (i < v_hi) {
-            float e[8];
-            masses8(ld_nc_v4(p + i), M, a.c, e);
-#pragma unroll
-            for (int t = 0; t < 8; ++t) ms[t] = (double)e[t];
-            for (int j = 0; j < nov; ++j) {
-                const int off = sh_ovid[j] - i * 8;
-                if (off >= 0 && off < 8) {
-#pragma unroll
-                    for (int t = 0; t < 8; ++t)
-                        if (t == off) ms[t] = sh_ovm[j];
-                }
-            }
-#pragma unroll
-            for (int t = 0; t < 8; ++t) lsum += ms[t];
-        } else {
-#pragma unroll
-            for (int t = 0; t < 8; ++t) ms[t] = 0.0;
-        }
-        const double incl = warp_incl_scan(lsum, lane);
+    int sl_sel = -1, sl_pos = -1;
+    double base_pos = 0.0;
+    for (int c0 = 0; c0 < n_sl && sl_sel < 0; c0 += 32) {
+        const double v = (c0 + lane < n_sl) ? sh_slice[warp * n_sl + c0 + lane] : 0.0;
+        const double incl = warp_incl_scan(v, lane);
         const unsigned hit = __ballot_sync(0xffffffffu, base + incl > target);
+        const unsigned pos = __ballot_sync(0xffffffffu, v > 0.0);
+        if (pos) {
+            const int lp = 31 - __clz(pos);
+            sl_pos = c0 + lp;
+            base_pos = base + __shfl_sync(0xffffffffu, incl - v, lp);
+        }
         if (hit) {
-            const int L = __ffs(hit) - 1;
-            int tok = -1;
-            if (lane == L) {
-                double cum = base + (incl - lsum);
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    cum += ms[t];
-                    if (tok < 0 && cum > target) tok = i * 8 + t;
-                }
-                if (tok < 0) {  // scan and sequential sums disagreed in the last bit
-#pragma unroll
-                    for (int t = 0; t < 8; ++t)
-                        if (ms[t] > 0.0) tok = i * 8 + t;
-                }
-                *dst = tok;
-            }
-            found = 1;
+            const int lh = __ffs(hit) - 1;
+            sl_sel = c0 + lh;
+            base += __shfl_sync(0xffffffffu, incl - v, lh);
         } else {
             base += __shfl_sync(0xffffffffu, incl, 31);
-#pragma unroll
-            for (int t = 0; t < 8; ++t)
-                if (ms[t] > 0.0) last_pos = i * 8 + t;
         }
     }
-    if (found < 0) {
-        // the segment's scanned mass fell short of its level-A sum by rounding: last positive token
+    bool take_last = false;
+    if (sl_sel < 0) {
+        if (sl_pos < 0) {  // no mass at all in the segment (cannot be selected with positive total; keep a valid token)
+            if (lane == 0) *dst = max(0, v_hi * 8 - 1);
+            return;
+        }
+        sl_sel = sl_pos;
+        base = base_pos;
+        take_last = true;
+    }
+    // the token inside the slice
+    const int i = v_lo + sl_sel * 32 + lane;
+    double ms[8];
+    double lsum = 0.0;
+    if (i < v_hi) {
+        float e[8];
+        masses8(ld_nc_v4(p + i), M, a.c, e);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) ms[t] = (double)e[t];
+        for (int j = 0; j < nov; ++j) {
+            const int off = sh_ovid[j] - i * 8;
+            if (off >= 0 && off < 8) {
+#pragma unroll
+                for (int t = 0; t < 8; ++t)
+                    if (t == off) ms[t] = sh_ovm[j];
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) lsum += ms[t];
+    } else {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) ms[t] = 0.0;
+    }
+    const double incl = warp_incl_scan(lsum, lane);
+    const unsigned hit = take_last ? 0u : __ballot_sync(0xffffffffu, base + incl > target);
+    if (hit) {
+        const int Lh = __ffs(hit) - 1;
+        if (lane == Lh) {
+            int tok = -1;
+            double cum = base + (incl - lsum);
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                cum += ms[t];
+                if (tok < 0 && cum > target) tok = i * 8 + t;
+            }
+            if (tok < 0) {  // scan and sequential sums disagreed in the last bit
+#pragma unroll
+                for (int t = 0; t < 8; ++t)
+                    if (ms[t] > 0.0) tok = i * 8 + t;
+            }
+            *dst = tok;
+        }
+    } else {
+        // the lanes' scanned mass fell short of the slice's sum by rounding: last token with positive mass
+        int last_pos = -1;
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+            if (ms[t] > 0.0) last_pos = i * 8 + t;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, o));
-        if (lane == 0) *dst = last_pos < 0 ? v_hi * 8 - 1 : last_pos;
+        if (lane == 0) *dst = last_pos < 0 ? max(0, v_hi * 8 - 1) : last_pos;
     }
+}
+
+static int launch_terminal(const TermArgs &ta, cudaStream_t st) {
+    const size_t smem = (size_t)TERM_WARPS * term_slices(ta.V) * sizeof(double);
+    if (smem > 200 * 1024) return SPECROLL_ELIMIT;
+    if (smem > 40 * 1024)
+        SR_CUDA_TRY(cudaFuncSetAttribute(terminal_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    terminal_kernel<<<ta.B, TERM_THREADS, smem, st>>>(ta);
+    SR_LAUNCH_CHECK();
+    return SPECROLL_OK;
 }
 
 }  // namespace specroll
@@ -507,9 +575,7 @@ extern "C" int specroll_verify(const specroll_verify_desc *d, const void *logits
     ta.k = d->k;
     ta.V = d->V;
     ta.c = c;
-    terminal_kernel<<<d->B, TERM_THREADS, 0, st>>>(ta);
-    SR_LAUNCH_CHECK();
-    return SPECROLL_OK;
+    return launch_terminal(ta, st);
 }
 
 // ------------------------------------------------------------------------------ allocation-free variant
