@@ -60,9 +60,10 @@ def test_tiny_config():
 
 
 @pytest.mark.parametrize("Hq,Hkv,D,N", [(12, 2, 128, 16), (28, 4, 128, 32), (40, 8, 128, 48), (10, 2, 64, 13),
-                                        (28, 4, 128, 64), (4, 4, 128, 1), (14, 2, 64, 37)])
+                                        (28, 4, 128, 64), (4, 4, 128, 1), (14, 2, 64, 37), (14, 2, 64, 30)])
 def test_group_sizes_head_dims_and_tree_sizes(Hq, Hkv, D, N):
-    # G = 6, 7, 5, 5, 7, 1, 7; rows = 96, 224, 240, 65, 448, 1, 259 (one to four row blocks)
+    # G = 6, 7, 5, 5, 7, 1, 7, 7; rows = 96, 224, 240, 65, 448, 1, 259, 210 (one to four row blocks; an even
+    # number of blocks runs two per work unit, an odd number one per unit)
     K = 5
     w = I.scaled(I.WORKLOADS["qwen7b"], B=5, N=N, K=K, Hq=Hq, Hkv=Hkv, D=D, kv_a=300, kv_b=900)
     x = I.attn_inputs(w)
@@ -83,6 +84,18 @@ def test_ragged_lengths_empty_cache_and_split_kv():
     check(o2, O2, lse2, edge=True)
     o3, O3, lse3 = run_both(w, x, lengths=[64, 5000, 80, 64, 65, 2049, 777])
     check(o3, O3, lse3)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,N", [(10, 2, 64, 13), (14, 2, 64, 30), (12, 2, 128, 16), (28, 4, 128, 32),
+                                        (14, 2, 128, 37)])
+def test_sequences_cut_into_many_chunks(Hq, Hkv, D, N):
+    # one sequence of 5000 tokens among short ones: ten chunks, merged by the kernel that runs after the
+    # attention kernel (one, two and three row blocks, both head dims); next to it a sequence cut in two,
+    # which the attention kernel merges itself only when no sequence has five chunks or more
+    w = I.scaled(I.WORKLOADS["qwen7b"], B=4, N=N, K=5, Hq=Hq, Hkv=Hkv, D=D, kv_a=300, kv_b=900)
+    x = I.attn_inputs(w)
+    o, O, lse = run_both(w, x, lengths=[5000, 64, 700, 129])
+    check(o, O, lse)
 
 
 def test_reduced_batches_of_the_large_configs():
