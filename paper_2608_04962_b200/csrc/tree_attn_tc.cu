@@ -193,7 +193,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     ok = false;
                     break;
                 }
-                const int w = atomicAdd(a.work_counter, 1);
+                // the first unit of a CTA is its own index (no round trip before the first loads); the counter
+                // hands out the units after those
+                const int w = u == 0 ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(a.work_counter, 1);
                 volatile UnitDesc *d = ring + slot;
                 if (w >= a.total_work) {
                     d->valid = 0;
