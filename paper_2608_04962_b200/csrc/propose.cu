@@ -336,6 +336,10 @@ struct ProposePlan {
     size_t off_status, off_xhat, off_z, off_zt, off_pval, off_pid, total;
 };
 
+// head_mlp_tc.cu
+int launch_head_mlp_tc(const void *xhat, int KX, const void *A, const void *bias, const void *h, float *z, int B,
+                       int K, int d, int32_t *status, cudaStream_t st);
+
 // lm_head_tc.cu
 int launch_lm_head_tc(const void *Zt, const void *W, int M, int V, int d, int k, int n_mblocks, int n_groups,
                       int tiles_per_group, float *pval, int32_t *pid, int32_t *status, cudaStream_t st);
@@ -461,7 +465,10 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
         dd, p.KX, d->ln_eps);
     SR_LAUNCH_CHECK();
 
-    {
+    if (!(d->flags & SPECROLL_PROPOSE_LEGACY_MMA)) {
+        int rc = launch_head_mlp_tc(xhat, p.KX, A, bias, hb, z, B, K, dd, status, st);
+        if (rc) return rc;
+    } else {
         int rc = set_smem(head_mlp_kernel, HeadTile::SMEM_BYTES);
         if (rc) return rc;
         dim3 grid((dd + HeadTile::BN - 1) / HeadTile::BN, (B + HeadTile::BM - 1) / HeadTile::BM, K);

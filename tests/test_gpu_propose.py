@@ -73,9 +73,11 @@ def test_tiny_config(peaked):
 
 
 @pytest.mark.parametrize("B,K,k,d,V,N", [(37, 4, 8, 512, 3000, 16), (130, 2, 8, 256, 1288, 9),
-                                         (9, 5, 16, 320, 2056, 24), (64, 4, 8, 1536, 8192, 16)])
+                                         (9, 5, 16, 320, 2056, 24), (64, 4, 8, 1536, 8192, 16),
+                                         (300, 2, 8, 192, 1288, 9), (100, 3, 8, 448, 2048, 12)])
 def test_ragged_shapes(B, K, k, d, V, N):
-    # rows and vocabulary not multiples of the 128-wide tiles; k above the fast-path size
+    # rows, hidden size and vocabulary not multiples of the 128-wide tiles; k above the fast-path size;
+    # batches on either side of the head kernel's 64 / 128 / 256-sequence blocks, and one above 256
     w = I.scaled(I.WORKLOADS["qwen1.5b"], B=B, K=K, k=k, d=d, V=V, N=N, alpha_heads=(0.025, 0.01, 0.006, 0.004, 0.003)[:K])
     x = I.propose_inputs(w, peaked=True)
     g = gpu_propose(w, x)
