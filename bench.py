@@ -188,7 +188,7 @@ def run_ours(args, w, layers):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     D.init("nccl")
-    wl = StepWorkload(w, dev, seed=rank, layers=layers)
+    wl = StepWorkload(w, dev, seed=rank, layers=layers, paged=args.paged)
     peaks = measured_peaks()
 
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
@@ -250,6 +250,24 @@ def run_ours(args, w, layers):
                    "frac": ver_gbs / peaks["hbm_gbs"], "note": "whole call (3 launches); bytes = logits once"},
     }
 
+    if args.paged:
+        # committing the accepted paths to every layer's pages (what follows a step in an engine; outside the
+        # metric's step).  Repeatable: the workload's lengths are not advanced, the same rows are rewritten.
+        len_out = torch.empty_like(wl.kv_len)
+        st_word = torch.zeros(1, dtype=torch.int32, device=dev)
+        for _ in range(3):
+            wl.commit(len_out, st_word)
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        for _ in range(5):
+            wl.commit(len_out, st_word)
+        c1.record()
+        torch.cuda.synchronize()
+        rows = int((wl.ver["n_acc"] + 1).sum().item())
+        phases["commit"] = {"ms": c0.elapsed_time(c1) / 5, "layers": wl.layers, "tokens_appended": rows,
+                            "bytes": rows * wl.layers * 2 * 2 * w.Hkv * w.D * 2, "status": int(st_word.item()),
+                            "note": "specroll_commit_path_layers, all layers in one launch; latency-bound (a few MB)"}
+
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         one, ctok, threads = oracle_sample_step(w, args.ref_seqs, wl.layers)
@@ -266,6 +284,8 @@ def run_ours(args, w, layers):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "N": w.N, "K": w.K, "k": w.k, "d": w.d, "V": w.V, "Hq": w.Hq,
                        "Hkv": w.Hkv, "D": w.D, "layers": wl.layers, "T_kv": wl.T_kv, "temperature": w.temperature,
+                       "kv_cache": "128-token pages in a seeded random order (specroll_tree_attn_paged)" if args.paged
+                       else "contiguous ragged (specroll_tree_attn)",
                        "parallelism": f"replicas x{world} (sharded by sequence, no collective)",
                        "l2": "inputs larger than L2: per-layer KV cache, logits and W each exceed 126 MB and every "
                              "layer has its own cache"},
@@ -383,6 +403,9 @@ def main():
     ap.add_argument("--ref-seqs", type=int, default=8, help="sequences per CPU-oracle sample step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--paged", action="store_true",
+                    help="keep the KV cache in 128-token pages (specroll_tree_attn_paged) and time the commit of the "
+                         "accepted paths after the step as well (reported beside the step, not inside it)")
     args = ap.parse_args()
     from paper_2608_04962_b200 import inputs as I
     w = I.WORKLOADS[args.workload]

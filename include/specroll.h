@@ -38,7 +38,8 @@ extern "C" {
 #define SPECROLL_EWORKSPACE 3 /* workspace too small or misaligned */
 #define SPECROLL_ECUDA 4      /* a CUDA runtime call or kernel launch failed */
 #define SPECROLL_ETIMEOUT 5   /* a bounded device-side wait ran out (read from a status word) */
-#define SPECROLL_ELIMIT 6     /* problem larger than the fixed limit of an allocation-free entry point */
+#define SPECROLL_ELIMIT 6     /* problem larger than a fixed limit: of an allocation-free entry point, of the kernel a
+                                 paged cache needs, or of a sequence's own pages */
 
 #define SPECROLL_MAX_NODES 64
 #define SPECROLL_MAX_HEADS 8
@@ -148,6 +149,65 @@ int specroll_tree_attn(const specroll_attn_desc *desc, const void *Q, const void
                        const int32_t *kv_indptr_host, const void *Kt, const void *Vt,
                        const int32_t *parent_host, void *O, float *lse, void *workspace,
                        size_t workspace_bytes, void *cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * The same attention over a paged cache, and the two operations that turn one speculative step
+ * into the next (the paper lists "accepted-path KV extraction" among the contents of generation
+ * time, Sec. on the experimental protocol, and gives no formula; the layout below is this
+ * library's).
+ *
+ * A layer's cache is a pool Kp,Vp[n_pages, SPECROLL_PAGE_TOKENS, Hkv, D] bf16.  Sequence b owns the
+ * slots page_indptr[b] .. page_indptr[b+1]-1 of page_table (i32, device); slot i names the pool
+ * page that holds its tokens [128 i, 128 i + 128).  kv_len[b] tokens are valid (device and host
+ * copies with the same values); a sequence may own more pages than it fills.
+ *
+ * specroll_tree_attn_paged computes exactly what specroll_tree_attn computes on the cache that the
+ * table describes.  It needs the tcgen05 kernel: Hq/Hkv <= 128 and B <= 4096, no
+ * SPECROLL_ATTN_LEGACY_MMA (else SPECROLL_ELIMIT).  SPECROLL_ATTN_REUSE_PLAN: same lengths and same
+ * page_indptr as the call that built the plan.  Page numbers outside [0, n_pages) read as zeros.
+ */
+#define SPECROLL_PAGE_TOKENS 128
+
+size_t specroll_tree_attn_paged_workspace_bytes(const specroll_attn_desc *desc,
+                                                const int32_t *kv_len_host);
+
+int specroll_tree_attn_paged(const specroll_attn_desc *desc, const void *Q, const void *Kp,
+                             const void *Vp, int64_t n_pages, const int32_t *page_table_dev,
+                             const int32_t *page_indptr_dev, const int32_t *kv_len_dev,
+                             const int32_t *kv_len_host, const void *Kt, const void *Vt,
+                             const int32_t *parent_host, void *O, float *lse, void *workspace,
+                             size_t workspace_bytes, void *cuda_stream);
+
+/* Appends the committed path of every sequence to one layer's paged cache: the tree rows
+ * Kt,Vt[b, path_node[b,i], :, :] for i = 0 .. n_acc[b] (the anchor and the accepted nodes, as
+ * specroll_verify wrote them) go to cache positions kv_len[b] + i.  The step's last token
+ * (out_tok[b, n_acc[b]]) has no key yet: it is the next step's anchor.
+ * kv_len_out[B] (device, nullable, may be kv_len itself) receives kv_len[b] + n_acc[b] + 1; pass it
+ * with the last layer only.  A token that does not fit the sequence's own pages is not written and
+ * sets *status (device word, nullable) to SPECROLL_ELIMIT; the length is advanced regardless, so
+ * the caller must check the word before relying on the cache.  All pointers device; nothing is
+ * allocated. */
+int specroll_commit_path(int32_t B, int32_t N, int32_t K, int32_t Hkv, int32_t D, const void *Kt,
+                         const void *Vt, const int32_t *path_node, const int32_t *n_acc, void *Kp,
+                         void *Vp, int64_t n_pages, const int32_t *page_table,
+                         const int32_t *page_indptr, const int32_t *kv_len, int32_t *kv_len_out,
+                         int32_t *status, void *cuda_stream);
+
+/* The same for all layers of a model in one launch per 64 layers: Kt, Vt, Kp, Vp are HOST arrays of
+ * n_layers device pointers (read during the call, not retained); every layer shares the page table,
+ * the lengths and n_pages.  kv_len_out is written once, after the last layer's copies. */
+int specroll_commit_path_layers(int32_t B, int32_t N, int32_t K, int32_t Hkv, int32_t D,
+                                int32_t n_layers, const void *const *Kt, const void *const *Vt,
+                                const int32_t *path_node, const int32_t *n_acc, void *const *Kp,
+                                void *const *Vp, int64_t n_pages, const int32_t *page_table,
+                                const int32_t *page_indptr, const int32_t *kv_len,
+                                int32_t *kv_len_out, int32_t *status, void *cuda_stream);
+
+/* Next step's input state: h_next[b,:] = hidden[b, term_node[b], :], the target's final hidden
+ * state at the node whose distribution (or residual) produced the step's last token.
+ * hidden[B,N,d] and h_next[B,d] bf16, d % 8 == 0, term_node[B] i32 as written by specroll_verify. */
+int specroll_gather_hidden(int32_t B, int32_t N, int32_t d, const void *hidden,
+                           const int32_t *term_node, void *h_next, void *cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
  * Exact target verification (App. B.2 Eq. "nodeaccept" / "noderesidual", Algorithm "Exact

@@ -204,3 +204,62 @@ def node_budget(C_hw, B_active, N_min=1, N_max=10) -> int:
     f = lib().specroll_ref_node_budget
     f.restype = C.c_int32
     return int(f(C.c_int32(C_hw), C.c_int32(B_active), C.c_int32(N_min), C.c_int32(N_max)))
+
+
+# ----------------------------------------------------------------------------------- between two steps
+# The paper names "accepted-path KV extraction" among the contents of generation time and gives no formula; the
+# page layout is the library's.  These are written out as plain loops over tokens: a paged cache is read token
+# by token through the table, and a committed path is appended token by token.
+
+PAGE_TOKENS = 128
+
+
+def paged_to_contiguous(Kp, Vp, page_table, page_indptr, kv_len):
+    """The cache that a page table describes, as the contiguous ragged arrays of ``tree_attn``:
+    token t of sequence b lives in pool page page_table[page_indptr[b] + t // 128] at row t % 128."""
+    Kp, Vp = _as(Kp, np.uint16), _as(Vp, np.uint16)
+    page_table, page_indptr, kv_len = (_as(x, np.int32) for x in (page_table, page_indptr, kv_len))
+    B = kv_len.shape[0]
+    indptr = np.zeros(B + 1, np.int32)
+    np.cumsum(kv_len, out=indptr[1:])
+    Kc = np.zeros((int(indptr[-1]),) + Kp.shape[2:], np.uint16)
+    Vc = np.zeros_like(Kc)
+    for b in range(B):
+        for t in range(int(kv_len[b])):
+            page = int(page_table[page_indptr[b] + t // PAGE_TOKENS])
+            Kc[indptr[b] + t] = Kp[page, t % PAGE_TOKENS]
+            Vc[indptr[b] + t] = Vp[page, t % PAGE_TOKENS]
+    return Kc, Vc, indptr
+
+
+def tree_attn_paged(Q, Kp, Vp, page_table, page_indptr, kv_len, Kt, Vt, parent, scale=None, want_lse=False):
+    """Tree attention over a paged cache = tree attention over the cache the table describes."""
+    Kc, Vc, indptr = paged_to_contiguous(Kp, Vp, page_table, page_indptr, kv_len)
+    return tree_attn(Q, Kc, Vc, indptr, Kt, Vt, parent, scale=scale, want_lse=want_lse)
+
+
+def commit_path(Kt, Vt, path_node, n_acc, Kp, Vp, page_table, page_indptr, kv_len):
+    """Appends tree rows path_node[b, 0..n_acc[b]] of every sequence to its paged cache.  Returns new copies
+    (Kp, Vp, kv_len); a token that does not fit the sequence's own pages is dropped and reported in ``overflow``."""
+    Kt, Vt, Kp, Vp = (_as(x, np.uint16) for x in (Kt, Vt, Kp, Vp))
+    path_node, n_acc, page_table, page_indptr, kv_len = (
+        _as(x, np.int32) for x in (path_node, n_acc, page_table, page_indptr, kv_len))
+    Kp, Vp, new_len = Kp.copy(), Vp.copy(), kv_len.copy()
+    overflow = False
+    for b in range(kv_len.shape[0]):
+        own = int(page_indptr[b + 1] - page_indptr[b])
+        for i in range(int(n_acc[b]) + 1):
+            pos = int(kv_len[b]) + i
+            if pos // PAGE_TOKENS >= own:
+                overflow = True
+                continue
+            page = int(page_table[page_indptr[b] + pos // PAGE_TOKENS])
+            Kp[page, pos % PAGE_TOKENS] = Kt[b, path_node[b, i]]
+            Vp[page, pos % PAGE_TOKENS] = Vt[b, path_node[b, i]]
+        new_len[b] = kv_len[b] + n_acc[b] + 1
+    return {"Kp": Kp, "Vp": Vp, "kv_len": new_len, "overflow": overflow}
+
+
+def gather_hidden(hidden, term_node):
+    hidden, term_node = _as(hidden, np.uint16), _as(term_node, np.int32)
+    return np.stack([hidden[b, term_node[b]] for b in range(hidden.shape[0])])

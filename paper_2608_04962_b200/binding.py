@@ -22,12 +22,15 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
            "specroll_propose_workspace_bytes", "specroll_propose", "specroll_workspace_status",
            "specroll_tree_draw",
            "specroll_tree_attn_workspace_bytes", "specroll_tree_attn",
+           "specroll_tree_attn_paged_workspace_bytes", "specroll_tree_attn_paged",
+           "specroll_commit_path", "specroll_commit_path_layers", "specroll_gather_hidden",
            "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static")
 
 
 PROPOSE_LEGACY_MMA = 1
 ATTN_LEGACY_MMA = 1
 ATTN_REUSE_PLAN = 2
+PAGE_TOKENS = 128
 
 
 class SpecrollError(RuntimeError):
@@ -66,11 +69,11 @@ def lib():
         l.specroll_node_budget.restype = C.c_int32
         l.specroll_node_budget.argtypes = [C.c_int32] * 4
         for n in ("specroll_propose_workspace_bytes", "specroll_verify_workspace_bytes",
-                  "specroll_tree_attn_workspace_bytes"):
+                  "specroll_tree_attn_workspace_bytes", "specroll_tree_attn_paged_workspace_bytes"):
             getattr(l, n).restype = C.c_size_t
         for n in ("specroll_propose", "specroll_workspace_status", "specroll_tree_draw", "specroll_tree_attn",
-                  "specroll_verify",
-                  "specroll_verify_static"):
+                  "specroll_verify", "specroll_verify_static", "specroll_tree_attn_paged", "specroll_commit_path",
+                  "specroll_commit_path_layers", "specroll_gather_hidden"):
             getattr(l, n).restype = C.c_int
         _lib = l
     return _lib
@@ -237,6 +240,104 @@ def tree_attn(Q, Kc, Vc, kv_indptr_dev, kv_indptr_host, Kt, Vt, parent, scale=No
         _check(lib().specroll_workspace_status(C.c_void_p(workspace.data_ptr()), _stream()),
                "specroll_workspace_status")
     return (out, lse) if want_lse else out
+
+
+def tree_attn_paged_workspace_bytes(B, N, Hq, Hkv, D, kv_len_host, scale=None) -> int:
+    kl = _host_i32(kv_len_host, "kv_len_host")
+    desc = AttnDesc(B, N, Hq, Hkv, D, scale if scale is not None else 1.0 / float(np.sqrt(D)), 0)
+    return int(lib().specroll_tree_attn_paged_workspace_bytes(C.byref(desc), kl.ctypes.data_as(C.c_void_p)))
+
+
+def tree_attn_paged(Q, Kp, Vp, page_table, page_indptr, kv_len_dev, kv_len_host, Kt, Vt, parent, scale=None,
+                    want_lse=False, workspace=None, out=None, lse=None, flags: int = 0, check_status: bool = False):
+    """specroll_tree_attn_paged.  Kp, Vp: [n_pages, 128, Hkv, D]; page_table, page_indptr, kv_len_dev: device
+    int32; kv_len_host: host copy of the lengths.  Returns O (and lse when asked)."""
+    parent = _host_i32(parent, "parent")
+    kl = _host_i32(kv_len_host, "kv_len_host")
+    B, N, Hq, D = Q.shape
+    Hkv = Kt.shape[2]
+    if kl.shape[0] != B or tuple(Kt.shape) != (B, N, Hkv, D) or tuple(Vt.shape) != (B, N, Hkv, D):
+        raise SpecrollError("tree_attn_paged: inconsistent shapes")
+    if tuple(Kp.shape[1:]) != (PAGE_TOKENS, Hkv, D) or Vp.shape != Kp.shape:
+        raise SpecrollError("tree_attn_paged: page pool must be [n_pages, 128, Hkv, D]")
+    if page_indptr.numel() != B + 1 or kv_len_dev.numel() != B:
+        raise SpecrollError("tree_attn_paged: page_indptr / kv_len_dev sizes")
+    if scale is None:
+        scale = 1.0 / float(np.sqrt(D))
+    desc = AttnDesc(B, N, Hq, Hkv, D, scale, flags)
+    dev = Q.device
+    if out is None:
+        out = torch.empty((B, N, Hq, D), dtype=torch.bfloat16, device=dev)
+    if want_lse and lse is None:
+        lse = torch.empty((B, N, Hq), dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = _workspace(lib().specroll_tree_attn_paged_workspace_bytes(
+            C.byref(desc), kl.ctypes.data_as(C.c_void_p)), dev)
+    bf = torch.bfloat16
+    rc = lib().specroll_tree_attn_paged(
+        C.byref(desc), _dev(Q, bf, "Q"), _dev(Kp, bf, "Kp"), _dev(Vp, bf, "Vp"), C.c_int64(Kp.shape[0]),
+        _dev(page_table, torch.int32, "page_table"), _dev(page_indptr, torch.int32, "page_indptr"),
+        _dev(kv_len_dev, torch.int32, "kv_len_dev"), kl.ctypes.data_as(C.c_void_p),
+        _dev(Kt, bf, "Kt"), _dev(Vt, bf, "Vt"), parent.ctypes.data_as(C.c_void_p),
+        _dev(out, bf, "O"), _dev(lse, torch.float32, "lse"), C.c_void_p(workspace.data_ptr()),
+        C.c_size_t(workspace.numel()), _stream())
+    _check(rc, "specroll_tree_attn_paged")
+    if check_status:
+        _check(lib().specroll_workspace_status(C.c_void_p(workspace.data_ptr()), _stream()),
+               "specroll_workspace_status")
+    return (out, lse) if want_lse else out
+
+
+def commit_path(Kt, Vt, path_node, n_acc, Kp, Vp, page_table, page_indptr, kv_len, kv_len_out=None, status=None):
+    """specroll_commit_path: appends the committed path's tree rows to one layer's paged cache (in place)."""
+    B, N, Hkv, D = Kt.shape
+    K = path_node.shape[1] - 1
+    bf = torch.bfloat16
+    rc = lib().specroll_commit_path(
+        B, N, K, Hkv, D, _dev(Kt, bf, "Kt"), _dev(Vt, bf, "Vt"), _dev(path_node, torch.int32, "path_node"),
+        _dev(n_acc, torch.int32, "n_acc"), _dev(Kp, bf, "Kp"), _dev(Vp, bf, "Vp"), C.c_int64(Kp.shape[0]),
+        _dev(page_table, torch.int32, "page_table"), _dev(page_indptr, torch.int32, "page_indptr"),
+        _dev(kv_len, torch.int32, "kv_len"), _dev(kv_len_out, torch.int32, "kv_len_out"),
+        _dev(status, torch.int32, "status"), _stream())
+    _check(rc, "specroll_commit_path")
+
+
+def commit_path_layers(Kt, Vt, path_node, n_acc, Kp, Vp, page_table, page_indptr, kv_len, kv_len_out=None,
+                       status=None):
+    """specroll_commit_path_layers: Kt, Vt, Kp, Vp are lists with one tensor per layer."""
+    n = len(Kt)
+    if not (len(Vt) == len(Kp) == len(Vp) == n) or n == 0:
+        raise SpecrollError("commit_path_layers: one tensor per layer in each list")
+    B, N, Hkv, D = Kt[0].shape
+    K = path_node.shape[1] - 1
+    bf = torch.bfloat16
+    arr = C.c_void_p * n
+    ptrs = [arr(*[_dev(t, bf, name).value for t in ts]) for ts, name in ((Kt, "Kt"), (Vt, "Vt"), (Kp, "Kp"), (Vp, "Vp"))]
+    for ts in (Kt, Vt):
+        if any(tuple(t.shape) != (B, N, Hkv, D) for t in ts):
+            raise SpecrollError("commit_path_layers: tree K/V shapes differ between layers")
+    for ts in (Kp, Vp):
+        if any(tuple(t.shape) != tuple(Kp[0].shape) for t in ts):
+            raise SpecrollError("commit_path_layers: page pools differ between layers")
+    rc = lib().specroll_commit_path_layers(
+        B, N, K, Hkv, D, n, ptrs[0], ptrs[1], _dev(path_node, torch.int32, "path_node"),
+        _dev(n_acc, torch.int32, "n_acc"), ptrs[2], ptrs[3], C.c_int64(Kp[0].shape[0]),
+        _dev(page_table, torch.int32, "page_table"), _dev(page_indptr, torch.int32, "page_indptr"),
+        _dev(kv_len, torch.int32, "kv_len"), _dev(kv_len_out, torch.int32, "kv_len_out"),
+        _dev(status, torch.int32, "status"), _stream())
+    _check(rc, "specroll_commit_path_layers")
+
+
+def gather_hidden(hidden, term_node, out=None):
+    """specroll_gather_hidden: hidden[B,N,d] bf16, term_node[B] -> h_next[B,d]."""
+    B, N, d = hidden.shape
+    if out is None:
+        out = torch.empty((B, d), dtype=torch.bfloat16, device=hidden.device)
+    rc = lib().specroll_gather_hidden(B, N, d, _dev(hidden, torch.bfloat16, "hidden"),
+                                      _dev(term_node, torch.int32, "term_node"), _dev(out, torch.bfloat16, "h_next"),
+                                      _stream())
+    _check(rc, "specroll_gather_hidden")
+    return out
 
 
 # ----------------------------------------------------------------------------------- verify

@@ -84,7 +84,8 @@ __device__ int block_exclusive_scan(int *data, int n, int *warp_tot) {
 //                   exclusive prefix of ns in that order                  (tcgen05 kernel, B <= PREP_MAX_B)
 // Also clears the status word and the scheduling counters.
 __global__ void __launch_bounds__(PREP_THREADS)
-attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles, int tile_tokens,
+attn_prep_kernel(const int32_t *__restrict__ kv_indptr, const int32_t *__restrict__ kv_len,
+                 const int32_t *__restrict__ page_indptr, int B, int chunk_tiles, int tile_tokens,
                  int32_t *__restrict__ item_start, int32_t *__restrict__ sorted_start,
                  int32_t *__restrict__ seq_at_rank, int32_t *__restrict__ unit_tab, int32_t *__restrict__ status,
                  int32_t *__restrict__ counters, int n_counters) {
@@ -101,7 +102,7 @@ attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles, 
             int acc = 0;
             for (int b = 0; b < B; ++b) {
                 item_start[b] = acc;
-                const int L = kv_indptr[b + 1] - kv_indptr[b];
+                const int L = kv_len ? kv_len[b] : kv_indptr[b + 1] - kv_indptr[b];
                 const int tiles = (L + tile_tokens - 1) / tile_tokens;
                 const int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
                 acc += ns < 1 ? 1 : ns;
@@ -111,7 +112,7 @@ attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles, 
         return;
     }
     for (int b = t; b < B; b += PREP_THREADS) {
-        const int L = kv_indptr[b + 1] - kv_indptr[b];
+        const int L = kv_len ? kv_len[b] : kv_indptr[b + 1] - kv_indptr[b];
         const int tiles = (L + tile_tokens - 1) / tile_tokens;
         int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
         if (ns < 1) ns = 1;
@@ -152,7 +153,9 @@ attn_prep_kernel(const int32_t *__restrict__ kv_indptr, int B, int chunk_tiles, 
                 r += (co > c) || (co == c && o < b);
             }
             const int ns = (int)sh_ns[b];
-            const int kv0 = kv_indptr[b], L = kv_indptr[b + 1] - kv0;
+            // contiguous cache: first token and length; paged cache: first slot of the page table and length
+            const int kv0 = kv_len ? page_indptr[b] : kv_indptr[b];
+            const int L = kv_len ? kv_len[b] : kv_indptr[b + 1] - kv0;
             const int first = item_start[b];  // written by this block; visible after the barriers above
             int4 *dst = reinterpret_cast<int4 *>(unit_tab) + 2 * (size_t)sh_tmp[r];
             for (int s = 0; s < ns; ++s) {
@@ -655,14 +658,20 @@ extern "C" size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *d
     return p.total;
 }
 
-extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, const void *Kc, const void *Vc,
-                                  const int32_t *kv_indptr_dev, const int32_t *kv_indptr_host, const void *Kt,
-                                  const void *Vt, const int32_t *parent_host, void *O, float *lse,
-                                  void *workspace, size_t workspace_bytes, void *cuda_stream) {
+// Common body of the two entry points.  Contiguous cache: kv_indptr_dev, T_kv = cached tokens.  Paged cache:
+// kv_len_dev, page_indptr_dev, page_table_dev, T_kv = tokens in the page pool.  indptr_host is the (derived)
+// prefix of the host lengths either way.
+static int run_tree_attn(const specroll_attn_desc *d, const void *Q, const void *Kc, const void *Vc, long long T_kv,
+                         const int32_t *kv_indptr_dev, const int32_t *kv_len_dev, const int32_t *page_indptr_dev,
+                         const int32_t *page_table_dev, const int32_t *indptr_host, const void *Kt, const void *Vt,
+                         const int32_t *parent_host, void *O, float *lse, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream) {
+    const bool paged = page_table_dev != nullptr;
     AttnPlan p;
-    if (make_attn_plan(d, kv_indptr_host, &p) != SPECROLL_OK) return SPECROLL_EINVAL;
-    if (!Q || !kv_indptr_dev || !Kt || !Vt || !O) return SPECROLL_EINVAL;
-    const long long T_kv = kv_indptr_host[d->B] - kv_indptr_host[0];
+    if (make_attn_plan(d, indptr_host, &p) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (!Q || !Kt || !Vt || !O) return SPECROLL_EINVAL;
+    if (paged ? (!kv_len_dev || !page_indptr_dev) : !kv_indptr_dev) return SPECROLL_EINVAL;
+    if (paged && !p.use_tc) return SPECROLL_ELIMIT;  // the mma.sync kernel reads a contiguous cache only
     if (T_kv > 0 && (!Kc || !Vc)) return SPECROLL_EINVAL;
     Topo topo;
     TopoMask mask;
@@ -681,6 +690,7 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
     a.Kt = static_cast<const __nv_bfloat16 *>(Kt);
     a.Vt = static_cast<const __nv_bfloat16 *>(Vt);
     a.kv_indptr = kv_indptr_dev;
+    a.page_table = page_table_dev;
     a.item_start = reinterpret_cast<int32_t *>(ws + p.off_items);
     a.O = static_cast<__nv_bfloat16 *>(O);
     a.lse = lse;
@@ -714,7 +724,8 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
     a.nodes_per_block = p.nodes_per_block;
     if (!(p.use_tc && (d->flags & SPECROLL_ATTN_REUSE_PLAN))) {
         // (the tcgen05 kernel leaves its scheduling counters cleared, so a kept plan can be run again as is)
-        attn_prep_kernel<<<1, PREP_THREADS, 0, st>>>(kv_indptr_dev, d->B, p.chunk_tiles, p.tile_tokens,
+        attn_prep_kernel<<<1, PREP_THREADS, 0, st>>>(kv_indptr_dev, paged ? kv_len_dev : nullptr, page_indptr_dev, d->B,
+                                                     p.chunk_tiles, p.tile_tokens,
                                                      reinterpret_cast<int32_t *>(ws + p.off_items),
                                                      p.use_tc ? sorted_start : nullptr, seq_at_rank,
                                                      p.use_tc ? unit_tab : nullptr, status, counters, p.n_counters);
@@ -728,4 +739,50 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
     }
     if (d->D == 128) return launch_attn<128>(a, mask, p, d->Hkv, n_out, st);
     return launch_attn<64>(a, mask, p, d->Hkv, n_out, st);
+}
+
+extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, const void *Kc, const void *Vc,
+                                  const int32_t *kv_indptr_dev, const int32_t *kv_indptr_host, const void *Kt,
+                                  const void *Vt, const int32_t *parent_host, void *O, float *lse,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!d || !kv_indptr_host || d->B < 0) return SPECROLL_EINVAL;
+    const long long T_kv = (long long)kv_indptr_host[d->B] - kv_indptr_host[0];
+    return run_tree_attn(d, Q, Kc, Vc, T_kv, kv_indptr_dev, nullptr, nullptr, nullptr, kv_indptr_host, Kt, Vt,
+                         parent_host, O, lse, workspace, workspace_bytes, cuda_stream);
+}
+
+// Prefix of the host lengths: what the planner takes.  False if a length is negative.
+static bool lengths_to_indptr(const int32_t *kv_len_host, int B, std::vector<int32_t> *ip) {
+    ip->assign((size_t)B + 1, 0);
+    long long acc = 0;
+    for (int b = 0; b < B; ++b) {
+        if (kv_len_host[b] < 0) return false;
+        acc += kv_len_host[b];
+        if (acc > 0x7fffffffLL) return false;
+        (*ip)[(size_t)b + 1] = (int32_t)acc;
+    }
+    return true;
+}
+
+extern "C" size_t specroll_tree_attn_paged_workspace_bytes(const specroll_attn_desc *d, const int32_t *kv_len_host) {
+    if (!d || !kv_len_host || d->B < 0 || d->B > (1 << 24)) return 0;
+    std::vector<int32_t> ip;
+    if (!lengths_to_indptr(kv_len_host, d->B, &ip)) return 0;
+    AttnPlan p;
+    if (make_attn_plan(d, ip.data(), &p) != SPECROLL_OK || !p.use_tc) return 0;
+    return p.total;
+}
+
+extern "C" int specroll_tree_attn_paged(const specroll_attn_desc *d, const void *Q, const void *Kp, const void *Vp,
+                                        int64_t n_pages, const int32_t *page_table_dev,
+                                        const int32_t *page_indptr_dev, const int32_t *kv_len_dev,
+                                        const int32_t *kv_len_host, const void *Kt, const void *Vt,
+                                        const int32_t *parent_host, void *O, float *lse, void *workspace,
+                                        size_t workspace_bytes, void *cuda_stream) {
+    if (!d || !kv_len_host || d->B < 0 || d->B > (1 << 24) || n_pages < 0 || n_pages > (1LL << 24) || !page_table_dev)
+        return SPECROLL_EINVAL;
+    std::vector<int32_t> ip;
+    if (!lengths_to_indptr(kv_len_host, d->B, &ip)) return SPECROLL_EINVAL;
+    return run_tree_attn(d, Q, Kp, Vp, n_pages * SPECROLL_PAGE_TOKENS, nullptr, kv_len_dev, page_indptr_dev,
+                         page_table_dev, ip.data(), Kt, Vt, parent_host, O, lse, workspace, workspace_bytes, cuda_stream);
 }

@@ -25,6 +25,9 @@ struct AttnArgs {
     int32_t total_work;           // items * Hkv * n_rb / nrb
     int32_t nodes_per_block;      // rows_per_block = nodes_per_block * G
     int32_t nrb;                  // row blocks per work unit: 1, or 2 (then n_rb is even)
+    // paged cache (tcgen05 kernel only): pool page of every 128-token tile; a chunk table row then carries the
+    // sequence's first slot in this table instead of its first token
+    const int32_t *page_table;
     int32_t merge_mode;           // chunks of a split sequence are merged 0: by the CTA that finishes last; 2: by a later kernel
 };
 

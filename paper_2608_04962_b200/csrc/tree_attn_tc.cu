@@ -242,15 +242,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     for (int bx = 0; bx < C::NBOX; ++bx)
                         tma_load_3d(q_s + blk * C::QB_BYTES + bx * BOX_BYTES, &tmQ, bx * 64, hkv * G,
                                     b * N + (rb + blk) * a.nodes_per_block, bar(C::B_QFULL));
-                // ---- K tiles, each followed by the V tile from two tiles back
+                // ---- K tiles, each followed by the V tile from two tiles back.  Paged cache: kv0 is the sequence's
+                //      first slot in the page table and a tile is one pool page; page numbers are fetched two
+                //      tiles ahead of their use, under the wait for a free stage.
+                const int n_kv = t_hi - t_lo;
+                const int32_t *pt = a.page_table ? a.page_table + kv0 + t_lo : nullptr;
+                int pg0 = (pt && n_kv > 0) ? __ldg(pt) : 0, pg1 = (pt && n_kv > 1) ? __ldg(pt + 1) : 0;
                 for (int it = 0; it < n_it && ok; ++it) {
+                    const int pg2 = (pt && it + 2 < n_kv) ? __ldg(pt + it + 2) : 0;
                     const int s = (int)(kt % KS);
                     if (!mbar_wait(bar(C::B_KEMPTY + s), ((kt / KS) & 1u) ^ 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
                     const bool tree = has_tree && (it == n_it - 1);
-                    const int tok = tree ? b * N : kv0 + (t_lo + it) * BN;
+                    const int tok = tree ? b * N : (pt ? pg0 * BN : kv0 + (t_lo + it) * BN);
+                    pg0 = pg1;
+                    pg1 = pg2;
                     const CUtensorMap *mk = tree ? &tmKt : &tmK;
                     const uint32_t dst = k_s + s * C::KV_BYTES;
                     mbar_arrive_expect_tx(bar(C::B_KFULL + s), C::KV_BYTES);

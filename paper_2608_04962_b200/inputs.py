@@ -294,3 +294,32 @@ def synthetic_candidates(w: Workload) -> Tuple[np.ndarray, np.ndarray]:
             ids[b, hd] = g.choice(w.V, size=w.k, replace=False)
     lg = -np.sort(-(g.standard_normal(size=(w.B, w.K, w.k), dtype=np.float32) * np.float32(1.5)), axis=-1)
     return ids, np.ascontiguousarray(lg, dtype=np.float32)
+
+
+def paged_cache(Kc, Vc, kv_indptr, spare_tokens: int, seed: int):
+    """Scatters a contiguous ragged cache into a pool of 128-token pages in a seeded random page order.
+
+    Every sequence gets room for ``spare_tokens`` more tokens; the pool has a few unused pages and unused rows
+    hold a bit pattern that is not zero, so that a kernel reading beyond a sequence's length would be noticed.
+    Returns Kp, Vp [n_pages, 128, Hkv, D] (uint16 bit patterns), page_table, page_indptr, kv_len (int32)."""
+    PAGE = 128
+    kv_indptr = np.asarray(kv_indptr, np.int64)
+    B = kv_indptr.shape[0] - 1
+    kv_len = (kv_indptr[1:] - kv_indptr[:-1]).astype(np.int32)
+    own = (kv_len.astype(np.int64) + spare_tokens + PAGE - 1) // PAGE
+    page_indptr = np.zeros(B + 1, np.int32)
+    np.cumsum(own, out=page_indptr[1:])
+    n_pages = int(page_indptr[-1]) + 3
+    g = rng(seed)
+    page_table = g.permutation(n_pages)[: int(page_indptr[-1])].astype(np.int32)
+    Kp = np.full((n_pages, PAGE) + Kc.shape[1:], 0x7F00, np.uint16)   # bf16 2^127: poisons any sum it enters
+    Vp = np.full((n_pages, PAGE) + Vc.shape[1:], 0x7F00, np.uint16)
+    for b in range(B):
+        for i in range(int((kv_len[b] + PAGE - 1) // PAGE)):
+            lo = int(kv_indptr[b]) + i * PAGE
+            hi = min(int(kv_indptr[b + 1]), lo + PAGE)
+            page = int(page_table[page_indptr[b] + i])
+            Kp[page, : hi - lo] = Kc[lo:hi]
+            Vp[page, : hi - lo] = Vc[lo:hi]
+    return Kp, Vp, page_table, page_indptr, kv_len
+

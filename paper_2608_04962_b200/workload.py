@@ -32,8 +32,9 @@ def _randn_bf16(gen, shape, std, device):
 class StepWorkload:
     """All tensors of one step for workload ``w`` on ``device`` (seed offset for replicas)."""
 
-    def __init__(self, w: I.Workload, device, seed: int = 0, layers: int | None = None):
+    def __init__(self, w: I.Workload, device, seed: int = 0, layers: int | None = None, paged: bool = False):
         self.w = w
+        self.paged = bool(paged)
         self.device = device
         self.layers = int(layers if layers is not None else w.layers)
         gen = torch.Generator(device=device)
@@ -73,11 +74,37 @@ class StepWorkload:
             self.Vt.append(_randn_bf16(gen, (B, N, w.Hkv, w.D), 1.0, device))
         self.O = [torch.empty((B, N, w.Hq, w.D), dtype=torch.bfloat16, device=device)
                   for _ in range(self.layers)]
+        if self.paged:
+            # the same caches scattered into pools of 128-token pages in a seeded random page order, with room
+            # for one more committed path per sequence; the contiguous copies are dropped
+            PAGE = S.PAGE_TOKENS
+            own = (L.astype(np.int64) + (K + 1) + PAGE - 1) // PAGE
+            pi = np.zeros(B + 1, np.int32)
+            np.cumsum(own, out=pi[1:])
+            self.n_pages = int(pi[-1]) + 3
+            pt = I.rng(1000 * w.cfg_id + 31 + seed).permutation(self.n_pages)[: int(pi[-1])].astype(np.int32)
+            tok = np.arange(self.T_kv, dtype=np.int64)
+            seq = np.repeat(np.arange(B), L)
+            t_in = tok - self.kv_indptr_host[:-1].astype(np.int64)[seq]
+            flat = pt[pi[:-1].astype(np.int64)[seq] + t_in // PAGE].astype(np.int64) * PAGE + t_in % PAGE
+            flat_d = torch.from_numpy(flat).to(device)
+            self.page_table = torch.from_numpy(pt).to(device)
+            self.page_indptr = torch.from_numpy(pi).to(device)
+            self.kv_len_host = L.astype(np.int32)
+            self.kv_len = torch.from_numpy(self.kv_len_host).to(device)
+            self.Kp, self.Vp = [], []
+            for l in range(self.layers):
+                for src, dst in ((self.Kc, self.Kp), (self.Vc, self.Vp)):
+                    pool = torch.zeros((self.n_pages * PAGE, w.Hkv, w.D), dtype=torch.bfloat16, device=device)
+                    pool[flat_d] = src[l]
+                    dst.append(pool.view(self.n_pages, PAGE, w.Hkv, w.D))
+                    src[l] = None
         # workspaces and outputs, allocated once
         self.ws_propose = torch.empty(S.propose_workspace_bytes(B, N, K, k, d, V, w.temperature),
                                       dtype=torch.uint8, device=device)
-        self.ws_attn = torch.empty(S.tree_attn_workspace_bytes(B, N, w.Hq, w.Hkv, w.D, self.kv_indptr_host),
-                                   dtype=torch.uint8, device=device)
+        ws_bytes = (S.tree_attn_paged_workspace_bytes(B, N, w.Hq, w.Hkv, w.D, self.kv_len_host) if self.paged else
+                    S.tree_attn_workspace_bytes(B, N, w.Hq, w.Hkv, w.D, self.kv_indptr_host))
+        self.ws_attn = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
         self.ws_verify = torch.empty(S.verify_workspace_bytes(B, N, K, k, V, w.temperature),
                                      dtype=torch.uint8, device=device)
         self.prop = None
@@ -114,9 +141,20 @@ class StepWorkload:
 
     def attn(self, layer: int):
         # every layer of a step sees the same KV lengths: layers after the first reuse the work plan
+        if self.paged:
+            return S.tree_attn_paged(self.Q[layer], self.Kp[layer], self.Vp[layer], self.page_table, self.page_indptr,
+                                     self.kv_len, self.kv_len_host, self.Kt[layer], self.Vt[layer], self.parent,
+                                     workspace=self.ws_attn, out=self.O[layer],
+                                     flags=S.ATTN_REUSE_PLAN if layer > 0 else 0)
         return S.tree_attn(self.Q[layer], self.Kc[layer], self.Vc[layer], self.kv_indptr, self.kv_indptr_host,
                            self.Kt[layer], self.Vt[layer], self.parent, workspace=self.ws_attn,
                            out=self.O[layer], flags=S.ATTN_REUSE_PLAN if layer > 0 else 0)
+
+    def commit(self, kv_len_out=None, status=None):
+        """Appends the committed paths of the last verification to every layer's paged cache (the workload's
+        own lengths are left alone, so that the step can be repeated)."""
+        S.commit_path_layers(self.Kt, self.Vt, self.ver["path_node"], self.ver["n_acc"], self.Kp, self.Vp,
+                             self.page_table, self.page_indptr, self.kv_len, kv_len_out=kv_len_out, status=status)
 
     def verify(self):
         p = self.prop
