@@ -246,6 +246,27 @@ int specroll_verify(const specroll_verify_desc *desc, const void *logits,
                     float *row_sum, float *min_margin, void *workspace, size_t workspace_bytes,
                     void *cuda_stream);
 
+/* The same verification against nucleus-truncated target distributions (App. "Implementation and
+ * Reproducibility Details": rollouts sample at temperature 1.0 and nucleus threshold 0.95).  p_n is
+ * replaced by its renormalised restriction to the nucleus: tokens in order of decreasing probability
+ * until their mass first reaches top_p, plus every token that ties with the last one taken (the
+ * paper does not say how ties are cut; this rule does not depend on the order of equal
+ * probabilities).  top_p in (0,1); top_p >= 1 is specroll_verify.  Acceptance, residuals and the
+ * terminal draw then use the truncated distributions, so the emitted tokens are exact samples of them.
+ * row_max / row_sum are still those of the plain softmax.  Optional outputs (device, nullable):
+ * nucleus_thr[B,N] fp32 = logit of the smallest kept token, nucleus_sum[B,N] fp32 = sum of
+ * exp((l - row_max)/T) over the kept tokens.  Workspace: specroll_verify_nucleus_workspace_bytes. */
+size_t specroll_verify_nucleus_workspace_bytes(const specroll_verify_desc *desc);
+
+int specroll_verify_nucleus(const specroll_verify_desc *desc, float top_p, const void *logits,
+                            const int32_t *parent_host, const int32_t *tree_tok,
+                            const uint8_t *tree_cand, const int32_t *cand_id,
+                            const float *cand_logit, const float *u_acc, const float *u_fin,
+                            int32_t *n_acc, int32_t *path_node, int32_t *out_tok,
+                            int32_t *term_node, int32_t *term_kind, float *row_max, float *row_sum,
+                            float *min_margin, float *nucleus_thr, float *nucleus_sum,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* ------------------------------------------------------------------------------------------
  * Allocation-free variant of specroll_verify.  (The paper has no counterpart: this is a
  * deployment convenience of this library, not a step of the method.)

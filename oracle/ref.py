@@ -173,7 +173,10 @@ def tree_attn(Q, Kc, Vc, kv_indptr, Kt, Vt, parent, scale=None, want_lse=False):
 
 
 def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin,
-           temperature=1.0):
+           temperature=1.0, top_p=None):
+    if top_p is not None:
+        return _verify_nucleus(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin,
+                               temperature, top_p)
     logits = _as(logits, np.uint16)
     parent, tree_tok = _as(parent, np.int32), _as(tree_tok, np.int32)
     tree_cand, cand_id = _as(tree_cand, np.uint8), _as(cand_id, np.int32)
@@ -198,6 +201,36 @@ def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fi
     return {"n_acc": n_acc, "path_node": path, "out_tok": out_tok, "term_node": term_node,
             "term_kind": term_kind, "row_max": row_max, "row_sum": row_sum, "min_margin": mm,
             "fin_margin": fm}
+
+
+def _verify_nucleus(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, temperature, top_p):
+    logits = _as(logits, np.uint16)
+    parent, tree_tok = _as(parent, np.int32), _as(tree_tok, np.int32)
+    tree_cand, cand_id = _as(tree_cand, np.uint8), _as(cand_id, np.int32)
+    cand_logit, u_acc, u_fin = (_as(x, np.float32) for x in (cand_logit, u_acc, u_fin))
+    B, N, V = logits.shape
+    _, K, k = cand_id.shape
+    n_acc = np.empty(B, np.int32)
+    path = np.empty((B, K + 1), np.int32)
+    out_tok = np.empty((B, K + 1), np.int32)
+    term_node = np.empty(B, np.int32)
+    term_kind = np.empty(B, np.int32)
+    row_max = np.empty((B, N), np.float64)
+    row_sum = np.empty((B, N), np.float64)
+    mm = np.empty(B, np.float64)
+    fm = np.empty(B, np.float64)
+    thr = np.full((B, N), np.nan)
+    ksum = np.full((B, N), np.nan)
+    nm = np.empty(B, np.float64)
+    rc = lib().specroll_ref_verify_nucleus(
+        B, N, K, k, V, C.c_double(float(np.float32(temperature))), C.c_double(float(np.float32(top_p))), _p(logits),
+        _p(parent), _p(tree_tok), _p(tree_cand), _p(cand_id), _p(cand_logit), _p(u_acc), _p(u_fin), _p(n_acc),
+        _p(path), _p(out_tok), _p(term_node), _p(term_kind), _p(row_max), _p(row_sum), _p(mm), _p(fm), _p(thr),
+        _p(ksum), _p(nm))
+    _chk(rc, "verify_nucleus")
+    return {"n_acc": n_acc, "path_node": path, "out_tok": out_tok, "term_node": term_node,
+            "term_kind": term_kind, "row_max": row_max, "row_sum": row_sum, "min_margin": mm,
+            "fin_margin": fm, "nucleus_thr": thr, "nucleus_sum": ksum, "nucleus_margin": nm}
 
 
 def node_budget(C_hw, B_active, N_min=1, N_max=10) -> int:

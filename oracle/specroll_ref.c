@@ -421,13 +421,59 @@ int specroll_ref_tree_attn(int B, int N, int Hq, int Hkv, int D, double scale, c
  * min_margin[B] = min |U - ratio| over tested slots (+inf if none);
  * fin_margin[B] = distance of u_fin*total to the nearest bracket end, over total.
  */
-int specroll_ref_verify(int B, int N, int K, int k, int V, double T, const uint16_t *logits,
+/* Nucleus truncation of one target distribution (the experiments sample the target at nucleus threshold 0.95,
+ * App. "Implementation and Reproducibility Details"; the paper does not say how ties are cut).  Reading: the
+ * tokens are taken in order of decreasing probability until their mass first reaches top_p, and every token
+ * that ties with the last one taken is kept as well, so the kept set does not depend on how equal
+ * probabilities are ordered.  p[V] (sums to 1) is replaced by its renormalised restriction to the kept set.
+ * thr_p = smallest kept probability, kept_mass = mass kept (before renormalising),
+ * margin = distance of top_p to the nearer of the two cumulative masses that bracket it. */
+typedef struct { double p; int v; } nuc_item;
+static int nuc_cmp(const void *a, const void *b)
+{
+    const nuc_item *x = (const nuc_item *)a, *y = (const nuc_item *)b;
+    if (x->p > y->p) return -1;
+    if (x->p < y->p) return 1;
+    return (x->v > y->v) - (x->v < y->v);
+}
+static void nucleus(int V, double *p, double top_p, nuc_item *scratch, double *thr_p, double *kept_mass,
+                    double *margin)
+{
+    for (int v = 0; v < V; ++v) {
+        scratch[v].p = p[v];
+        scratch[v].v = v;
+    }
+    qsort(scratch, (size_t)V, sizeof(nuc_item), nuc_cmp);
+    double cum = 0.0, above = 0.0; /* above = mass of the probabilities strictly larger than the current one */
+    int i = 0;
+    for (; i < V; ++i) {
+        if (i > 0 && scratch[i].p < scratch[i - 1].p) above = cum;
+        cum += scratch[i].p;
+        if (cum >= top_p) break;
+    }
+    if (i >= V) i = V - 1; /* rounding kept the total below top_p: keep everything */
+    const double pv = scratch[i].p;
+    double all = above; /* mass of everything >= pv */
+    for (int j = 0; j < V; ++j)
+        if (scratch[j].p == pv) all += scratch[j].p;
+    for (int v = 0; v < V; ++v) p[v] = (p[v] >= pv) ? p[v] / all : 0.0;
+    *thr_p = pv;
+    *kept_mass = all;
+    double m1 = top_p - above, m2 = all - top_p;
+    if (m1 < 0) m1 = -m1;
+    if (m2 < 0) m2 = -m2;
+    *margin = m1 < m2 ? m1 : m2;
+}
+
+static int verify_impl(int B, int N, int K, int k, int V, double T, double top_p, const uint16_t *logits,
                         const int32_t *parent, const int32_t *tree_tok, const uint8_t *tree_cand,
                         const int32_t *cand_id, const float *cand_logit, const float *u_acc,
                         const float *u_fin, int32_t *n_acc, int32_t *path_node, int32_t *out_tok,
                         int32_t *term_node, int32_t *term_kind, double *row_max, double *row_sum,
-                        double *min_margin, double *fin_margin)
+                        double *min_margin, double *fin_margin, double *nuc_thr, double *nuc_sum,
+                        double *nuc_margin)
 {
+    const int truncate = top_p > 0.0 && top_p < 1.0;
     int depth[REF_MAX_NODES];
     if (tree_depths(N, parent, depth) != REF_OK || k < 1 || k > REF_MAX_K || V < 1) return REF_EINVAL;
     for (int n = 0; n < N; ++n)
@@ -436,6 +482,8 @@ int specroll_ref_verify(int B, int N, int K, int k, int V, double T, const uint1
     for (int b = 0; b < B; ++b) {
         double *r = (double *)malloc(sizeof(double) * V);
         double *q = (double *)malloc(sizeof(double) * V);
+        nuc_item *scratch = truncate ? (nuc_item *)malloc(sizeof(nuc_item) * V) : NULL;
+        double nmin = INFINITY; /* smallest nucleus margin among the nodes whose distribution was used */
         /* softmax statistics of every node */
         for (int n = 0; n < N; ++n) {
             const uint16_t *lg = logits + ((size_t)b * N + n) * V;
@@ -459,6 +507,13 @@ int specroll_ref_verify(int B, int N, int K, int k, int V, double T, const uint1
             const uint16_t *lg = logits + ((size_t)b * N + u) * V;
             double mx = row_max[(size_t)b * N + u], s = row_sum[(size_t)b * N + u];
             for (int v = 0; v < V; ++v) r[v] = exp((bf16_to_f64(lg[v]) - mx) / T) / s;
+            if (truncate) { /* the target distribution of this node is its nucleus */
+                double thr_p, kept, mg;
+                nucleus(V, r, top_p, scratch, &thr_p, &kept, &mg);
+                if (mg < nmin) nmin = mg;
+                if (nuc_thr) nuc_thr[(size_t)b * N + u] = mx + T * log(thr_p * s); /* logit of the smallest kept token */
+                if (nuc_sum) nuc_sum[(size_t)b * N + u] = kept * s;               /* kept mass in units of exp((l-M)/T) */
+            }
             int nchild = 0, accepted = -1;
             for (int c = u + 1; c < N; ++c)
                 if (parent[c] == u) ++nchild;
@@ -534,10 +589,41 @@ int specroll_ref_verify(int B, int N, int K, int k, int V, double T, const uint1
         term_kind[b] = kind;
         if (min_margin) min_margin[b] = mm;
         if (fin_margin) fin_margin[b] = fm / total;
+        if (nuc_margin) nuc_margin[b] = nmin;
         free(r);
         free(q);
+        free(scratch);
     }
     return REF_OK;
+}
+
+int specroll_ref_verify(int B, int N, int K, int k, int V, double T, const uint16_t *logits,
+                        const int32_t *parent, const int32_t *tree_tok, const uint8_t *tree_cand,
+                        const int32_t *cand_id, const float *cand_logit, const float *u_acc,
+                        const float *u_fin, int32_t *n_acc, int32_t *path_node, int32_t *out_tok,
+                        int32_t *term_node, int32_t *term_kind, double *row_max, double *row_sum,
+                        double *min_margin, double *fin_margin)
+{
+    return verify_impl(B, N, K, k, V, T, 1.0, logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin,
+                       n_acc, path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, fin_margin,
+                       NULL, NULL, NULL);
+}
+
+/* The same walk against nucleus-truncated target distributions (top_p in (0,1); >= 1 keeps everything).
+ * Extra outputs: nuc_thr, nuc_sum [B,N], written for the nodes the walk visited only (others untouched):
+ * the logit of the smallest kept token and the kept mass in units of exp((l - M)/T);
+ * nuc_margin[B] = smallest distance of top_p to a bracketing cumulative mass over the visited nodes. */
+int specroll_ref_verify_nucleus(int B, int N, int K, int k, int V, double T, double top_p, const uint16_t *logits,
+                                const int32_t *parent, const int32_t *tree_tok, const uint8_t *tree_cand,
+                                const int32_t *cand_id, const float *cand_logit, const float *u_acc,
+                                const float *u_fin, int32_t *n_acc, int32_t *path_node, int32_t *out_tok,
+                                int32_t *term_node, int32_t *term_kind, double *row_max, double *row_sum,
+                                double *min_margin, double *fin_margin, double *nuc_thr, double *nuc_sum,
+                                double *nuc_margin)
+{
+    return verify_impl(B, N, K, k, V, T, top_p, logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc,
+                       u_fin, n_acc, path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin,
+                       fin_margin, nuc_thr, nuc_sum, nuc_margin);
 }
 
 /* Node budget N_t = clip(floor(C_hw / B_t), N_min, N_max)  (Eq. "verification-budget"). */

@@ -24,7 +24,8 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
            "specroll_tree_attn_workspace_bytes", "specroll_tree_attn",
            "specroll_tree_attn_paged_workspace_bytes", "specroll_tree_attn_paged",
            "specroll_commit_path", "specroll_commit_path_layers", "specroll_gather_hidden",
-           "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static")
+           "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static",
+           "specroll_verify_nucleus_workspace_bytes", "specroll_verify_nucleus")
 
 
 PROPOSE_LEGACY_MMA = 1
@@ -69,11 +70,12 @@ def lib():
         l.specroll_node_budget.restype = C.c_int32
         l.specroll_node_budget.argtypes = [C.c_int32] * 4
         for n in ("specroll_propose_workspace_bytes", "specroll_verify_workspace_bytes",
-                  "specroll_tree_attn_workspace_bytes", "specroll_tree_attn_paged_workspace_bytes"):
+                  "specroll_tree_attn_workspace_bytes", "specroll_tree_attn_paged_workspace_bytes",
+                  "specroll_verify_nucleus_workspace_bytes"):
             getattr(l, n).restype = C.c_size_t
         for n in ("specroll_propose", "specroll_workspace_status", "specroll_tree_draw", "specroll_tree_attn",
                   "specroll_verify", "specroll_verify_static", "specroll_tree_attn_paged", "specroll_commit_path",
-                  "specroll_commit_path_layers", "specroll_gather_hidden"):
+                  "specroll_commit_path_layers", "specroll_gather_hidden", "specroll_verify_nucleus"):
             getattr(l, n).restype = C.c_int
         _lib = l
     return _lib
@@ -348,6 +350,11 @@ def verify_workspace_bytes(B, N, K, k, V, temperature=1.0) -> int:
     return int(lib().specroll_verify_workspace_bytes(C.byref(desc)))
 
 
+def verify_nucleus_workspace_bytes(B, N, K, k, V, temperature=1.0) -> int:
+    desc = VerifyDesc(B, N, K, k, V, temperature, 0)
+    return int(lib().specroll_verify_nucleus_workspace_bytes(C.byref(desc)))
+
+
 def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, temperature=1.0,
            workspace=None, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
     """specroll_verify.  Device tensors in, dict of device tensors out."""
@@ -380,6 +387,45 @@ def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fi
         _dev(out["row_sum"], f32, "row_sum"), _dev(out.get("min_margin"), f32, "min_margin"),
         C.c_void_p(workspace.data_ptr()), C.c_size_t(workspace.numel()), _stream())
     _check(rc, "specroll_verify")
+    return out
+
+
+def verify_nucleus(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, top_p, temperature=1.0,
+                   workspace=None, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+    """specroll_verify_nucleus: verification against nucleus-truncated target distributions.
+    The returned dict also holds nucleus_thr and nucleus_sum [B,N]."""
+    parent = _host_i32(parent, "parent")
+    B, N, V = logits.shape
+    _, K, k = cand_id.shape
+    if parent.shape[0] != N or tuple(tree_tok.shape) != (B, N) or tuple(u_acc.shape) != (B, N):
+        raise SpecrollError("verify_nucleus: inconsistent shapes")
+    desc = VerifyDesc(B, N, K, k, V, temperature, 0)
+    dev = logits.device
+    i32, f32 = torch.int32, torch.float32
+    if out is None:
+        out = {"n_acc": torch.empty(B, dtype=i32, device=dev),
+               "path_node": torch.empty((B, K + 1), dtype=i32, device=dev),
+               "out_tok": torch.empty((B, K + 1), dtype=i32, device=dev),
+               "term_node": torch.empty(B, dtype=i32, device=dev),
+               "term_kind": torch.empty(B, dtype=i32, device=dev),
+               "row_max": torch.empty((B, N), dtype=f32, device=dev),
+               "row_sum": torch.empty((B, N), dtype=f32, device=dev),
+               "min_margin": torch.empty(B, dtype=f32, device=dev),
+               "nucleus_thr": torch.empty((B, N), dtype=f32, device=dev),
+               "nucleus_sum": torch.empty((B, N), dtype=f32, device=dev)}
+    if workspace is None:
+        workspace = _workspace(lib().specroll_verify_nucleus_workspace_bytes(C.byref(desc)), dev)
+    rc = lib().specroll_verify_nucleus(
+        C.byref(desc), C.c_float(top_p), _dev(logits, torch.bfloat16, "logits"), parent.ctypes.data_as(C.c_void_p),
+        _dev(tree_tok, i32, "tree_tok"), _dev(tree_cand, torch.uint8, "tree_cand"),
+        _dev(cand_id, i32, "cand_id"), _dev(cand_logit, f32, "cand_logit"), _dev(u_acc, f32, "u_acc"),
+        _dev(u_fin, f32, "u_fin"), _dev(out["n_acc"], i32, "n_acc"), _dev(out["path_node"], i32, "path_node"),
+        _dev(out["out_tok"], i32, "out_tok"), _dev(out["term_node"], i32, "term_node"),
+        _dev(out["term_kind"], i32, "term_kind"), _dev(out["row_max"], f32, "row_max"),
+        _dev(out["row_sum"], f32, "row_sum"), _dev(out.get("min_margin"), f32, "min_margin"),
+        _dev(out.get("nucleus_thr"), f32, "nucleus_thr"), _dev(out.get("nucleus_sum"), f32, "nucleus_sum"),
+        C.c_void_p(workspace.data_ptr()), C.c_size_t(workspace.numel()), _stream())
+    _check(rc, "specroll_verify_nucleus")
     return out
 
 

@@ -91,6 +91,106 @@ row_stats_kernel(const uint16_t *__restrict__ logits, int V, float c, float *__r
     }
 }
 
+// ------------------------------------------------------------------------------ nucleus threshold
+
+// Order-preserving 16-bit key of a bf16 value (-0 counts as +0): larger value <=> larger key.
+__device__ __forceinline__ uint32_t ord_key(uint32_t bits) {
+    if (bits == 0x8000u) bits = 0u;
+    return (bits & 0x8000u) ? (~bits & 0xffffu) : (bits | 0x8000u);
+}
+
+constexpr int NUC_THREADS = 512;
+
+// Nucleus of one row (sampling configuration of the experiments: threshold 0.95): tokens are taken in order of
+// decreasing probability until their mass first reaches top_p, and every token that ties with the last one
+// taken is kept too.  Equal probabilities are equal bf16 logits, so the kept set is "key >= threshold key", and
+// the threshold is found by a radix search over the 16 key bits, four bits per pass: each pass adds up, per
+// value of the next four bits, the mass of the tokens whose leading bits match the digits found so far
+// (private bins per thread in shared memory, no atomics), and picks the digit at which the mass from the top
+// reaches top_p * S.  Run by all NUC_THREADS threads of a CTA; the row comes from HBM once and from L2 after.
+// Leaves in st->prefix the threshold key (a token is kept iff ord_key(logit) >= key) and in st->keep the sum of
+// the kept exp((l - M)/T).
+struct NucleusSmem {
+    float bins[16][NUC_THREADS];
+    float wsum[NUC_THREADS / 32][16];
+    float above, keep;
+    uint32_t prefix;
+};
+
+__device__ void nucleus_row(const uint16_t *__restrict__ row_logits, int V, float c, float M, float target,
+                            NucleusSmem *st) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint4 *p = reinterpret_cast<const uint4 *>(row_logits);
+    const int nvec = V >> 3;
+    if (tid == 0) {
+        st->above = 0.f;
+        st->prefix = 0u;
+    }
+    __syncthreads();
+    for (int level = 0; level < 4; ++level) {
+        const int shift = 12 - 4 * level;
+        const uint32_t prefix = st->prefix;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) st->bins[j][tid] = 0.f;
+        for (int i0 = tid; i0 < nvec; i0 += 4 * NUC_THREADS) {
+            uint4 vv[4];  // four independent loads in flight; an absent one reads as -inf (no mass, lowest key range)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int i = i0 + q * NUC_THREADS;
+                vv[q] = i < nvec ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    const uint32_t bits = (t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu);
+                    const uint32_t key = ord_key(bits);
+                    if (level == 0 || (key >> (shift + 4)) == prefix)
+                        st->bins[(key >> shift) & 15u][tid] += ex2_approx((__uint_as_float(bits << 16) - M) * c);
+                }
+            }
+        }
+        // sixteen sums over the block
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float x = warp_sum(st->bins[j][tid]);
+            if (lane == 0) st->wsum[warp][j] = x;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            float tot[16];
+            for (int j = 0; j < 16; ++j) {
+                float x = 0.f;
+                for (int w2 = 0; w2 < NUC_THREADS / 32; ++w2) x += st->wsum[w2][j];
+                tot[j] = x;
+            }
+            // from the top digit down: first digit at which the mass reaches the target
+            float cum = st->above;
+            int sel = -1, low = 0;
+            for (int j = 15; j >= 0; --j) {
+                if (tot[j] > 0.f) low = j;
+            }
+            for (int j = 15; j >= 0; --j) {
+                if (cum + tot[j] >= target) {
+                    sel = j;
+                    break;
+                }
+                cum += tot[j];
+            }
+            if (sel < 0) {  // rounding kept the total below the target: keep everything
+                sel = low;
+                cum = st->above;
+                for (int j = 15; j > low; --j) cum += tot[j];
+            }
+            st->above = cum;
+            st->prefix = (prefix << 4) | (uint32_t)sel;
+            st->keep = cum + tot[sel];
+        }
+        __syncthreads();
+    }
+}
+
 // ------------------------------------------------------------------------------ walk
 
 struct WalkArgs {
@@ -112,133 +212,222 @@ struct WalkArgs {
     double T;
 };
 
-__global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(WalkArgs a, Topo topo) {
-    __shared__ double sh_r[WALK_WARPS][SPECROLL_MAX_TOPK];
-    __shared__ double sh_w[WALK_WARPS][SPECROLL_MAX_TOPK];
-    __shared__ float sh_cl[WALK_WARPS][SPECROLL_MAX_TOPK];
-    __shared__ int32_t sh_id[WALK_WARPS][SPECROLL_MAX_TOPK];
-    __shared__ double sh_bc[WALK_WARPS][2];  // broadcast slots: current max, accepted flag
+// What a warp carries from node to node of one sequence's walk.
+struct WalkState {
+    int nacc, kind;
+    double sigma;  // residual of a token outside the candidate set = sigma * p(token)
+    double p_off;
+    float mm;
+    bool have_residual;
+};
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.x * WALK_WARPS + warp;
-    if (b >= a.B) return;
-    double *r = sh_r[warp], *w = sh_w[warp];
-    float *cl = sh_cl[warp];
-    int32_t *id = sh_id[warp];
-    const int k = a.k, N = a.N, K = a.K;
+// Per-warp shared scratch of the walk.
+struct WalkSmem {
+    double r[SPECROLL_MAX_TOPK];
+    double w[SPECROLL_MAX_TOPK];
+    float cl[SPECROLL_MAX_TOPK];
+    int32_t id[SPECROLL_MAX_TOPK];
+    double bc[2];  // broadcast slots: current max, accepted flag
+};
 
-    int u = 0, nacc = 0, kind = 0;
-    double sigma = 1.0;  // residual of a token outside the candidate set = sigma * p(token)
-    double p_off = 0.0;
-    float mm = INFINITY;
-    bool have_residual = false;
+__device__ __forceinline__ void walk_begin(const WalkArgs &a, int b, int lane, WalkState *st) {
+    st->nacc = 0;
+    st->kind = 0;
+    st->sigma = 1.0;
+    st->p_off = 0.0;
+    st->mm = INFINITY;
+    st->have_residual = false;
     if (lane == 0) {
+        const int K = a.K;
         for (int i = 0; i <= K; ++i) a.path_node[(size_t)b * (K + 1) + i] = a.out_tok[(size_t)b * (K + 1) + i] = -1;
         a.path_node[(size_t)b * (K + 1)] = 0;
     }
-    for (;;) {
-        if (topo.n_child[u] == 0) {
-            kind = (u != 0) ? 1 : 0;
-            have_residual = false;
-            break;
-        }
-        const int hd = topo.depth[u];
-        const double M = (double)a.row_max[(size_t)b * N + u];
-        const double S = (double)a.row_sum[(size_t)b * N + u];
-        const uint16_t *lg = a.logits + ((size_t)b * N + u) * a.V;
-        for (int j = lane; j < k; j += 32) {
-            const int t = a.cand_id[((size_t)b * K + hd) * k + j];
-            id[j] = t;
-            cl[j] = a.cand_logit[((size_t)b * K + hd) * k + j];
-            const double l = (double)bf16_bits_to_float(lg[t]);
-            r[j] = exp((l - M) / a.T) / S;  // r = p_u on the candidates
+}
+
+// One node u (which has children), by one warp: the target's probabilities on the candidates of u's head -
+// S is the normaliser and thr the nucleus threshold key (0: none) of u's row - then u's children in slot order.
+// Returns the accepted child, or -1 when every child was rejected (the residual is then in sm->r, st->sigma).
+__device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, double S, uint32_t thr, int lane,
+                         WalkSmem *sm, WalkState *st) {
+    double *r = sm->r, *w = sm->w;
+    float *cl = sm->cl;
+    int32_t *id = sm->id;
+    const int k = a.k, N = a.N, K = a.K;
+    const int hd = topo.depth[u];
+    const double M = (double)a.row_max[(size_t)b * N + u];
+    const uint16_t *lg = a.logits + ((size_t)b * N + u) * a.V;
+    for (int j = lane; j < k; j += 32) {
+        const int t = a.cand_id[((size_t)b * K + hd) * k + j];
+        id[j] = t;
+        cl[j] = a.cand_logit[((size_t)b * K + hd) * k + j];
+        const uint32_t bits = lg[t];
+        const double l = (double)bf16_bits_to_float((uint16_t)bits);
+        r[j] = ord_key(bits) >= thr ? exp((l - M) / a.T) / S : 0.0;  // r = p_u on the candidates
+    }
+    __syncwarp();
+    st->sigma = 1.0;
+    if (lane == 0) {
+        double pc = 0.0;
+        for (int j = 0; j < k; ++j) pc += r[j];
+        st->p_off = 1.0 - pc;
+        if (st->p_off < 0.0) st->p_off = 0.0;
+    }
+    uint64_t taken = 0;
+    int accepted = -1;
+    for (int c = u + 1; c < N && accepted < 0; ++c) {
+        if (topo.parent[c] != u) continue;
+        // slot proposal q on the candidates not yet taken
+        if (lane == 0) {
+            double mx = -INFINITY;
+            for (int j = 0; j < k; ++j)
+                if (!((taken >> j) & 1) && (double)cl[j] > mx) mx = (double)cl[j];
+            sm->bc[0] = mx;
         }
         __syncwarp();
-        sigma = 1.0;
+        const double mx = sm->bc[0];
+        for (int j = lane; j < k; j += 32)
+            w[j] = ((taken >> j) & 1) ? 0.0 : exp(((double)cl[j] - mx) / a.T);
+        __syncwarp();
+        const int jc = a.tree_cand[(size_t)b * N + c];
         if (lane == 0) {
-            double pc = 0.0;
-            for (int j = 0; j < k; ++j) pc += r[j];
-            p_off = 1.0 - pc;
-            if (p_off < 0.0) p_off = 0.0;
-        }
-        uint64_t taken = 0;
-        int accepted = -1;
-        for (int c = u + 1; c < N && accepted < 0; ++c) {
-            if (topo.parent[c] != u) continue;
-            // slot proposal q on the candidates not yet taken
-            if (lane == 0) {
-                double mx = -INFINITY;
-                for (int j = 0; j < k; ++j)
-                    if (!((taken >> j) & 1) && (double)cl[j] > mx) mx = (double)cl[j];
-                sh_bc[warp][0] = mx;
-            }
-            __syncwarp();
-            const double mx = sh_bc[warp][0];
-            for (int j = lane; j < k; j += 32)
-                w[j] = ((taken >> j) & 1) ? 0.0 : exp(((double)cl[j] - mx) / a.T);
-            __syncwarp();
-            const int jc = a.tree_cand[(size_t)b * N + c];
-            if (lane == 0) {
-                double s = 0.0;
-                for (int j = 0; j < k; ++j) s += w[j];
-                const double qy = w[jc] / s;
-                double ratio;
-                if (qy > 0.0)
-                    ratio = r[jc] / qy;
-                else
-                    ratio = (r[jc] > 0.0) ? INFINITY : 0.0;
-                const double uu = (double)a.u_acc[(size_t)b * N + c];
-                const float mg = (float)fabs(uu - ratio);
-                if (mg < mm) mm = mg;
-                if (uu < (ratio < 1.0 ? ratio : 1.0)) {
-                    sh_bc[warp][1] = (double)c;
-                } else {
-                    sh_bc[warp][1] = -1.0;
-                    double Z = 0.0;
-                    for (int j = 0; j < k; ++j) {
-                        const double t = r[j] - w[j] / s;
-                        w[j] = t > 0.0 ? t : 0.0;
-                        Z += w[j];
-                    }
-                    Z += sigma * p_off;
-                    if (Z > 1e-300) {
-                        for (int j = 0; j < k; ++j) r[j] = w[j] / Z;
-                        sigma /= Z;
-                    }
+            double s = 0.0;
+            for (int j = 0; j < k; ++j) s += w[j];
+            const double qy = w[jc] / s;
+            double ratio;
+            if (qy > 0.0)
+                ratio = r[jc] / qy;
+            else
+                ratio = (r[jc] > 0.0) ? INFINITY : 0.0;
+            const double uu = (double)a.u_acc[(size_t)b * N + c];
+            const float mg = (float)fabs(uu - ratio);
+            if (mg < st->mm) st->mm = mg;
+            if (uu < (ratio < 1.0 ? ratio : 1.0)) {
+                sm->bc[1] = (double)c;
+            } else {
+                sm->bc[1] = -1.0;
+                double Z = 0.0;
+                for (int j = 0; j < k; ++j) {
+                    const double t = r[j] - w[j] / s;
+                    w[j] = t > 0.0 ? t : 0.0;
+                    Z += w[j];
+                }
+                Z += st->sigma * st->p_off;
+                if (Z > 1e-300) {
+                    for (int j = 0; j < k; ++j) r[j] = w[j] / Z;
+                    st->sigma /= Z;
                 }
             }
-            __syncwarp();
-            accepted = (int)sh_bc[warp][1];
-            taken |= 1ull << jc;
-            __syncwarp();
         }
-        if (accepted < 0) {
-            kind = 0;
-            have_residual = true;
-            break;
-        }
-        if (lane == 0) {
-            a.out_tok[(size_t)b * (K + 1) + nacc] = a.tree_tok[(size_t)b * N + accepted];
-            a.path_node[(size_t)b * (K + 1) + nacc + 1] = accepted;
-        }
-        ++nacc;
-        u = accepted;
+        __syncwarp();
+        accepted = (int)sm->bc[1];
+        taken |= 1ull << jc;
+        __syncwarp();
     }
-    // hand the residual over to the terminal draw
-    if (have_residual) {
-        const double S = (double)a.row_sum[(size_t)b * N + u];
-        sigma = __shfl_sync(0xffffffffu, sigma, 0);
+    if (accepted >= 0) {
+        if (lane == 0) {
+            a.out_tok[(size_t)b * (K + 1) + st->nacc] = a.tree_tok[(size_t)b * N + accepted];
+            a.path_node[(size_t)b * (K + 1) + st->nacc + 1] = accepted;
+        }
+        ++st->nacc;
+    }
+    return accepted;
+}
+
+// Results of a sequence and the hand-over of the residual (S = normaliser of u's row) to the terminal draw.
+__device__ __forceinline__ void walk_end(const WalkArgs &a, int b, int u, double S, int lane, WalkSmem *sm,
+                                         WalkState *st) {
+    const int k = a.k;
+    if (st->have_residual) {
+        const double sigma = __shfl_sync(0xffffffffu, st->sigma, 0);
         for (int j = lane; j < k; j += 32) {
-            a.ws_ovid[(size_t)b * k + j] = id[j];
-            a.ws_ovm[(size_t)b * k + j] = r[j] * S / sigma;
+            a.ws_ovid[(size_t)b * k + j] = sm->id[j];
+            a.ws_ovm[(size_t)b * k + j] = sm->r[j] * S / sigma;
         }
     }
     if (lane == 0) {
-        a.ws_nov[b] = have_residual ? k : 0;
-        a.n_acc[b] = nacc;
+        a.ws_nov[b] = st->have_residual ? k : 0;
+        a.n_acc[b] = st->nacc;
         a.term_node[b] = u;
-        a.term_kind[b] = kind;
-        if (a.min_margin) a.min_margin[b] = mm;
+        a.term_kind[b] = st->kind;
+        if (a.min_margin) a.min_margin[b] = st->mm;
+    }
+}
+
+// Plain target distributions: one warp per sequence.
+__global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(WalkArgs a, Topo topo) {
+    __shared__ WalkSmem sh[WALK_WARPS];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * WALK_WARPS + warp;
+    if (b >= a.B) return;
+    WalkSmem *sm = &sh[warp];
+    WalkState st;
+    walk_begin(a, b, lane, &st);
+    int u = 0;
+    for (;;) {
+        if (topo.n_child[u] == 0) {
+            st.kind = (u != 0) ? 1 : 0;
+            st.have_residual = false;
+            break;
+        }
+        const int acc = walk_node(a, topo, b, u, (double)a.row_sum[(size_t)b * a.N + u], 0u, lane, sm, &st);
+        if (acc < 0) {
+            st.kind = 0;
+            st.have_residual = true;
+            break;
+        }
+        u = acc;
+    }
+    walk_end(a, b, u, (double)a.row_sum[(size_t)b * a.N + u], lane, sm, &st);
+}
+
+// Nucleus-truncated target distributions: one CTA per sequence.  Only the nodes the walk visits need their
+// nucleus, and which they are is known only as the walk goes, so before each node all threads find that row's
+// threshold (nucleus_row) and warp 0 then does the node.  Thresholds and kept sums of the visited nodes are
+// left in thr_key / keep_sum (the terminal draw reads those of the last node).
+__global__ void __launch_bounds__(NUC_THREADS)
+walk_nucleus_kernel(WalkArgs a, Topo topo, float c, float top_p, uint32_t *__restrict__ thr_key,
+                    float *__restrict__ keep_sum, float *__restrict__ out_thr, float *__restrict__ out_sum) {
+    __shared__ NucleusSmem nuc;
+    __shared__ WalkSmem sm;
+    __shared__ int sh_next;  // next node, or -1 when the walk is over
+    const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    WalkState st;
+    if (warp == 0) walk_begin(a, b, lane, &st);
+    int u = 0;
+    for (;;) {
+        const size_t row = (size_t)b * a.N + u;
+        nucleus_row(a.logits + row * a.V, a.V, c, a.row_max[row], top_p * a.row_sum[row], &nuc);
+        const uint32_t thr = nuc.prefix;
+        const float keep = nuc.keep;
+        if (threadIdx.x == 0) {
+            thr_key[row] = thr;
+            keep_sum[row] = keep;
+            if (out_sum) out_sum[row] = keep;
+            if (out_thr) {  // the threshold as a logit: undo the key
+                const uint32_t bits = (thr & 0x8000u) ? (thr & 0x7fffu) : (~thr & 0xffffu);
+                out_thr[row] = __uint_as_float(bits << 16);
+            }
+        }
+        if (warp == 0) {
+            int next = -1;
+            if (topo.n_child[u] == 0) {
+                st.kind = (u != 0) ? 1 : 0;
+                st.have_residual = false;
+            } else {
+                next = walk_node(a, topo, b, u, (double)keep, thr, lane, &sm, &st);
+                if (next < 0) {
+                    st.kind = 0;
+                    st.have_residual = true;
+                }
+            }
+            if (next < 0) walk_end(a, b, u, (double)keep, lane, &sm, &st);
+            if (lane == 0) sh_next = next;
+        }
+        __syncthreads();
+        const int next = sh_next;
+        __syncthreads();
+        if (next < 0) break;
+        u = next;
     }
 }
 
@@ -251,18 +440,25 @@ struct TermArgs {
     const int32_t *n_acc, *term_node;
     const int32_t *ws_nov, *ws_ovid;
     const double *ws_ovm;
+    const uint32_t *thr_key;  // nucleus threshold per row (NULL: no truncation)
     int32_t *out_tok;
     int32_t B, N, K, k, V;
     float c;  // log2(e) / T
 };
 
-__device__ __forceinline__ void masses8(const uint4 &v, float M, float c, float (&e)[8]) {
+// Plain softmax masses of eight tokens; tokens below the nucleus threshold (thr = 0: none) weigh nothing.
+__device__ __forceinline__ void masses8(const uint4 &v, float M, float c, uint32_t thr, float (&e)[8]) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        e[2 * i] = ex2_approx((__uint_as_float(w[i] << 16) - M) * c);
-        e[2 * i + 1] = ex2_approx((__uint_as_float(w[i] & 0xffff0000u) - M) * c);
+        const float e0 = ex2_approx((__uint_as_float(w[i] << 16) - M) * c);
+        const float e1 = ex2_approx((__uint_as_float(w[i] & 0xffff0000u) - M) * c);
+        e[2 * i] = ord_key(w[i] & 0xffffu) >= thr ? e0 : 0.f;
+        e[2 * i + 1] = ord_key(w[i] >> 16) >= thr ? e1 : 0.f;
     }
+}
+__device__ __forceinline__ float mass1(uint16_t bits, float M, float c, uint32_t thr) {
+    return ord_key(bits) >= thr ? ex2_approx((bf16_bits_to_float(bits) - M) * c) : 0.f;
 }
 
 __device__ __forceinline__ double warp_incl_scan(double v, int lane) {
@@ -296,6 +492,7 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
     const int node = a.term_node[b];
     const int nov = a.ws_nov[b];
     const float M = a.row_max[(size_t)b * a.N + node];
+    const uint32_t thr = a.thr_key ? a.thr_key[(size_t)b * a.N + node] : 0u;
     const uint16_t *lg = a.logits + ((size_t)b * a.N + node) * a.V;
     const uint4 *p = reinterpret_cast<const uint4 *>(lg);
     const int nvec = a.V >> 3;
@@ -319,7 +516,7 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             float e[8];
-            masses8(v[q], M, a.c, e);
+            masses8(v[q], M, a.c, thr, e);
             double acc = 0.0;
 #pragma unroll
             for (int t = 0; t < 8; ++t) acc += (double)e[t];
@@ -333,7 +530,7 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
         for (int j = 0; j < nov; ++j) {
             const int t = sh_ovid[j], vi = t >> 3;
             const int w = min(TERM_WARPS - 1, vi / vpw), sl = (vi - w * vpw) >> 5;
-            sh_slice[w * n_sl + sl] += sh_ovm[j] - (double)ex2_approx((bf16_bits_to_float(lg[t]) - M) * a.c);
+            sh_slice[w * n_sl + sl] += sh_ovm[j] - (double)mass1(lg[t], M, a.c, thr);
         }
     }
     __syncthreads();
@@ -368,7 +565,7 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
         if (threadIdx.x == 0) {
             int tok = a.V - 1;
             for (; tok > 0; --tok) {
-                double ms = (double)ex2_approx((bf16_bits_to_float(lg[tok]) - M) * a.c);
+                double ms = (double)mass1(lg[tok], M, a.c, thr);
                 for (int j = 0; j < nov; ++j)
                     if (sh_ovid[j] == tok) ms = sh_ovm[j];
                 if (ms > 0.0) break;
@@ -419,7 +616,7 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
     double lsum = 0.0;
     if (i < v_hi) {
         float e[8];
-        masses8(ld_nc_v4(p + i), M, a.c, e);
+        masses8(ld_nc_v4(p + i), M, a.c, thr, e);
 #pragma unroll
         for (int t = 0; t < 8; ++t) ms[t] = (double)e[t];
         for (int j = 0; j < nov; ++j) {
@@ -491,31 +688,41 @@ static int check_verify_desc(const specroll_verify_desc *d) {
     return SPECROLL_OK;
 }
 
-extern "C" size_t specroll_verify_workspace_bytes(const specroll_verify_desc *d) {
-    if (check_verify_desc(d) != SPECROLL_OK) return 0;
+static size_t verify_ws_base(const specroll_verify_desc *d) {
     size_t B = (size_t)d->B, k = (size_t)d->k;
     return align_up(B * k * sizeof(double), 256) + align_up(B * k * sizeof(int32_t), 256) +
            align_up(B * sizeof(int32_t), 256) + 256;
 }
 
-extern "C" int specroll_verify(const specroll_verify_desc *d, const void *logits,
-                               const int32_t *parent_host, const int32_t *tree_tok,
-                               const uint8_t *tree_cand, const int32_t *cand_id,
-                               const float *cand_logit, const float *u_acc, const float *u_fin,
-                               int32_t *n_acc, int32_t *path_node, int32_t *out_tok,
-                               int32_t *term_node, int32_t *term_kind, float *row_max,
-                               float *row_sum, float *min_margin, void *workspace,
-                               size_t workspace_bytes, void *cuda_stream) {
+extern "C" size_t specroll_verify_workspace_bytes(const specroll_verify_desc *d) {
+    if (check_verify_desc(d) != SPECROLL_OK) return 0;
+    return verify_ws_base(d);
+}
+
+extern "C" size_t specroll_verify_nucleus_workspace_bytes(const specroll_verify_desc *d) {
+    if (check_verify_desc(d) != SPECROLL_OK) return 0;
+    const size_t rows = (size_t)d->B * d->N;
+    return verify_ws_base(d) + align_up(rows * sizeof(uint32_t), 256) + align_up(rows * sizeof(float), 256);
+}
+
+// top_p in (0, 1): the target distributions are their nuclei; otherwise the plain softmax.
+static int run_verify(const specroll_verify_desc *d, float top_p, const void *logits, const int32_t *parent_host,
+                      const int32_t *tree_tok, const uint8_t *tree_cand, const int32_t *cand_id,
+                      const float *cand_logit, const float *u_acc, const float *u_fin, int32_t *n_acc,
+                      int32_t *path_node, int32_t *out_tok, int32_t *term_node, int32_t *term_kind, float *row_max,
+                      float *row_sum, float *min_margin, float *nucleus_thr, float *nucleus_sum, void *workspace,
+                      size_t workspace_bytes, void *cuda_stream) {
     if (check_verify_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (!logits || !tree_tok || !tree_cand || !cand_id || !cand_logit || !u_acc || !u_fin || !n_acc ||
         !path_node || !out_tok || !term_node || !term_kind || !row_max || !row_sum)
         return SPECROLL_EINVAL;
+    const bool truncate = top_p > 0.f && top_p < 1.f;
     Topo topo;
     if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (!aligned16(logits)) return SPECROLL_EALIGN;
     if (d->B == 0) return SPECROLL_OK;
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-        workspace_bytes < specroll_verify_workspace_bytes(d))
+    const size_t need = truncate ? specroll_verify_nucleus_workspace_bytes(d) : verify_ws_base(d);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)
         return SPECROLL_EWORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const size_t B = (size_t)d->B, k = (size_t)d->k;
@@ -525,13 +732,16 @@ extern "C" int specroll_verify(const specroll_verify_desc *d, const void *logits
     int32_t *ws_ovid = reinterpret_cast<int32_t *>(ws);
     ws += align_up(B * k * sizeof(int32_t), 256);
     int32_t *ws_nov = reinterpret_cast<int32_t *>(ws);
+    ws += align_up(B * sizeof(int32_t), 256) + 256;
+    const size_t n_rows = B * (size_t)d->N;
+    uint32_t *thr_key = truncate ? reinterpret_cast<uint32_t *>(ws) : nullptr;
+    float *keep_sum = truncate ? reinterpret_cast<float *>(ws + align_up(n_rows * sizeof(uint32_t), 256)) : nullptr;
 
     const float c = (float)(1.4426950408889634 / (double)d->temperature);
     const int rows = d->B * d->N;
     row_stats_kernel<<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
                                                   row_sum);
     SR_LAUNCH_CHECK();
-
     WalkArgs wa;
     wa.logits = static_cast<const uint16_t *>(logits);
     wa.tree_tok = tree_tok;
@@ -556,7 +766,11 @@ extern "C" int specroll_verify(const specroll_verify_desc *d, const void *logits
     wa.k = d->k;
     wa.V = d->V;
     wa.T = (double)d->temperature;
-    walk_kernel<<<(d->B + WALK_WARPS - 1) / WALK_WARPS, WALK_WARPS * 32, 0, st>>>(wa, topo);
+    if (truncate)
+        walk_nucleus_kernel<<<d->B, NUC_THREADS, 0, st>>>(wa, topo, c, top_p, thr_key, keep_sum, nucleus_thr,
+                                                           nucleus_sum);
+    else
+        walk_kernel<<<(d->B + WALK_WARPS - 1) / WALK_WARPS, WALK_WARPS * 32, 0, st>>>(wa, topo);
     SR_LAUNCH_CHECK();
 
     TermArgs ta;
@@ -568,6 +782,7 @@ extern "C" int specroll_verify(const specroll_verify_desc *d, const void *logits
     ta.ws_nov = ws_nov;
     ta.ws_ovid = ws_ovid;
     ta.ws_ovm = ws_ovm;
+    ta.thr_key = thr_key;
     ta.out_tok = out_tok;
     ta.B = d->B;
     ta.N = d->N;
@@ -576,6 +791,34 @@ extern "C" int specroll_verify(const specroll_verify_desc *d, const void *logits
     ta.V = d->V;
     ta.c = c;
     return launch_terminal(ta, st);
+}
+
+extern "C" int specroll_verify(const specroll_verify_desc *d, const void *logits,
+                               const int32_t *parent_host, const int32_t *tree_tok,
+                               const uint8_t *tree_cand, const int32_t *cand_id,
+                               const float *cand_logit, const float *u_acc, const float *u_fin,
+                               int32_t *n_acc, int32_t *path_node, int32_t *out_tok,
+                               int32_t *term_node, int32_t *term_kind, float *row_max,
+                               float *row_sum, float *min_margin, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream) {
+    return run_verify(d, 1.0f, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
+                      path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, nullptr, nullptr,
+                      workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" int specroll_verify_nucleus(const specroll_verify_desc *d, float top_p, const void *logits,
+                                       const int32_t *parent_host, const int32_t *tree_tok,
+                                       const uint8_t *tree_cand, const int32_t *cand_id,
+                                       const float *cand_logit, const float *u_acc, const float *u_fin,
+                                       int32_t *n_acc, int32_t *path_node, int32_t *out_tok,
+                                       int32_t *term_node, int32_t *term_kind, float *row_max,
+                                       float *row_sum, float *min_margin, float *nucleus_thr,
+                                       float *nucleus_sum, void *workspace, size_t workspace_bytes,
+                                       void *cuda_stream) {
+    if (!(top_p > 0.f)) return SPECROLL_EINVAL;
+    return run_verify(d, top_p, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
+                      path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, nucleus_thr,
+                      nucleus_sum, workspace, workspace_bytes, cuda_stream);
 }
 
 // ------------------------------------------------------------------------------ allocation-free variant

@@ -32,9 +32,11 @@ def _randn_bf16(gen, shape, std, device):
 class StepWorkload:
     """All tensors of one step for workload ``w`` on ``device`` (seed offset for replicas)."""
 
-    def __init__(self, w: I.Workload, device, seed: int = 0, layers: int | None = None, paged: bool = False):
+    def __init__(self, w: I.Workload, device, seed: int = 0, layers: int | None = None, paged: bool = False,
+                 top_p: float | None = None):
         self.w = w
         self.paged = bool(paged)
+        self.top_p = top_p if (top_p is not None and 0.0 < top_p < 1.0) else None
         self.device = device
         self.layers = int(layers if layers is not None else w.layers)
         gen = torch.Generator(device=device)
@@ -105,7 +107,7 @@ class StepWorkload:
         ws_bytes = (S.tree_attn_paged_workspace_bytes(B, N, w.Hq, w.Hkv, w.D, self.kv_len_host) if self.paged else
                     S.tree_attn_workspace_bytes(B, N, w.Hq, w.Hkv, w.D, self.kv_indptr_host))
         self.ws_attn = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
-        self.ws_verify = torch.empty(S.verify_workspace_bytes(B, N, K, k, V, w.temperature),
+        self.ws_verify = torch.empty(S.verify_nucleus_workspace_bytes(B, N, K, k, V, w.temperature),
                                      dtype=torch.uint8, device=device)
         self.prop = None
         self.ver = None
@@ -158,6 +160,11 @@ class StepWorkload:
 
     def verify(self):
         p = self.prop
+        if self.top_p is not None:
+            self.ver = S.verify_nucleus(self.logits, self.parent, p["tree_tok"], p["tree_cand"], p["cand_id"],
+                                        p["cand_logit"], self.u_acc, self.u_fin, self.top_p,
+                                        temperature=self.w.temperature, workspace=self.ws_verify, out=self.ver)
+            return self.ver
         self.ver = S.verify(self.logits, self.parent, p["tree_tok"], p["tree_cand"], p["cand_id"],
                             p["cand_logit"], self.u_acc, self.u_fin, temperature=self.w.temperature,
                             workspace=self.ws_verify, out=self.ver)
