@@ -144,6 +144,11 @@ typedef struct {
 size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *desc,
                                           const int32_t *kv_indptr_host);
 
+/* Number of kernels one specroll_tree_attn call with this descriptor and these lengths enqueues
+ * (plan kernel unless the plan is reused, attention kernel, merge kernel when a sequence is cut into
+ * many chunks); -1 for an invalid descriptor.  (Housekeeping for reports; the paper has no counterpart.) */
+int specroll_tree_attn_launches(const specroll_attn_desc *desc, const int32_t *kv_indptr_host);
+
 int specroll_tree_attn(const specroll_attn_desc *desc, const void *Q, const void *Kc,
                        const void *Vc, const int32_t *kv_indptr_dev,
                        const int32_t *kv_indptr_host, const void *Kt, const void *Vt,

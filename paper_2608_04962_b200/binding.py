@@ -21,7 +21,7 @@ _lib = None
 EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
            "specroll_propose_workspace_bytes", "specroll_propose", "specroll_workspace_status",
            "specroll_tree_draw",
-           "specroll_tree_attn_workspace_bytes", "specroll_tree_attn",
+           "specroll_tree_attn_workspace_bytes", "specroll_tree_attn", "specroll_tree_attn_launches",
            "specroll_tree_attn_paged_workspace_bytes", "specroll_tree_attn_paged",
            "specroll_commit_path", "specroll_commit_path_layers", "specroll_gather_hidden",
            "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static",
@@ -75,7 +75,8 @@ def lib():
             getattr(l, n).restype = C.c_size_t
         for n in ("specroll_propose", "specroll_workspace_status", "specroll_tree_draw", "specroll_tree_attn",
                   "specroll_verify", "specroll_verify_static", "specroll_tree_attn_paged", "specroll_commit_path",
-                  "specroll_commit_path_layers", "specroll_gather_hidden", "specroll_verify_nucleus"):
+                  "specroll_commit_path_layers", "specroll_gather_hidden", "specroll_verify_nucleus",
+                  "specroll_tree_attn_launches"):
             getattr(l, n).restype = C.c_int
         _lib = l
     return _lib
@@ -205,6 +206,13 @@ def tree_attn_workspace_bytes(B, N, Hq, Hkv, D, kv_indptr_host, scale=None) -> i
     ip = _host_i32(kv_indptr_host, "kv_indptr_host")
     desc = AttnDesc(B, N, Hq, Hkv, D, scale if scale is not None else 1.0 / float(np.sqrt(D)), 0)
     return int(lib().specroll_tree_attn_workspace_bytes(C.byref(desc), ip.ctypes.data_as(C.c_void_p)))
+
+
+def tree_attn_launches(B, N, Hq, Hkv, D, kv_indptr_host, flags: int = 0) -> int:
+    """Kernels one tree_attn call enqueues for these lengths (the plan decides whether a merge kernel runs)."""
+    ip = _host_i32(kv_indptr_host, "kv_indptr_host")
+    desc = AttnDesc(B, N, Hq, Hkv, D, 1.0 / float(np.sqrt(D)), flags)
+    return int(lib().specroll_tree_attn_launches(C.byref(desc), ip.ctypes.data_as(C.c_void_p)))
 
 
 def tree_attn(Q, Kc, Vc, kv_indptr_dev, kv_indptr_host, Kt, Vt, parent, scale=None, want_lse=False,

@@ -658,6 +658,15 @@ extern "C" size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *d
     return p.total;
 }
 
+extern "C" int specroll_tree_attn_launches(const specroll_attn_desc *d, const int32_t *kv_indptr_host) {
+    AttnPlan p;
+    if (make_attn_plan(d, kv_indptr_host, &p) != SPECROLL_OK) return -1;
+    if (d->B == 0) return 0;
+    const bool split = p.items > d->B;
+    if (p.use_tc) return ((d->flags & SPECROLL_ATTN_REUSE_PLAN) ? 0 : 1) + 1 + ((p.merge_mode == 2 && split) ? 1 : 0);
+    return 1 + 1 + (split ? 1 : 0);
+}
+
 // Common body of the two entry points.  Contiguous cache: kv_indptr_dev, T_kv = cached tokens.  Paged cache:
 // kv_len_dev, page_indptr_dev, page_table_dev, T_kv = tokens in the page pool.  indptr_host is the (derived)
 // prefix of the host lengths either way.

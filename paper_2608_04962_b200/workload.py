@@ -186,11 +186,16 @@ class StepWorkload:
             events[3].record()
 
     # ---- bookkeeping for the report
-    LAUNCHES_PROPOSE, LAUNCHES_ATTN, LAUNCHES_VERIFY = 6, 2, 3   # kernels per call
+    LAUNCHES_PROPOSE, LAUNCHES_VERIFY = 6, 3   # kernels per call (layernorm, heads, correction, projection, merge,
+    #                                            draw; row statistics, walk, terminal draw)
 
     def launches_per_step(self) -> int:
-        # the attention prep kernel runs for the first layer only (the plan is reused afterwards)
-        return self.LAUNCHES_PROPOSE + 1 + self.layers * (self.LAUNCHES_ATTN - 1) + self.LAUNCHES_VERIFY
+        # the library says how many kernels an attention call enqueues: the plan kernel runs for the first layer
+        # only (the plan is reused afterwards), a merge kernel only when a sequence is cut into many chunks
+        w = self.w
+        first = S.tree_attn_launches(w.B, w.N, w.Hq, w.Hkv, w.D, self.kv_indptr_host)
+        later = S.tree_attn_launches(w.B, w.N, w.Hq, w.Hkv, w.D, self.kv_indptr_host, flags=S.ATTN_REUSE_PLAN)
+        return self.LAUNCHES_PROPOSE + first + (self.layers - 1) * later + self.LAUNCHES_VERIFY
 
     def tokens_per_step(self) -> int:
         return self.w.B * self.w.N
