@@ -103,90 +103,216 @@ constexpr int NUC_THREADS = 512;
 
 // Nucleus of one row (sampling configuration of the experiments: threshold 0.95): tokens are taken in order of
 // decreasing probability until their mass first reaches top_p, and every token that ties with the last one
-// taken is kept too.  Equal probabilities are equal bf16 logits, so the kept set is "key >= threshold key", and
-// the threshold is found by a radix search over the 16 key bits, four bits per pass: each pass adds up, per
-// value of the next four bits, the mass of the tokens whose leading bits match the digits found so far
-// (private bins per thread in shared memory, no atomics), and picks the digit at which the mass from the top
-// reaches top_p * S.  Run by all NUC_THREADS threads of a CTA; the row comes from HBM once and from L2 after.
-// Leaves in st->prefix the threshold key (a token is kept iff ord_key(logit) >= key) and in st->keep the sum of
-// the kept exp((l - M)/T).
+// taken is kept too.  Equal probabilities are equal bf16 logits, so the kept set is "key >= threshold key".
+// Run by all NUC_THREADS threads of a CTA; the row comes from HBM once and from L2 after.  Result: st->prefix =
+// threshold key (a token is kept iff ord_key(logit) >= key), st->keep = sum of the kept exp((l - M)/T).
+//
+// The threshold is searched from coarse to exact:
+//   A  sixteen bins of the distance below the maximum, e = (M - l) c in log2 units, two units wide (the last bin
+//      takes everything beyond 30): per-thread private bins in shared memory, no atomics; the bin where the mass
+//      from the top reaches top_p * S is selected;
+//   B  the same inside the selected bin, sixteen sub-bins of 1/8 unit;
+//   C  the keys of the tokens in the selected sub-bin are collected in shared memory (a few thousand at most);
+//   D  a radix search over the 16 key bits, four per pass, on that list alone finds the exact key.
+// A and B cost about a dozen instructions per token, C half of that; the bin index is the argument of the
+// exponential, which is needed anyway.  If the threshold lies in the catch-all bin or the list overflows, the
+// radix search runs over the whole row instead (nucleus_row_radix; same result, four full passes).
+constexpr int NUC_LIST = 8192;
+constexpr float NUC_WA = 2.0f, NUC_WB = 0.125f;
+
 struct NucleusSmem {
     float bins[16][NUC_THREADS];
     float wsum[NUC_THREADS / 32][16];
+    unsigned short list[NUC_LIST];
+    int n_list;
+    int sel;  // bin selected by the last level
     float above, keep;
     uint32_t prefix;
 };
 
-__device__ void nucleus_row(const uint16_t *__restrict__ row_logits, int V, float c, float M, float target,
-                            NucleusSmem *st) {
+// Sums the sixteen private bins over the block; thread 0 then picks, from the first bin on, the bin at which
+// above + running mass reaches the target (or the last bin with mass if rounding keeps the total below it) and
+// leaves it in st->sel, the mass before it in st->above and the mass up to and including it in st->keep.
+__device__ void nucleus_pick(NucleusSmem *st, float target, bool top_is_high_index) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint4 *p = reinterpret_cast<const uint4 *>(row_logits);
-    const int nvec = V >> 3;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const float x = warp_sum(st->bins[j][tid]);
+        if (lane == 0) st->wsum[warp][j] = x;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float tot[16];
+        for (int j = 0; j < 16; ++j) {
+            float x = 0.f;
+            for (int w2 = 0; w2 < NUC_THREADS / 32; ++w2) x += st->wsum[w2][j];
+            tot[top_is_high_index ? 15 - j : j] = x;  // tot[0] = most probable bin
+        }
+        float cum = st->above;
+        int sel = -1, last = 0;
+        for (int j = 0; j < 16; ++j)
+            if (tot[j] > 0.f) last = j;
+        for (int j = 0; j < 16; ++j) {
+            if (cum + tot[j] >= target) {
+                sel = j;
+                break;
+            }
+            cum += tot[j];
+        }
+        if (sel < 0) {
+            sel = last;
+            cum = st->above;
+            for (int j = 0; j < last; ++j) cum += tot[j];
+        }
+        st->above = cum;
+        st->keep = cum + tot[sel];
+        st->sel = top_is_high_index ? 15 - sel : sel;
+    }
+    __syncthreads();
+}
+
+// One radix pass of the key search: masses of the keys whose leading bits equal `prefix`, by their next four bits.
+__device__ __forceinline__ void nucleus_key_bin(NucleusSmem *st, uint32_t bits, int level, uint32_t prefix, float M,
+                                                float c) {
+    const int shift = 12 - 4 * level;
+    const uint32_t key = ord_key(bits);
+    if (level == 0 || (key >> (shift + 4)) == prefix)
+        st->bins[(key >> shift) & 15u][threadIdx.x] += ex2_approx((__uint_as_float(bits << 16) - M) * c);
+}
+
+// Exact search over the whole row (fallback): four passes, four key bits each.
+__device__ void nucleus_row_radix(const uint4 *__restrict__ p, int nvec, float c, float M, float target,
+                                  NucleusSmem *st) {
+    const int tid = threadIdx.x;
     if (tid == 0) {
         st->above = 0.f;
         st->prefix = 0u;
     }
     __syncthreads();
     for (int level = 0; level < 4; ++level) {
-        const int shift = 12 - 4 * level;
         const uint32_t prefix = st->prefix;
 #pragma unroll
         for (int j = 0; j < 16; ++j) st->bins[j][tid] = 0.f;
-        for (int i0 = tid; i0 < nvec; i0 += 4 * NUC_THREADS) {
-            uint4 vv[4];  // four independent loads in flight; an absent one reads as -inf (no mass, lowest key range)
+        for (int i = tid; i < nvec; i += NUC_THREADS) {
+            const uint4 v = ld_nc_v4(p + i);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int i = i0 + q * NUC_THREADS;
-                vv[q] = i < nvec ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    const uint32_t bits = (t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu);
-                    const uint32_t key = ord_key(bits);
-                    if (level == 0 || (key >> (shift + 4)) == prefix)
-                        st->bins[(key >> shift) & 15u][tid] += ex2_approx((__uint_as_float(bits << 16) - M) * c);
-                }
-            }
+            for (int t = 0; t < 8; ++t)
+                nucleus_key_bin(st, (t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu), level, prefix, M, c);
         }
-        // sixteen sums over the block
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const float x = warp_sum(st->bins[j][tid]);
-            if (lane == 0) st->wsum[warp][j] = x;
-        }
+        nucleus_pick(st, target, true);
+        if (tid == 0) st->prefix = (prefix << 4) | (uint32_t)st->sel;
         __syncthreads();
-        if (tid == 0) {
-            float tot[16];
-            for (int j = 0; j < 16; ++j) {
-                float x = 0.f;
-                for (int w2 = 0; w2 < NUC_THREADS / 32; ++w2) x += st->wsum[w2][j];
-                tot[j] = x;
-            }
-            // from the top digit down: first digit at which the mass reaches the target
-            float cum = st->above;
-            int sel = -1, low = 0;
-            for (int j = 15; j >= 0; --j) {
-                if (tot[j] > 0.f) low = j;
-            }
-            for (int j = 15; j >= 0; --j) {
-                if (cum + tot[j] >= target) {
-                    sel = j;
-                    break;
-                }
-                cum += tot[j];
-            }
-            if (sel < 0) {  // rounding kept the total below the target: keep everything
-                sel = low;
-                cum = st->above;
-                for (int j = 15; j > low; --j) cum += tot[j];
-            }
-            st->above = cum;
-            st->prefix = (prefix << 4) | (uint32_t)sel;
-            st->keep = cum + tot[sel];
+    }
+}
+
+__device__ void nucleus_row(const uint16_t *__restrict__ row_logits, int V, float c, float M, float target,
+                            NucleusSmem *st) {
+    const int tid = threadIdx.x;
+    const uint4 *p = reinterpret_cast<const uint4 *>(row_logits);
+    const int nvec = V >> 3;
+    const float Mc = M * c;
+    if (tid == 0) {
+        st->above = 0.f;
+        st->n_list = 0;
+    }
+    // the distance below the maximum, in log2 units, and the mass: e >= 0, mass = 2^-e
+    auto dist = [&](uint32_t bits) { return Mc - __uint_as_float(bits << 16) * c; };
+    // bin = e / width rounded to nearest, taken from the mantissa of e / width + 1.5 * 2^23 (float-to-int
+    // conversions share the special-function unit with the exponentials; this stays on the FMA and integer
+    // pipes).  Any monotone rule would do: the same one is used in every pass.
+    auto to_int = [](float x) { return (int)(__float_as_uint(x + 12582912.0f) - 0x4B400000u); };
+    auto bin_a = [&](float e) { return min(15, to_int(e * (1.0f / NUC_WA))); };
+    // ---- A
+#pragma unroll
+    for (int j = 0; j < 16; ++j) st->bins[j][tid] = 0.f;
+    __syncthreads();
+    for (int i0 = tid; i0 < nvec; i0 += 4 * NUC_THREADS) {
+        uint4 vv[4];  // four independent loads in flight; an absent one reads as -inf (no mass)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = i0 + q * NUC_THREADS;
+            vv[q] = i < nvec ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
         }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const float e = dist((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
+                st->bins[bin_a(e)][tid] += ex2_approx(-e);
+            }
+        }
+    }
+    nucleus_pick(st, target, false);
+    const int ja = st->sel;
+    if (ja == 15) {  // the cut lies among tokens 2^-30 below the maximum: exact search over the whole row
+        nucleus_row_radix(p, nvec, c, M, target, st);
+        return;
+    }
+    // ---- B
+    const float ea = ((float)ja - 0.5f) * NUC_WA;  // lower edge of bin ja under round-to-nearest
+    auto bin_b = [&](float e) { return max(0, min(15, to_int((e - ea) * (1.0f / NUC_WB)))); };
+#pragma unroll
+    for (int j = 0; j < 16; ++j) st->bins[j][tid] = 0.f;
+    for (int i0 = tid; i0 < nvec; i0 += 4 * NUC_THREADS) {
+        uint4 vv[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = i0 + q * NUC_THREADS;
+            vv[q] = i < nvec ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const float e = dist((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
+                if (bin_a(e) == ja) st->bins[bin_b(e)][tid] += ex2_approx(-e);
+            }
+        }
+    }
+    nucleus_pick(st, target, false);
+    const int jb = st->sel;
+    // ---- C
+    for (int i0 = tid; i0 < nvec; i0 += 4 * NUC_THREADS) {
+        uint4 vv[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = i0 + q * NUC_THREADS;
+            vv[q] = i < nvec ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const uint32_t bits = (t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu);
+                const float e = dist(bits);
+                if (bin_a(e) == ja && bin_b(e) == jb) {
+                    const int pos = atomicAdd(&st->n_list, 1);
+                    if (pos < NUC_LIST) st->list[pos] = (unsigned short)bits;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    const int n_list = st->n_list;
+    if (n_list > NUC_LIST) {  // more tokens in one sub-bin than the list holds: exact search over the whole row
+        __syncthreads();
+        nucleus_row_radix(p, nvec, c, M, target, st);
+        return;
+    }
+    // ---- D: st->above is the mass above the sub-bin; the key search runs on the list
+    if (tid == 0) st->prefix = 0u;
+    __syncthreads();
+    for (int level = 0; level < 4; ++level) {
+        const uint32_t prefix = st->prefix;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) st->bins[j][tid] = 0.f;
+        for (int i = tid; i < n_list; i += NUC_THREADS) nucleus_key_bin(st, st->list[i], level, prefix, M, c);
+        nucleus_pick(st, target, true);
+        if (tid == 0) st->prefix = (prefix << 4) | (uint32_t)st->sel;
         __syncthreads();
     }
 }
@@ -387,7 +513,8 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(WalkArgs a, Topo 
 __global__ void __launch_bounds__(NUC_THREADS)
 walk_nucleus_kernel(WalkArgs a, Topo topo, float c, float top_p, uint32_t *__restrict__ thr_key,
                     float *__restrict__ keep_sum, float *__restrict__ out_thr, float *__restrict__ out_sum) {
-    __shared__ NucleusSmem nuc;
+    extern __shared__ __align__(16) unsigned char nuc_raw[];  // NucleusSmem: above the static limit, hence dynamic
+    NucleusSmem &nuc = *reinterpret_cast<NucleusSmem *>(nuc_raw);
     __shared__ WalkSmem sm;
     __shared__ int sh_next;  // next node, or -1 when the walk is over
     const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -766,10 +893,16 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
     wa.k = d->k;
     wa.V = d->V;
     wa.T = (double)d->temperature;
-    if (truncate)
-        walk_nucleus_kernel<<<d->B, NUC_THREADS, 0, st>>>(wa, topo, c, top_p, thr_key, keep_sum, nucleus_thr,
-                                                           nucleus_sum);
-    else
+    if (truncate) {
+        static bool configured = false;
+        if (!configured) {
+            SR_CUDA_TRY(cudaFuncSetAttribute(walk_nucleus_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)sizeof(NucleusSmem)));
+            configured = true;
+        }
+        walk_nucleus_kernel<<<d->B, NUC_THREADS, sizeof(NucleusSmem), st>>>(wa, topo, c, top_p, thr_key, keep_sum,
+                                                                             nucleus_thr, nucleus_sum);
+    } else
         walk_kernel<<<(d->B + WALK_WARPS - 1) / WALK_WARPS, WALK_WARPS * 32, 0, st>>>(wa, topo);
     SR_LAUNCH_CHECK();
 
