@@ -393,6 +393,59 @@ def run_e2e(args, wl, dev, world):
             "ms_per_step": tmax / steps, "steps": steps}
 
 
+def run_calls(args, w, layers):
+    """Per-call timings, each entry point alone: 20 warm-up + 100 timed launches with CUDA events, median and
+    minimum; once with a 256 MB write between launches (cold L2: the roofline number) and once back to back.
+    Prints one JSON object (not the bench line)."""
+    import torch
+    from paper_2608_04962_b200.workload import StepWorkload
+    from paper_2608_04962_b200 import binding as S
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback of the hot path")
+    S.lib()
+    dev = torch.device("cuda", 0)
+    wl = StepWorkload(w, dev, layers=min(layers, 2), paged=args.paged, top_p=args.top_p)
+    peaks = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    wl.step()
+
+    def attn_planned():
+        wl.attn(0)
+
+    def attn_reuse():
+        wl.attn(1)
+
+    calls = {
+        "propose": (wl.propose, "tensor", (wl.lmhead_algorithmic_flops() + 2 * w.B * w.K * w.d * w.d) / 1e12,
+                    peaks["bf16_tflops"], "TFLOP/s"),
+        "tree_attn (plan kernel + attention)": (attn_planned, "hbm", wl.attn_algorithmic_bytes() / 1e9,
+                                                peaks["hbm_gbs"], "GB/s"),
+        "tree_attn (plan reused)": (attn_reuse, "hbm", wl.attn_algorithmic_bytes() / 1e9, peaks["hbm_gbs"], "GB/s"),
+        "verify": (wl.verify, "hbm", wl.rowstats_algorithmic_bytes() / 1e9, peaks["hbm_gbs"], "GB/s"),
+    }
+    out = {"workload": w.name, "peak_source": peaks["source"], "calls": {}}
+    for name, (fn, bound, work, peak, unit) in calls.items():
+        rec = {"bound": bound, "unit": unit, "peak": peak, "work_per_call": work}
+        for mode in ("cold_l2", "back_to_back"):
+            for _ in range(20):
+                fn()
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(100)]
+            for a, b in evs:
+                if mode == "cold_l2":
+                    flush.fill_(1)
+                a.record()
+                fn()
+                b.record()
+            torch.cuda.synchronize()
+            t = np.array([a.elapsed_time(b) for a, b in evs])
+            med, mn = float(np.median(t)), float(t.min())
+            rec[mode] = {"median_us": med * 1e3, "min_us": mn * 1e3, "achieved_median": work / (med * 1e-3),
+                         "frac_median": work / (med * 1e-3) / peak}
+        out["calls"][name] = rec
+    print(json.dumps(out), flush=True)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -410,12 +463,16 @@ def main():
     ap.add_argument("--paged", action="store_true",
                     help="keep the KV cache in 128-token pages (specroll_tree_attn_paged) and time the commit of the "
                          "accepted paths after the step as well (reported beside the step, not inside it)")
+    ap.add_argument("--calls", action="store_true",
+                    help="time each entry point alone (100 launches, cold and warm L2) instead of the step")
     args = ap.parse_args()
     from paper_2608_04962_b200 import inputs as I
     w = I.WORKLOADS[args.workload]
     layers = args.layers if args.layers is not None else w.layers
     if args.impl == "reference":
         return run_reference(args, w, layers)
+    if args.calls:
+        return run_calls(args, w, layers)
     return run_ours(args, w, layers)
 
 
