@@ -54,3 +54,27 @@ def test_descriptor_validation_needs_no_device(libpath):
     assert S.tree_attn_workspace_bytes(2, 8, 4, 2, 64, ip) > 0
     assert S.tree_attn_workspace_bytes(2, 8, 4, 3, 64, ip) == 0       # Hq % Hkv != 0
     assert S.tree_attn_workspace_bytes(2, 8, 4, 2, 96, ip) == 0       # head_dim
+
+
+def test_attention_plan_is_host_only_and_consistent(libpath):
+    """The planner (chunk length by simulated hand-out, cached per lengths) runs without a device."""
+    from paper_2608_04962_b200 import binding as S
+    from paper_2608_04962_b200 import inputs as I
+    for name in ("qwen1.5b", "qwen7b", "sweep7b_B8"):
+        w = I.WORKLOADS[name]
+        L = I.kv_lengths(w)
+        ip = np.zeros(w.B + 1, np.int32)
+        np.cumsum(L, out=ip[1:])
+        a = S.tree_attn_workspace_bytes(w.B, w.N, w.Hq, w.Hkv, w.D, ip)
+        b = S.tree_attn_workspace_bytes(w.B, w.N, w.Hq, w.Hkv, w.D, ip)          # second time from the cache
+        assert a == b and a > 0
+        assert S.tree_attn_paged_workspace_bytes(w.B, w.N, w.Hq, w.Hkv, w.D, L.astype(np.int32)) == a
+        first = S.tree_attn_launches(w.B, w.N, w.Hq, w.Hkv, w.D, ip)
+        later = S.tree_attn_launches(w.B, w.N, w.Hq, w.Hkv, w.D, ip, flags=S.ATTN_REUSE_PLAN)
+        assert first == later + 1 and later in (1, 2)                            # plan kernel only the first time
+    # a changed length changes the plan's key: no stale answer
+    ip2 = ip.copy()
+    ip2[-1] += 4096
+    assert S.tree_attn_workspace_bytes(w.B, w.N, w.Hq, w.Hkv, w.D, ip2) != 0
+    assert S.tree_attn_launches(w.B, w.N, w.Hq, w.Hkv, w.D, ip, flags=64) == -1  # unknown flag
+    assert S.verify_nucleus_workspace_bytes(4, 8, 3, 2, 1024) > S.verify_workspace_bytes(4, 8, 3, 2, 1024)
