@@ -195,6 +195,26 @@ def run_ours(args, w, layers):
     for _ in range(max(args.warmup, 3)):
         wl.step()
     torch.cuda.synchronize()
+    graph = None
+    if args.graph:
+        # the whole step as one CUDA graph: the entry points only enqueue work on the caller's stream (kernels,
+        # one memset; tensor maps travel as kernel arguments), so a step can be captured and replayed
+        try:
+            side = torch.cuda.Stream(dev)
+            side.wait_stream(torch.cuda.current_stream(dev))
+            with torch.cuda.stream(side):
+                wl.step()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    wl.step()
+            torch.cuda.current_stream(dev).wait_stream(side)
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+        except Exception as exc:                       # capture refused: time plain launches instead
+            print(f"bench: CUDA graph capture failed ({exc}); timing plain launches", file=sys.stderr)
+            graph = None
+            torch.cuda.synchronize()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -204,7 +224,10 @@ def run_ours(args, w, layers):
     t1 = torch.cuda.Event(enable_timing=True)
     t0.record()
     for i in range(args.steps):
-        wl.step(ev[i])
+        if graph is not None:
+            graph.replay()
+        else:
+            wl.step(ev[i])
     t1.record()
     torch.cuda.synchronize()
     D.barrier()
@@ -214,6 +237,12 @@ def run_ours(args, w, layers):
     tmax, tok_all = D.aggregate(elapsed_ms, tokens, device=dev)
     value = tok_all / (tmax * 1e-3)
 
+    if graph is not None:
+        # phase times are not visible inside a replayed graph: take them from a few plain steps afterwards
+        torch.cuda.synchronize()
+        for i in range(args.steps):
+            wl.step(ev[i])
+        torch.cuda.synchronize()
     prop_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
     attn_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
     ver_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))
@@ -286,7 +315,7 @@ def run_ours(args, w, layers):
                        "Hkv": w.Hkv, "D": w.D, "layers": wl.layers, "T_kv": wl.T_kv, "temperature": w.temperature,
                        "kv_cache": "128-token pages in a seeded random order (specroll_tree_attn_paged)" if args.paged
                        else "contiguous ragged (specroll_tree_attn)",
-                       "top_p": wl.top_p,
+                       "top_p": wl.top_p, "cuda_graph": graph is not None,
                        "parallelism": f"replicas x{world} (sharded by sequence, no collective)",
                        "l2": "inputs larger than L2: per-layer KV cache, logits and W each exceed 126 MB and every "
                              "layer has its own cache"},
@@ -463,6 +492,9 @@ def main():
     ap.add_argument("--paged", action="store_true",
                     help="keep the KV cache in 128-token pages (specroll_tree_attn_paged) and time the commit of the "
                          "accepted paths after the step as well (reported beside the step, not inside it)")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture the step in a CUDA graph and time replays instead of plain launches (the phase "
+                         "times and the roofline line then come from plain steps run afterwards)")
     ap.add_argument("--calls", action="store_true",
                     help="time each entry point alone (100 launches, cold and warm L2) instead of the step")
     args = ap.parse_args()
