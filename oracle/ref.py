@@ -296,3 +296,77 @@ def commit_path(Kt, Vt, path_node, n_acc, Kp, Vp, page_table, page_indptr, kv_le
 def gather_hidden(hidden, term_node):
     hidden, term_node = _as(hidden, np.uint16), _as(term_node, np.int32)
     return np.stack([hidden[b, term_node[b]] for b in range(hidden.shape[0])])
+
+
+# ----------------------------------------------------------------------------------- verifier feedback
+def reflex_feedback(logits_rows, W, cand_id, cand_logit, y_star, m, rho, k_support, temperature=1.0, eps=1e-6):
+    """Verifier-derived feedback of matured proposals and the memory update (Sec. 3.3 / 3.4: Eq. "support",
+    "distdir", "covdir", the RMS normalisation, Eq. "unified-feedback", Eq. "ema"; the magnitudes d_dist and
+    d_cov from Eq. "acceptance-gap-decomposition").  One record per row, written out step by step in fp64:
+
+      p = softmax(logits / T) over the vocabulary; q = softmax(cand_logit / T) on the k candidates C, zero elsewhere
+      S = C  u  Top_kS(p)  u  {y*}                (ties of Top by (logit desc, id asc))
+      p_S, q_S = p, q renormalised on S           (q lives on C, a subset of S, so q_S = q)
+      r_dist = sum_{v in S} (p_S(v) - q_S(v)) W_v
+      C* = Top_k(p),  O = C* \\ C,  b* = weakest candidate (last of the list, which is sorted by logit)
+      r_cov = sum_{y in O} p_S(y) (W_y - W_b*)
+      d_dist = p(C) TV(p_C, q_C),  d_cov = p(C*) - p(C)
+      rbar = r / (RMS(r) + eps);  g = d_dist rbar_dist + d_cov rbar_cov;  e = (d_dist + d_cov) g / (RMS(g) + eps)
+      m <- rho m + (1 - rho) e
+
+    logits_rows [R,V] and W [V,d] are bf16 bit patterns; m [R,d], rho [R] floats.  Returns the new memory and the
+    intermediate quantities."""
+    logits_rows, W = _as(logits_rows, np.uint16), _as(W, np.uint16)
+    cand_id, y_star = _as(cand_id, np.int32), _as(y_star, np.int32)
+    cand_logit = np.asarray(cand_logit, np.float32).astype(np.float64)
+    m = np.asarray(m, np.float64)
+    rho = np.asarray(rho, np.float64)
+    R, V = logits_rows.shape
+    k = cand_id.shape[1]
+    d = W.shape[1]
+    T = float(np.float32(temperature))
+    if k_support < k:
+        raise ValueError("the support budget must cover the target's top-k (k_support >= k)")
+    Wf = (W.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    out = {"m": np.empty((R, d)), "e": np.empty((R, d)), "d_dist": np.empty(R), "d_cov": np.empty(R),
+           "tv": np.empty(R), "p_C": np.empty(R), "support": []}
+    rms = lambda v: np.sqrt(np.mean(v * v))
+    for r in range(R):
+        l = (logits_rows[r].astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        p = np.exp((l - l.max()) / T)
+        p /= p.sum()
+        C = [int(c) for c in cand_id[r]]
+        q_c = np.exp((cand_logit[r] - cand_logit[r].max()) / T)
+        q_c /= q_c.sum()
+        order = np.lexsort((np.arange(V), -l))            # by (logit desc, id asc)
+        top_s = [int(v) for v in order[:k_support]]
+        S = []
+        for v in C + top_s + [int(y_star[r])]:
+            if v not in S:
+                S.append(v)
+        pS = {v: p[v] for v in S}
+        tot = sum(pS.values())
+        pS = {v: x / tot for v, x in pS.items()}
+        qS = {v: 0.0 for v in S}
+        for j, c in enumerate(C):
+            qS[c] += q_c[j]
+        r_dist = np.zeros(d)
+        for v in S:
+            r_dist += (pS[v] - qS[v]) * Wf[v]
+        c_star = [int(v) for v in order[:k]]
+        O = [v for v in c_star if v not in C]
+        b_star = C[-1]
+        r_cov = np.zeros(d)
+        for y in O:
+            r_cov += pS[y] * (Wf[y] - Wf[b_star])
+        pC = sum(p[c] for c in C)
+        tv = 0.5 * sum(abs(p[c] / pC - q_c[j]) for j, c in enumerate(C))
+        d_dist = pC * tv
+        d_cov = sum(p[v] for v in c_star) - pC
+        g = d_dist * r_dist / (rms(r_dist) + eps) + d_cov * r_cov / (rms(r_cov) + eps)
+        e = (d_dist + d_cov) * g / (rms(g) + eps)
+        out["m"][r] = rho[r] * m[r] + (1.0 - rho[r]) * e
+        out["e"][r] = e
+        out["d_dist"][r], out["d_cov"][r], out["tv"][r], out["p_C"][r] = d_dist, d_cov, tv, pC
+        out["support"].append(S)
+    return out
