@@ -452,6 +452,33 @@ def run_calls(args, w, layers):
         "tree_attn (plan reused)": (attn_reuse, "hbm", wl.attn_algorithmic_bytes() / 1e9, peaks["hbm_gbs"], "GB/s"),
         "verify": (wl.verify, "hbm", wl.rowstats_algorithmic_bytes() / 1e9, peaks["hbm_gbs"], "GB/s"),
     }
+    # the feedback call on one matured record per (sequence, head): a node of the matching depth, a random realised token
+    R = w.B * w.K
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(5)
+    depth = np.zeros(w.N, np.int64)
+    for n in range(1, w.N):
+        depth[n] = depth[wl.parent[n]] + 1
+    node_of_head = [int(np.flatnonzero(depth == min(h, depth.max()))[0]) for h in range(w.K)]
+    rec_row = (torch.arange(w.B, device=dev)[:, None] * w.N +
+               torch.tensor(node_of_head, device=dev)[None, :]).reshape(-1).to(torch.int32).contiguous()
+    rec_mem = torch.arange(R, device=dev, dtype=torch.int32)
+    y_star = torch.randint(0, w.V, (R,), generator=gen, device=dev, dtype=torch.int32)
+    rho = torch.full((R,), 0.9, device=dev)
+    mem = wl.m.reshape(R, w.d).clone()
+    k_support = 48
+    fb_ws = torch.empty(R * k_support * 4 + 512, dtype=torch.uint8, device=dev)
+    cid = wl.prop["cand_id"].reshape(R, w.k).contiguous()
+    clg = wl.prop["cand_logit"].reshape(R, w.k).contiguous()
+    rmax = wl.ver["row_max"].reshape(-1).contiguous()
+    rsum = wl.ver["row_sum"].reshape(-1).contiguous()
+
+    def feedback():
+        S.reflex_feedback(wl.logits, rec_row, rmax, rsum, cid, clg, y_star, wl.W, rho, rec_mem, mem, k_support,
+                          temperature=w.temperature, workspace=fb_ws)
+
+    fb_bytes = (R * w.V * 2 + R * (w.k + k_support + 1) * w.d * 2 + 2 * R * w.d * 4) / 1e9
+    calls["reflex_feedback (B K records, support 48)"] = (feedback, "hbm", fb_bytes, peaks["hbm_gbs"], "GB/s")
     out = {"workload": w.name, "peak_source": peaks["source"], "calls": {}}
     for name, (fn, bound, work, peak, unit) in calls.items():
         rec = {"bound": bound, "unit": unit, "peak": peak, "work_per_call": work}

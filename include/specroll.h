@@ -215,6 +215,42 @@ int specroll_gather_hidden(int32_t B, int32_t N, int32_t d, const void *hidden,
                            const int32_t *term_node, void *h_next, void *cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Verifier-derived feedback of matured proposals and the trajectory memory update (Sec. 3.3 Eq.
+ * "acceptance-gap-decomposition"; Sec. 3.4 Eq. "support", "distdir", "covdir", "unified-feedback",
+ * "ema").  It produces the memory m that specroll_propose consumes.  Per record r (one matured
+ * proposal node), with p = softmax(logits[rec_row[r]] / T) and q = softmax(cand_logit[r] / T) on the
+ * candidates C = cand_id[r, :] (sorted by logit, as specroll_propose writes them):
+ *   S = C u Top_kS(p) u {y_star[r]};  p_S, q_S = p, q renormalised on S
+ *   r_dist = sum_{v in S} (p_S(v) - q_S(v)) W_v
+ *   C* = Top_k(p), O = C* \ C, b* = weakest (last) candidate;  r_cov = sum_{y in O} p_S(y) (W_y - W_b*)
+ *   d_dist = p(C) TV(p_C, q_C),  d_cov = p(C*) - p(C)
+ *   rbar = r / (RMS(r) + eps);  g = d_dist rbar_dist + d_cov rbar_cov;  e = (d_dist + d_cov) g / (RMS(g) + eps)
+ *   m[rec_mem[r], :] <- rho[r] m[rec_mem[r], :] + (1 - rho[r]) e
+ * Top sets are ordered by (logit desc, id asc).  k <= k_support <= 64 (the support must cover the target's
+ * top-k).  The records of one call must address distinct memory rows.
+ *
+ * Shapes (device): logits[rows, V] bf16 with row_max, row_sum[rows] fp32 as specroll_verify wrote them;
+ * rec_row, rec_mem, y_star[R] i32; cand_id[R,k] i32; cand_logit[R,k] fp32; W[V,d] bf16; rho[R] fp32;
+ * m[mem_rows, d] fp32 in/out; d_dist, d_cov, tv[R] fp32 outputs, each nullable.
+ * What the paper builds on top (severity, discarding, sketches, reliability score, the choice of alpha) is
+ * left to the caller: it needs only these outputs. */
+typedef struct {
+    int32_t R, k, k_support, d, V;
+    float temperature;
+    float eps;     /* RMS stabiliser (> = 0) */
+    int32_t flags; /* reserved, must be 0 */
+} specroll_feedback_desc;
+
+size_t specroll_reflex_feedback_workspace_bytes(const specroll_feedback_desc *desc);
+
+int specroll_reflex_feedback(const specroll_feedback_desc *desc, const void *logits,
+                             const int32_t *rec_row, const float *row_max, const float *row_sum,
+                             const int32_t *cand_id, const float *cand_logit, const int32_t *y_star,
+                             const void *W, const float *rho, const int32_t *rec_mem, float *m,
+                             float *d_dist, float *d_cov, float *tv, void *workspace,
+                             size_t workspace_bytes, void *cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * Exact target verification (App. B.2 Eq. "nodeaccept" / "noderesidual", Algorithm "Exact
  * node-wise tree verification").
  *

@@ -25,7 +25,8 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
            "specroll_tree_attn_paged_workspace_bytes", "specroll_tree_attn_paged",
            "specroll_commit_path", "specroll_commit_path_layers", "specroll_gather_hidden",
            "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static",
-           "specroll_verify_nucleus_workspace_bytes", "specroll_verify_nucleus")
+           "specroll_verify_nucleus_workspace_bytes", "specroll_verify_nucleus",
+           "specroll_reflex_feedback_workspace_bytes", "specroll_reflex_feedback")
 
 
 PROPOSE_LEGACY_MMA = 1
@@ -55,6 +56,11 @@ class VerifyDesc(C.Structure):
                 ("V", C.c_int32), ("temperature", C.c_float), ("flags", C.c_int32)]
 
 
+class FeedbackDesc(C.Structure):
+    _fields_ = [("R", C.c_int32), ("k", C.c_int32), ("k_support", C.c_int32), ("d", C.c_int32), ("V", C.c_int32),
+                ("temperature", C.c_float), ("eps", C.c_float), ("flags", C.c_int32)]
+
+
 def lib():
     """The loaded library.  Raises if it is missing: the CUDA path is the only path."""
     global _lib
@@ -71,12 +77,12 @@ def lib():
         l.specroll_node_budget.argtypes = [C.c_int32] * 4
         for n in ("specroll_propose_workspace_bytes", "specroll_verify_workspace_bytes",
                   "specroll_tree_attn_workspace_bytes", "specroll_tree_attn_paged_workspace_bytes",
-                  "specroll_verify_nucleus_workspace_bytes"):
+                  "specroll_verify_nucleus_workspace_bytes", "specroll_reflex_feedback_workspace_bytes"):
             getattr(l, n).restype = C.c_size_t
         for n in ("specroll_propose", "specroll_workspace_status", "specroll_tree_draw", "specroll_tree_attn",
                   "specroll_verify", "specroll_verify_static", "specroll_tree_attn_paged", "specroll_commit_path",
                   "specroll_commit_path_layers", "specroll_gather_hidden", "specroll_verify_nucleus",
-                  "specroll_tree_attn_launches"):
+                  "specroll_tree_attn_launches", "specroll_reflex_feedback"):
             getattr(l, n).restype = C.c_int
         _lib = l
     return _lib
@@ -434,6 +440,33 @@ def verify_nucleus(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_a
         _dev(out.get("nucleus_thr"), f32, "nucleus_thr"), _dev(out.get("nucleus_sum"), f32, "nucleus_sum"),
         C.c_void_p(workspace.data_ptr()), C.c_size_t(workspace.numel()), _stream())
     _check(rc, "specroll_verify_nucleus")
+    return out
+
+
+def reflex_feedback(logits, rec_row, row_max, row_sum, cand_id, cand_logit, y_star, W, rho, rec_mem, m, k_support,
+                    temperature=1.0, eps=1e-6, workspace=None):
+    """specroll_reflex_feedback: verifier feedback of R matured records, memory ``m`` updated in place.
+    logits [rows, V] bf16 (any leading shape), row_max/row_sum [rows]; returns d_dist, d_cov, tv [R]."""
+    V = logits.shape[-1]
+    R, k = cand_id.shape
+    d = W.shape[1]
+    desc = FeedbackDesc(R, k, k_support, d, V, temperature, eps, 0)
+    dev = logits.device
+    f32, i32 = torch.float32, torch.int32
+    out = {n: torch.empty(R, dtype=f32, device=dev) for n in ("d_dist", "d_cov", "tv")}
+    need = lib().specroll_reflex_feedback_workspace_bytes(C.byref(desc))
+    if need == 0:
+        raise SpecrollError("reflex_feedback: invalid descriptor")
+    if workspace is None:
+        workspace = _workspace(need, dev)
+    rc = lib().specroll_reflex_feedback(
+        C.byref(desc), _dev(logits, torch.bfloat16, "logits"), _dev(rec_row, i32, "rec_row"),
+        _dev(row_max, f32, "row_max"), _dev(row_sum, f32, "row_sum"), _dev(cand_id, i32, "cand_id"),
+        _dev(cand_logit, f32, "cand_logit"), _dev(y_star, i32, "y_star"), _dev(W, torch.bfloat16, "W"),
+        _dev(rho, f32, "rho"), _dev(rec_mem, i32, "rec_mem"), _dev(m, f32, "m"), _dev(out["d_dist"], f32, "d_dist"),
+        _dev(out["d_cov"], f32, "d_cov"), _dev(out["tv"], f32, "tv"), C.c_void_p(workspace.data_ptr()),
+        C.c_size_t(workspace.numel()), _stream())
+    _check(rc, "specroll_reflex_feedback")
     return out
 
 

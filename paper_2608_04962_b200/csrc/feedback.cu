@@ -1,0 +1,442 @@
+// Verifier-derived feedback of matured proposals and the trajectory memory update (Sec. 3.3 Eq.
+// "acceptance-gap-decomposition"; Sec. 3.4 Eq. "support", "distdir", "covdir", the RMS normalisation, Eq.
+// "unified-feedback", Eq. "ema").  Per record (one matured proposal node):
+//
+//   p = softmax(logits / T) over the vocabulary; q = softmax(cand_logit / T) on the k candidates C
+//   S = C  u  Top_kS(p)  u  {y*};   p_S, q_S = p, q renormalised on S (q lives on C, so q_S = q)
+//   r_dist = sum_{v in S} (p_S(v) - q_S(v)) W_v
+//   C* = Top_k(p),  O = C* \ C,  b* = weakest candidate;   r_cov = sum_{y in O} p_S(y) (W_y - W_b*)
+//   d_dist = p(C) TV(p_C, q_C),   d_cov = p(C*) - p(C)
+//   rbar = r / (RMS(r) + eps);  g = d_dist rbar_dist + d_cov rbar_cov;  e = (d_dist + d_cov) g / (RMS(g) + eps)
+//   m <- rho m + (1 - rho) e
+//
+// Two kernels, one CTA per record each:
+//   feedback_topk_kernel   exact Top_kS of the record's logits row, ordered by (logit desc, id asc): a radix
+//                          search over the 16-bit order-preserving keys of the bf16 logits by COUNT (four bits per
+//                          pass) finds the key of the kS-th largest value; a pass collects the ids above it, an
+//                          ordered pass the first ids that tie with it; a rank sort orders the kS winners.
+//   feedback_kernel        the small quantities (q, p on S, the coefficient of every support row) by one warp,
+//                          then all threads gather the <= k + kS + 1 rows of W once and accumulate both
+//                          directions, three RMS reductions, and the memory update.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace specroll {
+
+namespace fb {
+constexpr int TOPK_THREADS = 512;
+constexpr int FB_THREADS = 256;
+constexpr int MAX_S = 2 * SPECROLL_MAX_TOPK + 1;  // candidates + Top_kS + y*
+
+__device__ __forceinline__ uint32_t ord_key16(uint32_t bits) {
+    if (bits == 0x8000u) bits = 0u;  // -0 counts as +0
+    return (bits & 0x8000u) ? (~bits & 0xffffu) : (bits | 0x8000u);
+}
+
+template <int THREADS>
+__device__ __forceinline__ int block_sum_int(int v, int *red) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    int t = 0;
+    for (int w = 0; w < THREADS / 32; ++w) t += red[w];
+    return t;
+}
+
+template <int THREADS>
+__device__ __forceinline__ float block_sum_f(float v, float *red) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int w = 0; w < THREADS / 32; ++w) t += red[w];
+    return t;
+}
+}  // namespace fb
+
+// top_id[r, 0..kS): ids of the kS largest logits of row rec_row[r], by (logit desc, id asc).
+__global__ void __launch_bounds__(fb::TOPK_THREADS)
+feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restrict__ rec_row, int V, int kS,
+                     int32_t *__restrict__ top_id) {
+    using namespace fb;
+    __shared__ int bins[16][TOPK_THREADS];
+    __shared__ int wsum[TOPK_THREADS / 32][16];
+    __shared__ int red[TOPK_THREADS / 32];
+    __shared__ int sh_above, sh_prefix, sh_n;
+    __shared__ int sel_id[SPECROLL_MAX_TOPK];
+    __shared__ uint32_t sel_key[SPECROLL_MAX_TOPK];
+    const int r = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint16_t *row = logits + (size_t)rec_row[r] * V;
+    const uint4 *p = reinterpret_cast<const uint4 *>(row);
+    const int nvec = V >> 3;
+    if (tid == 0) {
+        sh_above = 0;
+        sh_prefix = 0;
+        sh_n = 0;
+    }
+    __syncthreads();
+    // ---- key of the kS-th largest value: four radix passes over the counts
+    for (int level = 0; level < 4; ++level) {
+        const int shift = 12 - 4 * level;
+        const uint32_t prefix = (uint32_t)sh_prefix;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) bins[j][tid] = 0;
+        for (int i = tid; i < nvec; i += TOPK_THREADS) {
+            const uint4 v = ld_nc_v4(p + i);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const uint32_t key = ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
+                if (level == 0 || (key >> (shift + 4)) == prefix) bins[(key >> shift) & 15u][tid] += 1;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            int x = bins[j][tid];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            if (lane == 0) wsum[warp][j] = x;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int cum = sh_above, sel = 0;
+            for (int j = 15; j >= 0; --j) {
+                int tot = 0;
+                for (int w2 = 0; w2 < TOPK_THREADS / 32; ++w2) tot += wsum[w2][j];
+                if (cum + tot >= kS) {  // the kS-th largest has this digit
+                    sel = j;
+                    break;
+                }
+                cum += tot;
+                sel = j;  // (fewer than kS values in the row: ends at the lowest digit)
+            }
+            sh_above = cum;  // values whose key is larger than every key with this prefix
+            sh_prefix = (int)((prefix << 4) | (uint32_t)sel);
+        }
+        __syncthreads();
+    }
+    const uint32_t thr = (uint32_t)sh_prefix;
+    const int n_above = sh_above;           // keys strictly above the threshold key: all of them are winners
+    const int need = max(0, kS - n_above);  // winners among the ties, lowest ids first
+    // ---- winners above the threshold (any order; sorted below)
+    for (int i = tid; i < nvec; i += TOPK_THREADS) {
+        const uint4 v = ld_nc_v4(p + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const uint32_t key = ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
+            if (key > thr) {
+                const int pos = atomicAdd(&sh_n, 1);
+                if (pos < SPECROLL_MAX_TOPK) {
+                    sel_id[pos] = i * 8 + t;
+                    sel_key[pos] = key;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // ---- the first `need` ties in id order: every thread takes a contiguous piece of the row
+    {
+        const int per = (nvec + TOPK_THREADS - 1) / TOPK_THREADS;
+        const int lo = min(nvec, tid * per), hi = min(nvec, lo + per);
+        int cnt = 0;
+        for (int i = lo; i < hi; ++i) {
+            const uint4 v = ld_nc_v4(p + i);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+                cnt += ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu)) == thr;
+        }
+        // exclusive prefix of the counts over the threads
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int x = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += x;
+        }
+        if (lane == 31) red[warp] = incl;
+        __syncthreads();
+        int base = 0;
+        for (int w2 = 0; w2 < warp; ++w2) base += red[w2];
+        int rank = base + incl - cnt;  // ties before this thread's piece
+        if (cnt > 0 && rank < need) {
+            for (int i = lo; i < hi && rank < need; ++i) {
+                const uint4 v = ld_nc_v4(p + i);
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    if (rank < need && ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu)) == thr) {
+                        const int pos = n_above + rank;
+                        if (pos < SPECROLL_MAX_TOPK) {
+                            sel_id[pos] = i * 8 + t;
+                            sel_key[pos] = thr;
+                        }
+                        ++rank;
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // ---- order the winners by (key desc, id asc)
+    const int n_sel = min(kS, min(V, SPECROLL_MAX_TOPK));
+    if (tid < n_sel) {
+        const uint32_t ki = sel_key[tid];
+        const int ii = sel_id[tid];
+        int rk = 0;
+        for (int j = 0; j < n_sel; ++j) rk += (sel_key[j] > ki) || (sel_key[j] == ki && sel_id[j] < ii);
+        top_id[(size_t)r * kS + rk] = ii;
+    }
+}
+
+struct FeedbackArgs {
+    const uint16_t *logits;
+    const int32_t *rec_row;
+    const float *row_max, *row_sum;
+    const int32_t *cand_id;
+    const float *cand_logit;
+    const int32_t *y_star;
+    const __nv_bfloat16 *W;
+    const float *rho;
+    const int32_t *rec_mem;
+    const int32_t *top_id;
+    float *m;
+    float *d_dist, *d_cov, *tv;
+    int R, k, kS, d, V;
+    float inv_T, eps;
+};
+
+// MAXC = columns of the hidden dimension per thread (d <= 256 * MAXC)
+template <int MAXC>
+__global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a) {
+    using namespace fb;
+    __shared__ int s_id[MAX_S];
+    __shared__ float s_p[MAX_S];      // target mass exp((l - M)/T) / row_sum of the support tokens
+    __shared__ float s_adist[MAX_S];  // coefficient of W_v in r_dist
+    __shared__ float s_acov[MAX_S];   // coefficient of W_v in r_cov
+    __shared__ float s_q[SPECROLL_MAX_TOPK];
+    __shared__ int s_n;
+    __shared__ float s_dd, s_dc;
+    __shared__ float red[FB_THREADS / 32];
+    const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int k = a.k, kS = a.kS, d = a.d;
+    const size_t row = (size_t)a.rec_row[r];
+    const uint16_t *lg = a.logits + row * a.V;
+    const float M = a.row_max[row], Ssum = a.row_sum[row];
+    const int32_t *cid = a.cand_id + (size_t)r * k;
+    const float *cl = a.cand_logit + (size_t)r * k;
+    const int32_t *top = a.top_id + (size_t)r * kS;
+
+    if (warp == 0) {
+        // ---- q on the candidates
+        float mx = -INFINITY;
+        for (int j = lane; j < k; j += 32) mx = fmaxf(mx, cl[j]);
+        mx = warp_max(mx);
+        float qs = 0.f;
+        for (int j = lane; j < k; j += 32) {
+            const float w = __expf((cl[j] - mx) * a.inv_T);
+            s_q[j] = w;
+            qs += w;
+        }
+        qs = warp_sum(qs);
+        __syncwarp();
+        for (int j = lane; j < k; j += 32) s_q[j] /= qs;
+        // ---- S = C u Top_kS u {y*}, duplicates removed (first occurrence kept; the candidates come first)
+        const int n_raw = k + kS + 1;
+        if (lane == 0) s_n = 0;
+        __syncwarp();
+        for (int i0 = 0; i0 < n_raw; i0 += 32) {
+            const int i = i0 + lane;
+            int v = -1;
+            if (i < k)
+                v = cid[i];
+            else if (i < k + kS)
+                v = top[i - k];
+            else if (i == k + kS)
+                v = a.y_star[r];
+            bool fresh = v >= 0 && v < a.V;
+            if (fresh) {
+                for (int j = 0; j < i; ++j) {  // the same token earlier in the concatenation?
+                    const int u = j < k ? cid[j] : (j < k + kS ? top[j - k] : a.y_star[r]);
+                    if (u == v) {
+                        fresh = false;
+                        break;
+                    }
+                }
+            }
+            const unsigned bal = __ballot_sync(0xffffffffu, fresh);
+            const int base = s_n;
+            if (fresh) {
+                const int pos = base + __popc(bal & ((1u << lane) - 1u));
+                s_id[pos] = v;
+                s_p[pos] = __expf((__uint_as_float((uint32_t)lg[v] << 16) - M) * a.inv_T) / Ssum;
+            }
+            __syncwarp();
+            if (lane == 0) s_n = base + __popc(bal);
+            __syncwarp();
+        }
+        const int n = s_n;
+        // ---- masses: p(S), p(C), p(C*); TV on C
+        float pS = 0.f;
+        for (int i = lane; i < n; i += 32) pS += s_p[i];
+        pS = warp_sum(pS);
+        float pC = 0.f;
+        for (int j = lane; j < k; j += 32) pC += s_p[j];  // the first k support entries are the candidates
+        pC = warp_sum(pC);
+        float tvs = 0.f;
+        for (int j = lane; j < k; j += 32) tvs += fabsf(s_p[j] / pC - s_q[j]);
+        tvs = 0.5f * warp_sum(tvs);
+        // C* = the first k of Top_kS; O = C* \ C
+        float pCs = 0.f, cov_b = 0.f;
+        for (int i = lane; i < n; i += 32) s_acov[i] = 0.f;
+        __syncwarp();
+        for (int t = lane; t < k; t += 32) {
+            const int v = top[t];
+            const float pv = __expf((__uint_as_float((uint32_t)lg[v] << 16) - M) * a.inv_T) / Ssum;
+            pCs += pv;
+            bool inC = false;
+            for (int j = 0; j < k; ++j) inC |= (cid[j] == v);
+            if (!inC) {
+                // an omitted target-important token: +p_S(y) on its own row, -p_S(y) on the weakest candidate's
+                int pos = -1;
+                for (int i = k; i < n; ++i)
+                    if (s_id[i] == v) pos = i;
+                if (pos >= 0) s_acov[pos] = pv / pS;
+                cov_b += pv / pS;
+            }
+        }
+        pCs = warp_sum(pCs);
+        cov_b = warp_sum(cov_b);
+        __syncwarp();
+        for (int i = lane; i < n; i += 32) s_adist[i] = s_p[i] / pS - (i < k ? s_q[i] : 0.f);
+        if (lane == 0) {
+            s_acov[k - 1] -= cov_b;  // b* = last candidate (the list is sorted by logit)
+            const float dd = pC * tvs, dc = pCs - pC;
+            s_dd = dd;
+            s_dc = dc;
+            if (a.d_dist) a.d_dist[r] = dd;
+            if (a.d_cov) a.d_cov[r] = dc;
+            if (a.tv) a.tv[r] = tvs;
+        }
+    }
+    __syncthreads();
+    const int n = s_n;
+    const float dd = s_dd, dc = s_dc;
+    // ---- both directions: thread t owns columns t, t + 256, ...; the support rows of W are read once
+    float rd[MAXC], rc[MAXC];
+    const int ncol = (d + FB_THREADS - 1) / FB_THREADS;
+#pragma unroll
+    for (int c = 0; c < MAXC; ++c) rd[c] = rc[c] = 0.f;
+    for (int i = 0; i < n; ++i) {
+        const __nv_bfloat16 *wr = a.W + (size_t)s_id[i] * d;
+        const float ad = s_adist[i], ac = s_acov[i];
+#pragma unroll
+        for (int c = 0; c < MAXC; ++c) {
+            const int col = tid + c * FB_THREADS;
+            if (c < ncol && col < d) {
+                const float w = __bfloat162float(wr[col]);
+                rd[c] = fmaf(ad, w, rd[c]);
+                rc[c] = fmaf(ac, w, rc[c]);
+            }
+        }
+    }
+    float sd = 0.f, scv = 0.f;
+#pragma unroll
+    for (int c = 0; c < MAXC; ++c) {
+        sd += rd[c] * rd[c];
+        scv += rc[c] * rc[c];
+    }
+    sd = block_sum_f<FB_THREADS>(sd, red);
+    scv = block_sum_f<FB_THREADS>(scv, red);
+    const float fd = dd / (sqrtf(sd / d) + a.eps), fc = dc / (sqrtf(scv / d) + a.eps);
+    float sg = 0.f;
+#pragma unroll
+    for (int c = 0; c < MAXC; ++c) {
+        rd[c] = fd * rd[c] + fc * rc[c];  // g
+        sg += rd[c] * rd[c];
+    }
+    sg = block_sum_f<FB_THREADS>(sg, red);
+    const float fe = (dd + dc) / (sqrtf(sg / d) + a.eps);
+    const float rho = a.rho[r];
+    float *mr = a.m + (size_t)a.rec_mem[r] * d;
+#pragma unroll
+    for (int c = 0; c < MAXC; ++c) {
+        const int col = tid + c * FB_THREADS;
+        if (c < ncol && col < d) mr[col] = rho * mr[col] + (1.f - rho) * fe * rd[c];
+    }
+}
+
+}  // namespace specroll
+
+using namespace specroll;
+
+static int check_feedback_desc(const specroll_feedback_desc *d) {
+    if (!d || d->R < 0 || d->k < 1 || d->k > SPECROLL_MAX_TOPK || d->k_support < d->k ||
+        d->k_support > SPECROLL_MAX_TOPK || d->d < 8 || d->d > 12288 || d->V < 8 || (d->V % 8) || d->k_support > d->V ||
+        !(d->temperature > 0.f) || !(d->eps >= 0.f) || d->flags != 0)
+        return SPECROLL_EINVAL;
+    return SPECROLL_OK;
+}
+
+extern "C" size_t specroll_reflex_feedback_workspace_bytes(const specroll_feedback_desc *d) {
+    if (check_feedback_desc(d) != SPECROLL_OK) return 0;
+    return align_up((size_t)d->R * d->k_support * sizeof(int32_t), 256) + 256;
+}
+
+extern "C" int specroll_reflex_feedback(const specroll_feedback_desc *d, const void *logits, const int32_t *rec_row,
+                                        const float *row_max, const float *row_sum, const int32_t *cand_id,
+                                        const float *cand_logit, const int32_t *y_star, const void *W,
+                                        const float *rho, const int32_t *rec_mem, float *m, float *d_dist,
+                                        float *d_cov, float *tv, void *workspace, size_t workspace_bytes,
+                                        void *cuda_stream) {
+    if (check_feedback_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (!logits || !rec_row || !row_max || !row_sum || !cand_id || !cand_logit || !y_star || !W || !rho || !rec_mem || !m)
+        return SPECROLL_EINVAL;
+    if (!aligned16(logits) || !aligned16(W)) return SPECROLL_EALIGN;
+    if (d->R == 0) return SPECROLL_OK;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < specroll_reflex_feedback_workspace_bytes(d))
+        return SPECROLL_EWORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int32_t *top_id = static_cast<int32_t *>(workspace);
+    feedback_topk_kernel<<<d->R, fb::TOPK_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), rec_row, d->V,
+                                                            d->k_support, top_id);
+    SR_LAUNCH_CHECK();
+    FeedbackArgs a;
+    a.logits = static_cast<const uint16_t *>(logits);
+    a.rec_row = rec_row;
+    a.row_max = row_max;
+    a.row_sum = row_sum;
+    a.cand_id = cand_id;
+    a.cand_logit = cand_logit;
+    a.y_star = y_star;
+    a.W = static_cast<const __nv_bfloat16 *>(W);
+    a.rho = rho;
+    a.rec_mem = rec_mem;
+    a.top_id = top_id;
+    a.m = m;
+    a.d_dist = d_dist;
+    a.d_cov = d_cov;
+    a.tv = tv;
+    a.R = d->R;
+    a.k = d->k;
+    a.kS = d->k_support;
+    a.d = d->d;
+    a.V = d->V;
+    a.inv_T = 1.0f / d->temperature;
+    a.eps = d->eps;
+    if (d->d <= 8 * fb::FB_THREADS)
+        feedback_kernel<8><<<d->R, fb::FB_THREADS, 0, st>>>(a);
+    else if (d->d <= 24 * fb::FB_THREADS)
+        feedback_kernel<24><<<d->R, fb::FB_THREADS, 0, st>>>(a);
+    else
+        feedback_kernel<48><<<d->R, fb::FB_THREADS, 0, st>>>(a);
+    SR_LAUNCH_CHECK();
+    return SPECROLL_OK;
+}
