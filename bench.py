@@ -188,7 +188,7 @@ def run_ours(args, w, layers):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     D.init("nccl")
-    wl = StepWorkload(w, dev, seed=rank, layers=layers, paged=args.paged, top_p=args.top_p)
+    wl = StepWorkload(w, dev, seed=rank, layers=layers, paged=args.paged, top_p=args.top_p, lazy_stats=args.lazy_stats)
     peaks = measured_peaks()
 
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
@@ -315,7 +315,7 @@ def run_ours(args, w, layers):
                        "Hkv": w.Hkv, "D": w.D, "layers": wl.layers, "T_kv": wl.T_kv, "temperature": w.temperature,
                        "kv_cache": "128-token pages in a seeded random order (specroll_tree_attn_paged)" if args.paged
                        else "contiguous ragged (specroll_tree_attn)",
-                       "top_p": wl.top_p, "cuda_graph": graph is not None,
+                       "top_p": wl.top_p, "lazy_stats": bool(args.lazy_stats), "cuda_graph": graph is not None,
                        "parallelism": f"replicas x{world} (sharded by sequence, no collective)",
                        "l2": "inputs larger than L2: per-layer KV cache, logits and W each exceed 126 MB and every "
                              "layer has its own cache"},
@@ -516,6 +516,9 @@ def main():
     ap.add_argument("--top-p", type=float, default=None,
                     help="verify against nucleus-truncated target distributions (specroll_verify_nucleus); the "
                          "metric's step uses the plain temperature softmax (default)")
+    ap.add_argument("--lazy-stats", action="store_true",
+                    help="softmax statistics of the visited nodes only (SPECROLL_VERIFY_LAZY_STATS); the metric's step "
+                         "evaluates every node (default)")
     ap.add_argument("--paged", action="store_true",
                     help="keep the KV cache in 128-token pages (specroll_tree_attn_paged) and time the commit of the "
                          "accepted paths after the step as well (reported beside the step, not inside it)")

@@ -274,8 +274,14 @@ int specroll_reflex_feedback(const specroll_feedback_desc *desc, const void *log
 typedef struct {
     int32_t B, N, K, k, V;
     float temperature;
-    int32_t flags; /* reserved, must be 0 */
+    int32_t flags; /* 0, or SPECROLL_VERIFY_LAZY_STATS */
 } specroll_verify_desc;
+
+/* Compute the softmax statistics only of the rows the walk visits (at most K + 1 per sequence instead of all N):
+ * same walk and same tokens; row_max / row_sum are then written for the visited nodes only and the other entries
+ * are left untouched.  (The method evaluates every node's distribution; this reads fewer bytes, for callers that do
+ * not need the statistics of the nodes that were never reached.) */
+#define SPECROLL_VERIFY_LAZY_STATS 1
 
 size_t specroll_verify_workspace_bytes(const specroll_verify_desc *desc);
 

@@ -32,6 +32,7 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
 PROPOSE_LEGACY_MMA = 1
 ATTN_LEGACY_MMA = 1
 ATTN_REUSE_PLAN = 2
+VERIFY_LAZY_STATS = 1
 PAGE_TOKENS = 128
 
 
@@ -370,14 +371,14 @@ def verify_nucleus_workspace_bytes(B, N, K, k, V, temperature=1.0) -> int:
 
 
 def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, temperature=1.0,
-           workspace=None, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+           workspace=None, out: Optional[Dict[str, torch.Tensor]] = None, flags: int = 0) -> Dict[str, torch.Tensor]:
     """specroll_verify.  Device tensors in, dict of device tensors out."""
     parent = _host_i32(parent, "parent")
     B, N, V = logits.shape
     _, K, k = cand_id.shape
     if parent.shape[0] != N or tuple(tree_tok.shape) != (B, N) or tuple(u_acc.shape) != (B, N):
         raise SpecrollError("verify: inconsistent shapes")
-    desc = VerifyDesc(B, N, K, k, V, temperature, 0)
+    desc = VerifyDesc(B, N, K, k, V, temperature, flags)
     dev = logits.device
     i32, f32 = torch.int32, torch.float32
     if out is None:
@@ -405,7 +406,8 @@ def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fi
 
 
 def verify_nucleus(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, top_p, temperature=1.0,
-                   workspace=None, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+                   workspace=None, out: Optional[Dict[str, torch.Tensor]] = None,
+                   flags: int = 0) -> Dict[str, torch.Tensor]:
     """specroll_verify_nucleus: verification against nucleus-truncated target distributions.
     The returned dict also holds nucleus_thr and nucleus_sum [B,N]."""
     parent = _host_i32(parent, "parent")
@@ -413,7 +415,7 @@ def verify_nucleus(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_a
     _, K, k = cand_id.shape
     if parent.shape[0] != N or tuple(tree_tok.shape) != (B, N) or tuple(u_acc.shape) != (B, N):
         raise SpecrollError("verify_nucleus: inconsistent shapes")
-    desc = VerifyDesc(B, N, K, k, V, temperature, 0)
+    desc = VerifyDesc(B, N, K, k, V, temperature, flags)
     dev = logits.device
     i32, f32 = torch.int32, torch.float32
     if out is None:

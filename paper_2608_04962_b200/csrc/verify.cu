@@ -373,14 +373,13 @@ __device__ __forceinline__ void walk_begin(const WalkArgs &a, int b, int lane, W
 // One node u (which has children), by one warp: the target's probabilities on the candidates of u's head -
 // S is the normaliser and thr the nucleus threshold key (0: none) of u's row - then u's children in slot order.
 // Returns the accepted child, or -1 when every child was rejected (the residual is then in sm->r, st->sigma).
-__device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, double S, uint32_t thr, int lane,
+__device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, double M, double S, uint32_t thr, int lane,
                          WalkSmem *sm, WalkState *st) {
     double *r = sm->r, *w = sm->w;
     float *cl = sm->cl;
     int32_t *id = sm->id;
     const int k = a.k, N = a.N, K = a.K;
     const int hd = topo.depth[u];
-    const double M = (double)a.row_max[(size_t)b * N + u];
     const uint16_t *lg = a.logits + ((size_t)b * N + u) * a.V;
     for (int j = lane; j < k; j += 32) {
         const int t = a.cand_id[((size_t)b * K + hd) * k + j];
@@ -495,7 +494,8 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(WalkArgs a, Topo 
             st.have_residual = false;
             break;
         }
-        const int acc = walk_node(a, topo, b, u, (double)a.row_sum[(size_t)b * a.N + u], 0u, lane, sm, &st);
+        const int acc = walk_node(a, topo, b, u, (double)a.row_max[(size_t)b * a.N + u],
+                                  (double)a.row_sum[(size_t)b * a.N + u], 0u, lane, sm, &st);
         if (acc < 0) {
             st.kind = 0;
             st.have_residual = true;
@@ -506,16 +506,57 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(WalkArgs a, Topo 
     walk_end(a, b, u, (double)a.row_sum[(size_t)b * a.N + u], lane, sm, &st);
 }
 
-// Nucleus-truncated target distributions: one CTA per sequence.  Only the nodes the walk visits need their
-// nucleus, and which they are is known only as the walk goes, so before each node all threads find that row's
-// threshold (nucleus_row) and warp 0 then does the node.  Thresholds and kept sums of the visited nodes are
-// left in thr_key / keep_sum (the terminal draw reads those of the last node).
+// Maximum and sum of exponentials of one row by all NUC_THREADS threads of a CTA (same arithmetic as
+// row_stats_kernel); every thread returns with the result.
+__device__ void row_stats_row(const uint16_t *__restrict__ row_logits, int V, float c, float *sm_m, float *sm_s,
+                              float *M_out, float *S_out) {
+    const uint4 *p = reinterpret_cast<const uint4 *>(row_logits);
+    const int nvec = V >> 3;
+    float m = NEG_INF, s = 0.f;
+    int i = threadIdx.x;
+    for (; i + 3 * NUC_THREADS < nvec; i += 4 * NUC_THREADS) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld_nc_v4(p + i + u * NUC_THREADS);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) online_update(v[u], c, m, s);
+    }
+    for (; i < nvec; i += NUC_THREADS) online_update(ld_nc_v4(p + i), c, m, s);
+    const float mw = warp_max(m);
+    s = (m == NEG_INF) ? 0.f : s * ex2_approx((m - mw) * c);
+    s = warp_sum(s);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) {
+        sm_m[warp] = mw;
+        sm_s[warp] = s;
+    }
+    __syncthreads();
+    float mb = NEG_INF;
+    for (int w = 0; w < NUC_THREADS / 32; ++w) mb = fmaxf(mb, sm_m[w]);
+    float sb = 0.f;
+    for (int w = 0; w < NUC_THREADS / 32; ++w)
+        sb += (sm_m[w] == NEG_INF) ? 0.f : sm_s[w] * ex2_approx((sm_m[w] - mb) * c);
+    *M_out = mb;
+    *S_out = sb;
+}
+
+// One CTA per sequence, for the two variants in which something has to be computed per visited node before the
+// node can be walked, and which nodes are visited is known only as the walk goes:
+//   LAZY  the softmax statistics of a row are computed when the walk reaches it (at most K + 1 rows per
+//         sequence instead of all N), and written to row_max / row_sum for those rows only;
+//   NUC   the target distributions are their nuclei: the row's threshold is searched (nucleus_row) and left
+//         in thr_key / keep_sum (the terminal draw reads those of the last node).
+// Before each node all threads do that work, then warp 0 does the node.
+template <bool LAZY, bool NUC>
 __global__ void __launch_bounds__(NUC_THREADS)
-walk_nucleus_kernel(WalkArgs a, Topo topo, float c, float top_p, uint32_t *__restrict__ thr_key,
-                    float *__restrict__ keep_sum, float *__restrict__ out_thr, float *__restrict__ out_sum) {
-    extern __shared__ __align__(16) unsigned char nuc_raw[];  // NucleusSmem: above the static limit, hence dynamic
+walk_cta_kernel(WalkArgs a, Topo topo, float c, float top_p, float *__restrict__ row_max_w,
+                float *__restrict__ row_sum_w, uint32_t *__restrict__ thr_key, float *__restrict__ keep_sum,
+                float *__restrict__ out_thr, float *__restrict__ out_sum) {
+    extern __shared__ __align__(16) unsigned char nuc_raw[];  // NucleusSmem (NUC only): above the static limit
     NucleusSmem &nuc = *reinterpret_cast<NucleusSmem *>(nuc_raw);
     __shared__ WalkSmem sm;
+    __shared__ float sm_m[NUC_THREADS / 32], sm_s[NUC_THREADS / 32];
     __shared__ int sh_next;  // next node, or -1 when the walk is over
     const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     WalkState st;
@@ -523,16 +564,31 @@ walk_nucleus_kernel(WalkArgs a, Topo topo, float c, float top_p, uint32_t *__res
     int u = 0;
     for (;;) {
         const size_t row = (size_t)b * a.N + u;
-        nucleus_row(a.logits + row * a.V, a.V, c, a.row_max[row], top_p * a.row_sum[row], &nuc);
-        const uint32_t thr = nuc.prefix;
-        const float keep = nuc.keep;
-        if (threadIdx.x == 0) {
-            thr_key[row] = thr;
-            keep_sum[row] = keep;
-            if (out_sum) out_sum[row] = keep;
-            if (out_thr) {  // the threshold as a logit: undo the key
-                const uint32_t bits = (thr & 0x8000u) ? (thr & 0x7fffu) : (~thr & 0xffffu);
-                out_thr[row] = __uint_as_float(bits << 16);
+        float M, S;
+        if constexpr (LAZY) {
+            row_stats_row(a.logits + row * a.V, a.V, c, sm_m, sm_s, &M, &S);
+            if (threadIdx.x == 0) {
+                row_max_w[row] = M;
+                row_sum_w[row] = S;
+            }
+        } else {
+            M = a.row_max[row];
+            S = a.row_sum[row];
+        }
+        uint32_t thr = 0u;
+        float norm = S;
+        if constexpr (NUC) {
+            nucleus_row(a.logits + row * a.V, a.V, c, M, top_p * S, &nuc);
+            thr = nuc.prefix;
+            norm = nuc.keep;
+            if (threadIdx.x == 0) {
+                thr_key[row] = thr;
+                keep_sum[row] = norm;
+                if (out_sum) out_sum[row] = norm;
+                if (out_thr) {  // the threshold as a logit: undo the key
+                    const uint32_t bits = (thr & 0x8000u) ? (thr & 0x7fffu) : (~thr & 0xffffu);
+                    out_thr[row] = __uint_as_float(bits << 16);
+                }
             }
         }
         if (warp == 0) {
@@ -541,13 +597,13 @@ walk_nucleus_kernel(WalkArgs a, Topo topo, float c, float top_p, uint32_t *__res
                 st.kind = (u != 0) ? 1 : 0;
                 st.have_residual = false;
             } else {
-                next = walk_node(a, topo, b, u, (double)keep, thr, lane, &sm, &st);
+                next = walk_node(a, topo, b, u, (double)M, (double)norm, thr, lane, &sm, &st);
                 if (next < 0) {
                     st.kind = 0;
                     st.have_residual = true;
                 }
             }
-            if (next < 0) walk_end(a, b, u, (double)keep, lane, &sm, &st);
+            if (next < 0) walk_end(a, b, u, (double)norm, lane, &sm, &st);
             if (lane == 0) sh_next = next;
         }
         __syncthreads();
@@ -810,7 +866,7 @@ using namespace specroll;
 static int check_verify_desc(const specroll_verify_desc *d) {
     if (!d || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->K < 1 || d->K > SPECROLL_MAX_HEADS ||
         d->k < 1 || d->k > SPECROLL_MAX_TOPK || d->V < 8 || (d->V % 8) || d->k > d->V ||
-        !(d->temperature > 0.f) || d->flags != 0)
+        !(d->temperature > 0.f) || (d->flags & ~SPECROLL_VERIFY_LAZY_STATS) != 0)
         return SPECROLL_EINVAL;
     return SPECROLL_OK;
 }
@@ -866,9 +922,13 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
 
     const float c = (float)(1.4426950408889634 / (double)d->temperature);
     const int rows = d->B * d->N;
-    row_stats_kernel<<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
-                                                  row_sum);
-    SR_LAUNCH_CHECK();
+    const bool lazy = (d->flags & SPECROLL_VERIFY_LAZY_STATS) != 0;
+    if (!lazy) {
+        row_stats_kernel<<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
+                                                      row_sum);
+        SR_LAUNCH_CHECK();
+    }
+
     WalkArgs wa;
     wa.logits = static_cast<const uint16_t *>(logits);
     wa.tree_tok = tree_tok;
@@ -896,14 +956,24 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
     if (truncate) {
         static bool configured = false;
         if (!configured) {
-            SR_CUDA_TRY(cudaFuncSetAttribute(walk_nucleus_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            SR_CUDA_TRY(cudaFuncSetAttribute(walk_cta_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)sizeof(NucleusSmem)));
+            SR_CUDA_TRY(cudaFuncSetAttribute(walk_cta_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)sizeof(NucleusSmem)));
             configured = true;
         }
-        walk_nucleus_kernel<<<d->B, NUC_THREADS, sizeof(NucleusSmem), st>>>(wa, topo, c, top_p, thr_key, keep_sum,
-                                                                             nucleus_thr, nucleus_sum);
-    } else
+        if (lazy)
+            walk_cta_kernel<true, true><<<d->B, NUC_THREADS, sizeof(NucleusSmem), st>>>(
+                wa, topo, c, top_p, row_max, row_sum, thr_key, keep_sum, nucleus_thr, nucleus_sum);
+        else
+            walk_cta_kernel<false, true><<<d->B, NUC_THREADS, sizeof(NucleusSmem), st>>>(
+                wa, topo, c, top_p, row_max, row_sum, thr_key, keep_sum, nucleus_thr, nucleus_sum);
+    } else if (lazy) {
+        walk_cta_kernel<true, false><<<d->B, NUC_THREADS, 0, st>>>(wa, topo, c, 1.0f, row_max, row_sum, nullptr, nullptr,
+                                                                    nullptr, nullptr);
+    } else {
         walk_kernel<<<(d->B + WALK_WARPS - 1) / WALK_WARPS, WALK_WARPS * 32, 0, st>>>(wa, topo);
+    }
     SR_LAUNCH_CHECK();
 
     TermArgs ta;

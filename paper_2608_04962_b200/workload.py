@@ -33,8 +33,9 @@ class StepWorkload:
     """All tensors of one step for workload ``w`` on ``device`` (seed offset for replicas)."""
 
     def __init__(self, w: I.Workload, device, seed: int = 0, layers: int | None = None, paged: bool = False,
-                 top_p: float | None = None):
+                 top_p: float | None = None, lazy_stats: bool = False):
         self.w = w
+        self.verify_flags = S.VERIFY_LAZY_STATS if lazy_stats else 0
         self.paged = bool(paged)
         self.top_p = top_p if (top_p is not None and 0.0 < top_p < 1.0) else None
         self.device = device
@@ -163,11 +164,12 @@ class StepWorkload:
         if self.top_p is not None:
             self.ver = S.verify_nucleus(self.logits, self.parent, p["tree_tok"], p["tree_cand"], p["cand_id"],
                                         p["cand_logit"], self.u_acc, self.u_fin, self.top_p,
-                                        temperature=self.w.temperature, workspace=self.ws_verify, out=self.ver)
+                                        temperature=self.w.temperature, workspace=self.ws_verify, out=self.ver,
+                                        flags=self.verify_flags)
             return self.ver
         self.ver = S.verify(self.logits, self.parent, p["tree_tok"], p["tree_cand"], p["cand_id"],
                             p["cand_logit"], self.u_acc, self.u_fin, temperature=self.w.temperature,
-                            workspace=self.ws_verify, out=self.ver)
+                            workspace=self.ws_verify, out=self.ver, flags=self.verify_flags)
         return self.ver
 
     def step(self, events=None):

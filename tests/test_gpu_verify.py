@@ -124,3 +124,38 @@ def test_bad_arguments_are_refused_without_touching_the_device():
         S.verify(lg, parent, *args, temperature=0.0)
     with pytest.raises(S.SpecrollError):
         S.verify(lg, parent, *args, workspace=torch.empty(256, dtype=torch.uint8, device="cuda")[:16])
+
+
+@pytest.mark.parametrize("name,B,V,T", [("qwen1.5b", 32, 151936, 1.0), ("qwen7b", 16, 8200, 0.7)])
+def test_lazy_row_statistics_give_the_same_walk(name, B, V, T):
+    # statistics of the visited rows only: same tokens as the full pass; row_max / row_sum written where visited
+    w = I.scaled(I.WORKLOADS[name], B=B, V=V, temperature=T)
+    parent = I.topology(w)
+    cid, cl = I.synthetic_candidates(w)
+    d = ref.tree_draw(parent, np.zeros(w.B, np.int32), cid, cl, I.uniforms24(78, (w.B, w.N)), temperature=T)
+    lg = I.target_logits(w, parent, d["tree_tok"])
+    u_acc, u_fin = I.verify_uniforms(w)
+    o = ref.verify(lg, parent, d["tree_tok"], d["tree_cand"], cid, cl, u_acc, u_fin, temperature=T)
+    args = (dev_bf16(lg), parent, dev(d["tree_tok"]), dev(d["tree_cand"]), dev(cid), dev(cl), dev(u_acc), dev(u_fin))
+    out = {"n_acc": torch.empty(B, dtype=torch.int32, device="cuda"),
+           "path_node": torch.empty((B, w.K + 1), dtype=torch.int32, device="cuda"),
+           "out_tok": torch.empty((B, w.K + 1), dtype=torch.int32, device="cuda"),
+           "term_node": torch.empty(B, dtype=torch.int32, device="cuda"),
+           "term_kind": torch.empty(B, dtype=torch.int32, device="cuda"),
+           "row_max": torch.full((B, w.N), -7.0, device="cuda"), "row_sum": torch.full((B, w.N), -7.0, device="cuda"),
+           "min_margin": torch.empty(B, device="cuda")}
+    g = {k: host(v) for k, v in S.verify(*args, temperature=T, out=out, flags=S.VERIFY_LAZY_STATS).items()}
+    full = {k: host(v) for k, v in S.verify(*args, temperature=T).items()}
+    for key in ("n_acc", "path_node", "out_tok", "term_node", "term_kind"):
+        assert np.array_equal(g[key], full[key]), key               # the two GPU variants agree exactly
+    visited = np.zeros((B, w.N), bool)
+    for b in range(B):
+        visited[b, g["path_node"][b, : g["n_acc"][b] + 1]] = True
+        visited[b, g["term_node"][b]] = True
+    assert np.array_equal(g["row_max"][visited].astype(np.float64), o["row_max"][visited])
+    assert np.abs(g["row_sum"][visited] / o["row_sum"][visited] - 1).max() < 2e-5
+    assert (g["row_max"][~visited] == -7.0).all() and (g["row_sum"][~visited] == -7.0).all()
+    assert visited.sum() < 0.5 * visited.size                        # it does read fewer rows
+    same = (g["n_acc"] == o["n_acc"]) & (g["out_tok"] == o["out_tok"]).all(1)
+    assert (same | (o["min_margin"] < NEAR_TIE) | (o["fin_margin"] < 1e-6)).all()
+
