@@ -138,13 +138,21 @@ head_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                 tmem_ld32(taddr + (uint32_t)c, r);
                 tmem_ld_wait();
                 if (o < d) {
+                    // all residual loads first: taken one by one between the stores, each would cost a full
+                    // round trip to L2 (that made the epilogue three quarters of the kernel)
+                    float hv[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int b = min(b0 + c + i, B - 1);
+                        hv[i] = __bfloat162float(h[(size_t)b * d + o]);
+                    }
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const int b = b0 + c + i;
                         if (b < B) {
                             const float y = __uint_as_float(r[i]) + bo;
                             const float sl = y / (1.0f + __expf(-y));
-                            z[((size_t)b * K + hd) * d + o] = __bfloat162float(h[(size_t)b * d + o]) + sl;
+                            z[((size_t)b * K + hd) * d + o] = hv[i] + sl;
                         }
                     }
                 }
