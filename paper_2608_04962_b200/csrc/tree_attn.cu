@@ -509,13 +509,13 @@ static int compute_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_
     if (p->use_tc) {
         // row blocks are whole nodes: (node, head-in-group) rows of a block are one TMA box
         // The softmax of a row block costs the same whether the block is full or not, so the rows go into as
-        // few blocks as possible.  An even number of blocks is processed two per work unit (they share every
-        // K/V tile in shared memory); an odd number one per unit (the blocks' units run side by side on
-        // different SMs and the tile comes from L2 after the first read).
+        // few blocks as possible.  Every block is a work unit of its own; the units of one (chunk, KV head)
+        // are neighbours in the work order, run side by side on different SMs, and the K/V tiles reach the
+        // later ones from L2 (measured: DRAM reads stay at one pass over the cache).
         int npb = 128 / G;
         const int nb = (d->N + npb - 1) / npb;
         npb = (d->N + nb - 1) / nb;  // even out the blocks
-        p->nrb = (nb % 2 == 0) ? 2 : 1;
+        p->nrb = 1;
         p->nodes_per_block = npb;
         p->n_rb = nb;
         p->rows_per_block = npb * G;
