@@ -489,7 +489,7 @@ static long long estimate_makespan(const std::vector<int> &tiles, int ct, int co
 }
 
 struct AttnPlan {
-    int rows, n_rb, nrb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens, nodes_per_block, n_counters;
+    int rows, n_rb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens, nodes_per_block, n_counters;
     int merge_mode;  // tcgen05 path: 0 = split sequences are merged inside the attention kernel, 2 = by a kernel after it
     bool use_tc;
     size_t off_status, off_items, off_sorted, off_rank, off_tab, off_counters, off_po, off_pml, total;
@@ -515,12 +515,10 @@ static int compute_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_
         int npb = 128 / G;
         const int nb = (d->N + npb - 1) / npb;
         npb = (d->N + nb - 1) / nb;  // even out the blocks
-        p->nrb = 1;
         p->nodes_per_block = npb;
         p->n_rb = nb;
         p->rows_per_block = npb * G;
     } else {
-        p->nrb = 1;
         p->nodes_per_block = 0;
         p->n_rb = (p->rows + AT_MAX_WARPS * 16 - 1) / (AT_MAX_WARPS * 16);
         p->rows_per_block = ((p->rows + p->n_rb - 1) / p->n_rb + 15) / 16 * 16;
@@ -539,7 +537,7 @@ static int compute_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_
     // the candidate whose estimated finishing time is lowest (the kernel hands the units, longest first, to
     // whichever CTA is free, which a few microseconds of host time can play through).  At least 512 tokens,
     // so that the fp32 partials stay a small fraction of the KV bytes.
-    const long long ctas_per_tile = (long long)d->Hkv * p->n_rb / p->nrb;
+    const long long ctas_per_tile = (long long)d->Hkv * p->n_rb;
     auto chunk_for = [&](int per_sm_pct) -> int {
         long long c = (tiles_total * ctas_per_tile * 100 + (long long)PLAN_SMS * per_sm_pct - 1) / ((long long)PLAN_SMS * per_sm_pct);
         if (c < 512 / TT) c = 512 / TT;
@@ -727,8 +725,7 @@ static int run_tree_attn(const specroll_attn_desc *d, const void *Q, const void 
     a.unit_tab = unit_tab;
     a.work_counter = counters;
     a.split_counters = counters + 64;
-    a.total_work = p.items * d->Hkv * (p.n_rb / p.nrb);
-    a.nrb = p.nrb;
+    a.total_work = p.items * d->Hkv * p.n_rb;
     a.merge_mode = p.merge_mode;
     a.nodes_per_block = p.nodes_per_block;
     if (!(p.use_tc && (d->flags & SPECROLL_ATTN_REUSE_PLAN))) {

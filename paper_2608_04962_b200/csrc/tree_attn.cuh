@@ -22,9 +22,8 @@ struct AttnArgs {
     const int32_t *unit_tab;      // [items][8] per chunk in work order: b, chunk, n_chunks, first item, kv0, L, 0, 0
     int32_t *work_counter;        // next work unit to hand out
     int32_t *split_counters;      // [B, Hkv, n_rb] chunks of a (sequence, kv head, row block) that have finished
-    int32_t total_work;           // items * Hkv * n_rb / nrb
+    int32_t total_work;           // items * Hkv * n_rb
     int32_t nodes_per_block;      // rows_per_block = nodes_per_block * G
-    int32_t nrb;                  // row blocks per work unit: 1, or 2 (then n_rb is even)
     // paged cache (tcgen05 kernel only): pool page of every 128-token tile; a chunk table row then carries the
     // sequence's first slot in this table instead of its first token
     const int32_t *page_table;
