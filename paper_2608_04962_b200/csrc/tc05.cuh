@@ -54,6 +54,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
+// try_wait with an upper limit (ns) on how long the thread may stay suspended before it answers
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
 // Non-blocking probe (try_wait may suspend the thread for a while before it answers).
 __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -72,16 +85,16 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
-    uint32_t spins = 0;
     for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (((++spins) & 127u) == 0u) {
-            if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
-                // records which wait gave up: barrier address (shared window) and the parity waited for
-                *abort_flag = (int)(0x40000000u | (parity << 24) | (bar & 0xffffffu));
-                return false;
-            }
+        // The thread sleeps in the barrier unit until the phase completes or the hinted time (50 us) is up:
+        // a waiting warp then issues next to nothing, where a loop of short probes takes issue slots and
+        // ALU cycles away from the warps that have work.
+        if (mbar_try_wait_hint(bar, parity, 50000u)) return true;
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+            // records which wait gave up: barrier address (shared window) and the parity waited for
+            *abort_flag = (int)(0x40000000u | (parity << 24) | (bar & 0xffffffu));
+            return false;
         }
     }
 }

@@ -657,7 +657,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     bits0 = limit >= 32 ? 0xffffffffu : (limit <= 0 ? 0u : ((1u << limit) - 1u));
                     bits1 = limit >= 64 ? 0xffffffffu : (limit <= 32 ? 0u : ((1u << (limit - 32)) - 1u));
                 }
-                // ---- pass 1: maximum of this thread's 64 columns
                 uint32_t r0[32], r1[32];
                 float mx0 = -INFINITY, mx1 = -INFINITY;
                 auto max_group = [&](const uint32_t(&src)[32], uint32_t bc) {
@@ -673,77 +672,138 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                             if ((bc >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(src[i2]));
                     }
                 };
-                tmem_ld32(s_t + 64u * half, r0);
-                tmem_ld32(s_t + 64u * half + 32u, r1);
-                tmem_ld_wait();
-                max_group(r0, bits0);
-                max_group(r1, bits1);
-                // ---- exchange the partial maximum with the thread that has the row's other 64 columns.  It
-                //      travels as bf16: any common reference close to the true maximum will do.  Two slots,
-                //      alternating, so that a fast thread's next write cannot overtake a slow read.
-                const unsigned short mine = bf16_bits_rn(fmaxf(mx0, mx1));
-                const int px = (int)(use_pair & 1u) * 64;
-                xm[px + half * 32 + lane] = mine;
+                // Exchanges the partial maximum with the thread that has the row's other 64 columns and returns the
+                // row's maximum (scaled).  It travels as bf16: any common reference close to the true maximum
+                // will do.  Two slots, alternating, so that a fast thread's next write cannot overtake a slow read.
+                auto row_max = [&](float &mt) -> bool {
+                    const unsigned short mine = bf16_bits_rn(fmaxf(mx0, mx1));
+                    const int px = (int)(use_pair & 1u) * 64;
+                    xm[px + half * 32 + lane] = mine;
 #ifdef SPECROLL_TRACE
-                const long long tps_ = clock64();
+                    const long long tps_ = clock64();
 #endif
-                ok = group_sync(pair_bar, use_pair, abort_flag);
+                    bool k_ = group_sync(pair_bar, use_pair, abort_flag);
 #ifdef SPECROLL_TRACE
-                prof[4] += (unsigned long long)(clock64() - tps_);
+                    prof[4] += (unsigned long long)(clock64() - tps_);
 #endif
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const float mt = fmaxf(bf16_bits_to_float(mine), bf16_bits_to_float(xm[px + (half ^ 1) * 32 + lane])) * sc;
-                float alpha = 1.f;
-                const bool need = mt > m_used + RESCALE_LOG2;  // also true on the first admissible tile
-                if (need) {
-                    alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - mt);
-                    m_used = mt;
-                    l *= alpha;
-                }
-                if (__any_sync(0xffffffffu, need) && j > 0) {
-                    // rows of this warp change their reference maximum: rescale this thread's half of their
-                    // running outputs in TMEM.  The previous tile's P V must have landed first.
-                    ok = twait(2, bar(C::B_PVDONE + (int)((t - 1u) % SB)), ((t - 1u) / SB) & 1u);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll 1
-                    for (int c = 0; c < DH; c += 32) {
-                        uint32_t o[32];
-                        tmem_ld32(o_t + (uint32_t)c, o);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int i2 = 0; i2 < 32; ++i2) o[i2] = __float_as_uint(__uint_as_float(o[i2]) * alpha);
-                        tmem_st32(o_t + (uint32_t)c, o);
-                    }
-                    tmem_st_wait();
-                }
-                const float mref = (m_used == -INFINITY) ? 0.f : m_used;
-                // ---- pass 2: p = 2^(s*scale - m) as packed bf16 pairs.  Each 32-column group becomes 16 packed
-                //      columns, stored over S columns this thread has already read: [0,32) for the first thread
-                //      of the pair, [96,128) for the second.
-                float ls0 = 0.f, ls1 = 0.f;
-                auto exp_group = [&](const uint32_t(&src)[32], uint32_t bc, uint32_t dst_col) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i2 = 0; i2 < 32; i2 += 2) {
-                        float p0 = ex2_approx(fmaf(__uint_as_float(src[i2]), sc, -mref));
-                        float p1 = ex2_approx(fmaf(__uint_as_float(src[i2 + 1]), sc, -mref));
-                        if (!full) {
-                            p0 = ((bc >> i2) & 1u) ? p0 : 0.f;
-                            p1 = ((bc >> (i2 + 1)) & 1u) ? p1 : 0.f;
-                        }
-                        ls0 += p0;
-                        ls1 += p1;
-                        pk[i2 >> 1] = pack_bf16x2(p0, p1);
-                    }
-                    tmem_st16(dst_col, pk);
+                    k_ = __all_sync(0xffffffffu, k_);
+                    mt = fmaxf(bf16_bits_to_float(mine), bf16_bits_to_float(xm[px + (half ^ 1) * 32 + lane])) * sc;
+                    return k_;
                 };
-                exp_group(r0, bits0, s_t + 96u * half);
-                exp_group(r1, bits1, s_t + 96u * half + 16u);
-                tmem_st_wait();
-                l += ls0 + ls1;
+                // p = 2^(s*scale - m) of one 32-column group as 16 packed bf16 pairs; adds the values to ls0 / ls1
+                // and, if asked to, folds the scores into mx0 / mx1.  (Two copies of each loop: with the mask test
+                // inside one loop the compiler evaluates it for every element of the full tiles too.)
+                float ls0 = 0.f, ls1 = 0.f;
+                auto exp_group = [&](const uint32_t(&src)[32], uint32_t bc, float mref, bool with_max, uint32_t(&pk)[16]) {
+                    if (full) {
+#pragma unroll
+                        for (int i2 = 0; i2 < 32; i2 += 2) {
+                            const float s0 = __uint_as_float(src[i2]), s1 = __uint_as_float(src[i2 + 1]);
+                            if (with_max) {
+                                mx0 = fmaxf(mx0, s0);
+                                mx1 = fmaxf(mx1, s1);
+                            }
+                            const float p0 = ex2_approx(fmaf(s0, sc, -mref));
+                            const float p1 = ex2_approx(fmaf(s1, sc, -mref));
+                            ls0 += p0;
+                            ls1 += p1;
+                            pk[i2 >> 1] = pack_bf16x2(p0, p1);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i2 = 0; i2 < 32; i2 += 2) {
+                            const float s0 = __uint_as_float(src[i2]), s1 = __uint_as_float(src[i2 + 1]);
+                            const bool b0 = (bc >> i2) & 1u, b1 = (bc >> (i2 + 1)) & 1u;
+                            if (with_max) {
+                                if (b0) mx0 = fmaxf(mx0, s0);
+                                if (b1) mx0 = fmaxf(mx0, s1);
+                            }
+                            const float p0 = b0 ? ex2_approx(fmaf(s0, sc, -mref)) : 0.f;
+                            const float p1 = b1 ? ex2_approx(fmaf(s1, sc, -mref)) : 0.f;
+                            ls0 += p0;
+                            ls1 += p1;
+                            pk[i2 >> 1] = pack_bf16x2(p0, p1);
+                        }
+                    }
+                };
+                // P is stored over S columns this thread has already read: [0,32) for the first thread of the pair,
+                // [96,128) for the second
+                const uint32_t p_col = s_t + 96u * half;
+                bool done = false;
+                if (j > 0) {
+                    // ---- one pass with the reference maximum as it stands: the exponentials of the first group run
+                    //      while the second group is still on its way from TMEM, and the row maximum (found on the
+                    //      side) only has to confirm that the reference may stay; if it may not, for some row of
+                    //      this warp, the tile is done again below with the two passes of a first tile.
+                    uint32_t pk0[16], pk1[16];
+                    const float mref = (m_used == -INFINITY) ? 0.f : m_used;
+                    tmem_ld32(s_t + 64u * half, r0);
+                    tmem_ld_wait();
+                    tmem_ld32(s_t + 64u * half + 32u, r1);
+                    exp_group(r0, bits0, mref, false, pk0);
+                    tmem_ld_wait();
+                    exp_group(r1, bits1, mref, false, pk1);
+                    // A score above the reference by more than 2^8 makes its p, and so the sum, exceed 2^8: the
+                    // sum (which is there anyway) serves as the alarm; the two-pass path then decides exactly.
+                    mx0 = mx1 = (ls0 + ls1 <= 256.0f) ? -INFINITY : INFINITY;
+                    float mt;
+                    ok = row_max(mt);
+                    if (!ok) break;
+                    if (!__any_sync(0xffffffffu, mt > m_used + RESCALE_LOG2)) {
+                        tmem_st16(p_col, pk0);
+                        tmem_st16(p_col + 16u, pk1);
+                        tmem_st_wait();
+                        l += ls0 + ls1;
+                        done = true;
+                    }
+                }
+                if (!done) {
+                    // ---- pass 1: maximum of this thread's 64 columns
+                    mx0 = mx1 = -INFINITY;
+                    ls0 = ls1 = 0.f;
+                    tmem_ld32(s_t + 64u * half, r0);
+                    tmem_ld32(s_t + 64u * half + 32u, r1);
+                    tmem_ld_wait();
+                    max_group(r0, bits0);
+                    max_group(r1, bits1);
+                    float mt;
+                    ok = row_max(mt);
+                    if (!ok) break;
+                    float alpha = 1.f;
+                    const bool need = mt > m_used + RESCALE_LOG2;  // also true on the first admissible tile
+                    if (need) {
+                        alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - mt);
+                        m_used = mt;
+                        l *= alpha;
+                    }
+                    if (__any_sync(0xffffffffu, need) && j > 0) {
+                        // rows of this warp change their reference maximum: rescale this thread's half of their
+                        // running outputs in TMEM.  The previous tile's P V must have landed first.
+                        ok = twait(2, bar(C::B_PVDONE + (int)((t - 1u) % SB)), ((t - 1u) / SB) & 1u);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int c = 0; c < DH; c += 32) {
+                            uint32_t o[32];
+                            tmem_ld32(o_t + (uint32_t)c, o);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i2 = 0; i2 < 32; ++i2) o[i2] = __float_as_uint(__uint_as_float(o[i2]) * alpha);
+                            tmem_st32(o_t + (uint32_t)c, o);
+                        }
+                        tmem_st_wait();
+                    }
+                    // ---- pass 2: p = 2^(s*scale - m) as packed bf16 pairs, 16 packed columns per 32-column group
+                    const float mref = (m_used == -INFINITY) ? 0.f : m_used;
+                    uint32_t pk[16];
+                    exp_group(r0, bits0, mref, false, pk);
+                    tmem_st16(p_col, pk);
+                    exp_group(r1, bits1, mref, false, pk);
+                    tmem_st16(p_col + 16u, pk);
+                    tmem_st_wait();
+                    l += ls0 + ls1;
+                }
                 tc_fence_before();
                 mbar_arrive(bar(C::B_PREADY + sb));
                 if (ws == 0 && lane == 0) SR_TRACE(2, 2, t);
