@@ -492,7 +492,7 @@ struct AttnPlan {
     int rows, n_rb, rows_per_block, rows_pad, chunk_tiles, items, tile_tokens, nodes_per_block, n_counters;
     int merge_mode;  // tcgen05 path: 0 = split sequences are merged inside the attention kernel, 2 = by a kernel after it
     bool use_tc;
-    size_t off_status, off_items, off_sorted, off_rank, off_tab, off_counters, off_po, off_pml, total;
+    size_t off_status, off_items, off_sorted, off_rank, off_tab, off_counters, off_po, off_pml, off_hand, total;
 };
 
 static int compute_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
@@ -596,6 +596,8 @@ static int compute_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_
     o += align_up((size_t)items * d->Hkv * p->rows_pad * d->D * 4, 256);
     p->off_pml = o;
     o += align_up((size_t)items * d->Hkv * p->rows_pad * 2 * 4, 256);
+    p->off_hand = o;
+    o += (size_t)ATTN_HAND_CTAS * 4 * 128 * 4;
     p->total = o + 256;
     return SPECROLL_OK;
 }
@@ -703,6 +705,7 @@ static int run_tree_attn(const specroll_attn_desc *d, const void *Q, const void 
     a.lse = lse;
     a.part_o = reinterpret_cast<float *>(ws + p.off_po);
     a.part_ml = reinterpret_cast<float *>(ws + p.off_pml);
+    a.hand = reinterpret_cast<float *>(ws + p.off_hand);
     a.B = d->B;
     a.N = d->N;
     a.Hq = d->Hq;

@@ -27,8 +27,11 @@ struct AttnArgs {
     // paged cache (tcgen05 kernel only): pool page of every 128-token tile; a chunk table row then carries the
     // sequence's first slot in this table instead of its first token
     const int32_t *page_table;
+    float *hand;                  // [ATTN_HAND_CTAS][4][128] per-CTA hand-over area between two groups of warps of the tcgen05 kernel
     int32_t merge_mode;           // chunks of a split sequence are merged 0: by the CTA that finishes last; 2: by a later kernel
 };
+
+constexpr int ATTN_HAND_CTAS = 256;  // CTAs the hand-over area is sized for (the grid is one CTA per SM)
 
 // tcgen05 kernel (tree_attn_tc.cu).  T_kv = total cached tokens.  Launches the main kernel only.
 int launch_attn_tc(const AttnArgs &a, const TopoMask &mask, int D, long long T_kv, int32_t *status, cudaStream_t st);

@@ -74,7 +74,7 @@ struct UnitDesc {
     int32_t valid, b, hkv, rb, n_splits, kv0, L, t_lo, n_it, has_tree, item, item0;
 };
 
-template <int D>
+template <int D, bool TEAMS>
 struct Cfg {
     static constexpr int NBOX = D / 64;
     static constexpr int SB = 3;   // S buffers
@@ -91,14 +91,17 @@ struct Cfg {
     // barrier slots
     static constexpr int B_FULL = 0, B_EMPTY = B_FULL + RS, B_SFULL = B_EMPTY + RS, B_PREADY = B_SFULL + SB,
                          B_PVDONE = B_PREADY + SB, B_QFULL = B_PVDONE + SB, B_QFREE = B_QFULL + QS,
-                         B_UFULL = B_QFREE + QS, B_UEMPTY = B_UFULL + 2, B_PAIR = B_UEMPTY + 2, B_ALL = B_PAIR + 4,
+                         B_UFULL = B_QFREE + QS, B_UEMPTY = B_UFULL + 2, B_X = B_UEMPTY + 2, B_ALL = B_X + 4,
                          B_OFULL = B_ALL + 1, B_OFREE = B_OFULL + 1, B_HFULL = B_OFREE + 1, B_HFREE = B_HFULL + 1,
                          N_BARS = B_HFREE + 1;
     static constexpr int BAR_BYTES = (8 * N_BARS + 15) / 16 * 16;
-    static constexpr int XCH_BYTES = 1024;  // per lane group 256 bytes: the pairs' partial maxima as bf16
-    // hand-over from the softmax warps to the output warps: two shares of the row sum and the reference maximum
-    static constexpr int HAND_BYTES = 3 * 128 * 4;
-    static constexpr int EXTRA = BAR_BYTES + 16 + XCH_BYTES + 2 * 64 + HAND_BYTES;  // barriers, slot/abort/ticket, exchange, ring
+    // exchange area: the rows' reference maxima as one softmax team leaves them for the other ([2][128] fp32), or
+    // the partial row maxima of the pairs (per lane group [2 slots][2 halves][32 lanes] bf16)
+    static constexpr int XCH_BYTES = 1024;
+    static constexpr int EXTRA = BAR_BYTES + 16 + XCH_BYTES + 2 * 64;  // barriers, slot/abort/ticket, exchange, ring
+    // hand-over from the softmax warps to the output warps (per row: each team's share of the sum and the
+    // reference maximum it is relative to): in global memory, one area per CTA, because shared memory is full
+    static constexpr int HAND_FLOATS = 4 * 128;
     // The operand tiles need 1024-byte alignment.  The dynamic shared window starts 1024-aligned on this
     // architecture (checked at run time: the kernel reports an error instead of running misaligned).
     static constexpr int USED = QS * Q_BYTES + RS * KV_BYTES + EXTRA;
@@ -125,14 +128,14 @@ __device__ __forceinline__ unsigned short bf16_bits_rn(float x) {
 __device__ __forceinline__ float bf16_bits_to_float(unsigned short b) { return __uint_as_float((uint32_t)b << 16); }
 }  // namespace attc
 
-template <int D>
-__global__ void __launch_bounds__(attc::Cfg<D>::THREADS, 1)
+template <int D, bool TEAMS>
+__global__ void __launch_bounds__(attc::Cfg<D, TEAMS>::THREADS, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKt,
                     const __grid_constant__ CUtensorMap tmVt, AttnArgs a, TopoMask mask,
                     int32_t *__restrict__ status) {
     using namespace attc;
-    using C = Cfg<D>;
+    using C = Cfg<D, TEAMS>;
     constexpr int DH = D / 2;  // accumulator columns per thread of a pair (rescaling)
     constexpr int SB = C::SB, RS = C::RS, QS = C::QS, THREADS = C::THREADS;
     extern __shared__ unsigned char smem_raw[];
@@ -149,7 +152,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     volatile int *tickets = reinterpret_cast<volatile int *>(extra + 8);
     unsigned char *xch_base = extra + 16;
     volatile UnitDesc *ring = reinterpret_cast<volatile UnitDesc *>(extra + 16 + C::XCH_BYTES);  // 2 slots of 64 bytes
-    volatile float *hand = reinterpret_cast<volatile float *>(extra + 16 + C::XCH_BYTES + 128);  // [l share 0 | l share 1 | m][128 rows]
+    float *hand = a.hand + (size_t)blockIdx.x * C::HAND_FLOATS;  // [l of team 0 | l of team 1 | m of team 0 | m of team 1][128 rows]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int N = a.N, G = a.G;
@@ -188,10 +191,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (threadIdx.x == 0) {
         for (int i = 0; i < C::N_BARS; ++i) {
             uint32_t count = 1;
-            if (i >= C::B_PREADY && i < C::B_PREADY + SB) count = C::SOFTMAX_THREADS;
+            // a tile's P comes from one team, or from all softmax threads
+            if (i >= C::B_PREADY && i < C::B_PREADY + SB) count = TEAMS ? C::SOFTMAX_THREADS / 2 : C::SOFTMAX_THREADS;
             // a unit's descriptor is read by the MMA threads, the softmax threads and the output threads
             if (i >= C::B_UEMPTY && i < C::B_UEMPTY + 2) count = C::MMA_WARPS + C::SOFTMAX_THREADS + C::OUT_THREADS;
-            if (i >= C::B_PAIR && i < C::B_PAIR + 4) count = 64;
+            // exchange barriers: per team (reference maxima), or per lane group (the pairs' partial maxima)
+            if (i >= C::B_X && i < C::B_X + 4) count = TEAMS ? C::SOFTMAX_THREADS / 2 : 64;
             if (i == C::B_ALL || i == C::B_OFREE || i == C::B_HFREE) count = C::OUT_THREADS;
             if (i == C::B_HFULL) count = C::SOFTMAX_THREADS;
             mbar_init(bar(i), count);
@@ -492,10 +497,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         const uint32_t p_t = tmem_base + C::S_COL + 128u * (uint32_t)sb;
 #pragma unroll
                         for (int kk = 0; kk < BN / 16; ++kk) {
-                            // 16 tokens per operation: 2048 bytes (128 address units) down the V tile; P of tokens 0-63
-                            // sits in columns [0,32) of the S buffer, of tokens 64-127 in columns [96,128), 8 packed
-                            // columns per operation
-                            const uint32_t pcol = kk < 4 ? 8u * kk : 64u + 8u * kk;
+                            // 16 tokens per operation: 2048 bytes (128 address units) down the V tile, 8 packed columns
+                            // of P.  Teams: P sits in columns [0,64) of the S buffer; pairs: tokens 0-63 in columns
+                            // [0,32), tokens 64-127 in columns [96,128)
+                            const uint32_t pcol = TEAMS ? 8u * kk : (kk < 4 ? 8u * kk : 64u + 8u * kk);
                             umma_ts(o_t, p_t + pcol, desc(v_lo + 128u * kk), idesc_pv, (kk > 0 || j > 0) ? 1u : 0u);
                         }
                         umma_commit(bar(C::B_EMPTY + vs));
@@ -532,8 +537,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             ok = twait(1, bar(C::B_HFULL), u & 1u);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const float lt = hand[row] + hand[128 + row];
-            const float m_used = hand[256 + row];
+            // each team's share of the sum is relative to the reference as that team last knew it
+            const float l0 = __ldcg(hand + row), l1 = __ldcg(hand + 128 + row);
+            const float m0 = __ldcg(hand + 256 + row), m1 = __ldcg(hand + 384 + row);
+            const float m_used = fmaxf(m0, m1);
+            const float lt = (m0 == -INFINITY ? 0.f : l0 * ex2_approx(m0 - m_used)) +
+                             (m1 == -INFINITY ? 0.f : l1 * ex2_approx(m1 - m_used));
             mbar_arrive(bar(C::B_HFREE));
             // ---- the unit's last P V (operations complete in issue order, so it covers all)
             ok = twait(2, bar(C::B_OFULL), u & 1u);
@@ -606,219 +615,428 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (lane == 0 && lg == 2) SR_TRACE(3, 4, u);
         }
     } else {
-        // ------------------------------------------------------------------ softmax (8 warps, two threads per query row)
-        const int ws = warp - (1 + C::MMA_WARPS);
-        const int half = ws >> 2;  // which 64 of a tile's 128 columns, and which D/2 accumulator columns
-        const int lg = warp & 3;   // TMEM lane group of this warp
-        const int row = lg * 32 + lane;
-        const uint32_t t_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
-        const uint32_t o_t = t_lane + C::O_COL + (uint32_t)(half * DH);
-        const float sc = a.scale_log2;
-        // exchange area of this lane group, 256 bytes, touched by the group's two warps only: the partial maxima
-        // as bf16 [2 slots][2 halves][32 lanes]
-        volatile unsigned short *xm = reinterpret_cast<volatile unsigned short *>(xch_base + lg * 256);
-        uint32_t gt = 0;  // tiles processed so far (all units)
-        uint32_t use_pair = 0;
-        const uint32_t pair_bar = bar(C::B_PAIR + lg);
-        bool ok = true;
-        for (uint32_t u = 0; ok; ++u) {
-            const int slot = (int)(u & 1u);
-            ok = twait(0, bar(C::B_UFULL + slot), (u >> 1) & 1u);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            const int valid = ring[slot].valid, rb = ring[slot].rb, L = ring[slot].L, t_lo = ring[slot].t_lo;
-            const int n_it = ring[slot].n_it, has_tree = ring[slot].has_tree;
-            mbar_arrive(bar(C::B_UEMPTY + slot));
-            if (!valid) break;
-            const int gr = rb * a.rows_per_block + row;
-            const bool row_ok = row < a.rows_per_block && gr < a.rows;
-            const uint64_t anc = row_ok ? mask.anc[gr / G] : 0ull;
-            float m_used = -INFINITY, l = 0.f;  // l: this thread's share (its 64 columns of every tile)
-            for (int j = 0; j < n_it; ++j) {
-                const uint32_t t = gt + (uint32_t)j;
-                const int sb = (int)(t % SB);
-                ok = twait(1, bar(C::B_SFULL + sb), (t / SB) & 1u);
+        if constexpr (TEAMS) {
+            // ------------------------------------------------------------------ softmax (two teams of 4 warps)
+            // Team (t & 1) takes tile t, one thread per query row, so that the fixed latencies of a tile (TMEM
+            // loads and stores, barrier round trips) of one team run under the other team's exponentials.  The
+            // row's reference maximum is common to both teams, each keeps its own share of the row sum.  After the
+            // first two tiles of a unit a tile takes ONE pass: the exponentials are taken against the reference as
+            // this team knows it, nothing is stored yet, and the tile's sum serves as the alarm (a score more than
+            // 2^8 above the reference makes the sum exceed 2^8).  Then the thread looks at what the other team
+            // left after the tile before: if that reference differs from its own, or the alarm went off (both
+            // rare), the tile is done again from S with the two passes of a first tile, which can move the
+            // reference and rescale the accumulator.  The result is the same as doing two passes every time.
+            const int ws = warp - (1 + C::MMA_WARPS);
+            const int team = ws >> 2;
+            const int lg = warp & 3;  // TMEM lane group of this warp
+            const int row = lg * 32 + lane;
+            const uint32_t t_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
+            const uint32_t o_t = t_lane + C::O_COL;
+            const float sc = a.scale_log2;
+            volatile float *mref = reinterpret_cast<volatile float *>(xch_base);  // [2 slots][128 rows]
+            uint32_t gt = 0;  // tiles so far (all units, both teams)
+            bool ok = true;
+            for (uint32_t u = 0; ok; ++u) {
+                const int slot = (int)(u & 1u);
+                ok = twait(0, bar(C::B_UFULL + slot), (u >> 1) & 1u);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                tc_fence_after();
-                if (ws == 0 && lane == 0) SR_TRACE(2, 1, t);
-                const uint32_t s_t = t_lane + C::S_COL + 128u * (uint32_t)sb;
-                const bool tree = has_tree && (j == n_it - 1);
-                // columns >= limit are outside the sequence; this thread's columns start at 64 * half
-                const int limit = (tree ? 64 : (L - (t_lo + j) * BN)) - 64 * half;
-                const bool full = !tree && limit >= 64;
-                uint32_t bits0, bits1;  // admissible columns among this thread's 64, in two groups of 32
-                if (full) {
-                    bits0 = bits1 = 0xffffffffu;
-                } else if (tree) {
-                    bits0 = half == 0 ? (uint32_t)anc : 0u;
-                    bits1 = half == 0 ? (uint32_t)(anc >> 32) : 0u;
-                } else {
-                    bits0 = limit >= 32 ? 0xffffffffu : (limit <= 0 ? 0u : ((1u << limit) - 1u));
-                    bits1 = limit >= 64 ? 0xffffffffu : (limit <= 32 ? 0u : ((1u << (limit - 32)) - 1u));
-                }
-                uint32_t r0[32], r1[32];
-                float mx0 = -INFINITY, mx1 = -INFINITY;
-                auto max_group = [&](const uint32_t(&src)[32], uint32_t bc) {
-                    if (full) {
-#pragma unroll
-                        for (int i2 = 0; i2 < 32; i2 += 2) {
-                            mx0 = fmaxf(mx0, __uint_as_float(src[i2]));
-                            mx1 = fmaxf(mx1, __uint_as_float(src[i2 + 1]));
-                        }
-                    } else {
-#pragma unroll
-                        for (int i2 = 0; i2 < 32; ++i2)
-                            if ((bc >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(src[i2]));
-                    }
-                };
-                // Exchanges the partial maximum with the thread that has the row's other 64 columns and returns the
-                // row's maximum (scaled).  It travels as bf16: any common reference close to the true maximum
-                // will do.  Two slots, alternating, so that a fast thread's next write cannot overtake a slow read.
-                auto row_max = [&](float &mt) -> bool {
-                    const unsigned short mine = bf16_bits_rn(fmaxf(mx0, mx1));
-                    const int px = (int)(use_pair & 1u) * 64;
-                    xm[px + half * 32 + lane] = mine;
-#ifdef SPECROLL_TRACE
-                    const long long tps_ = clock64();
-#endif
-                    bool k_ = group_sync(pair_bar, use_pair, abort_flag);
-#ifdef SPECROLL_TRACE
-                    prof[4] += (unsigned long long)(clock64() - tps_);
-#endif
-                    k_ = __all_sync(0xffffffffu, k_);
-                    mt = fmaxf(bf16_bits_to_float(mine), bf16_bits_to_float(xm[px + (half ^ 1) * 32 + lane])) * sc;
-                    return k_;
-                };
-                // p = 2^(s*scale - m) of one 32-column group as 16 packed bf16 pairs; adds the values to ls0 / ls1
-                // and, if asked to, folds the scores into mx0 / mx1.  (Two copies of each loop: with the mask test
-                // inside one loop the compiler evaluates it for every element of the full tiles too.)
-                float ls0 = 0.f, ls1 = 0.f;
-                auto exp_group = [&](const uint32_t(&src)[32], uint32_t bc, float mref, bool with_max, uint32_t(&pk)[16]) {
-                    if (full) {
-#pragma unroll
-                        for (int i2 = 0; i2 < 32; i2 += 2) {
-                            const float s0 = __uint_as_float(src[i2]), s1 = __uint_as_float(src[i2 + 1]);
-                            if (with_max) {
-                                mx0 = fmaxf(mx0, s0);
-                                mx1 = fmaxf(mx1, s1);
-                            }
-                            const float p0 = ex2_approx(fmaf(s0, sc, -mref));
-                            const float p1 = ex2_approx(fmaf(s1, sc, -mref));
-                            ls0 += p0;
-                            ls1 += p1;
-                            pk[i2 >> 1] = pack_bf16x2(p0, p1);
-                        }
-                    } else {
-#pragma unroll
-                        for (int i2 = 0; i2 < 32; i2 += 2) {
-                            const float s0 = __uint_as_float(src[i2]), s1 = __uint_as_float(src[i2 + 1]);
-                            const bool b0 = (bc >> i2) & 1u, b1 = (bc >> (i2 + 1)) & 1u;
-                            if (with_max) {
-                                if (b0) mx0 = fmaxf(mx0, s0);
-                                if (b1) mx0 = fmaxf(mx0, s1);
-                            }
-                            const float p0 = b0 ? ex2_approx(fmaf(s0, sc, -mref)) : 0.f;
-                            const float p1 = b1 ? ex2_approx(fmaf(s1, sc, -mref)) : 0.f;
-                            ls0 += p0;
-                            ls1 += p1;
-                            pk[i2 >> 1] = pack_bf16x2(p0, p1);
-                        }
-                    }
-                };
-                // P is stored over S columns this thread has already read: [0,32) for the first thread of the pair,
-                // [96,128) for the second
-                const uint32_t p_col = s_t + 96u * half;
-                bool done = false;
-                if (j > 0) {
-                    // ---- one pass with the reference maximum as it stands: the exponentials of the first group run
-                    //      while the second group is still on its way from TMEM, and the row maximum (found on the
-                    //      side) only has to confirm that the reference may stay; if it may not, for some row of
-                    //      this warp, the tile is done again below with the two passes of a first tile.
-                    uint32_t pk0[16], pk1[16];
-                    const float mref = (m_used == -INFINITY) ? 0.f : m_used;
-                    tmem_ld32(s_t + 64u * half, r0);
-                    tmem_ld_wait();
-                    tmem_ld32(s_t + 64u * half + 32u, r1);
-                    exp_group(r0, bits0, mref, false, pk0);
-                    tmem_ld_wait();
-                    exp_group(r1, bits1, mref, false, pk1);
-                    // A score above the reference by more than 2^8 makes its p, and so the sum, exceed 2^8: the
-                    // sum (which is there anyway) serves as the alarm; the two-pass path then decides exactly.
-                    mx0 = mx1 = (ls0 + ls1 <= 256.0f) ? -INFINITY : INFINITY;
-                    float mt;
-                    ok = row_max(mt);
+                const int valid = ring[slot].valid, rb = ring[slot].rb, L = ring[slot].L, t_lo = ring[slot].t_lo;
+                const int n_it = ring[slot].n_it, has_tree = ring[slot].has_tree;
+                mbar_arrive(bar(C::B_UEMPTY + slot));
+                if (!valid) break;
+                const int gr = rb * a.rows_per_block + row;
+                const bool row_ok = row < a.rows_per_block && gr < a.rows;
+                const uint64_t anc = row_ok ? mask.anc[gr / G] : 0ull;
+                float m_used = -INFINITY, l = 0.f;  // reference maximum as this thread knows it; this team's share of the sum
+                for (int j = (int)((gt ^ (uint32_t)team) & 1u); j < n_it; j += 2) {
+                    const uint32_t t = gt + (uint32_t)j;
+                    const int sb = (int)(t % SB);
+                    ok = twait(1, bar(C::B_SFULL + sb), (t / SB) & 1u);
+                    ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                    if (!__any_sync(0xffffffffu, mt > m_used + RESCALE_LOG2)) {
-                        tmem_st16(p_col, pk0);
-                        tmem_st16(p_col + 16u, pk1);
+                    tc_fence_after();
+                    if (ws == 0 && lane == 0) SR_TRACE(2, 1, t);
+                    const uint32_t s_t = t_lane + C::S_COL + 128u * (uint32_t)sb;
+                    const bool tree = has_tree && (j == n_it - 1);
+                    // columns >= limit are outside the sequence (a tree tile has at most 64 rows of tree K/V)
+                    const int limit = tree ? 64 : (L - (t_lo + j) * BN);
+                    const bool full = !tree && limit >= BN;
+                    // admissible columns of 32-column group c
+                    auto bits_of = [&](int c) -> uint32_t {
+                        if (full) return 0xffffffffu;
+                        if (tree) return c == 0 ? (uint32_t)anc : (c == 1 ? (uint32_t)(anc >> 32) : 0u);
+                        const int lim = limit - 32 * c;
+                        return lim >= 32 ? 0xffffffffu : (lim <= 0 ? 0u : ((1u << lim) - 1u));
+                    };
+                    // p = 2^(s*scale - m) of one 32-column group as 16 packed bf16 pairs; adds the values to ls0 / ls1.
+                    // (Two copies of the loop: with the mask test inside one loop the compiler evaluates it for every
+                    // element of the full tiles too.)
+                    float ls0 = 0.f, ls1 = 0.f;
+                    auto exp_group = [&](const uint32_t(&src)[32], uint32_t bc, float mref_, uint32_t *pk) {
+                        if (full) {
+    #pragma unroll
+                            for (int i2 = 0; i2 < 32; i2 += 2) {
+                                const float p0 = ex2_approx(fmaf(__uint_as_float(src[i2]), sc, -mref_));
+                                const float p1 = ex2_approx(fmaf(__uint_as_float(src[i2 + 1]), sc, -mref_));
+                                ls0 += p0;
+                                ls1 += p1;
+                                pk[i2 >> 1] = pack_bf16x2(p0, p1);
+                            }
+                        } else {
+    #pragma unroll
+                            for (int i2 = 0; i2 < 32; i2 += 2) {
+                                const bool b0 = (bc >> i2) & 1u, b1 = (bc >> (i2 + 1)) & 1u;
+                                const float p0 = b0 ? ex2_approx(fmaf(__uint_as_float(src[i2]), sc, -mref_)) : 0.f;
+                                const float p1 = b1 ? ex2_approx(fmaf(__uint_as_float(src[i2 + 1]), sc, -mref_)) : 0.f;
+                                ls0 += p0;
+                                ls1 += p1;
+                                pk[i2 >> 1] = pack_bf16x2(p0, p1);
+                            }
+                        }
+                    };
+                    // The reference the other team left after tile t - 1.  Every tile waits for its predecessor's (also
+                    // the first tile of a unit, which does not use the value), so a slot is never written twice
+                    // between two reads.
+                    float m_pub = -INFINITY;
+                    auto predecessor = [&]() -> bool {
+                        if (t == 0u) return true;
+                        bool k_ = twait(4, bar(C::B_X + (int)((t - 1u) & 1u)), ((t - 1u) >> 1) & 1u);
+                        k_ = __all_sync(0xffffffffu, k_);
+                        if (k_ && j > 0) m_pub = mref[((t - 1u) & 1u) * 128u + row];
+                        return k_;
+                    };
+                    uint32_t x[32];
+                    bool done = false;
+                    if (j >= 2) {
+                        // ---- one pass against the reference as it stands; P stays in registers until the verdict
+                        uint32_t pk[64];
+                        const float mref_ = (m_used == -INFINITY) ? 0.f : m_used;
+    #pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            tmem_ld32(s_t + 32u * (uint32_t)c, x);
+                            tmem_ld_wait();
+                            exp_group(x, bits_of(c), mref_, pk + 16 * c);
+                        }
+                        ok = predecessor();
+                        if (!ok) break;
+                        const bool bad = !(ls0 + ls1 <= 256.0f) || m_pub != m_used;
+                        if (!__any_sync(0xffffffffu, bad)) {
+    #pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                uint32_t q[16];
+    #pragma unroll
+                                for (int i2 = 0; i2 < 16; ++i2) q[i2] = pk[16 * c + i2];
+                                tmem_st16(s_t + 16u * (uint32_t)c, q);
+                            }
+                            tmem_st_wait();
+                            l += ls0 + ls1;
+                            mref[(t & 1u) * 128u + row] = m_used;
+                            mbar_arrive(bar(C::B_X + (int)(t & 1u)));
+                            done = true;
+                        }
+                    }
+                    if (!done) {
+                        // ---- two passes.  First the row's maximum over the tile ...
+                        ls0 = ls1 = 0.f;
+                        float mx0 = -INFINITY, mx1 = -INFINITY;
+    #pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            tmem_ld32(s_t + 32u * (uint32_t)c, x);
+                            tmem_ld_wait();
+                            const uint32_t bc = bits_of(c);
+                            if (full) {
+    #pragma unroll
+                                for (int i2 = 0; i2 < 32; i2 += 2) {
+                                    mx0 = fmaxf(mx0, __uint_as_float(x[i2]));
+                                    mx1 = fmaxf(mx1, __uint_as_float(x[i2 + 1]));
+                                }
+                            } else {
+    #pragma unroll
+                                for (int i2 = 0; i2 < 32; ++i2)
+                                    if ((bc >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(x[i2]));
+                            }
+                        }
+                        const float mt = fmaxf(mx0, mx1) * sc;
+                        // ... then the reference: the other team's after the tile before (this thread's share of the sum
+                        // moves with it), raised if this tile's maximum is more than 2^8 above it
+                        ok = predecessor();
+                        if (!ok) break;
+                        if (j > 0 && m_pub != m_used) {
+                            l *= (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_pub);
+                            m_used = m_pub;
+                        }
+                        float alpha = 1.f;
+                        const bool need = mt > m_used + RESCALE_LOG2;  // also true on the first admissible tile
+                        if (need) {
+                            alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - mt);
+                            m_used = mt;
+                            l *= alpha;
+                        }
+                        mref[(t & 1u) * 128u + row] = m_used;  // known before the exponentials: the next tile need not wait for them
+                        mbar_arrive(bar(C::B_X + (int)(t & 1u)));
+                        if (__any_sync(0xffffffffu, need) && j > 0) {
+                            // rows of this warp change their reference maximum: rescale their running outputs in TMEM.
+                            // The previous tile's P V must have landed first (this tile's waits for the P written below).
+                            ok = twait(2, bar(C::B_PVDONE + (int)((t - 1u) % SB)), ((t - 1u) / SB) & 1u);
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (!ok) break;
+                            tc_fence_after();
+    #pragma unroll 1
+                            for (int c = 0; c < D; c += 32) {
+                                tmem_ld32(o_t + (uint32_t)c, x);
+                                tmem_ld_wait();
+    #pragma unroll
+                                for (int i2 = 0; i2 < 32; ++i2) x[i2] = __float_as_uint(__uint_as_float(x[i2]) * alpha);
+                                tmem_st32(o_t + (uint32_t)c, x);
+                            }
+                            tmem_st_wait();
+                        }
+                        // ... then p = 2^(s*scale - m) as packed bf16 pairs, group by group; 16 packed columns go over S
+                        // columns that have been read already
+                        const float mref_ = (m_used == -INFINITY) ? 0.f : m_used;
+    #pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t q[16];
+                            tmem_ld32(s_t + 32u * (uint32_t)c, x);
+                            tmem_ld_wait();
+                            exp_group(x, bits_of(c), mref_, q);
+                            tmem_st16(s_t + 16u * (uint32_t)c, q);
+                        }
                         tmem_st_wait();
                         l += ls0 + ls1;
-                        done = true;
                     }
+                    tc_fence_before();
+                    mbar_arrive(bar(C::B_PREADY + sb));
+                    if (ws == 0 && lane == 0) SR_TRACE(2, 2, t);
                 }
-                if (!done) {
-                    // ---- pass 1: maximum of this thread's 64 columns
-                    mx0 = mx1 = -INFINITY;
-                    ls0 = ls1 = 0.f;
-                    tmem_ld32(s_t + 64u * half, r0);
-                    tmem_ld32(s_t + 64u * half + 32u, r1);
-                    tmem_ld_wait();
-                    max_group(r0, bits0);
-                    max_group(r1, bits1);
-                    float mt;
-                    ok = row_max(mt);
-                    if (!ok) break;
-                    float alpha = 1.f;
-                    const bool need = mt > m_used + RESCALE_LOG2;  // also true on the first admissible tile
-                    if (need) {
-                        alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - mt);
-                        m_used = mt;
-                        l *= alpha;
-                    }
-                    if (__any_sync(0xffffffffu, need) && j > 0) {
-                        // rows of this warp change their reference maximum: rescale this thread's half of their
-                        // running outputs in TMEM.  The previous tile's P V must have landed first.
-                        ok = twait(2, bar(C::B_PVDONE + (int)((t - 1u) % SB)), ((t - 1u) / SB) & 1u);
-                        ok = __all_sync(0xffffffffu, ok);
-                        if (!ok) break;
-                        tc_fence_after();
-#pragma unroll 1
-                        for (int c = 0; c < DH; c += 32) {
-                            uint32_t o[32];
-                            tmem_ld32(o_t + (uint32_t)c, o);
-                            tmem_ld_wait();
-#pragma unroll
-                            for (int i2 = 0; i2 < 32; ++i2) o[i2] = __float_as_uint(__uint_as_float(o[i2]) * alpha);
-                            tmem_st32(o_t + (uint32_t)c, o);
-                        }
-                        tmem_st_wait();
-                    }
-                    // ---- pass 2: p = 2^(s*scale - m) as packed bf16 pairs, 16 packed columns per 32-column group
-                    const float mref = (m_used == -INFINITY) ? 0.f : m_used;
-                    uint32_t pk[16];
-                    exp_group(r0, bits0, mref, false, pk);
-                    tmem_st16(p_col, pk);
-                    exp_group(r1, bits1, mref, false, pk);
-                    tmem_st16(p_col + 16u, pk);
-                    tmem_st_wait();
-                    l += ls0 + ls1;
-                }
-                tc_fence_before();
-                mbar_arrive(bar(C::B_PREADY + sb));
-                if (ws == 0 && lane == 0) SR_TRACE(2, 2, t);
+                if (!ok) break;
+                // ---- end of the unit: each team leaves its share of the sum and the reference it is relative to for
+                //      the output warps and goes on with the next unit.  Those wait for the unit's last P V themselves.
+                gt += (uint32_t)n_it;
+                if (ws == 0 && lane == 0) SR_TRACE(2, 3, u);
+                ok = twait(3, bar(C::B_HFREE), (u & 1u) ^ 1u);  // the values of the unit before have been taken
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                hand[team * 128 + row] = l;
+                hand[256 + team * 128 + row] = m_used;
+                mbar_arrive(bar(C::B_HFULL));
             }
-            if (!ok) break;
-            // ---- hand the row's reference maximum and this thread's share of its sum to the output warps
-            //      and go on with the next unit; they wait for the unit's last P V themselves
-            gt += (uint32_t)n_it;
-            if (ws == 0 && lane == 0) SR_TRACE(2, 3, u);
-            ok = twait(3, bar(C::B_HFREE), (u & 1u) ^ 1u);  // the values of the unit before have been taken
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            hand[half * 128 + row] = l;
-            if (half == 0) hand[256 + row] = m_used;
-            mbar_arrive(bar(C::B_HFULL));
+        } else {
+            // ------------------------------------------------------------------ softmax (8 warps, two threads per query row)
+            const int ws = warp - (1 + C::MMA_WARPS);
+            const int half = ws >> 2;  // which 64 of a tile's 128 columns, and which D/2 accumulator columns
+            const int lg = warp & 3;   // TMEM lane group of this warp
+            const int row = lg * 32 + lane;
+            const uint32_t t_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
+            const uint32_t o_t = t_lane + C::O_COL + (uint32_t)(half * DH);
+            const float sc = a.scale_log2;
+            // exchange area of this lane group, 256 bytes, touched by the group's two warps only: the partial maxima
+            // as bf16 [2 slots][2 halves][32 lanes]
+            volatile unsigned short *xm = reinterpret_cast<volatile unsigned short *>(xch_base + lg * 256);
+            uint32_t gt = 0;  // tiles processed so far (all units)
+            uint32_t use_pair = 0;
+            const uint32_t pair_bar = bar(C::B_X + lg);
+            bool ok = true;
+            for (uint32_t u = 0; ok; ++u) {
+                const int slot = (int)(u & 1u);
+                ok = twait(0, bar(C::B_UFULL + slot), (u >> 1) & 1u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const int valid = ring[slot].valid, rb = ring[slot].rb, L = ring[slot].L, t_lo = ring[slot].t_lo;
+                const int n_it = ring[slot].n_it, has_tree = ring[slot].has_tree;
+                mbar_arrive(bar(C::B_UEMPTY + slot));
+                if (!valid) break;
+                const int gr = rb * a.rows_per_block + row;
+                const bool row_ok = row < a.rows_per_block && gr < a.rows;
+                const uint64_t anc = row_ok ? mask.anc[gr / G] : 0ull;
+                float m_used = -INFINITY, l = 0.f;  // l: this thread's share (its 64 columns of every tile)
+                for (int j = 0; j < n_it; ++j) {
+                    const uint32_t t = gt + (uint32_t)j;
+                    const int sb = (int)(t % SB);
+                    ok = twait(1, bar(C::B_SFULL + sb), (t / SB) & 1u);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (ws == 0 && lane == 0) SR_TRACE(2, 1, t);
+                    const uint32_t s_t = t_lane + C::S_COL + 128u * (uint32_t)sb;
+                    const bool tree = has_tree && (j == n_it - 1);
+                    // columns >= limit are outside the sequence; this thread's columns start at 64 * half
+                    const int limit = (tree ? 64 : (L - (t_lo + j) * BN)) - 64 * half;
+                    const bool full = !tree && limit >= 64;
+                    uint32_t bits0, bits1;  // admissible columns among this thread's 64, in two groups of 32
+                    if (full) {
+                        bits0 = bits1 = 0xffffffffu;
+                    } else if (tree) {
+                        bits0 = half == 0 ? (uint32_t)anc : 0u;
+                        bits1 = half == 0 ? (uint32_t)(anc >> 32) : 0u;
+                    } else {
+                        bits0 = limit >= 32 ? 0xffffffffu : (limit <= 0 ? 0u : ((1u << limit) - 1u));
+                        bits1 = limit >= 64 ? 0xffffffffu : (limit <= 32 ? 0u : ((1u << (limit - 32)) - 1u));
+                    }
+                    uint32_t r0[32], r1[32];
+                    float mx0 = -INFINITY, mx1 = -INFINITY;
+                    auto max_group = [&](const uint32_t(&src)[32], uint32_t bc) {
+                        if (full) {
+    #pragma unroll
+                            for (int i2 = 0; i2 < 32; i2 += 2) {
+                                mx0 = fmaxf(mx0, __uint_as_float(src[i2]));
+                                mx1 = fmaxf(mx1, __uint_as_float(src[i2 + 1]));
+                            }
+                        } else {
+    #pragma unroll
+                            for (int i2 = 0; i2 < 32; ++i2)
+                                if ((bc >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(src[i2]));
+                        }
+                    };
+                    // Exchanges the partial maximum with the thread that has the row's other 64 columns and returns the
+                    // row's maximum (scaled).  It travels as bf16: any common reference close to the true maximum
+                    // will do.  Two slots, alternating, so that a fast thread's next write cannot overtake a slow read.
+                    auto row_max = [&](float &mt) -> bool {
+                        const unsigned short mine = bf16_bits_rn(fmaxf(mx0, mx1));
+                        const int px = (int)(use_pair & 1u) * 64;
+                        xm[px + half * 32 + lane] = mine;
+    #ifdef SPECROLL_TRACE
+                        const long long tps_ = clock64();
+    #endif
+                        bool k_ = group_sync(pair_bar, use_pair, abort_flag);
+    #ifdef SPECROLL_TRACE
+                        prof[4] += (unsigned long long)(clock64() - tps_);
+    #endif
+                        k_ = __all_sync(0xffffffffu, k_);
+                        mt = fmaxf(bf16_bits_to_float(mine), bf16_bits_to_float(xm[px + (half ^ 1) * 32 + lane])) * sc;
+                        return k_;
+                    };
+                    // p = 2^(s*scale - m) of one 32-column group as 16 packed bf16 pairs; adds the values to ls0 / ls1
+                    // and, if asked to, folds the scores into mx0 / mx1.  (Two copies of each loop: with the mask test
+                    // inside one loop the compiler evaluates it for every element of the full tiles too.)
+                    float ls0 = 0.f, ls1 = 0.f;
+                    auto exp_group = [&](const uint32_t(&src)[32], uint32_t bc, float mref, bool with_max, uint32_t(&pk)[16]) {
+                        if (full) {
+    #pragma unroll
+                            for (int i2 = 0; i2 < 32; i2 += 2) {
+                                const float s0 = __uint_as_float(src[i2]), s1 = __uint_as_float(src[i2 + 1]);
+                                if (with_max) {
+                                    mx0 = fmaxf(mx0, s0);
+                                    mx1 = fmaxf(mx1, s1);
+                                }
+                                const float p0 = ex2_approx(fmaf(s0, sc, -mref));
+                                const float p1 = ex2_approx(fmaf(s1, sc, -mref));
+                                ls0 += p0;
+                                ls1 += p1;
+                                pk[i2 >> 1] = pack_bf16x2(p0, p1);
+                            }
+                        } else {
+    #pragma unroll
+                            for (int i2 = 0; i2 < 32; i2 += 2) {
+                                const float s0 = __uint_as_float(src[i2]), s1 = __uint_as_float(src[i2 + 1]);
+                                const bool b0 = (bc >> i2) & 1u, b1 = (bc >> (i2 + 1)) & 1u;
+                                if (with_max) {
+                                    if (b0) mx0 = fmaxf(mx0, s0);
+                                    if (b1) mx0 = fmaxf(mx0, s1);
+                                }
+                                const float p0 = b0 ? ex2_approx(fmaf(s0, sc, -mref)) : 0.f;
+                                const float p1 = b1 ? ex2_approx(fmaf(s1, sc, -mref)) : 0.f;
+                                ls0 += p0;
+                                ls1 += p1;
+                                pk[i2 >> 1] = pack_bf16x2(p0, p1);
+                            }
+                        }
+                    };
+                    // P is stored over S columns this thread has already read: [0,32) for the first thread of the pair,
+                    // [96,128) for the second
+                    const uint32_t p_col = s_t + 96u * half;
+                    bool done = false;
+                    if (j > 0) {
+                        // ---- one pass with the reference maximum as it stands: the exponentials of the first group run
+                        //      while the second group is still on its way from TMEM, and the row maximum (found on the
+                        //      side) only has to confirm that the reference may stay; if it may not, for some row of
+                        //      this warp, the tile is done again below with the two passes of a first tile.
+                        uint32_t pk0[16], pk1[16];
+                        const float mref = (m_used == -INFINITY) ? 0.f : m_used;
+                        tmem_ld32(s_t + 64u * half, r0);
+                        tmem_ld_wait();
+                        tmem_ld32(s_t + 64u * half + 32u, r1);
+                        exp_group(r0, bits0, mref, false, pk0);
+                        tmem_ld_wait();
+                        exp_group(r1, bits1, mref, false, pk1);
+                        // A score above the reference by more than 2^8 makes its p, and so the sum, exceed 2^8: the
+                        // sum (which is there anyway) serves as the alarm; the two-pass path then decides exactly.
+                        mx0 = mx1 = (ls0 + ls1 <= 256.0f) ? -INFINITY : INFINITY;
+                        float mt;
+                        ok = row_max(mt);
+                        if (!ok) break;
+                        if (!__any_sync(0xffffffffu, mt > m_used + RESCALE_LOG2)) {
+                            tmem_st16(p_col, pk0);
+                            tmem_st16(p_col + 16u, pk1);
+                            tmem_st_wait();
+                            l += ls0 + ls1;
+                            done = true;
+                        }
+                    }
+                    if (!done) {
+                        // ---- pass 1: maximum of this thread's 64 columns
+                        mx0 = mx1 = -INFINITY;
+                        ls0 = ls1 = 0.f;
+                        tmem_ld32(s_t + 64u * half, r0);
+                        tmem_ld32(s_t + 64u * half + 32u, r1);
+                        tmem_ld_wait();
+                        max_group(r0, bits0);
+                        max_group(r1, bits1);
+                        float mt;
+                        ok = row_max(mt);
+                        if (!ok) break;
+                        float alpha = 1.f;
+                        const bool need = mt > m_used + RESCALE_LOG2;  // also true on the first admissible tile
+                        if (need) {
+                            alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - mt);
+                            m_used = mt;
+                            l *= alpha;
+                        }
+                        if (__any_sync(0xffffffffu, need) && j > 0) {
+                            // rows of this warp change their reference maximum: rescale this thread's half of their
+                            // running outputs in TMEM.  The previous tile's P V must have landed first.
+                            ok = twait(2, bar(C::B_PVDONE + (int)((t - 1u) % SB)), ((t - 1u) / SB) & 1u);
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (!ok) break;
+                            tc_fence_after();
+    #pragma unroll 1
+                            for (int c = 0; c < DH; c += 32) {
+                                uint32_t o[32];
+                                tmem_ld32(o_t + (uint32_t)c, o);
+                                tmem_ld_wait();
+    #pragma unroll
+                                for (int i2 = 0; i2 < 32; ++i2) o[i2] = __float_as_uint(__uint_as_float(o[i2]) * alpha);
+                                tmem_st32(o_t + (uint32_t)c, o);
+                            }
+                            tmem_st_wait();
+                        }
+                        // ---- pass 2: p = 2^(s*scale - m) as packed bf16 pairs, 16 packed columns per 32-column group
+                        const float mref = (m_used == -INFINITY) ? 0.f : m_used;
+                        uint32_t pk[16];
+                        exp_group(r0, bits0, mref, false, pk);
+                        tmem_st16(p_col, pk);
+                        exp_group(r1, bits1, mref, false, pk);
+                        tmem_st16(p_col + 16u, pk);
+                        tmem_st_wait();
+                        l += ls0 + ls1;
+                    }
+                    tc_fence_before();
+                    mbar_arrive(bar(C::B_PREADY + sb));
+                    if (ws == 0 && lane == 0) SR_TRACE(2, 2, t);
+                }
+                if (!ok) break;
+                // ---- hand the row's reference maximum and this thread's share of its sum to the output warps
+                //      and go on with the next unit; they wait for the unit's last P V themselves
+                gt += (uint32_t)n_it;
+                if (ws == 0 && lane == 0) SR_TRACE(2, 3, u);
+                ok = twait(3, bar(C::B_HFREE), (u & 1u) ^ 1u);  // the values of the unit before have been taken
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                hand[half * 128 + row] = l;
+                hand[256 + half * 128 + row] = m_used;  // the same value from both threads of the pair
+                mbar_arrive(bar(C::B_HFULL));
+            }
         }
     }
 
@@ -862,9 +1080,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
 }
 
-template <int D>
+template <int D, bool TEAMS>
 static int launch_tc(const AttnArgs &a, const TopoMask &mask, long long T_kv, int32_t *status, cudaStream_t st) {
-    using C = attc::Cfg<D>;
+    using C = attc::Cfg<D, TEAMS>;
     CUtensorMap tmQ, tmK, tmV, tmKt, tmVt;
     int rc;
     const uint64_t tree_rows = (uint64_t)a.B * a.N;
@@ -883,10 +1101,11 @@ static int launch_tc(const AttnArgs &a, const TopoMask &mask, long long T_kv, in
         int dev = 0;
         SR_CUDA_TRY(cudaGetDevice(&dev));
         SR_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-        SR_CUDA_TRY(cudaFuncSetAttribute(tree_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+        SR_CUDA_TRY(cudaFuncSetAttribute(tree_attn_tc_kernel<D, TEAMS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
     }
-    const unsigned grid = (unsigned)(a.total_work < n_sm ? a.total_work : n_sm);
-    tree_attn_tc_kernel<D><<<grid, C::THREADS, C::SMEM, st>>>(tmQ, tmK, tmV, tmKt, tmVt, a, mask, status);
+    const int ctas = n_sm < ATTN_HAND_CTAS ? n_sm : ATTN_HAND_CTAS;  // every CTA has a hand-over area of its own
+    const unsigned grid = (unsigned)(a.total_work < ctas ? a.total_work : ctas);
+    tree_attn_tc_kernel<D, TEAMS><<<grid, C::THREADS, C::SMEM, st>>>(tmQ, tmK, tmV, tmKt, tmVt, a, mask, status);
     SR_LAUNCH_CHECK();
     return SPECROLL_OK;
 }
@@ -977,8 +1196,11 @@ extern "C" int specroll_debug_trace_read(unsigned long long *dst, unsigned int *
 #endif
 
 int launch_attn_tc(const AttnArgs &a, const TopoMask &mask, int D, long long T_kv, int32_t *status, cudaStream_t st) {
-    if (D == 128) return launch_tc<128>(a, mask, T_kv, status, st);
-    return launch_tc<64>(a, mask, T_kv, status, st);
+    // One row block per (sequence, KV head): the kernel is bound by HBM and the softmax with two threads per row
+    // is (slightly) the better one; more blocks: bound by the softmax, where the two alternating teams are faster.
+    const bool teams = a.n_rb > 1;
+    if (D == 128) return teams ? launch_tc<128, true>(a, mask, T_kv, status, st) : launch_tc<128, false>(a, mask, T_kv, status, st);
+    return teams ? launch_tc<64, true>(a, mask, T_kv, status, st) : launch_tc<64, false>(a, mask, T_kv, status, st);
 }
 
 }  // namespace specroll
