@@ -299,7 +299,8 @@ def gather_hidden(hidden, term_node):
 
 
 # ----------------------------------------------------------------------------------- verifier feedback
-def reflex_feedback(logits_rows, W, cand_id, cand_logit, y_star, m, rho, k_support, temperature=1.0, eps=1e-6):
+def reflex_feedback(logits_rows, W, cand_id, cand_logit, y_star, m, rho, k_support, temperature=1.0, eps=1e-6,
+                    severity=False, severity_min=0.03):
     """Verifier-derived feedback of matured proposals and the memory update (Sec. 3.3 / 3.4: Eq. "support",
     "distdir", "covdir", the RMS normalisation, Eq. "unified-feedback", Eq. "ema"; the magnitudes d_dist and
     d_cov from Eq. "acceptance-gap-decomposition").  One record per row, written out step by step in fp64:
@@ -313,6 +314,11 @@ def reflex_feedback(logits_rows, W, cand_id, cand_logit, y_star, m, rho, k_suppo
       d_dist = p(C) TV(p_C, q_C),  d_cov = p(C*) - p(C)
       rbar = r / (RMS(r) + eps);  g = d_dist rbar_dist + d_cov rbar_cov;  e = (d_dist + d_cov) g / (RMS(g) + eps)
       m <- rho m + (1 - rho) e
+
+    With ``severity`` (App. "Implementation details", paragraph "Verifier-derived feedback"): the observation's
+    severity  w = clip(0.3 TV(p_S, q_S) + 0.7 p_out, 0, 1),  p_out = 1 - p(C) the target mass outside the
+    candidates, weights it,  m <- rho m + (1 - rho) w e,  and an observation with w < severity_min is discarded
+    (the memory row keeps its value).  w and TV(p_S, q_S) are returned either way.
 
     logits_rows [R,V] and W [V,d] are bf16 bit patterns; m [R,d], rho [R] floats.  Returns the new memory and the
     intermediate quantities."""
@@ -329,7 +335,8 @@ def reflex_feedback(logits_rows, W, cand_id, cand_logit, y_star, m, rho, k_suppo
         raise ValueError("the support budget must cover the target's top-k (k_support >= k)")
     Wf = (W.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
     out = {"m": np.empty((R, d)), "e": np.empty((R, d)), "d_dist": np.empty(R), "d_cov": np.empty(R),
-           "tv": np.empty(R), "p_C": np.empty(R), "support": []}
+           "tv": np.empty(R), "p_C": np.empty(R), "support": [], "tv_S": np.empty(R), "w": np.empty(R),
+           "kept": np.ones(R, bool)}
     rms = lambda v: np.sqrt(np.mean(v * v))
     for r in range(R):
         l = (logits_rows[r].astype(np.uint32) << 16).view(np.float32).astype(np.float64)
@@ -365,8 +372,76 @@ def reflex_feedback(logits_rows, W, cand_id, cand_logit, y_star, m, rho, k_suppo
         d_cov = sum(p[v] for v in c_star) - pC
         g = d_dist * r_dist / (rms(r_dist) + eps) + d_cov * r_cov / (rms(r_cov) + eps)
         e = (d_dist + d_cov) * g / (rms(g) + eps)
-        out["m"][r] = rho[r] * m[r] + (1.0 - rho[r]) * e
+        tv_S = 0.5 * sum(abs(pS[v] - qS[v]) for v in S)
+        w = min(1.0, max(0.0, 0.3 * tv_S + 0.7 * (1.0 - pC)))
+        out["tv_S"][r], out["w"][r] = tv_S, w
+        if not severity:
+            out["m"][r] = rho[r] * m[r] + (1.0 - rho[r]) * e
+        elif w < severity_min:
+            out["m"][r] = m[r]
+            out["kept"][r] = False
+        else:
+            out["m"][r] = rho[r] * m[r] + (1.0 - rho[r]) * w * e
         out["e"][r] = e
         out["d_dist"][r], out["d_cov"][r], out["tv"][r], out["p_C"][r] = d_dist, d_cov, tv, pC
         out["support"].append(S)
     return out
+
+
+def reflex_sketch(X, Pi):
+    """Normalised random-projection sketch (Sec. 3.4 "Reliability from delayed alignment"; App. "Implementation
+    details": rank 24, seed 29): sketch(x) = Pi x / ||Pi x||_2, the zero vector when Pi x = 0.  X [R,d], Pi [rank,d]
+    (the projection's entries are an input: both sides are given the same matrix)."""
+    X, Pi = np.asarray(X, np.float64), np.asarray(Pi, np.float64)
+    out = np.zeros((X.shape[0], Pi.shape[0]))
+    for r in range(X.shape[0]):
+        y = np.array([float(np.dot(Pi[i], X[r])) for i in range(Pi.shape[0])])
+        nrm = np.sqrt(np.sum(y * y))
+        if nrm > 0.0:
+            out[r] = y / nrm
+    return out
+
+
+def reflex_gate(s, xi, slot, keep, n, mean, M2, n_fb, m, horizon, n_align_min, n_fb_min, alpha_lo, alpha_hi,
+                z_delta=0.60, mem_eps=1e-12):
+    """Reliability score and gate of every (trajectory, horizon) slot (Sec. 3.4 Eq. "reliability-score" and the
+    indicator of Eq. "reflex-correction"; App. "Implementation details": exact online sample moments, minimum
+    counts per horizon, correction interval per horizon).
+
+    Records r = 0..R-1 are taken in order; a kept record of slot j = slot[r] contributes its realised alignment
+    a_r = cos(s_r, xi_r) (0 when either sketch is the zero vector) to the slot's running count, mean and sum of
+    squared deviations (Welford's recurrences, which give the exact sample mean and variance), and counts as one
+    feedback observation.  Then, per slot with horizon h:
+        Rel = mean - z_delta * sqrt(M2 / (n - 1)) / sqrt(n)          (n >= 2; otherwise not eligible)
+        open = n >= n_align_min[h]  and  n_fb >= n_fb_min[h]  and  Rel > 0  and  RMS(m_slot) > mem_eps
+        alpha = alpha_lo[h] + (alpha_hi[h] - alpha_lo[h]) * min(Rel, 1)   if open, else 0
+    (the paper places the ratio in [alpha_lo, alpha_hi] for an eligible score without giving the map; the linear one
+    in the score is this implementation's reading).  Returns a [R] (nan for records not kept) and the updated
+    state, Rel [S] (-inf when n < 2) and alpha [S]."""
+    s, xi = np.asarray(s, np.float64), np.asarray(xi, np.float64)
+    n, n_fb = np.array(n, np.int64), np.array(n_fb, np.int64)
+    mean, M2 = np.array(mean, np.float64), np.array(M2, np.float64)
+    m = np.asarray(m, np.float64)
+    R, S = s.shape[0], n.shape[0]
+    a = np.full(R, np.nan)
+    for r in range(R):
+        if keep is not None and not keep[r]:
+            continue
+        j = int(slot[r])
+        ns, nx = np.sqrt(np.sum(s[r] ** 2)), np.sqrt(np.sum(xi[r] ** 2))
+        a[r] = float(np.dot(s[r], xi[r]) / (ns * nx)) if ns > 0.0 and nx > 0.0 else 0.0
+        n[j] += 1
+        delta = a[r] - mean[j]
+        mean[j] += delta / n[j]
+        M2[j] += delta * (a[r] - mean[j])
+        n_fb[j] += 1
+    rel = np.full(S, -np.inf)
+    alpha = np.zeros(S)
+    for j in range(S):
+        h = int(horizon[j])
+        if n[j] >= 2:
+            rel[j] = mean[j] - z_delta * np.sqrt(M2[j] / (n[j] - 1)) / np.sqrt(n[j])
+        rms = np.sqrt(np.mean(m[j] ** 2))
+        if n[j] >= n_align_min[h] and n_fb[j] >= n_fb_min[h] and rel[j] > 0.0 and rms > mem_eps:
+            alpha[j] = alpha_lo[h] + (alpha_hi[h] - alpha_lo[h]) * min(rel[j], 1.0)
+    return {"a": a, "n": n, "mean": mean, "M2": M2, "n_fb": n_fb, "rel": rel, "alpha": alpha}
