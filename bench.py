@@ -479,6 +479,34 @@ def run_calls(args, w, layers):
 
     fb_bytes = (R * w.V * 2 + R * (w.k + k_support + 1) * w.d * 2 + 2 * R * w.d * 4) / 1e9
     calls["reflex_feedback (B K records, support 48)"] = (feedback, "hbm", fb_bytes, peaks["hbm_gbs"], "GB/s")
+    # reliability side: sketches (rank 24) of the R feedback vectors, then alignments, online moments and the gate
+    # of the R slots (one record per slot here)
+    rank = 24
+    Pi = torch.randn((rank, w.d), generator=gen, device=dev)
+    e_vec = torch.randn((R, w.d), generator=gen, device=dev)
+    s_sk = S.reflex_sketch(mem, Pi)
+    xi_sk = S.reflex_sketch(e_vec, Pi)
+    slot = torch.arange(R, device=dev, dtype=torch.int32)
+    st_n = torch.zeros(R, dtype=torch.int32, device=dev)
+    st_fb = torch.zeros(R, dtype=torch.int32, device=dev)
+    st_mean = torch.zeros(R, device=dev)
+    st_M2 = torch.zeros(R, device=dev)
+    hz = (torch.arange(R, device=dev) % w.K).to(torch.int32)
+    n_al = torch.tensor([6, 16, 48, 48, 48][: w.K], dtype=torch.int32, device=dev)
+    n_fbm = torch.tensor([1, 2, 4, 4, 4][: w.K], dtype=torch.int32, device=dev)
+    a_lo = torch.tensor([0.010, 0.004, 0.0025, 0.0025, 0.0025][: w.K], device=dev)
+    a_hi = torch.tensor([0.025, 0.010, 0.0060, 0.0060, 0.0060][: w.K], device=dev)
+
+    def sketch():
+        S.reflex_sketch(e_vec, Pi)
+
+    def gate():
+        S.reflex_gate(s_sk, xi_sk, slot, None, st_n, st_mean, st_M2, st_fb, mem, hz, n_al, n_fbm, a_lo, a_hi)
+
+    calls["reflex_sketch (B K vectors, rank 24)"] = (sketch, "hbm", (R * w.d * 4 + rank * w.d * 4 + R * rank * 4) / 1e9,
+                                                     peaks["hbm_gbs"], "GB/s")
+    calls["reflex_gate (B K records, B K slots)"] = (gate, "hbm", (R * w.d * 4 + 2 * R * rank * 4 + 8 * R * 4) / 1e9,
+                                                    peaks["hbm_gbs"], "GB/s")
     out = {"workload": w.name, "peak_source": peaks["source"], "calls": {}}
     for name, (fn, bound, work, peak, unit) in calls.items():
         rec = {"bound": bound, "unit": unit, "peak": peak, "work_per_call": work}

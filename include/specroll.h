@@ -232,14 +232,22 @@ int specroll_gather_hidden(int32_t B, int32_t N, int32_t d, const void *hidden,
  * Shapes (device): logits[rows, V] bf16 with row_max, row_sum[rows] fp32 as specroll_verify wrote them;
  * rec_row, rec_mem, y_star[R] i32; cand_id[R,k] i32; cand_logit[R,k] fp32; W[V,d] bf16; rho[R] fp32;
  * m[mem_rows, d] fp32 in/out; d_dist, d_cov, tv[R] fp32 outputs, each nullable.
- * What the paper builds on top (severity, discarding, sketches, reliability score, the choice of alpha) is
- * left to the caller: it needs only these outputs. */
+ * Severity weighting and discarding: the flag below.  Sketches, reliability score and gate: specroll_reflex_sketch
+ * and specroll_reflex_gate. */
 typedef struct {
     int32_t R, k, k_support, d, V;
     float temperature;
     float eps;     /* RMS stabiliser (> = 0) */
-    int32_t flags; /* reserved, must be 0 */
+    int32_t flags; /* 0, or SPECROLL_FEEDBACK_SEVERITY */
+    float severity_min; /* with SPECROLL_FEEDBACK_SEVERITY: observations with w below it are discarded (paper: 0.03) */
 } specroll_feedback_desc;
+
+/* The observation's severity weights the update and small ones are discarded (App. "Implementation details",
+ * paragraph "Verifier-derived feedback"):  w = clip(0.3 TV(p_S, q_S) + 0.7 p_out, 0, 1)  with  p_out = 1 - p(C)
+ * the target mass outside the candidates;  m <- rho m + (1 - rho) w e  when  w >= severity_min, else the memory
+ * row is left as it is.  (How w enters the update is not printed in the paper; weighting the observation is
+ * this implementation's reading.) */
+#define SPECROLL_FEEDBACK_SEVERITY 1
 
 size_t specroll_reflex_feedback_workspace_bytes(const specroll_feedback_desc *desc);
 
@@ -249,6 +257,56 @@ int specroll_reflex_feedback(const specroll_feedback_desc *desc, const void *log
                              const void *W, const float *rho, const int32_t *rec_mem, float *m,
                              float *d_dist, float *d_cov, float *tv, void *workspace,
                              size_t workspace_bytes, void *cuda_stream);
+
+/* The same with two more outputs (device, each nullable): severity[R] fp32, the w above (written whether or
+ * not the flag is set), and e_out[R, d] fp32, the feedback vector e of every record (also of discarded ones),
+ * which specroll_reflex_sketch turns into the record's verifier-feedback sketch. */
+int specroll_reflex_feedback_ex(const specroll_feedback_desc *desc, const void *logits,
+                                const int32_t *rec_row, const float *row_max, const float *row_sum,
+                                const int32_t *cand_id, const float *cand_logit, const int32_t *y_star,
+                                const void *W, const float *rho, const int32_t *rec_mem, float *m,
+                                float *d_dist, float *d_cov, float *tv, float *severity, float *e_out,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Reliability from delayed alignment and the gate of the correction (Sec. 3.4, paragraphs "Reliability from
+ * delayed alignment" and "Gated hidden-state correction", Eq. "reliability-score" and the indicator of Eq.
+ * "reflex-correction"; App. "Implementation details", paragraph "Reflex configuration").
+ *
+ * specroll_reflex_sketch: normalised random-projection sketch of R vectors,
+ *   sketch[r, :] = Pi x_r / ||Pi x_r||_2   (the zero vector when Pi x_r = 0),  x_r = X[rows[r], :] (rows nullable:
+ *   then x_r = X[r, :]).  X[*, d] fp32, Pi[rank, d] fp32 (rank <= 32; the paper uses rank 24 and draws Pi with
+ *   seed 29; the matrix is an input here), sketch[R, rank] fp32.  Used at proposal time on the memory rows
+ *   (s_j) and at maturity on the feedback vectors (xi_j).
+ *
+ * specroll_reflex_gate: takes R matured records in order.  A kept record (keep nullable = all kept; else
+ * keep[r] != 0, e.g. severity >= severity_min) of slot j = slot[r] contributes its realised alignment
+ * a_r = cos(s_r, xi_r) (0 when either sketch is zero) to the slot's count n, mean and sum of squared
+ * deviations M2 (Welford's recurrences: the exact online sample moments) and to its feedback count n_fb.
+ * Then for every slot j (a trajectory-horizon pair) with horizon h = horizon[j]:
+ *   Rel = mean - z_delta sqrt(M2 / (n - 1)) / sqrt(n)      (n >= 2, else -inf)
+ *   open = n >= n_align_min[h] && n_fb >= n_fb_min[h] && Rel > 0 && RMS(m[j, :]) > mem_eps
+ *   alpha[j] = open ? alpha_lo[h] + (alpha_hi[h] - alpha_lo[h]) min(Rel, 1) : 0
+ * alpha is what specroll_propose takes per (sequence, head).  The paper puts the ratio of an eligible score
+ * inside [alpha_lo, alpha_hi] without printing the map; linear in the score is this implementation's reading.
+ * Shapes (device): s, xi[R, rank] fp32; slot[R] i32 in [0, S); keep[R] u8 nullable; n, n_fb[S] i32 in/out;
+ * mean, M2[S] fp32 in/out; m[S, d] fp32; horizon[S] i32 in [0, H); n_align_min, n_fb_min[H] i32; alpha_lo,
+ * alpha_hi[H] fp32; outputs a[R] (nullable; NaN for records not kept), rel[S], alpha[S] fp32. */
+typedef struct {
+    int32_t R, S, d, rank, H;
+    float z_delta; /* paper: 0.60 */
+    float mem_eps; /* a memory row with RMS at or below this is "negligible" */
+    int32_t flags; /* reserved, must be 0 */
+} specroll_gate_desc;
+
+int specroll_reflex_sketch(int32_t R, int32_t d, int32_t rank, const float *X, const int32_t *rows,
+                           const float *Pi, float *sketch, void *cuda_stream);
+
+int specroll_reflex_gate(const specroll_gate_desc *desc, const float *s, const float *xi,
+                         const int32_t *slot, const uint8_t *keep, int32_t *n, float *mean, float *M2,
+                         int32_t *n_fb, const float *m, const int32_t *horizon,
+                         const int32_t *n_align_min, const int32_t *n_fb_min, const float *alpha_lo,
+                         const float *alpha_hi, float *a, float *rel, float *alpha, void *cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
  * Exact target verification (App. B.2 Eq. "nodeaccept" / "noderesidual", Algorithm "Exact

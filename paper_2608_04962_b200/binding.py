@@ -26,13 +26,15 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
            "specroll_commit_path", "specroll_commit_path_layers", "specroll_gather_hidden",
            "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static",
            "specroll_verify_nucleus_workspace_bytes", "specroll_verify_nucleus",
-           "specroll_reflex_feedback_workspace_bytes", "specroll_reflex_feedback")
+           "specroll_reflex_feedback_workspace_bytes", "specroll_reflex_feedback", "specroll_reflex_feedback_ex",
+           "specroll_reflex_sketch", "specroll_reflex_gate")
 
 
 PROPOSE_LEGACY_MMA = 1
 ATTN_LEGACY_MMA = 1
 ATTN_REUSE_PLAN = 2
 VERIFY_LAZY_STATS = 1
+FEEDBACK_SEVERITY = 1
 PAGE_TOKENS = 128
 
 
@@ -59,7 +61,12 @@ class VerifyDesc(C.Structure):
 
 class FeedbackDesc(C.Structure):
     _fields_ = [("R", C.c_int32), ("k", C.c_int32), ("k_support", C.c_int32), ("d", C.c_int32), ("V", C.c_int32),
-                ("temperature", C.c_float), ("eps", C.c_float), ("flags", C.c_int32)]
+                ("temperature", C.c_float), ("eps", C.c_float), ("flags", C.c_int32), ("severity_min", C.c_float)]
+
+
+class GateDesc(C.Structure):
+    _fields_ = [("R", C.c_int32), ("S", C.c_int32), ("d", C.c_int32), ("rank", C.c_int32), ("H", C.c_int32),
+                ("z_delta", C.c_float), ("mem_eps", C.c_float), ("flags", C.c_int32)]
 
 
 def lib():
@@ -446,29 +453,73 @@ def verify_nucleus(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_a
 
 
 def reflex_feedback(logits, rec_row, row_max, row_sum, cand_id, cand_logit, y_star, W, rho, rec_mem, m, k_support,
-                    temperature=1.0, eps=1e-6, workspace=None):
-    """specroll_reflex_feedback: verifier feedback of R matured records, memory ``m`` updated in place.
-    logits [rows, V] bf16 (any leading shape), row_max/row_sum [rows]; returns d_dist, d_cov, tv [R]."""
+                    temperature=1.0, eps=1e-6, workspace=None, severity_min=None, want_e=False):
+    """specroll_reflex_feedback(_ex): verifier feedback of R matured records, memory ``m`` updated in place.
+    logits [rows, V] bf16 (any leading shape), row_max/row_sum [rows]; returns d_dist, d_cov, tv, severity [R]
+    (and e [R, d] with ``want_e``).  With ``severity_min`` the update is weighted by the severity and
+    observations below it are discarded."""
     V = logits.shape[-1]
     R, k = cand_id.shape
     d = W.shape[1]
-    desc = FeedbackDesc(R, k, k_support, d, V, temperature, eps, 0)
+    weighted = severity_min is not None
+    desc = FeedbackDesc(R, k, k_support, d, V, temperature, eps, FEEDBACK_SEVERITY if weighted else 0,
+                        float(severity_min) if weighted else 0.0)
     dev = logits.device
     f32, i32 = torch.float32, torch.int32
-    out = {n: torch.empty(R, dtype=f32, device=dev) for n in ("d_dist", "d_cov", "tv")}
+    out = {n: torch.empty(R, dtype=f32, device=dev) for n in ("d_dist", "d_cov", "tv", "severity")}
+    if want_e:
+        out["e"] = torch.empty((R, d), dtype=f32, device=dev)
     need = lib().specroll_reflex_feedback_workspace_bytes(C.byref(desc))
     if need == 0:
         raise SpecrollError("reflex_feedback: invalid descriptor")
     if workspace is None:
         workspace = _workspace(need, dev)
-    rc = lib().specroll_reflex_feedback(
+    rc = lib().specroll_reflex_feedback_ex(
         C.byref(desc), _dev(logits, torch.bfloat16, "logits"), _dev(rec_row, i32, "rec_row"),
         _dev(row_max, f32, "row_max"), _dev(row_sum, f32, "row_sum"), _dev(cand_id, i32, "cand_id"),
         _dev(cand_logit, f32, "cand_logit"), _dev(y_star, i32, "y_star"), _dev(W, torch.bfloat16, "W"),
         _dev(rho, f32, "rho"), _dev(rec_mem, i32, "rec_mem"), _dev(m, f32, "m"), _dev(out["d_dist"], f32, "d_dist"),
-        _dev(out["d_cov"], f32, "d_cov"), _dev(out["tv"], f32, "tv"), C.c_void_p(workspace.data_ptr()),
+        _dev(out["d_cov"], f32, "d_cov"), _dev(out["tv"], f32, "tv"), _dev(out["severity"], f32, "severity"),
+        _dev(out["e"], f32, "e") if want_e else None, C.c_void_p(workspace.data_ptr()),
         C.c_size_t(workspace.numel()), _stream())
-    _check(rc, "specroll_reflex_feedback")
+    _check(rc, "specroll_reflex_feedback_ex")
+    return out
+
+
+def reflex_sketch(X, Pi, rows=None):
+    """specroll_reflex_sketch: normalised random-projection sketches [R, rank] of the rows of X [*, d] fp32
+    (``rows`` [R] i32 selects them; all rows in order when None) under the projection Pi [rank, d] fp32."""
+    rank, d = Pi.shape
+    R = X.shape[0] if rows is None else rows.shape[0]
+    out = torch.empty((R, rank), dtype=torch.float32, device=X.device)
+    rc = lib().specroll_reflex_sketch(C.c_int32(R), C.c_int32(d), C.c_int32(rank), _dev(X, torch.float32, "X"),
+                                      _dev(rows, torch.int32, "rows") if rows is not None else None,
+                                      _dev(Pi, torch.float32, "Pi"), _dev(out, torch.float32, "sketch"), _stream())
+    _check(rc, "specroll_reflex_sketch")
+    return out
+
+
+def reflex_gate(s, xi, slot, keep, n, mean, M2, n_fb, m, horizon, n_align_min, n_fb_min, alpha_lo, alpha_hi,
+                z_delta=0.60, mem_eps=1e-12):
+    """specroll_reflex_gate: alignments of R matured records into the slots' online moments (n, mean, M2, n_fb
+    updated in place), then the reliability score and the correction ratio of every slot.  Returns a [R],
+    rel [S], alpha [S]."""
+    R, rank = s.shape
+    S, d = m.shape
+    H = n_align_min.shape[0]
+    dev = m.device
+    f32, i32 = torch.float32, torch.int32
+    desc = GateDesc(R, S, d, rank, H, z_delta, mem_eps, 0)
+    out = {"a": torch.empty(max(R, 1), dtype=f32, device=dev)[:R], "rel": torch.empty(S, dtype=f32, device=dev),
+           "alpha": torch.empty(S, dtype=f32, device=dev)}
+    rc = lib().specroll_reflex_gate(
+        C.byref(desc), _dev(s, f32, "s"), _dev(xi, f32, "xi"), _dev(slot, i32, "slot"),
+        _dev(keep, torch.uint8, "keep") if keep is not None else None, _dev(n, i32, "n"), _dev(mean, f32, "mean"),
+        _dev(M2, f32, "M2"), _dev(n_fb, i32, "n_fb"), _dev(m, f32, "m"), _dev(horizon, i32, "horizon"),
+        _dev(n_align_min, i32, "n_align_min"), _dev(n_fb_min, i32, "n_fb_min"), _dev(alpha_lo, f32, "alpha_lo"),
+        _dev(alpha_hi, f32, "alpha_hi"), _dev(out["a"], f32, "a"), _dev(out["rel"], f32, "rel"),
+        _dev(out["alpha"], f32, "alpha"), _stream())
+    _check(rc, "specroll_reflex_gate")
     return out
 
 

@@ -208,8 +208,11 @@ struct FeedbackArgs {
     const int32_t *top_id;
     float *m;
     float *d_dist, *d_cov, *tv;
+    float *severity, *e_out;  // optional outputs: w per record, the feedback vector e per record
     int R, k, kS, d, V;
     float inv_T, eps;
+    int weighted;        // the update is weighted by the severity, records below severity_min are discarded
+    float severity_min;
 };
 
 // MAXC = columns of the hidden dimension per thread (d <= 256 * MAXC)
@@ -222,7 +225,7 @@ __global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a
     __shared__ float s_acov[MAX_S];   // coefficient of W_v in r_cov
     __shared__ float s_q[SPECROLL_MAX_TOPK];
     __shared__ int s_n;
-    __shared__ float s_dd, s_dc;
+    __shared__ float s_dd, s_dc, s_w;
     __shared__ float red[FB_THREADS / 32];
     const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int k = a.k, kS = a.kS, d = a.d;
@@ -314,8 +317,18 @@ __global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a
         pCs = warp_sum(pCs);
         cov_b = warp_sum(cov_b);
         __syncwarp();
-        for (int i = lane; i < n; i += 32) s_adist[i] = s_p[i] / pS - (i < k ? s_q[i] : 0.f);
+        float tvS = 0.f;  // TV(p_S, q_S)
+        for (int i = lane; i < n; i += 32) {
+            const float ad = s_p[i] / pS - (i < k ? s_q[i] : 0.f);
+            s_adist[i] = ad;
+            tvS += fabsf(ad);
+        }
+        tvS = 0.5f * warp_sum(tvS);
         if (lane == 0) {
+            // severity of the observation: w = clip(0.3 TV(p_S, q_S) + 0.7 p_out, 0, 1), p_out = 1 - p(C)
+            const float w = fminf(1.f, fmaxf(0.f, 0.3f * tvS + 0.7f * (1.f - pC)));
+            s_w = w;
+            if (a.severity) a.severity[r] = w;
             s_acov[k - 1] -= cov_b;  // b* = last candidate (the list is sorted by logit)
             const float dd = pC * tvs, dc = pCs - pC;
             s_dd = dd;
@@ -364,11 +377,19 @@ __global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a
     sg = block_sum_f<FB_THREADS>(sg, red);
     const float fe = (dd + dc) / (sqrtf(sg / d) + a.eps);
     const float rho = a.rho[r];
+    const float w = s_w;
+    const bool keep = !a.weighted || w >= a.severity_min;
+    const float gain = (1.f - rho) * (a.weighted ? w : 1.f);
     float *mr = a.m + (size_t)a.rec_mem[r] * d;
+    float *er = a.e_out ? a.e_out + (size_t)r * d : nullptr;
 #pragma unroll
     for (int c = 0; c < MAXC; ++c) {
         const int col = tid + c * FB_THREADS;
-        if (c < ncol && col < d) mr[col] = rho * mr[col] + (1.f - rho) * fe * rd[c];
+        if (c < ncol && col < d) {
+            const float e = fe * rd[c];
+            if (er) er[col] = e;
+            if (keep) mr[col] = rho * mr[col] + gain * e;
+        }
     }
 }
 
@@ -379,7 +400,8 @@ using namespace specroll;
 static int check_feedback_desc(const specroll_feedback_desc *d) {
     if (!d || d->R < 0 || d->k < 1 || d->k > SPECROLL_MAX_TOPK || d->k_support < d->k ||
         d->k_support > SPECROLL_MAX_TOPK || d->d < 8 || d->d > 12288 || d->V < 8 || (d->V % 8) || d->k_support > d->V ||
-        !(d->temperature > 0.f) || !(d->eps >= 0.f) || d->flags != 0)
+        !(d->temperature > 0.f) || !(d->eps >= 0.f) || (d->flags & ~SPECROLL_FEEDBACK_SEVERITY) != 0 ||
+        ((d->flags & SPECROLL_FEEDBACK_SEVERITY) && !(d->severity_min >= 0.f)))
         return SPECROLL_EINVAL;
     return SPECROLL_OK;
 }
@@ -395,6 +417,16 @@ extern "C" int specroll_reflex_feedback(const specroll_feedback_desc *d, const v
                                         const float *rho, const int32_t *rec_mem, float *m, float *d_dist,
                                         float *d_cov, float *tv, void *workspace, size_t workspace_bytes,
                                         void *cuda_stream) {
+    return specroll_reflex_feedback_ex(d, logits, rec_row, row_max, row_sum, cand_id, cand_logit, y_star, W, rho, rec_mem,
+                                       m, d_dist, d_cov, tv, nullptr, nullptr, workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" int specroll_reflex_feedback_ex(const specroll_feedback_desc *d, const void *logits, const int32_t *rec_row,
+                                           const float *row_max, const float *row_sum, const int32_t *cand_id,
+                                           const float *cand_logit, const int32_t *y_star, const void *W,
+                                           const float *rho, const int32_t *rec_mem, float *m, float *d_dist,
+                                           float *d_cov, float *tv, float *severity, float *e_out, void *workspace,
+                                           size_t workspace_bytes, void *cuda_stream) {
     if (check_feedback_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (!logits || !rec_row || !row_max || !row_sum || !cand_id || !cand_logit || !y_star || !W || !rho || !rec_mem || !m)
         return SPECROLL_EINVAL;
@@ -424,6 +456,10 @@ extern "C" int specroll_reflex_feedback(const specroll_feedback_desc *d, const v
     a.d_dist = d_dist;
     a.d_cov = d_cov;
     a.tv = tv;
+    a.severity = severity;
+    a.e_out = e_out;
+    a.weighted = (d->flags & SPECROLL_FEEDBACK_SEVERITY) ? 1 : 0;
+    a.severity_min = d->severity_min;
     a.R = d->R;
     a.k = d->k;
     a.kS = d->k_support;
