@@ -553,6 +553,9 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="capture the step in a CUDA graph and time replays instead of plain launches (the phase "
                          "times and the roofline line then come from plain steps run afterwards)")
+    ap.add_argument("--chw", action="store_true",
+                    help="profile the verification capacity C_hw of Eq. verification-budget for the workload's shape "
+                         "(sweeps batch size and nodes per sequence; prints one JSON object)")
     ap.add_argument("--calls", action="store_true",
                     help="time each entry point alone (100 launches, cold and warm L2) instead of the step")
     args = ap.parse_args()
@@ -563,6 +566,18 @@ def main():
         return run_reference(args, w, layers)
     if args.calls:
         return run_calls(args, w, layers)
+    if args.chw:
+        import torch
+        from paper_2608_04962_b200 import binding as S
+        from paper_2608_04962_b200 import chw
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback of the hot path")
+        torch.cuda.set_device(0)
+        res = chw.profile(w, Bs=(256, 128, 64, 32, 16), Ns=(4, 8, 12, 16, 24, 32, 48, 64),
+                          device=torch.device("cuda", 0), warmup=args.warmup, steps=max(2, min(args.steps, 5)))
+        res["node_budget"] = {str(B): S.node_budget(res["C_hw"], B, 4, 64) for B in (256, 128, 64, 32, 16, 8)}
+        print(json.dumps(res), flush=True)
+        return 0
     return run_ours(args, w, layers)
 
 
