@@ -122,6 +122,27 @@ __device__ __forceinline__ bool group_sync(uint32_t bar, uint32_t &uses, volatil
     return ok;
 }
 
+// Two fp32 operations in one instruction (packed pairs in 64-bit registers): the softmax phase follows its
+// instruction count, and the scale-and-shift before the exponential and the running sums are pairwise anyway.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 __device__ __forceinline__ unsigned short bf16_bits_rn(float x) {
     return __bfloat16_as_ushort(__float2bfloat16_rn(x));
 }
@@ -675,16 +696,20 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     float ls0 = 0.f, ls1 = 0.f;
                     auto exp_group = [&](const uint32_t(&src)[32], uint32_t bc, float mref_, uint32_t *pk) {
                         if (full) {
-    #pragma unroll
+                            const uint64_t sc2 = pack_f32x2(sc, sc), nm2 = pack_f32x2(-mref_, -mref_);
+                            uint64_t ls2 = pack_f32x2(ls0, ls1);
+#pragma unroll
                             for (int i2 = 0; i2 < 32; i2 += 2) {
-                                const float p0 = ex2_approx(fmaf(__uint_as_float(src[i2]), sc, -mref_));
-                                const float p1 = ex2_approx(fmaf(__uint_as_float(src[i2 + 1]), sc, -mref_));
-                                ls0 += p0;
-                                ls1 += p1;
+                                float t0, t1;
+                                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(src[i2]), __uint_as_float(src[i2 + 1])), sc2, nm2),
+                                             t0, t1);
+                                const float p0 = ex2_approx(t0), p1 = ex2_approx(t1);
+                                ls2 = add_f32x2(ls2, pack_f32x2(p0, p1));
                                 pk[i2 >> 1] = pack_bf16x2(p0, p1);
                             }
+                            unpack_f32x2(ls2, ls0, ls1);
                         } else {
-    #pragma unroll
+#pragma unroll
                             for (int i2 = 0; i2 < 32; i2 += 2) {
                                 const bool b0 = (bc >> i2) & 1u, b1 = (bc >> (i2 + 1)) & 1u;
                                 const float p0 = b0 ? ex2_approx(fmaf(__uint_as_float(src[i2]), sc, -mref_)) : 0.f;
@@ -712,7 +737,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         // ---- one pass against the reference as it stands; P stays in registers until the verdict
                         uint32_t pk[64];
                         const float mref_ = (m_used == -INFINITY) ? 0.f : m_used;
-    #pragma unroll
+#pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             tmem_ld32(s_t + 32u * (uint32_t)c, x);
                             tmem_ld_wait();
@@ -722,10 +747,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         if (!ok) break;
                         const bool bad = !(ls0 + ls1 <= 256.0f) || m_pub != m_used;
                         if (!__any_sync(0xffffffffu, bad)) {
-    #pragma unroll
+#pragma unroll
                             for (int c = 0; c < 4; ++c) {
                                 uint32_t q[16];
-    #pragma unroll
+#pragma unroll
                                 for (int i2 = 0; i2 < 16; ++i2) q[i2] = pk[16 * c + i2];
                                 tmem_st16(s_t + 16u * (uint32_t)c, q);
                             }
@@ -740,19 +765,19 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         // ---- two passes.  First the row's maximum over the tile ...
                         ls0 = ls1 = 0.f;
                         float mx0 = -INFINITY, mx1 = -INFINITY;
-    #pragma unroll
+#pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             tmem_ld32(s_t + 32u * (uint32_t)c, x);
                             tmem_ld_wait();
                             const uint32_t bc = bits_of(c);
                             if (full) {
-    #pragma unroll
+#pragma unroll
                                 for (int i2 = 0; i2 < 32; i2 += 2) {
                                     mx0 = fmaxf(mx0, __uint_as_float(x[i2]));
                                     mx1 = fmaxf(mx1, __uint_as_float(x[i2 + 1]));
                                 }
                             } else {
-    #pragma unroll
+#pragma unroll
                                 for (int i2 = 0; i2 < 32; ++i2)
                                     if ((bc >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(x[i2]));
                             }
@@ -782,11 +807,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                             ok = __all_sync(0xffffffffu, ok);
                             if (!ok) break;
                             tc_fence_after();
-    #pragma unroll 1
+#pragma unroll 1
                             for (int c = 0; c < D; c += 32) {
                                 tmem_ld32(o_t + (uint32_t)c, x);
                                 tmem_ld_wait();
-    #pragma unroll
+#pragma unroll
                                 for (int i2 = 0; i2 < 32; ++i2) x[i2] = __float_as_uint(__uint_as_float(x[i2]) * alpha);
                                 tmem_st32(o_t + (uint32_t)c, x);
                             }
@@ -795,7 +820,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         // ... then p = 2^(s*scale - m) as packed bf16 pairs, group by group; 16 packed columns go over S
                         // columns that have been read already
                         const float mref_ = (m_used == -INFINITY) ? 0.f : m_used;
-    #pragma unroll
+#pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             uint32_t q[16];
                             tmem_ld32(s_t + 32u * (uint32_t)c, x);
@@ -878,13 +903,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     float mx0 = -INFINITY, mx1 = -INFINITY;
                     auto max_group = [&](const uint32_t(&src)[32], uint32_t bc) {
                         if (full) {
-    #pragma unroll
+#pragma unroll
                             for (int i2 = 0; i2 < 32; i2 += 2) {
                                 mx0 = fmaxf(mx0, __uint_as_float(src[i2]));
                                 mx1 = fmaxf(mx1, __uint_as_float(src[i2 + 1]));
                             }
                         } else {
-    #pragma unroll
+#pragma unroll
                             for (int i2 = 0; i2 < 32; ++i2)
                                 if ((bc >> i2) & 1u) mx0 = fmaxf(mx0, __uint_as_float(src[i2]));
                         }
@@ -896,13 +921,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         const unsigned short mine = bf16_bits_rn(fmaxf(mx0, mx1));
                         const int px = (int)(use_pair & 1u) * 64;
                         xm[px + half * 32 + lane] = mine;
-    #ifdef SPECROLL_TRACE
+#ifdef SPECROLL_TRACE
                         const long long tps_ = clock64();
-    #endif
+#endif
                         bool k_ = group_sync(pair_bar, use_pair, abort_flag);
-    #ifdef SPECROLL_TRACE
+#ifdef SPECROLL_TRACE
                         prof[4] += (unsigned long long)(clock64() - tps_);
-    #endif
+#endif
                         k_ = __all_sync(0xffffffffu, k_);
                         mt = fmaxf(bf16_bits_to_float(mine), bf16_bits_to_float(xm[px + (half ^ 1) * 32 + lane])) * sc;
                         return k_;
@@ -913,21 +938,24 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     float ls0 = 0.f, ls1 = 0.f;
                     auto exp_group = [&](const uint32_t(&src)[32], uint32_t bc, float mref, bool with_max, uint32_t(&pk)[16]) {
                         if (full) {
-    #pragma unroll
+                            const uint64_t sc2 = pack_f32x2(sc, sc), nm2 = pack_f32x2(-mref, -mref);
+                            uint64_t ls2 = pack_f32x2(ls0, ls1);
+#pragma unroll
                             for (int i2 = 0; i2 < 32; i2 += 2) {
                                 const float s0 = __uint_as_float(src[i2]), s1 = __uint_as_float(src[i2 + 1]);
                                 if (with_max) {
                                     mx0 = fmaxf(mx0, s0);
                                     mx1 = fmaxf(mx1, s1);
                                 }
-                                const float p0 = ex2_approx(fmaf(s0, sc, -mref));
-                                const float p1 = ex2_approx(fmaf(s1, sc, -mref));
-                                ls0 += p0;
-                                ls1 += p1;
+                                float t0, t1;
+                                unpack_f32x2(fma_f32x2(pack_f32x2(s0, s1), sc2, nm2), t0, t1);
+                                const float p0 = ex2_approx(t0), p1 = ex2_approx(t1);
+                                ls2 = add_f32x2(ls2, pack_f32x2(p0, p1));
                                 pk[i2 >> 1] = pack_bf16x2(p0, p1);
                             }
+                            unpack_f32x2(ls2, ls0, ls1);
                         } else {
-    #pragma unroll
+#pragma unroll
                             for (int i2 = 0; i2 < 32; i2 += 2) {
                                 const float s0 = __uint_as_float(src[i2]), s1 = __uint_as_float(src[i2 + 1]);
                                 const bool b0 = (bc >> i2) & 1u, b1 = (bc >> (i2 + 1)) & 1u;
@@ -1000,12 +1028,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                             ok = __all_sync(0xffffffffu, ok);
                             if (!ok) break;
                             tc_fence_after();
-    #pragma unroll 1
+#pragma unroll 1
                             for (int c = 0; c < DH; c += 32) {
                                 uint32_t o[32];
                                 tmem_ld32(o_t + (uint32_t)c, o);
                                 tmem_ld_wait();
-    #pragma unroll
+#pragma unroll
                                 for (int i2 = 0; i2 < 32; ++i2) o[i2] = __float_as_uint(__uint_as_float(o[i2]) * alpha);
                                 tmem_st32(o_t + (uint32_t)c, o);
                             }
