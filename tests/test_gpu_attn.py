@@ -105,6 +105,34 @@ def test_reduced_batches_of_the_large_configs():
         check(o, O, lse)
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,N", [(12, 2, 128, 16), (28, 4, 128, 32), (14, 2, 64, 37)])
+def test_scores_that_keep_growing_along_the_cache(Hq, Hkv, D, N):
+    # Keys whose magnitude grows 30-fold along the sequence: the row maxima keep rising from tile to tile by far
+    # more than the 2^8 the kernel tolerates before it moves a row's reference, so the alarm, the second pass, the
+    # rescaling of the accumulator and (with several row blocks) the hand-over of the reference between the two
+    # softmax teams all run many times per sequence; the chunks of the split sequences meet very different maxima.
+    w = I.scaled(I.WORKLOADS["qwen7b"], B=4, N=N, K=5, Hq=Hq, Hkv=Hkv, D=D, kv_a=300, kv_b=900)
+    x = dict(I.attn_inputs(w))
+    lengths = np.asarray([2300, 640, 131, 1500], np.int32)
+    ip = np.zeros(w.B + 1, np.int32)
+    np.cumsum(lengths, out=ip[1:])
+    g = I.rng(777)
+    Kc = g.standard_normal((int(ip[-1]), w.Hkv, w.D), dtype=np.float32)
+    for b in range(w.B):
+        ramp = 1.0 + 30.0 * np.arange(lengths[b], dtype=np.float32) / lengths[b]
+        Kc[ip[b]:ip[b + 1]] *= ramp[:, None, None]
+    x["kv_indptr"] = ip
+    x["Kc"] = I.f32_to_bf16_bits(Kc)
+    x["Vc"] = I.f32_to_bf16_bits(g.standard_normal((int(ip[-1]), w.Hkv, w.D), dtype=np.float32))
+    o = ref.tree_attn(x["Q"], x["Kc"], x["Vc"], x["kv_indptr"], x["Kt"], x["Vt"], x["parent"], want_lse=True)
+    O, lse = S.tree_attn(dev_bf16(x["Q"]), dev_bf16(x["Kc"]), dev_bf16(x["Vc"]), dev(x["kv_indptr"]), x["kv_indptr"],
+                         dev_bf16(x["Kt"]), dev_bf16(x["Vt"]), x["parent"], want_lse=True, flags=FLAGS["v"],
+                         check_status=True)
+    torch.cuda.synchronize()
+    # sharply peaked rows have |O| of a few units (one value row dominates): the bound scales with max(1, |O|)
+    check(o, host(O.float()).astype(np.float64), host(lse).astype(np.float64), edge=True)
+
+
 def test_scale_argument_and_topology_errors():
     w = I.scaled(I.WORKLOADS["tiny"], B=2)
     x = I.attn_inputs(w)
