@@ -11,10 +11,12 @@
 //   m <- rho m + (1 - rho) e
 //
 // Two kernels, one CTA per record each:
-//   feedback_topk_kernel   exact Top_kS of the record's logits row, ordered by (logit desc, id asc): a radix
-//                          search over the 16-bit order-preserving keys of the bf16 logits by COUNT (four bits per
-//                          pass) finds the key of the kS-th largest value; a pass collects the ids above it, an
-//                          ordered pass the first ids that tie with it; a rank sort orders the kS winners.
+//   feedback_topk_kernel   exact Top_kS of the record's logits row, ordered by (logit desc, id asc), on the 16-bit
+//                          order-preserving keys of the bf16 logits.  Two passes: a lower bound of the kS-th largest
+//                          key from the threads' own maxima, then the few elements at or above it ranked in shared
+//                          memory.  Fallback for rows with thousands of equal large values: a radix search by
+//                          COUNT (four bits per pass) for the key of the kS-th largest value, a pass for the ids
+//                          above it, an ordered pass for the first ids that tie with it, a rank sort.
 //   feedback_kernel        the small quantities (q, p on S, the coefficient of every support row) by one warp,
 //                          then all threads gather the <= k + kS + 1 rows of W once and accumulate both
 //                          directions, three RMS reductions, and the memory update.
@@ -26,6 +28,7 @@ namespace specroll {
 
 namespace fb {
 constexpr int TOPK_THREADS = 512;
+constexpr int TOPK_LIST_CAP = 2048;  // candidates of the list method
 constexpr int FB_THREADS = 256;
 constexpr int MAX_S = 2 * SPECROLL_MAX_TOPK + 1;  // candidates + Top_kS + y*
 
@@ -60,27 +63,31 @@ __device__ __forceinline__ float block_sum_f(float v, float *red) {
 }
 }  // namespace fb
 
-// top_id[r, 0..kS): ids of the kS largest logits of row rec_row[r], by (logit desc, id asc).
-__global__ void __launch_bounds__(fb::TOPK_THREADS)
-feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restrict__ rec_row, int V, int kS,
-                     int32_t *__restrict__ top_id) {
+// Shared memory of the top-k kernel: the list method and the radix fallback never run at the same time.
+struct TopkRadixSmem {
+    int bins[16][fb::TOPK_THREADS];
+    int wsum[fb::TOPK_THREADS / 32][16];
+    int red[fb::TOPK_THREADS / 32];
+    int sel_id[SPECROLL_MAX_TOPK];
+    uint32_t sel_key[SPECROLL_MAX_TOPK];
+};
+struct TopkListSmem {
+    uint32_t best[fb::TOPK_THREADS];     // every thread's largest key
+    uint32_t key[fb::TOPK_LIST_CAP];     // candidates: elements at or above the bound
+    int id[fb::TOPK_LIST_CAP];
+};
+
+// Exact Top_kS by a radix search over the counts (any row, also one with tens of thousands of equal values);
+// the fallback of the list method below.  top_id[0..kS): ids by (logit desc, id asc).
+__device__ void topk_radix(TopkRadixSmem &sm, int &sh_above, int &sh_prefix, int &sh_n, const uint4 *__restrict__ p,
+                           int nvec, int V, int kS, int32_t *__restrict__ top_id) {
     using namespace fb;
-    __shared__ int bins[16][TOPK_THREADS];
-    __shared__ int wsum[TOPK_THREADS / 32][16];
-    __shared__ int red[TOPK_THREADS / 32];
-    __shared__ int sh_above, sh_prefix, sh_n;
-    __shared__ int sel_id[SPECROLL_MAX_TOPK];
-    __shared__ uint32_t sel_key[SPECROLL_MAX_TOPK];
-    const int r = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint16_t *row = logits + (size_t)rec_row[r] * V;
-    const uint4 *p = reinterpret_cast<const uint4 *>(row);
-    const int nvec = V >> 3;
-    if (tid == 0) {
-        sh_above = 0;
-        sh_prefix = 0;
-        sh_n = 0;
-    }
-    __syncthreads();
+    auto &bins = sm.bins;
+    auto &wsum = sm.wsum;
+    auto &red = sm.red;
+    auto &sel_id = sm.sel_id;
+    auto &sel_key = sm.sel_key;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // ---- key of the kS-th largest value: four radix passes over the counts
     for (int level = 0; level < 4; ++level) {
         const int shift = 12 - 4 * level;
@@ -191,7 +198,94 @@ feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restr
         const int ii = sel_id[tid];
         int rk = 0;
         for (int j = 0; j < n_sel; ++j) rk += (sel_key[j] > ki) || (sel_key[j] == ki && sel_id[j] < ii);
-        top_id[(size_t)r * kS + rk] = ii;
+        top_id[rk] = ii;
+    }
+}
+
+// top_id[r, 0..kS): ids of the kS largest logits of row rec_row[r], by (logit desc, id asc).
+// List method, two passes over the row: (1) every thread finds the largest key of its strided share of the row; the
+// kS-th largest of those 512 values is a lower bound of the kS-th largest key of the row (there are at least kS
+// elements at or above it); (2) the elements at or above the bound, a few more than kS unless the large values
+// sit in few threads' shares, go into a list in shared memory, and an entry's rank in the list by (key desc, id
+// asc) is its place in the result.  A list longer than its capacity (a row with thousands of equal large values)
+// falls back to the radix search.
+__global__ void __launch_bounds__(fb::TOPK_THREADS)
+feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restrict__ rec_row, int V, int kS,
+                     int32_t *__restrict__ top_id) {
+    using namespace fb;
+    __shared__ union {
+        TopkRadixSmem radix;
+        TopkListSmem list;
+    } sm;
+    __shared__ int sh_above, sh_prefix, sh_n;
+    __shared__ uint32_t sh_bound;
+    const int r = blockIdx.x, tid = threadIdx.x;
+    const uint16_t *row = logits + (size_t)rec_row[r] * V;
+    const uint4 *p = reinterpret_cast<const uint4 *>(row);
+    const int nvec = V >> 3;
+    int32_t *out = top_id + (size_t)r * kS;
+    const int n_sel = min(kS, V);
+    if (tid == 0) sh_n = 0;
+    // ---- pass 1: the largest key of this thread's share
+    uint32_t best = 0u;
+    for (int i = tid; i < nvec; i += TOPK_THREADS) {
+        const uint4 v = ld_nc_v4(p + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int t = 0; t < 8; ++t) best = max(best, ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu)));
+    }
+    sm.list.best[tid] = best;
+    __syncthreads();
+    {
+        // the n_sel-th largest of the threads' values (ties broken by thread index: any of them will do as the bound)
+        int rk = 0;
+        for (int j = 0; j < TOPK_THREADS; ++j) {
+            const uint32_t o = sm.list.best[j];
+            rk += (o > best) || (o == best && j < tid);
+        }
+        if (rk == min(n_sel, TOPK_THREADS) - 1) sh_bound = best;
+    }
+    __syncthreads();
+    const uint32_t bound = sh_bound;
+    // ---- pass 2: everything at or above the bound
+    for (int i = tid; i < nvec; i += TOPK_THREADS) {
+        const uint4 v = ld_nc_v4(p + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const uint32_t key = ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
+            if (key >= bound) {
+                const int pos = atomicAdd(&sh_n, 1);
+                if (pos < TOPK_LIST_CAP) {
+                    sm.list.key[pos] = key;
+                    sm.list.id[pos] = i * 8 + t;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    const int n = sh_n;
+    if (n > TOPK_LIST_CAP || n < n_sel) {  // (n < n_sel cannot happen; the radix search is exact for every row)
+        __syncthreads();
+        if (tid == 0) {
+            sh_above = 0;
+            sh_prefix = 0;
+            sh_n = 0;
+        }
+        __syncthreads();
+        topk_radix(sm.radix, sh_above, sh_prefix, sh_n, p, nvec, V, kS, out);
+        return;
+    }
+    // ---- rank within the list
+    for (int e = tid; e < n; e += TOPK_THREADS) {
+        const uint32_t ke = sm.list.key[e];
+        const int ie = sm.list.id[e];
+        int rk = 0;
+        for (int j = 0; j < n; ++j) {
+            const uint32_t kj = sm.list.key[j];
+            rk += (kj > ke) || (kj == ke && sm.list.id[j] < ie);
+        }
+        if (rk < n_sel) out[rk] = ie;
     }
 }
 

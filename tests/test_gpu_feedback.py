@@ -88,3 +88,27 @@ def test_bad_arguments():
         S.reflex_feedback(*args, 2)            # support smaller than k
     with pytest.raises(S.SpecrollError):
         S.reflex_feedback(*args, 128)          # above the limit
+
+
+def test_thousands_of_equal_maxima_take_the_exact_fallback():
+    # more equal large values than the candidate list of the two-pass method holds: the radix search takes over,
+    # and the lowest ids win the ties, as in the oracle
+    R, V, d, k, kS = 2, 8192, 64, 4, 16
+    W, logits, rec_row, cand_id, cand_logit, y, m, rec_mem, rho = _case(33, R, V, d, k, R)
+    lf = np.full((R, V), -1.0, np.float32)
+    lf[:, 1::2] = 1.5                     # 4096 tokens share the maximum
+    lf[1, 4000] = 2.5
+    logits = I.f32_to_bf16_bits(lf)
+    rec_row = np.arange(R, dtype=np.int32)
+    o = ref.reflex_feedback(logits, W, cand_id, cand_logit, y, m[rec_mem], rho, kS)
+    row_max = lf.max(-1).astype(np.float32)
+    row_sum = np.exp(lf.astype(np.float64) - row_max[:, None]).sum(-1).astype(np.float32)
+    dm = dev(m.copy())
+    g = S.reflex_feedback(dev_bf16(logits), dev(rec_row), dev(row_max), dev(row_sum), dev(cand_id), dev(cand_logit),
+                          dev(y), dev_bf16(W), dev(rho), dev(rec_mem), dm, kS)
+    np.testing.assert_allclose(host(g["d_cov"]), o["d_cov"], rtol=2e-4, atol=1e-6)
+    np.testing.assert_allclose(host(g["d_dist"]), o["d_dist"], rtol=2e-4, atol=1e-6)
+    want = m.astype(np.float64).copy()
+    want[rec_mem] = o["m"]
+    np.testing.assert_allclose(host(dm), want, rtol=1e-3, atol=1e-4 * np.abs(want).max())
+
