@@ -696,18 +696,25 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     float ls0 = 0.f, ls1 = 0.f;
                     auto exp_group = [&](const uint32_t(&src)[32], uint32_t bc, float mref_, uint32_t *pk) {
                         if (full) {
+                            // in three sweeps (scale-and-shift, exponentials, sums and packing), so that no instruction
+                            // waits for the exponential issued just before it
                             const uint64_t sc2 = pack_f32x2(sc, sc), nm2 = pack_f32x2(-mref_, -mref_);
-                            uint64_t ls2 = pack_f32x2(ls0, ls1);
+                            float v[32];
 #pragma unroll
-                            for (int i2 = 0; i2 < 32; i2 += 2) {
-                                float t0, t1;
+                            for (int i2 = 0; i2 < 32; i2 += 2)
                                 unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(src[i2]), __uint_as_float(src[i2 + 1])), sc2, nm2),
-                                             t0, t1);
-                                const float p0 = ex2_approx(t0), p1 = ex2_approx(t1);
-                                ls2 = add_f32x2(ls2, pack_f32x2(p0, p1));
-                                pk[i2 >> 1] = pack_bf16x2(p0, p1);
+                                             v[i2], v[i2 + 1]);
+#pragma unroll
+                            for (int i2 = 0; i2 < 32; ++i2) v[i2] = ex2_approx(v[i2]);
+                            uint64_t ls2 = pack_f32x2(ls0, ls1), ls3 = pack_f32x2(0.f, 0.f);
+#pragma unroll
+                            for (int i2 = 0; i2 < 32; i2 += 4) {
+                                ls2 = add_f32x2(ls2, pack_f32x2(v[i2], v[i2 + 1]));
+                                ls3 = add_f32x2(ls3, pack_f32x2(v[i2 + 2], v[i2 + 3]));
+                                pk[i2 >> 1] = pack_bf16x2(v[i2], v[i2 + 1]);
+                                pk[(i2 >> 1) + 1] = pack_bf16x2(v[i2 + 2], v[i2 + 3]);
                             }
-                            unpack_f32x2(ls2, ls0, ls1);
+                            unpack_f32x2(add_f32x2(ls2, ls3), ls0, ls1);
                         } else {
 #pragma unroll
                             for (int i2 = 0; i2 < 32; i2 += 2) {
