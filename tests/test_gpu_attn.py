@@ -62,8 +62,8 @@ def test_tiny_config():
 @pytest.mark.parametrize("Hq,Hkv,D,N", [(12, 2, 128, 16), (28, 4, 128, 32), (40, 8, 128, 48), (10, 2, 64, 13),
                                         (28, 4, 128, 64), (4, 4, 128, 1), (14, 2, 64, 37), (14, 2, 64, 30)])
 def test_group_sizes_head_dims_and_tree_sizes(Hq, Hkv, D, N):
-    # G = 6, 7, 5, 5, 7, 1, 7, 7; rows = 96, 224, 240, 65, 448, 1, 259, 210 (one to four row blocks; an even
-    # number of blocks runs two per work unit, an odd number one per unit)
+    # G = 6, 7, 5, 5, 7, 1, 7, 7; rows = 96, 224, 240, 65, 448, 1, 259, 210 (one to four row blocks: the softmax
+    # with two threads per row for one block, the two alternating teams for more)
     K = 5
     w = I.scaled(I.WORKLOADS["qwen7b"], B=5, N=N, K=K, Hq=Hq, Hkv=Hkv, D=D, kv_a=300, kv_b=900)
     x = I.attn_inputs(w)

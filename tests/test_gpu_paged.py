@@ -34,7 +34,7 @@ def _gpu_paged(x, Kp, Vp, pt, pi, kl, **kw):
 
 @pytest.mark.parametrize("Hq,Hkv,D,N,lengths", [
     (12, 2, 128, 16, [700, 64, 1, 333, 129]),          # one row block
-    (28, 4, 128, 32, [900, 128, 70, 0, 257]),           # two row blocks per unit; an empty cache
+    (28, 4, 128, 32, [900, 128, 70, 0, 257]),           # two row blocks (two units per chunk and KV head); an empty cache
     (14, 2, 64, 37, [640, 64, 300, 127, 129]),          # three row blocks, head dim 64
     (12, 2, 128, 16, [5000, 64, 700, 129, 256]),        # a sequence cut into many chunks (merge kernel)
 ])
