@@ -309,6 +309,31 @@ int specroll_reflex_gate(const specroll_gate_desc *desc, const float *s, const f
                          const float *alpha_hi, float *a, float *rel, float *alpha, void *cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * The target's vocabulary projection with the verification's row statistics fused in, so that the
+ * logits of the tree nodes never reach memory (Sec. 3.2: p_u of every tree prefix from one packed
+ * target forward; App. B.2 uses, per node, the softmax normaliser and the probabilities of the node's
+ * candidate tokens only).  The paper does not describe this fusion; it computes the same quantities:
+ *   l[r, v]        = bf16( H[r, :] . W[v, :] )            (rounded as a storing projection would)
+ *   row_max[r]     = max_v l[r, v];   row_sum[r] = sum_v exp((l[r, v] - row_max[r]) / T)
+ *   want_logit[r,q] = l[r, want_id[r, q]]                  q < kw <= 8
+ * H[R, d] bf16 (rows = (sequence, node) in the order of the logits tensor of specroll_verify), W[V, d]
+ * bf16, want_id[R, kw] i32 (tokens in [0, V); nullable when kw == 0), row_max, row_sum[R] fp32,
+ * want_logit[R, kw] bf16.  d % 64 == 0, V % 8 == 0.  The workspace is scratch of this call.
+ *
+ * specroll_target_head_rows is the same product storing its logits[R, V] bf16: the one full row per
+ * sequence that the terminal draw reads (H then holds the hidden states of the terminal nodes, e.g. from
+ * specroll_gather_hidden).  status: one i32 on the device, SPECROLL_ETIMEOUT if a wait ran out. */
+size_t specroll_target_head_stats_workspace_bytes(int32_t R, int32_t d, int32_t V);
+
+int specroll_target_head_stats(int32_t R, int32_t d, int32_t V, float temperature, const void *H,
+                               const void *W, const int32_t *want_id, int32_t kw, float *row_max,
+                               float *row_sum, void *want_logit, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream);
+
+int specroll_target_head_rows(int32_t R, int32_t d, int32_t V, const void *H, const void *W,
+                              void *logits, int32_t *status, void *cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * Exact target verification (App. B.2 Eq. "nodeaccept" / "noderesidual", Algorithm "Exact
  * node-wise tree verification").
  *

@@ -445,3 +445,24 @@ def reflex_gate(s, xi, slot, keep, n, mean, M2, n_fb, m, horizon, n_align_min, n
         if n[j] >= n_align_min[h] and n_fb[j] >= n_fb_min[h] and rel[j] > 0.0 and rms > mem_eps:
             alpha[j] = alpha_lo[h] + (alpha_hi[h] - alpha_lo[h]) * min(rel[j], 1.0)
     return {"a": a, "n": n, "mean": mean, "M2": M2, "n_fb": n_fb, "rel": rel, "alpha": alpha}
+
+
+def target_head(H, W, temperature=1.0, want_id=None):
+    """The target's vocabulary projection followed by what the verification takes from it (Sec. 3.2, App. B.2):
+    l = bf16(H W^T) with H [R,d], W [V,d] bf16 bit patterns (products and sums in fp64, one rounding to bf16, as a
+    projection that stores bf16 logits does), row_max = max_v l, row_sum = sum_v exp((l - row_max)/T), and the logits
+    at want_id [R,kw].  Returns the logits as bf16 bit patterns too."""
+    H, W = _as(H, np.uint16), _as(W, np.uint16)
+    Hf = (H.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    Wf = (W.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    T = float(np.float32(temperature))
+    l64 = Hf @ Wf.T
+    bits = round_bf16(l64)
+    l = (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    row_max = l.max(-1)
+    row_sum = np.exp((l - row_max[:, None]) / T).sum(-1)
+    out = {"logits": bits, "row_max": row_max, "row_sum": row_sum}
+    if want_id is not None:
+        out["want_logit"] = np.take_along_axis(bits, np.asarray(want_id, np.int64), -1)
+    return out
+

@@ -27,7 +27,8 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
            "specroll_verify_workspace_bytes", "specroll_verify", "specroll_verify_static",
            "specroll_verify_nucleus_workspace_bytes", "specroll_verify_nucleus",
            "specroll_reflex_feedback_workspace_bytes", "specroll_reflex_feedback", "specroll_reflex_feedback_ex",
-           "specroll_reflex_sketch", "specroll_reflex_gate")
+           "specroll_reflex_sketch", "specroll_reflex_gate",
+           "specroll_target_head_stats_workspace_bytes", "specroll_target_head_stats", "specroll_target_head_rows")
 
 
 PROPOSE_LEGACY_MMA = 1
@@ -85,7 +86,8 @@ def lib():
         l.specroll_node_budget.argtypes = [C.c_int32] * 4
         for n in ("specroll_propose_workspace_bytes", "specroll_verify_workspace_bytes",
                   "specroll_tree_attn_workspace_bytes", "specroll_tree_attn_paged_workspace_bytes",
-                  "specroll_verify_nucleus_workspace_bytes", "specroll_reflex_feedback_workspace_bytes"):
+                  "specroll_verify_nucleus_workspace_bytes", "specroll_reflex_feedback_workspace_bytes",
+                  "specroll_target_head_stats_workspace_bytes"):
             getattr(l, n).restype = C.c_size_t
         for n in ("specroll_propose", "specroll_workspace_status", "specroll_tree_draw", "specroll_tree_attn",
                   "specroll_verify", "specroll_verify_static", "specroll_tree_attn_paged", "specroll_commit_path",
@@ -520,6 +522,45 @@ def reflex_gate(s, xi, slot, keep, n, mean, M2, n_fb, m, horizon, n_align_min, n
         _dev(alpha_hi, f32, "alpha_hi"), _dev(out["a"], f32, "a"), _dev(out["rel"], f32, "rel"),
         _dev(out["alpha"], f32, "alpha"), _stream())
     _check(rc, "specroll_reflex_gate")
+    return out
+
+
+def target_head_stats(H, W, want_id=None, temperature=1.0, workspace=None):
+    """specroll_target_head_stats: row_max, row_sum [R] and want_logit [R, kw] (bf16) of l = bf16(H W^T) without
+    storing l.  H [R, d] bf16, W [V, d] bf16, want_id [R, kw] i32 or None."""
+    R, d = H.shape
+    V = W.shape[0]
+    kw = 0 if want_id is None else want_id.shape[1]
+    dev = H.device
+    out = {"row_max": torch.empty(R, dtype=torch.float32, device=dev),
+           "row_sum": torch.empty(R, dtype=torch.float32, device=dev),
+           "want_logit": torch.empty((R, kw), dtype=torch.bfloat16, device=dev)}
+    need = lib().specroll_target_head_stats_workspace_bytes(C.c_int32(R), C.c_int32(d), C.c_int32(V))
+    if need == 0:
+        raise SpecrollError("target_head_stats: invalid shape")
+    if workspace is None:
+        workspace = _workspace(need, dev)
+    rc = lib().specroll_target_head_stats(
+        C.c_int32(R), C.c_int32(d), C.c_int32(V), C.c_float(temperature), _dev(H, torch.bfloat16, "H"),
+        _dev(W, torch.bfloat16, "W"), _dev(want_id, torch.int32, "want_id") if kw else None, C.c_int32(kw),
+        _dev(out["row_max"], torch.float32, "row_max"), _dev(out["row_sum"], torch.float32, "row_sum"),
+        _dev(out["want_logit"], torch.bfloat16, "want_logit") if kw else None, C.c_void_p(workspace.data_ptr()),
+        C.c_size_t(workspace.numel()), _stream())
+    _check(rc, "specroll_target_head_stats")
+    return out
+
+
+def target_head_rows(H, W, out=None):
+    """specroll_target_head_rows: logits [R, V] bf16 = bf16(H W^T)."""
+    R, d = H.shape
+    V = W.shape[0]
+    if out is None:
+        out = torch.empty((R, V), dtype=torch.bfloat16, device=H.device)
+    status = torch.zeros(1, dtype=torch.int32, device=H.device)
+    rc = lib().specroll_target_head_rows(C.c_int32(R), C.c_int32(d), C.c_int32(V), _dev(H, torch.bfloat16, "H"),
+                                         _dev(W, torch.bfloat16, "W"), _dev(out, torch.bfloat16, "logits"),
+                                         _dev(status, torch.int32, "status"), _stream())
+    _check(rc, "specroll_target_head_rows")
     return out
 
 
