@@ -507,6 +507,34 @@ def run_calls(args, w, layers):
                                                      peaks["hbm_gbs"], "GB/s")
     calls["reflex_gate (B K records, B K slots)"] = (gate, "hbm", (R * w.d * 4 + 2 * R * rank * 4 + 8 * R * 4) / 1e9,
                                                     peaks["hbm_gbs"], "GB/s")
+    # the target projection with fused row statistics over all (sequence, node) rows, and its storing form on one
+    # row per sequence (the terminal rows)
+    hid = (0.02 * torch.randn((w.B * w.N, w.d), generator=gen, device=dev)).to(torch.bfloat16)
+    want = wl.prop["cand_id"][:, 0, :].repeat_interleave(w.N, dim=0).contiguous()[:, : min(w.k, 8)].contiguous()
+    th_ws = torch.empty(S.lib().specroll_target_head_stats_workspace_bytes(w.B * w.N, w.d, w.V) + 256,
+                        dtype=torch.uint8, device=dev)
+    rows_out = torch.empty((w.B, w.V), dtype=torch.bfloat16, device=dev)
+
+    def head_stats():
+        S.target_head_stats(hid, wl.W, want, temperature=w.temperature, workspace=th_ws)
+
+    def head_rows():
+        S.target_head_rows(hid[: w.B], wl.W, out=rows_out)
+
+    hid3 = hid.reshape(w.B, w.N, w.d)
+    p_ = wl.prop
+
+    def verify_from_hidden():
+        S.verify_fused(hid3, wl.W, wl.parent, p_["tree_tok"], p_["tree_cand"], p_["cand_id"][:, :, : min(w.k, 8)].contiguous(),
+                       p_["cand_logit"][:, :, : min(w.k, 8)].contiguous(), wl.u_acc, wl.u_fin, temperature=w.temperature)
+
+    if w.k <= 8:
+        calls["verify_fused (projection + statistics + walk + terminal rows, from hidden states)"] = (
+            verify_from_hidden, "tensor", 2.0 * w.B * (w.N + 1) * w.d * w.V / 1e12, peaks["bf16_tflops"], "TFLOP/s")
+    calls["target_head_stats (B N rows, fused statistics)"] = (
+        head_stats, "tensor", 2.0 * w.B * w.N * w.d * w.V / 1e12, peaks["bf16_tflops"], "TFLOP/s")
+    calls["target_head_rows (B rows stored)"] = (
+        head_rows, "hbm", (w.V * w.d * 2 + w.B * w.V * 2) / 1e9, peaks["hbm_gbs"], "GB/s")
     out = {"workload": w.name, "peak_source": peaks["source"], "calls": {}}
     for name, (fn, bound, work, peak, unit) in calls.items():
         rec = {"bound": bound, "unit": unit, "peak": peak, "work_per_call": work}

@@ -376,6 +376,32 @@ int specroll_verify(const specroll_verify_desc *desc, const void *logits,
                     float *row_sum, float *min_margin, void *workspace, size_t workspace_bytes,
                     void *cuda_stream);
 
+/* Verification without the logits tensor (the same algorithm as specroll_verify, which see for the
+ * arguments; only where the target's numbers come from differs):
+ *   specroll_verify_want_ids     want_id[(b, u), j] = cand_id[b, depth(u), j], the tokens whose target logit the
+ *                                walk reads at node u (input of specroll_target_head_stats with kw = k <= 8);
+ *   specroll_verify_walk_sparse  the node-wise walk from row_max, row_sum[B*N] and cand_target[B, N, k] bf16 (the
+ *                                wanted logits); writes n_acc, path_node, the accepted tokens of out_tok, term_node,
+ *                                term_kind, min_margin (nullable) and leaves the residual in the workspace;
+ *   specroll_verify_terminal_rows  the step's last token from term_logits[B, V] bf16, the full logits row of
+ *                                every sequence's terminal node, with the same workspace.
+ * The workspace has specroll_verify_workspace_bytes(desc) bytes; desc.flags must be 0. */
+int specroll_verify_want_ids(const specroll_verify_desc *desc, const int32_t *parent_host,
+                             const int32_t *cand_id, int32_t *want_id, void *cuda_stream);
+
+int specroll_verify_walk_sparse(const specroll_verify_desc *desc, const void *cand_target,
+                                const float *row_max, const float *row_sum, const int32_t *parent_host,
+                                const int32_t *tree_tok, const uint8_t *tree_cand, const int32_t *cand_id,
+                                const float *cand_logit, const float *u_acc, int32_t *n_acc,
+                                int32_t *path_node, int32_t *out_tok, int32_t *term_node,
+                                int32_t *term_kind, float *min_margin, void *workspace,
+                                size_t workspace_bytes, void *cuda_stream);
+
+int specroll_verify_terminal_rows(const specroll_verify_desc *desc, const void *term_logits,
+                                  const float *row_max, const int32_t *n_acc, const int32_t *term_node,
+                                  const float *u_fin, int32_t *out_tok, void *workspace,
+                                  size_t workspace_bytes, void *cuda_stream);
+
 /* The same verification against nucleus-truncated target distributions (App. "Implementation and
  * Reproducibility Details": rollouts sample at temperature 1.0 and nucleus threshold 0.95).  p_n is
  * replaced by its renormalised restriction to the nucleus: tokens in order of decreasing probability

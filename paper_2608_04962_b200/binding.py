@@ -28,7 +28,8 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
            "specroll_verify_nucleus_workspace_bytes", "specroll_verify_nucleus",
            "specroll_reflex_feedback_workspace_bytes", "specroll_reflex_feedback", "specroll_reflex_feedback_ex",
            "specroll_reflex_sketch", "specroll_reflex_gate",
-           "specroll_target_head_stats_workspace_bytes", "specroll_target_head_stats", "specroll_target_head_rows")
+           "specroll_target_head_stats_workspace_bytes", "specroll_target_head_stats", "specroll_target_head_rows",
+           "specroll_verify_want_ids", "specroll_verify_walk_sparse", "specroll_verify_terminal_rows")
 
 
 PROPOSE_LEGACY_MMA = 1
@@ -411,6 +412,48 @@ def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fi
         _dev(out["row_sum"], f32, "row_sum"), _dev(out.get("min_margin"), f32, "min_margin"),
         C.c_void_p(workspace.data_ptr()), C.c_size_t(workspace.numel()), _stream())
     _check(rc, "specroll_verify")
+    return out
+
+
+def verify_fused(hidden, W, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, temperature=1.0):
+    """Exact verification from the target's final hidden states, without the logits tensor: the projection with
+    fused row statistics over all (sequence, node) rows (specroll_target_head_stats), the walk on the target logits
+    of the candidate tokens (specroll_verify_walk_sparse), then the one row per sequence that the terminal draw
+    needs (specroll_gather_hidden, specroll_target_head_rows, specroll_verify_terminal_rows).
+    hidden [B, N, d] bf16, W [V, d] bf16; the other arguments as for ``verify``.  Returns the same dict."""
+    parent = _host_i32(parent, "parent")
+    B, N, d = hidden.shape
+    V = W.shape[0]
+    _, K, k = cand_id.shape
+    desc = VerifyDesc(B, N, K, k, V, temperature, 0)
+    dev = hidden.device
+    i32, f32 = torch.int32, torch.float32
+    want = torch.empty((B * N, k), dtype=i32, device=dev)
+    rc = lib().specroll_verify_want_ids(C.byref(desc), parent.ctypes.data_as(C.c_void_p), _dev(cand_id, i32, "cand_id"),
+                                        _dev(want, i32, "want_id"), _stream())
+    _check(rc, "specroll_verify_want_ids")
+    st = target_head_stats(hidden.reshape(B * N, d), W, want, temperature=temperature)
+    out = {"n_acc": torch.empty(B, dtype=i32, device=dev), "path_node": torch.empty((B, K + 1), dtype=i32, device=dev),
+           "out_tok": torch.empty((B, K + 1), dtype=i32, device=dev), "term_node": torch.empty(B, dtype=i32, device=dev),
+           "term_kind": torch.empty(B, dtype=i32, device=dev), "row_max": st["row_max"].reshape(B, N),
+           "row_sum": st["row_sum"].reshape(B, N), "min_margin": torch.empty(B, dtype=f32, device=dev)}
+    ws = _workspace(lib().specroll_verify_workspace_bytes(C.byref(desc)), dev)
+    rc = lib().specroll_verify_walk_sparse(
+        C.byref(desc), _dev(st["want_logit"], torch.bfloat16, "cand_target"), _dev(st["row_max"], f32, "row_max"),
+        _dev(st["row_sum"], f32, "row_sum"), parent.ctypes.data_as(C.c_void_p), _dev(tree_tok, i32, "tree_tok"),
+        _dev(tree_cand, torch.uint8, "tree_cand"), _dev(cand_id, i32, "cand_id"), _dev(cand_logit, f32, "cand_logit"),
+        _dev(u_acc, f32, "u_acc"), _dev(out["n_acc"], i32, "n_acc"), _dev(out["path_node"], i32, "path_node"),
+        _dev(out["out_tok"], i32, "out_tok"), _dev(out["term_node"], i32, "term_node"),
+        _dev(out["term_kind"], i32, "term_kind"), _dev(out["min_margin"], f32, "min_margin"),
+        C.c_void_p(ws.data_ptr()), C.c_size_t(ws.numel()), _stream())
+    _check(rc, "specroll_verify_walk_sparse")
+    h_term = gather_hidden(hidden, out["term_node"])
+    rows = target_head_rows(h_term, W)
+    rc = lib().specroll_verify_terminal_rows(
+        C.byref(desc), _dev(rows, torch.bfloat16, "term_logits"), _dev(st["row_max"], f32, "row_max"),
+        _dev(out["n_acc"], i32, "n_acc"), _dev(out["term_node"], i32, "term_node"), _dev(u_fin, f32, "u_fin"),
+        _dev(out["out_tok"], i32, "out_tok"), C.c_void_p(ws.data_ptr()), C.c_size_t(ws.numel()), _stream())
+    _check(rc, "specroll_verify_terminal_rows")
     return out
 
 

@@ -321,6 +321,9 @@ __device__ void nucleus_row(const uint16_t *__restrict__ row_logits, int V, floa
 
 struct WalkArgs {
     const uint16_t *logits;
+    // sparse form (logits == NULL): the target logits of every node at the candidates of the node's head only,
+    // [B, N, k] bf16, as specroll_target_head_stats leaves them
+    const uint16_t *cand_target;
     const int32_t *tree_tok;
     const uint8_t *tree_cand;
     const int32_t *cand_id;
@@ -380,12 +383,13 @@ __device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, doub
     int32_t *id = sm->id;
     const int k = a.k, N = a.N, K = a.K;
     const int hd = topo.depth[u];
-    const uint16_t *lg = a.logits + ((size_t)b * N + u) * a.V;
+    const uint16_t *lg = a.logits ? a.logits + ((size_t)b * N + u) * a.V : nullptr;
+    const uint16_t *ct = a.cand_target ? a.cand_target + ((size_t)b * N + u) * k : nullptr;
     for (int j = lane; j < k; j += 32) {
         const int t = a.cand_id[((size_t)b * K + hd) * k + j];
         id[j] = t;
         cl[j] = a.cand_logit[((size_t)b * K + hd) * k + j];
-        const uint32_t bits = lg[t];
+        const uint32_t bits = lg ? lg[t] : ct[j];
         const double l = (double)bf16_bits_to_float((uint16_t)bits);
         r[j] = ord_key(bits) >= thr ? exp((l - M) / a.T) / S : 0.0;  // r = p_u on the candidates
     }
@@ -627,6 +631,7 @@ struct TermArgs {
     int32_t *out_tok;
     int32_t B, N, K, k, V;
     float c;  // log2(e) / T
+    int32_t row_per_seq;  // logits holds one row per sequence (that of its terminal node) instead of [B, N, V]
 };
 
 // Plain softmax masses of eight tokens; tokens below the nucleus threshold (thr = 0: none) weigh nothing.
@@ -676,7 +681,7 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
     const int nov = a.ws_nov[b];
     const float M = a.row_max[(size_t)b * a.N + node];
     const uint32_t thr = a.thr_key ? a.thr_key[(size_t)b * a.N + node] : 0u;
-    const uint16_t *lg = a.logits + ((size_t)b * a.N + node) * a.V;
+    const uint16_t *lg = a.logits + (a.row_per_seq ? (size_t)b : (size_t)b * a.N + node) * a.V;
     const uint4 *p = reinterpret_cast<const uint4 *>(lg);
     const int nvec = a.V >> 3;
     const int vpw = (nvec + TERM_WARPS - 1) / TERM_WARPS;  // vectors per warp segment
@@ -931,6 +936,7 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
 
     WalkArgs wa;
     wa.logits = static_cast<const uint16_t *>(logits);
+    wa.cand_target = nullptr;
     wa.tree_tok = tree_tok;
     wa.tree_cand = tree_cand;
     wa.cand_id = cand_id;
@@ -993,7 +999,123 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
     ta.k = d->k;
     ta.V = d->V;
     ta.c = c;
+    ta.row_per_seq = 0;
     return launch_terminal(ta, st);
+}
+
+// The hand-over area between the walk and the terminal draw inside a workspace (the layout of run_verify).
+static void carve_verify_ws(const specroll_verify_desc *d, void *workspace, double **ovm, int32_t **ovid, int32_t **nov) {
+    const size_t B = (size_t)d->B, k = (size_t)d->k;
+    char *ws = static_cast<char *>(workspace);
+    *ovm = reinterpret_cast<double *>(ws);
+    ws += align_up(B * k * sizeof(double), 256);
+    *ovid = reinterpret_cast<int32_t *>(ws);
+    ws += align_up(B * k * sizeof(int32_t), 256);
+    *nov = reinterpret_cast<int32_t *>(ws);
+}
+
+namespace specroll {
+// want_id[(b, u), j] = cand_id[b, depth(u), j]: the tokens whose target logit the walk reads at node u
+__global__ void want_ids_kernel(Topo topo, int B, int N, int K, int k, const int32_t *__restrict__ cand_id,
+                                int32_t *__restrict__ want_id) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)B * N * k) return;
+    const int j = (int)(i % k), u = (int)((i / k) % N), b = (int)(i / ((size_t)k * N));
+    const int hd = min((int)topo.depth[u], K - 1);  // (a node of the last level has no children; any valid token)
+    want_id[i] = cand_id[((size_t)b * K + hd) * k + j];
+}
+}  // namespace specroll
+
+extern "C" int specroll_verify_want_ids(const specroll_verify_desc *d, const int32_t *parent_host,
+                                        const int32_t *cand_id, int32_t *want_id, void *cuda_stream) {
+    if (check_verify_desc(d) != SPECROLL_OK || !cand_id || !want_id) return SPECROLL_EINVAL;
+    Topo topo;
+    if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
+    const size_t n = (size_t)d->B * d->N * d->k;
+    if (n == 0) return SPECROLL_OK;
+    want_ids_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        topo, d->B, d->N, d->K, d->k, cand_id, want_id);
+    SR_LAUNCH_CHECK();
+    return SPECROLL_OK;
+}
+
+extern "C" int specroll_verify_walk_sparse(const specroll_verify_desc *d, const void *cand_target,
+                                           const float *row_max, const float *row_sum, const int32_t *parent_host,
+                                           const int32_t *tree_tok, const uint8_t *tree_cand, const int32_t *cand_id,
+                                           const float *cand_logit, const float *u_acc, int32_t *n_acc,
+                                           int32_t *path_node, int32_t *out_tok, int32_t *term_node,
+                                           int32_t *term_kind, float *min_margin, void *workspace,
+                                           size_t workspace_bytes, void *cuda_stream) {
+    if (check_verify_desc(d) != SPECROLL_OK || d->flags != 0) return SPECROLL_EINVAL;
+    if (!cand_target || !row_max || !row_sum || !tree_tok || !tree_cand || !cand_id || !cand_logit || !u_acc || !n_acc ||
+        !path_node || !out_tok || !term_node || !term_kind)
+        return SPECROLL_EINVAL;
+    Topo topo;
+    if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (d->B == 0) return SPECROLL_OK;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < verify_ws_base(d))
+        return SPECROLL_EWORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    WalkArgs wa;
+    wa.logits = nullptr;
+    wa.cand_target = static_cast<const uint16_t *>(cand_target);
+    wa.tree_tok = tree_tok;
+    wa.tree_cand = tree_cand;
+    wa.cand_id = cand_id;
+    wa.cand_logit = cand_logit;
+    wa.u_acc = u_acc;
+    wa.row_max = row_max;
+    wa.row_sum = row_sum;
+    wa.n_acc = n_acc;
+    wa.path_node = path_node;
+    wa.out_tok = out_tok;
+    wa.term_node = term_node;
+    wa.term_kind = term_kind;
+    wa.min_margin = min_margin;
+    carve_verify_ws(d, workspace, &wa.ws_ovm, &wa.ws_ovid, &wa.ws_nov);
+    wa.B = d->B;
+    wa.N = d->N;
+    wa.K = d->K;
+    wa.k = d->k;
+    wa.V = d->V;
+    wa.T = (double)d->temperature;
+    walk_kernel<<<(d->B + WALK_WARPS - 1) / WALK_WARPS, WALK_WARPS * 32, 0, st>>>(wa, topo);
+    SR_LAUNCH_CHECK();
+    return SPECROLL_OK;
+}
+
+extern "C" int specroll_verify_terminal_rows(const specroll_verify_desc *d, const void *term_logits,
+                                             const float *row_max, const int32_t *n_acc, const int32_t *term_node,
+                                             const float *u_fin, int32_t *out_tok, void *workspace,
+                                             size_t workspace_bytes, void *cuda_stream) {
+    if (check_verify_desc(d) != SPECROLL_OK || d->flags != 0) return SPECROLL_EINVAL;
+    if (!term_logits || !row_max || !n_acc || !term_node || !u_fin || !out_tok) return SPECROLL_EINVAL;
+    if (!aligned16(term_logits)) return SPECROLL_EALIGN;
+    if (d->B == 0) return SPECROLL_OK;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < verify_ws_base(d))
+        return SPECROLL_EWORKSPACE;
+    TermArgs ta;
+    double *ovm;
+    int32_t *ovid, *nov;
+    carve_verify_ws(d, workspace, &ovm, &ovid, &nov);
+    ta.logits = static_cast<const uint16_t *>(term_logits);
+    ta.u_fin = u_fin;
+    ta.row_max = row_max;
+    ta.n_acc = n_acc;
+    ta.term_node = term_node;
+    ta.ws_nov = nov;
+    ta.ws_ovid = ovid;
+    ta.ws_ovm = ovm;
+    ta.thr_key = nullptr;
+    ta.out_tok = out_tok;
+    ta.B = d->B;
+    ta.N = d->N;
+    ta.K = d->K;
+    ta.k = d->k;
+    ta.V = d->V;
+    ta.c = (float)(1.4426950408889634 / (double)d->temperature);
+    ta.row_per_seq = 1;
+    return launch_terminal(ta, static_cast<cudaStream_t>(cuda_stream));
 }
 
 extern "C" int specroll_verify(const specroll_verify_desc *d, const void *logits,
