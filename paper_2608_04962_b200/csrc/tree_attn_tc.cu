@@ -18,15 +18,21 @@
 //   warp 2     one thread issues every  O += P V  (M=128, N=D, A = P from TMEM, B = V tile read
 //              MN-major from shared memory).  Two issuing threads, because one thread that also sits
 //              in the barrier waits left the tensor pipe idle more than half of the time.
-//   warps 3-10 softmax with TWO threads per query row (warps w and w+4 own the same 32 TMEM lanes
-//              and take columns 0-63 / 64-127 of each S tile).  The pair exchanges its two partial
-//              row maxima through shared memory once per tile.  At the end of a unit the threads
-//              leave the row's reference maximum and their shares of its sum in shared memory and go
-//              straight on to the next unit.
+//   warps 3-10 softmax, in one of two forms (template flag TEAMS, chosen by the number of row blocks):
+//              one row block (HBM-bound): TWO threads per query row (warps w and w+4 own the same 32 TMEM
+//              lanes and take columns 0-63 / 64-127 of each S tile); the pair exchanges one value per tile
+//              through shared memory.  More row blocks (softmax-bound): two TEAMS of four warps, one thread
+//              per row, team (t mod 2) takes tile t, so that one team's loads, stores and barrier round trips
+//              run under the other team's exponentials; the row's reference maximum travels from team to
+//              team through shared memory.  After the first tile(s) of a unit a tile takes one pass: the
+//              exponentials against the reference as it stands, the tile's sum as the alarm for a reference
+//              that has to move (then two passes from the S tile, which is still intact).  At the end of a
+//              unit the threads leave their reference maxima and their shares of the row sums in the
+//              workspace (one area per CTA) and go straight on to the next unit.
 //   warps 11-14 output: one thread per query row takes the finished accumulator out of TMEM (after
 //              the unit's last P V), normalises and stores it, or stores this chunk's fp32 partial.
-// P is written back to TMEM over parts of S that its writer has already read (columns [0,32) by
-// the first thread of a pair, [96,128) by the second), as packed bf16.  The output accumulator is
+// P is written back to TMEM over parts of S that its writer has already read (pairs: columns [0,32) by
+// the first thread, [96,128) by the second; teams: columns [0,64)), as packed bf16.  The output accumulator is
 // rescaled only when a row's reference maximum grows by more than 2^8 (rare).  Chunks of a split
 // sequence leave fp32 partials in the workspace; the CTA that finishes a sequence's last chunk
 // (atomic ticket, nobody waits) merges them, unless the plan leaves that to a kernel of its own.
