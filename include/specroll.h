@@ -140,6 +140,17 @@ typedef struct {
  * descriptor and the same kv_indptr values (typically the previous layer of the same step): do not
  * rebuild it.  Tensors (Q, K, V, O) may differ.  Ignored by the mma.sync kernel. */
 #define SPECROLL_ATTN_REUSE_PLAN 2
+/* The cache (Kc, Vc, or the pool and its page table) was last written before the kernel that
+ * precedes this call in the stream was launched, as is the case for every layer of a verification
+ * step whose cache was committed at the end of the step before.  Together with
+ * SPECROLL_ATTN_REUSE_PLAN this lets the attention kernel, which is launched as a programmatic
+ * dependent of that preceding kernel, fetch its first cache tiles while that kernel is still
+ * finishing; Q, the tree's K/V and the outputs are touched only after it has completed.  Without the
+ * flag nothing is read before then.  (Scheduling only; results do not depend on it.) */
+#define SPECROLL_ATTN_CACHE_SETTLED 4
+/* (The tcgen05 attention kernel is always launched with programmatic stream serialization; it waits
+ * for the kernel before it in the stream before it reads or writes anything, except as the flag above
+ * allows.  SPECROLL_ATTN_PDL=0 in the environment makes it an ordinary launch, for comparison.) */
 
 size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *desc,
                                           const int32_t *kv_indptr_host);

@@ -35,6 +35,7 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
 PROPOSE_LEGACY_MMA = 1
 ATTN_LEGACY_MMA = 1
 ATTN_REUSE_PLAN = 2
+ATTN_CACHE_SETTLED = 4
 VERIFY_LAZY_STATS = 1
 FEEDBACK_SEVERITY = 1
 PAGE_TOKENS = 128

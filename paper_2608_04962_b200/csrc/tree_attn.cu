@@ -497,7 +497,7 @@ struct AttnPlan {
 
 static int compute_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
     if (!d || !indptr_host || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->Hq < 1 || d->Hkv < 1 ||
-        (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || (d->flags & ~(SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN)) != 0 ||
+        (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || (d->flags & ~(SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN | SPECROLL_ATTN_CACHE_SETTLED)) != 0 ||
         !(d->scale > 0.f))
         return SPECROLL_EINVAL;
     const int G = d->Hq / d->Hkv;
@@ -632,7 +632,7 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     static unsigned next = 0;
     if (!d || !indptr_host || d->B < 0 || d->B > (1 << 24)) return compute_attn_plan(d, indptr_host, p);
     // what the key leaves out is checked here, so that a remembered plan never answers for an invalid call
-    if ((d->flags & ~(SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN)) != 0 || !(d->scale > 0.f)) return SPECROLL_EINVAL;
+    if ((d->flags & ~(SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN | SPECROLL_ATTN_CACHE_SETTLED)) != 0 || !(d->scale > 0.f)) return SPECROLL_EINVAL;
     const int key[7] = {d->B, d->N, d->Hq, d->Hkv, d->D, (int)(d->flags & SPECROLL_ATTN_LEGACY_MMA), 1};
     const size_t n = (size_t)d->B + 1;
     std::lock_guard<std::mutex> lock(mu);
@@ -731,6 +731,8 @@ static int run_tree_attn(const specroll_attn_desc *d, const void *Q, const void 
     a.total_work = p.items * d->Hkv * p.n_rb;
     a.merge_mode = p.merge_mode;
     a.nodes_per_block = p.nodes_per_block;
+    // early cache loads need a plan that is not being made by the kernel just before the attention kernel
+    a.early_cache = ((d->flags & SPECROLL_ATTN_CACHE_SETTLED) && (d->flags & SPECROLL_ATTN_REUSE_PLAN)) ? 1 : 0;
     if (!(p.use_tc && (d->flags & SPECROLL_ATTN_REUSE_PLAN))) {
         // (the tcgen05 kernel leaves its scheduling counters cleared, so a kept plan can be run again as is)
         attn_prep_kernel<<<1, PREP_THREADS, 0, st>>>(kv_indptr_dev, paged ? kv_len_dev : nullptr, page_indptr_dev, d->B,

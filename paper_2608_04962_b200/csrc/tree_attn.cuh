@@ -27,6 +27,7 @@ struct AttnArgs {
     // paged cache (tcgen05 kernel only): pool page of every 128-token tile; a chunk table row then carries the
     // sequence's first slot in this table instead of its first token
     const int32_t *page_table;
+    int early_cache;              // plan, cache and page table were complete before the preceding kernel was launched
     float *hand;                  // [ATTN_HAND_CTAS][4][128] per-CTA hand-over area between two groups of warps of the tcgen05 kernel
     int32_t merge_mode;           // chunks of a split sequence are merged 0: by the CTA that finishes last; 2: by a later kernel
 };

@@ -38,6 +38,7 @@
 // (atomic ticket, nobody waits) merges them, unless the plan leaves that to a kernel of its own.
 // TMEM columns: O: [0, 128);  S/P buffer i: [128 + 128 i, +128).
 #include <math.h>
+#include <stdlib.h>
 
 #include "tc05.cuh"
 #include "tree_attn.cuh"
@@ -248,6 +249,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Launched as a programmatic dependent of the kernel before it in the stream, this CTA may have done all
+    // of the above while that kernel was still finishing.  From here on it reads what earlier kernels wrote
+    // (the plan, the counters the launch before cleared, Q and the tree's K/V), so it waits for them to be
+    // complete.  The kernel after this one may be set up as early as its CTAs find room.
+    // Exception: when the caller has said that the plan and the cache were complete before that kernel was
+    // even launched, the loading thread fetches its first cache tiles right away and waits just before it
+    // needs Q (below).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const bool early = a.early_cache != 0;
+    if (!(early && warp == 0)) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // Sums the partials of all chunks of one (sequence, kv head, row block) for columns [col0, col0 + ncols) of one row;
     // run by the threads that own the row block, after the tickets showed that every chunk has been written.
@@ -374,11 +385,23 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     ok = false;
                     break;
                 }
-                mbar_arrive_expect_tx(bar(C::B_QFULL + qb), (uint32_t)(C::NBOX * 128 * a.rows_per_block));
+                auto load_q = [&]() {
+                    mbar_arrive_expect_tx(bar(C::B_QFULL + qb), (uint32_t)(C::NBOX * 128 * a.rows_per_block));
 #pragma unroll
-                for (int bx = 0; bx < C::NBOX; ++bx)
-                    tma_load_3d(q_s + qb * C::Q_BYTES + bx * BOX_BYTES, &tmQ, bx * 64, hkv * G, b * N + rb * a.nodes_per_block,
-                                bar(C::B_QFULL + qb));
+                    for (int bx = 0; bx < C::NBOX; ++bx)
+                        tma_load_3d(q_s + qb * C::Q_BYTES + bx * BOX_BYTES, &tmQ, bx * 64, hkv * G,
+                                    b * N + rb * a.nodes_per_block, bar(C::B_QFULL + qb));
+                };
+                // Early cache loads: the first unit's first three cache tiles (their stages are free, nothing
+                // here can block) go out before the kernel in front of this one has finished; Q and the tree's
+                // K/V may be that kernel's output, so they follow the wait.
+                bool q_pending = early && u == 0;
+                auto settle = [&]() {
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    load_q();
+                    q_pending = false;
+                };
+                if (!q_pending) load_q();
                 // ---- K tiles, each followed by the V tile from two tiles back.  Paged cache: kv0 is the sequence's
                 //      first slot in the page table and a tile is one pool page; page numbers are fetched two
                 //      tiles ahead of their use, under the wait for a free stage.
@@ -395,6 +418,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         break;
                     }
                     const bool tree = has_tree && (it == n_it - 1);
+                    if (q_pending && (tree || it >= 3)) settle();
                     const int tok = tree ? b * N : (pt ? pg0 * BN : kv0 + (t_lo + it) * BN);
                     pg0 = pg1;
                     pg1 = pg2;
@@ -418,6 +442,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     pv_tok[n_pend] = tok;
                     ++n_pend;
                 }
+                if (q_pending) settle();
                 // the unit's last V tiles go out now if their stages are already free; otherwise they wait
                 // behind the next unit's Q and first K tiles (never block here)
                 auto v_stage_free = [&]() {
@@ -434,6 +459,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     --n_pend;
                 }
             }
+            // (a thread that left the loop early has not waited yet; the counters touched at the end of the
+            // kernel are cleared by the launch before this one)
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             // flush the V tiles still pending (the last two tiles of the last unit)
             for (int i = 0; i < n_pend && ok; ++i) ok = load_v(pv_map[i], pv_h[i], pv_tok[i]);
             if (!ok) {
@@ -1146,7 +1174,24 @@ static int launch_tc(const AttnArgs &a, const TopoMask &mask, long long T_kv, in
     }
     const int ctas = n_sm < ATTN_HAND_CTAS ? n_sm : ATTN_HAND_CTAS;  // every CTA has a hand-over area of its own
     const unsigned grid = (unsigned)(a.total_work < ctas ? a.total_work : ctas);
-    tree_attn_tc_kernel<D, TEAMS><<<grid, C::THREADS, C::SMEM, st>>>(tmQ, tmK, tmV, tmKt, tmVt, a, mask, status);
+    // Programmatic stream serialization: the CTAs may be set up (barriers, tensor memory, zeroed Q buffers) while
+    // the kernel before this one in the stream is still running its last CTAs; the kernel itself waits for
+    // that kernel's completion before it reads anything (griddepcontrol.wait).
+    static const bool pdl = []() {
+        const char *e = getenv("SPECROLL_ATTN_PDL");
+        return !(e && e[0] == '0');
+    }();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(C::THREADS);
+    cfg.dynamicSmemBytes = C::SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    SR_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<D, TEAMS>, tmQ, tmK, tmV, tmKt, tmVt, a, mask, status));
     SR_LAUNCH_CHECK();
     return SPECROLL_OK;
 }

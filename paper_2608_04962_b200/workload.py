@@ -143,15 +143,17 @@ class StepWorkload:
         return self.prop
 
     def attn(self, layer: int):
-        # every layer of a step sees the same KV lengths: layers after the first reuse the work plan
+        # every layer of a step sees the same KV lengths: layers after the first reuse the work plan, and the
+        # caches were all written before the step began
+        later = S.ATTN_REUSE_PLAN | S.ATTN_CACHE_SETTLED
         if self.paged:
             return S.tree_attn_paged(self.Q[layer], self.Kp[layer], self.Vp[layer], self.page_table, self.page_indptr,
                                      self.kv_len, self.kv_len_host, self.Kt[layer], self.Vt[layer], self.parent,
                                      workspace=self.ws_attn, out=self.O[layer],
-                                     flags=S.ATTN_REUSE_PLAN if layer > 0 else 0)
+                                     flags=later if layer > 0 else 0)
         return S.tree_attn(self.Q[layer], self.Kc[layer], self.Vc[layer], self.kv_indptr, self.kv_indptr_host,
                            self.Kt[layer], self.Vt[layer], self.parent, workspace=self.ws_attn,
-                           out=self.O[layer], flags=S.ATTN_REUSE_PLAN if layer > 0 else 0)
+                           out=self.O[layer], flags=later if layer > 0 else 0)
 
     def commit(self, kv_len_out=None, status=None):
         """Appends the committed paths of the last verification to every layer's paged cache (the workload's

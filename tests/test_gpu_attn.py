@@ -147,6 +147,36 @@ def test_scale_argument_and_topology_errors():
         S.tree_attn(*args, bad)
 
 
+def test_layers_back_to_back_with_early_cache_loads():
+    # the layers of a step launched without a pause, every cache written beforehand: layers after the first
+    # may start loading their cache while the layer before is still finishing; each must match the oracle
+    if FLAGS["v"] != 0:
+        pytest.skip("a feature of the tcgen05 kernel")
+    w = I.scaled(I.WORKLOADS["qwen7b"], B=9, N=32)
+    lengths = np.array([2100, 64, 700, 129, 3300, 1, 0, 257, 1500], np.int32)
+    ip = np.zeros(w.B + 1, np.int32)
+    np.cumsum(lengths, out=ip[1:])
+    layers, want, args = 6, [], []
+    for layer in range(layers):
+        x = I.attn_inputs(w, layer=layer)
+        g = I.rng(950 + layer)
+        Kc = I.f32_to_bf16_bits(g.standard_normal((int(ip[-1]), w.Hkv, w.D), dtype=np.float32))
+        Vc = I.f32_to_bf16_bits(g.standard_normal((int(ip[-1]), w.Hkv, w.D), dtype=np.float32))
+        want.append(ref.tree_attn(x["Q"], Kc, Vc, ip, x["Kt"], x["Vt"], x["parent"])["O64"])
+        args.append((dev_bf16(x["Q"]), dev_bf16(Kc), dev_bf16(Vc), dev(ip), ip, dev_bf16(x["Kt"]), dev_bf16(x["Vt"]),
+                     x["parent"]))
+    ws = torch.empty(S.tree_attn_workspace_bytes(w.B, w.N, w.Hq, w.Hkv, w.D, ip), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    for rep in range(3):
+        outs = [S.tree_attn(*args[layer], workspace=ws,
+                            flags=(S.ATTN_REUSE_PLAN | S.ATTN_CACHE_SETTLED) if layer > 0 else 0)
+                for layer in range(layers)]
+        torch.cuda.synchronize()
+        for layer in range(layers):
+            diff = np.abs(host(outs[layer].float()) - want[layer])
+            assert (diff <= O_ATOL * np.maximum(1.0, np.abs(want[layer]))).all(), (rep, layer, diff.max())
+
+
 def test_plan_reuse_across_layers():
     # second call keeps the first call's work plan (same KV lengths, different tensors), as the layers of a
     # step do; results must still match the oracle, also for a third call
