@@ -788,6 +788,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         if (!ok) break;
                         const bool bad = !(ls0 + ls1 <= 256.0f) || m_pub != m_used;
                         if (!__any_sync(0xffffffffu, bad)) {
+                            // the reference stands: say so before storing P, the next tile's check waits for this
+                            mref[(t & 1u) * 128u + row] = m_used;
+                            mbar_arrive(bar(C::B_X + (int)(t & 1u)));
 #pragma unroll
                             for (int c = 0; c < 4; ++c) {
                                 uint32_t q[16];
@@ -797,8 +800,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                             }
                             tmem_st_wait();
                             l += ls0 + ls1;
-                            mref[(t & 1u) * 128u + row] = m_used;
-                            mbar_arrive(bar(C::B_X + (int)(t & 1u)));
                             done = true;
                         }
                     }
