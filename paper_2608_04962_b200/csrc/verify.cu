@@ -637,16 +637,25 @@ struct TermArgs {
 // Plain softmax masses of eight tokens; tokens below the nucleus threshold (thr = 0: none) weigh nothing.
 __device__ __forceinline__ void masses8(const uint4 &v, float M, float c, uint32_t thr, float (&e)[8]) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    if (thr == 0u) {  // (uniform over the CTA) no truncation: nothing to compare, a third of the instructions
+        const float nm = -M * c;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            e[2 * i] = ex2_approx(fmaf(__uint_as_float(w[i] << 16), c, nm));
+            e[2 * i + 1] = ex2_approx(fmaf(__uint_as_float(w[i] & 0xffff0000u), c, nm));
+        }
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const float e0 = ex2_approx((__uint_as_float(w[i] << 16) - M) * c);
-        const float e1 = ex2_approx((__uint_as_float(w[i] & 0xffff0000u) - M) * c);
+        const float e0 = ex2_approx(fmaf(__uint_as_float(w[i] << 16), c, -M * c));
+        const float e1 = ex2_approx(fmaf(__uint_as_float(w[i] & 0xffff0000u), c, -M * c));
         e[2 * i] = ord_key(w[i] & 0xffffu) >= thr ? e0 : 0.f;
         e[2 * i + 1] = ord_key(w[i] >> 16) >= thr ? e1 : 0.f;
     }
 }
 __device__ __forceinline__ float mass1(uint16_t bits, float M, float c, uint32_t thr) {
-    return ord_key(bits) >= thr ? ex2_approx((bf16_bits_to_float(bits) - M) * c) : 0.f;
+    return ord_key(bits) >= thr ? ex2_approx(fmaf(bf16_bits_to_float(bits), c, -M * c)) : 0.f;  // same form as masses8
 }
 
 __device__ __forceinline__ double warp_incl_scan(double v, int lane) {
@@ -705,11 +714,12 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
         for (int q = 0; q < 8; ++q) {
             float e[8];
             masses8(v[q], M, a.c, thr, e);
-            double acc = 0.0;
-#pragma unroll
-            for (int t = 0; t < 8; ++t) acc += (double)e[t];
+            // a slice's 256 masses are added pairwise in fp32 (relative error of a few 2^-24, the size of the
+            // exponentials' own error); everything above a slice is fp64.  (Converting every mass to fp64 first
+            // kept the conversion pipe busy for as long as the exponentials.)
+            float acc = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
             acc = warp_sum(acc);
-            if (lane == 0 && s0 + q < n_sl) sh_slice[warp * n_sl + s0 + q] = acc;
+            if (lane == 0 && s0 + q < n_sl) sh_slice[warp * n_sl + s0 + q] = (double)acc;
         }
     }
     __syncthreads();
