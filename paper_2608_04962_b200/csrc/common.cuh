@@ -69,13 +69,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// 2^x for two packed bf16 arguments at once (result packed bf16).
-__device__ __forceinline__ uint32_t ex2_bf16x2(uint32_t x) {
-    uint32_t y;
-    asm("ex2.approx.ftz.bf16x2 %0, %1;" : "=r"(y) : "r"(x));
-    return y;
-}
-
 // 16-byte streaming load that does not pollute L1.
 __device__ __forceinline__ uint4 ld_nc_v4(const void *p) {
     uint4 v;
