@@ -72,6 +72,8 @@ def test_attention_plan_is_host_only_and_consistent(libpath):
         first = S.tree_attn_launches(w.B, w.N, w.Hq, w.Hkv, w.D, ip)
         later = S.tree_attn_launches(w.B, w.N, w.Hq, w.Hkv, w.D, ip, flags=S.ATTN_REUSE_PLAN)
         assert first == later + 1 and later in (1, 2)                            # plan kernel only the first time
+        # the scheduling hint about the cache changes nothing that is counted
+        assert S.tree_attn_launches(w.B, w.N, w.Hq, w.Hkv, w.D, ip, flags=S.ATTN_REUSE_PLAN | S.ATTN_CACHE_SETTLED) == later
     # a changed length changes the plan's key: no stale answer
     ip2 = ip.copy()
     ip2[-1] += 4096
