@@ -226,14 +226,20 @@ feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restr
     int32_t *out = top_id + (size_t)r * kS;
     const int n_sel = min(kS, V);
     if (tid == 0) sh_n = 0;
-    // ---- pass 1: the largest key of this thread's share
-    uint32_t best = 0u;
-    for (int i = tid; i < nvec; i += TOPK_THREADS) {
+    // ---- pass 1: the largest key of this thread's share.  The order of the keys is the order of the values (with
+    //      -0 = +0), so the maximum is taken on the bf16 pairs as they come, one instruction per two logits, and
+    //      turned into a key once.
+    auto as_bf162 = [](uint32_t w_) { return *reinterpret_cast<const __nv_bfloat162 *>(&w_); };
+    __nv_bfloat162 mx2 = as_bf162(0xff80ff80u);  // (-inf, -inf)
+    for (int i = tid; i < nvec; i += 2 * TOPK_THREADS) {
         const uint4 v = ld_nc_v4(p + i);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int t = 0; t < 8; ++t) best = max(best, ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu)));
+        const int i1 = i + TOPK_THREADS;
+        const uint4 v1 = i1 < nvec ? ld_nc_v4(p + i1) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+        mx2 = __hmax2(__hmax2(__hmax2(as_bf162(v.x), as_bf162(v.y)), __hmax2(as_bf162(v.z), as_bf162(v.w))), mx2);
+        mx2 = __hmax2(__hmax2(__hmax2(as_bf162(v1.x), as_bf162(v1.y)), __hmax2(as_bf162(v1.z), as_bf162(v1.w))), mx2);
     }
+    const uint32_t mxb = *reinterpret_cast<const uint32_t *>(&mx2);
+    const uint32_t best = max(ord_key16(mxb & 0xffffu), ord_key16(mxb >> 16));
     sm.list.best[tid] = best;
     __syncthreads();
     {
@@ -247,14 +253,21 @@ feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restr
     }
     __syncthreads();
     const uint32_t bound = sh_bound;
-    // ---- pass 2: everything at or above the bound
+    // ---- pass 2: everything at or above the bound.  Compared as values, two at a time, against the bound's
+    //      value; a vector of eight with nothing to keep (nearly all of them) costs four compares and one branch.
+    const uint32_t bbits = (bound & 0x8000u) ? (bound & 0x7fffu) : (~bound & 0xffffu);  // the key undone
+    const __nv_bfloat162 bnd2 = as_bf162(bbits | (bbits << 16));
     for (int i = tid; i < nvec; i += TOPK_THREADS) {
         const uint4 v = ld_nc_v4(p + i);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t m[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m[j] = __hge2_mask(as_bf162(w[j]), bnd2);
+        if ((m[0] | m[1] | m[2] | m[3]) == 0u) continue;
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
-            const uint32_t key = ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
-            if (key >= bound) {
+            if ((m[t >> 1] >> (16 * (t & 1))) & 0xffffu) {
+                const uint32_t key = ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
                 const int pos = atomicAdd(&sh_n, 1);
                 if (pos < TOPK_LIST_CAP) {
                     sm.list.key[pos] = key;
