@@ -646,12 +646,18 @@ __device__ __forceinline__ void masses8(const uint4 &v, float M, float c, uint32
         }
         return;
     }
+    // the order of the keys is the order of the values (-0 = +0): compare two logits at a time with the
+    // threshold's value
+    const uint32_t tb = (thr & 0x8000u) ? (thr & 0x7fffu) : (~thr & 0xffffu);  // the key undone
+    const uint32_t tb2 = tb | (tb << 16);
+    const __nv_bfloat162 t2 = *reinterpret_cast<const __nv_bfloat162 *>(&tb2);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const float e0 = ex2_approx(fmaf(__uint_as_float(w[i] << 16), c, -M * c));
         const float e1 = ex2_approx(fmaf(__uint_as_float(w[i] & 0xffff0000u), c, -M * c));
-        e[2 * i] = ord_key(w[i] & 0xffffu) >= thr ? e0 : 0.f;
-        e[2 * i + 1] = ord_key(w[i] >> 16) >= thr ? e1 : 0.f;
+        const uint32_t keep = __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&w[i]), t2);
+        e[2 * i] = (keep & 0xffffu) ? e0 : 0.f;
+        e[2 * i + 1] = (keep >> 16) ? e1 : 0.f;
     }
 }
 __device__ __forceinline__ float mass1(uint16_t bits, float M, float c, uint32_t thr) {
