@@ -34,7 +34,9 @@ def _bits(t):
 @pytest.mark.parametrize("name,n_random", [("qwen1.5b", 3), ("qwen7b", 1), ("qwen14b", 1), ("sweep7b_B8", 1)])
 def test_full_size_step_sampled_against_the_oracle(name, n_random):
     w = I.WORKLOADS[name]
-    wl = StepWorkload(w, torch.device("cuda", 0), layers=1)
+    # three layers: the later ones keep the first one's plan and may load their first cache tiles while the layer
+    # before is still finishing, as all but the first layer of the benchmark's step do
+    wl = StepWorkload(w, torch.device("cuda", 0), layers=3)
     wl.step()
     torch.cuda.synchronize()
     assert S.workspace_status(wl.ws_attn) == 0 and S.workspace_status(wl.ws_propose) == 0
@@ -52,6 +54,20 @@ def test_full_size_step_sampled_against_the_oracle(name, n_random):
     got = wl.O[0][idx].float().cpu().numpy().astype(np.float64)
     err = np.abs(got - o["O64"]).max()
     assert err <= 1e-2, (name, err)
+    # ... and the last layer, on fewer sequences (the oracle's time)
+    few = picks[:3]
+    lens = np.array([ip[b + 1] - ip[b] for b in few], np.int32)
+    sub_ip = np.zeros(len(few) + 1, np.int32)
+    np.cumsum(lens, out=sub_ip[1:])
+    last = wl.layers - 1
+    Kc = np.concatenate([_bits(wl.Kc[last][ip[b]:ip[b + 1]]) for b in few], 0)
+    Vc = np.concatenate([_bits(wl.Vc[last][ip[b]:ip[b + 1]]) for b in few], 0)
+    fidx = torch.tensor(few, device=wl.device)
+    o = ref.tree_attn(_bits(wl.Q[last][fidx]), Kc, Vc, sub_ip, _bits(wl.Kt[last][fidx]), _bits(wl.Vt[last][fidx]), wl.parent)
+    got = wl.O[last][fidx].float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - o["O64"]).max()
+    assert err <= 1e-2, (name, "last layer", err)
+    assert torch.isfinite(wl.O[last].float()).all()
 
     # ---- verification: the oracle on the sampled sequences' logits, with the GPU's own proposal as input
     p = {k: v[idx].cpu().numpy() for k, v in wl.prop.items()}
