@@ -775,7 +775,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     uint32_t x[32];
                     bool done = false;
                     if (j >= 2) {
-                        // ---- one pass against the reference as it stands; P stays in registers until the verdict
+                        // ---- one pass against the reference as it stands; P stays in registers until the check below
                         uint32_t pk[64];
                         const float mref_ = (m_used == -INFINITY) ? 0.f : m_used;
 #pragma unroll
