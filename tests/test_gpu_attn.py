@@ -177,6 +177,51 @@ def test_layers_back_to_back_with_early_cache_loads():
             assert (diff <= O_ATOL * np.maximum(1.0, np.abs(want[layer]))).all(), (rep, layer, diff.max())
 
 
+@pytest.mark.parametrize("seed", [11, 12])
+def test_random_shapes_and_lengths(seed):
+    # seeded random head counts, group sizes, head dimensions, tree sizes, batch sizes and length mixes
+    # (empty caches, a few long sequences among short ones), two layers launched back to back each
+    if FLAGS["v"] != 0:
+        pytest.skip("the legacy kernel has its own cases")
+    rs = np.random.RandomState(seed)
+    for case in range(6):
+        Hkv = int(rs.choice([1, 2, 4, 8]))
+        G = int(rs.choice([1, 2, 4, 5, 6, 7]))
+        D = int(rs.choice([64, 128]))
+        N = int(rs.choice([1, 2, 5, 8, 16, 24, 32, 48, 64]))
+        B = int(rs.choice([1, 2, 3, 7, 12]))
+        base = I.WORKLOADS["qwen7b"]
+        w = I.scaled(base, B=B, N=N, Hq=Hkv * G, Hkv=Hkv, D=D, K=min(base.K, max(1, N - 1)))
+        if rs.randint(2):
+            lengths = rs.randint(0, 600, size=B)
+        else:
+            lengths = np.where(rs.rand(B) < 0.3, rs.randint(1500, 4000, size=B), rs.randint(0, 200, size=B))
+        lengths = lengths.astype(np.int32)
+        ip = np.zeros(B + 1, np.int32)
+        np.cumsum(lengths, out=ip[1:])
+        want, args = [], []
+        for layer in range(2):
+            x = I.attn_inputs(w, layer=layer)
+            g = I.rng(7000 + 100 * seed + 13 * case + layer)
+            T = max(int(ip[-1]), 1)
+            Kc = I.f32_to_bf16_bits(g.standard_normal((T, Hkv, D), dtype=np.float32))[:int(ip[-1])]
+            Vc = I.f32_to_bf16_bits(g.standard_normal((T, Hkv, D), dtype=np.float32))[:int(ip[-1])]
+            want.append(ref.tree_attn(x["Q"], Kc, Vc, ip, x["Kt"], x["Vt"], x["parent"])["O64"])
+            args.append((dev_bf16(x["Q"]), dev_bf16(Kc), dev_bf16(Vc), dev(ip), ip, dev_bf16(x["Kt"]),
+                         dev_bf16(x["Vt"]), x["parent"]))
+        ws = torch.empty(S.tree_attn_workspace_bytes(B, N, Hkv * G, Hkv, D, ip), dtype=torch.uint8, device="cuda")
+        torch.cuda.synchronize()
+        outs = [S.tree_attn(*args[layer], workspace=ws,
+                            flags=(S.ATTN_REUSE_PLAN | S.ATTN_CACHE_SETTLED) if layer > 0 else 0)
+                for layer in range(2)]
+        torch.cuda.synchronize()
+        assert S.workspace_status(ws) == 0
+        for layer in range(2):
+            diff = np.abs(host(outs[layer].float()) - want[layer])
+            assert (diff <= O_ATOL * np.maximum(1.0, np.abs(want[layer]))).all(), \
+                (case, dict(B=B, N=N, Hkv=Hkv, G=G, D=D), layer, diff.max(), lengths.tolist())
+
+
 def test_plan_reuse_across_layers():
     # second call keeps the first call's work plan (same KV lengths, different tensors), as the layers of a
     # step do; results must still match the oracle, also for a third call
