@@ -21,7 +21,7 @@
 //   warps 3-10 softmax, in one of two forms (template flag TEAMS, chosen by the number of row blocks):
 //              one row block (HBM-bound): TWO threads per query row (warps w and w+4 own the same 32 TMEM
 //              lanes and take columns 0-63 / 64-127 of each S tile); the pair exchanges one value per tile
-//              through shared memory.  More row blocks (softmax-bound): two TEAMS of four warps, one thread
+//              through shared memory.  More row blocks (bound by the loop S -> softmax -> P V): two TEAMS of four warps, one thread
 //              per row, team (t mod 2) takes tile t, so that one team's loads, stores and barrier round trips
 //              run under the other team's exponentials; the row's reference maximum travels from team to
 //              team through shared memory.  After the first tile(s) of a unit a tile takes one pass: the
@@ -37,6 +37,9 @@
 // sequence leave fp32 partials in the workspace; the CTA that finishes a sequence's last chunk
 // (atomic ticket, nobody waits) merges them, unless the plan leaves that to a kernel of its own.
 // TMEM columns: O: [0, 128);  S/P buffer i: [128 + 128 i, +128).
+// The kernel is launched as a programmatic dependent of the kernel before it in the stream: its CTAs are set up
+// while that kernel's last CTAs finish, and (when the caller has said that cache and plan are older than that
+// kernel) the loading thread fetches its first cache tiles before the wait that precedes every other access.
 #include <math.h>
 #include <stdlib.h>
 
