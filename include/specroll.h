@@ -175,7 +175,9 @@ int specroll_tree_attn(const specroll_attn_desc *desc, const void *Q, const void
  * A layer's cache is a pool Kp,Vp[n_pages, SPECROLL_PAGE_TOKENS, Hkv, D] bf16.  Sequence b owns the
  * slots page_indptr[b] .. page_indptr[b+1]-1 of page_table (i32, device); slot i names the pool
  * page that holds its tokens [128 i, 128 i + 128).  kv_len[b] tokens are valid (device and host
- * copies with the same values); a sequence may own more pages than it fills.
+ * copies with the same values); a sequence may own more pages than it fills.  Rows of a sequence's last
+ * page beyond kv_len[b] are read and multiplied by a zero weight: they must hold finite values (any
+ * finite bit pattern; a pool that was zero-filled once, or only ever written by the commit below, does).
  *
  * specroll_tree_attn_paged computes exactly what specroll_tree_attn computes on the cache that the
  * table describes.  It needs the tcgen05 kernel: Hq/Hkv <= 128 and B <= 4096, no
