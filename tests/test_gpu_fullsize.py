@@ -31,7 +31,8 @@ def _bits(t):
     return S.bf16_bits(t)
 
 
-@pytest.mark.parametrize("name,n_random", [("qwen1.5b", 3), ("qwen7b", 1), ("qwen14b", 1), ("sweep7b_B8", 1)])
+@pytest.mark.parametrize("name,n_random", [("qwen1.5b", 3), ("qwen7b", 1), ("qwen14b", 1), ("sweep7b_B8", 1),
+                                           ("sweep7b_B64", 0), ("sweep7b_B256", 0)])
 def test_full_size_step_sampled_against_the_oracle(name, n_random):
     w = I.WORKLOADS[name]
     # three layers: the later ones keep the first one's plan and may load their first cache tiles while the layer
