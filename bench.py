@@ -120,11 +120,26 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------ CPU oracle legs
 
 
+def use_host_cores_under_a_launcher():
+    """torchrun exports OMP_NUM_THREADS=1 to its ranks unless the caller set it.  The CPU legs run on rank 0 alone
+    (the other ranks do no CPU work) and are meant to use the machine's host cores, as they do when bench.py is
+    started directly: give the OpenMP runtime the cores this process may run on."""
+    if "TORCHELASTIC_RUN_ID" not in os.environ or os.environ.get("OMP_NUM_THREADS") != "1":
+        return
+    try:
+        import ctypes
+        ctypes.CDLL("libgomp.so.1").omp_set_num_threads(len(os.sched_getaffinity(0)))
+    except OSError:
+        pass
+
+
 def oracle_sample_step(w, n_seq: int, layers: int):
     """One pass of the whole path by the CPU oracle over the first n_seq sequences of `w`.
     Returns (seconds, tokens processed, threads)."""
     from oracle import ref
     from paper_2608_04962_b200 import inputs as I
+    ref.lib()
+    use_host_cores_under_a_launcher()
     ws = I.scaled(w, B=n_seq)
     x = I.propose_inputs(ws)
     a = I.attn_inputs(ws)
