@@ -281,9 +281,20 @@ int plan_head(int R, int V, HeadPlan *p) {
     using namespace thtc;
     p->n_mblocks = (R + BM - 1) / BM;
     const int n_tiles = (V + BN - 1) / BN;
-    int want = p->n_mblocks > 0 ? 148 / p->n_mblocks : 1;
-    if (want < 1) want = 1;
-    if (want > n_tiles) want = n_tiles;
+    // Number of vocabulary ranges: the CTAs (row blocks x ranges) run in waves of one per SM; the estimate of a
+    // plan is waves x (tiles per range + half a tile for a CTA's set-up and drain), and the candidate with the
+    // lowest estimate wins (with 32 row blocks: 9 ranges in two full waves instead of 4 ranges on 128 SMs).
+    int want = 1;
+    double best = -1.0;
+    for (int g = 1; g <= n_tiles && g <= 148; ++g) {
+        const int tpg = (n_tiles + g - 1) / g, ng = (n_tiles + tpg - 1) / tpg;
+        const long long ctas = (long long)(p->n_mblocks > 0 ? p->n_mblocks : 1) * ng;
+        const double est = (double)((ctas + 147) / 148) * ((double)tpg + 0.5);
+        if (best < 0.0 || est < best - 1e-9) {
+            best = est;
+            want = g;
+        }
+    }
     p->tiles_per_group = (n_tiles + want - 1) / want;
     p->n_groups = (n_tiles + p->tiles_per_group - 1) / p->tiles_per_group;
     size_t o = 0;
