@@ -106,6 +106,24 @@ def test_full_size_step_sampled_against_the_oracle(name, n_random):
     assert np.array_equal(p["tree_tok"], d["tree_tok"])
     np.testing.assert_allclose(p["slot_q"], d["slot_q"], rtol=1e-5)
 
+    # ---- the same chain with nothing of the GPU's in the oracle's inputs: for the sampled sequences whose
+    #      candidate lists the oracle reproduces id for id (no ties at the cut), the oracle's own lists, its own
+    #      draw and its own verification must give the GPU's tokens
+    oid3, ol3 = oid.reshape(len(picks), w.K, w.k), ol.reshape(len(picks), w.K, w.k).astype(np.float32)
+    clean = [i for i in range(len(picks)) if np.array_equal(oid3[i], p["cand_id"][i])]
+    if clean:
+        ci = np.array(clean)
+        d2 = ref.tree_draw(wl.parent, wl.anchor[idx].cpu().numpy()[ci], oid3[ci], ol3[ci],
+                           wl.u_draw[idx].cpu().numpy()[ci], temperature=w.temperature)
+        ov2 = ref.verify(_bits(wl.logits[idx])[ci], wl.parent, d2["tree_tok"], d2["tree_cand"], oid3[ci], ol3[ci],
+                         wl.u_acc[idx].cpu().numpy()[ci], wl.u_fin[idx].cpu().numpy()[ci], temperature=w.temperature)
+        for j, i in enumerate(clean):
+            if not np.array_equal(d2["tree_tok"][j], p["tree_tok"][i]):
+                continue   # a draw decided within rounding of a uniform (the lists' logits differ in their last bits)
+            same = gv["n_acc"][i] == ov2["n_acc"][j] and np.array_equal(gv["out_tok"][i], ov2["out_tok"][j]) and \
+                np.array_equal(gv["path_node"][i], ov2["path_node"][j])
+            assert same or ov2["min_margin"][j] < 1e-4 or ov2["fin_margin"][j] < 1e-6, (name, picks[i], "oracle-only chain")
+
     # ---- properties that hold for every sequence of the full batch
     n_acc = wl.ver["n_acc"].cpu().numpy()
     path = wl.ver["path_node"].cpu().numpy()
