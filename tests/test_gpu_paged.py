@@ -62,6 +62,14 @@ def test_plan_reuse_with_a_paged_cache():
     a = _gpu_paged(x, Kp, Vp, pt, pi, kl, workspace=ws)
     b = _gpu_paged(x, Kp, Vp, pt, pi, kl, workspace=ws, flags=S.ATTN_REUSE_PLAN)
     assert torch.equal(a, b)
+    # back to back, with the first pages of a call fetched while the call before is finishing
+    outs = [S.tree_attn_paged(dev_bf16(x["Q"]), dev_bf16(Kp), dev_bf16(Vp), dev(pt), dev(pi), dev(kl), kl,
+                              dev_bf16(x["Kt"]), dev_bf16(x["Vt"]), x["parent"], workspace=ws,
+                              flags=S.ATTN_REUSE_PLAN | S.ATTN_CACHE_SETTLED) for _ in range(4)]
+    torch.cuda.synchronize()
+    assert S.workspace_status(ws) == 0
+    for o in outs:
+        assert torch.equal(a, o)
 
 
 def test_paged_needs_the_tcgen05_kernel():
