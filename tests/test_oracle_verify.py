@@ -190,6 +190,40 @@ def test_million_trials_marginal_joint_first_slot_and_sandwich():
     assert ((out["term_kind"] == 1) == np.isin(out["term_node"], [2, 3, 4])).all()
 
 
+def test_temperature_other_than_one_marginal_first_slot_and_continuation():
+    # Same tree and tables at T = 0.7 and T = 1.3.  The target of every node is softmax(l / T), and the
+    # proposal of the draw is the head softmax at the same T (App. B.1 Eq. "nodep" / "slotq"), so
+    # the emitted tokens must follow softmax(l / T) and the first-slot acceptance must be
+    # 1 - TV(softmax(l / T), q_{u,1}) (App. B.2 Eq. "nodeaccept").  A temperature applied to only one
+    # of the two, or applied as a product instead of a quotient, fails every assertion below.
+    parent = np.array([-1, 0, 0, 1, 1], np.int32)
+    node_logits, cand_id, cand_logit = _vocab8_tables(77)
+    node_logits = node_logits * 0.5 + 0.3                      # not normalised: log-probabilities would hide a slip at T = 1 only
+    n = 400_000
+    for T, seed in ((0.7, 5), (1.3, 6)):
+        out = _run(parent, node_logits, cand_id, cand_logit, n, seed=seed, T=T)
+        T32 = np.float64(np.float32(T))
+        P = softmax(_f64(_bits(node_logits)) / T32, axis=-1)
+        P1 = softmax(_f64(_bits(node_logits)), axis=-1)
+        assert np.abs(P[0] - P1[0]).max() > 0.02               # the two temperatures are told apart by the test
+        freq = np.bincount(out["out_tok"][:, 0], minlength=8) / n
+        assert _within(freq, P[0], n).all(), (T, freq, P[0])
+        assert not _within(freq, P1[0], n).all()
+        q1 = np.zeros(8)
+        q1[cand_id[0]] = softmax(cand_logit[0].astype(np.float64) / T32)
+        a1 = np.mean((out["n_acc"] >= 1) & (out["path_node"][:, 1] == 1))
+        assert _within(a1, 1 - 0.5 * np.abs(P[0] - q1).sum(), n), (T, a1)
+        # slot_q recorded by the draw is the head softmax at T over what the earlier sibling left
+        first = out["tree_cand"][:, 1].astype(int)
+        np.testing.assert_allclose(out["slot_q"][:, 1], q1[cand_id[0]][first], rtol=1e-5)
+        for c in (1, 2):
+            sel = (out["n_acc"] >= 1) & (out["path_node"][:, 1] == c)
+            m = int(sel.sum())
+            assert m > 2000
+            f2 = np.bincount(out["out_tok"][sel, 1], minlength=8) / m
+            assert _within(f2, P[c], m).all(), (T, c, f2, P[c])
+
+
 def test_single_candidate_closed_form():
     # k = 1: q is a point mass on y, so y is accepted w.p. p(y) and the fallback is p off y.
     g = I.rng(5)
