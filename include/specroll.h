@@ -124,7 +124,8 @@ int specroll_tree_draw(int32_t B, int32_t N, int32_t K, int32_t k, float tempera
  *
  * Shapes: Q[B,N,Hq,D] bf16; Kc,Vc[T_kv,Hkv,D] bf16, sequence b owning rows
  * kv_indptr[b] .. kv_indptr[b+1]-1; kv_indptr_dev/_host[B+1] i32 (same values; the host copy
- * sizes the launch so no device read-back is needed); Kt,Vt[B,N,Hkv,D] bf16.
+ * sizes the launch so no device read-back is needed); kv_indptr[0] must be 0 (Kc and Vc point at
+ * the first sequence's first token), else SPECROLL_EINVAL; Kt,Vt[B,N,Hkv,D] bf16.
  * Outputs: O[B,N,Hq,D] bf16; lse[B,N,Hq] fp32 or NULL (natural-log sum-exp of the scaled scores).
  * Limits: D == 64 or 128, Hq % Hkv == 0, N <= 64.
  */
@@ -148,9 +149,13 @@ typedef struct {
  * finishing; Q, the tree's K/V and the outputs are touched only after it has completed.  Without the
  * flag nothing is read before then.  (Scheduling only; results do not depend on it.) */
 #define SPECROLL_ATTN_CACHE_SETTLED 4
-/* (The tcgen05 attention kernel is always launched with programmatic stream serialization; it waits
- * for the kernel before it in the stream before it reads or writes anything, except as the flag above
- * allows.  SPECROLL_ATTN_PDL=0 in the environment makes it an ordinary launch, for comparison.) */
+/* The tcgen05 attention kernels are launched with programmatic stream serialization: their CTAs are
+ * set up while the kernel before them in the stream finishes, and they wait for that kernel before
+ * they read or write anything, except as the flag above allows.  This flag makes the launch an
+ * ordinary one (for comparison; results do not depend on it). */
+#define SPECROLL_ATTN_NO_PDL 8
+#define SPECROLL_ATTN_ALL_FLAGS \
+    (SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN | SPECROLL_ATTN_CACHE_SETTLED | SPECROLL_ATTN_NO_PDL)
 
 size_t specroll_tree_attn_workspace_bytes(const specroll_attn_desc *desc,
                                           const int32_t *kv_indptr_host);

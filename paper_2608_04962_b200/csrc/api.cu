@@ -3,6 +3,10 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
+#include <utility>
+#include <vector>
+
 #include "common.cuh"
 
 namespace specroll {
@@ -13,6 +17,30 @@ static thread_local char g_msg[256];
 int note_cuda_error(cudaError_t e) {
     g_last_cuda = e;
     return SPECROLL_ECUDA;
+}
+
+int device_setup(const void *kernel, int dynamic_smem_bytes, int *n_sm) {
+    constexpr int MAX_DEV = 64;
+    static std::mutex mu;
+    static std::vector<std::pair<const void *, int>> done;  // (kernel, device) pairs whose limit has been raised
+    static int sm_count[MAX_DEV];                           // 0 = not asked yet
+    int dev = 0;
+    SR_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(mu);
+    if (n_sm) {
+        if (dev < 0 || dev >= MAX_DEV) {
+            SR_CUDA_TRY(cudaDeviceGetAttribute(n_sm, cudaDevAttrMultiProcessorCount, dev));
+        } else {
+            if (sm_count[dev] == 0) SR_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+            *n_sm = sm_count[dev];
+        }
+    }
+    if (!kernel) return SPECROLL_OK;
+    for (const auto &e : done)
+        if (e.first == kernel && e.second == dev) return SPECROLL_OK;
+    SR_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dynamic_smem_bytes));
+    done.emplace_back(kernel, dev);
+    return SPECROLL_OK;
 }
 
 int build_topo(const int32_t *parent_host, int N, int K, int k, Topo *t, TopoMask *m) {

@@ -21,6 +21,11 @@ int note_cuda_error(cudaError_t e);
 
 #define SR_LAUNCH_CHECK() SR_CUDA_TRY(cudaGetLastError())
 
+// Raises a kernel's dynamic shared-memory limit the first time the kernel is launched on the current device
+// (the attribute is per device), and optionally returns that device's SM count.  Thread-safe; later calls for
+// the same (kernel, device) cost one table look-up.  Returns SPECROLL_OK or SPECROLL_ECUDA.
+int device_setup(const void *kernel, int dynamic_smem_bytes, int *n_sm);
+
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

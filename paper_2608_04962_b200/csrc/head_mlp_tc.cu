@@ -178,12 +178,7 @@ static int launch_bn(const CUtensorMap &tmW, const void *xhat, int KX, const voi
     CUtensorMap tmX;
     int rc = make_tmap_2d_bf16(&tmX, xhat, (uint64_t)KX * B, (uint64_t)d, (uint64_t)d, BN);
     if (rc != SPECROLL_OK) return rc;
-    static bool configured = false;
-    if (!configured) {
-        SR_CUDA_TRY(cudaFuncSetAttribute(head_mlp_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         C::SMEM_BYTES));
-        configured = true;
-    }
+    if ((rc = device_setup(reinterpret_cast<const void *>(head_mlp_tc_kernel<BN>), C::SMEM_BYTES, nullptr)) != SPECROLL_OK) return rc;
     const dim3 grid((unsigned)((d + BM - 1) / BM), (unsigned)((B + BN - 1) / BN), (unsigned)K);
     head_mlp_tc_kernel<BN><<<grid, THREADS, C::SMEM_BYTES, st>>>(
         tmW, tmX, KX, static_cast<const __nv_bfloat16 *>(bias), static_cast<const __nv_bfloat16 *>(h), z, B, K, d,

@@ -253,12 +253,7 @@ int launch_lm_head_tc(const void *Zt, const void *W, int M, int V, int d, int k,
     if (rc != SPECROLL_OK) return rc;
     rc = make_tmap_2d_bf16(&tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)d, BN);
     if (rc != SPECROLL_OK) return rc;
-    static bool configured = false;
-    if (!configured) {
-        SR_CUDA_TRY(cudaFuncSetAttribute(lm_head_topk_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         SMEM_BYTES));
-        configured = true;
-    }
+    if ((rc = device_setup(reinterpret_cast<const void *>(lm_head_topk_tc_kernel), SMEM_BYTES, nullptr)) != SPECROLL_OK) return rc;
     lm_head_topk_tc_kernel<<<n_mblocks * n_groups, THREADS, SMEM_BYTES, st>>>(tmA, tmB, M, V, d, k, n_mblocks,
                                                                              n_groups, tiles_per_group, pval, pid,
                                                                              status);

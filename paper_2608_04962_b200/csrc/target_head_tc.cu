@@ -338,11 +338,7 @@ extern "C" int specroll_target_head_stats(int32_t R, int32_t d, int32_t V, float
     if (rc != SPECROLL_OK) return rc;
     rc = make_tmap_2d_bf16(&tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)d, BN);
     if (rc != SPECROLL_OK) return rc;
-    static bool configured = false;
-    if (!configured) {
-        SR_CUDA_TRY(cudaFuncSetAttribute(target_head_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-        configured = true;
-    }
+    if ((rc = device_setup(reinterpret_cast<const void *>(target_head_tc_kernel<false>), SMEM_BYTES, nullptr)) != SPECROLL_OK) return rc;
     const float c_log2 = 1.4426950408889634f / temperature;
     target_head_tc_kernel<false><<<p.n_mblocks * p.n_groups, THREADS, SMEM_BYTES, st>>>(
         tmA, tmB, R, V, d, p.n_mblocks, p.n_groups, p.tiles_per_group, c_log2, want_id, kw, pm, ps,
@@ -369,11 +365,7 @@ extern "C" int specroll_target_head_rows(int32_t R, int32_t d, int32_t V, const 
     if (rc != SPECROLL_OK) return rc;
     rc = make_tmap_2d_bf16(&tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)d, BN);
     if (rc != SPECROLL_OK) return rc;
-    static bool configured = false;
-    if (!configured) {
-        SR_CUDA_TRY(cudaFuncSetAttribute(target_head_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-        configured = true;
-    }
+    if ((rc = device_setup(reinterpret_cast<const void *>(target_head_tc_kernel<true>), SMEM_BYTES, nullptr)) != SPECROLL_OK) return rc;
     target_head_tc_kernel<true><<<p.n_mblocks * p.n_groups, THREADS, SMEM_BYTES, st>>>(
         tmA, tmB, R, V, d, p.n_mblocks, p.n_groups, p.tiles_per_group, 0.f, nullptr, 0, nullptr, nullptr, nullptr,
         static_cast<uint16_t *>(logits), status);

@@ -497,7 +497,7 @@ struct AttnPlan {
 
 static int compute_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_host, AttnPlan *p) {
     if (!d || !indptr_host || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->Hq < 1 || d->Hkv < 1 ||
-        (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || (d->flags & ~(SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN | SPECROLL_ATTN_CACHE_SETTLED)) != 0 ||
+        (d->Hq % d->Hkv) || (d->D != 64 && d->D != 128) || (d->flags & ~SPECROLL_ATTN_ALL_FLAGS) != 0 ||
         !(d->scale > 0.f))
         return SPECROLL_EINVAL;
     const int G = d->Hq / d->Hkv;
@@ -578,7 +578,7 @@ static int compute_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_
     // A sequence cut into many chunks is merged by a kernel of its own, over the whole GPU; with few chunks the
     // CTA that finishes a sequence's last chunk merges them while the others keep streaming.
     p->merge_mode = (p->use_tc && (max_tiles + p->chunk_tiles - 1) / p->chunk_tiles >= 5) ? 2 : 0;
-    p->n_counters = 64 + d->B * d->Hkv * p->n_rb;  // [0]: work counter; [64 ...]: per (b, hkv, rb) arrivals
+    p->n_counters = 64 + d->B * d->Hkv * p->n_rb;  // [0]: work counter, [1]: CTAs that have left; [64 ...]: per (b, hkv, rb) arrivals
     size_t o = 0;
     p->off_status = o;
     o += 256;
@@ -632,7 +632,7 @@ static int make_attn_plan(const specroll_attn_desc *d, const int32_t *indptr_hos
     static unsigned next = 0;
     if (!d || !indptr_host || d->B < 0 || d->B > (1 << 24)) return compute_attn_plan(d, indptr_host, p);
     // what the key leaves out is checked here, so that a remembered plan never answers for an invalid call
-    if ((d->flags & ~(SPECROLL_ATTN_LEGACY_MMA | SPECROLL_ATTN_REUSE_PLAN | SPECROLL_ATTN_CACHE_SETTLED)) != 0 || !(d->scale > 0.f)) return SPECROLL_EINVAL;
+    if ((d->flags & ~SPECROLL_ATTN_ALL_FLAGS) != 0 || !(d->scale > 0.f)) return SPECROLL_EINVAL;
     const int key[7] = {d->B, d->N, d->Hq, d->Hkv, d->D, (int)(d->flags & SPECROLL_ATTN_LEGACY_MMA), 1};
     const size_t n = (size_t)d->B + 1;
     std::lock_guard<std::mutex> lock(mu);
@@ -731,6 +731,7 @@ static int run_tree_attn(const specroll_attn_desc *d, const void *Q, const void 
     a.total_work = p.items * d->Hkv * p.n_rb;
     a.merge_mode = p.merge_mode;
     a.nodes_per_block = p.nodes_per_block;
+    a.no_pdl = (d->flags & SPECROLL_ATTN_NO_PDL) ? 1 : 0;
     // early cache loads need a plan that is not being made by the kernel just before the attention kernel
     a.early_cache = ((d->flags & SPECROLL_ATTN_CACHE_SETTLED) && (d->flags & SPECROLL_ATTN_REUSE_PLAN)) ? 1 : 0;
     if (!(p.use_tc && (d->flags & SPECROLL_ATTN_REUSE_PLAN))) {
@@ -756,8 +757,9 @@ extern "C" int specroll_tree_attn(const specroll_attn_desc *d, const void *Q, co
                                   const int32_t *kv_indptr_dev, const int32_t *kv_indptr_host, const void *Kt,
                                   const void *Vt, const int32_t *parent_host, void *O, float *lse,
                                   void *workspace, size_t workspace_bytes, void *cuda_stream) {
-    if (!d || !kv_indptr_host || d->B < 0) return SPECROLL_EINVAL;
-    const long long T_kv = (long long)kv_indptr_host[d->B] - kv_indptr_host[0];
+    // the cache tensors start at the first sequence's first token: token coordinates count from their base
+    if (!d || !kv_indptr_host || d->B < 0 || kv_indptr_host[0] != 0) return SPECROLL_EINVAL;
+    const long long T_kv = (long long)kv_indptr_host[d->B];
     return run_tree_attn(d, Q, Kc, Vc, T_kv, kv_indptr_dev, nullptr, nullptr, nullptr, kv_indptr_host, Kt, Vt,
                          parent_host, O, lse, workspace, workspace_bytes, cuda_stream);
 }

@@ -30,6 +30,7 @@ struct AttnArgs {
     int early_cache;              // plan, cache and page table were complete before the preceding kernel was launched
     float *hand;                  // [ATTN_HAND_CTAS][4][128] per-CTA hand-over area between two groups of warps of the tcgen05 kernel
     int32_t merge_mode;           // chunks of a split sequence are merged 0: by the CTA that finishes last; 2: by a later kernel
+    int32_t no_pdl;               // launch the attention kernel as an ordinary kernel, not as a programmatic dependent
 };
 
 constexpr int ATTN_HAND_CTAS = 256;  // CTAs the hand-over area is sized for (the grid is one CTA per SM)

@@ -41,38 +41,11 @@
 // while that kernel's last CTAs finish, and (when the caller has said that cache and plan are older than that
 // kernel) the loading thread fetches its first cache tiles before the wait that precedes every other access.
 #include <math.h>
-#include <stdlib.h>
 
 #include "tc05.cuh"
 #include "tree_attn.cuh"
 
 namespace specroll {
-
-// Optional instrumentation, off in normal builds.
-//   -DSPECROLL_TRACE: one thread per role adds up the SM cycles it spends in each kind of barrier wait (all CTAs).
-//   -DSPECROLL_TRACE_EVENTS (with the above): CTA 0 also records (event, index, SM clock) per role; each record
-//   costs a round trip to global memory, so the timeline it gives is stretched.
-#ifdef SPECROLL_TRACE
-__device__ unsigned long long g_trace[4][8192];
-__device__ unsigned int g_trace_n[4];
-__device__ unsigned long long g_prof[5][12];
-__device__ unsigned long long g_cta_ns[8][2][160];  // per launch (mod 8): start and end of each CTA (global timer)
-__device__ unsigned int g_launch_n;
-#endif
-#if defined(SPECROLL_TRACE) && defined(SPECROLL_TRACE_EVENTS)
-#define SR_TRACE(role, ev, idx)                                                                       \
-    do {                                                                                              \
-        if (blockIdx.x == 0) {                                                                        \
-            const unsigned n_ = g_trace_n[role]++;                                                    \
-            if (n_ < 4096) {                                                                          \
-                g_trace[role][2 * n_] = ((unsigned long long)(ev) << 32) | (unsigned)(idx);           \
-                g_trace[role][2 * n_ + 1] = (unsigned long long)clock64();                            \
-            }                                                                                         \
-        }                                                                                             \
-    } while (0)
-#else
-#define SR_TRACE(role, ev, idx)
-#endif
 
 namespace attc {
 constexpr int BN = 128;  // KV tokens per tile
@@ -187,20 +160,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int N = a.N, G = a.G;
-#ifdef SPECROLL_TRACE
-    unsigned long long prof[12] = {0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull};
-    const long long prof_t0 = clock64();
-    const unsigned launch_slot = *(volatile unsigned int *)&g_launch_n & 7u;
-    if (threadIdx.x == 0 && blockIdx.x < 160) g_cta_ns[launch_slot][0][blockIdx.x] = globaltimer_ns();
-    auto twait = [&](int slot, uint32_t b_, uint32_t par_) {
-        const long long t_ = clock64();
-        const bool r_ = mbar_wait(b_, par_, abort_flag);
-        prof[slot] += (unsigned long long)(clock64() - t_);
-        return r_;
-    };
-#else
     auto twait = [&](int, uint32_t b_, uint32_t par_) { return mbar_wait(b_, par_, abort_flag); };
-#endif
     // Ring stage and phase of tile t's K and V (t counts tiles over all units of this CTA): in load order
     // K0 K1 K2 V0 K3 V1 K4 V2 ... K(t) is load number 2t - 2 (t for the first two) and V(t) load number 2t + 3.
     auto k_slot = [&](uint32_t t, int &st, uint32_t &ph) {
@@ -381,7 +341,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 d->item = item0 + split;
                 d->item0 = item0;
                 mbar_arrive(bar(C::B_UFULL + slot));  // release: the descriptor is visible to whoever acquires
-                SR_TRACE(0, 0, u);
                 // ---- the unit's Q block, into the buffer whose unit (two back) has had every S computed
                 const int qb = (int)(u % QS);
                 if (u >= (uint32_t)QS && !twait(2, bar(C::B_QFREE + qb), (u / QS - 1u) & 1u)) {
@@ -432,7 +391,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     for (int bx = 0; bx < C::NBOX; ++bx)
                         tma_load_3d(dst + bx * BOX_BYTES, mk, bx * 64, hkv, tok, bar(C::B_FULL + s));
                     ++kt;
-                    SR_TRACE(0, 1, kt);
                     if (n_pend == 2) {
                         ok = load_v(pv_map[0], pv_h[0], pv_tok[0]);
                         pv_map[0] = pv_map[1];
@@ -525,7 +483,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         }
                         umma_commit(bar(C::B_SFULL + sb));
                         umma_commit(bar(C::B_EMPTY + ks));  // the stage is free once this S has been computed
-                        SR_TRACE(1, 1, ts);
                     }
                     umma_commit(bar(C::B_QFREE + qb));  // every S of the unit computed: its Q buffer may be replaced
                 }
@@ -563,7 +520,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         }
                         umma_commit(bar(C::B_EMPTY + vs));
                         umma_commit(bar(C::B_PVDONE + sb));
-                        SR_TRACE(1, 3, tp);
                     }
                     if (ok) umma_commit(bar(C::B_OFULL));  // the unit's accumulator is complete when this arrives
                 }
@@ -607,7 +563,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            if (lane == 0 && lg == 2) SR_TRACE(3, 3, u);
             const uint32_t o_t = t_lane + C::O_COL;
             const int n = row_ok ? gr / G : 0, g = row_ok ? gr % G : 0;
             const bool direct = (n_splits == 1);
@@ -670,7 +625,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     merge_rows(b, hkv, rb, n_splits, item0, row, 0, D);
                 }
             }
-            if (lane == 0 && lg == 2) SR_TRACE(3, 4, u);
         }
     } else {
         if constexpr (TEAMS) {
@@ -714,7 +668,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
-                    if (ws == 0 && lane == 0) SR_TRACE(2, 1, t);
                     const uint32_t s_t = t_lane + C::S_COL + 128u * (uint32_t)sb;
                     const bool tree = has_tree && (j == n_it - 1);
                     // columns >= limit are outside the sequence (a tree tile has at most 64 rows of tree K/V)
@@ -878,13 +831,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                     tc_fence_before();
                     mbar_arrive(bar(C::B_PREADY + sb));
-                    if (ws == 0 && lane == 0) SR_TRACE(2, 2, t);
                 }
                 if (!ok) break;
                 // ---- end of the unit: each team leaves its share of the sum and the reference it is relative to for
                 //      the output warps and goes on with the next unit.  Those wait for the unit's last P V themselves.
                 gt += (uint32_t)n_it;
-                if (ws == 0 && lane == 0) SR_TRACE(2, 3, u);
                 ok = twait(3, bar(C::B_HFREE), (u & 1u) ^ 1u);  // the values of the unit before have been taken
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -928,7 +879,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
-                    if (ws == 0 && lane == 0) SR_TRACE(2, 1, t);
                     const uint32_t s_t = t_lane + C::S_COL + 128u * (uint32_t)sb;
                     const bool tree = has_tree && (j == n_it - 1);
                     // columns >= limit are outside the sequence; this thread's columns start at 64 * half
@@ -966,13 +916,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         const unsigned short mine = bf16_bits_rn(fmaxf(mx0, mx1));
                         const int px = (int)(use_pair & 1u) * 64;
                         xm[px + half * 32 + lane] = mine;
-#ifdef SPECROLL_TRACE
-                        const long long tps_ = clock64();
-#endif
                         bool k_ = group_sync(pair_bar, use_pair, abort_flag);
-#ifdef SPECROLL_TRACE
-                        prof[4] += (unsigned long long)(clock64() - tps_);
-#endif
                         k_ = __all_sync(0xffffffffu, k_);
                         mt = fmaxf(bf16_bits_to_float(mine), bf16_bits_to_float(xm[px + (half ^ 1) * 32 + lane])) * sc;
                         return k_;
@@ -1096,13 +1040,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                     tc_fence_before();
                     mbar_arrive(bar(C::B_PREADY + sb));
-                    if (ws == 0 && lane == 0) SR_TRACE(2, 2, t);
                 }
                 if (!ok) break;
                 // ---- hand the row's reference maximum and this thread's share of its sum to the output warps
                 //      and go on with the next unit; they wait for the unit's last P V themselves
                 gt += (uint32_t)n_it;
-                if (ws == 0 && lane == 0) SR_TRACE(2, 3, u);
                 ok = twait(3, bar(C::B_HFREE), (u & 1u) ^ 1u);  // the values of the unit before have been taken
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -1114,14 +1056,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
 
     // ------------------------------------------------------------------ teardown
-#ifdef SPECROLL_TRACE
-    if (lane == 0 && (warp <= 3 || warp == 1 + C::MMA_WARPS + C::SOFTMAX_THREADS / 32)) {
-        const int role = warp <= 1 ? warp : (warp == 2 ? 4 : (warp == 3 ? 2 : 3));  // 0 producer, 1 / 4 MMA, 2 softmax, 3 output
-        if (warp == 0 && blockIdx.x < 160) g_cta_ns[launch_slot][1][blockIdx.x] = globaltimer_ns();
-        prof[11] = (unsigned long long)(clock64() - prof_t0);
-        for (int i = 0; i < 12; ++i) atomicAdd(&g_prof[role][i], prof[i]);
-    }
-#endif
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -1146,9 +1080,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (threadIdx.x == 0) {
             a.work_counter[0] = 0;
             a.work_counter[1] = 0;
-#ifdef SPECROLL_TRACE
-            g_launch_n = g_launch_n + 1u;
-#endif
         }
     }
 }
@@ -1169,22 +1100,13 @@ static int launch_tc(const AttnArgs &a, const TopoMask &mask, long long T_kv, in
     if ((rc = make_tmap_3d_bf16(&tmV, vc, D, a.Hkv, cache_rows, 1, attc::BN)) != SPECROLL_OK) return rc;
     if ((rc = make_tmap_3d_bf16(&tmKt, a.Kt, D, a.Hkv, tree_rows, 1, attc::BN)) != SPECROLL_OK) return rc;
     if ((rc = make_tmap_3d_bf16(&tmVt, a.Vt, D, a.Hkv, tree_rows, 1, attc::BN)) != SPECROLL_OK) return rc;
-    static int n_sm = 0;
-    if (n_sm == 0) {
-        int dev = 0;
-        SR_CUDA_TRY(cudaGetDevice(&dev));
-        SR_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-        SR_CUDA_TRY(cudaFuncSetAttribute(tree_attn_tc_kernel<D, TEAMS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
-    }
+    int n_sm = 0;
+    if ((rc = device_setup(reinterpret_cast<const void *>(tree_attn_tc_kernel<D, TEAMS>), C::SMEM, &n_sm)) != SPECROLL_OK) return rc;
     const int ctas = n_sm < ATTN_HAND_CTAS ? n_sm : ATTN_HAND_CTAS;  // every CTA has a hand-over area of its own
     const unsigned grid = (unsigned)(a.total_work < ctas ? a.total_work : ctas);
     // Programmatic stream serialization: the CTAs may be set up (barriers, tensor memory, zeroed Q buffers) while
     // the kernel before this one in the stream is still running its last CTAs; the kernel itself waits for
     // that kernel's completion before it reads anything (griddepcontrol.wait).
-    static const bool pdl = []() {
-        const char *e = getenv("SPECROLL_ATTN_PDL");
-        return !(e && e[0] == '0');
-    }();
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(C::THREADS);
@@ -1194,7 +1116,7 @@ static int launch_tc(const AttnArgs &a, const TopoMask &mask, long long T_kv, in
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
+    cfg.numAttrs = a.no_pdl ? 0 : 1;
     SR_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel<D, TEAMS>, tmQ, tmK, tmV, tmKt, tmVt, a, mask, status));
     SR_LAUNCH_CHECK();
     return SPECROLL_OK;
@@ -1265,25 +1187,6 @@ int launch_attn_merge_tc(const AttnArgs &a, int D, int items, cudaStream_t st) {
     return SPECROLL_OK;
 }
 
-#ifdef SPECROLL_TRACE
-extern "C" int specroll_debug_prof_read(unsigned long long *dst) {  // 5 roles x 12 counters; clears them
-    if (cudaMemcpyFromSymbol(dst, g_prof, sizeof(unsigned long long) * 60) != cudaSuccess) return 4;
-    unsigned long long z[60] = {0};
-    return cudaMemcpyToSymbol(g_prof, z, sizeof(z)) == cudaSuccess ? 0 : 4;
-}
-extern "C" int specroll_debug_cta_read(unsigned long long *dst, unsigned int *n_launches) {  // [8][2][160] times in ns
-    if (cudaMemcpyFromSymbol(n_launches, g_launch_n, 4) != cudaSuccess) return 4;
-    return cudaMemcpyFromSymbol(dst, g_cta_ns, sizeof(unsigned long long) * 8 * 2 * 160) == cudaSuccess ? 0 : 4;
-}
-extern "C" int specroll_debug_trace_reset(void) {
-    unsigned int z[4] = {0, 0, 0, 0};
-    return cudaMemcpyToSymbol(g_trace_n, z, sizeof(z)) == cudaSuccess ? 0 : 4;
-}
-extern "C" int specroll_debug_trace_read(unsigned long long *dst, unsigned int *counts) {
-    if (cudaMemcpyFromSymbol(counts, g_trace_n, 16) != cudaSuccess) return 4;
-    return cudaMemcpyFromSymbol(dst, g_trace, sizeof(unsigned long long) * 4 * 8192) == cudaSuccess ? 0 : 4;
-}
-#endif
 
 int launch_attn_tc(const AttnArgs &a, const TopoMask &mask, int D, long long T_kv, int32_t *status, cudaStream_t st) {
     // One row block per (sequence, KV head): the kernel is bound by HBM and the softmax with two threads per row

@@ -976,14 +976,10 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
     wa.V = d->V;
     wa.T = (double)d->temperature;
     if (truncate) {
-        static bool configured = false;
-        if (!configured) {
-            SR_CUDA_TRY(cudaFuncSetAttribute(walk_cta_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)sizeof(NucleusSmem)));
-            SR_CUDA_TRY(cudaFuncSetAttribute(walk_cta_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)sizeof(NucleusSmem)));
-            configured = true;
-        }
+        int rc_ = device_setup(reinterpret_cast<const void *>(walk_cta_kernel<false, true>), (int)sizeof(NucleusSmem), nullptr);
+        if (rc_ == SPECROLL_OK)
+            rc_ = device_setup(reinterpret_cast<const void *>(walk_cta_kernel<true, true>), (int)sizeof(NucleusSmem), nullptr);
+        if (rc_ != SPECROLL_OK) return rc_;
         if (lazy)
             walk_cta_kernel<true, true><<<d->B, NUC_THREADS, sizeof(NucleusSmem), st>>>(
                 wa, topo, c, top_p, row_max, row_sum, thr_key, keep_sum, nucleus_thr, nucleus_sum);
