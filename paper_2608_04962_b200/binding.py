@@ -36,6 +36,7 @@ PROPOSE_LEGACY_MMA = 1
 ATTN_LEGACY_MMA = 1
 ATTN_REUSE_PLAN = 2
 ATTN_CACHE_SETTLED = 4
+ATTN_NO_PDL = 8
 VERIFY_LAZY_STATS = 1
 FEEDBACK_SEVERITY = 1
 PAGE_TOKENS = 128

@@ -289,23 +289,26 @@ tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__rest
     slot_q[(size_t)b * N] = 1.0f;
     for (int n = 1; n < N; ++n) {
         const int u = topo.parent[n], hd = topo.depth[n] - 1;
-        double *w = sh_w[warp][hd];
+        const double *w = sh_w[warp][hd];
+        double w_left[SPECROLL_MAX_TOPK];  // used on the rare path below only
         const unsigned long long taken = sh_taken[warp][u];
         double s = 0.0;
         for (int j = 0; j < k; ++j)
             if (!((taken >> j) & 1ull)) s += w[j];
         if (!(s > 0.0)) {
             // every remaining weight underflowed against a taken candidate's logit: take the reference among
-            // the remaining ones instead (from here on this head's weights are relative to it)
+            // the remaining ones instead.  The head's table is shared by all parents of this depth, whose taken
+            // sets differ, so the weights of this one draw go into an array of their own.
             const float *cl = cand_logit + ((size_t)b * K + hd) * k;
             float mxf = -INFINITY;
             for (int j = 0; j < k; ++j)
                 if (!((taken >> j) & 1ull)) mxf = fmaxf(mxf, cl[j]);
             s = 0.0;
             for (int j = 0; j < k; ++j) {
-                w[j] = ((taken >> j) & 1ull) ? 0.0 : exp(((double)cl[j] - (double)mxf) / T);
-                s += w[j];
+                w_left[j] = ((taken >> j) & 1ull) ? 0.0 : exp(((double)cl[j] - (double)mxf) / T);
+                s += w_left[j];
             }
+            w = w_left;
         }
         // first remaining candidate whose cumulative probability exceeds the uniform (compared as masses)
         const double thr = (double)u_draw[(size_t)b * N + n] * s;

@@ -80,3 +80,18 @@ def test_attention_plan_is_host_only_and_consistent(libpath):
     assert S.tree_attn_workspace_bytes(w.B, w.N, w.Hq, w.Hkv, w.D, ip2) != 0
     assert S.tree_attn_launches(w.B, w.N, w.Hq, w.Hkv, w.D, ip, flags=64) == -1  # unknown flag
     assert S.verify_nucleus_workspace_bytes(4, 8, 3, 2, 1024) > S.verify_workspace_bytes(4, 8, 3, 2, 1024)
+
+
+def test_cache_offsets_must_start_at_zero(libpath):
+    """Token coordinates count from the base of Kc / Vc: an offset table that starts elsewhere is refused on the
+    host, before anything is enqueued (no device needed)."""
+    import ctypes as C
+    from paper_2608_04962_b200 import binding as S
+    desc = S.AttnDesc(2, 8, 4, 2, 64, 0.125, 0)
+    ip = np.array([5, 100, 300], np.int32)
+    parent = np.array([-1, 0, 0, 1, 1, 2, 3, 3], np.int32)
+    null = C.c_void_p(0)
+    rc = S.lib().specroll_tree_attn(C.byref(desc), null, null, null, null, ip.ctypes.data_as(C.c_void_p), null, null,
+                                    parent.ctypes.data_as(C.c_void_p), null, null, null, C.c_size_t(0), null)
+    assert rc == 1                                                                # SPECROLL_EINVAL
+    assert S.tree_attn_launches(2, 8, 4, 2, 64, np.array([0, 100, 300], np.int32), flags=S.ATTN_NO_PDL) >= 1

@@ -40,14 +40,20 @@ def run_both(w, x, lengths=None):
 
 
 def check(o, O, lse, edge=False):
-    """edge=False: the bar of the workloads (cache length >= 64, so |O| < 1): max abs <= 1e-2.
-    edge=True: degenerate caches (0 or 1 cached tokens) give |O| of several units, where the bf16
-    output spacing alone (2^-8 |O|) exceeds 1e-2; there the bound scales with max(1, |O|)."""
-    diff = np.abs(O - o["O64"])
-    if edge:
-        assert (diff <= O_ATOL * np.maximum(1.0, np.abs(o["O64"]))).all(), diff.max()
-    else:
-        assert diff.max() <= O_ATOL, diff.max()
+    """edge=False: the bar of the workloads everywhere: max abs <= 1e-2.
+    edge=True: the same bar for every element with |O| <= 1.  Where the softmax is concentrated on a few tokens
+    (degenerate caches of 0 or 1 tokens, scores that grow along the cache) |O| reaches several units and the
+    spacing of the bf16 output alone (2^-8 |O|) exceeds 1e-2; those elements, and only those, get the bound
+    scaled by |O|, and must in addition lie within one bf16 step of the oracle's rounded value."""
+    o64 = o["O64"]
+    diff = np.abs(O - o64)
+    big = (np.abs(o64) > 1.0) & edge
+    assert (diff[~big] <= O_ATOL).all(), diff[~big].max()
+    if big.any():
+        assert (diff[big] <= O_ATOL * np.abs(o64[big])).all(), (diff[big] / np.abs(o64[big])).max()
+        step = 2.0 ** (np.floor(np.log2(np.abs(o64[big]))) - 7)
+        rounded = I.bf16_bits_to_f32(I.f32_to_bf16_bits(o64[big].astype(np.float32))).astype(np.float64)
+        assert (np.abs(O[big] - rounded) <= step).all()
     err = diff.max()
     np.testing.assert_allclose(lse, o["lse"], atol=2e-3, rtol=0)
     return err

@@ -32,7 +32,8 @@ def _bits(t):
 
 
 @pytest.mark.parametrize("name,n_random", [("qwen1.5b", 3), ("qwen7b", 1), ("qwen14b", 1), ("sweep7b_B8", 1),
-                                           ("sweep7b_B64", 0), ("sweep7b_B256", 0)])
+                                           ("sweep7b_B16", 0), ("sweep7b_B32", 0), ("sweep7b_B64", 0),
+                                           ("sweep7b_B128", 0), ("sweep7b_B256", 0)])
 def test_full_size_step_sampled_against_the_oracle(name, n_random):
     w = I.WORKLOADS[name]
     # three layers: the later ones keep the first one's plan and may load their first cache tiles while the layer
@@ -97,10 +98,24 @@ def test_full_size_step_sampled_against_the_oracle(name, n_random):
     have = np.zeros_like(must)
     have[rows, gid] = True
     assert (have | ~must).all()
-    # 1e-3 absolute, plus 5e-4 relative for the large logits of the wide shapes: one element of the
-    # corrected state rounding to the neighbouring bf16 moves a logit by ulp(z) * |W|, which grows with
-    # the logit scale (d = 5120 gives logits around 6 and, on average, half a flipped element per row)
-    np.testing.assert_allclose(p["cand_logit"].reshape(-1, w.k), picked, atol=1e-3, rtol=5e-4)
+    # The bar is 1e-3 on a logit (= 1e-3 relative on its probability).  One explicit allowance: the GPU rounds the
+    # corrected state z~ to bf16 from an fp32 value, the oracle from the fp64 one, so an element that lies within
+    # the GPU's own error of the midpoint between two bf16 values may round to the other neighbour, which moves a
+    # logit by (bf16 step of z_i) * |W[v, i]|.  Those elements are found from the oracle's unrounded z~ (fp32 sums
+    # over d terms: 4e-6 relative is a generous bound on the GPU's error), the allowance is their worst case, and
+    # few logits may need it at all.
+    zc = hd["zc"].reshape(-1, w.d)
+    zt = I.bf16_bits_to_f32(hd["zt"].reshape(-1, w.d)).astype(np.float64)
+    step = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(zt), 1e-30))) - 7)
+    at_risk = np.abs(np.abs(zc - zt) - 0.5 * step) <= 4e-6 * np.abs(zc)
+    Wf = I.bf16_bits_to_f32(W).astype(np.float64)
+    allow = np.full(gid.shape, 1e-3)
+    for r in np.nonzero(at_risk.any(-1))[0]:
+        cols = np.nonzero(at_risk[r])[0]
+        allow[r] += (np.abs(Wf[gid[r]][:, cols]) * step[r, cols][None, :]).sum(-1)
+    dl = np.abs(p["cand_logit"].reshape(-1, w.k).astype(np.float64) - picked)
+    assert (dl <= allow).all(), (name, float((dl - allow).max()))
+    assert (dl > 1e-3).mean() < 0.01, (name, float((dl > 1e-3).mean()))
     d = ref.tree_draw(wl.parent, wl.anchor[idx].cpu().numpy(), p["cand_id"], p["cand_logit"],
                       wl.u_draw[idx].cpu().numpy(), temperature=w.temperature)
     assert np.array_equal(p["tree_tok"], d["tree_tok"])
@@ -142,3 +157,32 @@ def test_full_size_step_sampled_against_the_oracle(name, n_random):
     assert (np.sort(cid, -1)[..., 1:] != np.sort(cid, -1)[..., :-1]).all()
     cl = wl.prop["cand_logit"].cpu().numpy()
     assert (np.diff(cl, axis=-1) <= 0).all()
+
+
+def test_projection_and_top_k_of_a_whole_row_block():
+    """Every row of the first 128-row block of the projection's M dimension (32 sequences x 4 heads of the 1.5B
+    shape) against the oracle's full logits: the block is what one CTA column of the kernel owns."""
+    w = I.WORKLOADS["qwen1.5b"]
+    wl = StepWorkload(w, torch.device("cuda", 0), layers=1)
+    wl.propose()
+    torch.cuda.synchronize()
+    assert S.workspace_status(wl.ws_propose) == 0
+    n_seq = 128 // w.K
+    sl = slice(0, n_seq)
+    A, bias, W = _bits(wl.A), _bits(wl.bias), _bits(wl.W)
+    hd = ref.heads(_bits(wl.h[sl]), A, bias, m=wl.m[sl].cpu().numpy(), alpha=wl.alpha[sl].cpu().numpy(),
+                   clip_c=w.clip_c)
+    full = ref.lm_logits(hd["zt"], W)                             # [128, V]
+    oid, ol = ref.topk(full, w.k)
+    gid = wl.prop["cand_id"][sl].cpu().numpy().reshape(-1, w.k)
+    gl = wl.prop["cand_logit"][sl].cpu().numpy().reshape(-1, w.k).astype(np.float64)
+    rows = np.arange(full.shape[0])[:, None]
+    kth = ol[:, -1].astype(np.float64)
+    picked = full[rows, gid]
+    assert (picked >= kth[:, None] - 1e-3).all()                  # nothing below the cut (ties within 1e-3 aside)
+    must = full > (kth[:, None] + 1e-3)
+    have = np.zeros_like(must)
+    have[rows, gid] = True
+    assert (have | ~must).all()                                   # nothing above the cut is missing
+    assert np.abs(gl - picked).max() <= 1e-3
+    assert (np.diff(gl, axis=-1) <= 0).all()                      # lists sorted by logit

@@ -148,6 +148,28 @@ def test_tree_draw_alone_matches_exactly():
     assert np.array_equal(host(g["tree_tok"]), o["tree_tok"])
 
 
+def test_tree_draw_with_a_candidate_that_dwarfs_the_rest():
+    # One candidate of every head leads the others by more than 745 T, so that once it has been drawn the weights
+    # of the rest underflow against it and the draw has to renormalise over what is left (App. B.1 Eq. "slotq":
+    # q_{u,j} is a softmax over the remaining candidates only).  Two parents of the same depth draw from the same
+    # head: the second parent's first child must still see the leading candidate.
+    parent = np.array([-1, 0, 0, 1, 1, 1, 2, 2, 2], np.int32)
+    B, K, k = 64, 2, 4
+    g = I.rng(77)
+    cid = np.tile(np.arange(K * k, dtype=np.int32).reshape(1, K, k), (B, 1, 1))
+    cl = np.sort(g.standard_normal((B, K, k)).astype(np.float32), axis=-1)[..., ::-1].copy()
+    cl[..., 0] += 900.0
+    u = I.uniforms24(9, (B, parent.shape[0]))
+    anchor = np.zeros(B, np.int32)
+    for T in (1.0, 0.7):
+        o = ref.tree_draw(parent, anchor, cid, cl, u, temperature=T)
+        d = S.tree_draw(parent, dev(anchor), dev(cid), dev(cl), dev(u), temperature=T)
+        assert (o["tree_cand"][:, [1, 3, 6]] == 0).all()          # every first child takes the leading candidate
+        assert np.array_equal(host(d["tree_tok"]), o["tree_tok"])
+        assert np.array_equal(host(d["tree_cand"]), o["tree_cand"])
+        np.testing.assert_allclose(host(d["slot_q"]), o["slot_q"], rtol=1e-6)
+
+
 def test_bad_arguments():
     w = I.scaled(I.WORKLOADS["tiny"], B=2)
     x = I.propose_inputs(w)

@@ -42,7 +42,7 @@ def _same(a, b):
 
 
 def test_two_calls_in_a_row_match_the_workspace_entry_point():
-    # first call: many sequences, wide candidate lists -> fills most of the shared scratch
+    # first call: many sequences, wide candidate lists (B * k = 2400 of the 16384 candidate slots the scratch holds)
     args1 = _case(B=300, N=16, K=4, k=8, V=4096, seed=1, boost=6.0)
     want1 = S.verify(*args1)
     got1 = S.verify_static(*args1)
@@ -59,6 +59,21 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     got3 = S.verify_static(*args1)
     torch.cuda.synchronize()
     _same(got3, want1)
+
+
+def test_the_largest_admitted_problem_fits_the_scratch():
+    # exactly at both limits: B = 4096 sequences and B * k = 16384 candidate slots; small tree and vocabulary
+    args = _case(B=4096, N=5, K=2, k=4, V=512, seed=3, boost=4.0)
+    want = S.verify(*args)
+    got = S.verify_static(*args)
+    torch.cuda.synchronize()
+    _same(got, want)
+    # and a small problem right after it
+    args2 = _case(B=5, N=3, K=2, k=2, V=256, seed=4, boost=3.0)
+    got2 = S.verify_static(*args2)
+    want2 = S.verify(*args2)
+    torch.cuda.synchronize()
+    _same(got2, want2)
 
 
 def test_sizes_beyond_the_fixed_limit_are_refused_with_a_clear_error():
