@@ -129,8 +129,25 @@ def _stream() -> C.c_void_p:
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
+# Every device tensor this module allocates (outputs and workspaces) comes from this function.  The tests swap in
+# an allocator that surrounds each tensor with guard bytes and checks them afterwards (set_allocator); by default
+# it is torch.empty.
+_empty = torch.empty
+
+
+def set_allocator(fn=None):
+    """Replaces the allocator of outputs and workspaces (signature of torch.empty); None restores torch.empty."""
+    global _empty
+    _empty = torch.empty if fn is None else fn
+
+
+def alloc(*size, **kw) -> torch.Tensor:
+    """torch.empty through the current allocator (for callers that keep outputs and workspaces of their own)."""
+    return _empty(*size, **kw)
+
+
 def _workspace(nbytes: int, device) -> torch.Tensor:
-    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    return _empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
 
 
 def version() -> int:
@@ -175,11 +192,11 @@ def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0,
     desc = ProposeDesc(B, N, K, k, d, V, temperature, ln_eps, rms_eps, clip_c, flags)
     dev = h.device
     if out is None:
-        out = {"cand_id": torch.empty((B, K, k), dtype=torch.int32, device=dev),
-               "cand_logit": torch.empty((B, K, k), dtype=torch.float32, device=dev),
-               "tree_tok": torch.empty((B, N), dtype=torch.int32, device=dev),
-               "tree_cand": torch.empty((B, N), dtype=torch.uint8, device=dev),
-               "slot_q": torch.empty((B, N), dtype=torch.float32, device=dev)}
+        out = {"cand_id": _empty((B, K, k), dtype=torch.int32, device=dev),
+               "cand_logit": _empty((B, K, k), dtype=torch.float32, device=dev),
+               "tree_tok": _empty((B, N), dtype=torch.int32, device=dev),
+               "tree_cand": _empty((B, N), dtype=torch.uint8, device=dev),
+               "slot_q": _empty((B, N), dtype=torch.float32, device=dev)}
     if workspace is None:
         workspace = _workspace(lib().specroll_propose_workspace_bytes(C.byref(desc)), dev)
     bf = torch.bfloat16
@@ -204,9 +221,9 @@ def tree_draw(parent, anchor, cand_id, cand_logit, u_draw, temperature=1.0) -> D
     B, K, k = cand_id.shape
     N = parent.shape[0]
     dev = cand_id.device
-    out = {"tree_tok": torch.empty((B, N), dtype=torch.int32, device=dev),
-           "tree_cand": torch.empty((B, N), dtype=torch.uint8, device=dev),
-           "slot_q": torch.empty((B, N), dtype=torch.float32, device=dev)}
+    out = {"tree_tok": _empty((B, N), dtype=torch.int32, device=dev),
+           "tree_cand": _empty((B, N), dtype=torch.uint8, device=dev),
+           "slot_q": _empty((B, N), dtype=torch.float32, device=dev)}
     rc = lib().specroll_tree_draw(
         C.c_int32(B), C.c_int32(N), C.c_int32(K), C.c_int32(k), C.c_float(temperature),
         parent.ctypes.data_as(C.c_void_p), _dev(anchor, torch.int32, "anchor"),
@@ -251,9 +268,9 @@ def tree_attn(Q, Kc, Vc, kv_indptr_dev, kv_indptr_host, Kt, Vt, parent, scale=No
     desc = AttnDesc(B, N, Hq, Hkv, D, scale, flags)
     dev = Q.device
     if out is None:
-        out = torch.empty((B, N, Hq, D), dtype=torch.bfloat16, device=dev)
+        out = _empty((B, N, Hq, D), dtype=torch.bfloat16, device=dev)
     if want_lse and lse is None:
-        lse = torch.empty((B, N, Hq), dtype=torch.float32, device=dev)
+        lse = _empty((B, N, Hq), dtype=torch.float32, device=dev)
     if workspace is None:
         workspace = _workspace(lib().specroll_tree_attn_workspace_bytes(
             C.byref(desc), ip.ctypes.data_as(C.c_void_p)), dev)
@@ -296,9 +313,9 @@ def tree_attn_paged(Q, Kp, Vp, page_table, page_indptr, kv_len_dev, kv_len_host,
     desc = AttnDesc(B, N, Hq, Hkv, D, scale, flags)
     dev = Q.device
     if out is None:
-        out = torch.empty((B, N, Hq, D), dtype=torch.bfloat16, device=dev)
+        out = _empty((B, N, Hq, D), dtype=torch.bfloat16, device=dev)
     if want_lse and lse is None:
-        lse = torch.empty((B, N, Hq), dtype=torch.float32, device=dev)
+        lse = _empty((B, N, Hq), dtype=torch.float32, device=dev)
     if workspace is None:
         workspace = _workspace(lib().specroll_tree_attn_paged_workspace_bytes(
             C.byref(desc), kl.ctypes.data_as(C.c_void_p)), dev)
@@ -361,7 +378,7 @@ def gather_hidden(hidden, term_node, out=None):
     """specroll_gather_hidden: hidden[B,N,d] bf16, term_node[B] -> h_next[B,d]."""
     B, N, d = hidden.shape
     if out is None:
-        out = torch.empty((B, d), dtype=torch.bfloat16, device=hidden.device)
+        out = _empty((B, d), dtype=torch.bfloat16, device=hidden.device)
     rc = lib().specroll_gather_hidden(B, N, d, _dev(hidden, torch.bfloat16, "hidden"),
                                       _dev(term_node, torch.int32, "term_node"), _dev(out, torch.bfloat16, "h_next"),
                                       _stream())
@@ -394,14 +411,14 @@ def verify(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fi
     dev = logits.device
     i32, f32 = torch.int32, torch.float32
     if out is None:
-        out = {"n_acc": torch.empty(B, dtype=i32, device=dev),
-               "path_node": torch.empty((B, K + 1), dtype=i32, device=dev),
-               "out_tok": torch.empty((B, K + 1), dtype=i32, device=dev),
-               "term_node": torch.empty(B, dtype=i32, device=dev),
-               "term_kind": torch.empty(B, dtype=i32, device=dev),
-               "row_max": torch.empty((B, N), dtype=f32, device=dev),
-               "row_sum": torch.empty((B, N), dtype=f32, device=dev),
-               "min_margin": torch.empty(B, dtype=f32, device=dev)}
+        out = {"n_acc": _empty(B, dtype=i32, device=dev),
+               "path_node": _empty((B, K + 1), dtype=i32, device=dev),
+               "out_tok": _empty((B, K + 1), dtype=i32, device=dev),
+               "term_node": _empty(B, dtype=i32, device=dev),
+               "term_kind": _empty(B, dtype=i32, device=dev),
+               "row_max": _empty((B, N), dtype=f32, device=dev),
+               "row_sum": _empty((B, N), dtype=f32, device=dev),
+               "min_margin": _empty(B, dtype=f32, device=dev)}
     if workspace is None:
         workspace = _workspace(lib().specroll_verify_workspace_bytes(C.byref(desc)), dev)
     rc = lib().specroll_verify(
@@ -430,15 +447,15 @@ def verify_fused(hidden, W, parent, tree_tok, tree_cand, cand_id, cand_logit, u_
     desc = VerifyDesc(B, N, K, k, V, temperature, 0)
     dev = hidden.device
     i32, f32 = torch.int32, torch.float32
-    want = torch.empty((B * N, k), dtype=i32, device=dev)
+    want = _empty((B * N, k), dtype=i32, device=dev)
     rc = lib().specroll_verify_want_ids(C.byref(desc), parent.ctypes.data_as(C.c_void_p), _dev(cand_id, i32, "cand_id"),
                                         _dev(want, i32, "want_id"), _stream())
     _check(rc, "specroll_verify_want_ids")
     st = target_head_stats(hidden.reshape(B * N, d), W, want, temperature=temperature)
-    out = {"n_acc": torch.empty(B, dtype=i32, device=dev), "path_node": torch.empty((B, K + 1), dtype=i32, device=dev),
-           "out_tok": torch.empty((B, K + 1), dtype=i32, device=dev), "term_node": torch.empty(B, dtype=i32, device=dev),
-           "term_kind": torch.empty(B, dtype=i32, device=dev), "row_max": st["row_max"].reshape(B, N),
-           "row_sum": st["row_sum"].reshape(B, N), "min_margin": torch.empty(B, dtype=f32, device=dev)}
+    out = {"n_acc": _empty(B, dtype=i32, device=dev), "path_node": _empty((B, K + 1), dtype=i32, device=dev),
+           "out_tok": _empty((B, K + 1), dtype=i32, device=dev), "term_node": _empty(B, dtype=i32, device=dev),
+           "term_kind": _empty(B, dtype=i32, device=dev), "row_max": st["row_max"].reshape(B, N),
+           "row_sum": st["row_sum"].reshape(B, N), "min_margin": _empty(B, dtype=f32, device=dev)}
     ws = _workspace(lib().specroll_verify_workspace_bytes(C.byref(desc)), dev)
     rc = lib().specroll_verify_walk_sparse(
         C.byref(desc), _dev(st["want_logit"], torch.bfloat16, "cand_target"), _dev(st["row_max"], f32, "row_max"),
@@ -473,16 +490,16 @@ def verify_nucleus(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_a
     dev = logits.device
     i32, f32 = torch.int32, torch.float32
     if out is None:
-        out = {"n_acc": torch.empty(B, dtype=i32, device=dev),
-               "path_node": torch.empty((B, K + 1), dtype=i32, device=dev),
-               "out_tok": torch.empty((B, K + 1), dtype=i32, device=dev),
-               "term_node": torch.empty(B, dtype=i32, device=dev),
-               "term_kind": torch.empty(B, dtype=i32, device=dev),
-               "row_max": torch.empty((B, N), dtype=f32, device=dev),
-               "row_sum": torch.empty((B, N), dtype=f32, device=dev),
-               "min_margin": torch.empty(B, dtype=f32, device=dev),
-               "nucleus_thr": torch.empty((B, N), dtype=f32, device=dev),
-               "nucleus_sum": torch.empty((B, N), dtype=f32, device=dev)}
+        out = {"n_acc": _empty(B, dtype=i32, device=dev),
+               "path_node": _empty((B, K + 1), dtype=i32, device=dev),
+               "out_tok": _empty((B, K + 1), dtype=i32, device=dev),
+               "term_node": _empty(B, dtype=i32, device=dev),
+               "term_kind": _empty(B, dtype=i32, device=dev),
+               "row_max": _empty((B, N), dtype=f32, device=dev),
+               "row_sum": _empty((B, N), dtype=f32, device=dev),
+               "min_margin": _empty(B, dtype=f32, device=dev),
+               "nucleus_thr": _empty((B, N), dtype=f32, device=dev),
+               "nucleus_sum": _empty((B, N), dtype=f32, device=dev)}
     if workspace is None:
         workspace = _workspace(lib().specroll_verify_nucleus_workspace_bytes(C.byref(desc)), dev)
     rc = lib().specroll_verify_nucleus(
@@ -513,9 +530,9 @@ def reflex_feedback(logits, rec_row, row_max, row_sum, cand_id, cand_logit, y_st
                         float(severity_min) if weighted else 0.0)
     dev = logits.device
     f32, i32 = torch.float32, torch.int32
-    out = {n: torch.empty(R, dtype=f32, device=dev) for n in ("d_dist", "d_cov", "tv", "severity")}
+    out = {n: _empty(R, dtype=f32, device=dev) for n in ("d_dist", "d_cov", "tv", "severity")}
     if want_e:
-        out["e"] = torch.empty((R, d), dtype=f32, device=dev)
+        out["e"] = _empty((R, d), dtype=f32, device=dev)
     need = lib().specroll_reflex_feedback_workspace_bytes(C.byref(desc))
     if need == 0:
         raise SpecrollError("reflex_feedback: invalid descriptor")
@@ -538,7 +555,7 @@ def reflex_sketch(X, Pi, rows=None):
     (``rows`` [R] i32 selects them; all rows in order when None) under the projection Pi [rank, d] fp32."""
     rank, d = Pi.shape
     R = X.shape[0] if rows is None else rows.shape[0]
-    out = torch.empty((R, rank), dtype=torch.float32, device=X.device)
+    out = _empty((R, rank), dtype=torch.float32, device=X.device)
     rc = lib().specroll_reflex_sketch(C.c_int32(R), C.c_int32(d), C.c_int32(rank), _dev(X, torch.float32, "X"),
                                       _dev(rows, torch.int32, "rows") if rows is not None else None,
                                       _dev(Pi, torch.float32, "Pi"), _dev(out, torch.float32, "sketch"), _stream())
@@ -557,8 +574,8 @@ def reflex_gate(s, xi, slot, keep, n, mean, M2, n_fb, m, horizon, n_align_min, n
     dev = m.device
     f32, i32 = torch.float32, torch.int32
     desc = GateDesc(R, S, d, rank, H, z_delta, mem_eps, 0)
-    out = {"a": torch.empty(max(R, 1), dtype=f32, device=dev)[:R], "rel": torch.empty(S, dtype=f32, device=dev),
-           "alpha": torch.empty(S, dtype=f32, device=dev)}
+    out = {"a": _empty(max(R, 1), dtype=f32, device=dev)[:R], "rel": _empty(S, dtype=f32, device=dev),
+           "alpha": _empty(S, dtype=f32, device=dev)}
     rc = lib().specroll_reflex_gate(
         C.byref(desc), _dev(s, f32, "s"), _dev(xi, f32, "xi"), _dev(slot, i32, "slot"),
         _dev(keep, torch.uint8, "keep") if keep is not None else None, _dev(n, i32, "n"), _dev(mean, f32, "mean"),
@@ -577,9 +594,9 @@ def target_head_stats(H, W, want_id=None, temperature=1.0, workspace=None):
     V = W.shape[0]
     kw = 0 if want_id is None else want_id.shape[1]
     dev = H.device
-    out = {"row_max": torch.empty(R, dtype=torch.float32, device=dev),
-           "row_sum": torch.empty(R, dtype=torch.float32, device=dev),
-           "want_logit": torch.empty((R, kw), dtype=torch.bfloat16, device=dev)}
+    out = {"row_max": _empty(R, dtype=torch.float32, device=dev),
+           "row_sum": _empty(R, dtype=torch.float32, device=dev),
+           "want_logit": _empty((R, kw), dtype=torch.bfloat16, device=dev)}
     need = lib().specroll_target_head_stats_workspace_bytes(C.c_int32(R), C.c_int32(d), C.c_int32(V))
     if need == 0:
         raise SpecrollError("target_head_stats: invalid shape")
@@ -600,7 +617,7 @@ def target_head_rows(H, W, out=None):
     R, d = H.shape
     V = W.shape[0]
     if out is None:
-        out = torch.empty((R, V), dtype=torch.bfloat16, device=H.device)
+        out = _empty((R, V), dtype=torch.bfloat16, device=H.device)
     status = torch.zeros(1, dtype=torch.int32, device=H.device)
     rc = lib().specroll_target_head_rows(C.c_int32(R), C.c_int32(d), C.c_int32(V), _dev(H, torch.bfloat16, "H"),
                                          _dev(W, torch.bfloat16, "W"), _dev(out, torch.bfloat16, "logits"),
@@ -628,14 +645,14 @@ def verify_static(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_ac
     dev = logits.device
     i32, f32 = torch.int32, torch.float32
     if out is None:
-        out = {"n_acc": torch.empty(B, dtype=i32, device=dev),
-               "path_node": torch.empty((B, K + 1), dtype=i32, device=dev),
-               "out_tok": torch.empty((B, K + 1), dtype=i32, device=dev),
-               "term_node": torch.empty(B, dtype=i32, device=dev),
-               "term_kind": torch.empty(B, dtype=i32, device=dev),
-               "row_max": torch.empty((B, N), dtype=f32, device=dev),
-               "row_sum": torch.empty((B, N), dtype=f32, device=dev),
-               "min_margin": torch.empty(B, dtype=f32, device=dev)}
+        out = {"n_acc": _empty(B, dtype=i32, device=dev),
+               "path_node": _empty((B, K + 1), dtype=i32, device=dev),
+               "out_tok": _empty((B, K + 1), dtype=i32, device=dev),
+               "term_node": _empty(B, dtype=i32, device=dev),
+               "term_kind": _empty(B, dtype=i32, device=dev),
+               "row_max": _empty((B, N), dtype=f32, device=dev),
+               "row_sum": _empty((B, N), dtype=f32, device=dev),
+               "min_margin": _empty(B, dtype=f32, device=dev)}
     rc = lib().specroll_verify_static(
         C.byref(desc), _dev(logits, torch.bfloat16, "logits"), parent.ctypes.data_as(C.c_void_p),
         _dev(tree_tok, i32, "tree_tok"), _dev(tree_cand, torch.uint8, "tree_cand"),

@@ -19,6 +19,20 @@ def env_world() -> Tuple[int, int, int]:
             int(os.environ.get("WORLD_SIZE", "1")))
 
 
+def launch_plan(gpus: int, env=None):
+    """What ``--gpus N`` asks of this process.  ("run", None): go ahead as the rank the environment says (a launcher
+    started N ranks, or N == 1 and there is no launcher).  ("spawn", None): N > 1 and no launcher: the caller
+    starts N ranks itself.  ("refuse", message): a launcher started a different number of ranks than N."""
+    env = os.environ if env is None else env
+    ws = env.get("WORLD_SIZE")
+    if ws is None:
+        return ("run", None) if gpus <= 1 else ("spawn", None)
+    if int(ws) != int(gpus):
+        return ("refuse", f"--gpus {gpus} but the launcher started WORLD_SIZE={ws} ranks: start "
+                          f"--nproc-per-node {gpus}, or drop the launcher and let bench.py start its ranks")
+    return ("run", None)
+
+
 def init(backend: str) -> bool:
     """Joins the process group when launched with more than one rank.  Returns True if joined."""
     rank, _, world = env_world()

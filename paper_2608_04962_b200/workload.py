@@ -75,7 +75,7 @@ class StepWorkload:
             self.Vc.append(_randn_bf16(gen, (self.T_kv, w.Hkv, w.D), 1.0, device))
             self.Kt.append(_randn_bf16(gen, (B, N, w.Hkv, w.D), 1.0, device))
             self.Vt.append(_randn_bf16(gen, (B, N, w.Hkv, w.D), 1.0, device))
-        self.O = [torch.empty((B, N, w.Hq, w.D), dtype=torch.bfloat16, device=device)
+        self.O = [S.alloc((B, N, w.Hq, w.D), dtype=torch.bfloat16, device=device)
                   for _ in range(self.layers)]
         if self.paged:
             # the same caches scattered into pools of 128-token pages in a seeded random page order, with room
@@ -103,12 +103,12 @@ class StepWorkload:
                     dst.append(pool.view(self.n_pages, PAGE, w.Hkv, w.D))
                     src[l] = None
         # workspaces and outputs, allocated once
-        self.ws_propose = torch.empty(S.propose_workspace_bytes(B, N, K, k, d, V, w.temperature),
+        self.ws_propose = S.alloc(S.propose_workspace_bytes(B, N, K, k, d, V, w.temperature),
                                       dtype=torch.uint8, device=device)
         ws_bytes = (S.tree_attn_paged_workspace_bytes(B, N, w.Hq, w.Hkv, w.D, self.kv_len_host) if self.paged else
                     S.tree_attn_workspace_bytes(B, N, w.Hq, w.Hkv, w.D, self.kv_indptr_host))
-        self.ws_attn = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
-        self.ws_verify = torch.empty(S.verify_nucleus_workspace_bytes(B, N, K, k, V, w.temperature),
+        self.ws_attn = S.alloc(ws_bytes, dtype=torch.uint8, device=device)
+        self.ws_verify = S.alloc(S.verify_nucleus_workspace_bytes(B, N, K, k, V, w.temperature),
                                      dtype=torch.uint8, device=device)
         self.prop = None
         self.ver = None

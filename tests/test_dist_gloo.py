@@ -47,3 +47,13 @@ def test_single_process_aggregation_is_identity():
     from paper_2608_04962_b200 import dist as D
     assert D.env_world()[2] >= 1
     assert D.aggregate(3.5, 7.0) == (3.5, 7.0)
+
+
+def test_gpus_flag_against_the_launcher_environment():
+    from paper_2608_04962_b200 import dist as D
+    assert D.launch_plan(1, env={}) == ("run", None)
+    assert D.launch_plan(4, env={}) == ("spawn", None)                     # no launcher: bench.py starts the ranks
+    assert D.launch_plan(4, env={"WORLD_SIZE": "4"}) == ("run", None)
+    kind, msg = D.launch_plan(8, env={"WORLD_SIZE": "2"})
+    assert kind == "refuse" and "WORLD_SIZE=2" in msg
+    assert D.launch_plan(1, env={"WORLD_SIZE": "2"})[0] == "refuse"
