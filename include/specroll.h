@@ -41,12 +41,32 @@ extern "C" {
 #define SPECROLL_ELIMIT 6     /* problem larger than a fixed limit: of an allocation-free entry point, of the kernel a
                                  paged cache needs, or of a sequence's own pages */
 
+#define SPECROLL_EINDEX 7     /* debug build only: an index in a caller's device array is out of range */
+
 #define SPECROLL_MAX_NODES 64
 #define SPECROLL_MAX_HEADS 8
 #define SPECROLL_MAX_TOPK 64
 
 /* Library version (major * 10000 + minor * 100 + patch). */
 int specroll_version(void);
+
+/* Debug builds (compiled with -DSPECROLL_CHECK; the paper has no counterpart).  There the kernels check the
+ * indices they read from the caller's device arrays (candidate token ids and candidate slots of the
+ * verification walk, cache lengths of the attention plan):
+ * a bad index is not followed (index 0 is used instead, so the launch completes and nothing is read or
+ * written out of bounds) and the first one is remembered.  This call returns SPECROLL_OK, or
+ * SPECROLL_EINDEX with *detail (nullable) = the sequence or record it was found in; reset != 0 clears the
+ * memory.  It copies from the device synchronously: synchronise the streams the calls were enqueued on
+ * first.  In a normal build the checks do not exist and the call returns -1. */
+int specroll_check_status(int32_t *detail, int32_t reset);
+
+/* Debug builds only (the paper has no counterpart): arranges for one bounded device-side wait to run out, so
+ * that the path on which a kernel gives up can be tested without a fault or a hang.  what == 1: the next
+ * specroll_propose leaves out one barrier arrival in its projection kernel (nothing asynchronous is abandoned);
+ * the waiting warps give up after the debug build's 20 ms limit, the kernel returns, and
+ * specroll_workspace_status reports SPECROLL_ETIMEOUT.  Returns SPECROLL_OK, SPECROLL_EINVAL for an unknown
+ * `what`, -1 in a normal build (where nothing of this exists). */
+int specroll_check_inject(int32_t what);
 
 /* Human-readable text for a return code; for SPECROLL_ECUDA includes the last CUDA error
  * string seen by the calling thread.  The pointer stays valid until the thread's next call. */

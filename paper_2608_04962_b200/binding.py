@@ -15,10 +15,11 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libspecroll.so")
+# SPECROLL_LIB selects another build of the same library (the debug build with index checks, libspecroll_check.so)
+LIB_PATH = os.environ.get("SPECROLL_LIB") or os.path.join(_HERE, "libspecroll.so")
 _lib = None
 
-EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget",
+EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget", "specroll_check_status", "specroll_check_inject",
            "specroll_propose_workspace_bytes", "specroll_propose", "specroll_workspace_status",
            "specroll_tree_draw",
            "specroll_tree_attn_workspace_bytes", "specroll_tree_attn", "specroll_tree_attn_launches",
@@ -152,6 +153,15 @@ def _workspace(nbytes: int, device) -> torch.Tensor:
 
 def version() -> int:
     return int(lib().specroll_version())
+
+
+def check_status(reset: bool = True):
+    """specroll_check_status after a device synchronisation: (code, detail).  code is -1 for a normal build, 0 when
+    the debug build's index checks found nothing, else SPECROLL_EINDEX with detail = the sequence it was found in."""
+    torch.cuda.synchronize()
+    detail = C.c_int32(0)
+    rc = int(lib().specroll_check_status(C.byref(detail), C.c_int32(1 if reset else 0)))
+    return rc, int(detail.value)
 
 
 def workspace_status(workspace: torch.Tensor) -> int:

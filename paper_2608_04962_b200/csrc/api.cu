@@ -43,6 +43,22 @@ int device_setup(const void *kernel, int dynamic_smem_bytes, int *n_sm) {
     return SPECROLL_OK;
 }
 
+// readers of the per-translation-unit check words (debug builds register them at load time)
+static CheckReader *check_readers(int **n) {
+    static CheckReader readers[16];
+    static int count = 0;
+    *n = &count;
+    return readers;
+}
+
+void register_check_reader(CheckReader fn) {
+    int *n = nullptr;
+    CheckReader *r = check_readers(&n);
+    if (*n < 16) r[(*n)++] = fn;
+}
+
+int lm_head_arm_dropped_signal();  // lm_head_tc.cu
+
 int build_topo(const int32_t *parent_host, int N, int K, int k, Topo *t, TopoMask *m) {
     if (!parent_host || N < 1 || N > SPECROLL_MAX_NODES || parent_host[0] != -1) return SPECROLL_EINVAL;
     memset(t, 0, sizeof(*t));
@@ -81,11 +97,41 @@ const char *specroll_strerror(int code) {
         case SPECROLL_ELIMIT:
             return "problem exceeds the fixed size limit of this allocation-free entry point (use the "
                    "variant that takes a caller workspace)";
+        case SPECROLL_EINDEX:
+            return "an index read from a caller's device array is out of range (found by a build with index checks)";
         case SPECROLL_ECUDA:
             snprintf(g_msg, sizeof(g_msg), "CUDA error: %s", cudaGetErrorString(g_last_cuda));
             return g_msg;
         default: return "unknown error code";
     }
+}
+
+int specroll_check_status(int32_t *detail, int32_t reset) {
+    using namespace specroll;
+#ifndef SPECROLL_CHECK
+    (void)reset;
+    if (detail) *detail = 0;
+    return -1;
+#else
+    int *n = nullptr;
+    CheckReader *r = check_readers(&n);
+    int first = SPECROLL_OK;
+    for (int i = 0; i < *n; ++i) {
+        int where = 0;
+        const int rc = r[i](&where, reset);
+        if (rc != SPECROLL_OK && first == SPECROLL_OK) {
+            first = rc;
+            if (detail) *detail = where;
+        }
+    }
+    if (first == SPECROLL_OK && detail) *detail = 0;
+    return first;
+#endif
+}
+
+int specroll_check_inject(int32_t what) {
+    if (what == 1) return specroll::lm_head_arm_dropped_signal();
+    return SPECROLL_EINVAL;
 }
 
 int32_t specroll_node_budget(int32_t C_hw, int32_t B_active, int32_t N_min, int32_t N_max) {

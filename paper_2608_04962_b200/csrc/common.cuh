@@ -26,6 +26,43 @@ int note_cuda_error(cudaError_t e);
 // the same (kernel, device) cost one table look-up.  Returns SPECROLL_OK or SPECROLL_ECUDA.
 int device_setup(const void *kernel, int dynamic_smem_bytes, int *n_sm);
 
+// ---- index checks of debug builds (-DSPECROLL_CHECK)
+// No memory checker can be run on this code where it is developed, so a debug build makes the kernels check the
+// indices they read from caller-supplied device arrays (token ids, candidate slots, record rows).  A bad index is
+// never followed: the kernel notes the first one (a code and where) in a word of its translation unit and goes on
+// with index 0, so the launch completes and the context stays usable.  specroll_check_status reads the words.
+typedef int (*CheckReader)(int *detail, int reset);
+void register_check_reader(CheckReader fn);
+#ifdef SPECROLL_CHECK
+#define SR_CHECK_TU()                                                                                      \
+    static __device__ int sr_check_word[2];                                                                \
+    static int sr_check_read(int *detail, int reset) {                                                     \
+        int w_[2] = {0, 0};                                                                                \
+        if (cudaMemcpyFromSymbol(w_, sr_check_word, sizeof(w_)) != cudaSuccess) return SPECROLL_ECUDA;     \
+        if (reset) {                                                                                       \
+            const int z_[2] = {0, 0};                                                                      \
+            if (cudaMemcpyToSymbol(sr_check_word, z_, sizeof(z_)) != cudaSuccess) return SPECROLL_ECUDA;   \
+        }                                                                                                  \
+        if (detail) *detail = w_[1];                                                                       \
+        return w_[0];                                                                                      \
+    }                                                                                                      \
+    static const int sr_check_registered = (specroll::register_check_reader(sr_check_read), 0);             \
+    /* `index` if it lies in [0, n), else notes the failure and gives 0 */                                  \
+    static __device__ __forceinline__ int sr_checked(int index, int n, int where) {                         \
+        if (index >= 0 && index < n) return index;                                                          \
+        if (atomicCAS(&sr_check_word[0], 0, SPECROLL_EINDEX) == 0) sr_check_word[1] = where;                \
+        return 0;                                                                                           \
+    }
+#define SR_CHECK_FAIL(where)                                                        \
+    do {                                                                            \
+        if (atomicCAS(&sr_check_word[0], 0, SPECROLL_EINDEX) == 0) sr_check_word[1] = (where); \
+    } while (0)
+#define SR_CHECKED(index, n, where) sr_checked((index), (n), (where))
+#else
+#define SR_CHECK_TU()
+#define SR_CHECKED(index, n, where) (index)
+#endif
+
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -15,6 +15,20 @@
 
 namespace specroll {
 
+#ifdef SPECROLL_CHECK
+// Debug build only: when armed (specroll_check_inject(1)), CTA 0 leaves out the signal "first accumulator complete"
+// once.  The epilogue warps' wait for it then runs into its time limit, which is how the test reaches the path on
+// which every role gives up, tensor memory is released and the kernel returns SPECROLL_ETIMEOUT.  Only an arrival
+// on a barrier is left out: no copy or tensor operation is abandoned.
+static __device__ int g_drop_one_signal;
+int lm_head_arm_dropped_signal() {
+    const int one = 1;
+    return cudaMemcpyToSymbol(g_drop_one_signal, &one, sizeof(one)) == cudaSuccess ? SPECROLL_OK : SPECROLL_ECUDA;
+}
+#else
+int lm_head_arm_dropped_signal() { return -1; }
+#endif
+
 namespace lmtc {
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
@@ -173,7 +187,11 @@ lm_head_topk_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                         phase ^= 1u;
                     }
                 }
-                if (ok) umma_commit(tfull_bar(buf));  // accumulator complete
+                bool signal = ok;
+#ifdef SPECROLL_CHECK
+                if (t == 0 && blockIdx.x == 0 && atomicExch(&g_drop_one_signal, 0) == 1) signal = false;
+#endif
+                if (signal) umma_commit(tfull_bar(buf));  // accumulator complete
             }
         }
     } else {

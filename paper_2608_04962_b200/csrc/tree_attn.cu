@@ -28,6 +28,8 @@
 
 namespace specroll {
 
+SR_CHECK_TU()
+
 constexpr int AT_BN = 64;       // KV tokens per tile
 constexpr int AT_STAGES = 3;
 constexpr int AT_MAX_WARPS = 8; // 128 query rows per CTA
@@ -112,7 +114,13 @@ attn_prep_kernel(const int32_t *__restrict__ kv_indptr, const int32_t *__restric
         return;
     }
     for (int b = t; b < B; b += PREP_THREADS) {
-        const int L = kv_len ? kv_len[b] : kv_indptr[b + 1] - kv_indptr[b];
+        int L = kv_len ? kv_len[b] : kv_indptr[b + 1] - kv_indptr[b];
+#ifdef SPECROLL_CHECK
+        if (L < 0) {  // the device copy of the lengths disagrees with any host copy the planner can have seen
+            SR_CHECK_FAIL(b);
+            L = 0;
+        }
+#endif
         const int tiles = (L + tile_tokens - 1) / tile_tokens;
         int ns = (tiles + chunk_tiles - 1) / chunk_tiles;
         if (ns < 1) ns = 1;

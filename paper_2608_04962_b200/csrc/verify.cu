@@ -19,6 +19,8 @@
 
 namespace specroll {
 
+SR_CHECK_TU()
+
 constexpr int RS_THREADS = 256;
 constexpr int RS_UNROLL = 4;
 constexpr int WALK_WARPS = 4;
@@ -386,7 +388,7 @@ __device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, doub
     const uint16_t *lg = a.logits ? a.logits + ((size_t)b * N + u) * a.V : nullptr;
     const uint16_t *ct = a.cand_target ? a.cand_target + ((size_t)b * N + u) * k : nullptr;
     for (int j = lane; j < k; j += 32) {
-        const int t = a.cand_id[((size_t)b * K + hd) * k + j];
+        const int t = SR_CHECKED(a.cand_id[((size_t)b * K + hd) * k + j], a.V, b);
         id[j] = t;
         cl[j] = a.cand_logit[((size_t)b * K + hd) * k + j];
         const uint32_t bits = lg ? lg[t] : ct[j];
@@ -417,7 +419,7 @@ __device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, doub
         for (int j = lane; j < k; j += 32)
             w[j] = ((taken >> j) & 1) ? 0.0 : exp(((double)cl[j] - mx) / a.T);
         __syncwarp();
-        const int jc = a.tree_cand[(size_t)b * N + c];
+        const int jc = SR_CHECKED((int)a.tree_cand[(size_t)b * N + c], k, b);
         if (lane == 0) {
             double s = 0.0;
             for (int j = 0; j < k; ++j) s += w[j];
