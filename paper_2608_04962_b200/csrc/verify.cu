@@ -361,6 +361,19 @@ struct WalkSmem {
     double bc[2];  // broadcast slots: current max, accepted flag
 };
 
+// Everything the walk of one sequence can read, staged in shared memory in one round of independent loads (the
+// plain walk; the other forms read global memory node by node): per node the row's statistics, the acceptance
+// uniform, the drawn token and its slot; per head the candidate ids and proposal logits; per walkable node the
+// target logits at its head's candidates.
+struct WalkStage {
+    const float *rmax, *rsum, *uacc;  // [N]
+    const int32_t *ttok;              // [N]
+    const uint8_t *tcand;             // [N]
+    const int32_t *cid;               // [K, k]
+    const float *clog;                // [K, k]
+    const uint16_t *pre;              // [N, k]
+};
+
 __device__ __forceinline__ void walk_begin(const WalkArgs &a, int b, int lane, WalkState *st) {
     st->nacc = 0;
     st->kind = 0;
@@ -378,8 +391,9 @@ __device__ __forceinline__ void walk_begin(const WalkArgs &a, int b, int lane, W
 // One node u (which has children), by one warp: the target's probabilities on the candidates of u's head -
 // S is the normaliser and thr the nucleus threshold key (0: none) of u's row - then u's children in slot order.
 // Returns the accepted child, or -1 when every child was rejected (the residual is then in sm->r, st->sigma).
+// sg (nullable): the sequence's inputs staged in shared memory.
 __device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, double M, double S, uint32_t thr, int lane,
-                         WalkSmem *sm, WalkState *st) {
+                         WalkSmem *sm, WalkState *st, const WalkStage *sg = nullptr) {
     double *r = sm->r, *w = sm->w;
     float *cl = sm->cl;
     int32_t *id = sm->id;
@@ -388,75 +402,73 @@ __device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, doub
     const uint16_t *lg = a.logits ? a.logits + ((size_t)b * N + u) * a.V : nullptr;
     const uint16_t *ct = a.cand_target ? a.cand_target + ((size_t)b * N + u) * k : nullptr;
     for (int j = lane; j < k; j += 32) {
-        const int t = SR_CHECKED(a.cand_id[((size_t)b * K + hd) * k + j], a.V, b);
+        const int t = sg ? sg->cid[hd * k + j] : SR_CHECKED(a.cand_id[((size_t)b * K + hd) * k + j], a.V, b);
         id[j] = t;
-        cl[j] = a.cand_logit[((size_t)b * K + hd) * k + j];
-        const uint32_t bits = lg ? lg[t] : ct[j];
+        cl[j] = sg ? sg->clog[hd * k + j] : a.cand_logit[((size_t)b * K + hd) * k + j];
+        const uint32_t bits = sg ? sg->pre[u * k + j] : (lg ? lg[t] : ct[j]);
         const double l = (double)bf16_bits_to_float((uint16_t)bits);
         r[j] = ord_key(bits) >= thr ? exp((l - M) / a.T) / S : 0.0;  // r = p_u on the candidates
     }
     __syncwarp();
+    // Every lane holds one or two of the k candidates (j = lane, lane + 32); sums and maxima over the candidates
+    // are warp reductions, so that the state (sigma, p_off, the margin) is the same in every lane and nothing of
+    // the slot loop runs on one lane alone (k-long loops of fp64 divisions on one lane were most of the walk's time).
     st->sigma = 1.0;
-    if (lane == 0) {
+    {
         double pc = 0.0;
-        for (int j = 0; j < k; ++j) pc += r[j];
-        st->p_off = 1.0 - pc;
-        if (st->p_off < 0.0) st->p_off = 0.0;
+        for (int j = lane; j < k; j += 32) pc += r[j];
+        pc = warp_sum(pc);
+        st->p_off = pc < 1.0 ? 1.0 - pc : 0.0;
     }
     uint64_t taken = 0;
     int accepted = -1;
     for (int c = u + 1; c < N && accepted < 0; ++c) {
         if (topo.parent[c] != u) continue;
         // slot proposal q on the candidates not yet taken
-        if (lane == 0) {
-            double mx = -INFINITY;
-            for (int j = 0; j < k; ++j)
-                if (!((taken >> j) & 1) && (double)cl[j] > mx) mx = (double)cl[j];
-            sm->bc[0] = mx;
-        }
-        __syncwarp();
-        const double mx = sm->bc[0];
+        double mx = -INFINITY;
         for (int j = lane; j < k; j += 32)
+            if (!((taken >> j) & 1) && (double)cl[j] > mx) mx = (double)cl[j];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        double s = 0.0;
+        for (int j = lane; j < k; j += 32) {
             w[j] = ((taken >> j) & 1) ? 0.0 : exp(((double)cl[j] - mx) / a.T);
-        __syncwarp();
-        const int jc = SR_CHECKED((int)a.tree_cand[(size_t)b * N + c], k, b);
-        if (lane == 0) {
-            double s = 0.0;
-            for (int j = 0; j < k; ++j) s += w[j];
-            const double qy = w[jc] / s;
-            double ratio;
-            if (qy > 0.0)
-                ratio = r[jc] / qy;
-            else
-                ratio = (r[jc] > 0.0) ? INFINITY : 0.0;
-            const double uu = (double)a.u_acc[(size_t)b * N + c];
-            const float mg = (float)fabs(uu - ratio);
-            if (mg < st->mm) st->mm = mg;
-            if (uu < (ratio < 1.0 ? ratio : 1.0)) {
-                sm->bc[1] = (double)c;
-            } else {
-                sm->bc[1] = -1.0;
-                double Z = 0.0;
-                for (int j = 0; j < k; ++j) {
-                    const double t = r[j] - w[j] / s;
-                    w[j] = t > 0.0 ? t : 0.0;
-                    Z += w[j];
-                }
-                Z += st->sigma * st->p_off;
-                if (Z > 1e-300) {
-                    for (int j = 0; j < k; ++j) r[j] = w[j] / Z;
-                    st->sigma /= Z;
-                }
-            }
+            s += w[j];
         }
+        s = warp_sum(s);
         __syncwarp();
-        accepted = (int)sm->bc[1];
+        const int jc = SR_CHECKED((int)(sg ? sg->tcand[c] : a.tree_cand[(size_t)b * N + c]), k, b);
+        const double qy = w[jc] / s;
+        double ratio;
+        if (qy > 0.0)
+            ratio = r[jc] / qy;
+        else
+            ratio = (r[jc] > 0.0) ? INFINITY : 0.0;
+        const double uu = (double)(sg ? sg->uacc[c] : a.u_acc[(size_t)b * N + c]);
+        const float mg = (float)fabs(uu - ratio);
+        if (mg < st->mm) st->mm = mg;
+        __syncwarp();
+        if (uu < (ratio < 1.0 ? ratio : 1.0)) {
+            accepted = c;
+        } else {
+            double Z = 0.0;
+            for (int j = lane; j < k; j += 32) {
+                const double t = r[j] - w[j] / s;
+                w[j] = t > 0.0 ? t : 0.0;
+                Z += w[j];
+            }
+            Z = warp_sum(Z) + st->sigma * st->p_off;
+            if (Z > 1e-300) {
+                for (int j = lane; j < k; j += 32) r[j] = w[j] / Z;
+                st->sigma /= Z;
+            }
+            __syncwarp();
+        }
         taken |= 1ull << jc;
-        __syncwarp();
     }
     if (accepted >= 0) {
         if (lane == 0) {
-            a.out_tok[(size_t)b * (K + 1) + st->nacc] = a.tree_tok[(size_t)b * N + accepted];
+            a.out_tok[(size_t)b * (K + 1) + st->nacc] = sg ? sg->ttok[accepted] : a.tree_tok[(size_t)b * N + accepted];
             a.path_node[(size_t)b * (K + 1) + st->nacc + 1] = accepted;
         }
         ++st->nacc;
@@ -484,13 +496,66 @@ __device__ __forceinline__ void walk_end(const WalkArgs &a, int b, int u, double
     }
 }
 
-// Plain target distributions: one warp per sequence.
+// Bytes of shared memory the staged inputs of one sequence take (16-byte multiples per array).
+__host__ __device__ inline size_t walk_stage_bytes(int N, int K, int k) {
+    auto up = [](size_t x) { return (x + 15) / 16 * 16; };
+    return 4 * up((size_t)N * 4) + up((size_t)N) + 2 * up((size_t)K * k * 4) + up((size_t)N * k * 2);
+}
+
+// Plain target distributions: one warp per sequence.  Which nodes the walk visits depends on its decisions, but
+// what it can ask for does not, so with the dense logits everything is fetched up front (WalkStage): one round
+// trip to memory per sequence instead of four or five dependent ones per visited node, which is what the walk's
+// time consisted of.  Dynamic shared memory: WALK_WARPS * walk_stage_bytes.
 __global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(WalkArgs a, Topo topo) {
     __shared__ WalkSmem sh[WALK_WARPS];
+    extern __shared__ __align__(16) unsigned char sh_stage[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x * WALK_WARPS + warp;
     if (b >= a.B) return;
     WalkSmem *sm = &sh[warp];
+    const int N = a.N, K = a.K, k = a.k;
+    WalkStage stage;
+    const WalkStage *sg = nullptr;
+    if (a.logits) {
+        auto up = [](size_t x) { return (x + 15) / 16 * 16; };
+        unsigned char *p = sh_stage + (size_t)warp * walk_stage_bytes(N, K, k);
+        float *rmax = reinterpret_cast<float *>(p);
+        p += up((size_t)N * 4);
+        float *rsum = reinterpret_cast<float *>(p);
+        p += up((size_t)N * 4);
+        float *uacc = reinterpret_cast<float *>(p);
+        p += up((size_t)N * 4);
+        int32_t *ttok = reinterpret_cast<int32_t *>(p);
+        p += up((size_t)N * 4);
+        uint8_t *tcand = reinterpret_cast<uint8_t *>(p);
+        p += up((size_t)N);
+        int32_t *cid = reinterpret_cast<int32_t *>(p);
+        p += up((size_t)K * k * 4);
+        float *clog = reinterpret_cast<float *>(p);
+        p += up((size_t)K * k * 4);
+        uint16_t *pre = reinterpret_cast<uint16_t *>(p);
+        for (int n = lane; n < N; n += 32) {
+            rmax[n] = a.row_max[(size_t)b * N + n];
+            rsum[n] = a.row_sum[(size_t)b * N + n];
+            uacc[n] = a.u_acc[(size_t)b * N + n];
+            ttok[n] = a.tree_tok[(size_t)b * N + n];
+            tcand[n] = a.tree_cand[(size_t)b * N + n];
+        }
+        for (int e = lane; e < K * k; e += 32) {
+            cid[e] = SR_CHECKED(a.cand_id[(size_t)b * K * k + e], a.V, b);
+            clog[e] = a.cand_logit[(size_t)b * K * k + e];
+        }
+        for (int e = lane; e < N * k; e += 32) {
+            const int u = e / k, j = e - u * k;
+            if (topo.n_child[u] > 0) {  // (a node with children is at depth < K)
+                const int t = SR_CHECKED(a.cand_id[((size_t)b * K + topo.depth[u]) * k + j], a.V, b);
+                pre[e] = a.logits[((size_t)b * N + u) * a.V + t];
+            }
+        }
+        __syncwarp();
+        stage = WalkStage{rmax, rsum, uacc, ttok, tcand, cid, clog, pre};
+        sg = &stage;
+    }
     WalkState st;
     walk_begin(a, b, lane, &st);
     int u = 0;
@@ -500,8 +565,9 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(WalkArgs a, Topo 
             st.have_residual = false;
             break;
         }
-        const int acc = walk_node(a, topo, b, u, (double)a.row_max[(size_t)b * a.N + u],
-                                  (double)a.row_sum[(size_t)b * a.N + u], 0u, lane, sm, &st);
+        const double M = sg ? (double)sg->rmax[u] : (double)a.row_max[(size_t)b * N + u];
+        const double S = sg ? (double)sg->rsum[u] : (double)a.row_sum[(size_t)b * N + u];
+        const int acc = walk_node(a, topo, b, u, M, S, 0u, lane, sm, &st, sg);
         if (acc < 0) {
             st.kind = 0;
             st.have_residual = true;
@@ -509,7 +575,7 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(WalkArgs a, Topo 
         }
         u = acc;
     }
-    walk_end(a, b, u, (double)a.row_sum[(size_t)b * a.N + u], lane, sm, &st);
+    walk_end(a, b, u, sg ? (double)sg->rsum[u] : (double)a.row_sum[(size_t)b * N + u], lane, sm, &st);
 }
 
 // Maximum and sum of exponentials of one row by all NUC_THREADS threads of a CTA (same arithmetic as
@@ -992,7 +1058,12 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
         walk_cta_kernel<true, false><<<d->B, NUC_THREADS, 0, st>>>(wa, topo, c, 1.0f, row_max, row_sum, nullptr, nullptr,
                                                                     nullptr, nullptr);
     } else {
-        walk_kernel<<<(d->B + WALK_WARPS - 1) / WALK_WARPS, WALK_WARPS * 32, 0, st>>>(wa, topo);
+        const size_t stage = (size_t)WALK_WARPS * walk_stage_bytes(d->N, d->K, d->k);
+        if (stage > 40 * 1024) {  // beyond what a kernel may use without asking (together with its static arrays)
+            const int rc_ = device_setup(reinterpret_cast<const void *>(walk_kernel), 64 * 1024, nullptr);
+            if (rc_ != SPECROLL_OK) return rc_;
+        }
+        walk_kernel<<<(d->B + WALK_WARPS - 1) / WALK_WARPS, WALK_WARPS * 32, stage, st>>>(wa, topo);
     }
     SR_LAUNCH_CHECK();
 
