@@ -61,7 +61,7 @@ class ClockSampler:
     def __init__(self, gpu_index: int, period_s: float = 0.002):
         self.idx = gpu_index
         self.period = period_s
-        self.sm, self.reasons = [], set()
+        self.sm, self.power, self.reasons = [], [], set()
         self.max_mhz = None
         self._stop = False
         self._thread = None
@@ -72,6 +72,10 @@ class ClockSampler:
         while not self._stop:
             try:
                 self.sm.append(float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                try:
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
+                except Exception:
+                    pass
                 bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
                 for name, mask in self.REASONS:
                     if bits & mask:
@@ -114,6 +118,8 @@ class ClockSampler:
                 pass
             return out
         out.update(sm_mhz=float(np.median(self.sm)), reasons=sorted(self.reasons), samples=len(self.sm))
+        if self.power:
+            out.update(power_w_median=float(np.median(self.power)), power_w_max=float(np.max(self.power)))
         return out
 
 

@@ -259,8 +259,20 @@ topk_merge_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pi
 
 constexpr int DRAW_WARPS = 4;
 
-// One warp per sequence.  Lanes evaluate the exponentials; lane 0 does the short ordered sums so
-// that the arithmetic order is the plain sequential one.
+__device__ __forceinline__ double warp_incl_scan_f64(double v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// One warp per sequence.  The nodes are drawn one after the other (a child's distribution depends on what its
+// earlier siblings took), but within a node the work over the k candidates is spread over the lanes (lane j holds
+// candidates j and j + 32): their total, the running sums of the inverse-CDF walk and the first candidate whose
+// running sum exceeds the uniform come from warp scans and ballots.  (With k-long fp64 loops on one lane a draw of
+// 48 nodes took 40 us.)
 __global__ void __launch_bounds__(DRAW_WARPS * 32)
 tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__restrict__ anchor,
                  const int32_t *__restrict__ cand_id, const float *__restrict__ cand_logit,
@@ -270,6 +282,9 @@ tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__rest
     // child's distribution is these weights renormalised over the candidates its earlier siblings left.
     __shared__ double sh_w[DRAW_WARPS][SPECROLL_MAX_HEADS][SPECROLL_MAX_TOPK];
     __shared__ unsigned long long sh_taken[DRAW_WARPS][SPECROLL_MAX_NODES];
+    // the candidates' token ids, so that the loop over the nodes reads nothing from global memory (a load whose
+    // value the same iteration stores holds the warp for a memory round trip per node)
+    __shared__ int32_t sh_id[DRAW_WARPS][SPECROLL_MAX_HEADS][SPECROLL_MAX_TOPK];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x * DRAW_WARPS + warp;
     if (b >= B) return;
@@ -279,55 +294,62 @@ tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__rest
         float mxf = -INFINITY;
         for (int j = lane; j < k; j += 32) mxf = fmaxf(mxf, cl[j]);
         mxf = warp_max(mxf);
-        for (int j = lane; j < k; j += 32) sh_w[warp][hd][j] = exp(((double)cl[j] - (double)mxf) / T);
+        for (int j = lane; j < k; j += 32) {
+            sh_w[warp][hd][j] = exp(((double)cl[j] - (double)mxf) / T);
+            sh_id[warp][hd][j] = cand_id[((size_t)b * K + hd) * k + j];
+        }
     }
     for (int n = lane; n < N; n += 32) sh_taken[warp][n] = 0ull;
+    // the uniforms of the sequence's nodes, one round of loads (lane n holds nodes n and n + 32)
+    const float u_lo = lane < N ? u_draw[(size_t)b * N + lane] : 0.f;
+    const float u_hi = lane + 32 < N ? u_draw[(size_t)b * N + lane + 32] : 0.f;
     __syncwarp();
-    if (lane != 0) return;
-    tree_tok[(size_t)b * N] = anchor[b];
-    tree_cand[(size_t)b * N] = 255;
-    slot_q[(size_t)b * N] = 1.0f;
+    if (lane == 0) {
+        tree_tok[(size_t)b * N] = anchor[b];
+        tree_cand[(size_t)b * N] = 255;
+        slot_q[(size_t)b * N] = 1.0f;
+    }
     for (int n = 1; n < N; ++n) {
         const int u = topo.parent[n], hd = topo.depth[n] - 1;
         const double *w = sh_w[warp][hd];
-        double w_left[SPECROLL_MAX_TOPK];  // used on the rare path below only
         const unsigned long long taken = sh_taken[warp][u];
-        double s = 0.0;
-        for (int j = 0; j < k; ++j)
-            if (!((taken >> j) & 1ull)) s += w[j];
+        const bool ok0 = lane < k && !((taken >> lane) & 1ull);
+        const bool ok1 = lane + 32 < k && !((taken >> (lane + 32)) & 1ull);
+        double w0 = ok0 ? w[lane] : 0.0, w1 = ok1 ? w[lane + 32] : 0.0;
+        double s = warp_sum(w0 + w1);
         if (!(s > 0.0)) {
             // every remaining weight underflowed against a taken candidate's logit: take the reference among
-            // the remaining ones instead.  The head's table is shared by all parents of this depth, whose taken
-            // sets differ, so the weights of this one draw go into an array of their own.
+            // the remaining ones instead (the head's table is shared by all parents of this depth, whose taken
+            // sets differ, so the weights of this one draw stay in registers)
             const float *cl = cand_logit + ((size_t)b * K + hd) * k;
-            float mxf = -INFINITY;
-            for (int j = 0; j < k; ++j)
-                if (!((taken >> j) & 1ull)) mxf = fmaxf(mxf, cl[j]);
-            s = 0.0;
-            for (int j = 0; j < k; ++j) {
-                w_left[j] = ((taken >> j) & 1ull) ? 0.0 : exp(((double)cl[j] - (double)mxf) / T);
-                s += w_left[j];
-            }
-            w = w_left;
+            float mxf = fmaxf(ok0 ? cl[lane] : -INFINITY, ok1 ? cl[lane + 32] : -INFINITY);
+            mxf = warp_max(mxf);
+            w0 = ok0 ? exp(((double)cl[lane] - (double)mxf) / T) : 0.0;
+            w1 = ok1 ? exp(((double)cl[lane + 32] - (double)mxf) / T) : 0.0;
+            s = warp_sum(w0 + w1);
         }
         // first remaining candidate whose cumulative probability exceeds the uniform (compared as masses)
-        const double thr = (double)u_draw[(size_t)b * N + n] * s;
-        double cum = 0.0;
-        int sel = -1, last = -1;
-        for (int j = 0; j < k; ++j) {
-            if ((taken >> j) & 1ull) continue;
-            last = j;
-            cum += w[j];
-            if (cum > thr) {
-                sel = j;
-                break;
-            }
+        const float un = __shfl_sync(0xffffffffu, n < 32 ? u_lo : u_hi, n & 31);
+        const double thr = (double)un * s;
+        const double c0 = warp_incl_scan_f64(w0, lane);
+        const double c1 = __shfl_sync(0xffffffffu, c0, 31) + warp_incl_scan_f64(w1, lane);
+        const unsigned hit0 = __ballot_sync(0xffffffffu, ok0 && c0 > thr), hit1 = __ballot_sync(0xffffffffu, ok1 && c1 > thr);
+        const unsigned v0 = __ballot_sync(0xffffffffu, ok0), v1 = __ballot_sync(0xffffffffu, ok1);
+        int sel;
+        if (hit0)
+            sel = __ffs(hit0) - 1;
+        else if (hit1)
+            sel = 32 + __ffs(hit1) - 1;
+        else
+            sel = v1 ? 32 + (31 - __clz(v1)) : (31 - __clz(v0));  // none: the last remaining candidate
+        const double wsel = __shfl_sync(0xffffffffu, sel < 32 ? w0 : w1, sel & 31);
+        if (lane == 0) {
+            sh_taken[warp][u] = taken | (1ull << sel);
+            tree_tok[(size_t)b * N + n] = sh_id[warp][hd][sel];
+            tree_cand[(size_t)b * N + n] = (uint8_t)sel;
+            slot_q[(size_t)b * N + n] = (float)(wsel / s);
         }
-        if (sel < 0) sel = last;
-        sh_taken[warp][u] = taken | (1ull << sel);
-        tree_tok[(size_t)b * N + n] = cand_id[((size_t)b * K + hd) * k + sel];
-        tree_cand[(size_t)b * N + n] = (uint8_t)sel;
-        slot_q[(size_t)b * N + n] = (float)(w[sel] / s);
+        __syncwarp();
     }
 }
 
