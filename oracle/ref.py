@@ -84,6 +84,19 @@ def heads(h, A, bias, m=None, alpha=None, gamma=None, beta=None, ln_eps=1e-5, rm
     return {"xhat": xhat, "z": z, "zc": zc, "zt": zt}
 
 
+def prehead(h, m, alpha, rms_eps=1e-6, clip_c=0.0):
+    """The correction applied to the last hidden state (secondary form).  h [B,d] bf16 bits, m [B,d] fp32,
+    alpha [B] fp32.  Returns dict(hc fp64 unrounded, ht bf16 bits)."""
+    h = _as(h, np.uint16)
+    m, alpha = _as(m, np.float32), _as(alpha, np.float32)
+    B, d = h.shape
+    hc = np.empty((B, d), np.float64)
+    ht = np.empty((B, d), np.uint16)
+    _chk(lib().specroll_ref_prehead(B, d, C.c_double(rms_eps), C.c_double(clip_c), _p(h), _p(m), _p(alpha), _p(hc),
+                                    _p(ht)), "prehead")
+    return {"hc": hc, "ht": ht}
+
+
 def lm_logits(zt, W):
     zt, W = _as(zt, np.uint16), _as(W, np.uint16)
     zt2 = zt.reshape(-1, zt.shape[-1])
@@ -132,7 +145,11 @@ def tree_draw(parent, anchor, cand_id, cand_logit, u_draw, temperature=1.0):
 
 
 def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0, ln_eps=1e-5,
-            rms_eps=1e-6, clip_c=0.0, gamma=None, beta=None):
+            rms_eps=1e-6, clip_c=0.0, gamma=None, beta=None, pre_head=False):
+    """pre_head: m [B,d] and alpha [B] correct the hidden state before the heads (no correction after them)."""
+    if pre_head:
+        h = prehead(h, m, alpha, rms_eps=rms_eps, clip_c=clip_c)["ht"]
+        m, alpha = None, None
     h, A, bias, W = (_as(x, np.uint16) for x in (h, A, bias, W))
     anchor, parent = _as(anchor, np.int32), _as(parent, np.int32)
     m, alpha, u_draw = _as(m, np.float32), _as(alpha, np.float32), _as(u_draw, np.float32)

@@ -175,6 +175,47 @@ int specroll_ref_heads(int B, int K, int d, double ln_eps, double rms_eps, doubl
     return REF_OK;
 }
 
+/* ------------------------------------------------------------------ proposal: correction before the heads
+ *
+ * Secondary form of the bounded correction (Sec. 3.4, Eq. "reflex-correction", applied to the last hidden
+ * state instead of to each head's output; the wording of this repository's task statement: "Reflex applies
+ * its bounded correction to the last hidden state, the K future-token heads run over it").  One memory row
+ * and one ratio per sequence:
+ *     dh = alpha_b RMS(h_b) m_b / (RMS(m_b) + eps),   |dh|_2 <= clip_c |h_b|_2 if clip_c > 0,
+ *     h~_b = h_b + dh   (alpha_b = 0 or m NULL: h~_b = h_b exactly),  rounded to bf16 (it replaces h).
+ * hc[B,d] fp64 (unrounded), ht[B,d] bf16; either may be NULL.
+ */
+int specroll_ref_prehead(int B, int d, double rms_eps, double clip_c, const uint16_t *h, const float *m,
+                         const float *alpha, double *hc_out, uint16_t *ht_out)
+{
+    if (B < 0 || d < 1) return REF_EINVAL;
+    for (int b = 0; b < B; ++b) {
+        double a = (alpha && m) ? (double)alpha[b] : 0.0;
+        double coef = 0.0;
+        if (a != 0.0) {
+            const float *mv = m + (size_t)b * d;
+            double sh = 0.0, sm = 0.0;
+            for (int i = 0; i < d; ++i) {
+                double hv = bf16_to_f64(h[(size_t)b * d + i]);
+                sh += hv * hv;
+                sm += (double)mv[i] * (double)mv[i];
+            }
+            double rms_h = sqrt(sh / d), rms_m = sqrt(sm / d);
+            coef = a * rms_h / (rms_m + rms_eps);
+            double nd = fabs(coef) * sqrt(sm); /* |dh|_2 */
+            double nh = sqrt(sh);
+            if (clip_c > 0.0 && nd > clip_c * nh) coef *= clip_c * nh / nd;
+        }
+        for (int i = 0; i < d; ++i) {
+            double hv = bf16_to_f64(h[(size_t)b * d + i]);
+            double v = (a != 0.0) ? hv + coef * (double)m[(size_t)b * d + i] : hv;
+            if (hc_out) hc_out[(size_t)b * d + i] = v;
+            if (ht_out) ht_out[(size_t)b * d + i] = (a != 0.0) ? f64_to_bf16(v) : h[(size_t)b * d + i];
+        }
+    }
+    return REF_OK;
+}
+
 /* ------------------------------------------------------------------ proposal: vocabulary projection
  *
  * logits[r, v] = W_v . zt_r  (shared, frozen projection; Eq. "heads", second line).

@@ -1,8 +1,49 @@
 // Host-side construction of TMA tensor maps (driver entry point looked up at run time, so the
 // library does not link against the driver).
+#include <string.h>
+
+#include <mutex>
+
 #include "tc05.cuh"
 
 namespace specroll {
+
+// A tensor map is a pure function of (base pointer, extents, strides, box): the last few are remembered, so that
+// the calls of a step (the same caches, weights and activations layer after layer, step after step) do not encode
+// theirs again (encoding costs a few microseconds of host time per map, five maps per attention call).
+namespace {
+struct MapKey {
+    const void *base;
+    uint64_t a, b, c;
+    uint32_t box1, box2, rank;
+};
+struct MapEntry {
+    MapKey key;
+    CUtensorMap map;
+    bool used;
+};
+constexpr int MAP_CACHE = 128;
+std::mutex map_mu;
+MapEntry map_cache[MAP_CACHE];
+unsigned map_next = 0;
+
+bool map_lookup(const MapKey &k, CUtensorMap *out) {
+    std::lock_guard<std::mutex> lock(map_mu);
+    for (int i = 0; i < MAP_CACHE; ++i)
+        if (map_cache[i].used && memcmp(&map_cache[i].key, &k, sizeof(MapKey)) == 0) {
+            *out = map_cache[i].map;
+            return true;
+        }
+    return false;
+}
+void map_store(const MapKey &k, const CUtensorMap &m) {
+    std::lock_guard<std::mutex> lock(map_mu);
+    MapEntry &e = map_cache[map_next++ % MAP_CACHE];
+    e.key = k;
+    e.map = m;
+    e.used = true;
+}
+}  // namespace
 
 // ------------------------------------------------------------------------------ tensor maps
 
@@ -25,6 +66,16 @@ static EncodeTiledFn encode_tiled_fn() {
 // 3-D bf16 tensor [n2, n1, n0] (n0 innermost, contiguous), box [box2, box1, 64], 128-byte swizzle.
 int make_tmap_3d_bf16(CUtensorMap *map, const void *base, uint64_t n0, uint64_t n1, uint64_t n2, uint32_t box1,
                       uint32_t box2) {
+    MapKey key;
+    memset(&key, 0, sizeof(key));
+    key.base = base;
+    key.a = n0;
+    key.b = n1;
+    key.c = n2;
+    key.box1 = box1;
+    key.box2 = box2;
+    key.rank = 3;
+    if (map_lookup(key, map)) return SPECROLL_OK;
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return note_cuda_error(cudaErrorNotSupported);
     cuuint64_t dims[3] = {n0, n1, n2};
@@ -35,11 +86,21 @@ int make_tmap_3d_bf16(CUtensorMap *map, const void *base, uint64_t n0, uint64_t 
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return note_cuda_error(cudaErrorInvalidValue);
+    map_store(key, *map);
     return SPECROLL_OK;
 }
 
 int make_tmap_2d_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint64_t ld_elems,
                       uint32_t box_rows) {
+    MapKey key;
+    memset(&key, 0, sizeof(key));
+    key.base = base;
+    key.a = rows;
+    key.b = cols;
+    key.c = ld_elems;
+    key.box1 = box_rows;
+    key.rank = 2;
+    if (map_lookup(key, map)) return SPECROLL_OK;
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return note_cuda_error(cudaErrorNotSupported);
     cuuint64_t dims[2] = {cols, rows};
@@ -50,6 +111,7 @@ int make_tmap_2d_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return note_cuda_error(cudaErrorInvalidValue);
+    map_store(key, *map);
     return SPECROLL_OK;
 }
 

@@ -111,6 +111,47 @@ def test_reflex_clip_binds_only_above_threshold():
     assert (rel[0::2] < 0.05).all()
 
 
+def test_correction_before_the_heads_closed_form_abstention_clip_and_composition():
+    # the secondary form: one memory row and one ratio per sequence, applied to the last hidden state
+    w = I.scaled(I.WORKLOADS["tiny"], B=8)
+    x = I.propose_inputs(w, peaked=True)
+    hf = _f64(x["h"])
+    m1 = x["m"][:, 0, :].copy()
+    eps = 1e-6
+    # abstention: bit-identical hidden state
+    for kw in ({"m": m1, "alpha": np.zeros(w.B, np.float32)}, {"m": None, "alpha": None}):
+        o = ref.prehead(x["h"], kw["m"], kw["alpha"])
+        assert np.array_equal(o["ht"], x["h"]) and np.array_equal(o["hc"], hf)
+    # closed form of the step: |dh| = alpha |h| RMS(m) / (RMS(m) + eps), parallel to m
+    alpha = np.full(w.B, 0.03, np.float32)
+    o = ref.prehead(x["h"], m1, alpha, rms_eps=eps)
+    dh = o["hc"] - hf
+    mm = m1.astype(np.float64)
+    rms_m = np.sqrt((mm ** 2).mean(-1))
+    want = np.float64(np.float32(0.03)) * np.linalg.norm(hf, axis=-1) * rms_m / (rms_m + eps)
+    np.testing.assert_allclose(np.linalg.norm(dh, axis=-1), want, rtol=1e-12)
+    np.testing.assert_allclose((dh * mm).sum(-1) / (np.linalg.norm(dh, axis=-1) * np.linalg.norm(mm, axis=-1)), 1.0, rtol=1e-12)
+    assert np.array_equal(o["ht"], ref.round_bf16(o["hc"]))
+    # the clip binds exactly at clip_c |h| and only above it
+    alpha2 = np.where(np.arange(w.B) % 2 == 0, 0.05, 0.3).astype(np.float32)
+    o2 = ref.prehead(x["h"], m1, alpha2, clip_c=0.1)
+    rel = np.linalg.norm(o2["hc"] - hf, axis=-1) / np.linalg.norm(hf, axis=-1)
+    np.testing.assert_allclose(rel[1::2], 0.1, rtol=1e-12)
+    assert (rel[0::2] < 0.05).all() and (rel[0::2] > 0.0499).all()
+    # the proposal in this form = the ordinary proposal, without memory, run on the corrected hidden state
+    a = ref.propose(x["h"], x["anchor"], x["A"], x["bias"], x["W"], m1, alpha, x["parent"], x["u_draw"], k=w.k,
+                    pre_head=True)
+    b = ref.propose(o["ht"], x["anchor"], x["A"], x["bias"], x["W"], None, None, x["parent"], x["u_draw"], k=w.k)
+    for key in a:
+        assert np.array_equal(a[key], b[key]), key
+    # and it is not the per-head form: with the same memory for every head the two give different states
+    mk = np.repeat(m1[:, None, :], w.K, axis=1)
+    ak = np.repeat(alpha[:, None], w.K, axis=1)
+    post = ref.heads(x["h"], x["A"], x["bias"], m=mk, alpha=ak)["zc"]
+    pre = ref.heads(o["ht"], x["A"], x["bias"])["zc"]
+    assert np.abs(post - pre).max() > 1e-4
+
+
 def test_projection_against_numpy_and_topk_against_argsort():
     w = I.scaled(I.WORKLOADS["tiny"], B=3, V=777)
     x = I.propose_inputs(w, peaked=True)
