@@ -105,12 +105,19 @@ typedef struct {
     float ln_eps;      /* LayerNorm epsilon (1e-5 if the caller has no other value) */
     float rms_eps;     /* epsilon of the RMS normalisation of the memory */
     float clip_c;      /* <= 0: no L2 clip */
-    int32_t flags;     /* 0, or SPECROLL_PROPOSE_LEGACY_MMA */
+    int32_t flags;     /* 0, or an OR of the SPECROLL_PROPOSE_* / SPECROLL_REFLEX_* flags below */
 } specroll_propose_desc;
 
 /* Run the vocabulary projection on the mma.sync kernel instead of the tcgen05 one (kept for
  * comparison and for k > 8, where it is used anyway). */
 #define SPECROLL_PROPOSE_LEGACY_MMA 1
+/* Secondary form of the bounded correction (Sec. 3.4 Eq. "reflex-correction" applied once, to the last
+ * hidden state, before the heads; the paper's own form corrects each head's output and is the default):
+ *   h~_b = bf16(h_b + alpha_b RMS(h_b) m_b / (RMS(m_b) + rms_eps)),  |h~_b - h_b|_2 <= clip_c |h_b|_2,
+ * the heads and the projection then run on h~ and their outputs are not corrected.  With this flag
+ * m is [B, d] and alpha is [B] (one memory row and one ratio per sequence); alpha_b = 0 or NULL
+ * leaves h_b untouched bit for bit. */
+#define SPECROLL_REFLEX_PRE_HEAD 2
 
 size_t specroll_propose_workspace_bytes(const specroll_propose_desc *desc);
 

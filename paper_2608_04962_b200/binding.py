@@ -34,6 +34,7 @@ EXPORTS = ("specroll_version", "specroll_strerror", "specroll_node_budget", "spe
 
 
 PROPOSE_LEGACY_MMA = 1
+REFLEX_PRE_HEAD = 2
 ATTN_LEGACY_MMA = 1
 ATTN_REUSE_PLAN = 2
 ATTN_CACHE_SETTLED = 4
@@ -177,8 +178,8 @@ def node_budget(C_hw: int, B_active: int, N_min: int = 1, N_max: int = 10) -> in
 
 
 def propose_workspace_bytes(B, N, K, k, d, V, temperature=1.0, ln_eps=1e-5, rms_eps=1e-6,
-                            clip_c=0.0) -> int:
-    desc = ProposeDesc(B, N, K, k, d, V, temperature, ln_eps, rms_eps, clip_c, 0)
+                            clip_c=0.0, flags=0) -> int:
+    desc = ProposeDesc(B, N, K, k, d, V, temperature, ln_eps, rms_eps, clip_c, flags)
     return int(lib().specroll_propose_workspace_bytes(C.byref(desc)))
 
 
@@ -195,10 +196,16 @@ def propose(h, anchor, A, bias, W, m, alpha, parent, u_draw, k, temperature=1.0,
         raise SpecrollError("propose: inconsistent weight shapes")
     if tuple(u_draw.shape) != (B, N) or tuple(anchor.shape) != (B,):
         raise SpecrollError("propose: inconsistent u_draw / anchor shapes")
-    if m is not None and tuple(m.shape) != (B, K, d):
-        raise SpecrollError("propose: m must be [B,K,d]")
-    if alpha is not None and tuple(alpha.shape) != (B, K):
-        raise SpecrollError("propose: alpha must be [B,K]")
+    if flags & REFLEX_PRE_HEAD:
+        if m is not None and tuple(m.shape) != (B, d):
+            raise SpecrollError("propose: with REFLEX_PRE_HEAD m must be [B,d]")
+        if alpha is not None and tuple(alpha.shape) != (B,):
+            raise SpecrollError("propose: with REFLEX_PRE_HEAD alpha must be [B]")
+    else:
+        if m is not None and tuple(m.shape) != (B, K, d):
+            raise SpecrollError("propose: m must be [B,K,d]")
+        if alpha is not None and tuple(alpha.shape) != (B, K):
+            raise SpecrollError("propose: alpha must be [B,K]")
     desc = ProposeDesc(B, N, K, k, d, V, temperature, ln_eps, rms_eps, clip_c, flags)
     dev = h.device
     if out is None:

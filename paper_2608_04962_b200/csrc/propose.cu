@@ -124,6 +124,36 @@ reflex_kernel(const float *__restrict__ z, const float *__restrict__ m, const fl
     }
 }
 
+// Secondary form of the correction (SPECROLL_REFLEX_PRE_HEAD): applied to the last hidden state, one memory row
+// and one ratio per sequence.  ht[b,:] = bf16(h[b,:] + coef * m[b,:]), coef = alpha RMS(h) / (RMS(m) + eps), shrunk
+// so that |coef * m|_2 <= clip_c * |h|_2; alpha = 0 or no memory: ht = h bit for bit.
+__global__ void __launch_bounds__(RX_THREADS)
+prehead_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict__ m, const float *__restrict__ alpha,
+               __nv_bfloat16 *__restrict__ ht, int d, float rms_eps, float clip_c) {
+    __shared__ float red[RX_THREADS / 32];
+    const size_t r = blockIdx.x;
+    const __nv_bfloat16 *hr = h + r * d;
+    const float a = (alpha && m) ? alpha[r] : 0.f;
+    if (a != 0.f) {  // uniform across the block
+        const float *mr = m + r * d;
+        float sh = 0.f, sm = 0.f;
+        for (int i = threadIdx.x; i < d; i += RX_THREADS) {
+            const float hv = __bfloat162float(hr[i]), mv = mr[i];
+            sh += hv * hv;
+            sm += mv * mv;
+        }
+        sh = block_sum<RX_THREADS>(sh, red);
+        sm = block_sum<RX_THREADS>(sm, red);
+        const float rms_h = sqrtf(sh / d), rms_m = sqrtf(sm / d);
+        float coef = a * rms_h / (rms_m + rms_eps);
+        const float nd = fabsf(coef) * sqrtf(sm), nh = sqrtf(sh);
+        if (clip_c > 0.f && nd > clip_c * nh) coef *= clip_c * nh / nd;
+        for (int i = threadIdx.x; i < d; i += RX_THREADS) ht[r * d + i] = __float2bfloat16_rn(__bfloat162float(hr[i]) + coef * mr[i]);
+    } else {
+        for (int i = threadIdx.x; i < d; i += RX_THREADS) ht[r * d + i] = hr[i];
+    }
+}
+
 // ------------------------------------------------------------------------------ P4 projection + top-k
 
 // Sorted (descending value; earlier insertion wins ties) list of the KMAX best seen so far.
@@ -358,7 +388,7 @@ tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__rest
 struct ProposePlan {
     int KX, M, n_mblocks, n_tiles, n_groups, tiles_per_group;
     bool use_tc;  // tcgen05 projection kernel (k <= 8); otherwise the mma.sync one
-    size_t off_status, off_xhat, off_z, off_zt, off_pval, off_pid, total;
+    size_t off_status, off_xhat, off_z, off_zt, off_pval, off_pid, off_hc, total;
 };
 
 // head_mlp_tc.cu
@@ -373,7 +403,7 @@ static int make_plan(const specroll_propose_desc *d, bool affine, ProposePlan *p
     if (!d || d->B < 0 || d->N < 1 || d->N > SPECROLL_MAX_NODES || d->K < 1 || d->K > SPECROLL_MAX_HEADS ||
         d->k < 1 || d->k > SPECROLL_MAX_TOPK || d->d < 64 || (d->d % 64) || d->V < 8 || (d->V % 8) ||
         d->k > d->V || !(d->temperature > 0.f) || !(d->ln_eps >= 0.f) || !(d->rms_eps >= 0.f) ||
-        (d->flags & ~SPECROLL_PROPOSE_LEGACY_MMA) != 0 || d->d > 12288)
+        (d->flags & ~(SPECROLL_PROPOSE_LEGACY_MMA | SPECROLL_REFLEX_PRE_HEAD)) != 0 || d->d > 12288)
         return SPECROLL_EINVAL;
     p->KX = affine ? d->K : 1;
     p->M = d->B * d->K;
@@ -400,6 +430,8 @@ static int make_plan(const specroll_propose_desc *d, bool affine, ProposePlan *p
     o += align_up((size_t)p->M * p->n_groups * k * 4, 256);
     p->off_pid = o;
     o += align_up((size_t)p->M * p->n_groups * k * 4, 256);
+    p->off_hc = o;  // the corrected hidden state of the pre-head form
+    if (d->flags & SPECROLL_REFLEX_PRE_HEAD) o += align_up(B * dd * 2, 256);
     p->total = o + 256;
     return SPECROLL_OK;
 }
@@ -484,6 +516,15 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
     const int B = d->B, K = d->K, dd = d->d, k = d->k, V = d->V;
     int32_t *status = reinterpret_cast<int32_t *>(ws + p.off_status);
     SR_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int32_t), st));
+    const bool pre_head = (d->flags & SPECROLL_REFLEX_PRE_HEAD) != 0;
+    if (pre_head) {
+        // the correction moves the hidden state itself (m [B, d], alpha [B]); everything after it reads the
+        // corrected state, and the heads' outputs are not corrected again
+        __nv_bfloat16 *hc = reinterpret_cast<__nv_bfloat16 *>(ws + p.off_hc);
+        prehead_kernel<<<B, RX_THREADS, 0, st>>>(hb, m, alpha, hc, dd, d->rms_eps, d->clip_c);
+        SR_LAUNCH_CHECK();
+        hb = hc;
+    }
 
     layernorm_kernel<<<B, LN_THREADS, dd * sizeof(float), st>>>(
         hb, static_cast<const __nv_bfloat16 *>(ln_gamma), static_cast<const __nv_bfloat16 *>(ln_beta), xhat, B,
@@ -503,7 +544,8 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
         SR_LAUNCH_CHECK();
     }
 
-    reflex_kernel<<<B * K, RX_THREADS, 0, st>>>(z, m, alpha, zt, dd, d->rms_eps, d->clip_c);
+    reflex_kernel<<<B * K, RX_THREADS, 0, st>>>(z, pre_head ? nullptr : m, pre_head ? nullptr : alpha, zt, dd, d->rms_eps,
+                                               d->clip_c);
     SR_LAUNCH_CHECK();
 
     {

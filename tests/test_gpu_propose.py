@@ -125,6 +125,35 @@ def test_reflex_abstain_clip_and_affine_layernorm():
     check_candidates(w, x, g2, logit_atol=LOGIT_ATOL, gamma=gam, beta=bet)
 
 
+def test_correction_before_the_heads():
+    # secondary form of the bounded correction: one memory row and ratio per sequence, applied to h; the heads
+    # then run on the corrected state (the oracle's own pins fix that composition on the CPU)
+    w = I.scaled(I.WORKLOADS["qwen1.5b"], B=70, K=4, k=8, d=640, V=4104, N=16)
+    x = I.propose_inputs(w, peaked=True)
+    gg = I.rng(77)
+    m = gg.standard_normal((w.B, w.d)).astype(np.float32)
+    alpha = gg.uniform(0.02, 0.3, w.B).astype(np.float32)
+    alpha[::5] = 0.0                                          # some sequences abstain
+    for clip_c in (0.0, 0.05):                                # unclipped; clip binding for the larger ratios
+        wc = I.scaled(w, clip_c=clip_c)
+        ht = ref.prehead(x["h"], m, alpha, clip_c=clip_c)["ht"]
+        assert (ht[::5] == x["h"][::5]).all() and (ht[1] != x["h"][1]).any()
+        g = gpu_propose(wc, dict(x, m=m, alpha=alpha), flags=S.REFLEX_PRE_HEAD)
+        xo = dict(x, h=ht, m=None, alpha=None)
+        same, oid, ol = check_candidates(wc, xo, g, logit_atol=LOGIT_ATOL)
+        check_tree(wc, xo, g, same, oid=oid, ol=ol)
+        assert same.mean() > 0.9
+    # every ratio zero, or no memory at all: bit for bit the uncorrected proposal
+    g_plain = gpu_propose(w, dict(x, m=None, alpha=None))
+    for mm, aa in ((m, np.zeros(w.B, np.float32)), (None, None)):
+        g0 = gpu_propose(w, dict(x, m=mm, alpha=aa), flags=S.REFLEX_PRE_HEAD)
+        for key in ("cand_id", "cand_logit", "tree_tok", "tree_cand", "slot_q"):
+            assert np.array_equal(g0[key], g_plain[key]), key
+    # the per-head shapes of the default form are refused under the flag
+    with pytest.raises(S.SpecrollError):
+        gpu_propose(w, x, flags=S.REFLEX_PRE_HEAD)
+
+
 def test_tree_draw_alone_matches_exactly():
     for name in ("qwen1.5b", "qwen7b", "qwen14b"):
         w = I.scaled(I.WORKLOADS[name], B=200)
