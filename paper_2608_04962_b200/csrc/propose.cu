@@ -287,7 +287,7 @@ topk_merge_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pi
 
 // ------------------------------------------------------------------------------ P5 tree draw
 
-constexpr int DRAW_WARPS = 4;
+constexpr int DRAW_WARPS = 8;
 
 __device__ __forceinline__ double warp_incl_scan_f64(double v, int lane) {
 #pragma unroll
@@ -298,11 +298,12 @@ __device__ __forceinline__ double warp_incl_scan_f64(double v, int lane) {
     return v;
 }
 
-// One warp per sequence.  The nodes are drawn one after the other (a child's distribution depends on what its
-// earlier siblings took), but within a node the work over the k candidates is spread over the lanes (lane j holds
+// One CTA per sequence, one warp per parent node.  A child's distribution depends on what its earlier siblings
+// drew and on nothing else, so the children of different parents are drawn at the same time and only siblings
+// wait for each other; within a draw the work over the k candidates is spread over the lanes (lane j holds
 // candidates j and j + 32): their total, the running sums of the inverse-CDF walk and the first candidate whose
-// running sum exceeds the uniform come from warp scans and ballots.  (With k-long fp64 loops on one lane a draw of
-// 48 nodes took 40 us.)
+// running sum exceeds the uniform come from warp scans and ballots.  (Node after node on one warp, a draw of 48
+// nodes took 32 us: some twenty dependent fp64 operations and shuffles per node.)
 __global__ void __launch_bounds__(DRAW_WARPS * 32)
 tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__restrict__ anchor,
                  const int32_t *__restrict__ cand_id, const float *__restrict__ cand_logit,
@@ -310,76 +311,88 @@ tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__rest
                  uint8_t *__restrict__ tree_cand, float *__restrict__ slot_q) {
     // Softmax weights of every head's candidates, relative to the head's largest logit, once per sequence: a
     // child's distribution is these weights renormalised over the candidates its earlier siblings left.
-    __shared__ double sh_w[DRAW_WARPS][SPECROLL_MAX_HEADS][SPECROLL_MAX_TOPK];
-    __shared__ unsigned long long sh_taken[DRAW_WARPS][SPECROLL_MAX_NODES];
-    // the candidates' token ids, so that the loop over the nodes reads nothing from global memory (a load whose
-    // value the same iteration stores holds the warp for a memory round trip per node)
-    __shared__ int32_t sh_id[DRAW_WARPS][SPECROLL_MAX_HEADS][SPECROLL_MAX_TOPK];
+    __shared__ double sh_w[SPECROLL_MAX_HEADS][SPECROLL_MAX_TOPK];
+    __shared__ int32_t sh_id[SPECROLL_MAX_HEADS][SPECROLL_MAX_TOPK];
+    __shared__ float sh_u[SPECROLL_MAX_NODES];
+    __shared__ int8_t sh_parent[SPECROLL_MAX_NODES];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.x * DRAW_WARPS + warp;
-    if (b >= B) return;
+    const int b = blockIdx.x;
     const int N = topo.N;
-    for (int hd = 0; hd < K; ++hd) {
+    const double inv_T = 1.0 / T;  // (the largest logit minus itself over T would be a division with a zero numerator)
+    for (int hd = warp; hd < K; hd += DRAW_WARPS) {
         const float *cl = cand_logit + ((size_t)b * K + hd) * k;
         float mxf = -INFINITY;
         for (int j = lane; j < k; j += 32) mxf = fmaxf(mxf, cl[j]);
         mxf = warp_max(mxf);
         for (int j = lane; j < k; j += 32) {
-            sh_w[warp][hd][j] = exp(((double)cl[j] - (double)mxf) / T);
-            sh_id[warp][hd][j] = cand_id[((size_t)b * K + hd) * k + j];
+            sh_w[hd][j] = exp(((double)cl[j] - (double)mxf) * inv_T);
+            sh_id[hd][j] = cand_id[((size_t)b * K + hd) * k + j];
         }
     }
-    for (int n = lane; n < N; n += 32) sh_taken[warp][n] = 0ull;
-    // the uniforms of the sequence's nodes, one round of loads (lane n holds nodes n and n + 32)
-    const float u_lo = lane < N ? u_draw[(size_t)b * N + lane] : 0.f;
-    const float u_hi = lane + 32 < N ? u_draw[(size_t)b * N + lane + 32] : 0.f;
-    __syncwarp();
-    if (lane == 0) {
+    for (int n = threadIdx.x; n < N; n += DRAW_WARPS * 32) {
+        sh_u[n] = u_draw[(size_t)b * N + n];
+        sh_parent[n] = topo.parent[n];
+    }
+    if (threadIdx.x == 0) {
         tree_tok[(size_t)b * N] = anchor[b];
         tree_cand[(size_t)b * N] = 255;
         slot_q[(size_t)b * N] = 1.0f;
     }
-    for (int n = 1; n < N; ++n) {
-        const int u = topo.parent[n], hd = topo.depth[n] - 1;
-        const double *w = sh_w[warp][hd];
-        const unsigned long long taken = sh_taken[warp][u];
-        const bool ok0 = lane < k && !((taken >> lane) & 1ull);
-        const bool ok1 = lane + 32 < k && !((taken >> (lane + 32)) & 1ull);
-        double w0 = ok0 ? w[lane] : 0.0, w1 = ok1 ? w[lane + 32] : 0.0;
-        double s = warp_sum(w0 + w1);
-        if (!(s > 0.0)) {
-            // every remaining weight underflowed against a taken candidate's logit: take the reference among
-            // the remaining ones instead (the head's table is shared by all parents of this depth, whose taken
-            // sets differ, so the weights of this one draw stay in registers)
-            const float *cl = cand_logit + ((size_t)b * K + hd) * k;
-            float mxf = fmaxf(ok0 ? cl[lane] : -INFINITY, ok1 ? cl[lane + 32] : -INFINITY);
-            mxf = warp_max(mxf);
-            w0 = ok0 ? exp(((double)cl[lane] - (double)mxf) / T) : 0.0;
-            w1 = ok1 ? exp(((double)cl[lane + 32] - (double)mxf) / T) : 0.0;
-            s = warp_sum(w0 + w1);
+    __syncthreads();
+    int idx = 0;
+    for (int u = 0; u < N; ++u) {
+        if (topo.n_child[u] == 0) continue;
+        if ((idx++ % DRAW_WARPS) != warp) continue;
+        const int hd = topo.depth[u];  // the children of u are drawn by head depth(u) (0-based)
+        const double *w = sh_w[hd];
+        // children of u (a child's index is larger than its parent's), in slot order
+        const unsigned cm_lo = __ballot_sync(0xffffffffu, lane > u && lane < N && sh_parent[lane < N ? lane : 0] == u);
+        const unsigned cm_hi =
+            __ballot_sync(0xffffffffu, lane + 32 > u && lane + 32 < N && sh_parent[lane + 32 < N ? lane + 32 : 0] == u);
+        unsigned long long cm = ((unsigned long long)cm_hi << 32) | cm_lo;
+        unsigned long long taken = 0ull;
+        while (cm) {
+            const int n = __ffsll((long long)cm) - 1;
+            cm &= cm - 1;
+            const bool ok0 = lane < k && !((taken >> lane) & 1ull);
+            const bool ok1 = lane + 32 < k && !((taken >> (lane + 32)) & 1ull);
+            double w0 = ok0 ? w[lane] : 0.0, w1 = ok1 ? w[lane + 32] : 0.0;
+            // running sums over the remaining candidates; their total is the last one
+            double c0 = warp_incl_scan_f64(w0, lane);
+            double c1 = __shfl_sync(0xffffffffu, c0, 31);
+            if (k > 32) c1 += warp_incl_scan_f64(w1, lane);
+            double s = __shfl_sync(0xffffffffu, c1, 31);
+            if (!(s > 0.0)) {
+                // every remaining weight underflowed against a taken candidate's logit: take the reference among
+                // the remaining ones instead
+                const float *cl = cand_logit + ((size_t)b * K + hd) * k;
+                float mxf = fmaxf(ok0 ? cl[lane] : -INFINITY, ok1 ? cl[lane + 32] : -INFINITY);
+                mxf = warp_max(mxf);
+                w0 = ok0 ? exp(((double)cl[lane] - (double)mxf) * inv_T) : 0.0;
+                w1 = ok1 ? exp(((double)cl[lane + 32] - (double)mxf) * inv_T) : 0.0;
+                c0 = warp_incl_scan_f64(w0, lane);
+                c1 = __shfl_sync(0xffffffffu, c0, 31) + warp_incl_scan_f64(w1, lane);
+                s = __shfl_sync(0xffffffffu, c1, 31);
+            }
+            // first remaining candidate whose cumulative probability exceeds the uniform (compared as masses)
+            const double thr = (double)sh_u[n] * s;
+            const unsigned hit0 = __ballot_sync(0xffffffffu, ok0 && c0 > thr), hit1 = __ballot_sync(0xffffffffu, ok1 && c1 > thr);
+            const unsigned v0 = __ballot_sync(0xffffffffu, ok0), v1 = __ballot_sync(0xffffffffu, ok1);
+            int sel;
+            if (hit0)
+                sel = __ffs(hit0) - 1;
+            else if (hit1)
+                sel = 32 + __ffs(hit1) - 1;
+            else
+                sel = v1 ? 32 + (31 - __clz(v1)) : (31 - __clz(v0));  // none: the last remaining candidate
+            const double wsel = __shfl_sync(0xffffffffu, sel < 32 ? w0 : w1, sel & 31);
+            taken |= 1ull << sel;
+            if (lane == 0) {
+                tree_tok[(size_t)b * N + n] = sh_id[hd][sel];
+                tree_cand[(size_t)b * N + n] = (uint8_t)sel;
+                slot_q[(size_t)b * N + n] = (float)(wsel / s);
+            }
         }
-        // first remaining candidate whose cumulative probability exceeds the uniform (compared as masses)
-        const float un = __shfl_sync(0xffffffffu, n < 32 ? u_lo : u_hi, n & 31);
-        const double thr = (double)un * s;
-        const double c0 = warp_incl_scan_f64(w0, lane);
-        const double c1 = __shfl_sync(0xffffffffu, c0, 31) + warp_incl_scan_f64(w1, lane);
-        const unsigned hit0 = __ballot_sync(0xffffffffu, ok0 && c0 > thr), hit1 = __ballot_sync(0xffffffffu, ok1 && c1 > thr);
-        const unsigned v0 = __ballot_sync(0xffffffffu, ok0), v1 = __ballot_sync(0xffffffffu, ok1);
-        int sel;
-        if (hit0)
-            sel = __ffs(hit0) - 1;
-        else if (hit1)
-            sel = 32 + __ffs(hit1) - 1;
-        else
-            sel = v1 ? 32 + (31 - __clz(v1)) : (31 - __clz(v0));  // none: the last remaining candidate
-        const double wsel = __shfl_sync(0xffffffffu, sel < 32 ? w0 : w1, sel & 31);
-        if (lane == 0) {
-            sh_taken[warp][u] = taken | (1ull << sel);
-            tree_tok[(size_t)b * N + n] = sh_id[warp][hd][sel];
-            tree_cand[(size_t)b * N + n] = (uint8_t)sel;
-            slot_q[(size_t)b * N + n] = (float)(wsel / s);
-        }
-        __syncwarp();
     }
 }
 
@@ -446,7 +459,7 @@ static int launch_tree_draw(const Topo &topo, int B, int K, int k, float T, cons
                             const int32_t *cand_id, const float *cand_logit, const float *u_draw,
                             int32_t *tree_tok, uint8_t *tree_cand, float *slot_q, cudaStream_t st) {
     if (B == 0) return SPECROLL_OK;
-    tree_draw_kernel<<<(B + DRAW_WARPS - 1) / DRAW_WARPS, DRAW_WARPS * 32, 0, st>>>(
+    tree_draw_kernel<<<B, DRAW_WARPS * 32, 0, st>>>(
         topo, B, K, k, (double)T, anchor, cand_id, cand_logit, u_draw, tree_tok, tree_cand, slot_q);
     SR_LAUNCH_CHECK();
     return SPECROLL_OK;

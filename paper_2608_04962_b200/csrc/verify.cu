@@ -51,23 +51,111 @@ __device__ __forceinline__ void online_update(const uint4 &v, float c, float &m,
     s += acc;
 }
 
+// As online_update, with a second sum (of the current slice; SL) kept relative to the same running maximum.
+template <bool SL>
+__device__ __forceinline__ void online_update_slice(const uint4 &v, float c, float &m, float &s, float &sl) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float x[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        x[2 * i] = __uint_as_float(w[i] << 16);
+        x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+    float vm = x[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) vm = fmaxf(vm, x[i]);
+    if (vm > m) {
+        const float f = ex2_approx((m - vm) * c);  // m = -inf gives 0
+        s *= f;
+        if (SL) sl *= f;
+        m = vm;
+    }
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc += ex2_approx((x[i] - m) * c);
+    s += acc;
+    if (SL) sl += acc;
+}
+
+// How the statistics kernel cuts a row: groups of 128 8-token vectors (four loads of 32 consecutive vectors by one
+// warp); each of the kernel's warps takes one contiguous run of groups (gpw of them, the last warp what is left); a
+// run is cut into slices of up to four groups (4096 tokens).  Slices are numbered warp by warp, so in token order;
+// a warp with a short run has empty slices at its end.
+constexpr int RS_WARPS = RS_THREADS / 32;
+struct RowSlices {
+    int nvec, G, gpw, spw, n_sl;
+    __host__ __device__ explicit RowSlices(int V) {
+        nvec = V >> 3;
+        G = (nvec + 127) / 128;
+        gpw = (G + RS_WARPS - 1) / RS_WARPS;
+        spw = (gpw + 3) / 4;
+        n_sl = RS_WARPS * spw;
+    }
+    // groups [g_lo, g_hi) of slice t of warp w (empty: g_lo >= g_hi)
+    __host__ __device__ void groups(int w, int t, int *g_lo, int *g_hi) const {
+        const int run_hi = min_((w + 1) * gpw, G);
+        *g_lo = w * gpw + 4 * t;
+        *g_hi = min_(run_hi, *g_lo + 4);
+    }
+    // vectors [v_lo, v_hi) of slice s
+    __host__ __device__ void vectors(int s, int *v_lo, int *v_hi) const {
+        int g_lo, g_hi;
+        groups(s / spw, s % spw, &g_lo, &g_hi);
+        *v_lo = min_(nvec, g_lo * 128);
+        *v_hi = g_hi > g_lo ? min_(nvec, g_hi * 128) : *v_lo;
+    }
+    __host__ __device__ int slice_of_token(int tok) const {
+        const int g = (tok >> 3) / 128, w = g / gpw;
+        return w * spw + (g - w * gpw) / 4;
+    }
+    static __host__ __device__ int min_(int a, int b) { return a < b ? a : b; }
+};
+__host__ __device__ inline int row_slices(int V) { return RowSlices(V).n_sl; }
+
 // logits[rows, V] bf16; c = log2(e) / T.  row_max = max_v l_v, row_sum = sum_v exp((l_v - max)/T).
-__global__ void __launch_bounds__(RS_THREADS)
+// TAB: every slice also leaves tab[row, slice] = (R, sum over the slice of exp((l_v - R)/T)) with some R >= the
+// slice's logits: the terminal draw of a row then needs this table and one slice of the row instead of the row.
+// (The two warp reductions per slice are why a slice is as long as it is: the shuffle unit passes one warp
+// instruction per clock per SM, and ten shuffles per 1024 tokens cost a tenth of the kernel's time.)
+template <bool TAB>
+__global__ void __launch_bounds__(RS_THREADS, 8)
 row_stats_kernel(const uint16_t *__restrict__ logits, int V, float c, float *__restrict__ row_max,
-                 float *__restrict__ row_sum) {
+                 float *__restrict__ row_sum, float2 *__restrict__ tab) {
+    // a kernel launched behind this one as its programmatic dependent may start its own prologue as SMs free up; it
+    // waits for this grid's completion before it reads the statistics
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const size_t row = blockIdx.x;
     const uint4 *p = reinterpret_cast<const uint4 *>(logits + row * (size_t)V);
-    const int nvec = V >> 3;
+    const RowSlices rs(V);
+    const int nvec = rs.nvec;
     float m = NEG_INF, s = 0.f;
-    int i = threadIdx.x;
-    for (; i + (RS_UNROLL - 1) * RS_THREADS < nvec; i += RS_UNROLL * RS_THREADS) {
-        uint4 v[RS_UNROLL];
+    {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int t = 0; t < rs.spw; ++t) {
+            int g_lo, g_hi;
+            rs.groups(warp, t, &g_lo, &g_hi);
+            float sl = 0.f;
+#pragma unroll 1
+            for (int g = g_lo; g < g_hi; ++g) {
+                const int i0 = g * 128 + lane;
+                if (i0 + 3 * 32 < nvec) {  // (for lane 31: the whole group is inside the row)
+                    uint4 v[4];
 #pragma unroll
-        for (int u = 0; u < RS_UNROLL; ++u) v[u] = ld_nc_v4(p + i + u * RS_THREADS);
+                    for (int q = 0; q < 4; ++q) v[q] = ld_nc_v4(p + i0 + q * 32);
 #pragma unroll
-        for (int u = 0; u < RS_UNROLL; ++u) online_update(v[u], c, m, s);
+                    for (int q = 0; q < 4; ++q) online_update_slice<TAB>(v[q], c, m, s, sl);
+                } else {
+                    for (int q = 0; q < 4; ++q)
+                        if (i0 + q * 32 < nvec) online_update_slice<TAB>(ld_nc_v4(p + i0 + q * 32), c, m, s, sl);
+                }
+            }
+            if (TAB) {
+                const float R = warp_max(m);  // >= everything the warp has seen, this slice included
+                const float tot = warp_sum((m == NEG_INF) ? 0.f : sl * ex2_approx((m - R) * c));
+                if (lane == 0) tab[row * rs.n_sl + warp * rs.spw + t] = make_float2(R, tot);
+            }
+        }
     }
-    for (; i < nvec; i += RS_THREADS) online_update(ld_nc_v4(p + i), c, m, s);
 
     // warp, then block reduction of (m, s)
     float mw = warp_max(m);
@@ -359,6 +447,10 @@ struct WalkSmem {
     float cl[SPECROLL_MAX_TOPK];
     int32_t id[SPECROLL_MAX_TOPK];
     double bc[2];  // broadcast slots: current max, accepted flag
+    // per child of the node at hand (walk_node): 1 / s_i, the candidates taken before it, its own candidate
+    double inv_s[32];
+    uint32_t taken[32];
+    int32_t jc[32];
 };
 
 // Everything the walk of one sequence can read, staged in shared memory in one round of independent loads (the
@@ -372,6 +464,11 @@ struct WalkStage {
     const int32_t *cid;               // [K, k]
     const float *clog;                // [K, k]
     const uint16_t *pre;              // [N, k]
+    // optional (nullptr: computed per node): the tree's parent array, the proposal weights exp((c_j - max c)/T) of
+    // every head's candidates, the target probabilities of every walkable node's candidates
+    const int8_t *parent;  // [N]
+    const double *e;       // [K, k]
+    const double *p;       // [N, k]
 };
 
 __device__ __forceinline__ void walk_begin(const WalkArgs &a, int b, int lane, WalkState *st) {
@@ -392,8 +489,10 @@ __device__ __forceinline__ void walk_begin(const WalkArgs &a, int b, int lane, W
 // S is the normaliser and thr the nucleus threshold key (0: none) of u's row - then u's children in slot order.
 // Returns the accepted child, or -1 when every child was rejected (the residual is then in sm->r, st->sigma).
 // sg (nullable): the sequence's inputs staged in shared memory.
-__device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, double M, double S, uint32_t thr, int lane,
-                         WalkSmem *sm, WalkState *st, const WalkStage *sg = nullptr) {
+// emit = false: nothing is written to the results and the count of accepted tokens stays (the node is examined
+// on its own, before it is known whether the walk reaches it).
+__device__ int walk_node_seq(const WalkArgs &a, const Topo &topo, int b, int u, double M, double S, uint32_t thr,
+                                           int lane, WalkSmem *sm, WalkState *st, const WalkStage *sg, bool emit) {
     double *r = sm->r, *w = sm->w;
     float *cl = sm->cl;
     int32_t *id = sm->id;
@@ -401,13 +500,17 @@ __device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, doub
     const int hd = topo.depth[u];
     const uint16_t *lg = a.logits ? a.logits + ((size_t)b * N + u) * a.V : nullptr;
     const uint16_t *ct = a.cand_target ? a.cand_target + ((size_t)b * N + u) * k : nullptr;
+    // Quotients whose numerator can be exactly zero (the largest logit minus itself, a taken candidate's weight, a
+    // residual entry clamped to zero) are formed as products with a reciprocal: a double division with a zero
+    // numerator leaves the division's fast path, and one lane on the slow path holds up the whole warp at every slot.
+    const double inv_T = 1.0 / a.T, inv_S = 1.0 / S;
     for (int j = lane; j < k; j += 32) {
         const int t = sg ? sg->cid[hd * k + j] : SR_CHECKED(a.cand_id[((size_t)b * K + hd) * k + j], a.V, b);
         id[j] = t;
         cl[j] = sg ? sg->clog[hd * k + j] : a.cand_logit[((size_t)b * K + hd) * k + j];
         const uint32_t bits = sg ? sg->pre[u * k + j] : (lg ? lg[t] : ct[j]);
         const double l = (double)bf16_bits_to_float((uint16_t)bits);
-        r[j] = ord_key(bits) >= thr ? exp((l - M) / a.T) / S : 0.0;  // r = p_u on the candidates
+        r[j] = ord_key(bits) >= thr ? exp((l - M) * inv_T) * inv_S : 0.0;  // r = p_u on the candidates
     }
     __syncwarp();
     // Every lane holds one or two of the k candidates (j = lane, lane + 32); sums and maxima over the candidates
@@ -432,16 +535,17 @@ __device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, doub
         for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         double s = 0.0;
         for (int j = lane; j < k; j += 32) {
-            w[j] = ((taken >> j) & 1) ? 0.0 : exp(((double)cl[j] - mx) / a.T);
+            w[j] = ((taken >> j) & 1) ? 0.0 : exp(((double)cl[j] - mx) * inv_T);
             s += w[j];
         }
         s = warp_sum(s);
+        const double inv_s = 1.0 / s;
         __syncwarp();
         const int jc = SR_CHECKED((int)(sg ? sg->tcand[c] : a.tree_cand[(size_t)b * N + c]), k, b);
-        const double qy = w[jc] / s;
+        const double qy = w[jc] * inv_s;
         double ratio;
         if (qy > 0.0)
-            ratio = r[jc] / qy;
+            ratio = r[jc] > 0.0 ? r[jc] / qy : 0.0;
         else
             ratio = (r[jc] > 0.0) ? INFINITY : 0.0;
         const double uu = (double)(sg ? sg->uacc[c] : a.u_acc[(size_t)b * N + c]);
@@ -453,20 +557,21 @@ __device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, doub
         } else {
             double Z = 0.0;
             for (int j = lane; j < k; j += 32) {
-                const double t = r[j] - w[j] / s;
+                const double t = r[j] - w[j] * inv_s;
                 w[j] = t > 0.0 ? t : 0.0;
                 Z += w[j];
             }
             Z = warp_sum(Z) + st->sigma * st->p_off;
             if (Z > 1e-300) {
-                for (int j = lane; j < k; j += 32) r[j] = w[j] / Z;
-                st->sigma /= Z;
+                const double inv_Z = 1.0 / Z;
+                for (int j = lane; j < k; j += 32) r[j] = w[j] * inv_Z;
+                st->sigma *= inv_Z;
             }
             __syncwarp();
         }
         taken |= 1ull << jc;
     }
-    if (accepted >= 0) {
+    if (accepted >= 0 && emit) {
         if (lane == 0) {
             a.out_tok[(size_t)b * (K + 1) + st->nacc] = sg ? sg->ttok[accepted] : a.tree_tok[(size_t)b * N + accepted];
             a.path_node[(size_t)b * (K + 1) + st->nacc + 1] = accepted;
@@ -476,15 +581,173 @@ __device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, doub
     return accepted;
 }
 
+// The same node with the slots' dependent chain cut to its minimum (k <= 32 candidates and <= 32 children; anything
+// else, and weights that underflow, go to walk_node_seq).  Lane j holds candidate j (replicated over the warp when
+// k < 32, so that a sum over the candidates is log2 k shuffle steps), lane i holds child i.
+//   - What a slot's proposal is does not depend on the decisions before it: child i sees the candidates its earlier
+//     siblings did not draw, q_i(j) = e_j / s_i with e_j = exp((c_j - max c)/T) and s_i the sum of the remaining e_j
+//     (the same quotient as with the maximum of the remaining ones as reference).  All s_i at once, before the chain.
+//   - The residual is carried unnormalised: r = rho / Zc.  A rejection gives rho_j <- max(rho_j - Zc q_i(j), 0) and
+//     Zc <- sum_j rho_j + p_off, where p_off (the target's mass outside the candidates) stays what it was: dividing
+//     by Zc gives back the normalised update, with sigma = 1 / Zc.  One fused multiply-add and one sum per slot.
+//   - The acceptance test of child i needs rho at its own candidate and Zc as they were when the chain reached it;
+//     lane i keeps them and all ratios are formed together after the chain, which runs over all children whether or
+//     not an earlier one is accepted (the first accepted child decides; what follows it is ignored).
+__device__ int walk_node(const WalkArgs &a, const Topo &topo, int b, int u, double M, double S, uint32_t thr, int lane,
+                         WalkSmem *sm, WalkState *st, const WalkStage *sg = nullptr, bool emit = true) {
+    const int k = a.k, N = a.N, K = a.K;
+    // children of u, in slot order
+    const int8_t *par = (sg && sg->parent) ? sg->parent : nullptr;  // (a lane-indexed read of the by-value struct is slow)
+    const unsigned cm_lo = __ballot_sync(
+        0xffffffffu, lane > u && lane < N && (par ? par[lane < N ? lane : 0] : topo.parent[lane < N ? lane : 0]) == u);
+    const unsigned cm_hi = __ballot_sync(0xffffffffu, lane + 32 > u && lane + 32 < N &&
+                                                          (par ? par[lane + 32 < N ? lane + 32 : 0]
+                                                               : topo.parent[lane + 32 < N ? lane + 32 : 0]) == u);
+    const int m_lo = __popc(cm_lo), m = m_lo + __popc(cm_hi);
+    if (k > 32 || m > 32) return walk_node_seq(a, topo, b, u, M, S, thr, lane, sm, st, sg, emit);
+    const int hd = topo.depth[u];
+    int kp = 1;
+    while (kp < k) kp <<= 1;
+    const int j = lane & (kp - 1);
+    const bool have = j < k;
+    const double inv_T = 1.0 / a.T, inv_S = 1.0 / S;
+    // the candidates: token, proposal weight, target probability
+    const bool staged = sg && sg->p && sg->e;
+    double rho = 0.0, e = 0.0;
+    if (staged) {
+        if (have) {
+            rho = sg->p[u * k + j];
+            e = sg->e[hd * k + j];
+            if (lane < k) sm->id[j] = sg->cid[hd * k + j];
+        }
+    } else {
+        float clj = -INFINITY;
+        if (have) {
+            const int tok = sg ? sg->cid[hd * k + j] : SR_CHECKED(a.cand_id[((size_t)b * K + hd) * k + j], a.V, b);
+            clj = sg ? sg->clog[hd * k + j] : a.cand_logit[((size_t)b * K + hd) * k + j];
+            uint32_t bits;
+            if (sg)
+                bits = sg->pre[u * k + j];
+            else if (a.logits)
+                bits = a.logits[((size_t)b * N + u) * a.V + tok];
+            else
+                bits = a.cand_target[((size_t)b * N + u) * k + j];
+            const double l = (double)bf16_bits_to_float((uint16_t)bits);
+            rho = ord_key(bits) >= thr ? exp((l - M) * inv_T) * inv_S : 0.0;
+            if (lane < k) sm->id[j] = tok;
+        }
+        float mxf = clj;
+        for (int o = kp >> 1; o > 0; o >>= 1) mxf = fmaxf(mxf, __shfl_xor_sync(0xffffffffu, mxf, o));
+        e = have ? exp(((double)clj - (double)mxf) * inv_T) : 0.0;
+    }
+    double pc = rho;
+    for (int o = kp >> 1; o > 0; o >>= 1) pc += __shfl_xor_sync(0xffffffffu, pc, o);
+    const double p_off = pc < 1.0 ? 1.0 - pc : 0.0;
+    // the children: lane i holds child i
+    int c_i = 0, jc_i = 0;
+    double uu_i = 0.0;
+    if (lane < m) {
+        c_i = lane < m_lo ? (int)__fns(cm_lo, 0, lane + 1) : 32 + (int)__fns(cm_hi, 0, lane - m_lo + 1);
+        jc_i = SR_CHECKED((int)(sg ? sg->tcand[c_i] : a.tree_cand[(size_t)b * N + c_i]), k, b);
+        uu_i = (double)(sg ? sg->uacc[c_i] : a.u_acc[(size_t)b * N + c_i]);
+    }
+    unsigned taken_i = lane < m ? (1u << jc_i) : 0u;  // exclusive prefix OR over the children before i
+    {
+        unsigned incl = taken_i;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl |= t;
+        }
+        taken_i = incl & ~taken_i;
+    }
+    double s_i = 0.0;
+    if (staged) {
+        for (int jj = 0; jj < k; ++jj)
+            if (!((taken_i >> jj) & 1u)) s_i += sg->e[hd * k + jj];
+    } else {
+        for (int jj = 0; jj < k; ++jj) {
+            const double ej = __shfl_sync(0xffffffffu, e, jj);
+            if (!((taken_i >> jj) & 1u)) s_i += ej;
+        }
+    }
+    if (__ballot_sync(0xffffffffu, lane < m && !(s_i > 0.0 && s_i < INFINITY)))
+        return walk_node_seq(a, topo, b, u, M, S, thr, lane, sm, st, sg, emit);
+    // what a slot needs from its child, where every lane can read it without a shuffle
+    const double inv_s_i = lane < m ? 1.0 / s_i : 0.0;
+    if (lane < m) {
+        sm->inv_s[lane] = inv_s_i;
+        sm->taken[lane] = taken_i;
+        sm->jc[lane] = jc_i;
+    }
+    __syncwarp();
+    // the chain
+    double Zc = 1.0, my_rho = 0.0, my_Zc = 1.0;
+    for (int i = 0; i < m; ++i) {
+        const double q = ((sm->taken[i] >> j) & 1u) ? 0.0 : e * sm->inv_s[i];
+        const double rho_jc = __shfl_sync(0xffffffffu, rho, sm->jc[i]);
+        if (lane == i) {
+            my_rho = rho_jc;
+            my_Zc = Zc;
+        }
+        const double t = fmax(rho - Zc * q, 0.0);
+        double Zn = t;
+        for (int o = kp >> 1; o > 0; o >>= 1) Zn += __shfl_xor_sync(0xffffffffu, Zn, o);
+        Zn += p_off;
+        if (Zn > 1e-300 * Zc) {
+            rho = t;
+            Zc = Zn;
+        }
+    }
+    // child i's own proposal probability: its candidate is among those it can still draw
+    const double my_q = __shfl_sync(0xffffffffu, e, jc_i) * inv_s_i;
+    // every child's test at once
+    bool acc_i = false;
+    float mg_i = INFINITY;
+    if (lane < m) {
+        double ratio;
+        if (my_q > 0.0)
+            ratio = my_rho > 0.0 ? (my_rho / my_Zc) / my_q : 0.0;
+        else
+            ratio = my_rho > 0.0 ? INFINITY : 0.0;
+        acc_i = uu_i < (ratio < 1.0 ? ratio : 1.0);
+        mg_i = (float)fabs(uu_i - ratio);
+    }
+    const unsigned accmask = __ballot_sync(0xffffffffu, acc_i);
+    const int first = accmask ? __ffs(accmask) - 1 : -1;
+    float mg = (lane < m && (first < 0 || lane <= first)) ? mg_i : INFINITY;
+    mg = -warp_max(-mg);
+    if (mg < st->mm) st->mm = mg;
+    if (first >= 0) {
+        const int accepted = __shfl_sync(0xffffffffu, c_i, first);
+        if (emit) {
+            if (lane == 0) {
+                a.out_tok[(size_t)b * (K + 1) + st->nacc] = sg ? sg->ttok[accepted] : a.tree_tok[(size_t)b * N + accepted];
+                a.path_node[(size_t)b * (K + 1) + st->nacc + 1] = accepted;
+            }
+            ++st->nacc;
+        }
+        return accepted;
+    }
+    // all rejected: the residual, normalised as the callers expect it (r and sigma = 1 / Zc)
+    const double inv_Zc = 1.0 / Zc;
+    if (lane < k) sm->r[j] = rho * inv_Zc;
+    st->sigma = inv_Zc;
+    st->p_off = p_off;
+    __syncwarp();
+    return -1;
+}
+
 // Results of a sequence and the hand-over of the residual (S = normaliser of u's row) to the terminal draw.
 __device__ __forceinline__ void walk_end(const WalkArgs &a, int b, int u, double S, int lane, WalkSmem *sm,
                                          WalkState *st) {
     const int k = a.k;
     if (st->have_residual) {
         const double sigma = __shfl_sync(0xffffffffu, st->sigma, 0);
+        const double f = S / sigma;  // (one division; the entries may be zero)
         for (int j = lane; j < k; j += 32) {
             a.ws_ovid[(size_t)b * k + j] = sm->id[j];
-            a.ws_ovm[(size_t)b * k + j] = sm->r[j] * S / sigma;
+            a.ws_ovm[(size_t)b * k + j] = sm->r[j] * f;
         }
     }
     if (lane == 0) {
@@ -553,7 +816,7 @@ __global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(WalkArgs a, Topo 
             }
         }
         __syncwarp();
-        stage = WalkStage{rmax, rsum, uacc, ttok, tcand, cid, clog, pre};
+        stage = WalkStage{rmax, rsum, uacc, ttok, tcand, cid, clog, pre, nullptr, nullptr, nullptr};
         sg = &stage;
     }
     WalkState st;
@@ -741,6 +1004,138 @@ __device__ __forceinline__ double warp_incl_scan(double v, int lane) {
     return v;
 }
 
+// Pass 1 of the terminal draw by one warp: the plain softmax mass of every 32-vector slice of the segment
+// [v_lo, v_hi) of a row, eight slices' loads in flight, left in out[0 .. n_sl).
+__device__ __forceinline__ void term_slice_masses(const uint4 *__restrict__ p, int v_lo, int v_hi, int n_sl, float M, float c,
+                                                  uint32_t thr, int lane, double *out) {
+    for (int s0 = 0; s0 < n_sl; s0 += 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = v_lo + (s0 + q) * 32 + lane;
+            v[q] = (s0 + q < n_sl && i < v_hi) ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);  // -inf: no mass
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            float e[8];
+            masses8(v[q], M, c, thr, e);
+            // a slice's 256 masses are added pairwise in fp32 (relative error of a few 2^-24, the size of the
+            // exponentials' own error); everything above a slice is fp64.  (Converting every mass to fp64 first
+            // kept the conversion pipe busy for as long as the exponentials.)
+            float acc = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+            acc = warp_sum(acc);
+            if (lane == 0 && s0 + q < n_sl) out[s0 + q] = (double)acc;
+        }
+    }
+}
+
+// The masses of the eight tokens of vector i of a row (zero beyond v_hi), the residual entries in place of the
+// plain masses of their tokens; returns their sum.
+__device__ __forceinline__ double term_vector_masses(const uint4 *__restrict__ p, int i, int v_hi, float M, float c, uint32_t thr,
+                                                     int nov, const int32_t *ovid, const double *ovm, double (&ms)[8]) {
+    double lsum = 0.0;
+    if (i < v_hi) {
+        float e[8];
+        masses8(ld_nc_v4(p + i), M, c, thr, e);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) ms[t] = (double)e[t];
+        for (int j = 0; j < nov; ++j) {
+            const int off = ovid[j] - i * 8;
+            if (off >= 0 && off < 8) {
+#pragma unroll
+                for (int t = 0; t < 8; ++t)
+                    if (t == off) ms[t] = ovm[j];
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) lsum += ms[t];
+    } else {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) ms[t] = 0.0;
+    }
+    return lsum;
+}
+
+// The token inside a 32-vector slice, by the warp whose lanes hold the vectors' masses (ms, their sums lsum): the
+// first token whose running mass, from base on, exceeds the target; take_last: the last one with positive mass.
+__device__ __forceinline__ void term_pick_token(int i, const double (&ms)[8], double lsum, double base, double target,
+                                                bool take_last, int v_hi, int32_t *dst, int lane) {
+    const double incl = warp_incl_scan(lsum, lane);
+    const unsigned hit = take_last ? 0u : __ballot_sync(0xffffffffu, base + incl > target);
+    if (hit) {
+        const int Lh = __ffs(hit) - 1;
+        if (lane == Lh) {
+            int tok = -1;
+            double cum = base + (incl - lsum);
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                cum += ms[t];
+                if (tok < 0 && cum > target) tok = i * 8 + t;
+            }
+            if (tok < 0) {  // scan and sequential sums disagreed in the last bit
+#pragma unroll
+                for (int t = 0; t < 8; ++t)
+                    if (ms[t] > 0.0) tok = i * 8 + t;
+            }
+            *dst = tok;
+        }
+    } else {
+        // the lanes' scanned mass fell short of the slice's sum by rounding: last token with positive mass
+        int last_pos = -1;
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+            if (ms[t] > 0.0) last_pos = i * 8 + t;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, o));
+        if (lane == 0) *dst = last_pos < 0 ? max(0, v_hi * 8 - 1) : last_pos;
+    }
+}
+
+// Last step of the terminal draw by one warp, inside the segment [v_lo, v_hi) that holds the target mass: seg_slices =
+// the segment's n_sl slice masses (residual entries applied), base = the mass before the segment; ovid / ovm = the nov
+// residual entries.  Writes the token to *dst.
+__device__ void term_pick(const uint4 *__restrict__ p, const double *seg_slices, int n_sl, int v_lo, int v_hi, double base,
+                          double target, float M, float c, uint32_t thr, int nov, const int32_t *ovid, const double *ovm,
+                          int32_t *dst, int lane) {
+    // the slice inside the selected segment: first one whose running mass exceeds the target; if rounding made
+    // the slices fall short of the segment's own sum, the last slice with positive mass
+    int sl_sel = -1, sl_pos = -1;
+    double base_pos = 0.0;
+    for (int c0 = 0; c0 < n_sl && sl_sel < 0; c0 += 32) {
+        const double v = (c0 + lane < n_sl) ? seg_slices[c0 + lane] : 0.0;
+        const double incl = warp_incl_scan(v, lane);
+        const unsigned hit = __ballot_sync(0xffffffffu, base + incl > target);
+        const unsigned pos = __ballot_sync(0xffffffffu, v > 0.0);
+        if (pos) {
+            const int lp = 31 - __clz(pos);
+            sl_pos = c0 + lp;
+            base_pos = base + __shfl_sync(0xffffffffu, incl - v, lp);
+        }
+        if (hit) {
+            const int lh = __ffs(hit) - 1;
+            sl_sel = c0 + lh;
+            base += __shfl_sync(0xffffffffu, incl - v, lh);
+        } else {
+            base += __shfl_sync(0xffffffffu, incl, 31);
+        }
+    }
+    bool take_last = false;
+    if (sl_sel < 0) {
+        if (sl_pos < 0) {  // no mass at all in the segment (cannot be selected with positive total; keep a valid token)
+            if (lane == 0) *dst = max(0, v_hi * 8 - 1);
+            return;
+        }
+        sl_sel = sl_pos;
+        base = base_pos;
+        take_last = true;
+    }
+    // the token inside the slice
+    const int i = v_lo + sl_sel * 32 + lane;
+    double ms[8];
+    const double lsum = term_vector_masses(p, i, v_hi, M, c, thr, nov, ovid, ovm, ms);
+    term_pick_token(i, ms, lsum, base, target, take_last, v_hi, dst, lane);
+}
+
 // The vocabulary is cut into TERM_WARPS warp segments of vpw 8-token vectors, each walked in slices of 32 vectors (one per
 // lane).  Pass 1 (all warps, independent loads) leaves the fp64 mass of every slice in shared memory; the walk's
 // residual entries then replace the plain mass of their tokens; two scans pick the segment and the slice that
@@ -776,26 +1171,7 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
         sh_ovid[threadIdx.x] = a.ws_ovid[(size_t)b * a.k + threadIdx.x];
     }
 
-    // pass 1: plain softmax mass of every slice, eight slices' loads in flight
-    for (int s0 = 0; s0 < n_sl; s0 += 8) {
-        uint4 v[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int i = v_lo + (s0 + q) * 32 + lane;
-            v[q] = (s0 + q < n_sl && i < v_hi) ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);  // -inf: no mass
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            float e[8];
-            masses8(v[q], M, a.c, thr, e);
-            // a slice's 256 masses are added pairwise in fp32 (relative error of a few 2^-24, the size of the
-            // exponentials' own error); everything above a slice is fp64.  (Converting every mass to fp64 first
-            // kept the conversion pipe busy for as long as the exponentials.)
-            float acc = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
-            acc = warp_sum(acc);
-            if (lane == 0 && s0 + q < n_sl) sh_slice[warp * n_sl + s0 + q] = (double)acc;
-        }
-    }
+    term_slice_masses(p, v_lo, v_hi, n_sl, M, a.c, thr, lane, sh_slice + warp * n_sl);
     __syncthreads();
     // the walk's residual entries replace the plain mass of their tokens (at most k of them: one thread)
     if (threadIdx.x == 0) {
@@ -848,92 +1224,351 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
     }
     if (warp != wsel) return;
 
-    // the slice inside the selected segment: first one whose running mass exceeds the target; if rounding made
-    // the slices fall short of the segment's own sum, the last slice with positive mass
-    const double target = sh_base[1];
-    double base = sh_base[0];
-    int sl_sel = -1, sl_pos = -1;
-    double base_pos = 0.0;
-    for (int c0 = 0; c0 < n_sl && sl_sel < 0; c0 += 32) {
-        const double v = (c0 + lane < n_sl) ? sh_slice[warp * n_sl + c0 + lane] : 0.0;
-        const double incl = warp_incl_scan(v, lane);
-        const unsigned hit = __ballot_sync(0xffffffffu, base + incl > target);
-        const unsigned pos = __ballot_sync(0xffffffffu, v > 0.0);
-        if (pos) {
-            const int lp = 31 - __clz(pos);
-            sl_pos = c0 + lp;
-            base_pos = base + __shfl_sync(0xffffffffu, incl - v, lp);
-        }
-        if (hit) {
-            const int lh = __ffs(hit) - 1;
-            sl_sel = c0 + lh;
-            base += __shfl_sync(0xffffffffu, incl - v, lh);
-        } else {
-            base += __shfl_sync(0xffffffffu, incl, 31);
+    term_pick(p, sh_slice + warp * n_sl, n_sl, v_lo, v_hi, sh_base[0], sh_base[1], M, a.c, thr, nov, sh_ovid, sh_ovm, dst,
+              lane);
+}
+
+// ------------------------------------------------------------------------------ walk + terminal draw in one launch
+//
+// The plain verification after the row statistics, one cluster of S CTAs per sequence (S = 1: plain CTAs).
+//   (1) Everything a walk can read is staged in shared memory; what does not depend on the row statistics (the
+//       candidates, the uniforms, the target logits at the candidates) is fetched before the wait for the previous
+//       kernel in the stream, which this kernel is launched to overlap with (programmatic dependent launch).
+//   (2) Which nodes the walk reaches depends on its decisions, but what happens AT a node does not: its children
+//       are tried in slot order until one is accepted, each against the residual left by the rejections before it.
+//       So every node with children is examined on its own, one warp per node, all at once: the first accepted
+//       child (or none, and then the residual), and the smallest margin on the way.  The walk itself is then a
+//       chain of at most K + 1 look-ups.  Every CTA of a cluster does (1) and (2) for itself: same inputs, same
+//       arithmetic, same result, nothing to exchange.
+//   (3) The terminal draw over the last node's row.  With the statistics kernel's slice table (tab) the masses of the
+//       row's 4096-token slices are there already: pick the slice, then read that one slice of the row.  Without it
+//       the S * WT_WARPS warps of the cluster each take one segment of the vocabulary; the slice masses of the
+//       other CTAs are read through distributed shared memory by the cluster's first CTA, which finishes as
+//       terminal_kernel does.
+constexpr int WT_THREADS = 512;
+constexpr int WT_WARPS = WT_THREADS / 32;
+
+struct WtLayout {
+    size_t stage, ovm, first, mm, slices, seg, par, e, p, total;
+    int G, vpw, n_sl;
+};
+__host__ __device__ inline WtLayout wt_layout(int N, int K, int k, int V, int S, bool tab) {
+    WtLayout L;
+    auto up = [](size_t x) { return (x + 15) / 16 * 16; };
+    const int nvec = V >> 3;
+    if (tab) {  // the segments are the table's slices; only the selected one is cut into 32-vector slices
+        L.G = row_slices(V);
+        L.vpw = 4 * 128;
+        L.n_sl = L.vpw / 32;
+    } else {
+        L.G = S * WT_WARPS;
+        L.vpw = (nvec + L.G - 1) / L.G;
+        L.n_sl = (L.vpw + 31) / 32;
+    }
+    size_t o = 0;
+    L.stage = o;
+    o += up(walk_stage_bytes(N, K, k));
+    L.ovm = o;
+    o += up((size_t)N * k * sizeof(double));
+    L.first = o;
+    o += up((size_t)N * sizeof(int32_t));
+    L.mm = o;
+    o += up((size_t)N * sizeof(float));
+    L.slices = o;
+    o += up((size_t)(tab ? 1 : L.G) * L.n_sl * sizeof(double));
+    L.seg = o;
+    o += up((size_t)L.G * sizeof(double));
+    L.par = o;
+    o += up((size_t)N);
+    L.e = o;
+    o += up((size_t)K * k * sizeof(double));
+    L.p = o;
+    o += up((size_t)N * k * sizeof(double));
+    L.total = o;
+    return L;
+}
+
+__global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, Topo topo, const float *__restrict__ u_fin, float c,
+                                                               int S, const float2 *__restrict__ tab) {
+    __shared__ WalkSmem sh[WT_WARPS];
+    extern __shared__ __align__(16) unsigned char sh_dyn[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rank = S > 1 ? (int)cluster_ctarank() : 0;
+    const int b = blockIdx.x / S;
+    const int N = a.N, K = a.K, k = a.k;
+    const WtLayout L = wt_layout(N, K, k, a.V, S, tab != nullptr);
+    auto up = [](size_t x) { return (x + 15) / 16 * 16; };
+    unsigned char *p0 = sh_dyn + L.stage;
+    float *rmax = reinterpret_cast<float *>(p0);
+    p0 += up((size_t)N * 4);
+    float *rsum = reinterpret_cast<float *>(p0);
+    p0 += up((size_t)N * 4);
+    float *uacc = reinterpret_cast<float *>(p0);
+    p0 += up((size_t)N * 4);
+    int32_t *ttok = reinterpret_cast<int32_t *>(p0);
+    p0 += up((size_t)N * 4);
+    uint8_t *tcand = reinterpret_cast<uint8_t *>(p0);
+    p0 += up((size_t)N);
+    int32_t *cid = reinterpret_cast<int32_t *>(p0);
+    p0 += up((size_t)K * k * 4);
+    float *clog = reinterpret_cast<float *>(p0);
+    p0 += up((size_t)K * k * 4);
+    uint16_t *pre = reinterpret_cast<uint16_t *>(p0);
+    double *ovm = reinterpret_cast<double *>(sh_dyn + L.ovm);
+    int32_t *first = reinterpret_cast<int32_t *>(sh_dyn + L.first);
+    float *mmin = reinterpret_cast<float *>(sh_dyn + L.mm);
+    double *slices = reinterpret_cast<double *>(sh_dyn + L.slices);
+    double *seg = reinterpret_cast<double *>(sh_dyn + L.seg);
+    int8_t *par = reinterpret_cast<int8_t *>(sh_dyn + L.par);
+    double *we = reinterpret_cast<double *>(sh_dyn + L.e);
+    double *wp = reinterpret_cast<double *>(sh_dyn + L.p);
+    const double inv_T = 1.0 / a.T;
+    // (1) inputs of this call, none of them written by the kernel before this one
+    for (int n = tid; n < N; n += WT_THREADS) {
+        uacc[n] = a.u_acc[(size_t)b * N + n];
+        ttok[n] = a.tree_tok[(size_t)b * N + n];
+        tcand[n] = a.tree_cand[(size_t)b * N + n];
+        par[n] = topo.parent[n];
+    }
+    for (int e = tid; e < K * k; e += WT_THREADS) {
+        cid[e] = SR_CHECKED(a.cand_id[(size_t)b * K * k + e], a.V, b);
+        clog[e] = a.cand_logit[(size_t)b * K * k + e];
+    }
+    for (int e = tid; e < N * k; e += WT_THREADS) {
+        const int u = e / k, j = e - u * k;
+        if (topo.n_child[u] > 0) {  // (a node with children is at depth < K)
+            const int t = SR_CHECKED(a.cand_id[((size_t)b * K + topo.depth[u]) * k + j], a.V, b);
+            pre[e] = a.logits[((size_t)b * N + u) * a.V + t];
         }
     }
-    bool take_last = false;
-    if (sl_sel < 0) {
-        if (sl_pos < 0) {  // no mass at all in the segment (cannot be selected with positive total; keep a valid token)
-            if (lane == 0) *dst = max(0, v_hi * 8 - 1);
-            return;
-        }
-        sl_sel = sl_pos;
-        base = base_pos;
-        take_last = true;
+    // the proposal weights of every head's candidates, relative to the head's largest logit
+    __syncthreads();
+    for (int e = tid; e < K * k; e += WT_THREADS) {
+        const int hd = e / k;
+        float mx = -INFINITY;
+        for (int jj = 0; jj < k; ++jj) mx = fmaxf(mx, clog[hd * k + jj]);
+        we[e] = exp(((double)clog[e] - (double)mx) * inv_T);
     }
-    // the token inside the slice
-    const int i = v_lo + sl_sel * 32 + lane;
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the row statistics are complete from here on
+    for (int n = tid; n < N; n += WT_THREADS) {
+        rmax[n] = a.row_max[(size_t)b * N + n];
+        rsum[n] = a.row_sum[(size_t)b * N + n];
+    }
+    // the target probabilities of every walkable node's candidates (the statistics straight from global memory:
+    // one round trip for everything)
+    for (int e = tid; e < N * k; e += WT_THREADS) {
+        const int u = e / k;
+        if (topo.n_child[u] > 0) {
+            const double M = (double)a.row_max[(size_t)b * N + u], S = (double)a.row_sum[(size_t)b * N + u];
+            wp[e] = exp(((double)bf16_bits_to_float(pre[e]) - M) * inv_T) * (1.0 / S);
+        }
+    }
+    __syncthreads();
+    // (2) every node with children on its own
+    {
+        const WalkStage stage{rmax, rsum, uacc, ttok, tcand, cid, clog, pre, par, we, wp};
+        int idx = 0;
+        for (int u = 0; u < N; ++u) {
+            if (topo.n_child[u] == 0) continue;
+            if ((idx++ % WT_WARPS) != warp) continue;
+            WalkState st;
+            st.nacc = 0;
+            st.kind = 0;
+            st.sigma = 1.0;
+            st.p_off = 0.0;
+            st.mm = INFINITY;
+            st.have_residual = false;
+            const int acc = walk_node(a, topo, b, u, (double)rmax[u], (double)rsum[u], 0u, lane, &sh[warp], &st, &stage, false);
+            if (acc < 0) {
+                const double f = (double)rsum[u] / st.sigma;
+                for (int j = lane; j < k; j += 32) ovm[u * k + j] = sh[warp].r[j] * f;
+            }
+            if (lane == 0) {
+                first[u] = acc;
+                mmin[u] = st.mm;
+            }
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    // the walk: every thread follows the same chain
+    int u = 0, nacc = 0, kind = 0;
+    bool resid = false;
+    float mm = INFINITY;
+    const bool writer = (rank == 0 && tid == 0);
+    if (writer) {
+        for (int i = 0; i <= K; ++i) a.path_node[(size_t)b * (K + 1) + i] = a.out_tok[(size_t)b * (K + 1) + i] = -1;
+        a.path_node[(size_t)b * (K + 1)] = 0;
+    }
+    for (;;) {
+        if (topo.n_child[u] == 0) {
+            kind = (u != 0) ? 1 : 0;
+            break;
+        }
+        mm = fminf(mm, mmin[u]);
+        const int ch = first[u];
+        if (ch < 0) {
+            resid = true;
+            break;
+        }
+        if (writer) {
+            a.out_tok[(size_t)b * (K + 1) + nacc] = ttok[ch];
+            a.path_node[(size_t)b * (K + 1) + nacc + 1] = ch;
+        }
+        ++nacc;
+        u = ch;
+    }
+    if (writer) {
+        a.n_acc[b] = nacc;
+        a.term_node[b] = u;
+        a.term_kind[b] = kind;
+        if (a.min_margin) a.min_margin[b] = mm;
+    }
+
+    // (3) the terminal draw from row u: the residual (k entries over the plain masses) or the plain distribution
+    const int nov = resid ? k : 0;
+    const int32_t *ovid = cid + (resid ? topo.depth[u] : 0) * k;
+    const double *ovm_u = ovm + u * k;
+    const float M = rmax[u];
+    const uint16_t *lg = a.logits + ((size_t)b * N + u) * a.V;
+    const uint4 *p = reinterpret_cast<const uint4 *>(lg);
+    const int nvec = a.V >> 3, vpw = L.vpw, n_sl = L.n_sl, G = L.G;
+    if (tab) {
+        const float2 *tb = tab + ((size_t)b * N + u) * G;
+        for (int g = tid; g < G; g += WT_THREADS) {
+            const float2 e = tb[g];
+            seg[g] = (double)e.y * (double)ex2_approx((e.x - M) * c);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            const RowSlices rs(a.V);
+            for (int j = 0; j < nov; ++j) seg[rs.slice_of_token(ovid[j])] += ovm_u[j] - (double)mass1(pre[u * k + j], M, c, 0u);
+        }
+        __syncthreads();
+    } else {
+        {
+            const int g = rank * WT_WARPS + warp;
+            const int v_lo = min(nvec, g * vpw), v_hi = min(nvec, v_lo + vpw);
+            term_slice_masses(p, v_lo, v_hi, n_sl, M, c, 0u, lane, slices + (size_t)g * n_sl);
+        }
+        if (S > 1) {
+            cluster_sync_all();  // every CTA's slice masses are in its shared memory
+            if (rank == 0) {
+                const int per = WT_WARPS * n_sl;
+                for (int e = tid; e < (S - 1) * per; e += WT_THREADS) {
+                    const int r = 1 + e / per, o = r * per + (e - (r - 1) * per);
+                    slices[o] = ld_dsmem_f64(slices + o, r);
+                }
+            }
+            cluster_sync_all();  // the other CTAs may leave
+            if (rank != 0) return;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            for (int j = 0; j < nov; ++j) {
+                const int t = ovid[j], vi = t >> 3;
+                const int w = min(G - 1, vi / vpw), sl = (vi - w * vpw) >> 5;
+                slices[w * n_sl + sl] += ovm_u[j] - (double)mass1(pre[u * k + j], M, c, 0u);  // (staged: lg[t])
+            }
+        }
+        __syncthreads();
+        for (int g = warp; g < G; g += WT_WARPS) {
+            double acc = 0.0;
+            for (int sl = lane; sl < n_sl; sl += 32) acc += slices[g * n_sl + sl];
+            acc = warp_sum(acc);
+            if (lane == 0) seg[g] = acc;
+        }
+        __syncthreads();
+    }
+    __shared__ int sh_wsel;
+    __shared__ double sh_bt[2];
+    int32_t *dst = a.out_tok + (size_t)b * (K + 1) + nacc;
+    if (warp == 0) {
+        double total = 0.0;
+        for (int g0 = 0; g0 < G; g0 += 32) total += warp_sum(g0 + lane < G ? seg[g0 + lane] : 0.0);
+        const double target = (double)u_fin[b] * total;
+        int wsel = -1;
+        double base = 0.0;
+        for (int g0 = 0; g0 < G && wsel < 0; g0 += 32) {
+            const double v = g0 + lane < G ? seg[g0 + lane] : 0.0;
+            const double incl = warp_incl_scan(v, lane);
+            const unsigned hit = __ballot_sync(0xffffffffu, g0 + lane < G && base + incl > target);
+            if (hit) {
+                const int lh = __ffs(hit) - 1;
+                wsel = g0 + lh;
+                base += __shfl_sync(0xffffffffu, incl - v, lh);
+            } else {
+                base += __shfl_sync(0xffffffffu, incl, 31);
+            }
+        }
+        if (wsel < 0) {
+            // u_fin * total reached the total through rounding: take the last token with positive mass
+            if (lane == 0) {
+                int tok = a.V - 1;
+                for (; tok > 0; --tok) {
+                    double ms = (double)mass1(lg[tok], M, c, 0u);
+                    for (int j = 0; j < nov; ++j)
+                        if (ovid[j] == tok) ms = ovm_u[j];
+                    if (ms > 0.0) break;
+                }
+                *dst = tok;
+            }
+        } else if (!tab) {
+            const int v_lo = min(nvec, wsel * vpw), v_hi = min(nvec, v_lo + vpw);
+            term_pick(p, slices + (size_t)wsel * n_sl, n_sl, v_lo, v_hi, base, target, M, c, 0u, nov, ovid, ovm_u, dst, lane);
+        }
+        if (lane == 0) {
+            sh_wsel = wsel;
+            sh_bt[0] = base;
+            sh_bt[1] = target;
+        }
+    }
+    if (!tab) return;
+    // with the table: the selected slice of the row is read now, one 32-vector slice per warp, all warps at once;
+    // the warp whose slice holds the target keeps its vectors' masses in registers and picks the token
+    static_assert(4 * 128 / 32 == WT_WARPS, "one 32-vector slice of a table slice per warp");
+    __syncthreads();
+    const int wsel = sh_wsel;
+    if (wsel < 0) return;
+    double base = sh_bt[0];
+    const double target = sh_bt[1];
+    int v_lo, v_hi;
+    RowSlices(a.V).vectors(wsel, &v_lo, &v_hi);
+    const int i = v_lo + warp * 32 + lane;
     double ms[8];
-    double lsum = 0.0;
-    if (i < v_hi) {
-        float e[8];
-        masses8(ld_nc_v4(p + i), M, a.c, thr, e);
-#pragma unroll
-        for (int t = 0; t < 8; ++t) ms[t] = (double)e[t];
-        for (int j = 0; j < nov; ++j) {
-            const int off = sh_ovid[j] - i * 8;
-            if (off >= 0 && off < 8) {
-#pragma unroll
-                for (int t = 0; t < 8; ++t)
-                    if (t == off) ms[t] = sh_ovm[j];
-            }
-        }
-#pragma unroll
-        for (int t = 0; t < 8; ++t) lsum += ms[t];
-    } else {
-#pragma unroll
-        for (int t = 0; t < 8; ++t) ms[t] = 0.0;
+    const double lsum = term_vector_masses(p, i, v_hi, M, c, 0u, nov, ovid, ovm_u, ms);
+    {
+        const double sm_ = warp_sum(lsum);
+        if (lane == 0) slices[warp] = sm_;
     }
-    const double incl = warp_incl_scan(lsum, lane);
-    const unsigned hit = take_last ? 0u : __ballot_sync(0xffffffffu, base + incl > target);
+    __syncthreads();
+    // every warp finds the slice for itself (same numbers, same result)
+    const double v = lane < WT_WARPS ? slices[lane] : 0.0;
+    const double incl = warp_incl_scan(v, lane);
+    const unsigned hit = __ballot_sync(0xffffffffu, lane < WT_WARPS && base + incl > target);
+    const unsigned pos = __ballot_sync(0xffffffffu, v > 0.0);
+    bool take_last = false;
+    int sl_sel;
     if (hit) {
-        const int Lh = __ffs(hit) - 1;
-        if (lane == Lh) {
-            int tok = -1;
-            double cum = base + (incl - lsum);
-#pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                cum += ms[t];
-                if (tok < 0 && cum > target) tok = i * 8 + t;
-            }
-            if (tok < 0) {  // scan and sequential sums disagreed in the last bit
-#pragma unroll
-                for (int t = 0; t < 8; ++t)
-                    if (ms[t] > 0.0) tok = i * 8 + t;
-            }
-            *dst = tok;
-        }
+        sl_sel = __ffs(hit) - 1;
+    } else if (pos) {  // the slices fell short of the table's mass by rounding: the last slice with positive mass
+        sl_sel = 31 - __clz(pos);
+        take_last = true;
     } else {
-        // the lanes' scanned mass fell short of the slice's sum by rounding: last token with positive mass
-        int last_pos = -1;
-#pragma unroll
-        for (int t = 0; t < 8; ++t)
-            if (ms[t] > 0.0) last_pos = i * 8 + t;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, o));
-        if (lane == 0) *dst = last_pos < 0 ? max(0, v_hi * 8 - 1) : last_pos;
+        if (tid == 0) *dst = max(0, v_hi * 8 - 1);  // (no mass at all; keep a valid token)
+        return;
     }
+    base += __shfl_sync(0xffffffffu, incl - v, sl_sel);
+    if (warp != sl_sel) return;
+    term_pick_token(i, ms, lsum, base, target, take_last, v_hi, dst, lane);
+}
+
+// S CTAs per sequence: as many as keep the grid within about two CTAs per SM, a power of two up to the portable
+// cluster size.
+static int walk_term_split(int B) {
+    int S = 8;
+    while (S > 1 && (long long)B * S > 296) S >>= 1;
+    return S;
 }
 
 static int launch_terminal(const TermArgs &ta, cudaStream_t st) {
@@ -966,9 +1601,14 @@ static size_t verify_ws_base(const specroll_verify_desc *d) {
            align_up(B * sizeof(int32_t), 256) + 256;
 }
 
+// The slice table of the plain verification: one (reference, mass) pair per 4096-token slice of every row.
+static size_t verify_ws_table(const specroll_verify_desc *d) {
+    return align_up((size_t)d->B * d->N * row_slices(d->V) * sizeof(float2), 256);
+}
+
 extern "C" size_t specroll_verify_workspace_bytes(const specroll_verify_desc *d) {
     if (check_verify_desc(d) != SPECROLL_OK) return 0;
-    return verify_ws_base(d);
+    return verify_ws_base(d) + ((d->flags & SPECROLL_VERIFY_LAZY_STATS) ? 0 : verify_ws_table(d));
 }
 
 extern "C" size_t specroll_verify_nucleus_workspace_bytes(const specroll_verify_desc *d) {
@@ -983,7 +1623,7 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
                       const float *cand_logit, const float *u_acc, const float *u_fin, int32_t *n_acc,
                       int32_t *path_node, int32_t *out_tok, int32_t *term_node, int32_t *term_kind, float *row_max,
                       float *row_sum, float *min_margin, float *nucleus_thr, float *nucleus_sum, void *workspace,
-                      size_t workspace_bytes, void *cuda_stream) {
+                      size_t workspace_bytes, void *cuda_stream, bool table_optional = false) {
     if (check_verify_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (!logits || !tree_tok || !tree_cand || !cand_id || !cand_logit || !u_acc || !u_fin || !n_acc ||
         !path_node || !out_tok || !term_node || !term_kind || !row_max || !row_sum)
@@ -993,7 +1633,13 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
     if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (!aligned16(logits)) return SPECROLL_EALIGN;
     if (d->B == 0) return SPECROLL_OK;
-    const size_t need = truncate ? specroll_verify_nucleus_workspace_bytes(d) : verify_ws_base(d);
+    const bool lazy = (d->flags & SPECROLL_VERIFY_LAZY_STATS) != 0;
+    // the slice table serves the plain verification with all rows' statistics; a caller with fixed scratch
+    // (table_optional) goes without it when it does not fit
+    bool use_table = !truncate && !lazy;
+    if (use_table && table_optional && workspace_bytes < verify_ws_base(d) + verify_ws_table(d)) use_table = false;
+    const size_t need = truncate ? specroll_verify_nucleus_workspace_bytes(d)
+                                 : verify_ws_base(d) + (use_table ? verify_ws_table(d) : 0);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)
         return SPECROLL_EWORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -1011,10 +1657,14 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
 
     const float c = (float)(1.4426950408889634 / (double)d->temperature);
     const int rows = d->B * d->N;
-    const bool lazy = (d->flags & SPECROLL_VERIFY_LAZY_STATS) != 0;
+    float2 *tab = use_table ? reinterpret_cast<float2 *>(ws) : nullptr;  // (no nucleus arrays in this form)
     if (!lazy) {
-        row_stats_kernel<<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
-                                                      row_sum);
+        if (use_table)
+            row_stats_kernel<true><<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
+                                                                row_sum, tab);
+        else
+            row_stats_kernel<false><<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
+                                                                 row_sum, nullptr);
         SR_LAUNCH_CHECK();
     }
 
@@ -1058,12 +1708,34 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
         walk_cta_kernel<true, false><<<d->B, NUC_THREADS, 0, st>>>(wa, topo, c, 1.0f, row_max, row_sum, nullptr, nullptr,
                                                                     nullptr, nullptr);
     } else {
-        const size_t stage = (size_t)WALK_WARPS * walk_stage_bytes(d->N, d->K, d->k);
-        if (stage > 40 * 1024) {  // beyond what a kernel may use without asking (together with its static arrays)
-            const int rc_ = device_setup(reinterpret_cast<const void *>(walk_kernel), 64 * 1024, nullptr);
-            if (rc_ != SPECROLL_OK) return rc_;
+        // plain verification: the walk and the terminal draw in one launch, overlapping the statistics kernel's tail
+        constexpr int WT_SMEM_LIMIT = 160 * 1024;
+        const int S = use_table ? 1 : walk_term_split(d->B);
+        const WtLayout L = wt_layout(d->N, d->K, d->k, d->V, S, use_table);
+        if (L.total > (size_t)WT_SMEM_LIMIT) return SPECROLL_ELIMIT;
+        const int rc_ = device_setup(reinterpret_cast<const void *>(walk_term_kernel), WT_SMEM_LIMIT, nullptr);
+        if (rc_ != SPECROLL_OK) return rc_;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(d->B * S));
+        cfg.blockDim = dim3(WT_THREADS);
+        cfg.dynamicSmemBytes = L.total;
+        cfg.stream = st;
+        cudaLaunchAttribute attrs[2];
+        int na = 0;
+        attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attrs[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+        if (S > 1) {
+            attrs[na].id = cudaLaunchAttributeClusterDimension;
+            attrs[na].val.clusterDim.x = (unsigned)S;
+            attrs[na].val.clusterDim.y = 1;
+            attrs[na].val.clusterDim.z = 1;
+            ++na;
         }
-        walk_kernel<<<(d->B + WALK_WARPS - 1) / WALK_WARPS, WALK_WARPS * 32, stage, st>>>(wa, topo);
+        cfg.attrs = attrs;
+        cfg.numAttrs = na;
+        SR_CUDA_TRY(cudaLaunchKernelEx(&cfg, walk_term_kernel, wa, topo, u_fin, c, S, (const float2 *)tab));
+        return SPECROLL_OK;
     }
     SR_LAUNCH_CHECK();
 
@@ -1228,7 +1900,7 @@ extern "C" int specroll_verify_nucleus(const specroll_verify_desc *d, float top_
     if (!(top_p > 0.f)) return SPECROLL_EINVAL;
     return run_verify(d, top_p, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
                       path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, nucleus_thr,
-                      nucleus_sum, workspace, workspace_bytes, cuda_stream);
+                      nucleus_sum, workspace, workspace_bytes, cuda_stream, /*table_optional=*/true);
 }
 
 // ------------------------------------------------------------------------------ allocation-free variant
@@ -1257,7 +1929,7 @@ extern "C" int specroll_verify_static(const specroll_verify_desc *d, const void 
                                       float *row_sum, float *min_margin, void *cuda_stream) {
     if (check_verify_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (d->B > SPECROLL_STATIC_MAX_B || (long long)d->B * d->k > SPECROLL_STATIC_MAX_BK) return SPECROLL_ELIMIT;
-    if (specroll_verify_workspace_bytes(d) > STATIC_SCRATCH_BYTES) return SPECROLL_ELIMIT;
+    if (verify_ws_base(d) > STATIC_SCRATCH_BYTES) return SPECROLL_ELIMIT;
     int dev = -1;
     SR_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= MAX_DEVICES) return SPECROLL_ELIMIT;
@@ -1273,7 +1945,8 @@ extern "C" int specroll_verify_static(const specroll_verify_desc *d, const void 
         }
         scratch = g_scratch_addr[dev];
     }
-    return specroll_verify(d, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
-                           path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, scratch,
-                           STATIC_SCRATCH_BYTES, cuda_stream);
+    // (the slice table of the plain verification is used when it fits the scratch, else the row is read again)
+    return run_verify(d, 1.0f, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
+                      path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, nullptr, nullptr, scratch,
+                      STATIC_SCRATCH_BYTES, cuda_stream, true);
 }

@@ -108,8 +108,9 @@ class StepWorkload:
         ws_bytes = (S.tree_attn_paged_workspace_bytes(B, N, w.Hq, w.Hkv, w.D, self.kv_len_host) if self.paged else
                     S.tree_attn_workspace_bytes(B, N, w.Hq, w.Hkv, w.D, self.kv_indptr_host))
         self.ws_attn = S.alloc(ws_bytes, dtype=torch.uint8, device=device)
-        self.ws_verify = S.alloc(S.verify_nucleus_workspace_bytes(B, N, K, k, V, w.temperature),
-                                     dtype=torch.uint8, device=device)
+        self.ws_verify = S.alloc(max(S.verify_nucleus_workspace_bytes(B, N, K, k, V, w.temperature),
+                                     S.verify_workspace_bytes(B, N, K, k, V, w.temperature)),
+                                 dtype=torch.uint8, device=device)
         self.prop = None
         self.ver = None
         # target logits: N(0,1) background, one mode token per node boosted by +14
