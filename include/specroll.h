@@ -398,10 +398,7 @@ int specroll_target_head_rows(int32_t R, int32_t d, int32_t V, const void *H, co
  * (max logit and sum exp((l - max)/T) of every node); min_margin[B] fp32 or NULL (smallest
  * |u - ratio| over the tested slots; +inf if none).
  * Limits: V % 8 == 0, k <= 64, K <= 8, N <= 64.
- * Workspace: scratch of the call, specroll_verify_workspace_bytes(desc) bytes, 256-byte aligned.  Besides
- * the hand-over of the residual it holds, for every (sequence, node) row, the softmax mass of each
- * 4096-token slice of the row (written by the pass that computes the row statistics), so that the terminal
- * draw reads one slice of one row per sequence and not the row again.
+ * Workspace: scratch of the call, specroll_verify_workspace_bytes(desc) bytes, 256-byte aligned.
  */
 typedef struct {
     int32_t B, N, K, k, V;

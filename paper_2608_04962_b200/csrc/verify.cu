@@ -1,16 +1,19 @@
 // Exact target verification: softmax statistics of every tree node, the node-wise
 // accept / resample walk, and the terminal (fallback or bonus) draw.
 //
-// Three launches per call:
+// Two launches per plain call:
 //   row_stats_kernel    one CTA per (sequence, node) row: streams the bf16 logits once with
 //                       128-bit loads and keeps an online (max, sum-exp) pair per thread.
-//   walk_kernel         one warp per sequence.  The residual of the walk differs from p only
-//                       on the <= k candidates of the current node (the proposal is zero
-//                       elsewhere), so it is tracked as k numbers plus one scale for the
-//                       rest of the vocabulary, all in fp64.
-//   terminal_kernel     one CTA per sequence: inverse-CDF draw over the vocabulary in token
-//                       order with fp64 segment sums; the walk's <= k residual entries override
-//                       the plain softmax mass.
+//   walk_term_kernel    one CTA (or cluster) per sequence, launched to overlap the tail of the
+//                       statistics kernel: the walk, then the terminal draw.  The residual of the
+//                       walk differs from p only on the <= k candidates of the current node (the
+//                       proposal is zero elsewhere), so it is tracked as k numbers plus one scale
+//                       for the rest of the vocabulary, all in fp64; the terminal draw is an
+//                       inverse CDF over the vocabulary in token order with fp64 segment sums, the
+//                       walk's <= k residual entries overriding the plain softmax mass.
+// The other forms (statistics only of visited rows, nucleus targets, logits that were never
+// stored) use walk_kernel / walk_cta_kernel (one warp / one CTA per sequence) and
+// terminal_kernel (one CTA per sequence).
 #include <math.h>
 
 #include <mutex>
@@ -22,7 +25,6 @@ namespace specroll {
 SR_CHECK_TU()
 
 constexpr int RS_THREADS = 256;
-constexpr int RS_UNROLL = 4;
 constexpr int WALK_WARPS = 4;
 constexpr int TERM_THREADS = 512;  // two CTAs per SM
 constexpr int TERM_WARPS = TERM_THREADS / 32;
@@ -51,108 +53,36 @@ __device__ __forceinline__ void online_update(const uint4 &v, float c, float &m,
     s += acc;
 }
 
-// As online_update, with a second sum (of the current slice; SL) kept relative to the same running maximum.
-template <bool SL>
-__device__ __forceinline__ void online_update_slice(const uint4 &v, float c, float &m, float &s, float &sl) {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    float x[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        x[2 * i] = __uint_as_float(w[i] << 16);
-        x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-    float vm = x[0];
-#pragma unroll
-    for (int i = 1; i < 8; ++i) vm = fmaxf(vm, x[i]);
-    if (vm > m) {
-        const float f = ex2_approx((m - vm) * c);  // m = -inf gives 0
-        s *= f;
-        if (SL) sl *= f;
-        m = vm;
-    }
-    float acc = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc += ex2_approx((x[i] - m) * c);
-    s += acc;
-    if (SL) sl += acc;
-}
-
-// How the statistics kernel cuts a row: groups of 128 8-token vectors (four loads of 32 consecutive vectors by one
-// warp); each of the kernel's warps takes one contiguous run of groups (gpw of them, the last warp what is left); a
-// run is cut into slices of up to four groups (4096 tokens).  Slices are numbered warp by warp, so in token order;
-// a warp with a short run has empty slices at its end.
-constexpr int RS_WARPS = RS_THREADS / 32;
-struct RowSlices {
-    int nvec, G, gpw, spw, n_sl;
-    __host__ __device__ explicit RowSlices(int V) {
-        nvec = V >> 3;
-        G = (nvec + 127) / 128;
-        gpw = (G + RS_WARPS - 1) / RS_WARPS;
-        spw = (gpw + 3) / 4;
-        n_sl = RS_WARPS * spw;
-    }
-    // groups [g_lo, g_hi) of slice t of warp w (empty: g_lo >= g_hi)
-    __host__ __device__ void groups(int w, int t, int *g_lo, int *g_hi) const {
-        const int run_hi = min_((w + 1) * gpw, G);
-        *g_lo = w * gpw + 4 * t;
-        *g_hi = min_(run_hi, *g_lo + 4);
-    }
-    // vectors [v_lo, v_hi) of slice s
-    __host__ __device__ void vectors(int s, int *v_lo, int *v_hi) const {
-        int g_lo, g_hi;
-        groups(s / spw, s % spw, &g_lo, &g_hi);
-        *v_lo = min_(nvec, g_lo * 128);
-        *v_hi = g_hi > g_lo ? min_(nvec, g_hi * 128) : *v_lo;
-    }
-    __host__ __device__ int slice_of_token(int tok) const {
-        const int g = (tok >> 3) / 128, w = g / gpw;
-        return w * spw + (g - w * gpw) / 4;
-    }
-    static __host__ __device__ int min_(int a, int b) { return a < b ? a : b; }
-};
-__host__ __device__ inline int row_slices(int V) { return RowSlices(V).n_sl; }
-
 // logits[rows, V] bf16; c = log2(e) / T.  row_max = max_v l_v, row_sum = sum_v exp((l_v - max)/T).
-// TAB: every slice also leaves tab[row, slice] = (R, sum over the slice of exp((l_v - R)/T)) with some R >= the
-// slice's logits: the terminal draw of a row then needs this table and one slice of the row instead of the row.
-// (The two warp reductions per slice are why a slice is as long as it is: the shuffle unit passes one warp
-// instruction per clock per SM, and ten shuffles per 1024 tokens cost a tenth of the kernel's time.)
-template <bool TAB>
+// The row is cut into groups of 128 8-token vectors; a warp takes one contiguous run of groups and reads a group
+// with four loads of 32 consecutive vectors (2 KB in one piece per warp).  32 registers, so that eight CTAs fit an SM.
+constexpr int RS_WARPS = RS_THREADS / 32;
 __global__ void __launch_bounds__(RS_THREADS, 8)
 row_stats_kernel(const uint16_t *__restrict__ logits, int V, float c, float *__restrict__ row_max,
-                 float *__restrict__ row_sum, float2 *__restrict__ tab) {
+                 float *__restrict__ row_sum) {
     // a kernel launched behind this one as its programmatic dependent may start its own prologue as SMs free up; it
     // waits for this grid's completion before it reads the statistics
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const size_t row = blockIdx.x;
     const uint4 *p = reinterpret_cast<const uint4 *>(logits + row * (size_t)V);
-    const RowSlices rs(V);
-    const int nvec = rs.nvec;
+    const int nvec = V >> 3;
     float m = NEG_INF, s = 0.f;
     {
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-        for (int t = 0; t < rs.spw; ++t) {
-            int g_lo, g_hi;
-            rs.groups(warp, t, &g_lo, &g_hi);
-            float sl = 0.f;
+        const int G = (nvec + 127) / 128, gpw = (G + RS_WARPS - 1) / RS_WARPS;
+        const int g_hi = min(G, (warp + 1) * gpw);
 #pragma unroll 1
-            for (int g = g_lo; g < g_hi; ++g) {
-                const int i0 = g * 128 + lane;
-                if (i0 + 3 * 32 < nvec) {  // (for lane 31: the whole group is inside the row)
-                    uint4 v[4];
+        for (int g = warp * gpw; g < g_hi; ++g) {
+            const int i0 = g * 128 + lane;
+            if (i0 + 3 * 32 < nvec) {  // (for lane 31: the whole group is inside the row)
+                uint4 v[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) v[q] = ld_nc_v4(p + i0 + q * 32);
+                for (int q = 0; q < 4; ++q) v[q] = ld_nc_v4(p + i0 + q * 32);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) online_update_slice<TAB>(v[q], c, m, s, sl);
-                } else {
-                    for (int q = 0; q < 4; ++q)
-                        if (i0 + q * 32 < nvec) online_update_slice<TAB>(ld_nc_v4(p + i0 + q * 32), c, m, s, sl);
-                }
-            }
-            if (TAB) {
-                const float R = warp_max(m);  // >= everything the warp has seen, this slice included
-                const float tot = warp_sum((m == NEG_INF) ? 0.f : sl * ex2_approx((m - R) * c));
-                if (lane == 0) tab[row * rs.n_sl + warp * rs.spw + t] = make_float2(R, tot);
+                for (int q = 0; q < 4; ++q) online_update(v[q], c, m, s);
+            } else {
+                for (int q = 0; q < 4; ++q)
+                    if (i0 + q * 32 < nvec) online_update(ld_nc_v4(p + i0 + q * 32), c, m, s);
             }
         }
     }
@@ -1240,11 +1170,11 @@ __global__ void __launch_bounds__(TERM_THREADS) terminal_kernel(TermArgs a) {
 //       child (or none, and then the residual), and the smallest margin on the way.  The walk itself is then a
 //       chain of at most K + 1 look-ups.  Every CTA of a cluster does (1) and (2) for itself: same inputs, same
 //       arithmetic, same result, nothing to exchange.
-//   (3) The terminal draw over the last node's row.  With the statistics kernel's slice table (tab) the masses of the
-//       row's 4096-token slices are there already: pick the slice, then read that one slice of the row.  Without it
-//       the S * WT_WARPS warps of the cluster each take one segment of the vocabulary; the slice masses of the
-//       other CTAs are read through distributed shared memory by the cluster's first CTA, which finishes as
-//       terminal_kernel does.
+//   (3) The terminal draw over the last node's row: the S * WT_WARPS warps of the cluster each take one segment of
+//       the vocabulary; the slice masses of the other CTAs are read through distributed shared memory by the
+//       cluster's first CTA, which finishes as terminal_kernel does.  (Letting the statistics pass leave the mass
+//       of every slice of every row, so that this step reads a table and one slice, was tried: the table costs the
+//       statistics kernel as much as it saves here.)
 constexpr int WT_THREADS = 512;
 constexpr int WT_WARPS = WT_THREADS / 32;
 
@@ -1252,19 +1182,13 @@ struct WtLayout {
     size_t stage, ovm, first, mm, slices, seg, par, e, p, total;
     int G, vpw, n_sl;
 };
-__host__ __device__ inline WtLayout wt_layout(int N, int K, int k, int V, int S, bool tab) {
+__host__ __device__ inline WtLayout wt_layout(int N, int K, int k, int V, int S) {
     WtLayout L;
     auto up = [](size_t x) { return (x + 15) / 16 * 16; };
     const int nvec = V >> 3;
-    if (tab) {  // the segments are the table's slices; only the selected one is cut into 32-vector slices
-        L.G = row_slices(V);
-        L.vpw = 4 * 128;
-        L.n_sl = L.vpw / 32;
-    } else {
-        L.G = S * WT_WARPS;
-        L.vpw = (nvec + L.G - 1) / L.G;
-        L.n_sl = (L.vpw + 31) / 32;
-    }
+    L.G = S * WT_WARPS;
+    L.vpw = (nvec + L.G - 1) / L.G;
+    L.n_sl = (L.vpw + 31) / 32;
     size_t o = 0;
     L.stage = o;
     o += up(walk_stage_bytes(N, K, k));
@@ -1275,7 +1199,7 @@ __host__ __device__ inline WtLayout wt_layout(int N, int K, int k, int V, int S,
     L.mm = o;
     o += up((size_t)N * sizeof(float));
     L.slices = o;
-    o += up((size_t)(tab ? 1 : L.G) * L.n_sl * sizeof(double));
+    o += up((size_t)L.G * L.n_sl * sizeof(double));
     L.seg = o;
     o += up((size_t)L.G * sizeof(double));
     L.par = o;
@@ -1289,14 +1213,14 @@ __host__ __device__ inline WtLayout wt_layout(int N, int K, int k, int V, int S,
 }
 
 __global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, Topo topo, const float *__restrict__ u_fin, float c,
-                                                               int S, const float2 *__restrict__ tab) {
+                                                               int S) {
     __shared__ WalkSmem sh[WT_WARPS];
     extern __shared__ __align__(16) unsigned char sh_dyn[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rank = S > 1 ? (int)cluster_ctarank() : 0;
     const int b = blockIdx.x / S;
     const int N = a.N, K = a.K, k = a.k;
-    const WtLayout L = wt_layout(N, K, k, a.V, S, tab != nullptr);
+    const WtLayout L = wt_layout(N, K, k, a.V, S);
     auto up = [](size_t x) { return (x + 15) / 16 * 16; };
     unsigned char *p0 = sh_dyn + L.stage;
     float *rmax = reinterpret_cast<float *>(p0);
@@ -1433,19 +1357,7 @@ __global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, To
     const uint16_t *lg = a.logits + ((size_t)b * N + u) * a.V;
     const uint4 *p = reinterpret_cast<const uint4 *>(lg);
     const int nvec = a.V >> 3, vpw = L.vpw, n_sl = L.n_sl, G = L.G;
-    if (tab) {
-        const float2 *tb = tab + ((size_t)b * N + u) * G;
-        for (int g = tid; g < G; g += WT_THREADS) {
-            const float2 e = tb[g];
-            seg[g] = (double)e.y * (double)ex2_approx((e.x - M) * c);
-        }
-        __syncthreads();
-        if (tid == 0) {
-            const RowSlices rs(a.V);
-            for (int j = 0; j < nov; ++j) seg[rs.slice_of_token(ovid[j])] += ovm_u[j] - (double)mass1(pre[u * k + j], M, c, 0u);
-        }
-        __syncthreads();
-    } else {
+    {
         {
             const int g = rank * WT_WARPS + warp;
             const int v_lo = min(nvec, g * vpw), v_hi = min(nvec, v_lo + vpw);
@@ -1480,87 +1392,41 @@ __global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, To
         }
         __syncthreads();
     }
-    __shared__ int sh_wsel;
-    __shared__ double sh_bt[2];
+    if (warp != 0) return;
+    double total = 0.0;
+    for (int g0 = 0; g0 < G; g0 += 32) total += warp_sum(g0 + lane < G ? seg[g0 + lane] : 0.0);
+    const double target = (double)u_fin[b] * total;
+    int wsel = -1;
+    double base = 0.0;
+    for (int g0 = 0; g0 < G && wsel < 0; g0 += 32) {
+        const double v = g0 + lane < G ? seg[g0 + lane] : 0.0;
+        const double incl = warp_incl_scan(v, lane);
+        const unsigned hit = __ballot_sync(0xffffffffu, g0 + lane < G && base + incl > target);
+        if (hit) {
+            const int lh = __ffs(hit) - 1;
+            wsel = g0 + lh;
+            base += __shfl_sync(0xffffffffu, incl - v, lh);
+        } else {
+            base += __shfl_sync(0xffffffffu, incl, 31);
+        }
+    }
     int32_t *dst = a.out_tok + (size_t)b * (K + 1) + nacc;
-    if (warp == 0) {
-        double total = 0.0;
-        for (int g0 = 0; g0 < G; g0 += 32) total += warp_sum(g0 + lane < G ? seg[g0 + lane] : 0.0);
-        const double target = (double)u_fin[b] * total;
-        int wsel = -1;
-        double base = 0.0;
-        for (int g0 = 0; g0 < G && wsel < 0; g0 += 32) {
-            const double v = g0 + lane < G ? seg[g0 + lane] : 0.0;
-            const double incl = warp_incl_scan(v, lane);
-            const unsigned hit = __ballot_sync(0xffffffffu, g0 + lane < G && base + incl > target);
-            if (hit) {
-                const int lh = __ffs(hit) - 1;
-                wsel = g0 + lh;
-                base += __shfl_sync(0xffffffffu, incl - v, lh);
-            } else {
-                base += __shfl_sync(0xffffffffu, incl, 31);
-            }
-        }
-        if (wsel < 0) {
-            // u_fin * total reached the total through rounding: take the last token with positive mass
-            if (lane == 0) {
-                int tok = a.V - 1;
-                for (; tok > 0; --tok) {
-                    double ms = (double)mass1(lg[tok], M, c, 0u);
-                    for (int j = 0; j < nov; ++j)
-                        if (ovid[j] == tok) ms = ovm_u[j];
-                    if (ms > 0.0) break;
-                }
-                *dst = tok;
-            }
-        } else if (!tab) {
-            const int v_lo = min(nvec, wsel * vpw), v_hi = min(nvec, v_lo + vpw);
-            term_pick(p, slices + (size_t)wsel * n_sl, n_sl, v_lo, v_hi, base, target, M, c, 0u, nov, ovid, ovm_u, dst, lane);
-        }
+    if (wsel < 0) {
+        // u_fin * total reached the total through rounding: take the last token with positive mass
         if (lane == 0) {
-            sh_wsel = wsel;
-            sh_bt[0] = base;
-            sh_bt[1] = target;
+            int tok = a.V - 1;
+            for (; tok > 0; --tok) {
+                double ms = (double)mass1(lg[tok], M, c, 0u);
+                for (int j = 0; j < nov; ++j)
+                    if (ovid[j] == tok) ms = ovm_u[j];
+                if (ms > 0.0) break;
+            }
+            *dst = tok;
         }
-    }
-    if (!tab) return;
-    // with the table: the selected slice of the row is read now, one 32-vector slice per warp, all warps at once;
-    // the warp whose slice holds the target keeps its vectors' masses in registers and picks the token
-    static_assert(4 * 128 / 32 == WT_WARPS, "one 32-vector slice of a table slice per warp");
-    __syncthreads();
-    const int wsel = sh_wsel;
-    if (wsel < 0) return;
-    double base = sh_bt[0];
-    const double target = sh_bt[1];
-    int v_lo, v_hi;
-    RowSlices(a.V).vectors(wsel, &v_lo, &v_hi);
-    const int i = v_lo + warp * 32 + lane;
-    double ms[8];
-    const double lsum = term_vector_masses(p, i, v_hi, M, c, 0u, nov, ovid, ovm_u, ms);
-    {
-        const double sm_ = warp_sum(lsum);
-        if (lane == 0) slices[warp] = sm_;
-    }
-    __syncthreads();
-    // every warp finds the slice for itself (same numbers, same result)
-    const double v = lane < WT_WARPS ? slices[lane] : 0.0;
-    const double incl = warp_incl_scan(v, lane);
-    const unsigned hit = __ballot_sync(0xffffffffu, lane < WT_WARPS && base + incl > target);
-    const unsigned pos = __ballot_sync(0xffffffffu, v > 0.0);
-    bool take_last = false;
-    int sl_sel;
-    if (hit) {
-        sl_sel = __ffs(hit) - 1;
-    } else if (pos) {  // the slices fell short of the table's mass by rounding: the last slice with positive mass
-        sl_sel = 31 - __clz(pos);
-        take_last = true;
-    } else {
-        if (tid == 0) *dst = max(0, v_hi * 8 - 1);  // (no mass at all; keep a valid token)
         return;
     }
-    base += __shfl_sync(0xffffffffu, incl - v, sl_sel);
-    if (warp != sl_sel) return;
-    term_pick_token(i, ms, lsum, base, target, take_last, v_hi, dst, lane);
+    const int v_lo = min(nvec, wsel * vpw), v_hi = min(nvec, v_lo + vpw);
+    term_pick(p, slices + (size_t)wsel * n_sl, n_sl, v_lo, v_hi, base, target, M, c, 0u, nov, ovid, ovm_u, dst, lane);
 }
 
 // S CTAs per sequence: as many as keep the grid within about two CTAs per SM, a power of two up to the portable
@@ -1601,14 +1467,9 @@ static size_t verify_ws_base(const specroll_verify_desc *d) {
            align_up(B * sizeof(int32_t), 256) + 256;
 }
 
-// The slice table of the plain verification: one (reference, mass) pair per 4096-token slice of every row.
-static size_t verify_ws_table(const specroll_verify_desc *d) {
-    return align_up((size_t)d->B * d->N * row_slices(d->V) * sizeof(float2), 256);
-}
-
 extern "C" size_t specroll_verify_workspace_bytes(const specroll_verify_desc *d) {
     if (check_verify_desc(d) != SPECROLL_OK) return 0;
-    return verify_ws_base(d) + ((d->flags & SPECROLL_VERIFY_LAZY_STATS) ? 0 : verify_ws_table(d));
+    return verify_ws_base(d);
 }
 
 extern "C" size_t specroll_verify_nucleus_workspace_bytes(const specroll_verify_desc *d) {
@@ -1623,7 +1484,7 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
                       const float *cand_logit, const float *u_acc, const float *u_fin, int32_t *n_acc,
                       int32_t *path_node, int32_t *out_tok, int32_t *term_node, int32_t *term_kind, float *row_max,
                       float *row_sum, float *min_margin, float *nucleus_thr, float *nucleus_sum, void *workspace,
-                      size_t workspace_bytes, void *cuda_stream, bool table_optional = false) {
+                      size_t workspace_bytes, void *cuda_stream) {
     if (check_verify_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (!logits || !tree_tok || !tree_cand || !cand_id || !cand_logit || !u_acc || !u_fin || !n_acc ||
         !path_node || !out_tok || !term_node || !term_kind || !row_max || !row_sum)
@@ -1634,12 +1495,7 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
     if (!aligned16(logits)) return SPECROLL_EALIGN;
     if (d->B == 0) return SPECROLL_OK;
     const bool lazy = (d->flags & SPECROLL_VERIFY_LAZY_STATS) != 0;
-    // the slice table serves the plain verification with all rows' statistics; a caller with fixed scratch
-    // (table_optional) goes without it when it does not fit
-    bool use_table = !truncate && !lazy;
-    if (use_table && table_optional && workspace_bytes < verify_ws_base(d) + verify_ws_table(d)) use_table = false;
-    const size_t need = truncate ? specroll_verify_nucleus_workspace_bytes(d)
-                                 : verify_ws_base(d) + (use_table ? verify_ws_table(d) : 0);
+    const size_t need = truncate ? specroll_verify_nucleus_workspace_bytes(d) : verify_ws_base(d);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)
         return SPECROLL_EWORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -1657,14 +1513,9 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
 
     const float c = (float)(1.4426950408889634 / (double)d->temperature);
     const int rows = d->B * d->N;
-    float2 *tab = use_table ? reinterpret_cast<float2 *>(ws) : nullptr;  // (no nucleus arrays in this form)
     if (!lazy) {
-        if (use_table)
-            row_stats_kernel<true><<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
-                                                                row_sum, tab);
-        else
-            row_stats_kernel<false><<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
-                                                                 row_sum, nullptr);
+        row_stats_kernel<<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
+                                                      row_sum);
         SR_LAUNCH_CHECK();
     }
 
@@ -1710,8 +1561,8 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
     } else {
         // plain verification: the walk and the terminal draw in one launch, overlapping the statistics kernel's tail
         constexpr int WT_SMEM_LIMIT = 160 * 1024;
-        const int S = use_table ? 1 : walk_term_split(d->B);
-        const WtLayout L = wt_layout(d->N, d->K, d->k, d->V, S, use_table);
+        const int S = walk_term_split(d->B);
+        const WtLayout L = wt_layout(d->N, d->K, d->k, d->V, S);
         if (L.total > (size_t)WT_SMEM_LIMIT) return SPECROLL_ELIMIT;
         const int rc_ = device_setup(reinterpret_cast<const void *>(walk_term_kernel), WT_SMEM_LIMIT, nullptr);
         if (rc_ != SPECROLL_OK) return rc_;
@@ -1734,7 +1585,7 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
         }
         cfg.attrs = attrs;
         cfg.numAttrs = na;
-        SR_CUDA_TRY(cudaLaunchKernelEx(&cfg, walk_term_kernel, wa, topo, u_fin, c, S, (const float2 *)tab));
+        SR_CUDA_TRY(cudaLaunchKernelEx(&cfg, walk_term_kernel, wa, topo, u_fin, c, S));
         return SPECROLL_OK;
     }
     SR_LAUNCH_CHECK();
@@ -1900,7 +1751,7 @@ extern "C" int specroll_verify_nucleus(const specroll_verify_desc *d, float top_
     if (!(top_p > 0.f)) return SPECROLL_EINVAL;
     return run_verify(d, top_p, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
                       path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, nucleus_thr,
-                      nucleus_sum, workspace, workspace_bytes, cuda_stream, /*table_optional=*/true);
+                      nucleus_sum, workspace, workspace_bytes, cuda_stream);
 }
 
 // ------------------------------------------------------------------------------ allocation-free variant
@@ -1929,7 +1780,7 @@ extern "C" int specroll_verify_static(const specroll_verify_desc *d, const void 
                                       float *row_sum, float *min_margin, void *cuda_stream) {
     if (check_verify_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (d->B > SPECROLL_STATIC_MAX_B || (long long)d->B * d->k > SPECROLL_STATIC_MAX_BK) return SPECROLL_ELIMIT;
-    if (verify_ws_base(d) > STATIC_SCRATCH_BYTES) return SPECROLL_ELIMIT;
+    if (specroll_verify_workspace_bytes(d) > STATIC_SCRATCH_BYTES) return SPECROLL_ELIMIT;
     int dev = -1;
     SR_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= MAX_DEVICES) return SPECROLL_ELIMIT;
@@ -1945,8 +1796,7 @@ extern "C" int specroll_verify_static(const specroll_verify_desc *d, const void 
         }
         scratch = g_scratch_addr[dev];
     }
-    // (the slice table of the plain verification is used when it fits the scratch, else the row is read again)
-    return run_verify(d, 1.0f, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
-                      path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, nullptr, nullptr, scratch,
-                      STATIC_SCRATCH_BYTES, cuda_stream, true);
+    return specroll_verify(d, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
+                           path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, scratch,
+                           STATIC_SCRATCH_BYTES, cuda_stream);
 }
