@@ -17,10 +17,13 @@
 //                          memory.  Fallback for rows with thousands of equal large values: a radix search by
 //                          COUNT (four bits per pass) for the key of the kS-th largest value, a pass for the ids
 //                          above it, an ordered pass for the first ids that tie with it, a rank sort.
-//   feedback_kernel        the small quantities (q, p on S, the coefficient of every support row) by one warp,
-//                          then all threads gather the <= k + kS + 1 rows of W once and accumulate both
-//                          directions, three RMS reductions, and the memory update.
+//   feedback_vec_kernel    the small quantities (q, p on S, the coefficient of every support row) by one warp,
+//                          then the <= k + kS + 1 rows of W come through shared memory by asynchronous copies,
+//                          several rows in flight, and all threads accumulate both directions; three RMS
+//                          reductions, and the memory update.  (feedback_kernel: hidden sizes not a multiple of 8.)
 #include <math.h>
+
+#include <algorithm>
 
 #include "common.cuh"
 
@@ -73,8 +76,9 @@ struct TopkRadixSmem {
 };
 struct TopkListSmem {
     uint32_t best[fb::TOPK_THREADS];     // every thread's largest key
-    uint32_t key[fb::TOPK_LIST_CAP];     // candidates: elements at or above the bound
-    int id[fb::TOPK_LIST_CAP];
+    // candidates (elements at or above the bound): key in the upper word, the complement of the id in the lower one,
+    // so that "larger" is (key desc, id asc) and a rank is a count of one comparison per entry
+    unsigned long long ent[fb::TOPK_LIST_CAP];
 };
 
 // Exact Top_kS by a radix search over the counts (any row, also one with tens of thousands of equal values);
@@ -231,12 +235,19 @@ feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restr
     //      turned into a key once.
     auto as_bf162 = [](uint32_t w_) { return *reinterpret_cast<const __nv_bfloat162 *>(&w_); };
     __nv_bfloat162 mx2 = as_bf162(0xff80ff80u);  // (-inf, -inf)
-    for (int i = tid; i < nvec; i += 2 * TOPK_THREADS) {
-        const uint4 v = ld_nc_v4(p + i);
-        const int i1 = i + TOPK_THREADS;
-        const uint4 v1 = i1 < nvec ? ld_nc_v4(p + i1) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-        mx2 = __hmax2(__hmax2(__hmax2(as_bf162(v.x), as_bf162(v.y)), __hmax2(as_bf162(v.z), as_bf162(v.w))), mx2);
-        mx2 = __hmax2(__hmax2(__hmax2(as_bf162(v1.x), as_bf162(v1.y)), __hmax2(as_bf162(v1.z), as_bf162(v1.w))), mx2);
+    // (Taking the bound from the head of the row only, to read the row once, was tried: the bound is lower, the list
+    // several hundred entries long, and ranking it costs more than the second pass over a row that sits in L2.)
+    const int nvec1 = nvec;
+    for (int i = tid; i < nvec1; i += 4 * TOPK_THREADS) {  // four loads in flight per thread
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int iu = i + u * TOPK_THREADS;
+            v[u] = iu < nvec1 ? ld_nc_v4(p + iu) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            mx2 = __hmax2(__hmax2(__hmax2(as_bf162(v[u].x), as_bf162(v[u].y)), __hmax2(as_bf162(v[u].z), as_bf162(v[u].w))), mx2);
     }
     const uint32_t mxb = *reinterpret_cast<const uint32_t *>(&mx2);
     const uint32_t best = max(ord_key16(mxb & 0xffffu), ord_key16(mxb >> 16));
@@ -244,11 +255,11 @@ feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restr
     __syncthreads();
     {
         // the n_sel-th largest of the threads' values (ties broken by thread index: any of them will do as the bound)
+        // (compared as (value, thread) pairs in one word; the loads do not depend on the count: unrolled)
+        const uint32_t mine = (best << 10) | (uint32_t)(TOPK_THREADS - 1 - tid);
         int rk = 0;
-        for (int j = 0; j < TOPK_THREADS; ++j) {
-            const uint32_t o = sm.list.best[j];
-            rk += (o > best) || (o == best && j < tid);
-        }
+#pragma unroll 8
+        for (int j = 0; j < TOPK_THREADS; ++j) rk += ((sm.list.best[j] << 10) | (uint32_t)(TOPK_THREADS - 1 - j)) > mine;
         if (rk == min(n_sel, TOPK_THREADS) - 1) sh_bound = best;
     }
     __syncthreads();
@@ -257,21 +268,29 @@ feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restr
     //      value; a vector of eight with nothing to keep (nearly all of them) costs four compares and one branch.
     const uint32_t bbits = (bound & 0x8000u) ? (bound & 0x7fffu) : (~bound & 0xffffu);  // the key undone
     const __nv_bfloat162 bnd2 = as_bf162(bbits | (bbits << 16));
-    for (int i = tid; i < nvec; i += TOPK_THREADS) {
-        const uint4 v = ld_nc_v4(p + i);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        uint32_t m[4];
+    for (int i0 = tid; i0 < nvec; i0 += 8 * TOPK_THREADS) {  // eight loads in flight per thread
+        uint4 vv[8];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) m[j] = __hge2_mask(as_bf162(w[j]), bnd2);
-        if ((m[0] | m[1] | m[2] | m[3]) == 0u) continue;
+        for (int u = 0; u < 8; ++u) {
+            const int iu = i0 + u * TOPK_THREADS;
+            vv[u] = iu < nvec ? ld_nc_v4(p + iu) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+        }
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            if ((m[t >> 1] >> (16 * (t & 1))) & 0xffffu) {
-                const uint32_t key = ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
-                const int pos = atomicAdd(&sh_n, 1);
-                if (pos < TOPK_LIST_CAP) {
-                    sm.list.key[pos] = key;
-                    sm.list.id[pos] = i * 8 + t;
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * TOPK_THREADS;
+            if (i >= nvec) continue;  // (a -inf filler would pass a bound of -inf)
+            const uint32_t w[4] = {vv[u].x, vv[u].y, vv[u].z, vv[u].w};
+            uint32_t m[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) m[j] = __hge2_mask(as_bf162(w[j]), bnd2);
+            if ((m[0] | m[1] | m[2] | m[3]) == 0u) continue;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                if ((m[t >> 1] >> (16 * (t & 1))) & 0xffffu) {
+                    const uint32_t key = ord_key16((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
+                    const int pos = atomicAdd(&sh_n, 1);
+                    if (pos < TOPK_LIST_CAP)
+                        sm.list.ent[pos] = ((unsigned long long)key << 32) | (uint32_t)(0x7fffffff - (i * 8 + t));
                 }
             }
         }
@@ -291,14 +310,11 @@ feedback_topk_kernel(const uint16_t *__restrict__ logits, const int32_t *__restr
     }
     // ---- rank within the list
     for (int e = tid; e < n; e += TOPK_THREADS) {
-        const uint32_t ke = sm.list.key[e];
-        const int ie = sm.list.id[e];
+        const unsigned long long me = sm.list.ent[e];
         int rk = 0;
-        for (int j = 0; j < n; ++j) {
-            const uint32_t kj = sm.list.key[j];
-            rk += (kj > ke) || (kj == ke && sm.list.id[j] < ie);
-        }
-        if (rk < n_sel) out[rk] = ie;
+#pragma unroll 8
+        for (int j = 0; j < n; ++j) rk += sm.list.ent[j] > me;
+        if (rk < n_sel) out[rk] = 0x7fffffff - (int)(uint32_t)(me & 0xffffffffull);
     }
 }
 
@@ -318,31 +334,43 @@ struct FeedbackArgs {
     float *severity, *e_out;  // optional outputs: w per record, the feedback vector e per record
     int R, k, kS, d, V;
     float inv_T, eps;
+    int rows_per_stage;  // (vector kernel) support rows of W per batch in shared memory
     int weighted;        // the update is weighted by the severity, records below severity_min are discarded
     float severity_min;
 };
 
-// MAXC = columns of the hidden dimension per thread (d <= 256 * MAXC)
-template <int MAXC>
-__global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a) {
+// The small quantities of one record, in shared memory.
+struct FeedbackSmall {
+    int id[fb::MAX_S];
+    float p[fb::MAX_S];      // target mass exp((l - M)/T) / row_sum of the support tokens
+    float adist[fb::MAX_S];  // coefficient of W_v in r_dist
+    float acov[fb::MAX_S];   // coefficient of W_v in r_cov
+    float q[SPECROLL_MAX_TOPK];
+    int raw_id[fb::MAX_S];   // C, Top_kS, y* as they come (with duplicates)
+    float raw_p[fb::MAX_S];
+    int n;
+    float dd, dc, w;
+};
+
+// q, p on S, the coefficient of every support row, the scalar outputs.  All threads fetch the ids and the target
+// logits at them (two rounds of independent loads); one warp does the rest from shared memory.  Ends with a barrier.
+__device__ void feedback_small(const FeedbackArgs &a, int r, FeedbackSmall &s) {
     using namespace fb;
-    __shared__ int s_id[MAX_S];
-    __shared__ float s_p[MAX_S];      // target mass exp((l - M)/T) / row_sum of the support tokens
-    __shared__ float s_adist[MAX_S];  // coefficient of W_v in r_dist
-    __shared__ float s_acov[MAX_S];   // coefficient of W_v in r_cov
-    __shared__ float s_q[SPECROLL_MAX_TOPK];
-    __shared__ int s_n;
-    __shared__ float s_dd, s_dc, s_w;
-    __shared__ float red[FB_THREADS / 32];
-    const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int k = a.k, kS = a.kS, d = a.d;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int k = a.k, kS = a.kS;
     const size_t row = (size_t)a.rec_row[r];
     const uint16_t *lg = a.logits + row * a.V;
     const float M = a.row_max[row], Ssum = a.row_sum[row];
     const int32_t *cid = a.cand_id + (size_t)r * k;
     const float *cl = a.cand_logit + (size_t)r * k;
     const int32_t *top = a.top_id + (size_t)r * kS;
-
+    const int n_raw = k + kS + 1;
+    for (int i = tid; i < n_raw; i += blockDim.x) {
+        const int v = i < k ? cid[i] : (i < k + kS ? top[i - k] : a.y_star[r]);
+        s.raw_id[i] = v;
+        s.raw_p[i] = (v >= 0 && v < a.V) ? __expf((__uint_as_float((uint32_t)lg[v] << 16) - M) * a.inv_T) / Ssum : 0.f;
+    }
+    __syncthreads();
     if (warp == 0) {
         // ---- q on the candidates
         float mx = -INFINITY;
@@ -351,73 +379,65 @@ __global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a
         float qs = 0.f;
         for (int j = lane; j < k; j += 32) {
             const float w = __expf((cl[j] - mx) * a.inv_T);
-            s_q[j] = w;
+            s.q[j] = w;
             qs += w;
         }
         qs = warp_sum(qs);
         __syncwarp();
-        for (int j = lane; j < k; j += 32) s_q[j] /= qs;
+        for (int j = lane; j < k; j += 32) s.q[j] /= qs;
         // ---- S = C u Top_kS u {y*}, duplicates removed (first occurrence kept; the candidates come first)
-        const int n_raw = k + kS + 1;
-        if (lane == 0) s_n = 0;
+        if (lane == 0) s.n = 0;
         __syncwarp();
         for (int i0 = 0; i0 < n_raw; i0 += 32) {
             const int i = i0 + lane;
-            int v = -1;
-            if (i < k)
-                v = cid[i];
-            else if (i < k + kS)
-                v = top[i - k];
-            else if (i == k + kS)
-                v = a.y_star[r];
+            const int v = i < n_raw ? s.raw_id[i] : -1;
             bool fresh = v >= 0 && v < a.V;
             if (fresh) {
                 for (int j = 0; j < i; ++j) {  // the same token earlier in the concatenation?
-                    const int u = j < k ? cid[j] : (j < k + kS ? top[j - k] : a.y_star[r]);
-                    if (u == v) {
+                    if (s.raw_id[j] == v) {
                         fresh = false;
                         break;
                     }
                 }
             }
             const unsigned bal = __ballot_sync(0xffffffffu, fresh);
-            const int base = s_n;
+            const int base = s.n;
             if (fresh) {
                 const int pos = base + __popc(bal & ((1u << lane) - 1u));
-                s_id[pos] = v;
-                s_p[pos] = __expf((__uint_as_float((uint32_t)lg[v] << 16) - M) * a.inv_T) / Ssum;
+                s.id[pos] = v;
+                s.p[pos] = s.raw_p[i];
             }
             __syncwarp();
-            if (lane == 0) s_n = base + __popc(bal);
+            if (lane == 0) s.n = base + __popc(bal);
             __syncwarp();
         }
-        const int n = s_n;
+        const int n = s.n;
         // ---- masses: p(S), p(C), p(C*); TV on C
         float pS = 0.f;
-        for (int i = lane; i < n; i += 32) pS += s_p[i];
+        for (int i = lane; i < n; i += 32) pS += s.p[i];
         pS = warp_sum(pS);
         float pC = 0.f;
-        for (int j = lane; j < k; j += 32) pC += s_p[j];  // the first k support entries are the candidates
+        for (int j = lane; j < k; j += 32) pC += s.p[j];  // the first k support entries are the candidates
         pC = warp_sum(pC);
         float tvs = 0.f;
-        for (int j = lane; j < k; j += 32) tvs += fabsf(s_p[j] / pC - s_q[j]);
+        for (int j = lane; j < k; j += 32) tvs += fabsf(s.p[j] / pC - s.q[j]);
         tvs = 0.5f * warp_sum(tvs);
         // C* = the first k of Top_kS; O = C* \ C
         float pCs = 0.f, cov_b = 0.f;
-        for (int i = lane; i < n; i += 32) s_acov[i] = 0.f;
+        for (int i = lane; i < n; i += 32) s.acov[i] = 0.f;
         __syncwarp();
         for (int t = lane; t < k; t += 32) {
-            const int v = top[t];
-            const float pv = __expf((__uint_as_float((uint32_t)lg[v] << 16) - M) * a.inv_T) / Ssum;
+            const int v = s.raw_id[k + t];
+            const float pv = s.raw_p[k + t];
             pCs += pv;
             bool inC = false;
-            for (int j = 0; j < k; ++j) inC |= (cid[j] == v);
+            for (int j = 0; j < k; ++j) inC |= (s.raw_id[j] == v);
             if (!inC) {
                 // an omitted target-important token: +p_S(y) on its own row, -p_S(y) on the weakest candidate's
                 int pos = -1;
                 for (int i = k; i < n; ++i)
-                    if (s_id[i] == v) pos = i;
-                if (pos >= 0) s_acov[pos] = pv / pS;
+                    if (s.id[i] == v) pos = i;
+                if (pos >= 0) s.acov[pos] = pv / pS;
                 cov_b += pv / pS;
             }
         }
@@ -426,26 +446,42 @@ __global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a
         __syncwarp();
         float tvS = 0.f;  // TV(p_S, q_S)
         for (int i = lane; i < n; i += 32) {
-            const float ad = s_p[i] / pS - (i < k ? s_q[i] : 0.f);
-            s_adist[i] = ad;
+            const float ad = s.p[i] / pS - (i < k ? s.q[i] : 0.f);
+            s.adist[i] = ad;
             tvS += fabsf(ad);
         }
         tvS = 0.5f * warp_sum(tvS);
         if (lane == 0) {
             // severity of the observation: w = clip(0.3 TV(p_S, q_S) + 0.7 p_out, 0, 1), p_out = 1 - p(C)
             const float w = fminf(1.f, fmaxf(0.f, 0.3f * tvS + 0.7f * (1.f - pC)));
-            s_w = w;
+            s.w = w;
             if (a.severity) a.severity[r] = w;
-            s_acov[k - 1] -= cov_b;  // b* = last candidate (the list is sorted by logit)
+            s.acov[k - 1] -= cov_b;  // b* = last candidate (the list is sorted by logit)
             const float dd = pC * tvs, dc = pCs - pC;
-            s_dd = dd;
-            s_dc = dc;
+            s.dd = dd;
+            s.dc = dc;
             if (a.d_dist) a.d_dist[r] = dd;
             if (a.d_cov) a.d_cov[r] = dc;
             if (a.tv) a.tv[r] = tvs;
         }
     }
     __syncthreads();
+}
+
+// Hidden sizes that are not a multiple of eight: thread t owns columns t, t + 256, ...
+// MAXC = columns of the hidden dimension per thread (d <= 256 * MAXC)
+template <int MAXC>
+__global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a) {
+    using namespace fb;
+    __shared__ FeedbackSmall sm;
+    __shared__ float red[FB_THREADS / 32];
+    const int r = blockIdx.x, tid = threadIdx.x;
+    const int d = a.d;
+    feedback_small(a, r, sm);
+    const int *s_id = sm.id;
+    const float *s_adist = sm.adist, *s_acov = sm.acov;
+    const int s_n = sm.n;
+    const float s_dd = sm.dd, s_dc = sm.dc, s_w = sm.w;
     const int n = s_n;
     const float dd = s_dd, dc = s_dc;
     // ---- both directions: thread t owns columns t, t + 256, ...; the support rows of W are read once
@@ -496,6 +532,121 @@ __global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a
             const float e = fe * rd[c];
             if (er) er[col] = e;
             if (keep) mr[col] = rho * mr[col] + gain * e;
+        }
+    }
+}
+
+// Hidden sizes that are a multiple of eight: thread t owns the 8-column vectors t, t + 512, ... (NV of them), a row
+// of W is read with 128-bit loads, and four support rows are in flight at a time: a record's 57 rows of W are a few
+// hundred KB fetched by one CTA, so what bounds the kernel is how many bytes that CTA keeps in flight.
+constexpr int FBV_THREADS = 512;
+template <int NV>
+__global__ void __launch_bounds__(FBV_THREADS) feedback_vec_kernel(FeedbackArgs a) {
+    using namespace fb;
+    __shared__ FeedbackSmall sm;
+    __shared__ float red[FBV_THREADS / 32];
+    extern __shared__ __align__(16) unsigned char fb_stage[];  // [3][rows_per_stage][d] bf16
+    const int r = blockIdx.x, tid = threadIdx.x;
+    const int d = a.d, nvec = d >> 3;
+    feedback_small(a, r, sm);
+    const int n = sm.n;
+    const float dd = sm.dd, dc = sm.dc;
+    float rd[NV][8], rc[NV][8];
+#pragma unroll
+    for (int c = 0; c < NV; ++c)
+#pragma unroll
+        for (int t = 0; t < 8; ++t) rd[c][t] = rc[c][t] = 0.f;
+    // The support rows of W come through shared memory in batches of rps rows, three batches deep, by asynchronous
+    // copies: two batches are on their way while one is used.  (With plain loads into registers the compiler kept one
+    // row in flight at a time, to save registers: 57 round trips to memory one after the other.)
+    constexpr int STAGES = 3;
+    const int rps = a.rows_per_stage;
+    const size_t stage_bytes = (size_t)rps * d * 2;
+    const int nb = (n + rps - 1) / rps;
+    auto issue = [&](int batch) {
+        if (batch < nb) {
+            const uint32_t dst = smem_u32(fb_stage + (size_t)(batch % STAGES) * stage_bytes);
+            for (int ch = tid; ch < rps * nvec; ch += FBV_THREADS) {
+                const int q = ch / nvec, vi = ch - q * nvec, i = batch * rps + q;
+                if (i < n) cp_async16(dst + (uint32_t)ch * 16u, a.W + (size_t)sm.id[i] * d + (size_t)vi * 8, true);
+            }
+        }
+        cp_async_commit();  // (an empty group when there is nothing left: the count below stays the same)
+    };
+    issue(0);
+    issue(1);
+    for (int b = 0; b < nb; ++b) {
+        issue(b + 2);
+        cp_async_wait<2>();  // everything up to batch b has landed
+        __syncthreads();
+        const unsigned char *src = fb_stage + (size_t)(b % STAGES) * stage_bytes;
+        for (int q = 0; q < rps; ++q) {
+            const int i = b * rps + q;
+            if (i >= n) break;
+            const float ad = sm.adist[i], ac = sm.acov[i];
+#pragma unroll
+            for (int c = 0; c < NV; ++c) {
+                const int vi = tid + c * FBV_THREADS;
+                if (vi < nvec) {
+                    const uint4 v = *reinterpret_cast<const uint4 *>(src + ((size_t)q * nvec + vi) * 16);
+                    const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const float lo = __uint_as_float(w4[t] << 16), hi = __uint_as_float(w4[t] & 0xffff0000u);
+                        rd[c][2 * t] = fmaf(ad, lo, rd[c][2 * t]);
+                        rd[c][2 * t + 1] = fmaf(ad, hi, rd[c][2 * t + 1]);
+                        rc[c][2 * t] = fmaf(ac, lo, rc[c][2 * t]);
+                        rc[c][2 * t + 1] = fmaf(ac, hi, rc[c][2 * t + 1]);
+                    }
+                }
+            }
+        }
+        __syncthreads();  // the stage is free for the batch three further on
+    }
+    float sd = 0.f, scv = 0.f;
+#pragma unroll
+    for (int c = 0; c < NV; ++c)
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            sd += rd[c][t] * rd[c][t];
+            scv += rc[c][t] * rc[c][t];
+        }
+    sd = block_sum_f<FBV_THREADS>(sd, red);
+    scv = block_sum_f<FBV_THREADS>(scv, red);
+    const float fd = dd / (sqrtf(sd / d) + a.eps), fc = dc / (sqrtf(scv / d) + a.eps);
+    float sg = 0.f;
+#pragma unroll
+    for (int c = 0; c < NV; ++c)
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            rd[c][t] = fd * rd[c][t] + fc * rc[c][t];  // g
+            sg += rd[c][t] * rd[c][t];
+        }
+    sg = block_sum_f<FBV_THREADS>(sg, red);
+    const float fe = (dd + dc) / (sqrtf(sg / d) + a.eps);
+    const float rho = a.rho[r];
+    const float w = sm.w;
+    const bool keep = !a.weighted || w >= a.severity_min;
+    const float gain = (1.f - rho) * (a.weighted ? w : 1.f);
+    float4 *mr = reinterpret_cast<float4 *>(a.m + (size_t)a.rec_mem[r] * d);
+    float4 *er = a.e_out ? reinterpret_cast<float4 *>(a.e_out + (size_t)r * d) : nullptr;
+#pragma unroll
+    for (int c = 0; c < NV; ++c) {
+        const int vi = tid + c * FBV_THREADS;
+        if (vi < nvec) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float4 e = make_float4(fe * rd[c][4 * h], fe * rd[c][4 * h + 1], fe * rd[c][4 * h + 2], fe * rd[c][4 * h + 3]);
+                if (er) er[2 * vi + h] = e;
+                if (keep) {
+                    float4 mv = mr[2 * vi + h];
+                    mv.x = rho * mv.x + gain * e.x;
+                    mv.y = rho * mv.y + gain * e.y;
+                    mv.z = rho * mv.z + gain * e.z;
+                    mv.w = rho * mv.w + gain * e.w;
+                    mr[2 * vi + h] = mv;
+                }
+            }
         }
     }
 }
@@ -574,7 +725,25 @@ extern "C" int specroll_reflex_feedback_ex(const specroll_feedback_desc *d, cons
     a.V = d->V;
     a.inv_T = 1.0f / d->temperature;
     a.eps = d->eps;
-    if (d->d <= 8 * fb::FB_THREADS)
+    // (m and e_out rows start at multiples of d floats: 16-byte aligned when d % 8 == 0 and the bases are)
+    const bool vec = (d->d % 8) == 0 && aligned16(m) && (!e_out || aligned16(e_out));
+    // batches of at most 24 KB of W rows, three deep: three CTAs fit an SM
+    a.rows_per_stage = std::max(1, std::min(8, 24576 / (d->d * 2)));
+    const size_t fb_smem = (size_t)3 * a.rows_per_stage * d->d * 2;
+    if (vec) {
+        const void *kern = d->d <= 8 * FBV_THREADS    ? reinterpret_cast<const void *>(feedback_vec_kernel<1>)
+                           : d->d <= 16 * FBV_THREADS ? reinterpret_cast<const void *>(feedback_vec_kernel<2>)
+                                                      : reinterpret_cast<const void *>(feedback_vec_kernel<3>);
+        const int rc_ = device_setup(kern, 112 * 1024, nullptr);
+        if (rc_ != SPECROLL_OK) return rc_;
+    }
+    if (vec && d->d <= 8 * FBV_THREADS)
+        feedback_vec_kernel<1><<<d->R, FBV_THREADS, fb_smem, st>>>(a);
+    else if (vec && d->d <= 16 * FBV_THREADS)
+        feedback_vec_kernel<2><<<d->R, FBV_THREADS, fb_smem, st>>>(a);
+    else if (vec)
+        feedback_vec_kernel<3><<<d->R, FBV_THREADS, fb_smem, st>>>(a);
+    else if (d->d <= 8 * fb::FB_THREADS)
         feedback_kernel<8><<<d->R, fb::FB_THREADS, 0, st>>>(a);
     else if (d->d <= 24 * fb::FB_THREADS)
         feedback_kernel<24><<<d->R, fb::FB_THREADS, 0, st>>>(a);

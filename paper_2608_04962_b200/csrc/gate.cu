@@ -14,19 +14,51 @@ constexpr int SK_THREADS = 256;
 constexpr int MAX_RANK = 32;
 }  // namespace gt
 
-// One block per record: y = Pi x (rank dot products of length d, a warp each, round robin), then y / ||y||.
+// One block per record: y = Pi x (rank dot products of length d), then y / ||y||.  A warp takes the ranks warp,
+// warp + 8, ... (four at most) together, so x is read once per warp; with d % 4 == 0 and 16-byte aligned rows the
+// loads are 128-bit and independent of the running sums, several in flight per lane.  (A record's x and Pi's rows
+// are a few hundred KB fetched by one CTA: what bounds the kernel is how many bytes it keeps in flight.)
 __global__ void __launch_bounds__(gt::SK_THREADS) sketch_kernel(int d, int rank, const float *__restrict__ X,
                                                                  const int32_t *__restrict__ rows,
-                                                                 const float *__restrict__ Pi, float *__restrict__ sketch) {
+                                                                 const float *__restrict__ Pi, float *__restrict__ sketch,
+                                                                 int vec) {
     __shared__ float y[gt::MAX_RANK];
+    constexpr int NW = gt::SK_THREADS / 32, RPW = gt::MAX_RANK / NW;
     const int r = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float *x = X + (size_t)(rows ? rows[r] : r) * d;
-    for (int i = warp; i < rank; i += gt::SK_THREADS / 32) {
-        const float *p = Pi + (size_t)i * d;
-        float acc = 0.f;
-        for (int c = lane; c < d; c += 32) acc = fmaf(p[c], x[c], acc);
-        acc = warp_sum(acc);
-        if (lane == 0) y[i] = acc;
+    float acc[RPW];
+#pragma unroll
+    for (int q = 0; q < RPW; ++q) acc[q] = 0.f;
+    if (vec) {
+        const float4 *x4 = reinterpret_cast<const float4 *>(x);
+        const float4 *p4 = reinterpret_cast<const float4 *>(Pi);
+        const int d4 = d >> 2;
+#pragma unroll 2
+        for (int c = lane; c < d4; c += 32) {
+            const float4 xv = x4[c];
+#pragma unroll
+            for (int q = 0; q < RPW; ++q) {
+                const int i = warp + q * NW;
+                if (i < rank) {
+                    const float4 pv = p4[(size_t)i * d4 + c];
+                    acc[q] = fmaf(pv.x, xv.x, fmaf(pv.y, xv.y, fmaf(pv.z, xv.z, fmaf(pv.w, xv.w, acc[q]))));
+                }
+            }
+        }
+    } else {
+        for (int c = lane; c < d; c += 32) {
+            const float xv = x[c];
+#pragma unroll
+            for (int q = 0; q < RPW; ++q) {
+                const int i = warp + q * NW;
+                if (i < rank) acc[q] = fmaf(Pi[(size_t)i * d + c], xv, acc[q]);
+            }
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < RPW; ++q) {
+        const float t = warp_sum(acc[q]);
+        if (lane == 0 && warp + q * NW < rank) y[warp + q * NW] = t;
     }
     __syncthreads();
     if (warp == 0) {
@@ -71,24 +103,49 @@ __global__ void __launch_bounds__(256) gate_kernel(GateArgs g, const float *__re
     if (j >= g.S) return;
     int n = g.n[j], nfb = g.n_fb[j];
     float mean = g.mean[j], M2 = g.M2[j];
-    for (int r0 = 0; r0 < g.R; r0 += 32) {
-        const int r = r0 + lane;
-        const bool mine = r < g.R && g.slot[r] == j && (!g.keep || g.keep[r]);
-        unsigned bal = __ballot_sync(0xffffffffu, mine);
-        while (bal) {
-            const int src = __ffs(bal) - 1;
-            bal &= bal - 1;
-            const float av = a[r0 + src];
-            n += 1;
-            const float delta = av - mean;
-            mean += delta / (float)n;
-            M2 += delta * (av - mean);
-            nfb += 1;
+    // the records in batches of 256: a lane's eight loads of a batch are independent of the recurrences
+    for (int r0 = 0; r0 < g.R; r0 += 256) {
+        unsigned mine = 0u;
+        float av[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int r = r0 + q * 32 + lane;
+            const bool mq = r < g.R && g.slot[r] == j && (!g.keep || g.keep[r]);
+            mine |= (mq ? 1u : 0u) << q;
+            av[q] = r < g.R ? a[r] : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            unsigned bal = __ballot_sync(0xffffffffu, (mine >> q) & 1u);
+            while (bal) {
+                const int src = __ffs(bal) - 1;
+                bal &= bal - 1;
+                const float v = __shfl_sync(0xffffffffu, av[q], src);
+                n += 1;
+                const float delta = v - mean;
+                mean += delta / (float)n;
+                M2 += delta * (v - mean);
+                nfb += 1;
+            }
         }
     }
     float ss = 0.f;
     const float *mr = g.m + (size_t)j * g.d;
-    for (int c = lane; c < g.d; c += 32) ss = fmaf(mr[c], mr[c], ss);
+    if ((g.d % 4) == 0 && (reinterpret_cast<uintptr_t>(g.m) & 15u) == 0) {
+        const float4 *m4 = reinterpret_cast<const float4 *>(mr);
+        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int c = lane; c < (g.d >> 2); c += 32) {
+            const float4 v = m4[c];
+            s4[0] = fmaf(v.x, v.x, s4[0]);
+            s4[1] = fmaf(v.y, v.y, s4[1]);
+            s4[2] = fmaf(v.z, v.z, s4[2]);
+            s4[3] = fmaf(v.w, v.w, s4[3]);
+        }
+        ss = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+    } else {
+        for (int c = lane; c < g.d; c += 32) ss = fmaf(mr[c], mr[c], ss);
+    }
     ss = warp_sum(ss);
     if (lane == 0) {
         g.n[j] = n;
@@ -114,7 +171,8 @@ extern "C" int specroll_reflex_sketch(int32_t R, int32_t d, int32_t rank, const 
     if (R < 0 || d < 1 || rank < 1 || rank > gt::MAX_RANK) return SPECROLL_EINVAL;
     if (R == 0) return SPECROLL_OK;
     if (!X || !Pi || !sketch) return SPECROLL_EINVAL;
-    sketch_kernel<<<R, gt::SK_THREADS, 0, static_cast<cudaStream_t>(cuda_stream)>>>(d, rank, X, rows, Pi, sketch);
+    const int vec = (d % 4) == 0 && aligned16(X) && aligned16(Pi);
+    sketch_kernel<<<R, gt::SK_THREADS, 0, static_cast<cudaStream_t>(cuda_stream)>>>(d, rank, X, rows, Pi, sketch, vec);
     SR_LAUNCH_CHECK();
     return SPECROLL_OK;
 }
