@@ -285,6 +285,83 @@ topk_merge_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pi
     }
 }
 
+// The same for k <= 8, the size of the tensor-core projection's partial lists: every lane first keeps the k best of
+// its own share of the partial entries in registers (one pass, the loads independent of each other), then k rounds of
+// arg-best over the lanes' current best, the winner moving on to its next one.  (Re-reading all entries in each of
+// the k rounds made this kernel a tenth of the call at small batch.)
+__global__ void __launch_bounds__(128)
+topk_merge8_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pid, int M, int n_cand, int k,
+                   int32_t *__restrict__ cand_id, float *__restrict__ cand_logit) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 4 + warp;
+    if (r >= M) return;
+    const float *v = pval + (size_t)r * n_cand;
+    const int32_t *id = pid + (size_t)r * n_cand;
+    float lv[8];
+    int32_t li[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        lv[i] = -INFINITY;
+        li[i] = 0x7fffffff;
+    }
+    auto better = [](float x, int32_t t, float y, int32_t u) { return x > y || (x == y && t < u); };
+    for (int c0 = lane; c0 < n_cand; c0 += 4 * 32) {
+        float x[4];
+        int32_t t[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int c = c0 + q * 32;
+            x[q] = c < n_cand ? v[c] : -INFINITY;
+            t[q] = c < n_cand ? id[c] : 0x7fffffff;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (!better(x[q], t[q], lv[7], li[7])) continue;
+            // insert into the sorted list (best first)
+#pragma unroll
+            for (int i = 7; i > 0; --i) {
+                if (better(x[q], t[q], lv[i - 1], li[i - 1])) {
+                    lv[i] = lv[i - 1];
+                    li[i] = li[i - 1];
+                } else if (better(x[q], t[q], lv[i], li[i])) {
+                    lv[i] = x[q];
+                    li[i] = t[q];
+                }
+            }
+            if (better(x[q], t[q], lv[0], li[0])) {
+                lv[0] = x[q];
+                li[0] = t[q];
+            }
+        }
+    }
+    for (int j = 0; j < k; ++j) {
+        float bv = lv[0];
+        int32_t bi = li[0];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (better(ov, oi, bv, bi)) {
+                bv = ov;
+                bi = oi;
+            }
+        }
+        if (lv[0] == bv && li[0] == bi) {  // (ids are distinct: one lane) this lane's best was taken
+#pragma unroll
+            for (int i = 0; i < 7; ++i) {
+                lv[i] = lv[i + 1];
+                li[i] = li[i + 1];
+            }
+            lv[7] = -INFINITY;
+            li[7] = 0x7fffffff;
+        }
+        if (lane == 0) {
+            cand_id[(size_t)r * k + j] = bi;
+            cand_logit[(size_t)r * k + j] = bv;
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------ P5 tree draw
 
 constexpr int DRAW_WARPS = 8;
@@ -585,7 +662,10 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
         SR_LAUNCH_CHECK();
     }
 
-    topk_merge_kernel<<<(p.M + 3) / 4, 128, 0, st>>>(pval, pid, p.M, p.n_groups * k, k, cand_id, cand_logit);
+    if (k <= 8)
+        topk_merge8_kernel<<<(p.M + 3) / 4, 128, 0, st>>>(pval, pid, p.M, p.n_groups * k, k, cand_id, cand_logit);
+    else
+        topk_merge_kernel<<<(p.M + 3) / 4, 128, 0, st>>>(pval, pid, p.M, p.n_groups * k, k, cand_id, cand_logit);
     SR_LAUNCH_CHECK();
 
     return launch_tree_draw(topo, B, K, k, d->temperature, anchor_tok, cand_id, cand_logit, u_draw, tree_tok,
