@@ -21,6 +21,25 @@ int note_cuda_error(cudaError_t e);
 
 #define SR_LAUNCH_CHECK() SR_CUDA_TRY(cudaGetLastError())
 
+#ifdef __CUDACC__
+// Launch as the programmatic dependent of the kernel before it in the stream (pdl = false: an ordinary launch).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(bool pdl, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Raises a kernel's dynamic shared-memory limit the first time the kernel is launched on the current device
 // (the attribute is per device), and optionally returns that device's SM count.  Thread-safe; later calls for
 // the same (kernel, device) cost one table look-up.  Returns SPECROLL_OK or SPECROLL_ECUDA.
@@ -123,6 +142,12 @@ __device__ __forceinline__ uint4 ld_nc_v4(const void *p) {
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
+
+// Programmatic dependent launch: a kernel lets the next one in the stream start its prologue (pdl_launch_dependents)
+// and waits for the one before it to complete, with its memory visible (pdl_wait; returns at once in a kernel that
+// was launched the ordinary way).  Everything a kernel reads from, or writes to, global memory comes after its wait.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Thread-block clusters: this CTA's rank, a barrier over all threads of the cluster (release / acquire), and a
 // load from the same shared-memory offset in another CTA of the cluster.

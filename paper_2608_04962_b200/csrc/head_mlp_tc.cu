@@ -38,6 +38,7 @@ head_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     using C = Cfg<BN>;
     constexpr int STAGES = C::STAGES;
     extern __shared__ unsigned char smem_raw[];
+    pdl_launch_dependents();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // 1024-byte alignment for the 128-byte swizzle atoms
     unsigned char *aligned = smem_raw + (base - raw);
@@ -73,6 +74,7 @@ head_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // set up under the tail of the kernel before; its outputs are read from here on
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -180,10 +182,10 @@ static int launch_bn(const CUtensorMap &tmW, const void *xhat, int KX, const voi
     if (rc != SPECROLL_OK) return rc;
     if ((rc = device_setup(reinterpret_cast<const void *>(head_mlp_tc_kernel<BN>), C::SMEM_BYTES, nullptr)) != SPECROLL_OK) return rc;
     const dim3 grid((unsigned)((d + BM - 1) / BM), (unsigned)((B + BN - 1) / BN), (unsigned)K);
-    head_mlp_tc_kernel<BN><<<grid, THREADS, C::SMEM_BYTES, st>>>(
-        tmW, tmX, KX, static_cast<const __nv_bfloat16 *>(bias), static_cast<const __nv_bfloat16 *>(h), z, B, K, d,
-        status);
-    SR_LAUNCH_CHECK();
+    // (the dependent of the LayerNorm kernel in the stream)
+    SR_CUDA_TRY(launch_dependent(true, head_mlp_tc_kernel<BN>, grid, dim3(THREADS), C::SMEM_BYTES, st, tmW, tmX, KX,
+                                 static_cast<const __nv_bfloat16 *>(bias), static_cast<const __nv_bfloat16 *>(h), z, B, K, d,
+                                 status));
     return SPECROLL_OK;
 }
 

@@ -73,6 +73,7 @@ lm_head_topk_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                        float *__restrict__ pval, int32_t *__restrict__ pid, int32_t *__restrict__ status) {
     using namespace lmtc;
     extern __shared__ unsigned char smem_raw[];
+    pdl_launch_dependents();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // 1024-byte alignment for the 128-byte swizzle atoms
     unsigned char *aligned = smem_raw + (base - raw);
@@ -115,6 +116,7 @@ lm_head_topk_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // set up under the tail of the kernel before; its outputs are read from here on
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -272,10 +274,9 @@ int launch_lm_head_tc(const void *Zt, const void *W, int M, int V, int d, int k,
     rc = make_tmap_2d_bf16(&tmB, W, (uint64_t)V, (uint64_t)d, (uint64_t)d, BN);
     if (rc != SPECROLL_OK) return rc;
     if ((rc = device_setup(reinterpret_cast<const void *>(lm_head_topk_tc_kernel), SMEM_BYTES, nullptr)) != SPECROLL_OK) return rc;
-    lm_head_topk_tc_kernel<<<n_mblocks * n_groups, THREADS, SMEM_BYTES, st>>>(tmA, tmB, M, V, d, k, n_mblocks,
-                                                                             n_groups, tiles_per_group, pval, pid,
-                                                                             status);
-    SR_LAUNCH_CHECK();
+    // (the dependent of the correction kernel in the stream)
+    SR_CUDA_TRY(launch_dependent(true, lm_head_topk_tc_kernel, dim3(n_mblocks * n_groups), dim3(THREADS), SMEM_BYTES, st, tmA,
+                                 tmB, M, V, d, k, n_mblocks, n_groups, tiles_per_group, pval, pid, status));
     return SPECROLL_OK;
 }
 

@@ -31,6 +31,8 @@ layernorm_kernel(const __nv_bfloat16 *__restrict__ h, const __nv_bfloat16 *__res
                  int KX, float eps) {
     extern __shared__ float row[];  // d floats
     __shared__ float red[LN_THREADS / 32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int b = blockIdx.x;
     float s = 0.f;
     for (int i = threadIdx.x; i < d; i += LN_THREADS) {
@@ -100,6 +102,8 @@ __global__ void __launch_bounds__(RX_THREADS)
 reflex_kernel(const float *__restrict__ z, const float *__restrict__ m, const float *__restrict__ alpha,
               __nv_bfloat16 *__restrict__ zt, int d, float rms_eps, float clip_c) {
     __shared__ float red[RX_THREADS / 32];
+    pdl_launch_dependents();
+    pdl_wait();
     const size_t r = blockIdx.x;
     const float *zr = z + r * d;
     const float a = (alpha && m) ? alpha[r] : 0.f;
@@ -131,6 +135,7 @@ __global__ void __launch_bounds__(RX_THREADS)
 prehead_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict__ m, const float *__restrict__ alpha,
                __nv_bfloat16 *__restrict__ ht, int d, float rms_eps, float clip_c) {
     __shared__ float red[RX_THREADS / 32];
+    pdl_launch_dependents();
     const size_t r = blockIdx.x;
     const __nv_bfloat16 *hr = h + r * d;
     const float a = (alpha && m) ? alpha[r] : 0.f;
@@ -247,6 +252,8 @@ lm_head_topk_kernel(const __nv_bfloat16 *__restrict__ Zt, const __nv_bfloat16 *_
 __global__ void __launch_bounds__(128)
 topk_merge_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pid, int M, int n_cand, int k,
                   int32_t *__restrict__ cand_id, float *__restrict__ cand_logit) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x * 4 + warp;
     if (r >= M) return;
@@ -292,6 +299,8 @@ topk_merge_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pi
 __global__ void __launch_bounds__(128)
 topk_merge8_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pid, int M, int n_cand, int k,
                    int32_t *__restrict__ cand_id, float *__restrict__ cand_logit) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x * 4 + warp;
     if (r >= M) return;
@@ -392,6 +401,7 @@ tree_draw_kernel(Topo topo, int B, int K, int k, double T, const int32_t *__rest
     __shared__ int32_t sh_id[SPECROLL_MAX_HEADS][SPECROLL_MAX_TOPK];
     __shared__ float sh_u[SPECROLL_MAX_NODES];
     __shared__ int8_t sh_parent[SPECROLL_MAX_NODES];
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x;
     const int N = topo.N;
@@ -532,13 +542,12 @@ static int set_smem(Kern kern, int bytes) {
     return SPECROLL_OK;
 }
 
-static int launch_tree_draw(const Topo &topo, int B, int K, int k, float T, const int32_t *anchor,
+static int launch_tree_draw(bool pdl, const Topo &topo, int B, int K, int k, float T, const int32_t *anchor,
                             const int32_t *cand_id, const float *cand_logit, const float *u_draw,
                             int32_t *tree_tok, uint8_t *tree_cand, float *slot_q, cudaStream_t st) {
     if (B == 0) return SPECROLL_OK;
-    tree_draw_kernel<<<B, DRAW_WARPS * 32, 0, st>>>(
-        topo, B, K, k, (double)T, anchor, cand_id, cand_logit, u_draw, tree_tok, tree_cand, slot_q);
-    SR_LAUNCH_CHECK();
+    SR_CUDA_TRY(launch_dependent(pdl, tree_draw_kernel, dim3(B), dim3(DRAW_WARPS * 32), 0, st, topo, B, K, k, (double)T, anchor,
+                                 cand_id, cand_logit, u_draw, tree_tok, tree_cand, slot_q));
     return SPECROLL_OK;
 }
 
@@ -571,7 +580,7 @@ extern "C" int specroll_tree_draw(int32_t B, int32_t N, int32_t K, int32_t k, fl
     if (build_topo(parent_host, N, K, k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (!anchor_tok || !cand_id || !cand_logit || !u_draw || !tree_tok || !tree_cand || !slot_q)
         return SPECROLL_EINVAL;
-    return launch_tree_draw(topo, B, K, k, temperature, anchor_tok, cand_id, cand_logit, u_draw, tree_tok,
+    return launch_tree_draw(false, topo, B, K, k, temperature, anchor_tok, cand_id, cand_logit, u_draw, tree_tok,
                             tree_cand, slot_q, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -616,10 +625,12 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
         hb = hc;
     }
 
-    layernorm_kernel<<<B, LN_THREADS, dd * sizeof(float), st>>>(
-        hb, static_cast<const __nv_bfloat16 *>(ln_gamma), static_cast<const __nv_bfloat16 *>(ln_beta), xhat, B,
-        dd, p.KX, d->ln_eps);
-    SR_LAUNCH_CHECK();
+    // From here on every kernel is launched as the programmatic dependent of the one before it: it may set itself up
+    // (barriers, tensor memory, tensor-map prefetch) under the tail of its predecessor and waits for the predecessor's
+    // completion before it touches global memory.
+    SR_CUDA_TRY(launch_dependent(pre_head, layernorm_kernel, dim3(B), dim3(LN_THREADS), dd * sizeof(float), st, hb,
+                                 static_cast<const __nv_bfloat16 *>(ln_gamma), static_cast<const __nv_bfloat16 *>(ln_beta),
+                                 xhat, B, dd, p.KX, d->ln_eps));
 
     if (!(d->flags & SPECROLL_PROPOSE_LEGACY_MMA)) {
         int rc = launch_head_mlp_tc(xhat, p.KX, A, bias, hb, z, B, K, dd, status, st);
@@ -634,9 +645,9 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
         SR_LAUNCH_CHECK();
     }
 
-    reflex_kernel<<<B * K, RX_THREADS, 0, st>>>(z, pre_head ? nullptr : m, pre_head ? nullptr : alpha, zt, dd, d->rms_eps,
-                                               d->clip_c);
-    SR_LAUNCH_CHECK();
+    SR_CUDA_TRY(launch_dependent(true, reflex_kernel, dim3(B * K), dim3(RX_THREADS), 0, st, (const float *)z,
+                                 pre_head ? (const float *)nullptr : m, pre_head ? (const float *)nullptr : alpha, zt, dd,
+                                 d->rms_eps, d->clip_c));
 
     {
         const int grid = p.n_mblocks * p.n_groups;
@@ -662,12 +673,9 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
         SR_LAUNCH_CHECK();
     }
 
-    if (k <= 8)
-        topk_merge8_kernel<<<(p.M + 3) / 4, 128, 0, st>>>(pval, pid, p.M, p.n_groups * k, k, cand_id, cand_logit);
-    else
-        topk_merge_kernel<<<(p.M + 3) / 4, 128, 0, st>>>(pval, pid, p.M, p.n_groups * k, k, cand_id, cand_logit);
-    SR_LAUNCH_CHECK();
+    SR_CUDA_TRY(launch_dependent(true, k <= 8 ? topk_merge8_kernel : topk_merge_kernel, dim3((p.M + 3) / 4), dim3(128), 0, st,
+                                 (const float *)pval, (const int32_t *)pid, p.M, p.n_groups * k, k, cand_id, cand_logit));
 
-    return launch_tree_draw(topo, B, K, k, d->temperature, anchor_tok, cand_id, cand_logit, u_draw, tree_tok,
+    return launch_tree_draw(true, topo, B, K, k, d->temperature, anchor_tok, cand_id, cand_logit, u_draw, tree_tok,
                             tree_cand, slot_q, st);
 }
