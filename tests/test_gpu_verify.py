@@ -109,6 +109,31 @@ def test_lone_root_and_chain_and_star_topologies():
         check(w, o, g, lg)
 
 
+def test_wide_lists_wide_stars_and_underflowing_proposals():
+    # the node routine's fast form holds a candidate and a child per lane: more than 32 of either, and slot
+    # proposals whose weights underflow against a drawn candidate's logit, take the sequential form
+    cases = []
+    w = I.scaled(I.WORKLOADS["tiny"], B=24, N=16, V=2048, K=3, k=40)                       # k > 32
+    cases.append((w, I.topology(w), None))
+    star = [-1] + [0] * 39                                                                   # 39 children > 32
+    w = I.scaled(I.WORKLOADS["tiny"], B=24, N=40, V=2048, K=2, k=48, fixed_parent=tuple(star))
+    cases.append((w, np.array(star, np.int32), None))
+    w = I.scaled(I.WORKLOADS["tiny"], B=24, N=12, V=1024, K=3, k=8)                        # gaps of 2000 between candidates
+    cases.append((w, I.topology(w), 2000.0))
+    for w, parent, gap in cases:
+        cid, cl = I.synthetic_candidates(w)
+        if gap is not None:
+            cl = (-gap * np.arange(w.k, dtype=np.float32))[None, None, :].repeat(w.B, 0).repeat(w.K, 1).copy()
+        d = ref.tree_draw(parent, np.zeros(w.B, np.int32), cid, cl, I.uniforms24(13, (w.B, w.N)))
+        lg = I.target_logits(w, parent, d["tree_tok"], boost=5.0)
+        u_acc, u_fin = I.verify_uniforms(w)
+        o, g = run_both(w, parent, lg, d["tree_tok"], d["tree_cand"], cid, cl, u_acc, u_fin)
+        check(w, o, g, lg)
+        if gap is not None:
+            # a later sibling's proposal is a point mass on the best remaining candidate
+            assert (d["tree_cand"][:, 1:] < w.k).all()
+
+
 def test_bad_arguments_are_refused_without_touching_the_device():
     w = I.scaled(I.WORKLOADS["tiny"], B=2)
     parent = I.topology(w)
