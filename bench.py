@@ -371,7 +371,7 @@ def run_ours(args, w, layers):
         "tree_attn": {"ms": attn_ms, "ms_per_layer": attn_ms / wl.layers, "layers": wl.layers,
                       "tflops": wl.attn_algorithmic_flops() / attn_launch_s / 1e12},
         "verify": {"ms": ver_ms, "bound": "hbm", "achieved": ver_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                   "frac": ver_gbs / peaks["hbm_gbs"], "note": "whole call (3 launches); bytes = logits once"},
+                   "frac": ver_gbs / peaks["hbm_gbs"], "note": "whole call (%d launches); bytes = logits once" % wl.LAUNCHES_VERIFY},
     }
 
     a_f, p_f, v_f = phase_fractions(w, wl, prop_ms, attn_ms / wl.layers, ver_ms, peaks)

@@ -36,6 +36,7 @@ class StepWorkload:
                  top_p: float | None = None, lazy_stats: bool = False):
         self.w = w
         self.verify_flags = S.VERIFY_LAZY_STATS if lazy_stats else 0
+        self.lazy_stats = bool(lazy_stats)
         self.paged = bool(paged)
         self.top_p = top_p if (top_p is not None and 0.0 < top_p < 1.0) else None
         self.device = device
@@ -191,8 +192,15 @@ class StepWorkload:
             events[3].record()
 
     # ---- bookkeeping for the report
-    LAUNCHES_PROPOSE, LAUNCHES_VERIFY = 6, 3   # kernels per call (layernorm, heads, correction, projection, merge,
-    #                                            draw; row statistics, walk, terminal draw)
+    LAUNCHES_PROPOSE = 6   # kernels per call: layernorm, heads, correction, projection, merge, draw
+
+    @property
+    def LAUNCHES_VERIFY(self) -> int:
+        # plain verification with all rows' statistics: the statistics kernel, then walk + terminal draw in one;
+        # with a nucleus: statistics, walk, draw; statistics of the visited rows only: walk, draw
+        if self.lazy_stats:
+            return 2
+        return 3 if self.top_p is not None else 2
 
     def launches_per_step(self) -> int:
         # the library says how many kernels an attention call enqueues: the plan kernel runs for the first layer
