@@ -128,21 +128,25 @@ constexpr int NUC_THREADS = 512;
 // threshold key (a token is kept iff ord_key(logit) >= key), st->keep = sum of the kept exp((l - M)/T).
 //
 // The threshold is searched from coarse to exact:
-//   A  sixteen bins of the distance below the maximum, e = (M - l) c in log2 units, two units wide (the last bin
-//      takes everything beyond 30): per-thread private bins in shared memory, no atomics; the bin where the mass
-//      from the top reaches top_p * S is selected;
-//   B  the same inside the selected bin, sixteen sub-bins of 1/8 unit;
-//   C  the keys of the tokens in the selected sub-bin are collected in shared memory (a few thousand at most);
+//   A  256 bins of the distance below the maximum, e = (M - l) c in log2 units, 1/8 unit wide, 32 units in all:
+//      one pass, fixed-point masses added to counters in shared memory; the bin where the mass from the
+//      top reaches top_p * S is selected;
+//   C  the keys of the tokens in the selected bin are collected in shared memory (a few thousand at most);
 //   D  a radix search over the 16 key bits, four per pass, on that list alone finds the exact key.
-// A and B cost about a dozen instructions per token, C half of that; the bin index is the argument of the
-// exponential, which is needed anyway.  If the threshold lies in the catch-all bin or the list overflows, the
+// A costs about a dozen instructions per token, C half of that; the bin index is the argument of the
+// exponential, which is needed anyway.  If the threshold lies beyond the bins or the list overflows, the
 // radix search runs over the whole row instead (nucleus_row_radix; same result, four full passes).
+// (Two passes of sixteen private bins per thread in place of A, every token a load, an add and a store in
+// shared memory in each: 0.80 ms for the verification of the 1.5B shape against 0.28 without a nucleus.)
 constexpr int NUC_LIST = 8192;
-constexpr float NUC_WA = 2.0f, NUC_WB = 0.125f;
+constexpr int NUC_BINS = 256;
+constexpr float NUC_WB = 0.125f;
 
 struct NucleusSmem {
     float bins[16][NUC_THREADS];
     float wsum[NUC_THREADS / 32][16];
+    uint32_t c_lo, c_hi;  // bf16 bits of the ends of the interval of logits that fall into the selected bin
+    uint32_t fine_lo[NUC_BINS], fine_hi[NUC_BINS];  // 64-bit fixed-point masses of the fine bins, in two words
     unsigned short list[NUC_LIST];
     int n_list;
     int sel;  // bin selected by the last level
@@ -161,32 +165,44 @@ __device__ void nucleus_pick(NucleusSmem *st, float target, bool top_is_high_ind
         if (lane == 0) st->wsum[warp][j] = x;
     }
     __syncthreads();
-    if (tid == 0) {
+    if (warp == 0) {
+        // lane j adds bin j over the warps (in warp order); lane 0 then walks the sixteen totals
+        float x = 0.f;
+        if (lane < 16)
+            for (int w2 = 0; w2 < NUC_THREADS / 32; ++w2) x += st->wsum[w2][lane];
         float tot[16];
-        for (int j = 0; j < 16; ++j) {
-            float x = 0.f;
-            for (int w2 = 0; w2 < NUC_THREADS / 32; ++w2) x += st->wsum[w2][j];
-            tot[top_is_high_index ? 15 - j : j] = x;  // tot[0] = most probable bin
-        }
-        float cum = st->above;
-        int sel = -1, last = 0;
-        for (int j = 0; j < 16; ++j)
-            if (tot[j] > 0.f) last = j;
-        for (int j = 0; j < 16; ++j) {
-            if (cum + tot[j] >= target) {
-                sel = j;
-                break;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) tot[j] = __shfl_sync(0xffffffffu, x, top_is_high_index ? 15 - j : j);  // tot[0] = most probable bin
+        if (lane == 0) {
+            float cum = st->above;
+            int sel = -1, last = 0;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (tot[j] > 0.f) last = j;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                if (sel < 0) {
+                    if (cum + tot[j] >= target)
+                        sel = j;
+                    else
+                        cum += tot[j];
+                }
             }
-            cum += tot[j];
+            float tsel = 0.f;
+            if (sel < 0) {
+                sel = last;
+                cum = st->above;
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (j < last) cum += tot[j];
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (j == sel) tsel = tot[j];
+            st->above = cum;
+            st->keep = cum + tsel;
+            st->sel = top_is_high_index ? 15 - sel : sel;
         }
-        if (sel < 0) {
-            sel = last;
-            cum = st->above;
-            for (int j = 0; j < last; ++j) cum += tot[j];
-        }
-        st->above = cum;
-        st->keep = cum + tot[sel];
-        st->sel = top_is_high_index ? 15 - sel : sel;
     }
     __syncthreads();
 }
@@ -198,6 +214,22 @@ __device__ __forceinline__ void nucleus_key_bin(NucleusSmem *st, uint32_t bits, 
     const uint32_t key = ord_key(bits);
     if (level == 0 || (key >> (shift + 4)) == prefix)
         st->bins[(key >> shift) & 15u][threadIdx.x] += ex2_approx((__uint_as_float(bits << 16) - M) * c);
+}
+
+// Four vectors of a row, NUC_THREADS apart, for one thread.  All four in range (every round but the last): plain
+// loads one after the other, so that all four are in flight together; a load under a condition of its own ends up
+// behind the use of the one before it.  Absent vectors read as -inf.
+__device__ __forceinline__ void nucleus_load4(const uint4 *__restrict__ p, int i0, int nvec, uint4 (&vv)[4]) {
+    if (i0 + 3 * NUC_THREADS < nvec) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) vv[q] = ld_nc_v4(p + i0 + q * NUC_THREADS);
+    } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = i0 + q * NUC_THREADS;
+            vv[q] = i < nvec ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+        }
+    }
 }
 
 // Exact search over the whole row (fallback): four passes, four key bits each.
@@ -242,76 +274,160 @@ __device__ void nucleus_row(const uint16_t *__restrict__ row_logits, int V, floa
     // conversions share the special-function unit with the exponentials; this stays on the FMA and integer
     // pipes).  Any monotone rule would do: the same one is used in every pass.
     auto to_int = [](float x) { return (int)(__float_as_uint(x + 12582912.0f) - 0x4B400000u); };
-    auto bin_a = [&](float e) { return min(15, to_int(e * (1.0f / NUC_WA))); };
-    // ---- A
-#pragma unroll
-    for (int j = 0; j < 16; ++j) st->bins[j][tid] = 0.f;
-    __syncthreads();
-    for (int i0 = tid; i0 < nvec; i0 += 4 * NUC_THREADS) {
-        uint4 vv[4];  // four independent loads in flight; an absent one reads as -inf (no mass)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int i = i0 + q * NUC_THREADS;
-            vv[q] = i < nvec ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
-#pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const float e = dist((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
-                st->bins[bin_a(e)][tid] += ex2_approx(-e);
-            }
-        }
-    }
-    nucleus_pick(st, target, false);
-    const int ja = st->sel;
-    if (ja == 15) {  // the cut lies among tokens 2^-30 below the maximum: exact search over the whole row
+    // ---- A: one pass, 256 bins of 1/8 unit over the first 32 units below the maximum, masses as 32-bit fixed point
+    //      (round to nearest; the row's largest element is 2^32) added to counters in shared memory: integer
+    //      sums do not depend on the order of the atomics, so the result is the same from run to run.  Tokens
+    //      further down fall outside the bins; a cut among them goes to the exact search below.
+    auto bin_ab = [&](float e) { return to_int(e * (1.0f / NUC_WB)); };  // (>= 0; >= NUC_BINS: outside)
+    // (one copy of the counters per warp, in the storage of the private bins of the later steps: only the lanes
+    // of a warp can meet at a counter.  Rows of more than 2^20 tokens could overflow a counter: exact search.)
+    if (nvec > (1 << 17)) {
         nucleus_row_radix(p, nvec, c, M, target, st);
         return;
     }
-    // ---- B
-    const float ea = ((float)ja - 0.5f) * NUC_WA;  // lower edge of bin ja under round-to-nearest
-    auto bin_b = [&](float e) { return max(0, min(15, to_int((e - ea) * (1.0f / NUC_WB)))); };
-#pragma unroll
-    for (int j = 0; j < 16; ++j) st->bins[j][tid] = 0.f;
+    static_assert(sizeof(st->bins) >= (NUC_THREADS / 32) * 2 * NUC_BINS * sizeof(uint32_t), "per-warp fine bins fit");
+    uint32_t *wfine = reinterpret_cast<uint32_t *>(&st->bins[0][0]) + (tid >> 5) * 2 * NUC_BINS;
+    for (int j = tid; j < (NUC_THREADS / 32) * 2 * NUC_BINS; j += NUC_THREADS) reinterpret_cast<uint32_t *>(&st->bins[0][0])[j] = 0u;
+    __syncthreads();
     for (int i0 = tid; i0 < nvec; i0 += 4 * NUC_THREADS) {
-        uint4 vv[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int i = i0 + q * NUC_THREADS;
-            vv[q] = i < nvec ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-        }
+        uint4 vv[4];  // four independent loads in flight; an absent one reads as -inf (no mass)
+        nucleus_load4(p, i0, nvec, vv);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
 #pragma unroll
             for (int t = 0; t < 8; ++t) {
                 const float e = dist((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
-                if (bin_a(e) == ja) st->bins[bin_b(e)][tid] += ex2_approx(-e);
+                const int j = bin_ab(e);
+                if (j < NUC_BINS) {
+                    // the two halves of the 32-bit mass go to counters of their own: a warp's share of the row is at
+                    // most 2^16 tokens, so neither can overflow, and the additions need no result back
+                    const uint32_t v = __float2uint_rn(ex2_approx(-e) * 4294967296.0f);
+                    atomicAdd(&wfine[j], v & 0xffffu);
+                    if (v >> 16) atomicAdd(&wfine[NUC_BINS + j], v >> 16);  // (most tokens are far below the maximum)
+                }
             }
         }
     }
-    nucleus_pick(st, target, false);
-    const int jb = st->sel;
-    // ---- C
-    for (int i0 = tid; i0 < nvec; i0 += 4 * NUC_THREADS) {
-        uint4 vv[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int i = i0 + q * NUC_THREADS;
-            vv[q] = i < nvec ? ld_nc_v4(p + i) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+    __syncthreads();
+    for (int j = tid; j < NUC_BINS; j += NUC_THREADS) {
+        unsigned long long tot = 0ull;
+        for (int w2 = 0; w2 < NUC_THREADS / 32; ++w2) {
+            const uint32_t *wf = reinterpret_cast<const uint32_t *>(&st->bins[0][0]) + w2 * 2 * NUC_BINS;
+            tot += ((unsigned long long)wf[NUC_BINS + j] << 16) + wf[j];
         }
+        st->fine_lo[j] = (uint32_t)tot;
+        st->fine_hi[j] = (uint32_t)(tot >> 32);
+    }
+    __syncthreads();
+    if (tid < 32) {
+        // the bin at which the mass from the top reaches the target: every lane takes eight consecutive bins
+        const unsigned long long tgt = (unsigned long long)((double)target * 4294967296.0);
+        unsigned long long mine = 0ull;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
+        auto fine = [&](int j) { return ((unsigned long long)st->fine_hi[j] << 32) | st->fine_lo[j]; };
 #pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const uint32_t bits = (t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu);
-                const float e = dist(bits);
-                if (bin_a(e) == ja && bin_b(e) == jb) {
-                    const int pos = atomicAdd(&st->n_list, 1);
-                    if (pos < NUC_LIST) st->list[pos] = (unsigned short)bits;
+        for (int q = 0; q < NUC_BINS / 32; ++q) mine += fine(tid * (NUC_BINS / 32) + q);
+        unsigned long long incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long x = __shfl_up_sync(0xffffffffu, incl, o);
+            if (tid >= o) incl += x;
+        }
+        const unsigned hit = __ballot_sync(0xffffffffu, incl >= tgt);
+        if (hit == 0u) {
+            if (tid == 0) st->sel = -1;  // the cut lies further down than the bins reach
+        } else if (tid == __ffs(hit) - 1) {
+            unsigned long long cum = incl - mine;
+            int j = tid * (NUC_BINS / 32);
+            while (cum + fine(j) < tgt) cum += fine(j++);  // (ends inside this lane's bins)
+            st->sel = j;
+            st->above = (float)((double)cum * (1.0 / 4294967296.0));
+            st->keep = (float)((double)(cum + fine(j)) * (1.0 / 4294967296.0));
+        }
+    }
+    __syncthreads();
+    const int jb = st->sel;
+    if (jb < 0) {  // exact search over the whole row
+        nucleus_row_radix(p, nvec, c, M, target, st);
+        return;
+    }
+    // ---- C: the tokens of bin jb.  The bin index does not increase with the logit, so they are the logits of an
+    //      interval, whose two ends thread 0 finds by bisection over the 16-bit keys (between the most negative finite
+    //      value and the row's maximum) with the very rule of pass A; the pass then compares packed bf16 pairs with
+    //      the two ends and looks closer only at vectors that hold a member (a few per cent).
+    if (tid == 0) {
+        auto bits_of_key = [](uint32_t key) { return (key & 0x8000u) ? (key & 0x7fffu) : (~key & 0xffffu); };
+        auto bin_of_key = [&](uint32_t key) { return bin_ab(dist(bits_of_key(key))); };
+        const uint32_t k_min = ord_key(0xff7fu), k_max = ord_key(__float_as_uint(M) >> 16);
+        // smallest key whose bin is <= jb (the bins fall as the keys rise; bin(k_max) = 0 <= jb)
+        uint32_t lo = k_min, hi = k_max;
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (bin_of_key(mid) <= jb)
+                hi = mid;
+            else
+                lo = mid + 1;
+        }
+        const uint32_t k_lo = lo;
+        // largest key whose bin is >= jb (bin(k_lo) = jb: pass A found a token there)
+        lo = k_lo;
+        hi = k_max;
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi + 1) >> 1;
+            if (bin_of_key(mid) >= jb)
+                lo = mid;
+            else
+                hi = mid - 1;
+        }
+        st->c_lo = bits_of_key(k_lo);
+        st->c_hi = bits_of_key(lo);
+    }
+    __syncthreads();
+    {
+        auto as_bf162 = [](uint32_t w_) { return *reinterpret_cast<const __nv_bfloat162 *>(&w_); };
+        const __nv_bfloat162 lo2 = as_bf162(st->c_lo | (st->c_lo << 16)), hi2 = as_bf162(st->c_hi | (st->c_hi << 16));
+        // (the loop bound is the same for all lanes of a warp: the body votes and scans over the whole warp; an
+        // absent vector reads as -inf, which no interval of finite ends holds)
+        for (int ib = tid & ~31; ib < nvec; ib += 4 * NUC_THREADS) {
+            const int i0 = ib + (tid & 31);
+            uint4 vv[4];
+            nucleus_load4(p, i0, nvec, vv);
+            // the members among this thread's 32 logits, as one bit each; one reservation in the list per warp and
+            // round: the lanes' counts are scanned over the warp
+            uint32_t member = 0u;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const uint32_t mk = __hge2_mask(as_bf162(w[t]), lo2) & __hle2_mask(as_bf162(w[t]), hi2);
+                    member |= ((mk & 1u) | ((mk >> 15) & 2u)) << (8 * q + 2 * t);
+                }
+            }
+            if (__ballot_sync(0xffffffffu, member != 0u) == 0u) continue;
+            const int cnt = __popc(member);
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int x = __shfl_up_sync(0xffffffffu, incl, o);
+                if ((tid & 31) >= o) incl += x;
+            }
+            int base = 0;
+            if ((tid & 31) == 31) base = atomicAdd(&st->n_list, incl);
+            base = __shfl_sync(0xffffffffu, base, 31);
+            int pos = base + incl - cnt;
+            if (cnt) {  // (element 8 q + 2 t + half of this round)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t w[4] = {vv[q].x, vv[q].y, vv[q].z, vv[q].w};
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        if ((member >> (8 * q + t)) & 1u) {
+                            if (pos < NUC_LIST) st->list[pos] = (unsigned short)((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xffffu));
+                            ++pos;
+                        }
+                    }
                 }
             }
         }
