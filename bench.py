@@ -416,6 +416,15 @@ def run_ours(args, w, layers):
         names = ["tiny", "qwen1.5b", "qwen7b", "qwen14b"] + [f"sweep7b_B{b}" for b in (256, 128, 64, 32, 16, 8)]
         for nm in names:
             if nm == w.name and layers == w.layers and not (args.paged or args.top_p or args.lazy_stats):
+                # the headline's own numbers (all layers back to back; on the large shapes the board is at its power
+                # limit then), and beside them the same calls in a three-layer step like the other entries
+                short = measure_workload(I.WORKLOADS[nm], dev, 3, 5, peaks, local)
+                headline_entry["three_layer_step"] = {
+                    k_: short[k_] for k_ in ("layers_run", "attn_us_per_layer", "attn_bound", "attn_frac", "propose_ms",
+                                             "propose_bound", "propose_frac", "verify_ms", "verify_frac", "clocks")}
+                headline_entry["three_layer_step"]["note"] = (
+                    "the same calls in a step of three attention layers, as for the other entries: no sustained "
+                    "load, so not what the full step reaches")
                 workloads.append(headline_entry)
             else:
                 workloads.append(measure_workload(I.WORKLOADS[nm], dev, 3, 5, peaks, local))
