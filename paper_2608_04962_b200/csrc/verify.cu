@@ -324,7 +324,6 @@ __device__ void nucleus_row(const uint16_t *__restrict__ row_logits, int V, floa
         // the bin at which the mass from the top reaches the target: every lane takes eight consecutive bins
         const unsigned long long tgt = (unsigned long long)((double)target * 4294967296.0);
         unsigned long long mine = 0ull;
-#pragma unroll
         auto fine = [&](int j) { return ((unsigned long long)st->fine_hi[j] << 32) | st->fine_lo[j]; };
 #pragma unroll
         for (int q = 0; q < NUC_BINS / 32; ++q) mine += fine(tid * (NUC_BINS / 32) + q);
