@@ -229,6 +229,105 @@ def phase_fractions(w, wl, prop_ms, attn_layer_ms, ver_ms, peaks):
     return attn, prop, ver
 
 
+def measure_power_roof(wl, local, secs=2.0):
+    """The board's power limit as a roof for the attention kernel (rank 0, one GPU).  Board power (NVML, 50 Hz, median of
+    the second half of each loop) of: the idle context, a device-to-device copy at full speed, a bf16 GEMM loop, and
+    this workload's attention layers back to back.  With the energy per byte of the copy and per FLOP of the GEMM, a
+    kernel with the attention's mix of bytes and FLOPs can sustain at most `max_hbm_frac` of the copy rate under the
+    board's limit.  None when NVML is not there."""
+    import threading
+    import torch
+    try:
+        import pynvml as nv
+        nv.nvmlInit()
+        phys, vis = local, os.environ.get("CUDA_VISIBLE_DEVICES")
+        if vis:
+            ids = [x for x in vis.split(",") if x.strip() != ""]
+            if local < len(ids) and ids[local].strip().isdigit():
+                phys = int(ids[local])
+        h = nv.nvmlDeviceGetHandleByIndex(phys)
+        limit_w = nv.nvmlDeviceGetPowerManagementLimit(h) / 1000.0
+    except Exception:
+        return None
+    dev = torch.device("cuda", local)
+
+    def loop(body):
+        stop, out = threading.Event(), []
+
+        def run():
+            while not stop.is_set():
+                try:
+                    out.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
+                except Exception:
+                    pass
+                time.sleep(0.02)
+
+        th = threading.Thread(target=run, daemon=True)
+        torch.cuda.synchronize()
+        th.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        t0, n = time.perf_counter(), 0
+        while time.perf_counter() - t0 < secs:
+            n += body()
+            torch.cuda.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        stop.set()
+        th.join(timeout=2)
+        tail = sorted(out[len(out) // 2:]) or [float("nan")]
+        return tail[len(tail) // 2], n, e0.elapsed_time(e1) * 1e-3
+
+    def idle():
+        time.sleep(0.1)
+        return 0
+
+    try:
+        src = torch.empty(2 << 30, dtype=torch.uint8, device=dev)
+        dst = torch.empty_like(src)
+        A = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+        Bm = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+    except Exception:
+        return None
+
+    def copy():
+        for _ in range(8):
+            dst.copy_(src)
+        return 8
+
+    def gemm():
+        for _ in range(40):
+            torch.matmul(A, Bm)
+        return 40
+
+    def attn():
+        for l in range(wl.layers):
+            wl.attn(l)
+        return wl.layers
+
+    idle_w, _, _ = loop(idle)
+    copy_w, nc, tc = loop(copy)
+    gemm_w, ng, tg = loop(gemm)
+    attn_w, na, ta = loop(attn)
+    copy_gbs = nc * 2 * src.numel() / tc / 1e9
+    gemm_tf = ng * 2 * 8192 ** 3 / tg / 1e12
+    attn_gbs = na * wl.attn_algorithmic_bytes() / ta / 1e9
+    attn_tf = na * wl.attn_algorithmic_flops() / ta / 1e12
+    del src, dst, A, Bm
+    torch.cuda.empty_cache()
+    x_h, x_t = attn_gbs / copy_gbs, attn_tf / gemm_tf
+    denom = (copy_w - idle_w) + (x_t / x_h) * (gemm_w - idle_w)
+    max_h = (limit_w - idle_w) / denom if denom > 0 else float("nan")
+    return {"limit_w": limit_w, "idle_w": idle_w, "copy_w": copy_w, "copy_gbs_read_plus_write": copy_gbs,
+            "gemm_w": gemm_w, "gemm_tflops": gemm_tf, "attn_w": attn_w, "attn_gbs_sustained": attn_gbs,
+            "attn_tflops_sustained": attn_tf,
+            "model_w": idle_w + x_h * (copy_w - idle_w) + x_t * (gemm_w - idle_w),
+            "max_frac_of_copy_rate": max_h, "attn_frac_of_copy_rate": x_h, "attn_frac_of_power_roof": x_h / max_h,
+            "note": "power = idle + (copy - idle) * (bytes/s over the copy's) + (gemm - idle) * (FLOP/s over the GEMM's); "
+                    "max_frac_of_copy_rate = the largest byte rate, as a fraction of the copy's, that a kernel with the "
+                    "attention's ratio of FLOPs to bytes sustains under limit_w by that model; loops of %.0f s each" % secs}
+
+
 def measure_workload(w, dev, layers, steps, peaks, local):
     """One entry of the `workloads` array: the step of workload `w` with `layers` attention layers (enough for the
     per-layer time: every layer has its own cache, larger than L2), its per-call times and roofline fractions, and
@@ -406,6 +505,9 @@ def run_ours(args, w, layers):
     # ---- every other configuration, in the same process: three attention layers each (per-layer time; every layer
     #      has its own cache), the full-depth step put together from the per-call times
     workloads = None
+    power_roof = None
+    if world == 1 and not args.no_workloads:
+        power_roof = measure_power_roof(wl, local)
     if world == 1 and not args.no_workloads:
         from paper_2608_04962_b200 import inputs as I
         del wl
@@ -451,7 +553,7 @@ def run_ours(args, w, layers):
                        "l2": "inputs larger than L2: per-layer KV cache, logits and W each exceed 126 MB and every "
                              "layer has its own cache"},
             "clocks": clocks, "e2e": e2e, "e2e_fused": e2e_fused, "gpu_launches": launches,
-            "roofline": roofline, "cpu_baseline": cpu, "phases": phases,
+            "roofline": dict(roofline, power_roof=power_roof), "cpu_baseline": cpu, "phases": phases,
             "accepted": {"aal": aal, "acceptance_rate": ar}, "workloads": workloads}
     print(json.dumps(line), flush=True)
     D.finish()
