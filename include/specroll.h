@@ -17,6 +17,8 @@
  *     overlap on the device.
  *   - Return value: SPECROLL_OK or an error code; on error nothing has been enqueued
  *     (except SPECROLL_ECUDA, where earlier launches of the call may have been).
+ *   - An empty batch (B = 0, or R = 0 records) is valid: the descriptor and the topology are
+ *     checked, nothing is enqueued, and the per-sequence arrays, which are empty, may be NULL.
  *   - Tree topology: parent_host[N] with parent[0] = -1 and 0 <= parent[n] < n; the tree is
  *     shared by all B sequences of a call.  depth(n) <= K, every node has <= k children,
  *     N <= 64.  The children of a node, in increasing node index, are its ordered slots.

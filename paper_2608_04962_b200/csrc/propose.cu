@@ -578,6 +578,7 @@ extern "C" int specroll_tree_draw(int32_t B, int32_t N, int32_t K, int32_t k, fl
         return SPECROLL_EINVAL;
     Topo topo;
     if (build_topo(parent_host, N, K, k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (B == 0) return SPECROLL_OK;  // (an empty batch has empty arrays: their pointers may be NULL)
     if (!anchor_tok || !cand_id || !cand_logit || !u_draw || !tree_tok || !tree_cand || !slot_q)
         return SPECROLL_EINVAL;
     return launch_tree_draw(false, topo, B, K, k, temperature, anchor_tok, cand_id, cand_logit, u_draw, tree_tok,
@@ -593,11 +594,12 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
     ProposePlan p;
     const bool affine = ln_gamma || ln_beta;
     if (make_plan(d, affine, &p) != SPECROLL_OK) return SPECROLL_EINVAL;
+    Topo topo;
+    if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (d->B == 0) return SPECROLL_OK;  // (an empty batch has empty arrays: their pointers may be NULL)
     if (!h || !anchor_tok || !A || !bias || !W || !u_draw || !cand_id || !cand_logit || !tree_tok ||
         !tree_cand || !slot_q)
         return SPECROLL_EINVAL;
-    Topo topo;
-    if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (!aligned16(h) || !aligned16(A) || !aligned16(bias) || !aligned16(W) || !aligned16(m) ||
         !aligned16(ln_gamma) || !aligned16(ln_beta))
         return SPECROLL_EALIGN;

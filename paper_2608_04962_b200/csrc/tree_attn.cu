@@ -686,6 +686,11 @@ static int run_tree_attn(const specroll_attn_desc *d, const void *Q, const void 
     const bool paged = page_table_dev != nullptr;
     AttnPlan p;
     if (make_attn_plan(d, indptr_host, &p) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (d->B == 0) {  // (an empty batch has empty arrays: their pointers may be NULL)
+        Topo topo0;
+        TopoMask mask0;
+        return build_topo(parent_host, d->N, -1, -1, &topo0, &mask0) == SPECROLL_OK ? SPECROLL_OK : SPECROLL_EINVAL;
+    }
     if (!Q || !Kt || !Vt || !O) return SPECROLL_EINVAL;
     if (paged ? (!kv_len_dev || !page_indptr_dev) : !kv_indptr_dev) return SPECROLL_EINVAL;
     if (paged && !p.use_tc) return SPECROLL_ELIMIT;  // the mma.sync kernel reads a contiguous cache only

@@ -1601,14 +1601,14 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
                       float *row_sum, float *min_margin, float *nucleus_thr, float *nucleus_sum, void *workspace,
                       size_t workspace_bytes, void *cuda_stream) {
     if (check_verify_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
-    if (!logits || !tree_tok || !tree_cand || !cand_id || !cand_logit || !u_acc || !u_fin || !n_acc ||
-        !path_node || !out_tok || !term_node || !term_kind || !row_max || !row_sum)
-        return SPECROLL_EINVAL;
     const bool truncate = top_p > 0.f && top_p < 1.f;
     Topo topo;
     if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (d->B == 0) return SPECROLL_OK;  // (an empty batch has empty arrays: their pointers may be NULL)
+    if (!logits || !tree_tok || !tree_cand || !cand_id || !cand_logit || !u_acc || !u_fin || !n_acc ||
+        !path_node || !out_tok || !term_node || !term_kind || !row_max || !row_sum)
+        return SPECROLL_EINVAL;
     if (!aligned16(logits)) return SPECROLL_EALIGN;
-    if (d->B == 0) return SPECROLL_OK;
     const bool lazy = (d->flags & SPECROLL_VERIFY_LAZY_STATS) != 0;
     const size_t need = truncate ? specroll_verify_nucleus_workspace_bytes(d) : verify_ws_base(d);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)

@@ -95,3 +95,25 @@ def test_cache_offsets_must_start_at_zero(libpath):
                                     parent.ctypes.data_as(C.c_void_p), null, null, null, C.c_size_t(0), null)
     assert rc == 1                                                                # SPECROLL_EINVAL
     assert S.tree_attn_launches(2, 8, 4, 2, 64, np.array([0, 100, 300], np.int32), flags=S.ATTN_NO_PDL) >= 1
+
+
+def test_an_empty_batch_is_valid_and_needs_no_device(libpath):
+    """B = 0: descriptor and topology are checked, nothing is enqueued, the (empty) arrays may be NULL."""
+    import ctypes as C
+    from paper_2608_04962_b200 import binding as S
+    L, null = S.lib(), C.c_void_p(0)
+    parent = np.array([-1, 0, 0, 1], np.int32)
+    pp = parent.ctypes.data_as(C.c_void_p)
+    pd = S.ProposeDesc(0, 4, 2, 2, 64, 64, 1.0, 1e-5, 1e-6, 0.0, 0)
+    assert L.specroll_propose(C.byref(pd), *([null] * 9), pp, *([null] * 7), C.c_size_t(0), null) == 0
+    assert L.specroll_tree_draw(C.c_int32(0), C.c_int32(4), C.c_int32(2), C.c_int32(2), C.c_float(1.0), pp,
+                                *([null] * 8)) == 0
+    vd = S.VerifyDesc(0, 4, 2, 2, 64, 1.0, 0)
+    assert L.specroll_verify(C.byref(vd), null, pp, *([null] * 15), C.c_size_t(0), null) == 0
+    ad = S.AttnDesc(0, 4, 4, 2, 64, 0.125, 0)
+    ip = np.zeros(1, np.int32)
+    assert L.specroll_tree_attn(C.byref(ad), null, null, null, null, ip.ctypes.data_as(C.c_void_p), null, null, pp, null,
+                                null, null, C.c_size_t(0), null) == 0
+    # a malformed tree is still refused
+    bad = np.array([-1, 2, 0, 1], np.int32)
+    assert L.specroll_verify(C.byref(vd), null, bad.ctypes.data_as(C.c_void_p), *([null] * 15), C.c_size_t(0), null) == 1

@@ -59,3 +59,25 @@ def test_star_of_sixty_three_children():
     u_acc, u_fin = I.verify_uniforms(w)
     o, gv = run_both(w, parent, lg, d["tree_tok"], d["tree_cand"], cid, cl, u_acc, u_fin)
     check_verify(w, o, gv, lg)
+
+
+def test_empty_batch_is_accepted_and_launches_nothing_wrong():
+    # B = 0 (a scheduler round with no live sequence): every entry point returns without touching its outputs
+    d, V, K, k, N = 128, 1024, 3, 4, 8
+    z = lambda shape, dt: torch.zeros(shape, dtype=dt, device="cuda")
+    parent = I.best_first_topology(N, K, k)
+    p = S.propose(z((0, d), torch.bfloat16), z((0,), torch.int32), z((K, d, d), torch.bfloat16), z((K, d), torch.bfloat16),
+                  z((V, d), torch.bfloat16), None, None, parent, z((0, N), torch.float32), k=k)
+    assert p["cand_id"].shape == (0, K, k) and p["tree_tok"].shape == (0, N)
+    t = S.tree_draw(parent, z((0,), torch.int32), z((0, K, k), torch.int32), z((0, K, k), torch.float32),
+                    z((0, N), torch.float32))
+    assert t["tree_tok"].shape == (0, N)
+    Hq, Hkv, D = 4, 2, 64
+    ip = np.zeros(1, np.int32)
+    O = S.tree_attn(z((0, N, Hq, D), torch.bfloat16), z((0, Hkv, D), torch.bfloat16), z((0, Hkv, D), torch.bfloat16),
+                    dev(ip), ip, z((0, N, Hkv, D), torch.bfloat16), z((0, N, Hkv, D), torch.bfloat16), parent)
+    assert O.shape[0] == 0
+    v = S.verify(z((0, N, V), torch.bfloat16), parent, z((0, N), torch.int32), z((0, N), torch.uint8),
+                 z((0, K, k), torch.int32), z((0, K, k), torch.float32), z((0, N), torch.float32), z((0,), torch.float32))
+    torch.cuda.synchronize()
+    assert v["n_acc"].shape == (0,) and v["out_tok"].shape == (0, K + 1)
