@@ -686,10 +686,10 @@ extern "C" int specroll_reflex_feedback_ex(const specroll_feedback_desc *d, cons
                                            float *d_cov, float *tv, float *severity, float *e_out, void *workspace,
                                            size_t workspace_bytes, void *cuda_stream) {
     if (check_feedback_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (d->R == 0) return SPECROLL_OK;  // (no records: the per-record arrays are empty and may be NULL)
     if (!logits || !rec_row || !row_max || !row_sum || !cand_id || !cand_logit || !y_star || !W || !rho || !rec_mem || !m)
         return SPECROLL_EINVAL;
     if (!aligned16(logits) || !aligned16(W)) return SPECROLL_EALIGN;
-    if (d->R == 0) return SPECROLL_OK;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
         workspace_bytes < specroll_reflex_feedback_workspace_bytes(d))
         return SPECROLL_EWORKSPACE;

@@ -75,12 +75,12 @@ static int commit_layers(int32_t B, int32_t N, int32_t K, int32_t Hkv, int32_t D
     if (B < 0 || N < 1 || N > SPECROLL_MAX_NODES || K < 1 || K > SPECROLL_MAX_HEADS || Hkv < 1 || (D != 64 && D != 128) ||
         n_pages < 0 || n_pages > (1LL << 24) || n_layers < 1)
         return SPECROLL_EINVAL;
+    if (B == 0) return SPECROLL_OK;  // (an empty batch has empty arrays: their pointers may be NULL)
     if (!Kt || !Vt || !path_node || !n_acc || !Kp || !Vp || !page_table || !page_indptr || !kv_len) return SPECROLL_EINVAL;
     for (int l = 0; l < n_layers; ++l) {
         if (!Kt[l] || !Vt[l] || !Kp[l] || !Vp[l]) return SPECROLL_EINVAL;
         if (!aligned16(Kt[l]) || !aligned16(Vt[l]) || !aligned16(Kp[l]) || !aligned16(Vp[l])) return SPECROLL_EALIGN;
     }
-    if (B == 0) return SPECROLL_OK;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int row_vec = Hkv * D / 8;  // 16-byte vectors per token row
     for (int l0 = 0; l0 < n_layers; l0 += COMMIT_MAX_LAYERS) {
@@ -126,9 +126,9 @@ extern "C" int specroll_commit_path_layers(int32_t B, int32_t N, int32_t K, int3
 extern "C" int specroll_gather_hidden(int32_t B, int32_t N, int32_t d, const void *hidden, const int32_t *term_node,
                                       void *h_next, void *cuda_stream) {
     if (B < 0 || N < 1 || N > SPECROLL_MAX_NODES || d < 8 || (d % 8)) return SPECROLL_EINVAL;
+    if (B == 0) return SPECROLL_OK;  // (an empty batch has empty arrays: their pointers may be NULL)
     if (!hidden || !term_node || !h_next) return SPECROLL_EINVAL;
     if (!aligned16(hidden) || !aligned16(h_next)) return SPECROLL_EALIGN;
-    if (B == 0) return SPECROLL_OK;
     gather_hidden_kernel<<<(unsigned)B, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         static_cast<const uint4 *>(hidden), term_node, N, d / 8, static_cast<uint4 *>(h_next));
     SR_LAUNCH_CHECK();

@@ -1770,12 +1770,12 @@ extern "C" int specroll_verify_walk_sparse(const specroll_verify_desc *d, const 
                                            int32_t *term_kind, float *min_margin, void *workspace,
                                            size_t workspace_bytes, void *cuda_stream) {
     if (check_verify_desc(d) != SPECROLL_OK || d->flags != 0) return SPECROLL_EINVAL;
+    Topo topo;
+    if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
+    if (d->B == 0) return SPECROLL_OK;  // (an empty batch has empty arrays: their pointers may be NULL)
     if (!cand_target || !row_max || !row_sum || !tree_tok || !tree_cand || !cand_id || !cand_logit || !u_acc || !n_acc ||
         !path_node || !out_tok || !term_node || !term_kind)
         return SPECROLL_EINVAL;
-    Topo topo;
-    if (build_topo(parent_host, d->N, d->K, d->k, &topo, nullptr) != SPECROLL_OK) return SPECROLL_EINVAL;
-    if (d->B == 0) return SPECROLL_OK;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < verify_ws_base(d))
         return SPECROLL_EWORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -1812,9 +1812,9 @@ extern "C" int specroll_verify_terminal_rows(const specroll_verify_desc *d, cons
                                              const float *u_fin, int32_t *out_tok, void *workspace,
                                              size_t workspace_bytes, void *cuda_stream) {
     if (check_verify_desc(d) != SPECROLL_OK || d->flags != 0) return SPECROLL_EINVAL;
+    if (d->B == 0) return SPECROLL_OK;  // (an empty batch has empty arrays: their pointers may be NULL)
     if (!term_logits || !row_max || !n_acc || !term_node || !u_fin || !out_tok) return SPECROLL_EINVAL;
     if (!aligned16(term_logits)) return SPECROLL_EALIGN;
-    if (d->B == 0) return SPECROLL_OK;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < verify_ws_base(d))
         return SPECROLL_EWORKSPACE;
     TermArgs ta;
