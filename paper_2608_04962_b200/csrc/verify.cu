@@ -32,7 +32,8 @@ constexpr float NEG_INF = -INFINITY;
 
 // ------------------------------------------------------------------------------ row statistics
 
-__device__ __forceinline__ void online_update(const uint4 &v, float c, float &m, float &s) {
+// nmc = -m c rides along with the running maximum m, so that an exponent is one fused multiply-add.
+__device__ __forceinline__ void online_update(const uint4 &v, float c, float &m, float &nmc, float &s) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     float x[8];
 #pragma unroll
@@ -46,10 +47,11 @@ __device__ __forceinline__ void online_update(const uint4 &v, float c, float &m,
     if (vm > m) {
         s *= ex2_approx((m - vm) * c);  // m = -inf gives 0
         m = vm;
+        nmc = -vm * c;
     }
     float acc = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc += ex2_approx((x[i] - m) * c);
+    for (int i = 0; i < 8; ++i) acc += ex2_approx(fmaf(x[i], c, nmc));
     s += acc;
 }
 
@@ -66,7 +68,7 @@ row_stats_kernel(const uint16_t *__restrict__ logits, int V, float c, float *__r
     const size_t row = blockIdx.x;
     const uint4 *p = reinterpret_cast<const uint4 *>(logits + row * (size_t)V);
     const int nvec = V >> 3;
-    float m = NEG_INF, s = 0.f;
+    float m = NEG_INF, nmc = 0.f, s = 0.f;
     {
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
         const int G = (nvec + 127) / 128, gpw = (G + RS_WARPS - 1) / RS_WARPS;
@@ -79,10 +81,10 @@ row_stats_kernel(const uint16_t *__restrict__ logits, int V, float c, float *__r
 #pragma unroll
                 for (int q = 0; q < 4; ++q) v[q] = ld_nc_v4(p + i0 + q * 32);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) online_update(v[q], c, m, s);
+                for (int q = 0; q < 4; ++q) online_update(v[q], c, m, nmc, s);
             } else {
                 for (int q = 0; q < 4; ++q)
-                    if (i0 + q * 32 < nvec) online_update(ld_nc_v4(p + i0 + q * 32), c, m, s);
+                    if (i0 + q * 32 < nvec) online_update(ld_nc_v4(p + i0 + q * 32), c, m, nmc, s);
             }
         }
     }
@@ -892,16 +894,16 @@ __device__ void row_stats_row(const uint16_t *__restrict__ row_logits, int V, fl
                               float *M_out, float *S_out) {
     const uint4 *p = reinterpret_cast<const uint4 *>(row_logits);
     const int nvec = V >> 3;
-    float m = NEG_INF, s = 0.f;
+    float m = NEG_INF, nmc = 0.f, s = 0.f;
     int i = threadIdx.x;
     for (; i + 3 * NUC_THREADS < nvec; i += 4 * NUC_THREADS) {
         uint4 v[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) v[u] = ld_nc_v4(p + i + u * NUC_THREADS);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) online_update(v[u], c, m, s);
+        for (int u = 0; u < 4; ++u) online_update(v[u], c, m, nmc, s);
     }
-    for (; i < nvec; i += NUC_THREADS) online_update(ld_nc_v4(p + i), c, m, s);
+    for (; i < nvec; i += NUC_THREADS) online_update(ld_nc_v4(p + i), c, m, nmc, s);
     const float mw = warp_max(m);
     s = (m == NEG_INF) ? 0.f : s * ex2_approx((m - mw) * c);
     s = warp_sum(s);
