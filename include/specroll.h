@@ -400,7 +400,10 @@ int specroll_target_head_rows(int32_t R, int32_t d, int32_t V, const void *H, co
  * (max logit and sum exp((l - max)/T) of every node); min_margin[B] fp32 or NULL (smallest
  * |u - ratio| over the tested slots; +inf if none).
  * Limits: V % 8 == 0, k <= 64, K <= 8, N <= 64.
- * Workspace: scratch of the call, specroll_verify_workspace_bytes(desc) bytes, 256-byte aligned.
+ * Workspace: scratch of the call, specroll_verify_workspace_bytes(desc) bytes, 256-byte aligned: the residual the
+ * walk hands to the terminal draw (12 bytes per candidate slot of a sequence) and, without
+ * SPECROLL_VERIFY_LAZY_STATS, 64 bytes per logits row in which the statistics pass leaves the maximum and the sum
+ * of each eighth of the row, so that the terminal draw reads only the eighth that holds the drawn token.
  */
 typedef struct {
     int32_t B, N, K, k, V;
@@ -481,7 +484,9 @@ int specroll_verify_nucleus(const specroll_verify_desc *desc, float top_p, const
  * fails for lack of memory or stalls every stream while the driver serialises the device), and a
  * plain-C client that only receives device pointers from another component and owns no allocator.
  *
- * Same arguments, outputs and results as specroll_verify, minus `workspace`: the scratch is a
+ * Same arguments, outputs and results as specroll_verify, minus `workspace` (where the per-row table of
+ * specroll_verify's workspace does not fit the fixed array beside the residual, the terminal draw reads its whole
+ * row instead): the scratch is a
  * fixed array inside the library image (about 0.2 MB, present once on every GPU that loads the
  * library, until the process exits).  The call performs no cudaMalloc/cudaFree and calls no
  * allocating routine.

@@ -59,9 +59,25 @@ __device__ __forceinline__ void online_update(const uint4 &v, float c, float &m,
 // The row is cut into groups of 128 8-token vectors; a warp takes one contiguous run of groups and reads a group
 // with four loads of 32 consecutive vectors (2 KB in one piece per warp).  32 registers, so that eight CTAs fit an SM.
 constexpr int RS_WARPS = RS_THREADS / 32;
+
+// The run of 8-token vectors that warp w of the statistics kernel takes of a row of nvec vectors, [v_lo, v_hi).
+__host__ __device__ inline void rs_run(int nvec, int w, int *v_lo, int *v_hi) {
+    const int G = (nvec + 127) / 128, gpw = (G + RS_WARPS - 1) / RS_WARPS;
+    const int g_lo = w * gpw < G ? w * gpw : G, g_hi = g_lo + gpw < G ? g_lo + gpw : G;
+    *v_lo = g_lo * 128 < nvec ? g_lo * 128 : nvec;
+    *v_hi = g_hi * 128 < nvec ? g_hi * 128 : nvec;
+}
+__host__ __device__ inline int rs_run_of_vec(int nvec, int vi) {
+    const int G = (nvec + 127) / 128, gpw = (G + RS_WARPS - 1) / RS_WARPS;
+    return (vi / 128) / gpw;
+}
+
+// run_tab (nullable): [rows][RS_WARPS] (m, s) of every warp's run, s = sum over the run of exp((l - m)/T): what the
+// warps hand to the final reduction anyway.  The terminal draw of a row then finds the eighth of the row that holds
+// its target from these and reads only that.
 __global__ void __launch_bounds__(RS_THREADS, 8)
 row_stats_kernel(const uint16_t *__restrict__ logits, int V, float c, float *__restrict__ row_max,
-                 float *__restrict__ row_sum) {
+                 float *__restrict__ row_sum, float2 *__restrict__ run_tab) {
     // a kernel launched behind this one as its programmatic dependent may start its own prologue as SMs free up; it
     // waits for this grid's completion before it reads the statistics
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -98,6 +114,7 @@ row_stats_kernel(const uint16_t *__restrict__ logits, int V, float c, float *__r
     if (lane == 0) {
         sm_m[warp] = mw;
         sm_s[warp] = s;
+        if (run_tab) run_tab[row * RS_WARPS + warp] = make_float2(mw, s);
     }
     __syncthreads();
     if (warp == 0) {
@@ -1330,7 +1347,7 @@ __host__ __device__ inline WtLayout wt_layout(int N, int K, int k, int V, int S)
 }
 
 __global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, Topo topo, const float *__restrict__ u_fin, float c,
-                                                               int S) {
+                                                               int S, const float2 *__restrict__ run_tab) {
     __shared__ WalkSmem sh[WT_WARPS];
     extern __shared__ __align__(16) unsigned char sh_dyn[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1473,11 +1490,46 @@ __global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, To
     const float M = rmax[u];
     const uint16_t *lg = a.logits + ((size_t)b * N + u) * a.V;
     const uint4 *p = reinterpret_cast<const uint4 *>(lg);
-    const int nvec = a.V >> 3, vpw = L.vpw, n_sl = L.n_sl, G = L.G;
+    const int nvec = a.V >> 3, G = L.G;
+    // With the statistics kernel's table of the row's eight runs (run_tab; then S = 1): the run that holds the target
+    // is found from the table and only that eighth of the row is read, cut into G segments like a whole row
+    // otherwise.  v_base, nvec_r: the vectors the draw works on; base0: the mass before them.
+    __shared__ int sh_run;
+    __shared__ double sh_b0t[2];
+    int v_base = 0, nvec_r = nvec;
+    if (run_tab) {
+        if (warp == 0) {
+            const float2 e = lane < RS_WARPS ? run_tab[((size_t)b * N + u) * RS_WARPS + lane] : make_float2(-INFINITY, 0.f);
+            double v = (lane < RS_WARPS && e.x != -INFINITY) ? (double)e.y * (double)ex2_approx((e.x - M) * c) : 0.0;
+            for (int j = 0; j < nov; ++j)
+                if (rs_run_of_vec(nvec, ovid[j] >> 3) == lane) v += ovm_u[j] - (double)mass1(pre[u * k + j], M, c, 0u);
+            v = fmax(v, 0.0);  // (a run whose mass was all in overridden tokens, after rounding)
+            const double incl = warp_incl_scan(v, lane);
+            const double total = __shfl_sync(0xffffffffu, incl, 31);
+            const double target = (double)u_fin[b] * total;
+            const unsigned hit = __ballot_sync(0xffffffffu, lane < RS_WARPS && incl > target);
+            const unsigned pos = __ballot_sync(0xffffffffu, v > 0.0);
+            // (rounding kept the target at or above the total: the last run with mass; the draw inside it then ends
+            // at its last token with mass)
+            const int r = hit ? __ffs(hit) - 1 : (pos ? 31 - __clz(pos) : 0);
+            const double b0 = __shfl_sync(0xffffffffu, incl - v, r);
+            if (lane == 0) {
+                sh_run = r;
+                sh_b0t[0] = b0;
+                sh_b0t[1] = target;
+            }
+        }
+        __syncthreads();
+        int v_end;
+        rs_run(nvec, sh_run, &v_base, &v_end);
+        nvec_r = v_end - v_base;
+    }
+    const int vpw = (nvec_r + G - 1) / G > 0 ? (nvec_r + G - 1) / G : 1;  // vectors per warp segment
+    const int n_sl = (vpw + 31) / 32;                                     // slices per segment (<= the layout's)
     {
         {
             const int g = rank * WT_WARPS + warp;
-            const int v_lo = min(nvec, g * vpw), v_hi = min(nvec, v_lo + vpw);
+            const int v_lo = v_base + min(nvec_r, g * vpw), v_hi = v_base + min(nvec_r, g * vpw + vpw);
             term_slice_masses(p, v_lo, v_hi, n_sl, M, c, 0u, lane, slices + (size_t)g * n_sl);
         }
         if (S > 1) {
@@ -1495,7 +1547,8 @@ __global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, To
         __syncthreads();
         if (tid == 0) {
             for (int j = 0; j < nov; ++j) {
-                const int t = ovid[j], vi = t >> 3;
+                const int t = ovid[j], vi = (t >> 3) - v_base;
+                if (vi < 0 || vi >= nvec_r) continue;  // (outside the run the draw works on)
                 const int w = min(G - 1, vi / vpw), sl = (vi - w * vpw) >> 5;
                 slices[w * n_sl + sl] += ovm_u[j] - (double)mass1(pre[u * k + j], M, c, 0u);  // (staged: lg[t])
             }
@@ -1510,11 +1563,17 @@ __global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, To
         __syncthreads();
     }
     if (warp != 0) return;
-    double total = 0.0;
-    for (int g0 = 0; g0 < G; g0 += 32) total += warp_sum(g0 + lane < G ? seg[g0 + lane] : 0.0);
-    const double target = (double)u_fin[b] * total;
+    double target, base;
+    if (run_tab) {
+        base = sh_b0t[0];
+        target = sh_b0t[1];
+    } else {
+        double total = 0.0;
+        for (int g0 = 0; g0 < G; g0 += 32) total += warp_sum(g0 + lane < G ? seg[g0 + lane] : 0.0);
+        target = (double)u_fin[b] * total;
+        base = 0.0;
+    }
     int wsel = -1;
-    double base = 0.0;
     for (int g0 = 0; g0 < G && wsel < 0; g0 += 32) {
         const double v = g0 + lane < G ? seg[g0 + lane] : 0.0;
         const double incl = warp_incl_scan(v, lane);
@@ -1529,9 +1588,10 @@ __global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, To
     }
     int32_t *dst = a.out_tok + (size_t)b * (K + 1) + nacc;
     if (wsel < 0) {
-        // u_fin * total reached the total through rounding: take the last token with positive mass
+        // the target reached the end of the masses through rounding: take the last token with positive mass (from the
+        // end of the vectors the draw worked on, downwards)
         if (lane == 0) {
-            int tok = a.V - 1;
+            int tok = (v_base + nvec_r) * 8 - 1;
             for (; tok > 0; --tok) {
                 double ms = (double)mass1(lg[tok], M, c, 0u);
                 for (int j = 0; j < nov; ++j)
@@ -1542,7 +1602,7 @@ __global__ void __launch_bounds__(WT_THREADS, 2) walk_term_kernel(WalkArgs a, To
         }
         return;
     }
-    const int v_lo = min(nvec, wsel * vpw), v_hi = min(nvec, v_lo + vpw);
+    const int v_lo = v_base + min(nvec_r, wsel * vpw), v_hi = v_base + min(nvec_r, wsel * vpw + vpw);
     term_pick(p, slices + (size_t)wsel * n_sl, n_sl, v_lo, v_hi, base, target, M, c, 0u, nov, ovid, ovm_u, dst, lane);
 }
 
@@ -1584,9 +1644,14 @@ static size_t verify_ws_base(const specroll_verify_desc *d) {
            align_up(B * sizeof(int32_t), 256) + 256;
 }
 
+// The statistics kernel's table of every row's eight runs (plain verification with all rows' statistics).
+static size_t verify_ws_runs(const specroll_verify_desc *d) {
+    return align_up((size_t)d->B * d->N * RS_WARPS * sizeof(float2), 256);
+}
+
 extern "C" size_t specroll_verify_workspace_bytes(const specroll_verify_desc *d) {
     if (check_verify_desc(d) != SPECROLL_OK) return 0;
-    return verify_ws_base(d);
+    return verify_ws_base(d) + ((d->flags & SPECROLL_VERIFY_LAZY_STATS) ? 0 : verify_ws_runs(d));
 }
 
 extern "C" size_t specroll_verify_nucleus_workspace_bytes(const specroll_verify_desc *d) {
@@ -1601,7 +1666,7 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
                       const float *cand_logit, const float *u_acc, const float *u_fin, int32_t *n_acc,
                       int32_t *path_node, int32_t *out_tok, int32_t *term_node, int32_t *term_kind, float *row_max,
                       float *row_sum, float *min_margin, float *nucleus_thr, float *nucleus_sum, void *workspace,
-                      size_t workspace_bytes, void *cuda_stream) {
+                      size_t workspace_bytes, void *cuda_stream, bool runs_optional = false) {
     if (check_verify_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
     const bool truncate = top_p > 0.f && top_p < 1.f;
     Topo topo;
@@ -1612,7 +1677,13 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
         return SPECROLL_EINVAL;
     if (!aligned16(logits)) return SPECROLL_EALIGN;
     const bool lazy = (d->flags & SPECROLL_VERIFY_LAZY_STATS) != 0;
-    const size_t need = truncate ? specroll_verify_nucleus_workspace_bytes(d) : verify_ws_base(d);
+    // the table of the rows' runs serves the plain verification with all rows' statistics; a caller with a fixed
+    // scratch, or with the nucleus form's workspace, goes without it when it does not fit (the terminal draw then
+    // reads the whole row, spread over a cluster for small batches)
+    bool use_runs = !truncate && !lazy;
+    if (use_runs && runs_optional && workspace_bytes < verify_ws_base(d) + verify_ws_runs(d)) use_runs = false;
+    const size_t need = truncate ? specroll_verify_nucleus_workspace_bytes(d)
+                                 : verify_ws_base(d) + (use_runs ? verify_ws_runs(d) : 0);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need)
         return SPECROLL_EWORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -1630,9 +1701,10 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
 
     const float c = (float)(1.4426950408889634 / (double)d->temperature);
     const int rows = d->B * d->N;
+    float2 *run_tab = use_runs ? reinterpret_cast<float2 *>(ws) : nullptr;  // (behind the hand-over area; no nucleus arrays in this form)
     if (!lazy) {
         row_stats_kernel<<<rows, RS_THREADS, 0, st>>>(static_cast<const uint16_t *>(logits), d->V, c, row_max,
-                                                      row_sum);
+                                                      row_sum, run_tab);
         SR_LAUNCH_CHECK();
     }
 
@@ -1678,7 +1750,7 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
     } else {
         // plain verification: the walk and the terminal draw in one launch, overlapping the statistics kernel's tail
         constexpr int WT_SMEM_LIMIT = 160 * 1024;
-        const int S = walk_term_split(d->B);
+        const int S = use_runs ? 1 : walk_term_split(d->B);
         const WtLayout L = wt_layout(d->N, d->K, d->k, d->V, S);
         if (L.total > (size_t)WT_SMEM_LIMIT) return SPECROLL_ELIMIT;
         const int rc_ = device_setup(reinterpret_cast<const void *>(walk_term_kernel), WT_SMEM_LIMIT, nullptr);
@@ -1702,7 +1774,7 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
         }
         cfg.attrs = attrs;
         cfg.numAttrs = na;
-        SR_CUDA_TRY(cudaLaunchKernelEx(&cfg, walk_term_kernel, wa, topo, u_fin, c, S));
+        SR_CUDA_TRY(cudaLaunchKernelEx(&cfg, walk_term_kernel, wa, topo, u_fin, c, S, (const float2 *)run_tab));
         return SPECROLL_OK;
     }
     SR_LAUNCH_CHECK();
@@ -1868,7 +1940,7 @@ extern "C" int specroll_verify_nucleus(const specroll_verify_desc *d, float top_
     if (!(top_p > 0.f)) return SPECROLL_EINVAL;
     return run_verify(d, top_p, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
                       path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, nucleus_thr,
-                      nucleus_sum, workspace, workspace_bytes, cuda_stream);
+                      nucleus_sum, workspace, workspace_bytes, cuda_stream, /*runs_optional=*/true);
 }
 
 // ------------------------------------------------------------------------------ allocation-free variant
@@ -1897,7 +1969,7 @@ extern "C" int specroll_verify_static(const specroll_verify_desc *d, const void 
                                       float *row_sum, float *min_margin, void *cuda_stream) {
     if (check_verify_desc(d) != SPECROLL_OK) return SPECROLL_EINVAL;
     if (d->B > SPECROLL_STATIC_MAX_B || (long long)d->B * d->k > SPECROLL_STATIC_MAX_BK) return SPECROLL_ELIMIT;
-    if (specroll_verify_workspace_bytes(d) > STATIC_SCRATCH_BYTES) return SPECROLL_ELIMIT;
+    if (verify_ws_base(d) > STATIC_SCRATCH_BYTES) return SPECROLL_ELIMIT;
     int dev = -1;
     SR_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= MAX_DEVICES) return SPECROLL_ELIMIT;
@@ -1913,7 +1985,9 @@ extern "C" int specroll_verify_static(const specroll_verify_desc *d, const void 
         }
         scratch = g_scratch_addr[dev];
     }
-    return specroll_verify(d, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
-                           path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, scratch,
-                           STATIC_SCRATCH_BYTES, cuda_stream);
+    // (the table of the rows' runs is used when it fits the scratch beside the hand-over area, else the terminal draw
+    // reads the whole row)
+    return run_verify(d, 1.0f, logits, parent_host, tree_tok, tree_cand, cand_id, cand_logit, u_acc, u_fin, n_acc,
+                      path_node, out_tok, term_node, term_kind, row_max, row_sum, min_margin, nullptr, nullptr, scratch,
+                      STATIC_SCRATCH_BYTES, cuda_stream, /*runs_optional=*/true);
 }
