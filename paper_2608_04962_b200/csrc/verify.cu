@@ -951,7 +951,7 @@ template <bool LAZY, bool NUC>
 __global__ void __launch_bounds__(NUC_THREADS)
 walk_cta_kernel(WalkArgs a, Topo topo, float c, float top_p, float *__restrict__ row_max_w,
                 float *__restrict__ row_sum_w, uint32_t *__restrict__ thr_key, float *__restrict__ keep_sum,
-                float *__restrict__ out_thr, float *__restrict__ out_sum) {
+                float *__restrict__ out_thr, float *__restrict__ out_sum, int thr_ready) {
     extern __shared__ __align__(16) unsigned char nuc_raw[];  // NucleusSmem (NUC only): above the static limit
     NucleusSmem &nuc = *reinterpret_cast<NucleusSmem *>(nuc_raw);
     __shared__ WalkSmem sm;
@@ -977,10 +977,15 @@ walk_cta_kernel(WalkArgs a, Topo topo, float c, float top_p, float *__restrict__
         uint32_t thr = 0u;
         float norm = S;
         if constexpr (NUC) {
-            nucleus_row(a.logits + row * a.V, a.V, c, M, top_p * S, &nuc);
-            thr = nuc.prefix;
-            norm = nuc.keep;
-            if (threadIdx.x == 0) {
+            if (thr_ready && topo.n_child[u] > 0) {  // (left by nucleus_rows_kernel for every node with children)
+                thr = thr_key[row];
+                norm = keep_sum[row];
+            } else {
+                nucleus_row(a.logits + row * a.V, a.V, c, M, top_p * S, &nuc);
+                thr = nuc.prefix;
+                norm = nuc.keep;
+            }
+            if (threadIdx.x == 0 && !(thr_ready && topo.n_child[u] > 0)) {
                 thr_key[row] = thr;
                 keep_sum[row] = norm;
                 if (out_sum) out_sum[row] = norm;
@@ -1010,6 +1015,41 @@ walk_cta_kernel(WalkArgs a, Topo topo, float c, float top_p, float *__restrict__
         __syncthreads();
         if (next < 0) break;
         u = next;
+    }
+}
+
+// The nucleus thresholds of every node with children, one CTA per (sequence, such node), all at once: which of
+// them the walk visits is not known yet, but a row's threshold depends on the row alone, and one pass of all
+// of them over the machine costs less than the visited ones one after the other inside a sequence's walk.  (A
+// sequence that ends at a leaf still needs that leaf's threshold for its last token: the walk kernel finds it.)
+#ifndef NUC_AHEAD_ROWS_PER_SM
+#define NUC_AHEAD_ROWS_PER_SM 5
+#endif
+struct NodeList {
+    int32_t n;
+    int8_t node[SPECROLL_MAX_NODES];
+};
+
+__global__ void __launch_bounds__(NUC_THREADS)
+nucleus_rows_kernel(const uint16_t *__restrict__ logits, int V, int N, NodeList nodes, float c, float top_p,
+                    const float *__restrict__ row_max, const float *__restrict__ row_sum,
+                    uint32_t *__restrict__ thr_key, float *__restrict__ keep_sum, float *__restrict__ out_thr,
+                    float *__restrict__ out_sum) {
+    extern __shared__ __align__(16) unsigned char nuc_raw[];
+    NucleusSmem &nuc = *reinterpret_cast<NucleusSmem *>(nuc_raw);
+    const int b = blockIdx.x / nodes.n, u = nodes.node[blockIdx.x - b * nodes.n];
+    const size_t row = (size_t)b * N + u;
+    const float M = row_max[row], S = row_sum[row];
+    nucleus_row(logits + row * V, V, c, M, top_p * S, &nuc);
+    if (threadIdx.x == 0) {
+        const uint32_t thr = nuc.prefix;
+        thr_key[row] = thr;
+        keep_sum[row] = nuc.keep;
+        if (out_sum) out_sum[row] = nuc.keep;
+        if (out_thr) {  // the threshold as a logit: undo the key
+            const uint32_t bits = (thr & 0x8000u) ? (thr & 0x7fffu) : (~thr & 0xffffu);
+            out_thr[row] = __uint_as_float(bits << 16);
+        }
     }
 }
 
@@ -1738,15 +1778,33 @@ static int run_verify(const specroll_verify_desc *d, float top_p, const void *lo
         if (rc_ == SPECROLL_OK)
             rc_ = device_setup(reinterpret_cast<const void *>(walk_cta_kernel<true, true>), (int)sizeof(NucleusSmem), nullptr);
         if (rc_ != SPECROLL_OK) return rc_;
-        if (lazy)
+        if (lazy) {
             walk_cta_kernel<true, true><<<d->B, NUC_THREADS, sizeof(NucleusSmem), st>>>(
-                wa, topo, c, top_p, row_max, row_sum, thr_key, keep_sum, nucleus_thr, nucleus_sum);
-        else
+                wa, topo, c, top_p, row_max, row_sum, thr_key, keep_sum, nucleus_thr, nucleus_sum, 0);
+        } else {
+            NodeList nodes;
+            nodes.n = 0;
+            for (int u = 0; u < d->N; ++u)
+                if (topo.n_child[u] > 0) nodes.node[nodes.n++] = (int8_t)u;
+            // Worth it while those rows are few enough to be searched side by side (small batches, whose walks
+            // would otherwise search three or four rows one after the other on a nearly empty machine); with
+            // more rows than that, searching only the visited ones inside the walk is less work and faster.
+            int n_sm = 0;
+            rc_ = device_setup(reinterpret_cast<const void *>(nucleus_rows_kernel), (int)sizeof(NucleusSmem), &n_sm);
+            if (rc_ != SPECROLL_OK) return rc_;
+            const bool ahead = nodes.n > 0 && d->B * nodes.n <= NUC_AHEAD_ROWS_PER_SM * n_sm;
+            if (ahead) {
+                nucleus_rows_kernel<<<d->B * nodes.n, NUC_THREADS, sizeof(NucleusSmem), st>>>(
+                    static_cast<const uint16_t *>(logits), d->V, d->N, nodes, c, top_p, row_max, row_sum, thr_key, keep_sum,
+                    nucleus_thr, nucleus_sum);
+                SR_LAUNCH_CHECK();
+            }
             walk_cta_kernel<false, true><<<d->B, NUC_THREADS, sizeof(NucleusSmem), st>>>(
-                wa, topo, c, top_p, row_max, row_sum, thr_key, keep_sum, nucleus_thr, nucleus_sum);
+                wa, topo, c, top_p, row_max, row_sum, thr_key, keep_sum, nucleus_thr, nucleus_sum, ahead ? 1 : 0);
+        }
     } else if (lazy) {
         walk_cta_kernel<true, false><<<d->B, NUC_THREADS, 0, st>>>(wa, topo, c, 1.0f, row_max, row_sum, nullptr, nullptr,
-                                                                    nullptr, nullptr);
+                                                                    nullptr, nullptr, 0);
     } else {
         // plain verification: the walk and the terminal draw in one launch, overlapping the statistics kernel's tail
         constexpr int WT_SMEM_LIMIT = 160 * 1024;

@@ -197,10 +197,11 @@ class StepWorkload:
     @property
     def LAUNCHES_VERIFY(self) -> int:
         # plain verification with all rows' statistics: the statistics kernel, then walk + terminal draw in one;
-        # with a nucleus: statistics, walk, draw; statistics of the visited rows only: walk, draw
+        # with a nucleus: statistics, thresholds of the nodes with children, walk, draw; statistics of the visited
+        # rows only: walk, draw
         if self.lazy_stats:
             return 2
-        return 3 if self.top_p is not None else 2
+        return 4 if self.top_p is not None else 2
 
     def launches_per_step(self) -> int:
         # the library says how many kernels an attention call enqueues: the plan kernel runs for the first layer
