@@ -727,7 +727,8 @@ def run_calls(args, w, layers):
     rho = torch.full((R,), 0.9, device=dev)
     mem = wl.m.reshape(R, w.d).clone()
     k_support = 48
-    fb_ws = torch.empty(R * k_support * 4 + 512, dtype=torch.uint8, device=dev)
+    fb_ws = torch.empty(S.reflex_feedback_workspace_bytes(R, w.k, k_support, w.d, w.V, w.temperature), dtype=torch.uint8,
+                        device=dev)
     cid = wl.prop["cand_id"].reshape(R, w.k).contiguous()
     clg = wl.prop["cand_logit"].reshape(R, w.k).contiguous()
     rmax = wl.ver["row_max"].reshape(-1).contiguous()

@@ -533,6 +533,11 @@ def verify_nucleus(logits, parent, tree_tok, tree_cand, cand_id, cand_logit, u_a
     return out
 
 
+def reflex_feedback_workspace_bytes(R, k, k_support, d, V, temperature=1.0, eps=1e-6) -> int:
+    desc = FeedbackDesc(R, k, k_support, d, V, temperature, eps, 0, 0.0)
+    return int(lib().specroll_reflex_feedback_workspace_bytes(C.byref(desc)))
+
+
 def reflex_feedback(logits, rec_row, row_max, row_sum, cand_id, cand_logit, y_star, W, rho, rec_mem, m, k_support,
                     temperature=1.0, eps=1e-6, workspace=None, severity_min=None, want_e=False):
     """specroll_reflex_feedback(_ex): verifier feedback of R matured records, memory ``m`` updated in place.

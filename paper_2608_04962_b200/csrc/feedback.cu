@@ -17,15 +17,17 @@
 //                          memory.  Fallback for rows with thousands of equal large values: a radix search by
 //                          COUNT (four bits per pass) for the key of the kS-th largest value, a pass for the ids
 //                          above it, an ordered pass for the first ids that tie with it, a rank sort.
-//   feedback_vec_kernel    the small quantities (q, p on S, the coefficient of every support row) by one warp,
-//                          then the <= k + kS + 1 rows of W come through shared memory by asynchronous copies,
-//                          several rows in flight, and all threads accumulate both directions; three RMS
-//                          reductions, and the memory update.  (feedback_kernel: hidden sizes not a multiple of 8.)
+//   feedback_vec_kernel    the small quantities (q, p on S, the coefficient of every support row; repeated tokens
+//                          found by all threads, the rest by one warp), then the <= k + kS + 1 rows of W come
+//                          through shared memory as bulk copies of whole rows, three batches in flight, and the
+//                          threads accumulate both directions; three RMS reductions, and the memory update.
+//                          (feedback_kernel: hidden sizes not a multiple of 8.)
 #include <math.h>
 
 #include <algorithm>
 
 #include "common.cuh"
+#include "tc05.cuh"
 
 namespace specroll {
 
@@ -62,6 +64,17 @@ __device__ __forceinline__ float block_sum_f(float v, float *red) {
     __syncthreads();
     float t = 0.f;
     for (int w = 0; w < THREADS / 32; ++w) t += red[w];
+    return t;
+}
+// the same for a CTA of any whole number of warps
+__device__ __forceinline__ float block_sum_rt(float v, float *red) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int w = 0; w < nw; ++w) t += red[w];
     return t;
 }
 }  // namespace fb
@@ -348,6 +361,8 @@ struct FeedbackSmall {
     float q[SPECROLL_MAX_TOPK];
     int raw_id[fb::MAX_S];   // C, Top_kS, y* as they come (with duplicates)
     float raw_p[fb::MAX_S];
+    int first[fb::MAX_S];    // raw index of the first occurrence of the same token (-1: not a token of the vocabulary)
+    int where[fb::MAX_S];    // the raw entry's place in S (-1: none)
     int n;
     float dd, dc, w;
 };
@@ -369,6 +384,15 @@ __device__ void feedback_small(const FeedbackArgs &a, int r, FeedbackSmall &s) {
         const int v = i < k ? cid[i] : (i < k + kS ? top[i - k] : a.y_star[r]);
         s.raw_id[i] = v;
         s.raw_p[i] = (v >= 0 && v < a.V) ? __expf((__uint_as_float((uint32_t)lg[v] << 16) - M) * a.inv_T) / Ssum : 0.f;
+        s.first[i] = (v >= 0 && v < a.V) ? i : -1;
+    }
+    __syncthreads();
+    // the first occurrence of every token in the concatenation: all pairs (i, j < i), spread over the CTA (matches
+    // are rare: a candidate that is also among the target's largest, y* among either)
+    for (int pp = tid; pp < n_raw * 64; pp += blockDim.x) {
+        const int i = pp >> 6;
+        for (int j = pp & 63; j < i; j += 64)
+            if (s.raw_id[j] == s.raw_id[i] && s.first[i] >= 0) atomicMin(&s.first[i], j);
     }
     __syncthreads();
     if (warp == 0) {
@@ -391,27 +415,25 @@ __device__ void feedback_small(const FeedbackArgs &a, int r, FeedbackSmall &s) {
         for (int i0 = 0; i0 < n_raw; i0 += 32) {
             const int i = i0 + lane;
             const int v = i < n_raw ? s.raw_id[i] : -1;
-            bool fresh = v >= 0 && v < a.V;
-            if (fresh) {
-                for (int j = 0; j < i; ++j) {  // the same token earlier in the concatenation?
-                    if (s.raw_id[j] == v) {
-                        fresh = false;
-                        break;
-                    }
-                }
-            }
+            const bool fresh = i < n_raw && s.first[i] == i;
             const unsigned bal = __ballot_sync(0xffffffffu, fresh);
             const int base = s.n;
             if (fresh) {
                 const int pos = base + __popc(bal & ((1u << lane) - 1u));
                 s.id[pos] = v;
                 s.p[pos] = s.raw_p[i];
+                s.where[i] = pos;
             }
             __syncwarp();
             if (lane == 0) s.n = base + __popc(bal);
             __syncwarp();
         }
         const int n = s.n;
+        for (int i = lane; i < n_raw; i += 32) {  // repeated tokens: the place of their first occurrence
+            const int f = s.first[i];
+            if (f != i) s.where[i] = f < 0 ? -1 : s.where[f];
+        }
+        __syncwarp();
         // ---- masses: p(S), p(C), p(C*); TV on C
         float pS = 0.f;
         for (int i = lane; i < n; i += 32) pS += s.p[i];
@@ -427,17 +449,14 @@ __device__ void feedback_small(const FeedbackArgs &a, int r, FeedbackSmall &s) {
         for (int i = lane; i < n; i += 32) s.acov[i] = 0.f;
         __syncwarp();
         for (int t = lane; t < k; t += 32) {
-            const int v = s.raw_id[k + t];
             const float pv = s.raw_p[k + t];
             pCs += pv;
-            bool inC = false;
-            for (int j = 0; j < k; ++j) inC |= (s.raw_id[j] == v);
+            const int f = s.first[k + t];
+            const bool inC = f >= 0 && f < k;  // (first seen among the candidates, which come first)
             if (!inC) {
                 // an omitted target-important token: +p_S(y) on its own row, -p_S(y) on the weakest candidate's
-                int pos = -1;
-                for (int i = k; i < n; ++i)
-                    if (s.id[i] == v) pos = i;
-                if (pos >= 0) s.acov[pos] = pv / pS;
+                const int pos = s.where[k + t];
+                if (pos >= k) s.acov[pos] = pv / pS;
                 cov_b += pv / pS;
             }
         }
@@ -536,73 +555,146 @@ __global__ void __launch_bounds__(fb::FB_THREADS) feedback_kernel(FeedbackArgs a
     }
 }
 
-// Hidden sizes that are a multiple of eight: thread t owns the 8-column vectors t, t + 512, ... (NV of them), a row
-// of W is read with 128-bit loads, and four support rows are in flight at a time: a record's 57 rows of W are a few
-// hundred KB fetched by one CTA, so what bounds the kernel is how many bytes that CTA keeps in flight.
+// Hidden sizes that are a multiple of eight.  The support rows of W come through shared memory in batches of rps
+// rows, three batches deep, as bulk copies of whole rows issued by one thread and counted on an mbarrier per stage
+// (asynchronous copies issued by all threads cost more instructions in address arithmetic than the sums they feed).
+// A row is nvec 8-column vectors.  When a row is shorter than the CTA (NV = 1), the threads form groups of nvec,
+// group g takes rows g, g + groups, ... of every batch, and the groups' partial sums are added through shared
+// memory at the end; otherwise the CTA has ceil(nvec / NV) threads (rounded up to whole warps) and thread t owns
+// the vectors t, t + blockDim, ... (NV of them) of every row.
 constexpr int FBV_THREADS = 512;
+constexpr int FBV_STAGES = 3;
+
+// Row groups of the vector kernel: as many as fit the CTA, at most one per row of a batch.
+__host__ __device__ inline int fbv_groups(int d, int rows_per_stage) {
+    const int nvec = d >> 3;
+    if (nvec >= FBV_THREADS) return 1;
+    const int g = FBV_THREADS / nvec;
+    return g < rows_per_stage ? g : rows_per_stage;
+}
+// Threads of the vector kernel's CTA for hidden size d with NV vectors per thread.
+__host__ __device__ inline int fbv_threads(int d, int NV) {
+    const int nvec = d >> 3;
+    if (NV == 1) return FBV_THREADS;
+    return ((nvec + NV - 1) / NV + 31) / 32 * 32;
+}
+
+__device__ __forceinline__ void fbv_bulk_row(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
 template <int NV>
-__global__ void __launch_bounds__(FBV_THREADS) feedback_vec_kernel(FeedbackArgs a) {
+__global__ void __launch_bounds__(FBV_THREADS, NV <= 2 ? 2 : 1) feedback_vec_kernel(FeedbackArgs a) {
     using namespace fb;
     __shared__ FeedbackSmall sm;
     __shared__ float red[FBV_THREADS / 32];
-    extern __shared__ __align__(16) unsigned char fb_stage[];  // [3][rows_per_stage][d] bf16
-    const int r = blockIdx.x, tid = threadIdx.x;
+    __shared__ __align__(8) unsigned long long full[FBV_STAGES];
+    __shared__ volatile int abort_flag;
+    extern __shared__ __align__(16) unsigned char fb_stage[];  // [3][rows_per_stage][d] bf16; then the groups' partial sums
+    const int r = blockIdx.x, tid = threadIdx.x, tpb = blockDim.x;
     const int d = a.d, nvec = d >> 3;
-    feedback_small(a, r, sm);
+    if (tid == 0) {
+        for (int s = 0; s < FBV_STAGES; ++s) mbar_init(smem_u32(&full[s]), 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    feedback_small(a, r, sm);  // (ends with a barrier)
     const int n = sm.n;
-    const float dd = sm.dd, dc = sm.dc;
+    const float dd = sm.dd, dc = sm.dc, sev = sm.w;
+    const int *sh_id = sm.id;
+    const float *sh_ad = sm.adist, *sh_ac = sm.acov;
     float rd[NV][8], rc[NV][8];
 #pragma unroll
     for (int c = 0; c < NV; ++c)
 #pragma unroll
         for (int t = 0; t < 8; ++t) rd[c][t] = rc[c][t] = 0.f;
-    // The support rows of W come through shared memory in batches of rps rows, three batches deep, by asynchronous
-    // copies: two batches are on their way while one is used.  (With plain loads into registers the compiler kept one
-    // row in flight at a time, to save registers: 57 round trips to memory one after the other.)
-    constexpr int STAGES = 3;
     const int rps = a.rows_per_stage;
-    const size_t stage_bytes = (size_t)rps * d * 2;
+    const uint32_t row_bytes = (uint32_t)d * 2u;
+    const size_t stage_bytes = (size_t)rps * row_bytes;
     const int nb = (n + rps - 1) / rps;
-    auto issue = [&](int batch) {
-        if (batch < nb) {
-            const uint32_t dst = smem_u32(fb_stage + (size_t)(batch % STAGES) * stage_bytes);
-            for (int ch = tid; ch < rps * nvec; ch += FBV_THREADS) {
-                const int q = ch / nvec, vi = ch - q * nvec, i = batch * rps + q;
-                if (i < n) cp_async16(dst + (uint32_t)ch * 16u, a.W + (size_t)sm.id[i] * d + (size_t)vi * 8, true);
-            }
-        }
-        cp_async_commit();  // (an empty group when there is nothing left: the count below stays the same)
+    const int groups = NV == 1 ? fbv_groups(d, rps) : 1;
+    const int grp = NV == 1 ? tid / nvec : 0, vi0 = NV == 1 ? tid - grp * nvec : tid;
+    auto issue = [&](int batch) {  // one thread
+        const int s = batch % FBV_STAGES;
+        const int rows = min(rps, n - batch * rps);
+        const uint32_t bar = smem_u32(&full[s]);
+        mbar_arrive_expect_tx(bar, (uint32_t)rows * row_bytes);
+        const uint32_t dst = smem_u32(fb_stage + (size_t)s * stage_bytes);
+        for (int q = 0; q < rows; ++q)
+            fbv_bulk_row(dst + (uint32_t)q * row_bytes, a.W + (size_t)sh_id[batch * rps + q] * d, row_bytes, bar);
     };
-    issue(0);
-    issue(1);
+    if (tid == 0)
+        for (int b = 0; b < FBV_STAGES && b < nb; ++b) issue(b);
+    bool ok = true;
     for (int b = 0; b < nb; ++b) {
-        issue(b + 2);
-        cp_async_wait<2>();  // everything up to batch b has landed
-        __syncthreads();
-        const unsigned char *src = fb_stage + (size_t)(b % STAGES) * stage_bytes;
-        for (int q = 0; q < rps; ++q) {
-            const int i = b * rps + q;
-            if (i >= n) break;
-            const float ad = sm.adist[i], ac = sm.acov[i];
+        ok = mbar_wait(smem_u32(&full[b % FBV_STAGES]), (uint32_t)(b / FBV_STAGES) & 1u, &abort_flag);
+        if (ok && grp < groups) {
+            const unsigned char *src = fb_stage + (size_t)(b % FBV_STAGES) * stage_bytes;
+            const int rows = min(rps, n - b * rps);
+            for (int q = grp; q < rows; q += groups) {
+                const int i = b * rps + q;
+                const float ad = sh_ad[i], ac = sh_ac[i];
 #pragma unroll
-            for (int c = 0; c < NV; ++c) {
-                const int vi = tid + c * FBV_THREADS;
-                if (vi < nvec) {
-                    const uint4 v = *reinterpret_cast<const uint4 *>(src + ((size_t)q * nvec + vi) * 16);
-                    const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+                for (int c = 0; c < NV; ++c) {
+                    const int vi = vi0 + c * tpb;
+                    if (vi < nvec) {
+                        const uint4 v = *reinterpret_cast<const uint4 *>(src + ((size_t)q * nvec + vi) * 16);
+                        const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        const float lo = __uint_as_float(w4[t] << 16), hi = __uint_as_float(w4[t] & 0xffff0000u);
-                        rd[c][2 * t] = fmaf(ad, lo, rd[c][2 * t]);
-                        rd[c][2 * t + 1] = fmaf(ad, hi, rd[c][2 * t + 1]);
-                        rc[c][2 * t] = fmaf(ac, lo, rc[c][2 * t]);
-                        rc[c][2 * t + 1] = fmaf(ac, hi, rc[c][2 * t + 1]);
+                        for (int t = 0; t < 4; ++t) {
+                            const float lo = __uint_as_float(w4[t] << 16), hi = __uint_as_float(w4[t] & 0xffff0000u);
+                            rd[c][2 * t] = fmaf(ad, lo, rd[c][2 * t]);
+                            rd[c][2 * t + 1] = fmaf(ad, hi, rd[c][2 * t + 1]);
+                            rc[c][2 * t] = fmaf(ac, lo, rc[c][2 * t]);
+                            rc[c][2 * t + 1] = fmaf(ac, hi, rc[c][2 * t + 1]);
+                        }
                     }
                 }
             }
         }
-        __syncthreads();  // the stage is free for the batch three further on
+        // the stage is free for the batch three further on; a wait that ran out ends the record for every thread
+        if (__syncthreads_or(!ok)) {
+            ok = false;
+            break;
+        }
+        if (tid == 0 && b + FBV_STAGES < nb) {
+            fence_proxy_async();  // the stage's readers are done (barrier above) before the copy engine writes it again
+            issue(b + FBV_STAGES);
+        }
     }
+    if (!ok) {
+        // (cannot happen with valid arguments: a bulk copy of a readable row always completes; the record is marked
+        // instead of left looking valid, and the memory is not touched)
+        if (tid == 0) {
+            if (a.d_dist) a.d_dist[r] = nanf("");
+            if (a.d_cov) a.d_cov[r] = nanf("");
+        }
+        return;
+    }
+    if (NV == 1 && groups > 1) {
+        // add the groups' partial sums: group g > 0 leaves its 16 numbers, group 0 collects
+        float *part = reinterpret_cast<float *>(fb_stage);  // [groups - 1][16][nvec]; the stages are free now
+        if (grp > 0 && grp < groups) {
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                part[((size_t)(grp - 1) * 16 + t) * nvec + vi0] = rd[0][t];
+                part[((size_t)(grp - 1) * 16 + 8 + t) * nvec + vi0] = rc[0][t];
+                rd[0][t] = rc[0][t] = 0.f;
+            }
+        }
+        __syncthreads();
+        if (grp == 0) {
+            for (int g = 1; g < groups; ++g)
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    rd[0][t] += part[((size_t)(g - 1) * 16 + t) * nvec + vi0];
+                    rc[0][t] += part[((size_t)(g - 1) * 16 + 8 + t) * nvec + vi0];
+                }
+        }
+    }
+    // (from here on only the threads with vectors of their own hold anything but zeros)
     float sd = 0.f, scv = 0.f;
 #pragma unroll
     for (int c = 0; c < NV; ++c)
@@ -611,8 +703,8 @@ __global__ void __launch_bounds__(FBV_THREADS) feedback_vec_kernel(FeedbackArgs 
             sd += rd[c][t] * rd[c][t];
             scv += rc[c][t] * rc[c][t];
         }
-    sd = block_sum_f<FBV_THREADS>(sd, red);
-    scv = block_sum_f<FBV_THREADS>(scv, red);
+    sd = block_sum_rt(sd, red);
+    scv = block_sum_rt(scv, red);
     const float fd = dd / (sqrtf(sd / d) + a.eps), fc = dc / (sqrtf(scv / d) + a.eps);
     float sg = 0.f;
 #pragma unroll
@@ -622,18 +714,18 @@ __global__ void __launch_bounds__(FBV_THREADS) feedback_vec_kernel(FeedbackArgs 
             rd[c][t] = fd * rd[c][t] + fc * rc[c][t];  // g
             sg += rd[c][t] * rd[c][t];
         }
-    sg = block_sum_f<FBV_THREADS>(sg, red);
+    sg = block_sum_rt(sg, red);
     const float fe = (dd + dc) / (sqrtf(sg / d) + a.eps);
     const float rho = a.rho[r];
-    const float w = sm.w;
-    const bool keep = !a.weighted || w >= a.severity_min;
-    const float gain = (1.f - rho) * (a.weighted ? w : 1.f);
+    const bool keep = !a.weighted || sev >= a.severity_min;
+    const float gain = (1.f - rho) * (a.weighted ? sev : 1.f);
     float4 *mr = reinterpret_cast<float4 *>(a.m + (size_t)a.rec_mem[r] * d);
     float4 *er = a.e_out ? reinterpret_cast<float4 *>(a.e_out + (size_t)r * d) : nullptr;
+    const bool owner = NV > 1 || grp == 0;
 #pragma unroll
     for (int c = 0; c < NV; ++c) {
-        const int vi = tid + c * FBV_THREADS;
-        if (vi < nvec) {
+        const int vi = vi0 + c * tpb;
+        if (owner && vi < nvec) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const float4 e = make_float4(fe * rd[c][4 * h], fe * rd[c][4 * h + 1], fe * rd[c][4 * h + 2], fe * rd[c][4 * h + 3]);
@@ -726,10 +818,13 @@ extern "C" int specroll_reflex_feedback_ex(const specroll_feedback_desc *d, cons
     a.inv_T = 1.0f / d->temperature;
     a.eps = d->eps;
     // (m and e_out rows start at multiples of d floats: 16-byte aligned when d % 8 == 0 and the bases are)
-    const bool vec = (d->d % 8) == 0 && aligned16(m) && (!e_out || aligned16(e_out));
+    // (bulk copies of W rows: 16-byte aligned rows)
+    const bool vec = (d->d % 8) == 0 && aligned16(m) && (!e_out || aligned16(e_out)) && aligned16(W);
     // batches of at most 24 KB of W rows, three deep: three CTAs fit an SM
     a.rows_per_stage = std::max(1, std::min(8, 24576 / (d->d * 2)));
-    const size_t fb_smem = (size_t)3 * a.rows_per_stage * d->d * 2;
+    const size_t fb_smem =
+        std::max((size_t)FBV_STAGES * a.rows_per_stage * d->d * 2,
+                 (size_t)(fbv_groups(d->d, a.rows_per_stage) - 1) * 16 * (size_t)(d->d >> 3) * sizeof(float));
     if (vec) {
         const void *kern = d->d <= 8 * FBV_THREADS    ? reinterpret_cast<const void *>(feedback_vec_kernel<1>)
                            : d->d <= 16 * FBV_THREADS ? reinterpret_cast<const void *>(feedback_vec_kernel<2>)
@@ -738,11 +833,11 @@ extern "C" int specroll_reflex_feedback_ex(const specroll_feedback_desc *d, cons
         if (rc_ != SPECROLL_OK) return rc_;
     }
     if (vec && d->d <= 8 * FBV_THREADS)
-        feedback_vec_kernel<1><<<d->R, FBV_THREADS, fb_smem, st>>>(a);
+        feedback_vec_kernel<1><<<d->R, fbv_threads(d->d, 1), fb_smem, st>>>(a);
     else if (vec && d->d <= 16 * FBV_THREADS)
-        feedback_vec_kernel<2><<<d->R, FBV_THREADS, fb_smem, st>>>(a);
+        feedback_vec_kernel<2><<<d->R, fbv_threads(d->d, 2), fb_smem, st>>>(a);
     else if (vec)
-        feedback_vec_kernel<3><<<d->R, FBV_THREADS, fb_smem, st>>>(a);
+        feedback_vec_kernel<3><<<d->R, fbv_threads(d->d, 3), fb_smem, st>>>(a);
     else if (d->d <= 8 * fb::FB_THREADS)
         feedback_kernel<8><<<d->R, fb::FB_THREADS, 0, st>>>(a);
     else if (d->d <= 24 * fb::FB_THREADS)
