@@ -109,6 +109,30 @@ def test_lone_root_and_chain_and_star_topologies():
         check(w, o, g, lg)
 
 
+@pytest.mark.parametrize("V", [8, 1032, 8200, 40008])
+def test_terminal_draw_alone_over_ragged_vocabularies(V):
+    """A lone root: the step is the terminal draw from the root's softmax.  Nearly flat logits spread the drawn tokens
+    over the whole vocabulary, so every eighth of the row (the unit the draw narrows down to first) is hit, with
+    vocabulary sizes that leave the eighths empty, partial or ragged; u_fin is stratified and includes 0."""
+    B = 640
+    w = I.scaled(I.WORKLOADS["tiny"], B=B, N=1, V=V, K=3, k=4, fixed_parent=(-1,))
+    parent = np.array([-1], np.int32)
+    cid, cl = I.synthetic_candidates(w)
+    d = ref.tree_draw(parent, np.zeros(B, np.int32), cid, cl, I.uniforms24(3, (B, 1)))
+    lg = I.target_logits(w, parent, d["tree_tok"], flat=True)
+    u_acc, _ = I.verify_uniforms(w)
+    u_fin = ((np.arange(B) + 0.5) / B).astype(np.float32)
+    u_fin[0] = 0.0
+    u_fin[-1] = np.float32(1.0 - 1e-4)
+    o, g = run_both(w, parent, lg, d["tree_tok"], d["tree_cand"], cid, cl, u_acc, u_fin)
+    check(w, o, g, lg)
+    assert (g["n_acc"] == 0).all() and (g["term_kind"] == 0).all()
+    tok = g["out_tok"][:, 0]
+    assert tok.min() >= 0 and tok.max() < V
+    if V >= 8200:
+        assert len(set((tok.astype(np.int64) * 8 // V).tolist())) == 8
+
+
 def test_wide_lists_wide_stars_and_underflowing_proposals():
     # the node routine's fast form holds a candidate and a child per lane: more than 32 of either, and slot
     # proposals whose weights underflow against a drawn candidate's logit, take the sequential form
