@@ -586,7 +586,7 @@ __device__ __forceinline__ void fbv_bulk_row(uint32_t dst, const void *src, uint
 }
 
 template <int NV>
-__global__ void __launch_bounds__(FBV_THREADS, NV <= 2 ? 2 : 1) feedback_vec_kernel(FeedbackArgs a) {
+__global__ void __launch_bounds__(FBV_THREADS, NV == 1 ? 3 : (NV == 2 ? 2 : 1)) feedback_vec_kernel(FeedbackArgs a) {
     using namespace fb;
     __shared__ FeedbackSmall sm;
     __shared__ float red[FBV_THREADS / 32];
@@ -820,8 +820,8 @@ extern "C" int specroll_reflex_feedback_ex(const specroll_feedback_desc *d, cons
     // (m and e_out rows start at multiples of d floats: 16-byte aligned when d % 8 == 0 and the bases are)
     // (bulk copies of W rows: 16-byte aligned rows)
     const bool vec = (d->d % 8) == 0 && aligned16(m) && (!e_out || aligned16(e_out)) && aligned16(W);
-    // batches of at most 24 KB of W rows, three deep: three CTAs fit an SM
-    a.rows_per_stage = std::max(1, std::min(8, 24576 / (d->d * 2)));
+    // batches of at most 20 KB of W rows, three deep: three CTAs fit an SM
+    a.rows_per_stage = std::max(1, std::min(8, 20480 / (d->d * 2)));
     const size_t fb_smem =
         std::max((size_t)FBV_STAGES * a.rows_per_stage * d->d * 2,
                  (size_t)(fbv_groups(d->d, a.rows_per_stage) - 1) * 16 * (size_t)(d->d >> 3) * sizeof(float));
