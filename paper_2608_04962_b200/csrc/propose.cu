@@ -296,6 +296,76 @@ topk_merge_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pi
 // its own share of the partial entries in registers (one pass, the loads independent of each other), then k rounds of
 // arg-best over the lanes' current best, the winner moving on to its next one.  (Re-reading all entries in each of
 // the k rounds made this kernel a tenth of the call at small batch.)
+struct Top8 {
+    float v[8];
+    int32_t i[8];
+};
+__device__ __forceinline__ bool tk_better(float x, int32_t t, float y, int32_t u) { return x > y || (x == y && t < u); }
+__device__ __forceinline__ void tk_init(Top8 &L) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        L.v[i] = -INFINITY;
+        L.i[i] = 0x7fffffff;
+    }
+}
+// insert into the sorted list (best first) if it belongs there
+__device__ __forceinline__ void tk_insert(Top8 &L, float x, int32_t t) {
+    if (!tk_better(x, t, L.v[7], L.i[7])) return;
+#pragma unroll
+    for (int i = 7; i > 0; --i) {
+        if (tk_better(x, t, L.v[i - 1], L.i[i - 1])) {
+            L.v[i] = L.v[i - 1];
+            L.i[i] = L.i[i - 1];
+        } else if (tk_better(x, t, L.v[i], L.i[i])) {
+            L.v[i] = x;
+            L.i[i] = t;
+        }
+    }
+    if (tk_better(x, t, L.v[0], L.i[0])) {
+        L.v[0] = x;
+        L.i[0] = t;
+    }
+}
+// the best of the lanes' current best; the lane that held it moves on to its next one (ids are distinct: one lane)
+__device__ __forceinline__ void tk_pop_best(Top8 &L, float &bv, int32_t &bi) {
+    bv = L.v[0];
+    bi = L.i[0];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (tk_better(ov, oi, bv, bi)) {
+            bv = ov;
+            bi = oi;
+        }
+    }
+    if (L.v[0] == bv && L.i[0] == bi) {
+#pragma unroll
+        for (int i = 0; i < 7; ++i) {
+            L.v[i] = L.v[i + 1];
+            L.i[i] = L.i[i + 1];
+        }
+        L.v[7] = -INFINITY;
+        L.i[7] = 0x7fffffff;
+    }
+}
+// a lane's share of the entries [c_lo, c_hi) of one row's partial lists, four independent loads at a time
+__device__ __forceinline__ void tk_scan(Top8 &L, const float *__restrict__ v, const int32_t *__restrict__ id, int c_lo,
+                                        int c_hi, int lane) {
+    for (int c0 = c_lo + lane; c0 < c_hi; c0 += 4 * 32) {
+        float x[4];
+        int32_t t[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int c = c0 + q * 32;
+            x[q] = c < c_hi ? v[c] : -INFINITY;
+            t[q] = c < c_hi ? id[c] : 0x7fffffff;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) tk_insert(L, x[q], t[q]);
+    }
+}
+
 __global__ void __launch_bounds__(128)
 topk_merge8_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pid, int M, int n_cand, int k,
                    int32_t *__restrict__ cand_id, float *__restrict__ cand_logit) {
@@ -304,66 +374,56 @@ topk_merge8_kernel(const float *__restrict__ pval, const int32_t *__restrict__ p
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x * 4 + warp;
     if (r >= M) return;
+    Top8 L;
+    tk_init(L);
+    tk_scan(L, pval + (size_t)r * n_cand, pid + (size_t)r * n_cand, 0, n_cand, lane);
+    for (int j = 0; j < k; ++j) {
+        float bv;
+        int32_t bi;
+        tk_pop_best(L, bv, bi);
+        if (lane == 0) {
+            cand_id[(size_t)r * k + j] = bi;
+            cand_logit[(size_t)r * k + j] = bv;
+        }
+    }
+}
+
+// The same with a CTA of eight warps per row, for rows with many partial lists (few rows in the projection, so
+// every CTA of the projection kernel has a list for each of them): a warp merges an eighth of the entries, warp 0
+// the eight results.  (One warp per row took 24 us on 32 rows of 148 lists, a tenth of the call.)
+constexpr int MERGE_WIDE_WARPS = 8;
+__global__ void __launch_bounds__(MERGE_WIDE_WARPS * 32)
+topk_merge8_wide_kernel(const float *__restrict__ pval, const int32_t *__restrict__ pid, int M, int n_cand, int k,
+                        int32_t *__restrict__ cand_id, float *__restrict__ cand_logit) {
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ float sv[MERGE_WIDE_WARPS * 8];
+    __shared__ int32_t si[MERGE_WIDE_WARPS * 8];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x;
     const float *v = pval + (size_t)r * n_cand;
     const int32_t *id = pid + (size_t)r * n_cand;
-    float lv[8];
-    int32_t li[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        lv[i] = -INFINITY;
-        li[i] = 0x7fffffff;
-    }
-    auto better = [](float x, int32_t t, float y, int32_t u) { return x > y || (x == y && t < u); };
-    for (int c0 = lane; c0 < n_cand; c0 += 4 * 32) {
-        float x[4];
-        int32_t t[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int c = c0 + q * 32;
-            x[q] = c < n_cand ? v[c] : -INFINITY;
-            t[q] = c < n_cand ? id[c] : 0x7fffffff;
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            if (!better(x[q], t[q], lv[7], li[7])) continue;
-            // insert into the sorted list (best first)
-#pragma unroll
-            for (int i = 7; i > 0; --i) {
-                if (better(x[q], t[q], lv[i - 1], li[i - 1])) {
-                    lv[i] = lv[i - 1];
-                    li[i] = li[i - 1];
-                } else if (better(x[q], t[q], lv[i], li[i])) {
-                    lv[i] = x[q];
-                    li[i] = t[q];
-                }
-            }
-            if (better(x[q], t[q], lv[0], li[0])) {
-                lv[0] = x[q];
-                li[0] = t[q];
-            }
+    const int per = (n_cand + MERGE_WIDE_WARPS - 1) / MERGE_WIDE_WARPS;
+    Top8 L;
+    tk_init(L);
+    tk_scan(L, v, id, min(n_cand, warp * per), min(n_cand, warp * per + per), lane);
+    for (int j = 0; j < 8; ++j) {
+        float bv;
+        int32_t bi;
+        tk_pop_best(L, bv, bi);
+        if (lane == 0) {
+            sv[warp * 8 + j] = bv;
+            si[warp * 8 + j] = bi;
         }
     }
+    __syncthreads();
+    if (warp != 0) return;
+    tk_init(L);
+    tk_scan(L, sv, si, 0, MERGE_WIDE_WARPS * 8, lane);
     for (int j = 0; j < k; ++j) {
-        float bv = lv[0];
-        int32_t bi = li[0];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (better(ov, oi, bv, bi)) {
-                bv = ov;
-                bi = oi;
-            }
-        }
-        if (lv[0] == bv && li[0] == bi) {  // (ids are distinct: one lane) this lane's best was taken
-#pragma unroll
-            for (int i = 0; i < 7; ++i) {
-                lv[i] = lv[i + 1];
-                li[i] = li[i + 1];
-            }
-            lv[7] = -INFINITY;
-            li[7] = 0x7fffffff;
-        }
+        float bv;
+        int32_t bi;
+        tk_pop_best(L, bv, bi);
         if (lane == 0) {
             cand_id[(size_t)r * k + j] = bi;
             cand_logit[(size_t)r * k + j] = bv;
@@ -675,8 +735,13 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
         SR_LAUNCH_CHECK();
     }
 
-    SR_CUDA_TRY(launch_dependent(true, k <= 8 ? topk_merge8_kernel : topk_merge_kernel, dim3((p.M + 3) / 4), dim3(128), 0, st,
-                                 (const float *)pval, (const int32_t *)pid, p.M, p.n_groups * k, k, cand_id, cand_logit));
+    if (k <= 8 && p.n_groups * k >= 512)
+        SR_CUDA_TRY(launch_dependent(true, topk_merge8_wide_kernel, dim3(p.M), dim3(MERGE_WIDE_WARPS * 32), 0, st,
+                                     (const float *)pval, (const int32_t *)pid, p.M, p.n_groups * k, k, cand_id, cand_logit));
+    else
+        SR_CUDA_TRY(launch_dependent(true, k <= 8 ? topk_merge8_kernel : topk_merge_kernel, dim3((p.M + 3) / 4), dim3(128), 0,
+                                     st, (const float *)pval, (const int32_t *)pid, p.M, p.n_groups * k, k, cand_id,
+                                     cand_logit));
 
     return launch_tree_draw(true, topo, B, K, k, d->temperature, anchor_tok, cand_id, cand_logit, u_draw, tree_tok,
                             tree_cand, slot_q, st);
