@@ -20,22 +20,27 @@ namespace specroll {
 namespace hmtc {
 constexpr int BM = 128, BK = 64, UMMA_K = 16, THREADS = 192;
 constexpr int W_BYTES = BM * BK * 2;
-template <int BN>
+// DEEP: for grids of at most one CTA per SM, where what a CTA keeps in flight is all the machine has in flight: a
+// stage holds two 64-wide slices of the contraction side by side (two boxes per operand), so a weight row arrives as
+// 256 contiguous bytes instead of 128 (the weights are row-major [d_out, d_in]: every row of a box is its own DRAM
+// page) and the ring holds twice the bytes; one CTA per SM.  Needs d % 128 == 0.
+template <int BN, bool DEEP>
 struct Cfg {
-    static constexpr int X_BYTES = BN * BK * 2;
-    static constexpr int STAGE_BYTES = W_BYTES + X_BYTES;
+    static constexpr int NBOX = DEEP ? 2 : 1;
+    static constexpr int X_BYTES = BN * BK * 2;  // one box
+    static constexpr int STAGE_BYTES = NBOX * (W_BYTES + X_BYTES);
     static constexpr int STAGES = BN == 64 ? 4 : (BN == 128 ? 3 : 4);
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 }  // namespace hmtc
 
-template <int BN>
+template <int BN, bool DEEP>
 __global__ void __launch_bounds__(hmtc::THREADS)
 head_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, int KX,
                    const __nv_bfloat16 *__restrict__ bias, const __nv_bfloat16 *__restrict__ h,
                    float *__restrict__ z, int B, int K, int d, int32_t *__restrict__ status) {
     using namespace hmtc;
-    using C = Cfg<BN>;
+    using C = Cfg<BN, DEEP>;
     constexpr int STAGES = C::STAGES;
     extern __shared__ unsigned char smem_raw[];
     pdl_launch_dependents();
@@ -53,7 +58,8 @@ head_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int o0 = blockIdx.x * BM, b0 = blockIdx.y * BN, hd = blockIdx.z;
-    const int KB = d / BK;
+    constexpr int NBOX = C::NBOX;
+    const int KB = d / (BK * NBOX);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -89,10 +95,13 @@ head_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                     ok = false;
                     break;
                 }
-                const uint32_t sw = base + stage * C::STAGE_BYTES, sx = sw + W_BYTES;
+                const uint32_t sw = base + stage * C::STAGE_BYTES, sx = sw + NBOX * W_BYTES;
                 mbar_arrive_expect_tx(full_bar(stage), C::STAGE_BYTES);
-                tma_load_2d(sw, &tmW, kb * BK, w_row, full_bar(stage));
-                tma_load_2d(sx, &tmX, kb * BK, x_row, full_bar(stage));
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx) {
+                    tma_load_2d(sw + bx * W_BYTES, &tmW, (kb * NBOX + bx) * BK, w_row, full_bar(stage));
+                    tma_load_2d(sx + bx * C::X_BYTES, &tmX, (kb * NBOX + bx) * BK, x_row, full_bar(stage));
+                }
             }
             if (!ok) {
                 // aborting: let the copies already in flight land before the CTA goes away
@@ -116,11 +125,15 @@ head_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                     break;
                 }
                 tc_fence_after();
-                const uint32_t sw = base + stage * C::STAGE_BYTES, sx = sw + W_BYTES;
-                const uint64_t adesc = smem_desc_sw128(sw, 1024, 0), bdesc = smem_desc_sw128(sx, 1024, 0);
+                const uint32_t sw = base + stage * C::STAGE_BYTES, sx = sw + NBOX * W_BYTES;
 #pragma unroll
-                for (int kk = 0; kk < BK / UMMA_K; ++kk)  // 16 inputs further = 32 bytes = 2 descriptor address units
-                    umma_ss(tmem_base, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+                for (int bx = 0; bx < NBOX; ++bx) {
+                    const uint64_t adesc = smem_desc_sw128(sw + bx * W_BYTES, 1024, 0);
+                    const uint64_t bdesc = smem_desc_sw128(sx + bx * C::X_BYTES, 1024, 0);
+#pragma unroll
+                    for (int kk = 0; kk < BK / UMMA_K; ++kk)  // 16 inputs further = 32 bytes = 2 descriptor address units
+                        umma_ss(tmem_base, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb | bx | kk) != 0 ? 1u : 0u);
+                }
                 umma_commit(empty_bar(stage));  // stage reusable once these MMAs have read it
             }
             if (ok) umma_commit(acc_bar);  // accumulator complete
@@ -172,21 +185,33 @@ head_mlp_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     }
 }
 
+template <int BN, bool DEEP>
+static int launch_bn2(const CUtensorMap &tmW, const CUtensorMap &tmX, int KX, const void *bias, const void *h, float *z,
+                      int B, int K, int d, int32_t *status, cudaStream_t st, dim3 grid) {
+    using namespace hmtc;
+    using C = Cfg<BN, DEEP>;
+    const int rc = device_setup(reinterpret_cast<const void *>(head_mlp_tc_kernel<BN, DEEP>), C::SMEM_BYTES, nullptr);
+    if (rc != SPECROLL_OK) return rc;
+    // (the dependent of the LayerNorm kernel in the stream)
+    SR_CUDA_TRY(launch_dependent(true, head_mlp_tc_kernel<BN, DEEP>, grid, dim3(THREADS), C::SMEM_BYTES, st, tmW, tmX, KX,
+                                 static_cast<const __nv_bfloat16 *>(bias), static_cast<const __nv_bfloat16 *>(h), z, B, K, d,
+                                 status));
+    return SPECROLL_OK;
+}
+
 template <int BN>
 static int launch_bn(const CUtensorMap &tmW, const void *xhat, int KX, const void *bias, const void *h, float *z,
                      int B, int K, int d, int32_t *status, cudaStream_t st) {
     using namespace hmtc;
-    using C = Cfg<BN>;
     CUtensorMap tmX;
     int rc = make_tmap_2d_bf16(&tmX, xhat, (uint64_t)KX * B, (uint64_t)d, (uint64_t)d, BN);
     if (rc != SPECROLL_OK) return rc;
-    if ((rc = device_setup(reinterpret_cast<const void *>(head_mlp_tc_kernel<BN>), C::SMEM_BYTES, nullptr)) != SPECROLL_OK) return rc;
+    int n_sm = 0;
+    if ((rc = device_setup(nullptr, 0, &n_sm)) != SPECROLL_OK) return rc;
     const dim3 grid((unsigned)((d + BM - 1) / BM), (unsigned)((B + BN - 1) / BN), (unsigned)K);
-    // (the dependent of the LayerNorm kernel in the stream)
-    SR_CUDA_TRY(launch_dependent(true, head_mlp_tc_kernel<BN>, grid, dim3(THREADS), C::SMEM_BYTES, st, tmW, tmX, KX,
-                                 static_cast<const __nv_bfloat16 *>(bias), static_cast<const __nv_bfloat16 *>(h), z, B, K, d,
-                                 status));
-    return SPECROLL_OK;
+    if (BN < 256 && (d % (2 * BK)) == 0 && (long long)grid.x * grid.y * grid.z <= n_sm)
+        return launch_bn2<BN, BN < 256>(tmW, tmX, KX, bias, h, z, B, K, d, status, st, grid);
+    return launch_bn2<BN, false>(tmW, tmX, KX, bias, h, z, B, K, d, status, st, grid);
 }
 
 // Host launcher.  xhat[KX, B, d], A[K, d, d] (row = output unit), bias[K, d], h[B, d] bf16; z[B, K, d] fp32.
