@@ -388,8 +388,8 @@ topk_merge8_kernel(const float *__restrict__ pval, const int32_t *__restrict__ p
     }
 }
 
-// The same with a CTA of eight warps per row, for rows with many partial lists (few rows in the projection, so
-// every CTA of the projection kernel has a list for each of them): a warp merges an eighth of the entries, warp 0
+// The same with a CTA of eight warps per row, for rows with 32 or more partial lists (few rows in the projection, so
+// many CTAs of the projection kernel have a list for each of them): a warp merges an eighth of the entries, warp 0
 // the eight results.  (One warp per row took 24 us on 32 rows of 148 lists, a tenth of the call.)
 constexpr int MERGE_WIDE_WARPS = 8;
 __global__ void __launch_bounds__(MERGE_WIDE_WARPS * 32)
@@ -735,7 +735,7 @@ extern "C" int specroll_propose(const specroll_propose_desc *d, const void *h, c
         SR_LAUNCH_CHECK();
     }
 
-    if (k <= 8 && p.n_groups * k >= 512)
+    if (k <= 8 && p.n_groups * k >= 256)
         SR_CUDA_TRY(launch_dependent(true, topk_merge8_wide_kernel, dim3(p.M), dim3(MERGE_WIDE_WARPS * 32), 0, st,
                                      (const float *)pval, (const int32_t *)pid, p.M, p.n_groups * k, k, cand_id, cand_logit));
     else
